@@ -1,0 +1,382 @@
+/*
+ * CPU oracle for greedy RNN-Transducer decoding: the sequential frame-by-frame
+ * procedure (Algorithm 1, "RNN-T Inference Algorithm") and windowed decoding
+ * (Algorithm 2, "WIND Algorithm").
+ *
+ * THIS IS TEST INFRASTRUCTURE.  It is deliberately plain and slow: nested loops,
+ * every sum accumulated in fp64 in index order, no blocking, no SIMD, no BLAS.
+ * Only the tests, the smoke check and the benchmark's CPU-baseline leg may call
+ * it; the CUDA library shares no code with it.
+ *
+ * Model (the paper treats decoder and joiner as black boxes; Section "Background:
+ * RNN-T" only fixes their roles):
+ *   decoder  = embedding table + L-layer LSTM (gate order i,f,g,o; two bias
+ *              vectors; zero initial state), fed ONE token per update; the
+ *              start-of-sequence input is the blank id;
+ *   joiner   = W_out * act(W_enc*f + b_enc + W_pred*h_top + b_pred) + b_out,
+ *              act = ReLU or tanh; argmax is taken on the logits (softmax is
+ *              monotone), lowest index winning ties.
+ *
+ * Safeguard against staying on one frame forever ("max symbols per frame", S):
+ * a counter of consecutive emissions on the current frame; when it reaches S
+ * the S-th token is still emitted and fed to the decoder, then t advances by
+ * one.  The counter resets whenever t advances.
+ *
+ * Pins (see tests): WIND(W) == sequential for every W; brute-force tabulation
+ * of joint argmaxes on tiny models; LSTM / linear layers against library fp64
+ * routines and closed forms; S honoured; jump-size support.
+ * The paper prints no worked numeric example, so token-level agreement with the
+ * paper's own runs is "parity unpinned"; the pins above are what fixes this code.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+typedef struct {
+    int32_t D, E, P, L, H, V;
+    int32_t blank_id;
+    int32_t act; /* 0 = ReLU, 1 = tanh */
+    const float* emb;         /* [V+1, E] */
+    const float* const* w_ih; /* L x [4P, in_l], in_0 = E, in_l = P */
+    const float* const* w_hh; /* L x [4P, P] */
+    const float* const* b_ih; /* L x [4P] */
+    const float* const* b_hh; /* L x [4P] */
+    const float* w_enc;       /* [H, D] */
+    const float* b_enc;       /* [H] */
+    const float* w_pred;      /* [H, P] */
+    const float* b_pred;      /* [H] */
+    const float* w_out;       /* [V+1, H] */
+    const float* b_out;       /* [V+1] */
+} oracle_model_t;
+
+typedef struct {
+    int64_t steps;          /* loop iterations (joint evaluations) */
+    int64_t joint_rows;     /* joint rows evaluated */
+    int64_t pred_updates;   /* decoder updates, excluding the start-of-sequence one */
+    int64_t forced;         /* forced advances by the S rule */
+    int64_t low_margin;     /* decisions whose top-2 logit margin < margin_thr */
+    int64_t decisions;      /* frame-level decisions taken (Alg. 1 sense) */
+    int64_t emit_frames;    /* frames with at least one emission */
+    int64_t jump_hist[65];  /* jump sizes 0..64 (WIND only; W <= 64 recorded) */
+} oracle_stats_t;
+
+/* ------------------------------------------------------------------------- */
+/* y = W x + b, W [n_out, n_in] fp32 row-major, x fp64, fp64 accumulate       */
+/* ------------------------------------------------------------------------- */
+void oracle_linear(const float* W, const float* b, const double* x, int n_out, int n_in, double* y) {
+    for (int o = 0; o < n_out; ++o) {
+        double acc = b ? (double)b[o] : 0.0;
+        const float* row = W + (size_t)o * n_in;
+        for (int k = 0; k < n_in; ++k) acc += (double)row[k] * x[k];
+        y[o] = acc;
+    }
+}
+
+static double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
+
+/*
+ * One LSTM stack update for one token.  h, c: [L, P] fp64, updated in place.
+ * Layer l: gates = W_ih x + b_ih + W_hh h + b_hh, split as (i, f, g, o);
+ * c <- sigma(f)*c + sigma(i)*tanh(g); h <- sigma(o)*tanh(c); x of layer l+1 is
+ * the new h of layer l.
+ */
+void oracle_lstm_step(const oracle_model_t* m, int32_t tok, double* h, double* c) {
+    const int P = m->P;
+    double* x = (double*)malloc(sizeof(double) * (size_t)(m->E > P ? m->E : P));
+    double* ga = (double*)malloc(sizeof(double) * 4 * (size_t)P);
+    double* gb = (double*)malloc(sizeof(double) * 4 * (size_t)P);
+    for (int k = 0; k < m->E; ++k) x[k] = (double)m->emb[(size_t)tok * m->E + k];
+    int n_in = m->E;
+    for (int l = 0; l < m->L; ++l) {
+        double* hl = h + (size_t)l * P;
+        double* cl = c + (size_t)l * P;
+        oracle_linear(m->w_ih[l], m->b_ih[l], x, 4 * P, n_in, ga);
+        oracle_linear(m->w_hh[l], m->b_hh[l], hl, 4 * P, P, gb);
+        for (int j = 0; j < P; ++j) {
+            double gi = sigmoid(ga[j] + gb[j]);
+            double gf = sigmoid(ga[P + j] + gb[P + j]);
+            double gg = tanh(ga[2 * P + j] + gb[2 * P + j]);
+            double go = sigmoid(ga[3 * P + j] + gb[3 * P + j]);
+            cl[j] = gf * cl[j] + gi * gg;
+            hl[j] = go * tanh(cl[j]);
+        }
+        for (int j = 0; j < P; ++j) x[j] = hl[j];
+        n_in = P;
+    }
+    free(x); free(ga); free(gb);
+}
+
+/* pred_proj = W_pred h_top + b_pred */
+void oracle_pred_proj(const oracle_model_t* m, const double* h, double* g) {
+    oracle_linear(m->w_pred, m->b_pred, h + (size_t)(m->L - 1) * m->P, m->H, m->P, g);
+}
+
+/* enc_proj[t,:] = W_enc enc[t,:] + b_enc for t < T */
+void oracle_enc_proj(const oracle_model_t* m, const float* enc, int T, double* out) {
+    double* x = (double*)malloc(sizeof(double) * (size_t)m->D);
+    for (int t = 0; t < T; ++t) {
+        for (int k = 0; k < m->D; ++k) x[k] = (double)enc[(size_t)t * m->D + k];
+        oracle_linear(m->w_enc, m->b_enc, x, m->H, m->D, out + (size_t)t * m->H);
+    }
+    free(x);
+}
+
+/* logits = W_out act(encp + g) + b_out ; z is scratch [H] */
+void oracle_joint_logits(const oracle_model_t* m, const double* encp, const double* g, double* z, double* logits) {
+    for (int k = 0; k < m->H; ++k) {
+        double s = encp[k] + g[k];
+        z[k] = (m->act == 0) ? (s > 0.0 ? s : 0.0) : tanh(s);
+    }
+    oracle_linear(m->w_out, m->b_out, z, m->V + 1, m->H, logits);
+}
+
+/* lowest index on ties; also returns the top-2 margin */
+static int argmax_margin(const double* v, int n, double* margin) {
+    int best = 0;
+    for (int i = 1; i < n; ++i)
+        if (v[i] > v[best]) best = i;
+    double second = -INFINITY;
+    for (int i = 0; i < n; ++i)
+        if (i != best && v[i] > second) second = v[i];
+    if (margin) *margin = v[best] - second;
+    return best;
+}
+
+typedef struct {
+    double *h, *c, *g, *z, *logits, *encp;
+} scratch_t;
+
+static void scratch_alloc(const oracle_model_t* m, int T, scratch_t* s) {
+    s->h = (double*)calloc((size_t)m->L * m->P, sizeof(double));
+    s->c = (double*)calloc((size_t)m->L * m->P, sizeof(double));
+    s->g = (double*)malloc(sizeof(double) * (size_t)m->H);
+    s->z = (double*)malloc(sizeof(double) * (size_t)m->H);
+    s->logits = (double*)malloc(sizeof(double) * (size_t)(m->V + 1) * 64);
+    s->encp = (double*)malloc(sizeof(double) * (size_t)(T > 0 ? T : 1) * m->H);
+}
+static void scratch_free(scratch_t* s) {
+    free(s->h); free(s->c); free(s->g); free(s->z); free(s->logits); free(s->encp);
+}
+
+/* start of sequence: zero state, feed the blank id once */
+static void decoder_start(const oracle_model_t* m, scratch_t* s) {
+    memset(s->h, 0, sizeof(double) * (size_t)m->L * m->P);
+    memset(s->c, 0, sizeof(double) * (size_t)m->L * m->P);
+    oracle_lstm_step(m, m->blank_id, s->h, s->c);
+    oracle_pred_proj(m, s->h, s->g);
+}
+static void decoder_feed(const oracle_model_t* m, scratch_t* s, int32_t tok) {
+    oracle_lstm_step(m, tok, s->h, s->c);
+    oracle_pred_proj(m, s->h, s->g);
+}
+
+/*
+ * Algorithm 1: one frame, one decision per iteration.
+ * Returns the number of tokens (may exceed max_out; only the first max_out are stored).
+ */
+int32_t oracle_decode_seq(const oracle_model_t* m, const float* enc, int32_t T, int32_t S, double margin_thr,
+                          int32_t* out_tokens, int32_t* out_frames, int32_t max_out, oracle_stats_t* st) {
+    scratch_t s;
+    scratch_alloc(m, T, &s);
+    oracle_enc_proj(m, enc, T, s.encp);
+    decoder_start(m, &s);
+    int32_t n_out = 0, t = 0, count = 0, last_emit_frame = -1;
+    while (t < T) {
+        oracle_joint_logits(m, s.encp + (size_t)t * m->H, s.g, s.z, s.logits);
+        double margin;
+        int label = argmax_margin(s.logits, m->V + 1, &margin);
+        if (st) {
+            st->steps++; st->joint_rows++; st->decisions++;
+            if (margin < margin_thr) st->low_margin++;
+        }
+        if (label != m->blank_id) {
+            if (n_out < max_out) { out_tokens[n_out] = label; out_frames[n_out] = t; }
+            n_out++;
+            if (st) { st->pred_updates++; if (t != last_emit_frame) st->emit_frames++; }
+            last_emit_frame = t;
+            decoder_feed(m, &s, label);
+            count++;
+            if (count == S) { t += 1; count = 0; if (st) st->forced++; }
+        } else {
+            t += 1;
+            count = 0;
+        }
+    }
+    scratch_free(&s);
+    return n_out;
+}
+
+/*
+ * Algorithm 2: n = min(W, T - t) frames share the current decoder state.
+ * All blank: t += n.  Otherwise i = first non-blank row, emit labels[i] at
+ * frame t+i and set t += i (the next window starts ON the emitting frame).
+ */
+int32_t oracle_decode_wind(const oracle_model_t* m, const float* enc, int32_t T, int32_t W, int32_t S,
+                           double margin_thr, int32_t* out_tokens, int32_t* out_frames, int32_t max_out,
+                           oracle_stats_t* st) {
+    if (W < 1 || W > 64) return -1;
+    scratch_t s;
+    scratch_alloc(m, T, &s);
+    oracle_enc_proj(m, enc, T, s.encp);
+    decoder_start(m, &s);
+    const int NV = m->V + 1;
+    int32_t n_out = 0, t = 0, count = 0, last_emit_frame = -1;
+    int labels[64];
+    double margins[64];
+    while (t < T) {
+        int n = (W < T - t) ? W : (T - t);
+        for (int w = 0; w < n; ++w) {
+            oracle_joint_logits(m, s.encp + (size_t)(t + w) * m->H, s.g, s.z, s.logits + (size_t)w * NV);
+            labels[w] = argmax_margin(s.logits + (size_t)w * NV, NV, &margins[w]);
+        }
+        if (st) { st->steps++; st->joint_rows += n; }
+        int i = -1;
+        for (int w = 0; w < n; ++w)
+            if (labels[w] != m->blank_id) { i = w; break; }
+        if (i < 0) {
+            if (st) {
+                st->jump_hist[n]++;
+                st->decisions += n;
+                for (int w = 0; w < n; ++w) if (margins[w] < margin_thr) st->low_margin++;
+            }
+            t += n;
+            count = 0;
+            continue;
+        }
+        if (st) {
+            st->jump_hist[i]++;
+            st->decisions += i + 1;
+            for (int w = 0; w <= i; ++w) if (margins[w] < margin_thr) st->low_margin++;
+        }
+        if (i > 0) count = 0;
+        t += i;
+        if (n_out < max_out) { out_tokens[n_out] = labels[i]; out_frames[n_out] = t; }
+        n_out++;
+        if (st) { st->pred_updates++; if (t != last_emit_frame) st->emit_frames++; }
+        last_emit_frame = t;
+        decoder_feed(m, &s, labels[i]);
+        count++;
+        if (count == S) { t += 1; count = 0; if (st) st->forced++; }
+    }
+    scratch_free(&s);
+    return n_out;
+}
+
+/*
+ * Batched front end: utterances are independent, so this is a plain loop over
+ * them (OpenMP across utterances only).  W == 0 selects Algorithm 1.
+ * enc [B, T, D]; out_tokens/out_frames [B, max_out]; out_len [B]; stats summed.
+ */
+void oracle_decode_batch(const oracle_model_t* m, const float* enc, const int32_t* enc_len, int32_t B, int32_t T,
+                         int32_t W, int32_t S, double margin_thr, int32_t* out_tokens, int32_t* out_frames,
+                         int32_t* out_len, int32_t max_out, oracle_stats_t* st_total) {
+    oracle_stats_t* sts = (oracle_stats_t*)calloc((size_t)B, sizeof(oracle_stats_t));
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        const float* e = enc + (size_t)b * T * m->D;
+        int32_t* ot = out_tokens + (size_t)b * max_out;
+        int32_t* of = out_frames + (size_t)b * max_out;
+        if (W == 0)
+            out_len[b] = oracle_decode_seq(m, e, enc_len[b], S, margin_thr, ot, of, max_out, &sts[b]);
+        else
+            out_len[b] = oracle_decode_wind(m, e, enc_len[b], W, S, margin_thr, ot, of, max_out, &sts[b]);
+    }
+    if (st_total) {
+        memset(st_total, 0, sizeof(*st_total));
+        for (int b = 0; b < B; ++b) {
+            st_total->steps += sts[b].steps;
+            st_total->joint_rows += sts[b].joint_rows;
+            st_total->pred_updates += sts[b].pred_updates;
+            st_total->forced += sts[b].forced;
+            st_total->low_margin += sts[b].low_margin;
+            st_total->decisions += sts[b].decisions;
+            st_total->emit_frames += sts[b].emit_frames;
+            for (int k = 0; k < 65; ++k) st_total->jump_hist[k] += sts[b].jump_hist[k];
+        }
+    }
+    free(sts);
+}
+
+/*
+ * Replay check of a (token, frame) sequence produced elsewhere against the
+ * sequential definition.  Walk frames from 0; the sequence implies one choice
+ * at every decision of Algorithm 1 (the listed token at its frame, blank at
+ * every frame that is left without having hit the S cap).  Each implied choice
+ * must be the oracle's argmax, or its oracle logit must lie within
+ * `margin_thr` of the oracle's maximum (a low-margin decision: counted).
+ * Returns 0 when consistent, else a positive code; *bad_pos gets the frame.
+ *   1: implied choice loses by more than the margin
+ *   2: frames not non-decreasing / out of range / more than S tokens on a frame
+ *   3: token out of range or equal to blank
+ */
+int32_t oracle_replay_verify(const oracle_model_t* m, const float* enc, int32_t T, int32_t S, double margin_thr,
+                             const int32_t* tokens, const int32_t* frames, int32_t n, int64_t* n_decisions,
+                             int64_t* n_low_margin, int64_t* n_not_argmax, int32_t* bad_pos) {
+    scratch_t s;
+    scratch_alloc(m, T, &s);
+    oracle_enc_proj(m, enc, T, s.encp);
+    decoder_start(m, &s);
+    int32_t rc = 0, t = 0, count = 0, idx = 0;
+    int64_t dec = 0, low = 0, notmax = 0;
+    for (int k = 0; k < n && !rc; ++k) {
+        if (tokens[k] < 0 || tokens[k] > m->V || tokens[k] == m->blank_id) { rc = 3; *bad_pos = k; }
+        if (frames[k] < 0 || frames[k] >= T || (k > 0 && frames[k] < frames[k - 1])) { rc = 2; *bad_pos = k; }
+    }
+    while (!rc && t < T) {
+        oracle_joint_logits(m, s.encp + (size_t)t * m->H, s.g, s.z, s.logits);
+        double margin;
+        int best = argmax_margin(s.logits, m->V + 1, &margin);
+        int choice = (idx < n && frames[idx] == t) ? tokens[idx] : m->blank_id;
+        if (idx < n && frames[idx] < t) { rc = 2; *bad_pos = t; break; }
+        dec++;
+        if (margin < margin_thr) low++;
+        if (choice != best) {
+            notmax++;
+            if (!(s.logits[choice] >= s.logits[best] - margin_thr)) { rc = 1; *bad_pos = t; break; }
+        }
+        if (choice != m->blank_id) {
+            decoder_feed(m, &s, choice);
+            idx++;
+            count++;
+            if (count == S) { t += 1; count = 0; }
+        } else {
+            t += 1;
+            count = 0;
+        }
+    }
+    if (!rc && idx != n) { rc = 2; *bad_pos = T; }
+    if (n_decisions) *n_decisions = dec;
+    if (n_low_margin) *n_low_margin = low;
+    if (n_not_argmax) *n_not_argmax = notmax;
+    scratch_free(&s);
+    return rc;
+}
+
+/*
+ * Teacher-forced window logits: feed `prefix` (after the start-of-sequence
+ * blank) to the decoder, then evaluate the joint at frames t0 .. t0+n-1,
+ * n = min(W, T - t0).  logits [W, V+1] fp64; rows >= n are left untouched.
+ * Optionally returns pred_proj (g, [H]) and the top-layer state.
+ */
+int32_t oracle_eval_joint_window(const oracle_model_t* m, const float* enc, int32_t T, const int32_t* prefix,
+                                 int32_t prefix_len, int32_t t0, int32_t W, double* logits, double* g_out,
+                                 double* h_out, double* c_out) {
+    scratch_t s;
+    scratch_alloc(m, 0, &s);
+    decoder_start(m, &s);
+    for (int k = 0; k < prefix_len; ++k) decoder_feed(m, &s, prefix[k]);
+    int n = (W < T - t0) ? W : (T - t0);
+    if (n < 0) n = 0;
+    double* ep = (double*)malloc(sizeof(double) * (size_t)m->H);
+    for (int w = 0; w < n; ++w) {
+        oracle_enc_proj(m, enc + (size_t)(t0 + w) * m->D, 1, ep);
+        oracle_joint_logits(m, ep, s.g, s.z, logits + (size_t)w * (m->V + 1));
+    }
+    if (g_out) memcpy(g_out, s.g, sizeof(double) * (size_t)m->H);
+    if (h_out) memcpy(h_out, s.h, sizeof(double) * (size_t)m->L * m->P);
+    if (c_out) memcpy(c_out, s.c, sizeof(double) * (size_t)m->L * m->P);
+    free(ep);
+    scratch_free(&s);
+    return n;
+}

@@ -1,0 +1,358 @@
+"""Pins for the CPU oracle: closed forms, library fp64 routines, brute force, invariants.
+
+The paper prints no worked numeric example, so the oracle is fixed by what the
+paper and the mathematics fix instead:
+  * Algorithm 2 returns exactly Algorithm 1's result for every window size
+    (results section: identical accuracy at every W; method section: frames
+    skipped by a jump are blank under the same decoder state);
+  * the blank / non-blank rules of the background section, checked by brute
+    force with an independent evaluator that re-runs a library LSTM over the
+    whole prefix;
+  * linear layers and the LSTM cell against library fp64 routines and closed forms.
+"""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from naive_model import NaiveModel, random_weights
+
+
+def rng(seed):
+    return np.random.default_rng(seed)
+
+
+# ---------------------------------------------------------------------------
+# linear layers, LSTM cell, joint: library routines and closed forms
+# ---------------------------------------------------------------------------
+def test_linear_matches_fp64_matmul():
+    r = rng(1)
+    W = r.standard_normal((37, 53)).astype(np.float32)
+    b = r.standard_normal(37).astype(np.float32)
+    x = r.standard_normal(53)
+    y = oracle.linear(W, b, x)
+    ref = W.astype(np.float64) @ x + b.astype(np.float64)
+    assert np.max(np.abs(y - ref)) < 1e-12
+    # a transposed operand or a dropped bias must show
+    assert np.max(np.abs(y - (W.astype(np.float64) @ x))) > 1e-3
+    y0 = oracle.linear(W, None, x)
+    assert np.max(np.abs(y0 - W.astype(np.float64) @ x)) < 1e-12
+
+
+def test_linear_unit_vectors_pick_columns():
+    W = np.arange(12, dtype=np.float32).reshape(3, 4)
+    for k in range(4):
+        x = np.zeros(4)
+        x[k] = 1.0
+        assert np.array_equal(oracle.linear(W, None, x), W[:, k].astype(np.float64))
+
+
+def test_lstm_zero_weights_closed_form():
+    # all matrices zero: gates are the bias sums; from zero state
+    # c = sigma(bi) * tanh(bg), h = sigma(bo) * tanh(c); f plays no role at step 1,
+    # at step 2 c2 = sigma(bf) * c + sigma(bi) * tanh(bg).
+    P, E, V = 3, 2, 4
+    w = random_weights(rng(2), 2, E, P, 1, 2, V)
+    w["w_ih"] = [np.zeros((4 * P, E), np.float32)]
+    w["w_hh"] = [np.zeros((4 * P, P), np.float32)]
+    bi, bf, bg, bo = 0.3, -0.7, 1.1, 0.4
+    b = np.concatenate([np.full(P, v, np.float32) for v in (bi, bf, bg, bo)])
+    w["b_ih"] = [b / 2]
+    w["b_hh"] = [b / 2]
+    m = oracle.Model(w)
+    sig = lambda v: 1.0 / (1.0 + np.exp(-np.float64(np.float32(v))))
+    bg64 = np.float64(np.float32(bg))
+    h, c = oracle.lstm_step(m, 1, np.zeros((1, P)), np.zeros((1, P)))
+    c1 = sig(bi) * np.tanh(bg64)
+    assert np.allclose(c, c1, atol=1e-7) and np.allclose(h, sig(bo) * np.tanh(c1), atol=1e-7)
+    h, c = oracle.lstm_step(m, 2, h, c)
+    c2 = sig(bf) * c1 + sig(bi) * np.tanh(bg64)
+    assert np.allclose(c, c2, atol=1e-7) and np.allclose(h, sig(bo) * np.tanh(c2), atol=1e-7)
+
+
+def test_lstm_all_zero_gives_zero_state():
+    P, E, V = 4, 3, 5
+    w = random_weights(rng(3), 2, E, P, 2, 2, V)
+    for k in ("w_ih", "w_hh", "b_ih", "b_hh"):
+        w[k] = [np.zeros_like(a) for a in w[k]]
+    m = oracle.Model(w)
+    h, c = oracle.lstm_step(m, 2, np.zeros((2, P)), np.zeros((2, P)))
+    assert np.all(h == 0) and np.all(c == 0)
+
+
+@pytest.mark.parametrize("L", [1, 2, 3])
+def test_lstm_matches_torch_lstm(L):
+    r = rng(10 + L)
+    D, E, P, H, V = 5, 7, 6, 4, 9
+    w = random_weights(r, D, E, P, L, H, V, bias_scale=0.5, emb_zero_blank=False)
+    m = oracle.Model(w)
+    nm = NaiveModel(w)
+    prefix = [3, 0, 8, 8, 1]
+    h = np.zeros((L, P))
+    c = np.zeros((L, P))
+    h, c = oracle.lstm_step(m, w["blank_id"], h, c)
+    for k, tok in enumerate(prefix):
+        h, c = oracle.lstm_step(m, tok, h, c)
+        h_top, hn, cn = nm.decoder(prefix[: k + 1])
+        assert np.max(np.abs(h - hn.numpy())) < 1e-12
+        assert np.max(np.abs(c - cn.numpy())) < 1e-12
+    g = oracle.pred_proj(m, h)
+    ref = w["w_pred"].astype(np.float64) @ h[-1] + w["b_pred"].astype(np.float64)
+    assert np.max(np.abs(g - ref)) < 1e-12
+
+
+@pytest.mark.parametrize("act", [0, 1])
+def test_enc_proj_and_joint_match_fp64(act):
+    r = rng(20 + act)
+    D, E, P, H, V = 6, 4, 5, 8, 7
+    w = random_weights(r, D, E, P, 1, H, V, act=act, bias_scale=0.3)
+    m = oracle.Model(w)
+    enc = r.standard_normal((9, D)).astype(np.float32)
+    ep = oracle.enc_proj(m, enc)
+    ref = enc.astype(np.float64) @ w["w_enc"].astype(np.float64).T + w["b_enc"].astype(np.float64)
+    assert np.max(np.abs(ep - ref)) < 1e-12
+    g = r.standard_normal(H)
+    lg = oracle.joint_logits(m, ep[4], g)
+    s = ref[4] + g
+    z = np.maximum(s, 0) if act == 0 else np.tanh(s)
+    ref_l = w["w_out"].astype(np.float64) @ z + w["b_out"].astype(np.float64)
+    assert np.max(np.abs(lg - ref_l)) < 1e-12
+    # the other activation must differ (guards against an ignored act flag)
+    z2 = np.tanh(s) if act == 0 else np.maximum(s, 0)
+    assert np.max(np.abs(lg - (w["w_out"].astype(np.float64) @ z2 + w["b_out"]))) > 1e-3
+
+
+def test_eval_joint_window_matches_independent_evaluator():
+    r = rng(30)
+    D, E, P, H, V = 5, 4, 6, 7, 6
+    w = random_weights(r, D, E, P, 2, H, V, act=1, bias_scale=0.2, blank_id=2)
+    m = oracle.Model(w)
+    nm = NaiveModel(w)
+    T = 11
+    enc = r.standard_normal((T, D)).astype(np.float32)
+    prefix = [0, 5, 1, 1]
+    for t0, W in [(0, 4), (9, 4), (3, 1), (10, 16)]:
+        lg, g, h, c = oracle.eval_joint_window(m, enc, T, prefix, t0, W)
+        assert lg.shape[0] == min(W, T - t0)
+        for k in range(lg.shape[0]):
+            assert np.max(np.abs(lg[k] - nm.logits(enc[t0 + k], prefix))) < 1e-11
+
+
+# ---------------------------------------------------------------------------
+# brute force: tabulate argmax joint(t, prefix) with the independent evaluator
+# ---------------------------------------------------------------------------
+def brute_force_greedy(nm, enc, S):
+    """Algorithm 1's rules walked on independently evaluated logits.
+
+    Background-section rules: a non-blank label is appended and the frame is kept;
+    blank advances the frame and keeps the decoder input.  The S cap forces an
+    advance after the S-th consecutive emission on one frame.
+    """
+    T = enc.shape[0]
+    hyp, frames, t, count = [], [], 0, 0
+    while t < T:
+        lg = nm.logits(enc[t], hyp)
+        label = int(np.argmax(lg))  # numpy argmax returns the first maximum
+        if label != nm.blank:
+            hyp.append(label)
+            frames.append(t)
+            count += 1
+            if count == S:
+                t += 1
+                count = 0
+        else:
+            t += 1
+            count = 0
+    return hyp, frames
+
+
+@pytest.mark.parametrize("seed,blank_id,act,S,bias", [
+    (0, None, 0, 2, 0.0), (1, 0, 1, 3, 0.5), (2, 1, 0, 1, -0.5), (3, None, 1, 4, 1.0), (4, 2, 0, 2, 0.3),
+    (5, None, 0, 3, -2.0),
+])
+def test_sequential_greedy_matches_brute_force(seed, blank_id, act, S, bias):
+    r = rng(100 + seed)
+    D, E, P, H, V, L = 3, 3, 4, 4, 3, 1 + seed % 2
+    w = random_weights(r, D, E, P, L, H, V, blank_id=blank_id, act=act, blank_bias=bias, bias_scale=0.3,
+                       emb_zero_blank=False)
+    nm = NaiveModel(w)
+    m = oracle.Model(w)
+    T = 6
+    enc = r.standard_normal((1, T, D)).astype(np.float32)
+    hyp, frames = brute_force_greedy(nm, enc[0], S)
+    tok, frm, n, st = oracle.decode_batch(m, enc, np.array([T], np.int32), W=0, S=S)
+    assert list(tok[0, : n[0]]) == hyp
+    assert list(frm[0, : n[0]]) == frames
+    for W in (1, 2, 3, 5, 6, 11):
+        tokw, frmw, nw, _ = oracle.decode_batch(m, enc, np.array([T], np.int32), W=W, S=S)
+        assert list(tokw[0, : nw[0]]) == hyp, W
+        assert list(frmw[0, : nw[0]]) == frames, W
+
+
+def test_brute_force_table_over_all_reachable_prefixes():
+    # tiny enough to enumerate: T=4, V=2, S=2 -> every (t, prefix) reachable under the cap
+    r = rng(200)
+    D, E, P, H, V, S, T = 2, 2, 3, 3, 2, 2, 4
+    w = random_weights(r, D, E, P, 1, H, V, blank_bias=0.2, bias_scale=0.2, emb_zero_blank=False)
+    nm, m = NaiveModel(w), oracle.Model(w)
+    enc = r.standard_normal((T, D)).astype(np.float32)
+    checked = 0
+    for n in range(0, 4):
+        for prefix in itertools.product(range(V), repeat=n):
+            for t0 in range(T):
+                lg, *_ = oracle.eval_joint_window(m, enc, T, list(prefix), t0, 1)
+                ref = nm.logits(enc[t0], list(prefix))
+                assert int(np.argmax(lg[0])) == int(np.argmax(ref))
+                assert np.max(np.abs(lg[0] - ref)) < 1e-11
+                checked += 1
+    assert checked == (1 + 2 + 4 + 8) * T
+
+
+# ---------------------------------------------------------------------------
+# invariants of the decoding loops
+# ---------------------------------------------------------------------------
+def small_case(seed, B=3, T=40, bias=1.0, S=3, V=12, L=1, act=0, blank_id=None):
+    r = rng(300 + seed)
+    D, E, P, H = 8, 6, 7, 10
+    w = random_weights(r, D, E, P, L, H, V, blank_id=blank_id, act=act, blank_bias=bias, bias_scale=0.1)
+    lens = r.integers(0, T + 1, size=B).astype(np.int32)
+    lens[0] = T
+    enc = r.standard_normal((B, T, D)).astype(np.float32)
+    for b in range(B):
+        enc[b, lens[b]:] = np.nan  # poison: padded frames must never be decoded
+    return w, enc, lens
+
+
+@pytest.mark.parametrize("seed,bias,S", [(0, 1.0, 3), (1, 0.0, 2), (2, 2.0, 5), (3, -1.0, 1), (4, 1.5, 10), (5, 0.7, 4)])
+def test_wind_equals_sequential_for_every_window(seed, bias, S):
+    w, enc, lens = small_case(seed, bias=bias, S=S, L=1 + seed % 2, act=seed % 2, blank_id=None if seed % 3 else 0)
+    m = oracle.Model(w)
+    T = enc.shape[1]
+    tok0, frm0, n0, st0 = oracle.decode_batch(m, enc, lens, W=0, S=S)
+    assert n0.sum() > 0 or bias > 1.9
+    for W in (1, 2, 3, 4, 8, 16, T, T + 5):
+        if W > 64:
+            continue
+        tok, frm, n, st = oracle.decode_batch(m, enc, lens, W=W, S=S)
+        assert np.array_equal(n, n0), W
+        assert np.array_equal(tok, tok0), W
+        assert np.array_equal(frm, frm0), W
+        # jumps lie in [0, W]; every frame is consumed exactly once by a jump or a forced advance
+        hist = np.array(st["jump_hist"])
+        assert hist[W + 1:].sum() == 0
+        assert (hist * np.arange(65)).sum() + st["forced"] == lens.sum()
+        assert hist.sum() == st["steps"]
+        assert st["forced"] == st0["forced"]
+        assert st["pred_updates"] == n.sum()
+        if W > 1:
+            assert st["steps"] <= st0["steps"]
+
+
+def test_max_symbols_is_honoured():
+    for seed, S in [(0, 1), (1, 2), (2, 3)]:
+        w, enc, lens = small_case(10 + seed, bias=-3.0, S=S)  # blank strongly disfavoured
+        m = oracle.Model(w)
+        for W in (0, 1, 4):
+            tok, frm, n, st = oracle.decode_batch(m, enc, lens, W=W, S=S)
+            for b in range(len(lens)):
+                f = frm[b, : n[b]]
+                assert np.all(np.diff(f) >= 0)
+                if n[b]:
+                    assert np.bincount(f).max() <= S
+                    assert f.max() < lens[b]
+            # with blank this unlikely nearly every frame hits the cap
+            assert st["forced"] > 0.5 * lens.sum()
+            assert n.sum() >= S * st["forced"]
+
+
+def test_huge_cap_equals_uncapped_when_loop_terminates():
+    w, enc, lens = small_case(20, bias=1.2, S=3)
+    m = oracle.Model(w)
+    a = oracle.decode_batch(m, enc, lens, W=4, S=50)
+    b = oracle.decode_batch(m, enc, lens, W=4, S=1000)
+    if a[3]["forced"] == 0:
+        assert np.array_equal(a[0][:, :50], b[0][:, :50]) and np.array_equal(a[2], b[2])
+
+
+def test_all_blank_and_zero_length():
+    w, enc, lens = small_case(30, bias=50.0)
+    lens[1] = 0
+    m = oracle.Model(w)
+    for W in (0, 1, 4, 16):
+        tok, frm, n, st = oracle.decode_batch(m, enc, lens, W=W, S=3)
+        assert n.sum() == 0 and st["pred_updates"] == 0
+        if W:
+            assert st["steps"] == sum(-(-int(l) // W) for l in lens)
+
+
+def test_batch_equals_single_and_padding_is_never_read():
+    w, enc, lens = small_case(40, B=4, bias=0.8)
+    m = oracle.Model(w)
+    tok, frm, n, _ = oracle.decode_batch(m, enc, lens, W=4, S=3)
+    for b in range(4):
+        e1 = np.ascontiguousarray(enc[b : b + 1, : max(1, lens[b])])
+        t1, f1, n1, _ = oracle.decode_batch(m, e1, lens[b : b + 1], W=4, S=3, max_out=tok.shape[1])
+        assert n1[0] == n[b]
+        assert np.array_equal(t1[0, : n1[0]], tok[b, : n[b]])
+        assert np.array_equal(f1[0, : n1[0]], frm[b, : n[b]])
+
+
+def test_output_overflow_reports_full_count():
+    w, enc, lens = small_case(50, bias=-3.0, S=3)
+    m = oracle.Model(w)
+    full = oracle.decode_batch(m, enc, lens, W=4, S=3)
+    cut = oracle.decode_batch(m, enc, lens, W=4, S=3, max_out=5)
+    assert np.array_equal(full[2], cut[2])
+    assert np.array_equal(full[0][:, :5], cut[0])
+
+
+# ---------------------------------------------------------------------------
+# replay check: accepts the oracle's own result, rejects a planted mistake
+# ---------------------------------------------------------------------------
+def test_replay_accepts_own_output_and_rejects_mistakes():
+    w, enc, lens = small_case(60, B=2, bias=0.9, S=3)
+    m = oracle.Model(w)
+    tok, frm, n, st = oracle.decode_batch(m, enc, lens, W=4, S=3)
+    b = 0
+    T = int(lens[b])
+    tk, fr = tok[b, : n[b]].copy(), frm[b, : n[b]].copy()
+    assert n[b] >= 3
+    ok = oracle.replay_verify(m, enc[b], T, 3, tk, fr, margin_thr=0.0)
+    assert ok["rc"] == 0 and ok["not_argmax"] == 0
+    seq = oracle.decode_batch(m, enc[b : b + 1], lens[b : b + 1], W=0, S=3)
+    assert ok["decisions"] == seq[3]["decisions"]
+    # drop a token: the frame is then implied blank, which the oracle does not agree with
+    bad = oracle.replay_verify(m, enc[b], T, 3, np.delete(tk, 1), np.delete(fr, 1), margin_thr=0.0)
+    assert bad["rc"] == 1
+    # frames out of order
+    fr2 = fr.copy()
+    fr2[0], fr2[-1] = fr[-1], fr[0]
+    if fr[0] != fr[-1]:
+        assert oracle.replay_verify(m, enc[b], T, 3, tk, fr2)["rc"] == 2
+    # blank as a token
+    tk3 = tk.copy()
+    tk3[0] = w["blank_id"]
+    assert oracle.replay_verify(m, enc[b], T, 3, tk3, fr)["rc"] == 3
+    # a wrong token is tolerated only inside the margin
+    lg, *_ = oracle.eval_joint_window(m, enc[b], T, [], int(fr[0]), 1)
+    order = np.argsort(-lg[0])
+    second = int(order[1]) if int(order[1]) != w["blank_id"] else int(order[2])
+    gap = lg[0][order[0]] - lg[0][second]
+    tk4 = tk.copy()
+    tk4[0] = second
+    # with a margin below the gap the first decision fails; whatever follows is irrelevant
+    assert oracle.replay_verify(m, enc[b], T, 3, tk4[:1], fr[:1], margin_thr=gap * 0.5)["rc"] in (1, 2)
+    res = oracle.replay_verify(m, enc[b], T, 3, tk4[:1], fr[:1], margin_thr=gap * 0.5)
+    assert res["rc"] == 1 and res["bad_pos"] == fr[0]
+
+
+def test_low_margin_count_matches_direct_count():
+    w, enc, lens = small_case(70, B=1, bias=0.9, S=3)
+    m = oracle.Model(w)
+    thr = 0.3
+    _, _, _, st = oracle.decode_batch(m, enc, lens, W=0, S=3, margin_thr=thr)
+    _, _, _, stw = oracle.decode_batch(m, enc, lens, W=4, S=3, margin_thr=thr)
+    assert st["low_margin"] == stw["low_margin"] and st["decisions"] == stw["decisions"]
+    assert 0 < st["low_margin"] < st["decisions"]
