@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of batched greedy WIND decoding on synthetic data (one JSON line on stdout).
+
+A "step" is one pass of the whole hot path over one batch: a single
+``wind_decode_greedy`` call (encoder projection, start-of-sequence decoder update,
+device-resident decoding loop) on the B = 128 FastConformer-Large-shaped workload.
+Metric: RTFx = audio seconds decoded per second at 80 ms per encoder frame.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME] [--window W]
+
+With N > 1 (under torchrun) every rank decodes its own replica of the batch: the path
+has no exchange step, so there is no collective in it; ranks only meet at the barrier
+and at the max-over-ranks of the device time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FRAME_SECONDS = 0.08
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ---------------------------------------------------------------------------
+# clocks during the timed region
+# ---------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str | None):
+        self.uuid = uuid
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+            if self.uuid:
+                cmd += ["-i", self.uuid]
+            self.proc = subprocess.Popen(cmd, stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    sm.append(float(parts[0])); mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ---------------------------------------------------------------------------
+# rank plumbing (barrier + max over ranks); gloo on CPU in the tests, nccl on GPUs
+# ---------------------------------------------------------------------------
+def dist_setup(n_gpus: int, backend: str | None = None):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        if not dist.is_initialized():
+            dist.init_process_group(backend=backend or "nccl", rank=rank, world_size=world)
+    return rank, local, world
+
+
+def barrier(world: int, device=None):
+    if world > 1:
+        import torch.distributed as dist
+        if device is not None and dist.get_backend() == "nccl":
+            dist.barrier(device_ids=[device.index])
+        else:
+            dist.barrier()
+
+
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if (device is not None and dist.get_backend() == "nccl") else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_rtfx(audio_seconds_per_rank_step: float, steps: int, ms_local: float, world: int, device=None):
+    """Whole-job RTFx from per-rank device time: every rank decodes its own replica."""
+    ms = max_over_ranks(ms_local, world, device)
+    total_audio = audio_seconds_per_rank_step * steps * world
+    return total_audio / (ms * 1e-3), ms / steps
+
+
+# ---------------------------------------------------------------------------
+# CPU baseline: the oracle as it stands, on a bounded sample of the workload
+# ---------------------------------------------------------------------------
+def oracle_sample(cfg, enc, lens, seconds_target: float, cores: int):
+    """First k utterances (batch order) whose estimated oracle cost is about `seconds_target`."""
+    macs_per_row = cfg.H * (cfg.V + 1)
+    est_rate = 0.6e9 * cores  # fp64 MAC/s, rough
+    budget = seconds_target * est_rate
+    # rows per frame at window W on this generator: about (tokens per frame) * min(W, a few) + 1
+    rows_per_frame = 3.0 * min(cfg.W, 8) * 0.6 + 1.0
+    acc, k = 0.0, 0
+    while k < len(lens) and (k < 1 or acc + lens[k] * rows_per_frame * macs_per_row <= budget):
+        acc += lens[k] * rows_per_frame * macs_per_row
+        k += 1
+    return k
+
+
+def run_cpu_baseline(cfg, weights, enc, lens, W, seconds_target=15.0):
+    import oracle
+    cores = os.cpu_count() or 1
+    k = oracle_sample(cfg, enc, lens, seconds_target, cores)
+    om = oracle.Model(weights)
+    sub = np.ascontiguousarray(enc[:k])
+    t0 = time.perf_counter()
+    _, _, on, st = oracle.decode_batch(om, sub, lens[:k], W=W, S=cfg.S)
+    dt = time.perf_counter() - t0
+    audio = float(lens[:k].sum()) * FRAME_SECONDS
+    return dict(value=audio / dt, unit="audio-s/s", cores=cores, kind="oracle",
+                sample=f"first {k} of {cfg.B} utterances ({int(lens[:k].sum())} frames), W={W}, one run, {dt:.1f} s",
+                seconds=dt, steps=st["steps"])
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3_large_b128")
+    ap.add_argument("--window", type=int, default=0, help="override the workload's window (0 = its default)")
+    ap.add_argument("--kernels", type=int, default=0, help="0 auto, 1 plain-ALU kernels, 2 tensor-core kernels")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the W=1 comparison, e2e and per-kernel timing legs")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+
+    import wind_synth as ws
+    cfg = ws.CONFIGS[args.workload]
+    W = args.window or cfg.W
+
+    if args.impl == "reference":
+        return reference_arm(args, cfg, W)
+
+    import torch
+    import paper_2505_13765_b200 as pkg
+
+    rank, local, world = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    pkg.load_library()
+    pkg.wind_set_kernels(args.kernels)
+    peaks = load_peaks()
+
+    weights = ws.make_model(cfg)
+    enc_np, lens_np = ws.make_enc(cfg, pad="zero")
+    model = pkg.WindModel(weights, device=dev)
+    B, T, D = enc_np.shape
+    max_out = T * cfg.S
+    enc_h = torch.from_numpy(enc_np).to(model.torch_dtype).pin_memory()
+    len_h = torch.from_numpy(lens_np).pin_memory()
+    enc_d = enc_h.to(dev)
+    len_d = len_h.to(dev)
+    tok_d = torch.full((B, max_out), -1, dtype=torch.int32, device=dev)
+    frm_d = torch.full((B, max_out), -1, dtype=torch.int32, device=dev)
+    ol_d = torch.zeros(B, dtype=torch.int32, device=dev)
+    wsb = pkg.alloc_workspace(model, B, T, max(W, 1), host_staging_max_out=max_out)
+    stream = torch.cuda.current_stream()
+    audio_s = float(lens_np.sum()) * FRAME_SECONDS
+
+    def step(window=W):
+        pkg.wind_decode_greedy(model, enc_d, len_d, window, cfg.S, tok_d, frm_d, ol_d, wsb, stream=stream)
+
+    def timed(fn, k):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier(world, dev)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(k):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier(world, dev)
+        return e0.elapsed_time(e1)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    uuid = None
+    try:
+        uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        pass
+    sampler = ClockSampler(uuid)
+    sampler.start()
+    ms_local = timed(step, args.steps)
+    clocks = sampler.stop()
+    stats = pkg.wind_read_stats(wsb, stream)
+    value, ms_per_step = aggregate_rtfx(audio_s, args.steps, ms_local, world, dev)
+    launches = (stats["launches_setup"] + stats["steps"] * stats["launches_per_step"]) * args.steps
+    tokens = stats["tokens"]
+
+    out = {
+        "metric": "greedy WIND RTFx (audio-s/s at 80 ms/frame)", "value": value, "unit": "audio-s/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "frames": int(lens_np.sum()), "T_max": int(lens_np.max()), "W": W,
+                   "max_symbols": cfg.S, "D": cfg.D, "E": cfg.E, "P": cfg.P, "L": cfg.L, "H": cfg.H, "V": cfg.V,
+                   "l2": "inputs larger than L2 (enc and enc_proj are each > 126 MB)",
+                   "multi_gpu": "replicas only (no exchange step in the path)"},
+        "frames_per_s": float(lens_np.sum()) * args.steps * world / (ms_per_step * args.steps * 1e-3),
+        "loop_steps": stats["steps"], "us_per_loop_step": ms_per_step * 1e3 / max(1, stats["steps"]),
+        "tokens": tokens, "tokens_per_frame": tokens / max(1, stats["frames"]),
+        "launches_per_token": (stats["launches_setup"] + stats["steps"] * stats["launches_per_step"]) / max(1, tokens),
+        "jump_hist": stats["jump_hist"][: W + 1], "kernels": {1: "simt", 2: "tensor"}.get(stats["kernels"], "?"),
+        "gpu_launches": launches, "clocks": clocks,
+    }
+
+    if rank == 0 and not args.no_extras:
+        # same library at W = 1 (the sequential baseline)
+        if W != 1:
+            for _ in range(2):
+                step(1)
+            k1 = max(1, min(args.steps, 3))
+            ms1 = timed(lambda: step(1), k1) if world == 1 else None
+            if ms1 is not None:
+                st1 = pkg.wind_read_stats(wsb, stream)
+                out["w1"] = {"value": audio_s * k1 / (ms1 * 1e-3), "ms_per_step": ms1 / k1, "loop_steps": st1["steps"]}
+                out["speedup_vs_w1"] = (ms1 / k1) / ms_per_step
+        # end to end through the host-buffer entry point: H2D of enc and lengths, D2H of the outputs, every step
+        if world == 1:
+            tok_h = torch.empty((B, max_out), dtype=torch.int32).pin_memory()
+            frm_h = torch.empty((B, max_out), dtype=torch.int32).pin_memory()
+            ol_h = torch.empty(B, dtype=torch.int32).pin_memory()
+
+            def step_host():
+                pkg.wind_decode_greedy_host(model, enc_h, len_h, W, cfg.S, tok_h, frm_h, ol_h, wsb, stream=stream)
+
+            step_host()
+            ke = max(1, min(args.steps, 3))
+            ms_e = timed(step_host, ke)
+            out["e2e"] = {"value": audio_s * ke / (ms_e * 1e-3), "unit": "audio-s/s",
+                          "h2d_bytes_per_step": int(enc_h.numel() * enc_h.element_size() + len_h.numel() * 4),
+                          "d2h_bytes_per_step": int((tok_h.numel() + frm_h.numel() + ol_h.numel()) * 4)}
+    elif world > 1:
+        # every rank must take part in the same collectives: none are issued in the extras
+        pass
+
+    if rank == 0:
+        out["roofline"] = roofline(pkg, model, cfg, W, enc_d, len_d, tok_d, frm_d, ol_d, wsb, stream, stats, peaks) \
+            if (world == 1 and not args.no_extras) else None
+        if not args.no_cpu_baseline and world == 1:
+            cb = run_cpu_baseline(cfg, weights, enc_np, lens_np, W)
+            out["cpu_baseline"] = cb
+        else:
+            out["cpu_baseline"] = None
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def roofline(pkg, model, cfg, W, enc_d, len_d, tok_d, frm_d, ol_d, wsb, stream, stats, peaks):
+    """Roofline entry for the fused joint kernel, the dominant kernel of the loop.
+
+    Algorithmic work per launch = 2 * H * (V+1) flop per evaluated window row (rows of finished
+    utterances and tile padding do not count); rows per launch = joint_rows / steps of the decode.
+    The launch duration comes from CUDA events recorded around every launch of the kernel on its
+    stream by the library's per-kernel timing entry point, over one full decode of the workload.
+    """
+    prof = getattr(pkg, "wind_profile_decode", None)
+    if prof is None:
+        return None
+    res = prof(model, enc_d, len_d, W, cfg.S, tok_d, frm_d, ol_d, wsb, stream=stream)
+    rows_per_launch = stats["joint_rows"] / max(1, stats["steps"])
+    flop = 2.0 * cfg.H * (cfg.V + 1) * rows_per_launch
+    dur_s = res["joint_ms"] * 1e-3 / max(1, res["joint_launches"])
+    achieved = flop / dur_s / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    return {"kernel": "fused windowed joint", "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+            "frac": achieved / peak, "peak_source": peaks["source"] + " sustained bf16", "traffic": None,
+            "avg_launch_us": dur_s * 1e6, "rows_per_launch": rows_per_launch,
+            "per_kernel_ms": {k: res[k] for k in res if k.endswith("_ms")}}
+
+
+def reference_arm(args, cfg, W):
+    """The oracle as it stands, timed on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import wind_synth as ws
+    weights = ws.make_model(cfg)
+    enc_np, lens_np = ws.make_enc(cfg, pad="zero")
+    per_step_target = max(2.0, min(15.0, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        run_cpu_baseline(cfg, weights, enc_np, lens_np, W, per_step_target)
+    vals, secs = [], []
+    for _ in range(max(1, args.steps)):
+        cb = run_cpu_baseline(cfg, weights, enc_np, lens_np, W, per_step_target)
+        vals.append(cb["value"]); secs.append(cb["seconds"])
+    value = float(np.sum([v * s for v, s in zip(vals, secs)]) / np.sum(secs))
+    cb["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": "greedy WIND RTFx (audio-s/s at 80 ms/frame)", "value": value, "unit": "audio-s/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(np.mean(secs)) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "W": W, "sample": cb["sample"]},
+        "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": value, "unit": "audio-s/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,197 @@
+/*
+ * wind.h -- C ABI of the B200 (sm_100a) library for batched greedy RNN-Transducer
+ * decoding with windowed non-blank detection (WIND).
+ *
+ * The library computes, per utterance, exactly what the sequential greedy procedure
+ * computes (Algorithm 1, "RNN-T Inference Algorithm"): scan the encoder frames left to
+ * right; at frame t evaluate the joiner on (enc[t], decoder state) and take the argmax;
+ * a non-blank label is appended, fed to the decoder and t is kept; blank keeps the
+ * decoder state and advances t (rules 1 and 2 of the background section).  With a window
+ * W > 1 it follows Algorithm 2 ("WIND Algorithm"): the joiner is evaluated on
+ * enc[t : t+n], n = min(W, len - t), against the ONE current decoder state, every row's
+ * argmax is taken, and the decoder jumps to the first non-blank row (t += i, label
+ * appended) or past the whole window (t += n) when all rows are blank.  W = 1 is the
+ * sequential baseline.  The batch runs in lock step (one joiner call and one masked
+ * decoder update per step for all utterances), which the paper describes in prose only
+ * (method section, last paragraph; CUDA-graph paragraph of the analysis section).
+ *
+ * Model (the paper leaves decoder and joiner abstract; these are the shapes used here):
+ *   decoder : embedding [V+1, E] + L-layer LSTM (hidden P, gate order i,f,g,o, biases
+ *             b_ih + b_hh, zero initial state), one token per update; the
+ *             start-of-sequence input is blank_id;
+ *   joiner  : logits = W_out * act(W_enc*f + b_enc + W_pred*h_top + b_pred) + b_out,
+ *             V+1 logits, argmax with the lowest index winning ties.
+ * max_symbols (S): after S consecutive emissions on one frame the S-th token is still
+ * emitted and fed to the decoder, then t advances by one; the count resets whenever t
+ * advances (the safeguard the paper mentions in a footnote of the beam-search section).
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless the parameter comment says "host".
+ *   - All buffers are caller-owned and borrowed for the duration of the call; the
+ *     library allocates no device memory.  Weight matrices are row-major [out, in].
+ *   - dtype WIND_DT_BF16: enc, emb and all weight matrices are bf16 (uint16 bit
+ *     patterns), biases fp32, all accumulation and recurrent state fp32.
+ *     dtype WIND_DT_F32: everything fp32, plain FMA arithmetic (no tf32).
+ *   - Calls enqueue work on `stream`, synchronise that stream once at the end to read the
+ *     device status word, and return it.  Errors detectable on the host return before
+ *     any launch.  Every device-side wait is bounded; a wait that runs out sets
+ *     WIND_ERR_TIMEOUT instead of hanging.
+ *   - Results are deterministic run to run.
+ */
+#ifndef WIND_H_
+#define WIND_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    WIND_OK = 0,
+    WIND_ERR_INVALID_ARG = 1,     /* null pointer, non-positive size, W < 1, blank_id > V, ... */
+    WIND_ERR_UNSUPPORTED = 2,     /* shape outside what the kernels handle (see wind_decode_greedy) */
+    WIND_ERR_CUDA = 3,            /* a CUDA runtime/driver call failed; see wind_last_cuda_error() */
+    WIND_ERR_OUTPUT_OVERFLOW = 4, /* some utterance produced more than max_out tokens */
+    WIND_ERR_TIMEOUT = 5,         /* a bounded device-side wait ran out */
+    WIND_ERR_INTERNAL = 6,        /* step cap exceeded or inconsistent device state */
+    WIND_ERR_WORKSPACE = 7        /* workspace too small or misaligned */
+} wind_status_t;
+
+typedef enum { WIND_ACT_RELU = 0, WIND_ACT_TANH = 1 } wind_act_t;
+typedef enum { WIND_DT_F32 = 0, WIND_DT_BF16 = 1 } wind_dtype_t;
+
+/* Which kernels run the bf16 path.  AUTO picks the tensor-core (tcgen05/TMA) kernels
+ * when the shapes allow (D, E, P, H multiples of 64) and the plain-ALU kernels otherwise. */
+typedef enum { WIND_KERNELS_AUTO = 0, WIND_KERNELS_SIMT = 1, WIND_KERNELS_TENSOR = 2 } wind_kernels_t;
+
+typedef struct {
+    int32_t D, E, P, L, H, V;  /* V labels; logits are V+1 wide; 1 <= L <= 8 */
+    int32_t blank_id;          /* 0..V; also the start-of-sequence decoder input */
+    int32_t act;               /* wind_act_t */
+    int32_t dtype;             /* wind_dtype_t: element type of enc, emb and the weight matrices */
+    int32_t reserved;
+    const void* emb;           /* [V+1, E] */
+    const void* const* w_ih;   /* HOST array of L device pointers: [4P, E] for l = 0, [4P, P] for l > 0 */
+    const void* const* w_hh;   /* HOST array of L device pointers: [4P, P] */
+    const float* const* b_ih;  /* HOST array of L device pointers: [4P] fp32 */
+    const float* const* b_hh;  /* HOST array of L device pointers: [4P] fp32 */
+    const void* w_enc;         /* [H, D] */
+    const float* b_enc;        /* [H] */
+    const void* w_pred;        /* [H, P] */
+    const float* b_pred;       /* [H] */
+    const void* w_out;         /* [V+1, H] */
+    const float* b_out;        /* [V+1] */
+} wind_model_t;
+
+/* Counters of the last decode that used a workspace (read back with wind_read_stats). */
+typedef struct {
+    int64_t steps;         /* lock-step iterations of the decoding loop */
+    int64_t joint_rows;    /* joiner rows evaluated for decisions (sum of n over steps and utterances) */
+    int64_t tokens;        /* tokens emitted (= decoder updates after the start-of-sequence one) */
+    int64_t forced;        /* forced advances by the max_symbols rule */
+    int64_t frames;        /* sum of enc_len */
+    int64_t jump_hist[65]; /* jump sizes 0..min(W,64): i on an emission, n on an all-blank window */
+    int32_t status;        /* device status word (wind_status_t) */
+    int32_t launches_per_step; /* kernel nodes in one loop iteration */
+    int32_t launches_setup;    /* kernel launches outside the loop (projection, init, first decoder update) */
+    int32_t kernels;           /* wind_kernels_t actually used */
+} wind_stats_t;
+
+/*
+ * Bytes of device workspace needed by wind_decode_greedy / wind_eval_joint_window for
+ * batches up to B utterances of up to T frames and window W.  Holds enc_proj [B,T,H],
+ * the decoder state, the per-row argmax keys (8 bytes per window row: the window logits
+ * themselves -- W x (V+1) floats per utterance in the paper's memory analysis -- never
+ * leave the chip) and control words.  Grows with W only by the key array.
+ */
+wind_status_t wind_workspace_bytes(const wind_model_t* m, int32_t B, int32_t T, int32_t W, size_t* bytes);
+
+/*
+ * Batched greedy decoding (Algorithm 2; Algorithm 1 when W == 1).
+ *   enc        [B, T, D] row-major, element type m->dtype.  Frames t >= enc_len[b] are
+ *              never read for a decision (they may hold NaN).
+ *   enc_len    [B] int32, 0 <= enc_len[b] <= T.
+ *   W          window, 1 <= W <= 64.   max_symbols >= 1.
+ *   out_tokens [B, max_out] int32; out_frames [B, max_out] int32 (0-based encoder frame at
+ *              which the token was emitted, non-decreasing, each value at most
+ *              max_symbols times); out_len [B] int32.  Entries beyond out_len[b] are
+ *              left untouched.  max_out = T * max_symbols always suffices; if an utterance
+ *              needs more than max_out it stops there, the others finish, and the call
+ *              returns WIND_ERR_OUTPUT_OVERFLOW.
+ *   workspace  device memory, 256-byte aligned, at least wind_workspace_bytes(m,B,T,W).
+ *              Calls sharing a workspace must not overlap in time.
+ *   stream     cudaStream_t (0 = default stream).
+ * WIND_ERR_UNSUPPORTED: L > 8, W > 64, B*T*H or B*max_out beyond 2^31-1 elements.
+ */
+wind_status_t wind_decode_greedy(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B,
+                                 int32_t T, int32_t W, int32_t max_symbols, int32_t* out_tokens,
+                                 int32_t* out_frames, int32_t* out_len, int32_t max_out, void* workspace,
+                                 size_t workspace_bytes, void* stream);
+
+/*
+ * Extra workspace (added to wind_workspace_bytes) that wind_decode_greedy_host needs for
+ * staging enc, enc_len and the three outputs on the device.
+ */
+wind_status_t wind_host_staging_bytes(const wind_model_t* m, int32_t B, int32_t T, int32_t max_out, size_t* bytes);
+
+/*
+ * Same decode, but enc, enc_len, out_tokens, out_frames and out_len are HOST pointers
+ * (pinned memory gives asynchronous copies).  The call copies enc and enc_len to the
+ * device, decodes, copies the outputs back and synchronises the stream.  The model's
+ * weights stay device pointers.  workspace: device, at least wind_workspace_bytes +
+ * wind_host_staging_bytes.
+ */
+wind_status_t wind_decode_greedy_host(const wind_model_t* m, const void* enc_host, const int32_t* enc_len_host,
+                                      int32_t B, int32_t T, int32_t W, int32_t max_symbols,
+                                      int32_t* out_tokens_host, int32_t* out_frames_host, int32_t* out_len_host,
+                                      int32_t max_out, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Teacher-forced window logits, for parity checks: runs the same projection, decoder and
+ * fused joiner kernels as the decode, with the argmax epilogue replaced by a store.
+ *   prefix [B, U] int32, prefix_len [B] (tokens fed after the start-of-sequence blank;
+ *   U >= max prefix_len), t0 [B] window start (0 <= t0[b] <= enc_len[b]).
+ *   logits [B, W, V+1] fp32; rows w >= min(W, enc_len[b] - t0[b]) are left untouched.
+ */
+wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B,
+                                     int32_t T, int32_t W, const int32_t* prefix, int32_t U,
+                                     const int32_t* prefix_len, const int32_t* t0, float* logits, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+
+/* Per-kernel device times of one decode, from CUDA events recorded on `stream` around
+ * every kernel launch (milliseconds summed over launches, and launch counts). */
+typedef struct {
+    double enc_proj_ms, joint_ms, control_ms, pred_ms;
+    int64_t enc_proj_launches, joint_launches, control_launches, pred_launches;
+} wind_profile_t;
+
+/*
+ * Measurement aid: the same decode as wind_decode_greedy (same kernels, same results), but
+ * the loop is driven from the host in bursts of steps so that every launch can be
+ * bracketed by a pair of CUDA events on `stream`.  Slower than wind_decode_greedy (events
+ * and one synchronisation per burst); use it to attribute time to kernels, not as the
+ * decoding path.  The paper has no counterpart; its timing is wall clock only.
+ */
+wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B,
+                                  int32_t T, int32_t W, int32_t max_symbols, int32_t* out_tokens,
+                                  int32_t* out_frames, int32_t* out_len, int32_t max_out, void* workspace,
+                                  size_t workspace_bytes, void* stream, wind_profile_t* host_out);
+
+/* Copies the counters of the last decode that used `workspace` to host memory (synchronises `stream`). */
+wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t* host_out);
+
+/* Process-wide choice of kernels for the bf16 path (default AUTO).  Returns the previous value. */
+int32_t wind_set_kernels(int32_t kernels);
+
+/* Human-readable name of a status code (static string). */
+const char* wind_status_string(wind_status_t s);
+
+/* Text of the last CUDA error seen by this thread inside the library (static/thread-local string). */
+const char* wind_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WIND_H_ */

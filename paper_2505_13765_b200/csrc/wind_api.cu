@@ -1,0 +1,429 @@
+// C ABI entry points: argument checks, workspace carving, launch sequence, and the
+// device-resident decoding loop (a CUDA-graph WHILE node whose body is two lock steps).
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "wind_internal.cuh"
+
+namespace wind {
+
+static thread_local char g_cuda_err[256] = "";
+static int g_kernels = WIND_KERNELS_AUTO;
+
+static wind_status_t cuda_fail(cudaError_t e, const char* where) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", where, cudaGetErrorString(e));
+    return WIND_ERR_CUDA;
+}
+#define WIND_CUDA(expr)                                              \
+    do {                                                             \
+        cudaError_t e__ = (expr);                                    \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #expr);        \
+    } while (0)
+
+static wind_status_t check_model(const wind_model_t* m) {
+    if (!m) return WIND_ERR_INVALID_ARG;
+    if (m->D < 1 || m->E < 1 || m->P < 1 || m->L < 1 || m->H < 1 || m->V < 1) return WIND_ERR_INVALID_ARG;
+    if (m->blank_id < 0 || m->blank_id > m->V) return WIND_ERR_INVALID_ARG;
+    if (m->act != WIND_ACT_RELU && m->act != WIND_ACT_TANH) return WIND_ERR_INVALID_ARG;
+    if (m->dtype != WIND_DT_F32 && m->dtype != WIND_DT_BF16) return WIND_ERR_INVALID_ARG;
+    if (m->L > kMaxLayers) return WIND_ERR_UNSUPPORTED;
+    return WIND_OK;
+}
+
+static wind_status_t check_shape(const wind_model_t* m, int B, int T, int W) {
+    if (B < 1 || T < 1 || W < 1) return WIND_ERR_INVALID_ARG;
+    if (W > kMaxWindow) return WIND_ERR_UNSUPPORTED;
+    if ((long long)B * T * m->H > 0x7fffffffLL || (long long)B * T * m->D > 0x7fffffffLL) return WIND_ERR_UNSUPPORTED;
+    if ((long long)B * W > 0x7fffffffLL) return WIND_ERR_UNSUPPORTED;
+    return WIND_OK;
+}
+
+static wind_status_t check_weights(const wind_model_t* m) {
+    if (!m->emb || !m->w_ih || !m->w_hh || !m->b_ih || !m->b_hh || !m->w_enc || !m->b_enc || !m->w_pred || !m->b_pred ||
+        !m->w_out || !m->b_out)
+        return WIND_ERR_INVALID_ARG;
+    for (int l = 0; l < m->L; ++l)
+        if (!m->w_ih[l] || !m->w_hh[l] || !m->b_ih[l] || !m->b_hh[l]) return WIND_ERR_INVALID_ARG;
+    return WIND_OK;
+}
+
+static void fill_call(Call& c, const wind_model_t* m, const void* enc, const int32_t* enc_len, int B, int T, int W, int S,
+                      int32_t* out_tokens, int32_t* out_frames, int32_t* out_len, int max_out, void* ws, cudaStream_t stream) {
+    memset(&c, 0, sizeof(c));
+    c.m = *m;
+    for (int l = 0; l < m->L; ++l) {
+        c.w_ih[l] = m->w_ih[l];
+        c.w_hh[l] = m->w_hh[l];
+        c.b_ih[l] = m->b_ih[l];
+        c.b_hh[l] = m->b_hh[l];
+    }
+    c.m.w_ih = nullptr; c.m.w_hh = nullptr; c.m.b_ih = nullptr; c.m.b_hh = nullptr;  // host arrays: not part of the key
+    c.m.reserved = 0;
+    c.enc = enc; c.enc_len = enc_len;
+    c.B = B; c.T = T; c.W = W; c.S = S; c.max_out = max_out;
+    c.out_tokens = out_tokens; c.out_frames = out_frames; c.out_len = out_len;
+    c.ws = static_cast<uint8_t*>(ws);
+    c.lay = make_layout(*m, B, T, W, max_out);
+    c.stream = stream;
+}
+
+static bool use_tensor(const Call& c) {
+    if (c.m.dtype != WIND_DT_BF16) return false;
+    if (g_kernels == WIND_KERNELS_SIMT) return false;
+    return tc_supported(c.m, c.B, c.T, c.W);
+}
+
+// ---------------------------------------------------------------------------
+// Decoding loop as a CUDA graph: WHILE(active > 0) { step(parity 1->0); step(parity 0->1) }.
+// A lock step is joint -> control -> decoder update; kernels of a step that starts with
+// active == 0 return at once, so the second step of the last iteration is a no-op.
+// Kernel arguments are baked into the graph, hence the cache keyed by the whole call.
+// ---------------------------------------------------------------------------
+struct LoopGraph {
+    Call key;
+    int tensor;
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    unsigned long long last_use = 0;
+};
+static std::mutex g_mutex;
+static std::vector<LoopGraph> g_graphs;
+static unsigned long long g_use_counter = 0;
+static cudaStream_t g_capture_stream = nullptr;
+constexpr size_t kMaxGraphs = 12;
+
+static cudaError_t enqueue_step(const Call& c, bool tensor, int parity_in, cudaGraphConditionalHandle handle, int use_handle) {
+    cudaError_t e;
+    e = tensor ? tc_joint(c, nullptr) : simt_joint(c, nullptr);
+    if (e != cudaSuccess) return e;
+    e = launch_control(c, handle, use_handle);
+    if (e != cudaSuccess) return e;
+    return tensor ? tc_pred_step(c, parity_in) : simt_pred_step(c, parity_in);
+}
+
+static bool same_key(const Call& a, const Call& b) {
+    Call x = a, y = b;
+    x.stream = nullptr; y.stream = nullptr;
+    return memcmp(&x, &y, sizeof(Call)) == 0;
+}
+
+static wind_status_t get_loop_graph(const Call& c, bool tensor, cudaGraphExec_t* exec_out) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    for (auto& g : g_graphs)
+        if (g.tensor == (int)tensor && same_key(g.key, c)) {
+            g.last_use = ++g_use_counter;
+            *exec_out = g.exec;
+            return WIND_OK;
+        }
+    if (!g_capture_stream) WIND_CUDA(cudaStreamCreateWithFlags(&g_capture_stream, cudaStreamNonBlocking));
+    LoopGraph g;
+    g.key = c;
+    g.tensor = tensor;
+    WIND_CUDA(cudaGraphCreate(&g.graph, 0));
+    cudaGraphConditionalHandle handle;
+    WIND_CUDA(cudaGraphConditionalHandleCreate(&handle, g.graph, 1, cudaGraphCondAssignDefault));
+    cudaGraphNodeParams np = {cudaGraphNodeTypeConditional};
+    np.conditional.handle = handle;
+    np.conditional.type = cudaGraphCondTypeWhile;
+    np.conditional.size = 1;
+    cudaGraphNode_t node;
+    WIND_CUDA(cudaGraphAddNode(&node, g.graph, nullptr, 0, &np));
+    cudaGraph_t body = np.conditional.phGraph_out[0];
+    Call cc = c;
+    cc.stream = g_capture_stream;
+    WIND_CUDA(cudaStreamBeginCaptureToGraph(g_capture_stream, body, nullptr, nullptr, 0, cudaStreamCaptureModeRelaxed));
+    cudaError_t e1 = enqueue_step(cc, tensor, 1, handle, 1);
+    cudaError_t e2 = e1 == cudaSuccess ? enqueue_step(cc, tensor, 0, handle, 1) : e1;
+    cudaGraph_t ended = nullptr;
+    cudaError_t e3 = cudaStreamEndCapture(g_capture_stream, &ended);
+    if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) {
+        cudaGraphDestroy(g.graph);
+        return cuda_fail(e1 != cudaSuccess ? e1 : (e2 != cudaSuccess ? e2 : e3), "capture of the decoding loop");
+    }
+    cudaError_t e4 = cudaGraphInstantiate(&g.exec, g.graph, 0);
+    if (e4 != cudaSuccess) {
+        cudaGraphDestroy(g.graph);
+        return cuda_fail(e4, "cudaGraphInstantiate");
+    }
+    if (g_graphs.size() >= kMaxGraphs) {
+        size_t victim = 0;
+        for (size_t i = 1; i < g_graphs.size(); ++i)
+            if (g_graphs[i].last_use < g_graphs[victim].last_use) victim = i;
+        cudaGraphExecDestroy(g_graphs[victim].exec);
+        cudaGraphDestroy(g_graphs[victim].graph);
+        g_graphs.erase(g_graphs.begin() + victim);
+    }
+    g.last_use = ++g_use_counter;
+    g_graphs.push_back(g);
+    *exec_out = g.exec;
+    return WIND_OK;
+}
+
+// Enqueue the whole decode on c.stream (no synchronisation).
+static wind_status_t enqueue_decode(const Call& c) {
+    const bool tensor = use_tensor(c);
+    if (c.m.dtype == WIND_DT_BF16 && g_kernels == WIND_KERNELS_TENSOR && !tensor) return WIND_ERR_UNSUPPORTED;
+    const int per_step = 2 + (tensor ? tc_pred_launches(c) : simt_pred_launches(c));
+    const int setup = 2 + (tensor ? tc_pred_launches(c) : simt_pred_launches(c));
+    if (tensor) WIND_CUDA(tc_prepare(c));
+    WIND_CUDA(launch_init(c, tensor ? WIND_KERNELS_TENSOR : WIND_KERNELS_SIMT, per_step, setup));
+    WIND_CUDA(tensor ? tc_enc_proj(c) : simt_enc_proj(c));
+    WIND_CUDA(tensor ? tc_pred_step(c, 0) : simt_pred_step(c, 0));  // start of sequence: h[0] (zeros) -> h[1]
+    const char* mode = getenv("WIND_LOOP");
+    if (mode && strcmp(mode, "host") == 0) {
+        // bring-up aid: fixed-size bursts of steps, the host polls the active count between bursts
+        cudaGraphConditionalHandle none{};
+        for (;;) {
+            for (int k = 0; k < 8; ++k) {
+                WIND_CUDA(enqueue_step(c, tensor, 1, none, 0));
+                WIND_CUDA(enqueue_step(c, tensor, 0, none, 0));
+            }
+            Ctrl hc;
+            WIND_CUDA(cudaMemcpyAsync(&hc, c.ctrl(), sizeof(Ctrl), cudaMemcpyDeviceToHost, c.stream));
+            WIND_CUDA(cudaStreamSynchronize(c.stream));
+            if (hc.active == 0) break;
+        }
+        return WIND_OK;
+    }
+    cudaGraphExec_t exec = nullptr;
+    wind_status_t s = get_loop_graph(c, tensor, &exec);
+    if (s != WIND_OK) return s;
+    WIND_CUDA(cudaGraphLaunch(exec, c.stream));
+    return WIND_OK;
+}
+
+static wind_status_t read_status(const Call& c) {
+    int32_t st = 0;
+    WIND_CUDA(cudaMemcpyAsync(&st, &c.ctrl()->status, sizeof(int32_t), cudaMemcpyDeviceToHost, c.stream));
+    WIND_CUDA(cudaStreamSynchronize(c.stream));
+    return (wind_status_t)st;
+}
+
+static wind_status_t check_decode_args(const wind_model_t* m, const void* enc, const int32_t* enc_len, int B, int T, int W,
+                                       int S, const int32_t* ot, const int32_t* of, const int32_t* ol, int max_out,
+                                       const void* ws) {
+    wind_status_t s = check_model(m);
+    if (s != WIND_OK) return s;
+    s = check_weights(m);
+    if (s != WIND_OK) return s;
+    s = check_shape(m, B, T, W);
+    if (s != WIND_OK) return s;
+    if (!enc || !enc_len || !ot || !of || !ol || !ws) return WIND_ERR_INVALID_ARG;
+    if (S < 1 || max_out < 1) return WIND_ERR_INVALID_ARG;
+    if ((long long)B * max_out > 0x7fffffffLL) return WIND_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(ws) % kAlign) return WIND_ERR_WORKSPACE;
+    return WIND_OK;
+}
+
+}  // namespace wind
+
+using namespace wind;
+
+extern "C" {
+
+wind_status_t wind_workspace_bytes(const wind_model_t* m, int32_t B, int32_t T, int32_t W, size_t* bytes) {
+    wind_status_t s = check_model(m);
+    if (s != WIND_OK) return s;
+    s = check_shape(m, B, T, W);
+    if (s != WIND_OK) return s;
+    if (!bytes) return WIND_ERR_INVALID_ARG;
+    *bytes = make_layout(*m, B, T, W, 1).total;
+    return WIND_OK;
+}
+
+wind_status_t wind_host_staging_bytes(const wind_model_t* m, int32_t B, int32_t T, int32_t max_out, size_t* bytes) {
+    wind_status_t s = check_model(m);
+    if (s != WIND_OK) return s;
+    s = check_shape(m, B, T, 1);
+    if (s != WIND_OK) return s;
+    if (!bytes || max_out < 1) return WIND_ERR_INVALID_ARG;
+    *bytes = make_layout(*m, B, T, 1, max_out).st_total;
+    return WIND_OK;
+}
+
+wind_status_t wind_decode_greedy(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B, int32_t T,
+                                 int32_t W, int32_t max_symbols, int32_t* out_tokens, int32_t* out_frames, int32_t* out_len,
+                                 int32_t max_out, void* workspace, size_t workspace_bytes, void* stream) {
+    wind_status_t s = check_decode_args(m, enc, enc_len, B, T, W, max_symbols, out_tokens, out_frames, out_len, max_out, workspace);
+    if (s != WIND_OK) return s;
+    Call c;
+    fill_call(c, m, enc, enc_len, B, T, W, max_symbols, out_tokens, out_frames, out_len, max_out, workspace, (cudaStream_t)stream);
+    if (workspace_bytes < c.lay.total) return WIND_ERR_WORKSPACE;
+    s = enqueue_decode(c);
+    if (s != WIND_OK) return s;
+    return read_status(c);
+}
+
+wind_status_t wind_decode_greedy_host(const wind_model_t* m, const void* enc_host, const int32_t* enc_len_host, int32_t B,
+                                      int32_t T, int32_t W, int32_t max_symbols, int32_t* out_tokens_host,
+                                      int32_t* out_frames_host, int32_t* out_len_host, int32_t max_out, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+    wind_status_t s = check_decode_args(m, enc_host, enc_len_host, B, T, W, max_symbols, out_tokens_host, out_frames_host,
+                                        out_len_host, max_out, workspace);
+    if (s != WIND_OK) return s;
+    Layout lay = make_layout(*m, B, T, W, max_out);
+    if (workspace_bytes < lay.total + lay.st_total) return WIND_ERR_WORKSPACE;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t es = m->dtype == WIND_DT_BF16 ? 2 : 4;
+    void* d_enc = ws + lay.st_enc;
+    int32_t* d_len = reinterpret_cast<int32_t*>(ws + lay.st_len);
+    int32_t* d_tok = reinterpret_cast<int32_t*>(ws + lay.st_tok);
+    int32_t* d_frm = reinterpret_cast<int32_t*>(ws + lay.st_frm);
+    int32_t* d_olen = reinterpret_cast<int32_t*>(ws + lay.st_olen);
+    WIND_CUDA(cudaMemcpyAsync(d_enc, enc_host, es * (size_t)B * T * m->D, cudaMemcpyHostToDevice, st));
+    WIND_CUDA(cudaMemcpyAsync(d_len, enc_len_host, sizeof(int32_t) * B, cudaMemcpyHostToDevice, st));
+    Call c;
+    fill_call(c, m, d_enc, d_len, B, T, W, max_symbols, d_tok, d_frm, d_olen, max_out, workspace, st);
+    s = enqueue_decode(c);
+    if (s != WIND_OK) return s;
+    WIND_CUDA(cudaMemcpyAsync(out_tokens_host, d_tok, sizeof(int32_t) * (size_t)B * max_out, cudaMemcpyDeviceToHost, st));
+    WIND_CUDA(cudaMemcpyAsync(out_frames_host, d_frm, sizeof(int32_t) * (size_t)B * max_out, cudaMemcpyDeviceToHost, st));
+    WIND_CUDA(cudaMemcpyAsync(out_len_host, d_olen, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, st));
+    return read_status(c);
+}
+
+wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B, int32_t T,
+                                     int32_t W, const int32_t* prefix, int32_t U, const int32_t* prefix_len, const int32_t* t0,
+                                     float* logits, void* workspace, size_t workspace_bytes, void* stream) {
+    wind_status_t s = check_model(m);
+    if (s != WIND_OK) return s;
+    s = check_weights(m);
+    if (s != WIND_OK) return s;
+    s = check_shape(m, B, T, W);
+    if (s != WIND_OK) return s;
+    if (!enc || !enc_len || !prefix_len || !t0 || !logits || !workspace || U < 0 || (U > 0 && !prefix)) return WIND_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return WIND_ERR_WORKSPACE;
+    Call c;
+    // the control arrays double as scratch outputs here: out_len is reset by the init kernel
+    fill_call(c, m, enc, enc_len, B, T, W, 1, nullptr, nullptr, nullptr, 1, workspace, (cudaStream_t)stream);
+    if (workspace_bytes < c.lay.total) return WIND_ERR_WORKSPACE;
+    c.out_len = c.count();  // any int32 [B] scratch: init writes zeros to it
+    const bool tensor = use_tensor(c);
+    if (c.m.dtype == WIND_DT_BF16 && g_kernels == WIND_KERNELS_TENSOR && !tensor) return WIND_ERR_UNSUPPORTED;
+    if (tensor) WIND_CUDA(tc_prepare(c));
+    WIND_CUDA(launch_init(c, tensor ? WIND_KERNELS_TENSOR : WIND_KERNELS_SIMT, 0, 0));
+    WIND_CUDA(tensor ? tc_enc_proj(c) : simt_enc_proj(c));
+    WIND_CUDA(launch_set_t(c, t0));  // also sets active = B, so the decoder updates run even if every length is 0
+    int parity = 0;
+    WIND_CUDA(tensor ? tc_pred_step(c, parity) : simt_pred_step(c, parity));  // start of sequence
+    parity ^= 1;
+    for (int u = 0; u < U; ++u) {
+        WIND_CUDA(launch_force_tokens(c, prefix, U, prefix_len, u));
+        WIND_CUDA(tensor ? tc_pred_step(c, parity) : simt_pred_step(c, parity));
+        parity ^= 1;
+    }
+    WIND_CUDA(launch_set_t(c, t0));
+    WIND_CUDA(tensor ? tc_joint(c, logits) : simt_joint(c, logits));
+    return read_status(c);
+}
+
+wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B, int32_t T,
+                                  int32_t W, int32_t max_symbols, int32_t* out_tokens, int32_t* out_frames, int32_t* out_len,
+                                  int32_t max_out, void* workspace, size_t workspace_bytes, void* stream,
+                                  wind_profile_t* host_out) {
+    wind_status_t s = check_decode_args(m, enc, enc_len, B, T, W, max_symbols, out_tokens, out_frames, out_len, max_out, workspace);
+    if (s != WIND_OK) return s;
+    if (!host_out) return WIND_ERR_INVALID_ARG;
+    Call c;
+    fill_call(c, m, enc, enc_len, B, T, W, max_symbols, out_tokens, out_frames, out_len, max_out, workspace, (cudaStream_t)stream);
+    if (workspace_bytes < c.lay.total) return WIND_ERR_WORKSPACE;
+    const bool tensor = use_tensor(c);
+    if (c.m.dtype == WIND_DT_BF16 && g_kernels == WIND_KERNELS_TENSOR && !tensor) return WIND_ERR_UNSUPPORTED;
+    memset(host_out, 0, sizeof(*host_out));
+    constexpr int kBurst = 32;              // steps per burst
+    constexpr int kEvents = 3 * kBurst + 1; // joint | control | pred boundaries
+    std::vector<cudaEvent_t> ev(kEvents);
+    for (auto& e : ev) WIND_CUDA(cudaEventCreate(&e));
+    auto destroy = [&]() { for (auto& e : ev) cudaEventDestroy(e); };
+    const int pred_l = tensor ? tc_pred_launches(c) : simt_pred_launches(c);
+    if (tensor) WIND_CUDA(tc_prepare(c));
+    WIND_CUDA(launch_init(c, tensor ? WIND_KERNELS_TENSOR : WIND_KERNELS_SIMT, 2 + pred_l, 2 + pred_l));
+    WIND_CUDA(cudaEventRecord(ev[0], c.stream));
+    WIND_CUDA(tensor ? tc_enc_proj(c) : simt_enc_proj(c));
+    WIND_CUDA(cudaEventRecord(ev[1], c.stream));
+    WIND_CUDA(tensor ? tc_pred_step(c, 0) : simt_pred_step(c, 0));
+    WIND_CUDA(cudaEventRecord(ev[2], c.stream));
+    WIND_CUDA(cudaStreamSynchronize(c.stream));
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, ev[0], ev[1]); host_out->enc_proj_ms += ms; host_out->enc_proj_launches += 1;
+    cudaEventElapsedTime(&ms, ev[1], ev[2]); host_out->pred_ms += ms; host_out->pred_launches += pred_l;
+    cudaGraphConditionalHandle none{};
+    int parity = 1;
+    for (;;) {
+        Ctrl before;
+        WIND_CUDA(cudaMemcpyAsync(&before, c.ctrl(), sizeof(Ctrl), cudaMemcpyDeviceToHost, c.stream));
+        WIND_CUDA(cudaStreamSynchronize(c.stream));
+        if (before.active == 0) break;
+        WIND_CUDA(cudaEventRecord(ev[0], c.stream));
+        for (int k = 0; k < kBurst; ++k) {
+            WIND_CUDA(tensor ? tc_joint(c, nullptr) : simt_joint(c, nullptr));
+            WIND_CUDA(cudaEventRecord(ev[3 * k + 1], c.stream));
+            WIND_CUDA(launch_control(c, none, 0));
+            WIND_CUDA(cudaEventRecord(ev[3 * k + 2], c.stream));
+            WIND_CUDA(tensor ? tc_pred_step(c, parity) : simt_pred_step(c, parity));
+            WIND_CUDA(cudaEventRecord(ev[3 * k + 3], c.stream));
+            parity ^= 1;
+        }
+        Ctrl after;
+        WIND_CUDA(cudaMemcpyAsync(&after, c.ctrl(), sizeof(Ctrl), cudaMemcpyDeviceToHost, c.stream));
+        WIND_CUDA(cudaStreamSynchronize(c.stream));
+        const int live = after.step - before.step;  // steps of this burst that did real work
+        for (int k = 0; k < live && k < kBurst; ++k) {
+            cudaEventElapsedTime(&ms, ev[3 * k], ev[3 * k + 1]); host_out->joint_ms += ms;
+            cudaEventElapsedTime(&ms, ev[3 * k + 1], ev[3 * k + 2]); host_out->control_ms += ms;
+            cudaEventElapsedTime(&ms, ev[3 * k + 2], ev[3 * k + 3]); host_out->pred_ms += ms;
+        }
+        host_out->joint_launches += live;
+        host_out->control_launches += live;
+        host_out->pred_launches += (int64_t)live * pred_l;
+    }
+    destroy();
+    return read_status(c);
+}
+
+wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t* host_out) {
+    if (!workspace || !host_out) return WIND_ERR_INVALID_ARG;
+    Ctrl hc;
+    WIND_CUDA(cudaMemcpyAsync(&hc, workspace, sizeof(Ctrl), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    WIND_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    memset(host_out, 0, sizeof(*host_out));
+    host_out->steps = hc.step;
+    host_out->joint_rows = hc.joint_rows;
+    host_out->tokens = hc.tokens;
+    host_out->forced = hc.forced;
+    host_out->frames = hc.frames;
+    for (int k = 0; k < 65; ++k) host_out->jump_hist[k] = hc.jump_hist[k];
+    host_out->status = hc.status;
+    host_out->launches_per_step = hc.launches_per_step;
+    host_out->launches_setup = hc.launches_setup;
+    host_out->kernels = hc.kernels;
+    return WIND_OK;
+}
+
+int32_t wind_set_kernels(int32_t kernels) {
+    int32_t prev = g_kernels;
+    if (kernels >= WIND_KERNELS_AUTO && kernels <= WIND_KERNELS_TENSOR) g_kernels = kernels;
+    return prev;
+}
+
+const char* wind_status_string(wind_status_t s) {
+    switch (s) {
+        case WIND_OK: return "WIND_OK";
+        case WIND_ERR_INVALID_ARG: return "WIND_ERR_INVALID_ARG";
+        case WIND_ERR_UNSUPPORTED: return "WIND_ERR_UNSUPPORTED";
+        case WIND_ERR_CUDA: return "WIND_ERR_CUDA";
+        case WIND_ERR_OUTPUT_OVERFLOW: return "WIND_ERR_OUTPUT_OVERFLOW";
+        case WIND_ERR_TIMEOUT: return "WIND_ERR_TIMEOUT";
+        case WIND_ERR_INTERNAL: return "WIND_ERR_INTERNAL";
+        case WIND_ERR_WORKSPACE: return "WIND_ERR_WORKSPACE";
+    }
+    return "WIND_ERR_UNKNOWN";
+}
+
+const char* wind_last_cuda_error(void) { return g_cuda_err; }
+
+}  // extern "C"

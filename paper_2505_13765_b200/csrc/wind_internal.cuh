@@ -1,0 +1,162 @@
+// Internal declarations shared by the translation units of the library:
+// workspace layout, device control block, argmax key packing, launch prototypes.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "wind.h"
+
+namespace wind {
+
+constexpr int kMaxLayers = 8;
+constexpr int kMaxWindow = 64;
+constexpr size_t kAlign = 256;
+
+// Device control block, first thing in the workspace.
+struct Ctrl {
+    int32_t status;   // wind_status_t, sticky (first error wins)
+    int32_t active;   // utterances with t < len after the last control update
+    int32_t step;     // loop iterations executed
+    int32_t step_cap; // hard bound on step
+    int64_t joint_rows;
+    int64_t tokens;
+    int64_t forced;
+    int64_t frames;
+    int64_t jump_hist[65];
+    int32_t launches_per_step;
+    int32_t launches_setup;
+    int32_t kernels;
+    int32_t pad;
+};
+
+// Byte offsets of every workspace region (all multiples of kAlign).
+struct Layout {
+    size_t ctrl;       // Ctrl
+    size_t t;          // int32 [B]   current frame per utterance
+    size_t count;      // int32 [B]   consecutive emissions on the current frame
+    size_t emit_tok;   // int32 [B]   token to feed to the decoder this step, -1 = none
+    size_t keys;       // uint64 [B*W] packed (logit, label) argmax keys, 0 = empty
+    size_t h;          // fp32 [2][L][B][P]  LSTM hidden state, ping-pong by step parity
+    size_t c;          // fp32 [L][B][P]     LSTM cell state
+    size_t pred_proj;  // fp32 [B][H]
+    size_t xh;         // bf16 [2][L][Bpad][in_l + P] decoder GEMM operand rows (tensor path)
+    size_t enc_proj;   // elem [B*T][H]
+    size_t total;
+    // host staging (wind_decode_greedy_host), placed after `total`
+    size_t st_enc, st_len, st_tok, st_frm, st_olen, st_total;
+    int32_t Bpad;      // B rounded up to 16 (tensor path operand rows)
+    int32_t xh_stride[kMaxLayers];  // elements per row of layer l's operand = in_l + P
+    size_t xh_layer_off[kMaxLayers]; // byte offset of layer l inside one parity's block
+    size_t xh_parity_bytes;
+};
+
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_out) {
+    Layout L{};
+    const size_t es = (m.dtype == WIND_DT_BF16) ? 2 : 4;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    L.ctrl = take(sizeof(Ctrl));
+    L.t = take(sizeof(int32_t) * B);
+    L.count = take(sizeof(int32_t) * B);
+    L.emit_tok = take(sizeof(int32_t) * B);
+    L.keys = take(sizeof(uint64_t) * (size_t)B * W);
+    L.h = take(sizeof(float) * 2 * (size_t)m.L * B * m.P);
+    L.c = take(sizeof(float) * (size_t)m.L * B * m.P);
+    L.pred_proj = take(sizeof(float) * (size_t)B * m.H);
+    L.Bpad = (B + 15) / 16 * 16;
+    size_t xb = 0;
+    for (int l = 0; l < m.L; ++l) {
+        L.xh_stride[l] = (l == 0 ? m.E : m.P) + m.P;
+        L.xh_layer_off[l] = xb;
+        xb = align_up(xb + (size_t)L.Bpad * L.xh_stride[l] * 2);
+    }
+    L.xh_parity_bytes = xb;
+    L.xh = take(2 * xb);
+    L.enc_proj = take(es * (size_t)B * T * m.H);
+    L.total = off;
+    L.st_enc = take(es * (size_t)B * T * m.D);
+    L.st_len = take(sizeof(int32_t) * B);
+    L.st_tok = take(sizeof(int32_t) * (size_t)B * (max_out > 0 ? max_out : 1));
+    L.st_frm = take(sizeof(int32_t) * (size_t)B * (max_out > 0 ? max_out : 1));
+    L.st_olen = take(sizeof(int32_t) * B);
+    L.st_total = off - L.total;
+    return L;
+}
+
+// Everything a kernel launcher needs for one call (host-side bundle, passed by value).
+struct Call {
+    wind_model_t m;
+    const void* w_ih[kMaxLayers];
+    const void* w_hh[kMaxLayers];
+    const float* b_ih[kMaxLayers];
+    const float* b_hh[kMaxLayers];
+    const void* enc;
+    const int32_t* enc_len;
+    int32_t B, T, W, S, max_out;
+    int32_t* out_tokens;
+    int32_t* out_frames;
+    int32_t* out_len;
+    uint8_t* ws;
+    Layout lay;
+    cudaStream_t stream;
+
+    Ctrl* ctrl() const { return reinterpret_cast<Ctrl*>(ws + lay.ctrl); }
+    int32_t* t() const { return reinterpret_cast<int32_t*>(ws + lay.t); }
+    int32_t* count() const { return reinterpret_cast<int32_t*>(ws + lay.count); }
+    int32_t* emit_tok() const { return reinterpret_cast<int32_t*>(ws + lay.emit_tok); }
+    unsigned long long* keys() const { return reinterpret_cast<unsigned long long*>(ws + lay.keys); }
+    float* h(int parity) const {
+        return reinterpret_cast<float*>(ws + lay.h) + (size_t)parity * m.L * B * m.P;
+    }
+    float* c() const { return reinterpret_cast<float*>(ws + lay.c); }
+    float* pred_proj() const { return reinterpret_cast<float*>(ws + lay.pred_proj); }
+    void* enc_proj() const { return ws + lay.enc_proj; }
+    __nv_bfloat16* xh(int parity, int l) const {
+        return reinterpret_cast<__nv_bfloat16*>(ws + lay.xh + (size_t)parity * lay.xh_parity_bytes + lay.xh_layer_off[l]);
+    }
+};
+
+// ---------------------------------------------------------------------------
+// argmax key: (orderable fp32 logit) << 32 | (0xFFFFFFFF - label); max key = max logit,
+// lowest label on equal logits.  0 is "empty".
+// ---------------------------------------------------------------------------
+__host__ __device__ inline uint32_t orderable_f32(uint32_t bits) {
+    return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+}
+__device__ inline unsigned long long pack_key(float logit, uint32_t label) {
+    return ((unsigned long long)orderable_f32(__float_as_uint(logit)) << 32) | (unsigned long long)(0xFFFFFFFFu - label);
+}
+__host__ __device__ inline uint32_t key_label(unsigned long long key) {
+    return 0xFFFFFFFFu - (uint32_t)(key & 0xFFFFFFFFull);
+}
+
+__device__ inline void set_status(Ctrl* ctrl, int32_t s) { atomicCAS(&ctrl->status, 0, s); }
+
+// ---------------------------------------------------------------------------
+// launchers (each enqueues on call.stream; returns cudaGetLastError())
+// ---------------------------------------------------------------------------
+// plain-ALU kernels (fp32 path, and bf16 path when the tensor kernels do not apply)
+cudaError_t simt_enc_proj(const Call& c);
+cudaError_t simt_pred_step(const Call& c, int parity_in);            // all layers + pred_proj
+cudaError_t simt_joint(const Call& c, float* logits_out /*nullable*/);
+int simt_pred_launches(const Call& c);
+
+// control
+cudaError_t launch_init(const Call& c, int kernels_used, int launches_per_step, int launches_setup);
+cudaError_t launch_control(const Call& c, cudaGraphConditionalHandle handle, int use_handle);
+cudaError_t launch_force_tokens(const Call& c, const int32_t* prefix, int U, const int32_t* prefix_len, int u);
+cudaError_t launch_set_t(const Call& c, const int32_t* t0);
+
+// tensor-core kernels (bf16 path)
+bool tc_supported(const wind_model_t& m, int B, int T, int W);
+cudaError_t tc_prepare(const Call& c);   // builds tensor maps for this call (host only)
+cudaError_t tc_enc_proj(const Call& c);
+cudaError_t tc_pred_step(const Call& c, int parity_in);
+cudaError_t tc_joint(const Call& c, float* logits_out);
+int tc_pred_launches(const Call& c);
+
+}  // namespace wind

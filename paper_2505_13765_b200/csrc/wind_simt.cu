@@ -1,0 +1,292 @@
+// Plain-ALU (FFMA) kernels: the fp32 path, and the bf16 path for shapes the tensor-core
+// kernels do not take.  On the bf16 path the operands are rounded where the tensor path
+// rounds them (enc_proj, the joint's activation output and the LSTM's h input go through
+// bf16), so both kernel sets compute the same quantities.
+#include "wind_internal.cuh"
+
+namespace wind {
+
+template <typename T> __device__ __forceinline__ float ldf(const T* p);
+template <> __device__ __forceinline__ float ldf<float>(const float* p) { return *p; }
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+template <typename T> __device__ __forceinline__ float round_like(float x);
+template <> __device__ __forceinline__ float round_like<float>(float x) { return x; }
+template <> __device__ __forceinline__ float round_like<__nv_bfloat16>(float x) {
+    return __bfloat162float(__float2bfloat16_rn(x));
+}
+template <typename T> __device__ __forceinline__ void stf(T* p, float x);
+template <> __device__ __forceinline__ void stf<float>(float* p, float x) { *p = x; }
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ---------------------------------------------------------------------------
+// enc_proj[r, :] = enc[r, :] . W_enc^T + b_enc for valid rows r = b*T + t, t < len[b]
+// 64x64 output tile, 16x16 threads, 4x4 outputs each, K tiles of 16.
+// ---------------------------------------------------------------------------
+template <typename TW>
+__global__ void __launch_bounds__(256) enc_proj_simt_kernel(const TW* __restrict__ enc, const int32_t* __restrict__ enc_len,
+                                                            const TW* __restrict__ w_enc, const float* __restrict__ b_enc,
+                                                            TW* __restrict__ enc_proj, int B, int T, int D, int H) {
+    __shared__ float As[16][65];
+    __shared__ float Bs[16][65];
+    const long long rows = (long long)B * T;
+    const long long r0 = (long long)blockIdx.x * 64;
+    const int h0 = blockIdx.y * 64;
+    // skip tiles without a valid row
+    {
+        long long rl = r0 + 63 < rows ? r0 + 63 : rows - 1;
+        int b0 = (int)(r0 / T), b1 = (int)(rl / T);
+        bool any = false;
+        for (int b = b0; b <= b1; ++b) {
+            long long first = (long long)b * T > r0 ? (long long)b * T : r0;
+            if (first <= rl && first - (long long)b * T < enc_len[b]) any = true;
+        }
+        if (!any) return;
+    }
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int k0 = 0; k0 < D; k0 += 16) {
+        for (int e = threadIdx.x; e < 64 * 16; e += 256) {
+            int rr = e >> 4, kk = e & 15;
+            long long r = r0 + rr;
+            float v = 0.f;
+            if (r < rows && k0 + kk < D) {
+                int b = (int)(r / T);
+                int t = (int)(r - (long long)b * T);
+                if (t < enc_len[b]) v = ldf(enc + r * D + k0 + kk);
+            }
+            As[kk][rr] = v;
+            int hh = h0 + rr;
+            Bs[kk][rr] = (hh < H && k0 + kk < D) ? ldf(w_enc + (size_t)hh * D + k0 + kk) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        long long r = r0 + ty * 4 + i;
+        if (r >= rows) continue;
+        int b = (int)(r / T);
+        int t = (int)(r - (long long)b * T);
+        if (t >= enc_len[b]) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int hh = h0 + tx * 4 + j;
+            if (hh < H) stf(enc_proj + r * H + hh, acc[i][j] + b_enc[hh]);
+        }
+    }
+}
+
+cudaError_t simt_enc_proj(const Call& c) {
+    long long rows = (long long)c.B * c.T;
+    dim3 grid((unsigned)((rows + 63) / 64), (unsigned)((c.m.H + 63) / 64));
+    if (rows == 0) return cudaSuccess;
+    if (c.m.dtype == WIND_DT_BF16)
+        enc_proj_simt_kernel<__nv_bfloat16><<<grid, 256, 0, c.stream>>>(
+            (const __nv_bfloat16*)c.enc, c.enc_len, (const __nv_bfloat16*)c.m.w_enc, c.m.b_enc,
+            (__nv_bfloat16*)c.enc_proj(), c.B, c.T, c.m.D, c.m.H);
+    else
+        enc_proj_simt_kernel<float><<<grid, 256, 0, c.stream>>>((const float*)c.enc, c.enc_len, (const float*)c.m.w_enc,
+                                                                  c.m.b_enc, (float*)c.enc_proj(), c.B, c.T, c.m.D, c.m.H);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// One LSTM layer for all utterances; block j owns hidden unit j (its 4 gate rows).
+// x = emb[emit_tok[b]] (layer 0) or the new h of the layer below; utterances with
+// emit_tok[b] < 0 keep their state (h copied to the other parity buffer).
+// ---------------------------------------------------------------------------
+template <typename TW>
+__global__ void __launch_bounds__(128) lstm_layer_simt_kernel(const Ctrl* __restrict__ ctrl, const int32_t* __restrict__ emit_tok,
+                                                              const TW* __restrict__ emb, const float* __restrict__ x_below,
+                                                              const TW* __restrict__ w_ih, const TW* __restrict__ w_hh,
+                                                              const float* __restrict__ b_ih, const float* __restrict__ b_hh,
+                                                              const float* __restrict__ h_in, float* __restrict__ h_out,
+                                                              float* __restrict__ c_state, int B, int n_in, int P) {
+    if (ctrl->active == 0) return;
+    extern __shared__ float sm[];  // 4 rows x (n_in + P)
+    const int j = blockIdx.x;
+    const int K = n_in + P;
+    for (int e = threadIdx.x; e < 4 * K; e += blockDim.x) {
+        int g = e / K, k = e - g * K;
+        size_t row = (size_t)g * P + j;
+        sm[e] = (k < n_in) ? ldf(w_ih + row * n_in + k) : ldf(w_hh + row * P + (k - n_in));
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    float bias[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) bias[g] = b_ih[g * P + j] + b_hh[g * P + j];
+    for (int b = warp; b < B; b += nw) {
+        const int tok = emit_tok[b];
+        const float* hb = h_in + (size_t)b * P;
+        if (tok < 0) {
+            if (lane == 0) h_out[(size_t)b * P + j] = hb[j];
+            continue;
+        }
+        float a[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int k = lane; k < K; k += 32) {
+            float x;
+            if (k < n_in)
+                x = x_below ? round_like<TW>(x_below[(size_t)b * P + k]) : ldf(emb + (size_t)tok * n_in + k);
+            else
+                x = round_like<TW>(hb[k - n_in]);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) a[g] = fmaf(sm[g * K + k], x, a[g]);
+        }
+#pragma unroll
+        for (int g = 0; g < 4; ++g) a[g] = warp_sum(a[g]);
+        if (lane == 0) {
+            float gi = 1.f / (1.f + expf(-(a[0] + bias[0])));
+            float gf = 1.f / (1.f + expf(-(a[1] + bias[1])));
+            float gg = tanhf(a[2] + bias[2]);
+            float go = 1.f / (1.f + expf(-(a[3] + bias[3])));
+            float cc = gf * c_state[(size_t)b * P + j] + gi * gg;
+            c_state[(size_t)b * P + j] = cc;
+            h_out[(size_t)b * P + j] = go * tanhf(cc);
+        }
+    }
+}
+
+// pred_proj[b, o] = W_pred[o, :] . h_top[b, :] + b_pred[o]; block o owns output o.
+template <typename TW>
+__global__ void __launch_bounds__(128) pred_proj_simt_kernel(const Ctrl* __restrict__ ctrl, const TW* __restrict__ w_pred,
+                                                             const float* __restrict__ b_pred, const float* __restrict__ h_top,
+                                                             float* __restrict__ pred_proj, int B, int P, int H) {
+    if (ctrl->active == 0) return;
+    extern __shared__ float sm[];
+    const int o = blockIdx.x;
+    for (int k = threadIdx.x; k < P; k += blockDim.x) sm[k] = ldf(w_pred + (size_t)o * P + k);
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    for (int b = warp; b < B; b += nw) {
+        float a = 0.f;
+        for (int k = lane; k < P; k += 32) a = fmaf(sm[k], round_like<TW>(h_top[(size_t)b * P + k]), a);
+        a = warp_sum(a);
+        if (lane == 0) pred_proj[(size_t)b * H + o] = a + b_pred[o];
+    }
+}
+
+template <typename TW>
+static cudaError_t simt_pred_step_t(const Call& c, int parity_in) {
+    const int P = c.m.P, B = c.B;
+    for (int l = 0; l < c.m.L; ++l) {
+        const int n_in = l == 0 ? c.m.E : P;
+        const float* x_below = l == 0 ? nullptr : c.h(1 - parity_in) + (size_t)(l - 1) * B * P;
+        size_t smem = sizeof(float) * 4 * (size_t)(n_in + P);
+        if (smem > 48 * 1024)
+            cudaFuncSetAttribute(lstm_layer_simt_kernel<TW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        lstm_layer_simt_kernel<TW><<<P, 128, smem, c.stream>>>(
+            c.ctrl(), c.emit_tok(), (const TW*)c.m.emb, x_below, (const TW*)c.w_ih[l], (const TW*)c.w_hh[l], c.b_ih[l],
+            c.b_hh[l], c.h(parity_in) + (size_t)l * B * P, c.h(1 - parity_in) + (size_t)l * B * P,
+            c.c() + (size_t)l * B * P, B, n_in, P);
+    }
+    pred_proj_simt_kernel<TW><<<c.m.H, 128, sizeof(float) * P, c.stream>>>(
+        c.ctrl(), (const TW*)c.m.w_pred, c.m.b_pred, c.h(1 - parity_in) + (size_t)(c.m.L - 1) * B * P, c.pred_proj(), B, P,
+        c.m.H);
+    return cudaGetLastError();
+}
+
+cudaError_t simt_pred_step(const Call& c, int parity_in) {
+    return c.m.dtype == WIND_DT_BF16 ? simt_pred_step_t<__nv_bfloat16>(c, parity_in) : simt_pred_step_t<float>(c, parity_in);
+}
+int simt_pred_launches(const Call& c) { return c.m.L + 1; }
+
+// ---------------------------------------------------------------------------
+// Windowed joint for one utterance per block: z[w] = act(enc_proj[b, t+w] + pred_proj[b]),
+// logits[w, v] = W_out[v] . z[w] + b_out[v]; per-row argmax key (or the logits themselves).
+// Rows are taken in chunks of 8 so the activation tile stays small.
+// ---------------------------------------------------------------------------
+template <typename TW>
+__global__ void __launch_bounds__(256) joint_simt_kernel(const Ctrl* __restrict__ ctrl, const int32_t* __restrict__ t_cur,
+                                                         const int32_t* __restrict__ enc_len, const TW* __restrict__ enc_proj,
+                                                         const float* __restrict__ pred_proj, const TW* __restrict__ w_out,
+                                                         const float* __restrict__ b_out, unsigned long long* __restrict__ keys,
+                                                         float* __restrict__ logits_out, int T, int W, int H, int NV, int act) {
+    if (ctrl->active == 0) return;
+    extern __shared__ float z[];  // [8][H]
+    __shared__ unsigned long long skey[8];
+    const int b = blockIdx.x;
+    const int t = t_cur[b], len = enc_len[b];
+    if (t >= len) return;
+    const int n = min(W, len - t);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    for (int w0 = 0; w0 < n; w0 += 8) {
+        const int nc = min(8, n - w0);
+        __syncthreads();
+        if (threadIdx.x < 8) skey[threadIdx.x] = 0ull;
+        for (int e = threadIdx.x; e < nc * H; e += blockDim.x) {
+            int w = e / H, k = e - w * H;
+            float s = ldf(enc_proj + ((size_t)b * T + t + w0 + w) * H + k) + pred_proj[(size_t)b * H + k];
+            s = act == WIND_ACT_RELU ? fmaxf(s, 0.f) : tanhf(s);
+            z[e] = round_like<TW>(s);
+        }
+        __syncthreads();
+        for (int v = warp; v < NV; v += nw) {
+            float a[8];
+#pragma unroll
+            for (int w = 0; w < 8; ++w) a[w] = 0.f;
+            for (int k = lane; k < H; k += 32) {
+                float wv = ldf(w_out + (size_t)v * H + k);
+#pragma unroll
+                for (int w = 0; w < 8; ++w)
+                    if (w < nc) a[w] = fmaf(wv, z[w * H + k], a[w]);
+            }
+#pragma unroll
+            for (int w = 0; w < 8; ++w) {
+                if (w < nc) {
+                    float s = warp_sum(a[w]) + b_out[v];
+                    if (lane == 0) {
+                        if (logits_out) logits_out[((size_t)b * W + w0 + w) * NV + v] = s;
+                        atomicMax(&skey[w], pack_key(s, (uint32_t)v));
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < nc) keys[(size_t)b * W + w0 + threadIdx.x] = skey[threadIdx.x];
+    }
+}
+
+cudaError_t simt_joint(const Call& c, float* logits_out) {
+    size_t smem = sizeof(float) * 8 * (size_t)c.m.H;
+    if (c.B == 0) return cudaSuccess;
+    if (c.m.dtype == WIND_DT_BF16) {
+        if (smem > 48 * 1024)
+            cudaFuncSetAttribute(joint_simt_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        joint_simt_kernel<__nv_bfloat16><<<c.B, 256, smem, c.stream>>>(
+            c.ctrl(), c.t(), c.enc_len, (const __nv_bfloat16*)c.enc_proj(), c.pred_proj(), (const __nv_bfloat16*)c.m.w_out,
+            c.m.b_out, c.keys(), logits_out, c.T, c.W, c.m.H, c.m.V + 1, c.m.act);
+    } else {
+        if (smem > 48 * 1024)
+            cudaFuncSetAttribute(joint_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        joint_simt_kernel<float><<<c.B, 256, smem, c.stream>>>(c.ctrl(), c.t(), c.enc_len, (const float*)c.enc_proj(),
+                                                                c.pred_proj(), (const float*)c.m.w_out, c.m.b_out, c.keys(),
+                                                                logits_out, c.T, c.W, c.m.H, c.m.V + 1, c.m.act);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace wind

@@ -1,0 +1,319 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+
+Comparison rule for (token, frame) sequences: bit-exact against the oracle's
+sequential result (Algorithm 1), except at decisions whose oracle top-2 logit
+margin is below 0.05; there the GPU's choice must still lie within 0.05 of the
+oracle's maximum (checked by replaying the GPU's sequence through the oracle),
+and the number of such decisions is reported.  Joint logits: 1e-4 abs on the
+fp32 path, 2e-2 abs on the bf16-weight path.
+"""
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import pytest
+
+import oracle
+import wind_synth as ws
+from naive_model import random_weights
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+MARGIN = 0.05
+TOL = {"f32": 1e-4, "bf16": 2e-2}
+
+
+@pytest.fixture(scope="module")
+def pkg():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2505_13765_b200 as p
+    p.load_library()
+    return p
+
+
+def check_against_oracle(pkg, weights, enc, lens, W, S, kernels=0, expect_exact=None, sample=None):
+    """Decode on the GPU, compare with the oracle.  Returns a report dict."""
+    prev = pkg.wind_set_kernels(kernels)
+    try:
+        model = pkg.WindModel(weights)
+        tok, frm, olen, stats, st = pkg.decode(model, enc, lens, W, S)
+    finally:
+        pkg.wind_set_kernels(prev)
+    assert st == 0
+    om = oracle.Model(weights)
+    B = enc.shape[0]
+    idx = list(range(B)) if sample is None else list(sample)
+    sub = np.ascontiguousarray(enc[idx])
+    otok, ofrm, on, ost = oracle.decode_batch(om, sub, lens[idx], W=0, S=S, max_out=tok.shape[1])
+
+    def replay(k):
+        b = idx[k]
+        return oracle.replay_verify(om, enc[b], int(lens[b]), S, tok[b, : olen[b]], frm[b, : olen[b]], MARGIN)
+
+    with ThreadPoolExecutor(8) as ex:
+        reps = list(ex.map(replay, range(len(idx))))
+    exact = 0
+    off_argmax = 0
+    for k, b in enumerate(idx):
+        r = reps[k]
+        assert r["rc"] == 0, f"utterance {b}: replay failed {r}"
+        off_argmax += r["not_argmax"]
+        same = on[k] == olen[b] and np.array_equal(otok[k, : on[k]], tok[b, : olen[b]]) and \
+            np.array_equal(ofrm[k, : on[k]], frm[b, : olen[b]])
+        exact += bool(same)
+        if r["not_argmax"] == 0:
+            assert same, f"utterance {b}: every decision is the oracle argmax yet the sequences differ"
+        f = frm[b, : olen[b]]
+        assert np.all(np.diff(f) >= 0)
+        if len(f):
+            assert f.max() < lens[b] and np.bincount(f).max() <= S
+        assert np.all(tok[b, olen[b]:] == -1)  # untouched beyond out_len
+    rep = dict(exact=exact, n=len(idx), off_argmax=off_argmax, low_margin_oracle=ost["low_margin"],
+               decisions=ost["decisions"], stats=stats)
+    if expect_exact:
+        assert exact == len(idx), rep
+    if sample is None:
+        assert stats["frames"] == int(lens.sum())
+        assert stats["tokens"] == int(olen.sum())
+        hist = np.array(stats["jump_hist"])
+        assert (hist * np.arange(65)).sum() + stats["forced"] == int(lens.sum())
+        assert hist[W + 1:].sum() == 0
+    print(f"[parity] W={W} S={S} exact {exact}/{len(idx)} utterances, {off_argmax} decisions off the oracle argmax "
+          f"(all inside {MARGIN}); oracle low-margin decisions {ost['low_margin']}/{ost['decisions']}")
+    return rep, (tok, frm, olen)
+
+
+def ragged_case(seed, B, T, D, E, P, L, H, V, act=0, blank_id=None, bias=1.0, dtype="f32"):
+    r = np.random.default_rng(1000 + seed)
+    w = random_weights(r, D, E, P, L, H, V, blank_id=blank_id, act=act, blank_bias=bias, bias_scale=0.1)
+    w["dtype"] = dtype
+    if dtype == "bf16":
+        for k in ("emb", "w_enc", "w_pred", "w_out"):
+            w[k] = ws.bf16_round(w[k])
+        w["w_ih"] = [ws.bf16_round(a) for a in w["w_ih"]]
+        w["w_hh"] = [ws.bf16_round(a) for a in w["w_hh"]]
+    lens = r.integers(0, T + 1, size=B).astype(np.int32)
+    lens[0] = T
+    if B > 2:
+        lens[1] = 0
+        lens[2] = 1
+    enc = r.standard_normal((B, T, D)).astype(np.float32)
+    if dtype == "bf16":
+        enc = ws.bf16_round(enc)
+    for b in range(B):
+        enc[b, lens[b]:] = np.nan
+    return w, enc, lens
+
+
+# ---------------------------------------------------------------------------
+# fp32 path
+# ---------------------------------------------------------------------------
+def test_cfg1_tiny_fp32(pkg):
+    cfg = ws.CONFIGS["cfg1_tiny"]
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="nan")
+    rep, out4 = check_against_oracle(pkg, weights, enc, lens, cfg.W, cfg.S)
+    rep1, out1 = check_against_oracle(pkg, weights, enc, lens, 1, cfg.S)
+    if rep["off_argmax"] == 0 and rep1["off_argmax"] == 0:
+        for a, b in zip(out4, out1):
+            assert np.array_equal(a, b)
+    rate = None
+    om = oracle.Model(weights)
+    _, _, _, st = oracle.decode_batch(om, enc, lens, W=0, S=cfg.S)
+    rate = st["emit_frames"] / lens.sum()
+    print(f"[cfg1] oracle non-blank frame rate on the workload sample: {rate:.3f}")
+
+
+@pytest.mark.parametrize("seed,W,S,act,blank0,L,bias", [
+    (0, 1, 3, 0, False, 1, 1.0), (1, 2, 2, 1, True, 2, 0.5), (2, 3, 1, 0, False, 1, 0.0), (3, 4, 5, 1, False, 3, 1.5),
+    (4, 8, 10, 0, True, 2, 1.0), (5, 16, 4, 0, False, 1, 2.0), (6, 64, 3, 1, False, 1, 1.0), (7, 5, 2, 0, False, 1, -3.0),
+])
+def test_fp32_ragged_shapes(pkg, seed, W, S, act, blank0, L, bias):
+    # odd sizes on purpose: nothing is a multiple of a tile
+    w, enc, lens = ragged_case(seed, B=7, T=53, D=37, E=29, P=41, L=L, H=67, V=45, act=act,
+                               blank_id=0 if blank0 else None, bias=bias)
+    check_against_oracle(pkg, w, enc, lens, W, S)
+
+
+def test_fp32_window_invariance_on_gpu(pkg):
+    w, enc, lens = ragged_case(20, B=5, T=80, D=32, E=32, P=32, L=1, H=64, V=30, bias=1.0)
+    outs = []
+    for W in (1, 2, 4, 8, 16, 64):
+        rep, out = check_against_oracle(pkg, w, enc, lens, W, 4)
+        outs.append((rep, out))
+    if all(r["off_argmax"] == 0 for r, _ in outs):
+        for _, o in outs[1:]:
+            for a, b in zip(o, outs[0][1]):
+                assert np.array_equal(a, b)
+
+
+def test_fp32_joint_logits(pkg):
+    w, enc, lens = ragged_case(30, B=6, T=40, D=48, E=24, P=40, L=2, H=72, V=50, act=1, bias=0.7)
+    logits_parity(pkg, w, enc, lens, W=4, S=3, tol=TOL["f32"], n_windows=24)
+
+
+def logits_parity(pkg, weights, enc, lens, W, S, tol, n_windows, kernels=0, seed=0):
+    """Teacher-forced logits at oracle-chosen prefixes and frames."""
+    om = oracle.Model(weights)
+    B, T, _ = enc.shape
+    otok, ofrm, on, _ = oracle.decode_batch(om, enc, lens, W=0, S=S)
+    r = np.random.default_rng(seed)
+    prev = pkg.wind_set_kernels(kernels)
+    model = pkg.WindModel(weights)
+    worst = 0.0
+    rows = 0
+    try:
+        for rep in range(max(1, n_windows // B)):
+            t0 = np.array([r.integers(0, max(1, lens[b])) if lens[b] else 0 for b in range(B)], np.int32)
+            if rep == 0:
+                t0[0] = max(0, lens[0] - 1)  # a window truncated by the end of the utterance
+            plen = np.array([int(np.searchsorted(ofrm[b, : on[b]], t0[b], side="left")) for b in range(B)], np.int32)
+            U = max(1, int(plen.max()))
+            prefix = np.zeros((B, U), np.int32)
+            for b in range(B):
+                prefix[b, : plen[b]] = otok[b, : plen[b]]
+            d = model.device
+            enc_d = pkg.to_device_enc(model, enc)
+            logits = torch.full((B, W, model.dims["V"] + 1), float("nan"), dtype=torch.float32, device=d)
+            wsb = pkg.alloc_workspace(model, B, T, W)
+            pkg.wind_eval_joint_window(model, enc_d, torch.from_numpy(lens).to(d), W, torch.from_numpy(prefix).to(d),
+                                       torch.from_numpy(plen).to(d), torch.from_numpy(t0).to(d), logits, wsb)
+            got = logits.cpu().numpy()
+            for b in range(B):
+                ref, *_ = oracle.eval_joint_window(om, enc[b], int(lens[b]), prefix[b, : plen[b]], int(t0[b]), W)
+                n = ref.shape[0]
+                assert n == max(0, min(W, lens[b] - t0[b]))
+                if n:
+                    err = np.max(np.abs(got[b, :n].astype(np.float64) - ref))
+                    worst = max(worst, float(err))
+                    rows += n
+                assert np.all(np.isnan(got[b, n:]))  # rows past the window are left untouched
+    finally:
+        pkg.wind_set_kernels(prev)
+    print(f"[logits] {rows} rows, worst abs error {worst:.3e} (tolerance {tol})")
+    assert rows > 0 and worst < tol
+
+
+# ---------------------------------------------------------------------------
+# bf16-weight path
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("kernels", [1, 0])
+def test_bf16_ragged_small(pkg, kernels):
+    # odd sizes: always the plain-ALU kernels
+    w, enc, lens = ragged_case(40, B=6, T=45, D=40, E=24, P=40, L=2, H=56, V=35, bias=1.0, dtype="bf16")
+    check_against_oracle(pkg, w, enc, lens, 4, 3, kernels=kernels)
+    logits_parity(pkg, w, enc, lens, W=4, S=3, tol=TOL["bf16"], n_windows=12, kernels=kernels)
+
+
+@pytest.mark.parametrize("kernels", [1, 0])
+@pytest.mark.parametrize("name,B,lo,hi,W", [
+    ("cfg3_large_b128", 5, 1, 150, 8), ("cfg3_large_b128", 3, 100, 300, 1), ("cfg4_xl_r25", 4, 20, 140, 16),
+    ("cfg4_xl_r50", 4, 20, 140, 4), ("cfg5_bigvocab", 3, 10, 60, 16),
+])
+def test_bf16_model_shapes_small_batches(pkg, kernels, name, B, lo, hi, W):
+    cfg = ws.small_variant(ws.CONFIGS[name], B, lo, hi)
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="nan")
+    rep, _ = check_against_oracle(pkg, weights, enc, lens, W, cfg.S, kernels=kernels)
+    assert rep["stats"]["kernels"] == (1 if kernels == 1 else rep["stats"]["kernels"])
+
+
+@pytest.mark.parametrize("kernels", [1, 0])
+@pytest.mark.parametrize("name,W", [("cfg3_large_b128", 8), ("cfg5_bigvocab", 16)])
+def test_bf16_joint_logits(pkg, kernels, name, W):
+    cfg = ws.small_variant(ws.CONFIGS[name], 8, 30, 90)
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="nan")
+    logits_parity(pkg, weights, enc, lens, W=W, S=cfg.S, tol=TOL["bf16"], n_windows=128 if name.startswith("cfg3") else 16,
+                  kernels=kernels)
+
+
+def test_cfg2_large_b1(pkg):
+    cfg = ws.CONFIGS["cfg2_large_b1"]
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="nan")
+    check_against_oracle(pkg, weights, enc, lens, cfg.W, cfg.S)
+
+
+def test_cfg3_full_batch_sampled_utterances(pkg):
+    # the launch configuration the benchmark times (B = 128, lengths 125..2500, W = 8);
+    # the oracle replays a sample of utterances (the shortest few, plus two drawn at random)
+    cfg = ws.CONFIGS["cfg3_large_b128"]
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="nan")
+    order = np.argsort(lens)
+    sample = sorted(set(order[:6].tolist() + [int(order[40]), int(order[64])]))
+    rep, out8 = check_against_oracle(pkg, weights, enc, lens, cfg.W, cfg.S, sample=sample)
+    st = rep["stats"]
+    assert st["frames"] == int(lens.sum())
+    hist = np.array(st["jump_hist"])
+    assert (hist * np.arange(65)).sum() + st["forced"] == int(lens.sum())
+    # properties that hold at any size
+    tok, frm, olen = out8
+    for b in range(cfg.B):
+        f = frm[b, : olen[b]]
+        assert np.all(np.diff(f) >= 0) and (len(f) == 0 or (f.max() < lens[b] and np.bincount(f).max() <= cfg.S))
+        assert np.all((tok[b, : olen[b]] >= 0) & (tok[b, : olen[b]] < cfg.V))
+
+
+# ---------------------------------------------------------------------------
+# behaviour of the interface
+# ---------------------------------------------------------------------------
+def test_determinism_and_workspace_reuse(pkg):
+    cfg = ws.small_variant(ws.CONFIGS["cfg3_large_b128"], 6, 10, 120)
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="nan")
+    model = pkg.WindModel(weights)
+    a = pkg.decode(model, enc, lens, 8, cfg.S)
+    b = pkg.decode(model, enc, lens, 8, cfg.S)
+    for x, y in zip(a[:3], b[:3]):
+        assert np.array_equal(x, y)
+    assert a[3] == b[3]
+
+
+def test_output_overflow_is_reported(pkg):
+    w, enc, lens = ragged_case(50, B=4, T=30, D=16, E=16, P=16, L=1, H=32, V=20, bias=-3.0)
+    model = pkg.WindModel(w)
+    tok, frm, olen, stats, st = pkg.decode(model, enc, lens, 4, 3, max_out=5, check=False)
+    assert st == pkg.binding.WIND_ERR_OUTPUT_OVERFLOW
+    assert olen.max() == 5
+    full = pkg.decode(model, enc, lens, 4, 3)
+    for b in range(4):
+        n = min(5, full[2][b])
+        assert np.array_equal(tok[b, :n], full[0][b, :n])
+
+
+def test_host_buffer_entry_point_matches_device_entry_point(pkg):
+    cfg = ws.small_variant(ws.CONFIGS["cfg3_large_b128"], 4, 10, 90)
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="zero")
+    model = pkg.WindModel(weights)
+    ref = pkg.decode(model, enc, lens, 8, cfg.S)
+    B, T, _ = enc.shape
+    max_out = T * cfg.S
+    enc_h = torch.from_numpy(enc).to(model.torch_dtype).pin_memory()
+    len_h = torch.from_numpy(lens).pin_memory()
+    tok_h = torch.full((B, max_out), -1, dtype=torch.int32).pin_memory()
+    frm_h = torch.full((B, max_out), -1, dtype=torch.int32).pin_memory()
+    ol_h = torch.zeros(B, dtype=torch.int32).pin_memory()
+    wsb = pkg.alloc_workspace(model, B, T, 8, host_staging_max_out=max_out)
+    pkg.wind_decode_greedy_host(model, enc_h, len_h, 8, cfg.S, tok_h, frm_h, ol_h, wsb)
+    assert np.array_equal(ol_h.numpy(), ref[2])
+    for b in range(B):
+        assert np.array_equal(tok_h.numpy()[b, : ref[2][b]], ref[0][b, : ref[2][b]])
+        assert np.array_equal(frm_h.numpy()[b, : ref[2][b]], ref[1][b, : ref[2][b]])
+
+
+def test_workspace_too_small_is_rejected(pkg):
+    w, enc, lens = ragged_case(60, B=2, T=10, D=8, E=8, P=8, L=1, H=8, V=5)
+    model = pkg.WindModel(w)
+    d = model.device
+    enc_d = pkg.to_device_enc(model, enc)
+    tok = torch.zeros((2, 30), dtype=torch.int32, device=d)
+    small = torch.empty(1024, dtype=torch.uint8, device=d)
+    st = pkg.wind_decode_greedy(model, enc_d, torch.from_numpy(lens).to(d), 4, 3, tok, tok.clone(), tok[:, 0].clone(), small,
+                                check=False)
+    assert st == pkg.binding.WIND_ERR_WORKSPACE

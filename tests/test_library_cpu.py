@@ -1,0 +1,93 @@
+"""Host-side checks of the CUDA library that need no GPU: it loads, exports every symbol the
+header declares, sizes its workspace as documented and rejects bad arguments before any launch."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+import paper_2505_13765_b200 as pkg
+from paper_2505_13765_b200 import binding as bd
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    entry.build()
+    return pkg.load_library()
+
+
+def large_model(**kw):
+    d = dict(D=512, E=640, P=640, L=1, H=640, V=1024, blank_id=1024, act=0, dtype=1)
+    d.update(kw)
+    return bd.wind_model_t(**d)
+
+
+def test_every_declared_symbol_is_exported(lib):
+    text = open(os.path.join(ROOT, "include", "wind.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(wind_[a-z_]+)\s*\(", text))
+    assert declared == set(bd.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_status_strings(lib):
+    names = [pkg.wind_status_string(i) for i in range(8)]
+    assert names[0] == "WIND_OK" and len(set(names)) == 8
+    assert pkg.wind_status_string(99) == "WIND_ERR_UNKNOWN"
+
+
+def test_workspace_grows_with_window_only_by_the_key_array(lib):
+    # The paper's memory analysis: WIND's only extra state is the window's logits,
+    # W x (V+1) floats per utterance (16 x 1025 = 16400 floats for W = 16).  Here the
+    # logits stay on chip and only an 8-byte argmax key per window row is kept.
+    m = large_model()
+    B, T = 128, 2500
+    base = pkg.wind_workspace_bytes(m, B, T, 1)
+    for W in (2, 4, 8, 16, 64):
+        extra = pkg.wind_workspace_bytes(m, B, T, W) - base
+        assert extra == 8 * B * (W - 1)
+        assert extra <= 4 * B * W * (m.V + 1)  # far below the paper's W x (V+1) floats per utterance
+    assert 16 * 1025 == 16400
+    # dominated by enc_proj [B, T, H] in bf16
+    assert base >= 2 * B * T * m.H and base < 2 * B * T * m.H * 1.02 + (1 << 22)
+
+
+def test_invalid_arguments_are_rejected_on_the_host(lib):
+    m = large_model()
+    n = C.c_size_t(0)
+    ref = C.byref(m)
+    assert lib.wind_workspace_bytes(None, 1, 1, 1, C.byref(n)) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_workspace_bytes(ref, 0, 10, 1, C.byref(n)) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_workspace_bytes(ref, 1, 10, 0, C.byref(n)) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_workspace_bytes(ref, 1, 10, 65, C.byref(n)) == bd.WIND_ERR_UNSUPPORTED
+    assert lib.wind_workspace_bytes(ref, 1, 10, 4, None) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_workspace_bytes(C.byref(large_model(blank_id=1025)), 1, 10, 4, C.byref(n)) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_workspace_bytes(C.byref(large_model(L=9)), 1, 10, 4, C.byref(n)) == bd.WIND_ERR_UNSUPPORTED
+    assert lib.wind_workspace_bytes(C.byref(large_model(act=2)), 1, 10, 4, C.byref(n)) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_workspace_bytes(ref, 4096, 4096, 4, C.byref(n)) == bd.WIND_ERR_UNSUPPORTED  # > 2^31 elements
+    # null weights / buffers: rejected before any CUDA call (this machine may have no GPU at all)
+    args = [ref, None, None, 1, 10, 4, 5, None, None, None, 50, None, 0, None]
+    assert lib.wind_decode_greedy(*args) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_decode_greedy_host(*args) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_eval_joint_window(ref, None, None, 1, 10, 4, None, 0, None, None, None, None, 0, None) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_read_stats(None, None, None) == bd.WIND_ERR_INVALID_ARG
+
+
+def test_set_kernels_round_trip(lib):
+    prev = pkg.wind_set_kernels(bd.WIND_KERNELS_SIMT)
+    assert pkg.wind_set_kernels(prev) == bd.WIND_KERNELS_SIMT
+    assert pkg.wind_set_kernels(77) == prev  # out of range: unchanged
+    assert pkg.wind_set_kernels(prev) == prev
+
+
+def test_product_path_does_not_touch_the_oracle():
+    pkg_dir = os.path.join(ROOT, "paper_2505_13765_b200")
+    for dirpath, _, files in os.walk(pkg_dir):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                src = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in src, f
