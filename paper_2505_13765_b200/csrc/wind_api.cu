@@ -107,6 +107,7 @@ static cudaError_t enqueue_step(const Call& c, bool tensor, int parity_in, cudaG
 static bool same_key(const Call& a, const Call& b) {
     Call x = a, y = b;
     x.stream = nullptr; y.stream = nullptr;
+    x.tc = nullptr; y.tc = nullptr;
     return memcmp(&x, &y, sizeof(Call)) == 0;
 }
 
@@ -163,7 +164,7 @@ static wind_status_t get_loop_graph(const Call& c, bool tensor, cudaGraphExec_t*
 }
 
 // Enqueue the whole decode on c.stream (no synchronisation).
-static wind_status_t enqueue_decode(const Call& c) {
+static wind_status_t enqueue_decode(Call& c) {
     const bool tensor = use_tensor(c);
     if (c.m.dtype == WIND_DT_BF16 && g_kernels == WIND_KERNELS_TENSOR && !tensor) return WIND_ERR_UNSUPPORTED;
     const int per_step = 2 + (tensor ? tc_pred_launches(c) : simt_pred_launches(c));

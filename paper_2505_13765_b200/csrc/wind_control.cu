@@ -7,14 +7,16 @@ namespace wind {
 
 // Reset all per-call state.  Block 0 also fills the control block.
 __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, int32_t* count, int32_t* emit_tok,
-                                                   unsigned long long* keys, float* h, float* c, int32_t* out_len,
+                                                   unsigned long long* keys, float* h, float* c, uint32_t* hb, int32_t* out_len,
                                                    const int32_t* __restrict__ enc_len, int B, int W, size_t n_h, size_t n_c,
+                                                   size_t n_hb_words,
                                                    int blank, int step_cap, int kernels_used, int launches_per_step,
                                                    int launches_setup) {
     const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t gstride = (size_t)gridDim.x * blockDim.x;
     for (size_t i = gtid; i < n_h; i += gstride) h[i] = 0.f;
     for (size_t i = gtid; i < n_c; i += gstride) c[i] = 0.f;
+    for (size_t i = gtid; i < n_hb_words; i += gstride) hb[i] = 0u;
     for (size_t i = gtid; i < (size_t)B * W; i += gstride) keys[i] = 0ull;
     for (size_t i = gtid; i < (size_t)B; i += gstride) {
         t[i] = 0;
@@ -62,8 +64,9 @@ cudaError_t launch_init(const Call& c, int kernels_used, int launches_per_step, 
     int blocks = (int)((n_h + 255) / 256);
     if (blocks > 296) blocks = 296;
     if (blocks < 1) blocks = 1;
-    init_kernel<<<blocks, 256, 0, c.stream>>>(c.ctrl(), c.t(), c.count(), c.emit_tok(), c.keys(), c.h(0), c.c(), c.out_len,
-                                              c.enc_len, c.B, c.W, n_h, n_c, c.m.blank_id, (int)step_cap, kernels_used,
+    init_kernel<<<blocks, 256, 0, c.stream>>>(c.ctrl(), c.t(), c.count(), c.emit_tok(), c.keys(), c.h(0), c.c(),
+                                              reinterpret_cast<uint32_t*>(c.hb(0, 0)), c.out_len, c.enc_len, c.B, c.W, n_h, n_c,
+                                              (size_t)c.m.L * c.lay.Bpad * c.m.P, c.m.blank_id, (int)step_cap, kernels_used,
                                               launches_per_step, launches_setup);
     return cudaGetLastError();
 }

@@ -41,15 +41,13 @@ struct Layout {
     size_t h;          // fp32 [2][L][B][P]  LSTM hidden state, ping-pong by step parity
     size_t c;          // fp32 [L][B][P]     LSTM cell state
     size_t pred_proj;  // fp32 [B][H]
-    size_t xh;         // bf16 [2][L][Bpad][in_l + P] decoder GEMM operand rows (tensor path)
+    size_t hb;         // bf16 [2][L][Bpad][P] LSTM hidden state as tensor-core operand rows (tensor path)
     size_t enc_proj;   // elem [B*T][H]
     size_t total;
     // host staging (wind_decode_greedy_host), placed after `total`
     size_t st_enc, st_len, st_tok, st_frm, st_olen, st_total;
     int32_t Bpad;      // B rounded up to 16 (tensor path operand rows)
-    int32_t xh_stride[kMaxLayers];  // elements per row of layer l's operand = in_l + P
-    size_t xh_layer_off[kMaxLayers]; // byte offset of layer l inside one parity's block
-    size_t xh_parity_bytes;
+    int32_t pad_;
 };
 
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -68,14 +66,7 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     L.c = take(sizeof(float) * (size_t)m.L * B * m.P);
     L.pred_proj = take(sizeof(float) * (size_t)B * m.H);
     L.Bpad = (B + 15) / 16 * 16;
-    size_t xb = 0;
-    for (int l = 0; l < m.L; ++l) {
-        L.xh_stride[l] = (l == 0 ? m.E : m.P) + m.P;
-        L.xh_layer_off[l] = xb;
-        xb = align_up(xb + (size_t)L.Bpad * L.xh_stride[l] * 2);
-    }
-    L.xh_parity_bytes = xb;
-    L.xh = take(2 * xb);
+    L.hb = take(2 * (size_t)m.L * L.Bpad * m.P * 2);
     L.enc_proj = take(es * (size_t)B * T * m.H);
     L.total = off;
     L.st_enc = take(es * (size_t)B * T * m.D);
@@ -103,6 +94,7 @@ struct Call {
     uint8_t* ws;
     Layout lay;
     cudaStream_t stream;
+    const void* tc;   // tensor maps of this call (host memory owned by the tensor-kernel module)
 
     Ctrl* ctrl() const { return reinterpret_cast<Ctrl*>(ws + lay.ctrl); }
     int32_t* t() const { return reinterpret_cast<int32_t*>(ws + lay.t); }
@@ -115,8 +107,8 @@ struct Call {
     float* c() const { return reinterpret_cast<float*>(ws + lay.c); }
     float* pred_proj() const { return reinterpret_cast<float*>(ws + lay.pred_proj); }
     void* enc_proj() const { return ws + lay.enc_proj; }
-    __nv_bfloat16* xh(int parity, int l) const {
-        return reinterpret_cast<__nv_bfloat16*>(ws + lay.xh + (size_t)parity * lay.xh_parity_bytes + lay.xh_layer_off[l]);
+    __nv_bfloat16* hb(int parity, int l) const {
+        return reinterpret_cast<__nv_bfloat16*>(ws + lay.hb) + ((size_t)parity * m.L + l) * lay.Bpad * m.P;
     }
 };
 
@@ -153,7 +145,7 @@ cudaError_t launch_set_t(const Call& c, const int32_t* t0);
 
 // tensor-core kernels (bf16 path)
 bool tc_supported(const wind_model_t& m, int B, int T, int W);
-cudaError_t tc_prepare(const Call& c);   // builds tensor maps for this call (host only)
+cudaError_t tc_prepare(Call& c);         // builds the tensor maps of this call (host only), sets c.tc
 cudaError_t tc_enc_proj(const Call& c);
 cudaError_t tc_pred_step(const Call& c, int parity_in);
 cudaError_t tc_joint(const Call& c, float* logits_out);
