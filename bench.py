@@ -179,6 +179,9 @@ def main():
     ap.add_argument("--workload", default="cfg3_large_b128")
     ap.add_argument("--window", type=int, default=0, help="override the workload's window (0 = its default)")
     ap.add_argument("--kernels", type=int, default=0, help="0 auto, 1 plain-ALU kernels, 2 tensor-core kernels")
+    ap.add_argument("--batch", type=int, default=0, help="override the number of utterances (profiling captures of a small case)")
+    ap.add_argument("--len-lo", type=int, default=0, help="override the shortest utterance length, frames")
+    ap.add_argument("--len-hi", type=int, default=0, help="override the longest utterance length, frames")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the W=1 comparison, e2e and per-kernel timing legs")
     args = ap.parse_args()
@@ -187,6 +190,8 @@ def main():
 
     import wind_synth as ws
     cfg = ws.CONFIGS[args.workload]
+    if args.batch or args.len_lo or args.len_hi:
+        cfg = ws.small_variant(cfg, args.batch or cfg.B, args.len_lo or cfg.len_lo, args.len_hi or cfg.len_hi)
     W = args.window or cfg.W
 
     if args.impl == "reference":
