@@ -160,6 +160,39 @@ wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, con
                                      const int32_t* prefix_len, const int32_t* t0, float* logits, void* workspace,
                                      size_t workspace_bytes, void* stream);
 
+/*
+ * Largest workspace, in bytes, that wind_eval_joint_window_static can serve: the size of the
+ * scratch array compiled into the library.
+ */
+#define WIND_STATIC_WORKSPACE_BYTES (16u * 1024u * 1024u)
+
+/*
+ * wind_eval_joint_window for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this entry point exists only for the sake of such callers.)
+ *
+ * Some callers of this library run where cudaMalloc is off limits: inside a stream-ordered
+ * section that must not synchronise the device, in a process whose memory pool is owned and
+ * fully handed out by another component, or in a real-time loop that is not allowed to touch
+ * the driver's allocator.  They cannot size and allocate the `workspace` the other entry points
+ * ask for.  This variant takes the same inputs and writes the same `logits`, but keeps all of
+ * its scratch (enc_proj, decoder state, keys, control words) in one array of
+ * WIND_STATIC_WORKSPACE_BYTES that is part of the library image: every GPU on which the
+ * library's kernels are loaded holds those bytes until the process exits.
+ *
+ *   - Nothing is allocated or freed, here or in any library routine the call uses.
+ *   - If wind_workspace_bytes(m, B, T, W) exceeds WIND_STATIC_WORKSPACE_BYTES the call returns
+ *     WIND_ERR_WORKSPACE before any launch; use wind_eval_joint_window with your own workspace.
+ *   - The first call on each device looks up the device address of the array (with that
+ *     device current).  Make that first call outside any stream capture.
+ *   - All calls on one device share the one array, which still holds what the previous call
+ *     left; every call re-initialises the parts that must start from zero.  Two calls that
+ *     overlap on the GPU (different streams, or different host threads) race on it: serialise them.
+ * Arguments, results and error codes are otherwise those of wind_eval_joint_window.
+ */
+wind_status_t wind_eval_joint_window_static(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B,
+                                            int32_t T, int32_t W, const int32_t* prefix, int32_t U,
+                                            const int32_t* prefix_len, const int32_t* t0, float* logits, void* stream);
+
 /* Per-kernel device times of one decode, from CUDA events recorded on `stream` around
  * every kernel launch (milliseconds summed over launches, and launch counts). */
 typedef struct {

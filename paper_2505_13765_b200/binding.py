@@ -30,7 +30,7 @@ WIND_KERNELS_AUTO, WIND_KERNELS_SIMT, WIND_KERNELS_TENSOR = 0, 1, 2
 
 EXPORTS = [
     "wind_workspace_bytes", "wind_decode_greedy", "wind_host_staging_bytes", "wind_decode_greedy_host",
-    "wind_eval_joint_window", "wind_profile_decode", "wind_read_stats", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
+    "wind_eval_joint_window", "wind_eval_joint_window_static", "wind_profile_decode", "wind_read_stats", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
 ]
 
 _vp = C.c_void_p
@@ -95,6 +95,8 @@ def load_library():
     L.wind_profile_decode.restype = i32
     L.wind_eval_joint_window.argtypes = [mp, _vp, _vp, i32, i32, i32, _vp, i32, _vp, _vp, _vp, _vp, C.c_size_t, _vp]
     L.wind_eval_joint_window.restype = i32
+    L.wind_eval_joint_window_static.argtypes = [mp, _vp, _vp, i32, i32, i32, _vp, i32, _vp, _vp, _vp, _vp]
+    L.wind_eval_joint_window_static.restype = i32
     L.wind_read_stats.argtypes = [_vp, _vp, C.POINTER(wind_stats_t)]
     L.wind_read_stats.restype = i32
     L.wind_set_kernels.argtypes = [i32]
@@ -282,6 +284,25 @@ def wind_eval_joint_window(model: WindModel, enc, enc_len, W: int, prefix, prefi
                                   prefix.data_ptr() if U else None, U, prefix_len.data_ptr(), t0.data_ptr(),
                                   logits.data_ptr(), _ws_ptr(workspace), _ws_bytes(workspace), _stream_ptr(stream))
     if st != WIND_OK:
+        raise WindError(st)
+    return st
+
+
+WIND_STATIC_WORKSPACE_BYTES = 16 * 1024 * 1024
+
+
+def wind_eval_joint_window_static(model: WindModel, enc, enc_len, W: int, prefix, prefix_len, t0, logits, stream=None,
+                                  check: bool = True) -> int:
+    """wind_eval_joint_window without a caller workspace: for callers that cannot allocate device
+    memory.  Scratch is the library's built-in array of WIND_STATIC_WORKSPACE_BYTES; larger problems
+    are rejected with WIND_ERR_WORKSPACE.  Calls sharing a device must not overlap on the GPU."""
+    L = load_library()
+    B, T, D = enc.shape
+    U = prefix.shape[1] if prefix is not None and prefix.numel() else 0
+    st = L.wind_eval_joint_window_static(model.ref, enc.data_ptr(), enc_len.data_ptr(), B, T, W,
+                                         prefix.data_ptr() if U else None, U, prefix_len.data_ptr(), t0.data_ptr(),
+                                         logits.data_ptr(), _stream_ptr(stream))
+    if check and st != WIND_OK:
         raise WindError(st)
     return st
 

@@ -322,6 +322,38 @@ wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, con
     return read_status(c);
 }
 
+// Scratch of wind_eval_joint_window_static.  In host code `g_static_ws` is only a handle for
+// the runtime's symbol lookup, never a device address: the address is resolved below.
+static __device__ __align__(256) unsigned char g_static_ws[WIND_STATIC_WORKSPACE_BYTES];
+constexpr int kMaxDevices = 64;
+static void* g_static_ws_addr[kMaxDevices] = {};
+static std::mutex g_static_mutex;
+
+wind_status_t wind_eval_joint_window_static(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B,
+                                            int32_t T, int32_t W, const int32_t* prefix, int32_t U,
+                                            const int32_t* prefix_len, const int32_t* t0, float* logits, void* stream) {
+    size_t need = 0;
+    wind_status_t s = wind_workspace_bytes(m, B, T, W, &need);
+    if (s != WIND_OK) return s;
+    if (need > (size_t)WIND_STATIC_WORKSPACE_BYTES) return WIND_ERR_WORKSPACE;
+    int dev = -1;
+    WIND_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return WIND_ERR_UNSUPPORTED;
+    void* ws = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ws_addr[dev]) {
+            // once per device, with that device current: the array's address on this device
+            void* addr = nullptr;
+            WIND_CUDA(cudaGetSymbolAddress(&addr, g_static_ws));
+            g_static_ws_addr[dev] = addr;
+        }
+        ws = g_static_ws_addr[dev];
+    }
+    return wind_eval_joint_window(m, enc, enc_len, B, T, W, prefix, U, prefix_len, t0, logits, ws,
+                                  (size_t)WIND_STATIC_WORKSPACE_BYTES, stream);
+}
+
 wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B, int32_t T,
                                   int32_t W, int32_t max_symbols, int32_t* out_tokens, int32_t* out_frames, int32_t* out_len,
                                   int32_t max_out, void* workspace, size_t workspace_bytes, void* stream,
