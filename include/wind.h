@@ -193,19 +193,24 @@ wind_status_t wind_eval_joint_window_static(const wind_model_t* m, const void* e
                                             int32_t T, int32_t W, const int32_t* prefix, int32_t U,
                                             const int32_t* prefix_len, const int32_t* t0, float* logits, void* stream);
 
-/* Per-kernel device times of one decode, from CUDA events recorded on `stream` around
- * every kernel launch (milliseconds summed over launches, and launch counts). */
+/* Per-kernel device times of one decode (milliseconds summed over launches, and launch counts):
+ * CUDA events recorded on `stream` around every launch on the plain-ALU path; on the tensor-core
+ * path the loop's phases as timed inside the persistent kernel. */
 typedef struct {
     double enc_proj_ms, joint_ms, control_ms, pred_ms;
     int64_t enc_proj_launches, joint_launches, control_launches, pred_launches;
+    /* tensor-core path only (zero otherwise): the decoding loop is one persistent kernel, so the
+     * figures above are its phases, timed from inside the kernel; loop_ms is its wall time,
+     * lstm_ms + proj_ms = pred_ms */
+    double loop_ms, lstm_ms, proj_ms;
 } wind_profile_t;
 
 /*
- * Measurement aid: the same decode as wind_decode_greedy (same kernels, same results), but
- * the loop is driven from the host in bursts of steps so that every launch can be
- * bracketed by a pair of CUDA events on `stream`.  Slower than wind_decode_greedy (events
- * and one synchronisation per burst); use it to attribute time to kernels, not as the
- * decoding path.  The paper has no counterpart; its timing is wall clock only.
+ * Measurement aid: the same decode as wind_decode_greedy (same kernels, same results) with the
+ * time attributed to its parts.  On the plain-ALU path the loop is driven from the host in bursts
+ * of steps so that every launch can be bracketed by a pair of CUDA events on `stream` (slower than
+ * wind_decode_greedy: events and one synchronisation per burst).  The paper has no counterpart; its
+ * timing is wall clock only.
  */
 wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B,
                                   int32_t T, int32_t W, int32_t max_symbols, int32_t* out_tokens,

@@ -96,12 +96,12 @@ static cudaStream_t g_capture_stream = nullptr;
 constexpr size_t kMaxGraphs = 12;
 
 static cudaError_t enqueue_step(const Call& c, bool tensor, int parity_in, cudaGraphConditionalHandle handle, int use_handle) {
-    cudaError_t e;
-    e = tensor ? tc_joint(c, nullptr) : simt_joint(c, nullptr);
+    (void)tensor;
+    cudaError_t e = simt_joint(c, nullptr);
     if (e != cudaSuccess) return e;
     e = launch_control(c, handle, use_handle);
     if (e != cudaSuccess) return e;
-    return tensor ? tc_pred_step(c, parity_in) : simt_pred_step(c, parity_in);
+    return simt_pred_step(c, parity_in);
 }
 
 static bool same_key(const Call& a, const Call& b) {
@@ -167,20 +167,28 @@ static wind_status_t get_loop_graph(const Call& c, bool tensor, cudaGraphExec_t*
 static wind_status_t enqueue_decode(Call& c) {
     const bool tensor = use_tensor(c);
     if (c.m.dtype == WIND_DT_BF16 && g_kernels == WIND_KERNELS_TENSOR && !tensor) return WIND_ERR_UNSUPPORTED;
-    const int per_step = 2 + (tensor ? tc_pred_launches(c) : simt_pred_launches(c));
-    const int setup = 2 + (tensor ? tc_pred_launches(c) : simt_pred_launches(c));
-    if (tensor) WIND_CUDA(tc_prepare(c));
-    WIND_CUDA(launch_init(c, tensor ? WIND_KERNELS_TENSOR : WIND_KERNELS_SIMT, per_step, setup));
-    WIND_CUDA(tensor ? tc_enc_proj(c) : simt_enc_proj(c));
-    WIND_CUDA(tensor ? tc_pred_step(c, 0) : simt_pred_step(c, 0));  // start of sequence: h[0] (zeros) -> h[1]
+    if (tensor) {
+        // projection and gate table once, then the whole loop as one persistent kernel
+        WIND_CUDA(tc_prepare(c));
+        WIND_CUDA(launch_init(c, WIND_KERNELS_TENSOR, 0, tc_setup_launches(c)));
+        WIND_CUDA(tc_enc_proj(c));
+        WIND_CUDA(tc_gate_table(c));
+        WIND_CUDA(tc_loop(c, nullptr, 0, nullptr, nullptr));
+        return WIND_OK;
+    }
+    const int per_step = 2 + simt_pred_launches(c);
+    const int setup = 2 + simt_pred_launches(c);
+    WIND_CUDA(launch_init(c, WIND_KERNELS_SIMT, per_step, setup));
+    WIND_CUDA(simt_enc_proj(c));
+    WIND_CUDA(simt_pred_step(c, 0));  // start of sequence: h[0] (zeros) -> h[1]
     const char* mode = getenv("WIND_LOOP");
     if (mode && strcmp(mode, "host") == 0) {
         // bring-up aid: fixed-size bursts of steps, the host polls the active count between bursts
         cudaGraphConditionalHandle none{};
         for (;;) {
             for (int k = 0; k < 8; ++k) {
-                WIND_CUDA(enqueue_step(c, tensor, 1, none, 0));
-                WIND_CUDA(enqueue_step(c, tensor, 0, none, 0));
+                WIND_CUDA(enqueue_step(c, false, 1, none, 0));
+                WIND_CUDA(enqueue_step(c, false, 0, none, 0));
             }
             Ctrl hc;
             WIND_CUDA(cudaMemcpyAsync(&hc, c.ctrl(), sizeof(Ctrl), cudaMemcpyDeviceToHost, c.stream));
@@ -190,7 +198,7 @@ static wind_status_t enqueue_decode(Call& c) {
         return WIND_OK;
     }
     cudaGraphExec_t exec = nullptr;
-    wind_status_t s = get_loop_graph(c, tensor, &exec);
+    wind_status_t s = get_loop_graph(c, false, &exec);
     if (s != WIND_OK) return s;
     WIND_CUDA(cudaGraphLaunch(exec, c.stream));
     return WIND_OK;
@@ -305,20 +313,28 @@ wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, con
     c.out_len = c.count();  // any int32 [B] scratch: init writes zeros to it
     const bool tensor = use_tensor(c);
     if (c.m.dtype == WIND_DT_BF16 && g_kernels == WIND_KERNELS_TENSOR && !tensor) return WIND_ERR_UNSUPPORTED;
-    if (tensor) WIND_CUDA(tc_prepare(c));
-    WIND_CUDA(launch_init(c, tensor ? WIND_KERNELS_TENSOR : WIND_KERNELS_SIMT, 0, 0));
-    WIND_CUDA(tensor ? tc_enc_proj(c) : simt_enc_proj(c));
+    if (tensor) {
+        WIND_CUDA(tc_prepare(c));
+        WIND_CUDA(launch_init(c, WIND_KERNELS_TENSOR, 0, 0));
+        WIND_CUDA(tc_enc_proj(c));
+        WIND_CUDA(tc_gate_table(c));
+        WIND_CUDA(launch_set_t(c, t0));
+        WIND_CUDA(tc_loop(c, prefix, U, prefix_len, logits));
+        return read_status(c);
+    }
+    WIND_CUDA(launch_init(c, WIND_KERNELS_SIMT, 0, 0));
+    WIND_CUDA(simt_enc_proj(c));
     WIND_CUDA(launch_set_t(c, t0));  // also sets active = B, so the decoder updates run even if every length is 0
     int parity = 0;
-    WIND_CUDA(tensor ? tc_pred_step(c, parity) : simt_pred_step(c, parity));  // start of sequence
+    WIND_CUDA(simt_pred_step(c, parity));  // start of sequence
     parity ^= 1;
     for (int u = 0; u < U; ++u) {
         WIND_CUDA(launch_force_tokens(c, prefix, U, prefix_len, u));
-        WIND_CUDA(tensor ? tc_pred_step(c, parity) : simt_pred_step(c, parity));
+        WIND_CUDA(simt_pred_step(c, parity));
         parity ^= 1;
     }
     WIND_CUDA(launch_set_t(c, t0));
-    WIND_CUDA(tensor ? tc_joint(c, logits) : simt_joint(c, logits));
+    WIND_CUDA(simt_joint(c, logits));
     return read_status(c);
 }
 
@@ -367,18 +383,52 @@ wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const 
     const bool tensor = use_tensor(c);
     if (c.m.dtype == WIND_DT_BF16 && g_kernels == WIND_KERNELS_TENSOR && !tensor) return WIND_ERR_UNSUPPORTED;
     memset(host_out, 0, sizeof(*host_out));
+    if (tensor) {
+        // the loop is one kernel: its phases are timed from inside (SM cycles of CTA 0, scaled by the
+        // kernel's wall time from the global timer); the projection is bracketed by events as usual
+        cudaEvent_t e0, e1;
+        WIND_CUDA(cudaEventCreate(&e0));
+        WIND_CUDA(cudaEventCreate(&e1));
+        WIND_CUDA(tc_prepare(c));
+        WIND_CUDA(launch_init(c, WIND_KERNELS_TENSOR, 0, tc_setup_launches(c)));
+        WIND_CUDA(cudaEventRecord(e0, c.stream));
+        WIND_CUDA(tc_enc_proj(c));
+        WIND_CUDA(cudaEventRecord(e1, c.stream));
+        WIND_CUDA(tc_gate_table(c));
+        WIND_CUDA(tc_loop(c, nullptr, 0, nullptr, nullptr));
+        Ctrl hc;
+        WIND_CUDA(cudaMemcpyAsync(&hc, c.ctrl(), sizeof(Ctrl), cudaMemcpyDeviceToHost, c.stream));
+        WIND_CUDA(cudaStreamSynchronize(c.stream));
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        cudaEventDestroy(e0);
+        cudaEventDestroy(e1);
+        host_out->enc_proj_ms = ms;
+        host_out->enc_proj_launches = 1;
+        const double cyc = (double)(hc.phase_cycles[0] + hc.phase_cycles[1] + hc.phase_cycles[2]);
+        const double ms_per_cycle = cyc > 0 ? (double)hc.loop_ns * 1e-6 / cyc : 0.0;
+        host_out->joint_ms = hc.phase_cycles[0] * ms_per_cycle;
+        host_out->pred_ms = (hc.phase_cycles[1] + hc.phase_cycles[2]) * ms_per_cycle;
+        host_out->control_ms = 0.0;   // the control step runs inside the decoder-update phase
+        host_out->joint_launches = hc.step;       // phases, not launches: one joint phase per lock step
+        host_out->pred_launches = hc.step + 1;
+        host_out->control_launches = 0;
+        host_out->loop_ms = (double)hc.loop_ns * 1e-6;
+        host_out->lstm_ms = hc.phase_cycles[1] * ms_per_cycle;
+        host_out->proj_ms = hc.phase_cycles[2] * ms_per_cycle;
+        return (wind_status_t)hc.status;
+    }
     constexpr int kBurst = 32;              // steps per burst
     constexpr int kEvents = 3 * kBurst + 1; // joint | control | pred boundaries
     std::vector<cudaEvent_t> ev(kEvents);
     for (auto& e : ev) WIND_CUDA(cudaEventCreate(&e));
     auto destroy = [&]() { for (auto& e : ev) cudaEventDestroy(e); };
-    const int pred_l = tensor ? tc_pred_launches(c) : simt_pred_launches(c);
-    if (tensor) WIND_CUDA(tc_prepare(c));
-    WIND_CUDA(launch_init(c, tensor ? WIND_KERNELS_TENSOR : WIND_KERNELS_SIMT, 2 + pred_l, 2 + pred_l));
+    const int pred_l = simt_pred_launches(c);
+    WIND_CUDA(launch_init(c, WIND_KERNELS_SIMT, 2 + pred_l, 2 + pred_l));
     WIND_CUDA(cudaEventRecord(ev[0], c.stream));
-    WIND_CUDA(tensor ? tc_enc_proj(c) : simt_enc_proj(c));
+    WIND_CUDA(simt_enc_proj(c));
     WIND_CUDA(cudaEventRecord(ev[1], c.stream));
-    WIND_CUDA(tensor ? tc_pred_step(c, 0) : simt_pred_step(c, 0));
+    WIND_CUDA(simt_pred_step(c, 0));
     WIND_CUDA(cudaEventRecord(ev[2], c.stream));
     WIND_CUDA(cudaStreamSynchronize(c.stream));
     float ms = 0.f;
@@ -393,11 +443,11 @@ wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const 
         if (before.active == 0) break;
         WIND_CUDA(cudaEventRecord(ev[0], c.stream));
         for (int k = 0; k < kBurst; ++k) {
-            WIND_CUDA(tensor ? tc_joint(c, nullptr) : simt_joint(c, nullptr));
+            WIND_CUDA(simt_joint(c, nullptr));
             WIND_CUDA(cudaEventRecord(ev[3 * k + 1], c.stream));
             WIND_CUDA(launch_control(c, none, 0));
             WIND_CUDA(cudaEventRecord(ev[3 * k + 2], c.stream));
-            WIND_CUDA(tensor ? tc_pred_step(c, parity) : simt_pred_step(c, parity));
+            WIND_CUDA(simt_pred_step(c, parity));
             WIND_CUDA(cudaEventRecord(ev[3 * k + 3], c.stream));
             parity ^= 1;
         }

@@ -7,9 +7,9 @@ namespace wind {
 
 // Reset all per-call state.  Block 0 also fills the control block.
 __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, int32_t* count, int32_t* emit_tok,
-                                                   unsigned long long* keys, float* h, float* c, uint32_t* hb, int32_t* out_len,
-                                                   const int32_t* __restrict__ enc_len, int B, int W, size_t n_h, size_t n_c,
-                                                   size_t n_hb_words,
+                                                   unsigned long long* keys, float* h, float* c, uint32_t* hb, uint32_t* z,
+                                                   int32_t* out_len, const int32_t* __restrict__ enc_len, int B, size_t n_keys,
+                                                   size_t n_h, size_t n_c, size_t n_hb_words, size_t n_z_words,
                                                    int blank, int step_cap, int kernels_used, int launches_per_step,
                                                    int launches_setup) {
     const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -17,9 +17,11 @@ __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, int32
     for (size_t i = gtid; i < n_h; i += gstride) h[i] = 0.f;
     for (size_t i = gtid; i < n_c; i += gstride) c[i] = 0.f;
     for (size_t i = gtid; i < n_hb_words; i += gstride) hb[i] = 0u;
-    for (size_t i = gtid; i < (size_t)B * W; i += gstride) keys[i] = 0ull;
+    for (size_t i = gtid; i < n_z_words; i += gstride) z[i] = 0u;
+    for (size_t i = gtid; i < n_keys; i += gstride) keys[i] = 0ull;
     for (size_t i = gtid; i < (size_t)B; i += gstride) {
         t[i] = 0;
+        t[B + i] = 0;
         count[i] = 0;
         emit_tok[i] = blank;  // start of sequence: every decoder is fed the blank id once
         out_len[i] = 0;
@@ -53,6 +55,10 @@ __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, int32
             ctrl->launches_setup = launches_setup;
             ctrl->kernels = kernels_used;
             ctrl->pad = 0;
+            ctrl->bar = 0u;
+            ctrl->abort = 0;
+            for (int k = 0; k < 4; ++k) ctrl->phase_cycles[k] = 0;
+            ctrl->loop_ns = 0;
         }
     }
 }
@@ -61,13 +67,19 @@ cudaError_t launch_init(const Call& c, int kernels_used, int launches_per_step, 
     size_t n_h = 2 * (size_t)c.m.L * c.B * c.m.P, n_c = (size_t)c.m.L * c.B * c.m.P;
     long long step_cap = (long long)c.T * (c.S + 1) + 2;
     if (step_cap > 0x7fffffff) step_cap = 0x7fffffff;
-    int blocks = (int)((n_h + 255) / 256);
-    if (blocks > 296) blocks = 296;
+    const bool bf = c.m.dtype == WIND_DT_BF16;
+    const size_t n_hb_words = bf ? (size_t)c.m.L * c.lay.Bpad * c.m.P : 0;       // 2 parities x bf16 = one word per element
+    const size_t n_z_words = bf ? (size_t)c.lay.rows_pad * c.m.H / 2 : 0;
+    size_t biggest = n_h > n_z_words ? n_h : n_z_words;
+    if (n_hb_words > biggest) biggest = n_hb_words;
+    int blocks = (int)((biggest + 255) / 256);
+    if (blocks > 592) blocks = 592;
     if (blocks < 1) blocks = 1;
     init_kernel<<<blocks, 256, 0, c.stream>>>(c.ctrl(), c.t(), c.count(), c.emit_tok(), c.keys(), c.h(0), c.c(),
-                                              reinterpret_cast<uint32_t*>(c.hb(0, 0)), c.out_len, c.enc_len, c.B, c.W, n_h, n_c,
-                                              (size_t)c.m.L * c.lay.Bpad * c.m.P, c.m.blank_id, (int)step_cap, kernels_used,
-                                              launches_per_step, launches_setup);
+                                              reinterpret_cast<uint32_t*>(c.hb(0, 0)), reinterpret_cast<uint32_t*>(c.z()),
+                                              c.out_len, c.enc_len, c.B, 2 * (size_t)c.lay.rows_pad, n_h, n_c, n_hb_words,
+                                              n_z_words, c.m.blank_id, (int)step_cap, kernels_used, launches_per_step,
+                                              launches_setup);
     return cudaGetLastError();
 }
 
@@ -176,7 +188,7 @@ cudaError_t launch_force_tokens(const Call& c, const int32_t* prefix, int U, con
 __global__ void set_t_kernel(Ctrl* ctrl, int32_t* t, const int32_t* __restrict__ t0, int B) {
     int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b == 0) ctrl->active = B;
-    if (b < B) t[b] = t0[b];
+    if (b < B) { t[b] = t0[b]; t[B + b] = t0[b]; }
 }
 cudaError_t launch_set_t(const Call& c, const int32_t* t0) {
     set_t_kernel<<<(c.B + 127) / 128, 128, 0, c.stream>>>(c.ctrl(), c.t(), t0, c.B);

@@ -29,25 +29,32 @@ struct Ctrl {
     int32_t launches_setup;
     int32_t kernels;
     int32_t pad;
+    // persistent loop kernel
+    uint32_t bar;             // grid barrier: arrivals so far (monotonic within a call)
+    int32_t abort;            // some CTA gave up: everybody leaves
+    long long phase_cycles[4];  // SM cycles spent in the joint / decoder-update / projection phases (CTA 0), [3] unused
+    long long loop_ns;        // wall time of the loop kernel (CTA 0, global timer)
 };
 
 // Byte offsets of every workspace region (all multiples of kAlign).
 struct Layout {
     size_t ctrl;       // Ctrl
-    size_t t;          // int32 [B]   current frame per utterance
+    size_t t;          // int32 [2][B] current frame per utterance (the loop kernel ping-pongs by step parity)
     size_t count;      // int32 [B]   consecutive emissions on the current frame
     size_t emit_tok;   // int32 [B]   token to feed to the decoder this step, -1 = none
-    size_t keys;       // uint64 [B*W] packed (logit, label) argmax keys, 0 = empty
-    size_t h;          // fp32 [2][L][B][P]  LSTM hidden state, ping-pong by step parity
+    size_t keys;       // uint64 [2][rows_pad] packed (logit, label) argmax keys, 0 = empty (second half: loop kernel)
+    size_t h;          // fp32 [2][L][B][P]  LSTM hidden state, ping-pong by step parity (plain-ALU path)
     size_t c;          // fp32 [L][B][P]     LSTM cell state
-    size_t pred_proj;  // fp32 [B][H]
+    size_t pred_proj;  // fp32 [B][H]        (plain-ALU path)
     size_t hb;         // bf16 [2][L][Bpad][P] LSTM hidden state as tensor-core operand rows (tensor path)
+    size_t z;          // bf16 [rows_pad][H] joint activations act(enc_proj + pred_proj), the joint GEMM's operand (tensor path)
+    size_t g0;         // fp32 [V+1][4P] layer-0 gate pre-activations of every token: W_ih emb[tok] + b_ih + b_hh (tensor path)
     size_t enc_proj;   // elem [B*T][H]
     size_t total;
     // host staging (wind_decode_greedy_host), placed after `total`
     size_t st_enc, st_len, st_tok, st_frm, st_olen, st_total;
-    int32_t Bpad;      // B rounded up to 16 (tensor path operand rows)
-    int32_t pad_;
+    int32_t Bpad;      // B rounded up to 128 (tensor path operand rows)
+    int32_t rows_pad;  // B*W rounded up to 256 (window rows incl. tile padding)
 };
 
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -58,15 +65,19 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
     L.ctrl = take(sizeof(Ctrl));
-    L.t = take(sizeof(int32_t) * B);
+    const bool bf = m.dtype == WIND_DT_BF16;
+    L.rows_pad = (int32_t)(((size_t)B * W + 255) / 256 * 256);
+    L.t = take(sizeof(int32_t) * 2 * B);
     L.count = take(sizeof(int32_t) * B);
     L.emit_tok = take(sizeof(int32_t) * B);
-    L.keys = take(sizeof(uint64_t) * (size_t)B * W);
+    L.keys = take(sizeof(uint64_t) * 2 * (size_t)L.rows_pad);
     L.h = take(sizeof(float) * 2 * (size_t)m.L * B * m.P);
     L.c = take(sizeof(float) * (size_t)m.L * B * m.P);
     L.pred_proj = take(sizeof(float) * (size_t)B * m.H);
-    L.Bpad = (B + 15) / 16 * 16;
-    L.hb = take(2 * (size_t)m.L * L.Bpad * m.P * 2);
+    L.Bpad = (B + 127) / 128 * 128;
+    L.hb = take(bf ? 2 * (size_t)m.L * L.Bpad * m.P * 2 : 0);
+    L.z = take(bf ? (size_t)L.rows_pad * m.H * 2 : 0);
+    L.g0 = take(bf ? sizeof(float) * (size_t)(m.V + 1) * 4 * m.P : 0);
     L.enc_proj = take(es * (size_t)B * T * m.H);
     L.total = off;
     L.st_enc = take(es * (size_t)B * T * m.D);
@@ -97,16 +108,18 @@ struct Call {
     const void* tc;   // tensor maps of this call (host memory owned by the tensor-kernel module)
 
     Ctrl* ctrl() const { return reinterpret_cast<Ctrl*>(ws + lay.ctrl); }
-    int32_t* t() const { return reinterpret_cast<int32_t*>(ws + lay.t); }
+    int32_t* t() const { return reinterpret_cast<int32_t*>(ws + lay.t); }   // [2][B]; the per-phase kernels use [0]
     int32_t* count() const { return reinterpret_cast<int32_t*>(ws + lay.count); }
     int32_t* emit_tok() const { return reinterpret_cast<int32_t*>(ws + lay.emit_tok); }
-    unsigned long long* keys() const { return reinterpret_cast<unsigned long long*>(ws + lay.keys); }
+    unsigned long long* keys() const { return reinterpret_cast<unsigned long long*>(ws + lay.keys); }  // [2][rows_pad]
     float* h(int parity) const {
         return reinterpret_cast<float*>(ws + lay.h) + (size_t)parity * m.L * B * m.P;
     }
     float* c() const { return reinterpret_cast<float*>(ws + lay.c); }
     float* pred_proj() const { return reinterpret_cast<float*>(ws + lay.pred_proj); }
     void* enc_proj() const { return ws + lay.enc_proj; }
+    __nv_bfloat16* z() const { return reinterpret_cast<__nv_bfloat16*>(ws + lay.z); }
+    float* g0() const { return reinterpret_cast<float*>(ws + lay.g0); }
     __nv_bfloat16* hb(int parity, int l) const {
         return reinterpret_cast<__nv_bfloat16*>(ws + lay.hb) + ((size_t)parity * m.L + l) * lay.Bpad * m.P;
     }
@@ -145,10 +158,13 @@ cudaError_t launch_set_t(const Call& c, const int32_t* t0);
 
 // tensor-core kernels (bf16 path)
 bool tc_supported(const wind_model_t& m, int B, int T, int W);
-cudaError_t tc_prepare(Call& c);         // builds the tensor maps of this call (host only), sets c.tc
+cudaError_t tc_prepare(Call& c);         // builds the tensor maps and the tile plan of this call (host only), sets c.tc
 cudaError_t tc_enc_proj(const Call& c);
-cudaError_t tc_pred_step(const Call& c, int parity_in);
-cudaError_t tc_joint(const Call& c, float* logits_out);
-int tc_pred_launches(const Call& c);
+cudaError_t tc_gate_table(const Call& c);  // g0[tok] = W_ih[0] emb[tok] + b_ih[0] + b_hh[0] for every token
+// The whole decoding loop as one persistent cooperative kernel.  prefix == nullptr: greedy
+// decoding until every utterance is done.  Otherwise teacher forcing: feed prefix tokens, then
+// store the window logits at t (set beforehand in both t buffers) to logits_out.
+cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* prefix_len, float* logits_out);
+int tc_setup_launches(const Call& c);
 
 }  // namespace wind

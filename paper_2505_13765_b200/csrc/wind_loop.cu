@@ -1,0 +1,797 @@
+// The decoding loop of the bf16 path as ONE persistent cooperative kernel (sm_100a).
+//
+// One CTA per SM stays resident for the whole decode.  A lock step of the batch
+// (Algorithm 2 applied to every utterance at once) is three phases separated by grid
+// barriers; every phase is a tensor-core GEMM whose operands arrive by TMA and whose
+// accumulator lives in tensor memory:
+//
+//   J  joint      logits^T [vocab tile 128, window rows N] = W_out tile . z^T, epilogue = per-row
+//                 argmax over the tile's 128 vocabulary entries by warp shuffles, combined across
+//                 vocabulary tiles with a 64-bit atomicMax on (logit, label) keys.  The logits never
+//                 leave the chip.  When every CTA owns exactly one tile, its W_out tile is loaded
+//                 once and stays in shared memory for the whole decode.
+//   L  decoder    gates [utterances 128, 4 x units] = h . W_hh^T (+ x . W_ih^T for upper layers);
+//                 the epilogue first does the control step for its utterances -- first-non-blank
+//                 scan of the window's keys, jump, emission, max-symbols rule (one CTA per
+//                 utterance tile writes the results, the others only need the token) -- then the
+//                 LSTM cell update.  Layer 0's input term W_ih emb[tok] + b comes from a table
+//                 computed once per call, so the embedding costs no GEMM work inside the loop.
+//   P  projection pred_proj [utterances 128, H slice] = h_top . W_pred^T + b_pred, epilogue =
+//                 z[b, w, slice] = act(enc_proj[b, t_b + w, slice] + pred_proj) for the next window.
+//
+// Roles per CTA: warp 0 issues TMA, warp 1 issues tcgen05.mma, warps 2..5 run the epilogues
+// (one thread per tensor-memory lane).  State that one phase reads while another CTA writes it
+// is double-buffered by step parity (t, keys), so a phase never reads what it writes.
+//
+// Every wait is bounded (mbarrier waits and the grid barrier): a CTA that runs out of patience
+// flags WIND_ERR_TIMEOUT, raises the global abort word, and every CTA leaves at its next wait.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <mutex>
+
+#include "wind_internal.cuh"
+#include "wind_ptx.cuh"
+#include "wind_loop.cuh"
+
+namespace wind {
+
+constexpr int LOOP_THREADS = 192;
+constexpr int LOOP_MAX_STAGES = 12;
+constexpr uint32_t LOOP_A_BYTES = 128 * BK * 2;  // one K block of a 128-row operand tile
+constexpr uint32_t LOOP_TMEM_COLS = 512;
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ int ld_volatile_i32(const int* p) {
+    int v;
+    asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// generic-proxy writes of this thread become visible to later async-proxy (TMA) reads
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// 32 lanes x 8 consecutive columns
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// One stage of the exchange that turns "every lane holds 2*HALF columns" into "every lane holds HALF
+// columns, reduced over lane pairs": lanes with bit HALF set keep the upper columns.
+template <int HALF>
+__device__ __forceinline__ void argmax_exchange(float* v, int* id, int lane) {
+    const bool up = (lane & HALF) != 0;
+#pragma unroll
+    for (int c = 0; c < HALF; ++c) {
+        const float sv = up ? v[c] : v[c + HALF];
+        const int si = up ? id[c] : id[c + HALF];
+        const float kv = up ? v[c + HALF] : v[c];
+        const int ki = up ? id[c + HALF] : id[c];
+        const float rv = __shfl_xor_sync(0xffffffffu, sv, HALF);
+        const int ri = __shfl_xor_sync(0xffffffffu, si, HALF);
+        const bool take = (rv > kv) || (rv == kv && ri < ki);   // lowest label on equal logits
+        v[c] = take ? rv : kv;
+        id[c] = take ? ri : ki;
+    }
+}
+
+struct PipeState {
+    uint32_t it;    // K blocks pushed (producer) or consumed (MMA issuer) so far, over the whole kernel
+    uint32_t acc;   // accumulator uses so far (MMA issuer and epilogue count the same items)
+};
+
+__global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_constant__ LoopMaps M, const LoopParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[LOOP_MAX_STAGES], empty_bar[LOOP_MAX_STAGES], stat_bar, acc_full, acc_empty;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int s_abort;      // this CTA has given up
+    __shared__ int s_active;     // utterances still decoding (set in the projection phase)
+    __shared__ int s_red[4];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cta = blockIdx.x, G = gridDim.x;
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* stat = smem;                       // stationary W_out tile: kb_h blocks of 128 x 64 bf16
+    uint8_t* ring = smem + p.stat_bytes;        // stages of [128-row operand block | small operand block]
+    const int S = p.stages;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        s_active = 0;
+        for (int s = 0; s < S; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        mbar_init(&stat_bar, 1);
+        mbar_init(&acc_full, 1);
+        mbar_init(&acc_empty, 4);
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(&tmem_slot, LOOP_TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+
+    if (p.j_stationary && cta < p.j_items && threadIdx.x == 0) {
+        const int vt = cta % p.vt_count;
+        mbar_expect_tx(&stat_bar, (uint32_t)p.kb_h * LOOP_A_BYTES);
+        for (int kb = 0; kb < p.kb_h; ++kb) tma_load_2d(stat + (size_t)kb * LOOP_A_BYTES, &M.w_out, kb * BK, vt * 128, &stat_bar);
+    }
+
+    PipeState ps{0u, 0u};
+    uint32_t epoch = 0;          // grid barrier target (thread 0)
+    int step = -1;               // -1: start of sequence
+    int pin = 0;                 // hb[pin] holds the current decoder state
+    long long clk_last = 0, cyc[3] = {0, 0, 0};
+    unsigned long long ns0 = 0;
+    if (cta == 0 && threadIdx.x == 0) { clk_last = clock64(); ns0 = globaltimer_ns(); }
+    int exit_status = 0;
+
+    // ----- helpers -------------------------------------------------------------------------
+    // Grid barrier for all threads of all CTAs; false when the kernel is being abandoned.
+    auto grid_sync = [&](int phase_kind) -> bool {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            epoch += (uint32_t)G;
+            if (s_abort) {
+                atomicExch(&p.ctrl->abort, 1);
+            } else {
+                __threadfence();
+                atomicAdd(&p.ctrl->bar, 1u);
+                unsigned long long t0 = 0;
+                for (uint32_t it = 1;; ++it) {
+                    if ((int32_t)(ld_acquire_u32(&p.ctrl->bar) - epoch) >= 0) break;
+                    if ((it & 63u) == 0u) {
+                        if (ld_volatile_i32(&p.ctrl->abort)) { s_abort = 2; break; }
+                        const unsigned long long now = globaltimer_ns();
+                        if (t0 == 0) t0 = now;
+                        else if (now - t0 > kWaitLimitNs) { s_abort = 1; atomicExch(&p.ctrl->abort, 1); break; }
+                    }
+                }
+                __threadfence();
+            }
+            if (cta == 0) {
+                const long long now = clock64();
+                cyc[phase_kind] += now - clk_last;
+                clk_last = now;
+            }
+        }
+        __syncthreads();
+        return s_abort == 0;
+    };
+
+    const int e = threadIdx.x - 64;            // epilogue thread 0..127 (warps 2..5)
+    const int q = warp & 3;                    // tensor-memory lane quadrant of this warp
+    const int row_in_tile = q * 32 + lane;     // the tensor-memory lane (accumulator row) of this thread
+    const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
+
+    for (;;) {
+        // =====================================================================================
+        // L phases: control step (layer 0 of a decoding step) + LSTM cell update, one phase per layer
+        // =====================================================================================
+        for (int l = 0; l < p.L; ++l) {
+            const int n_tile = 4 * p.slots;
+            const int segs = l == 0 ? 1 : 2;
+            const uint32_t b_bytes = (uint32_t)n_tile * BK * 2;
+            if (warp == 0) {
+                if (lane == 0) {
+                    fence_proxy_async_all();
+                    for (int i = cta; i < p.l_items; i += G) {
+                        const int mt = i / p.ug_count, ug = i - mt * p.ug_count;
+                        for (int sg = 0; sg < segs; ++sg) {
+                            const CUtensorMap* ma = (l == 0 || sg == 1) ? &M.hb[pin][l] : &M.hb[pin ^ 1][l - 1];
+                            const CUtensorMap* mb = (l == 0 || sg == 1) ? &M.w_hh[l] : &M.w_ih[l];
+                            for (int kb = 0; kb < p.kb_p; ++kb) {
+                                const int s = ps.it % S;
+                                if (!mbar_wait(&empty_bar[s], ((ps.it / S) & 1) ^ 1, &s_abort)) goto l_done;
+                                uint8_t* a_dst = ring + (size_t)s * p.stage_bytes;
+                                uint8_t* b_dst = a_dst + LOOP_A_BYTES;
+                                mbar_expect_tx(&full_bar[s], LOOP_A_BYTES + b_bytes);
+                                tma_load_2d(a_dst, ma, kb * BK, mt * 128, &full_bar[s]);
+                                for (int g = 0; g < 4; ++g)
+                                    tma_load_2d(b_dst + (size_t)g * p.slots * 128, mb, kb * BK, g * p.P + ug * p.ul, &full_bar[s]);
+                                ++ps.it;
+                            }
+                        }
+                    }
+                }
+            } else if (warp == 1) {
+                if (lane == 0) {
+                    const uint32_t idesc = idesc_bf16(128, n_tile);
+                    for (int i = cta; i < p.l_items; i += G) {
+                        if (!mbar_wait(&acc_empty, (ps.acc & 1) ^ 1, &s_abort)) goto l_done;
+                        tc_fence_after();
+                        const int kbs = segs * p.kb_p;
+                        for (int kb = 0; kb < kbs; ++kb) {
+                            const int s = ps.it % S;
+                            if (!mbar_wait(&full_bar[s], (ps.it / S) & 1, &s_abort)) goto l_done;
+                            tc_fence_after();
+                            const uint32_t a_addr = smem_u32(ring + (size_t)s * p.stage_bytes);
+                            const uint64_t adesc = smem_desc_sw128(a_addr);
+                            const uint64_t bdesc = smem_desc_sw128(a_addr + LOOP_A_BYTES);
+#pragma unroll
+                            for (int k = 0; k < BK / 16; ++k)
+                                tc_mma_bf16(tmem_base, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+                            tc_commit(&empty_bar[s]);
+                            ++ps.it;
+                        }
+                        tc_commit(&acc_full);
+                        ++ps.acc;
+                    }
+                }
+            } else {
+                const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
+                int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
+                const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
+                unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
+                for (int i = cta; i < p.l_items; i += G) {
+                    const int mt = i / p.ug_count, ug = i - mt * p.ug_count;
+                    const int b = mt * 128 + row_in_tile;
+                    // ---- which token does utterance b feed to its decoder in this step? ----
+                    int tok = -1;
+                    if (b < p.B) {
+                        if (step < 0) {
+                            tok = p.blank;
+                        } else if (p.forced) {
+                            tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
+                        } else if (l > 0) {
+                            tok = p.emit_tok[b];
+                        } else {
+                            // control step (Algorithm 2's branch): first non-blank row of the window
+                            int t = t_cur[b];
+                            const int len = p.enc_len[b];
+                            if (t < len) {
+                                const int n = min(p.W, len - t);
+                                int first = -1, label = p.blank;
+                                bool bad = false;
+                                for (int w0 = 0; w0 < n && first < 0; w0 += 8) {
+                                    unsigned long long kk[8];
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) kk[j] = (w0 + j < n) ? keys_cur[(size_t)b * p.W + w0 + j] : 0ull;
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) {
+                                        if (w0 + j < n && first < 0) {
+                                            uint32_t lab = key_label(kk[j]);
+                                            if (kk[j] == 0ull || lab >= (uint32_t)p.NV) { bad = true; lab = (uint32_t)p.blank; }
+                                            if ((int)lab != p.blank) { first = w0 + j; label = (int)lab; }
+                                        }
+                                    }
+                                }
+                                if (first >= 0) tok = label;
+                                if (ug == 0) {
+                                    // this CTA records the step for its utterances
+                                    int cnt = p.count[b];
+                                    int jump, forced = 0, emitted = 0;
+                                    if (first < 0) {
+                                        jump = n;
+                                        t += n;
+                                        cnt = 0;
+                                    } else {
+                                        jump = first;
+                                        if (first > 0) cnt = 0;
+                                        t += first;
+                                        const int pos = p.out_len[b];
+                                        if (pos < p.max_out) {
+                                            p.out_tokens[(size_t)b * p.max_out + pos] = label;
+                                            p.out_frames[(size_t)b * p.max_out + pos] = t;
+                                            p.out_len[b] = pos + 1;
+                                            emitted = 1;
+                                            cnt += 1;
+                                            if (cnt == p.S) { t += 1; cnt = 0; forced = 1; }
+                                        } else {
+                                            set_status(p.ctrl, WIND_ERR_OUTPUT_OVERFLOW);  // this utterance stops here
+                                            t = len;
+                                            tok = -1;
+                                        }
+                                    }
+                                    if (bad) set_status(p.ctrl, WIND_ERR_INTERNAL);
+                                    t_nxt[b] = t;
+                                    p.count[b] = cnt;
+                                    for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
+                                    atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
+                                    atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->joint_rows), (unsigned long long)n);
+                                    if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
+                                    if (forced) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
+                                }
+                            } else if (ug == 0) {
+                                t_nxt[b] = t;
+                            }
+                            if (ug == 0) p.emit_tok[b] = tok;
+                        }
+                    }
+                    // ---- LSTM cell update of units [ug*ul, ug*ul + ul) for utterance b ----
+                    const float* bi = p.b_ih[l];
+                    const float* bh = p.b_hh[l];
+                    float* cst = p.c_state + ((size_t)l * p.B + (b < p.B ? b : 0)) * p.P;
+                    const __nv_bfloat16* hin = p.hb + (((size_t)pin * p.L + l) * p.Bpad + (b < p.B ? b : 0)) * p.P;
+                    __nv_bfloat16* hout = p.hb + (((size_t)(pin ^ 1) * p.L + l) * p.Bpad + (b < p.B ? b : 0)) * p.P;
+                    const bool live = b < p.B && tok >= 0;
+                    const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full, ps.acc & 1, &s_abort));
+                    tc_fence_after();
+                    if (ready) {
+                        for (int u0 = 0; u0 < p.ul; u0 += 8) {
+                            float pre[4][8];
+#pragma unroll
+                            for (int g = 0; g < 4; ++g) tmem_ld8(tq + (uint32_t)(g * p.slots + u0), pre[g]);
+                            if (b < p.B) {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    const int unit = ug * p.ul + u0 + j;
+                                    if (u0 + j < p.ul && unit < p.P) {
+                                        if (live) {
+                                            float add[4];
+#pragma unroll
+                                            for (int g = 0; g < 4; ++g)
+                                                add[g] = l == 0 ? p.g0[(size_t)tok * 4 * p.P + (size_t)g * p.P + unit]
+                                                                : bi[g * p.P + unit] + bh[g * p.P + unit];
+                                            const float gi = sigmoid_f(pre[0][j] + add[0]);
+                                            const float gf = sigmoid_f(pre[1][j] + add[1]);
+                                            const float gg = tanhf(pre[2][j] + add[2]);
+                                            const float go = sigmoid_f(pre[3][j] + add[3]);
+                                            const float cc = gf * cst[unit] + gi * gg;
+                                            cst[unit] = cc;
+                                            hout[unit] = __float2bfloat16_rn(go * tanhf(cc));
+                                        } else {
+                                            hout[unit] = hin[unit];
+                                        }
+                                    }
+                                }
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty);
+                    ++ps.acc;
+                    if (!ready) goto l_done;
+                }
+                if (cta == 0 && e == 0 && l == 0 && step >= 0 && !p.forced) p.ctrl->step = step + 1;
+                fence_proxy_async_all();
+            }
+        l_done:
+            // keep the role threads' counters in step: the MMA issuer and the epilogue count items alike,
+            // producer and MMA issuer count K blocks alike; lanes other than 0 of warps 0/1 hold no state
+            if (!grid_sync(1)) goto done;
+        }
+        pin ^= 1;
+        if (p.forced && step + 1 < p.U) { ++step; continue; }
+
+        // =====================================================================================
+        // P phase: pred_proj for every utterance, then the next window's joint activations z
+        // =====================================================================================
+        {
+            const int n_tile = p.np;
+            const uint32_t b_bytes = (uint32_t)n_tile * BK * 2;
+            const int32_t* t_new = p.t2 + (size_t)((step + 1) & 1) * p.B;
+            if (warp == 0) {
+                if (lane == 0) {
+                    fence_proxy_async_all();
+                    for (int i = cta; i < p.p_items; i += G) {
+                        const int mt = i / p.hg_count, hg = i - mt * p.hg_count;
+                        for (int kb = 0; kb < p.kb_p; ++kb) {
+                            const int s = ps.it % S;
+                            if (!mbar_wait(&empty_bar[s], ((ps.it / S) & 1) ^ 1, &s_abort)) goto p_done;
+                            uint8_t* a_dst = ring + (size_t)s * p.stage_bytes;
+                            mbar_expect_tx(&full_bar[s], LOOP_A_BYTES + b_bytes);
+                            tma_load_2d(a_dst, &M.hb[pin][p.L - 1], kb * BK, mt * 128, &full_bar[s]);
+                            tma_load_2d(a_dst + LOOP_A_BYTES, &M.w_pred, kb * BK, hg * p.np, &full_bar[s]);
+                            ++ps.it;
+                        }
+                    }
+                }
+            } else if (warp == 1) {
+                if (lane == 0) {
+                    const uint32_t idesc = idesc_bf16(128, n_tile);
+                    for (int i = cta; i < p.p_items; i += G) {
+                        if (!mbar_wait(&acc_empty, (ps.acc & 1) ^ 1, &s_abort)) goto p_done;
+                        tc_fence_after();
+                        for (int kb = 0; kb < p.kb_p; ++kb) {
+                            const int s = ps.it % S;
+                            if (!mbar_wait(&full_bar[s], (ps.it / S) & 1, &s_abort)) goto p_done;
+                            tc_fence_after();
+                            const uint32_t a_addr = smem_u32(ring + (size_t)s * p.stage_bytes);
+                            const uint64_t adesc = smem_desc_sw128(a_addr);
+                            const uint64_t bdesc = smem_desc_sw128(a_addr + LOOP_A_BYTES);
+#pragma unroll
+                            for (int k = 0; k < BK / 16; ++k)
+                                tc_mma_bf16(tmem_base, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+                            tc_commit(&empty_bar[s]);
+                            ++ps.it;
+                        }
+                        tc_commit(&acc_full);
+                        ++ps.acc;
+                    }
+                }
+            } else {
+                // utterances still decoding, counted by every CTA (they all take the same exit)
+                {
+                    int cnt = 0;
+                    for (int b = e; b < p.B; b += 128) cnt += t_new[b] < p.enc_len[b];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+                    if (lane == 0) s_red[warp - 2] = cnt;
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (e == 0) s_active = s_red[0] + s_red[1] + s_red[2] + s_red[3];
+                }
+                for (int i = cta; i < p.p_items; i += G) {
+                    const int mt = i / p.hg_count, hg = i - mt * p.hg_count;
+                    const int b = mt * 128 + row_in_tile;
+                    const int h0 = hg * p.np;
+                    int t = 0, n = 0;
+                    if (b < p.B) {
+                        t = t_new[b];
+                        n = min(p.W, p.enc_len[b] - t);   // <= 0 when the utterance is done
+                    }
+                    const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full, ps.acc & 1, &s_abort));
+                    tc_fence_after();
+                    if (ready) {
+                        for (int c0 = 0; c0 < n_tile; c0 += 16) {
+                            float g[16];
+                            tmem_ld16(tq + (uint32_t)c0, g);
+                            if (b < p.B && n > 0) {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) g[j] += p.b_pred[h0 + c0 + j];
+                                for (int w0 = 0; w0 < p.W; w0 += 4) {
+                                    uint4 ev[4][2];
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) {
+                                        if (w0 + j < n) {
+                                            const uint4* src = reinterpret_cast<const uint4*>(
+                                                p.enc_proj + ((size_t)b * p.T + t + w0 + j) * p.H + h0 + c0);
+                                            ev[j][0] = src[0];
+                                            ev[j][1] = src[1];
+                                        }
+                                    }
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) {
+                                        if (w0 + j < p.W) {
+                                            uint4 o0 = make_uint4(0, 0, 0, 0), o1 = make_uint4(0, 0, 0, 0);
+                                            if (w0 + j < n) {
+                                                const __nv_bfloat162* eb = reinterpret_cast<const __nv_bfloat162*>(&ev[j][0]);
+                                                uint32_t wds[8];
+#pragma unroll
+                                                for (int k = 0; k < 8; ++k) {
+                                                    const float2 e2 = __bfloat1622float2(eb[k]);
+                                                    float z0 = e2.x + g[2 * k], z1 = e2.y + g[2 * k + 1];
+                                                    z0 = p.act == WIND_ACT_RELU ? fmaxf(z0, 0.f) : tanh_fast(z0);
+                                                    z1 = p.act == WIND_ACT_RELU ? fmaxf(z1, 0.f) : tanh_fast(z1);
+                                                    wds[k] = pack_bf16x2(z0, z1);
+                                                }
+                                                o0 = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+                                                o1 = make_uint4(wds[4], wds[5], wds[6], wds[7]);
+                                            }
+                                            uint4* dst = reinterpret_cast<uint4*>(p.z + ((size_t)b * p.W + w0 + j) * p.H + h0 + c0);
+                                            dst[0] = o0;
+                                            dst[1] = o1;
+                                        }
+                                    }
+                                }
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty);
+                    ++ps.acc;
+                    if (!ready) goto p_done;
+                }
+                fence_proxy_async_all();
+            }
+        p_done:
+            if (!grid_sync(2)) goto done;
+        }
+        if (!p.forced && s_active == 0) break;
+        if (!p.forced && step + 1 >= p.step_cap) { exit_status = WIND_ERR_INTERNAL; break; }
+        ++step;
+
+        // =====================================================================================
+        // J phase: window logits on tensor cores, per-row argmax in the epilogue
+        // =====================================================================================
+        {
+            const int n_tile = p.nj;
+            const uint32_t z_bytes = (uint32_t)n_tile * BK * 2;
+            unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
+            if (warp == 0) {
+                if (lane == 0) {
+                    fence_proxy_async_all();
+                    for (int i = cta; i < p.j_items; i += G) {
+                        const int rg = i / p.vt_count, vt = i - rg * p.vt_count;
+                        for (int kb = 0; kb < p.kb_h; ++kb) {
+                            const int s = ps.it % S;
+                            if (!mbar_wait(&empty_bar[s], ((ps.it / S) & 1) ^ 1, &s_abort)) goto j_done;
+                            uint8_t* a_dst = ring + (size_t)s * p.stage_bytes;
+                            if (p.j_stationary) {
+                                mbar_expect_tx(&full_bar[s], z_bytes);
+                                tma_load_2d(a_dst, &M.z, kb * BK, rg * n_tile, &full_bar[s]);
+                            } else {
+                                mbar_expect_tx(&full_bar[s], LOOP_A_BYTES + z_bytes);
+                                tma_load_2d(a_dst, &M.w_out, kb * BK, vt * 128, &full_bar[s]);
+                                tma_load_2d(a_dst + LOOP_A_BYTES, &M.z, kb * BK, rg * n_tile, &full_bar[s]);
+                            }
+                            ++ps.it;
+                        }
+                    }
+                }
+            } else if (warp == 1) {
+                if (lane == 0) {
+                    const uint32_t idesc = idesc_bf16(128, n_tile);
+                    if (p.j_stationary && cta < p.j_items) {
+                        if (!mbar_wait(&stat_bar, 0, &s_abort)) goto j_done;
+                    }
+                    for (int i = cta; i < p.j_items; i += G) {
+                        if (!mbar_wait(&acc_empty, (ps.acc & 1) ^ 1, &s_abort)) goto j_done;
+                        tc_fence_after();
+                        for (int kb = 0; kb < p.kb_h; ++kb) {
+                            const int s = ps.it % S;
+                            if (!mbar_wait(&full_bar[s], (ps.it / S) & 1, &s_abort)) goto j_done;
+                            tc_fence_after();
+                            const uint32_t st_addr = smem_u32(ring + (size_t)s * p.stage_bytes);
+                            const uint64_t adesc = smem_desc_sw128(p.j_stationary ? smem_u32(stat + (size_t)kb * LOOP_A_BYTES) : st_addr);
+                            const uint64_t bdesc = smem_desc_sw128(p.j_stationary ? st_addr : st_addr + LOOP_A_BYTES);
+#pragma unroll
+                            for (int k = 0; k < BK / 16; ++k)
+                                tc_mma_bf16(tmem_base, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+                            tc_commit(&empty_bar[s]);
+                            ++ps.it;
+                        }
+                        tc_commit(&acc_full);
+                        ++ps.acc;
+                    }
+                }
+            } else {
+                const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
+                for (int i = cta; i < p.j_items; i += G) {
+                    const int rg = i / p.vt_count, vt = i - rg * p.vt_count;
+                    const int v = vt * 128 + row_in_tile;            // this thread's vocabulary entry
+                    const bool v_ok = v < p.NV;
+                    const float bias = v_ok ? p.b_out[v] : 0.f;
+                    const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full, ps.acc & 1, &s_abort));
+                    tc_fence_after();
+                    if (ready) {
+                        for (int c0 = 0; c0 < n_tile; c0 += 32) {
+                            float val[32];
+                            tmem_ld16(tq + (uint32_t)c0, val);
+                            if (c0 + 16 < n_tile) {
+                                tmem_ld16(tq + (uint32_t)(c0 + 16), val + 16);
+                            } else {
+#pragma unroll
+                                for (int j = 16; j < 32; ++j) val[j] = -INFINITY;
+                            }
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) val[j] = v_ok ? val[j] + bias : -INFINITY;
+                            const int row = rg * n_tile + c0 + lane;      // the window row whose result this lane ends up with
+                            if (p.logits_out) {
+                                // teacher-forced evaluation: store the logits of the rows inside the window
+                                bool row_ok = false;
+                                if (row < p.rows && c0 + lane < n_tile) {
+                                    const int b = row / p.W, w = row - b * p.W;
+                                    row_ok = t_cur[b] + w < p.enc_len[b];
+                                }
+                                const uint32_t okmask = __ballot_sync(0xffffffffu, row_ok);
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    if (((okmask >> j) & 1u) && v_ok)
+                                        p.logits_out[(size_t)(rg * n_tile + c0 + j) * p.NV + v] = val[j];
+                            } else {
+                                int id[32];
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) id[j] = v;
+                                argmax_exchange<16>(val, id, lane);
+                                argmax_exchange<8>(val, id, lane);
+                                argmax_exchange<4>(val, id, lane);
+                                argmax_exchange<2>(val, id, lane);
+                                argmax_exchange<1>(val, id, lane);
+                                if (row < p.rows && c0 + lane < n_tile && val[0] > -INFINITY)
+                                    atomicMax(&keys_cur[row], pack_key(val[0], (uint32_t)id[0]));
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty);
+                    ++ps.acc;
+                    if (!ready) goto j_done;
+                }
+            }
+        j_done:
+            if (!grid_sync(0)) goto done;
+        }
+        if (p.forced) break;
+    }
+done:
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, LOOP_TMEM_COLS);
+    }
+    if (threadIdx.x == 0) {
+        if (s_abort == 1) set_status(p.ctrl, WIND_ERR_TIMEOUT);
+        if (cta == 0) {
+            if (exit_status) set_status(p.ctrl, exit_status);
+            p.ctrl->active = s_active;
+            for (int k = 0; k < 3; ++k) p.ctrl->phase_cycles[k] = cyc[k];
+            p.ctrl->loop_ns = (long long)(globaltimer_ns() - ns0);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// host side: tile plan, tensor maps, launch
+// ---------------------------------------------------------------------------
+static PFN_cuTensorMapEncodeTiled g_encode_loop = nullptr;
+static std::mutex g_loop_mutex;
+static int g_sm_count[64] = {};
+static int g_smem_optin[64] = {};
+static int g_attr_smem = 0;
+
+static cudaError_t loop_device_info(int* sms, int* smem_optin) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_loop_mutex);
+    if (!g_sm_count[dev]) {
+        int n = 0, sm = 0;
+        if ((e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&sm, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess) return e;
+        g_sm_count[dev] = n;
+        g_smem_optin[dev] = sm;
+    }
+    *sms = g_sm_count[dev];
+    *smem_optin = g_smem_optin[dev];
+    return cudaSuccess;
+}
+
+static cudaError_t get_encode_loop() {
+    std::lock_guard<std::mutex> lock(g_loop_mutex);
+    if (g_encode_loop) return cudaSuccess;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (qres != cudaDriverEntryPointSuccess || !fn) return cudaErrorNotSupported;
+    g_encode_loop = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(fn);
+    return cudaSuccess;
+}
+
+// bf16 matrix [rows, cols] row-major, box = box_rows x 64 columns, 128-byte swizzle, zero fill outside
+static cudaError_t loop_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode_loop(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+// Tile plan: how each phase's GEMM is cut into items (one item = one accumulator), sized so that a
+// phase is one wave over the grid whenever the shapes allow.
+cudaError_t loop_plan(const Call& c, LoopPlan* out) {
+    LoopPlan pl{};
+    int sms = 0, smem_optin = 0;
+    cudaError_t e = loop_device_info(&sms, &smem_optin);
+    if (e != cudaSuccess) return e;
+    const wind_model_t& m = c.m;
+    const int G = sms;
+    const int rows = c.B * c.W;
+    const int NV = m.V + 1;
+    pl.grid = G;
+    pl.kb_h = m.H / BK;
+    pl.kb_p = m.P / BK;
+    // joint: vocabulary tiles of 128 x window-row groups of nj
+    pl.vt_count = (NV + 127) / 128;
+    pl.nj = 256;
+    for (int cand : {16, 32, 64, 96, 128, 160, 192, 224, 256}) {
+        if ((long long)pl.vt_count * ((rows + cand - 1) / cand) <= G) { pl.nj = cand; break; }
+    }
+    pl.rg_count = (rows + pl.nj - 1) / pl.nj;
+    pl.j_items = pl.vt_count * pl.rg_count;
+    // decoder: utterance tiles of 128 x unit groups of ul (4 gates x `slots` rows per item)
+    pl.mt_count = (c.B + 127) / 128;
+    int groups_wanted = G / pl.mt_count;
+    if (groups_wanted < 1) groups_wanted = 1;
+    pl.ul = (m.P + groups_wanted - 1) / groups_wanted;
+    if (pl.ul > 64) pl.ul = 64;
+    pl.slots = 8;
+    while (pl.slots < pl.ul) pl.slots *= 2;
+    pl.ug_count = (m.P + pl.ul - 1) / pl.ul;
+    pl.l_items = pl.mt_count * pl.ug_count;
+    // projection: utterance tiles x H slices of np
+    pl.np = 16;
+    pl.hg_count = m.H / pl.np;
+    pl.p_items = pl.mt_count * pl.hg_count;
+    // shared memory: [stationary W_out tile] [ring of stages]
+    const int budget = smem_optin - 2048;   // static shared memory of the kernel and the 1 KB alignment slack
+    const uint32_t small_ops = (uint32_t)(4 * pl.slots > pl.np ? 4 * pl.slots : pl.np) * BK * 2;
+    const uint32_t stat_bytes = (uint32_t)pl.kb_h * LOOP_A_BYTES;
+    const uint32_t stage_stat = LOOP_A_BYTES + small_ops;
+    pl.j_stationary = pl.j_items <= G && pl.nj <= 128 && (long long)stat_bytes + 3ll * stage_stat + 1024 <= budget;
+    if (pl.j_stationary) {
+        pl.stat_bytes = stat_bytes;
+        pl.stage_bytes = stage_stat;
+    } else {
+        const uint32_t zb = (uint32_t)pl.nj * BK * 2;
+        pl.stat_bytes = 0;
+        pl.stage_bytes = LOOP_A_BYTES + (zb > small_ops ? zb : small_ops);
+    }
+    pl.stage_bytes = (pl.stage_bytes + 1023u) / 1024u * 1024u;
+    int stages = (int)((budget - 1024 - (long long)pl.stat_bytes) / pl.stage_bytes);
+    if (stages > LOOP_MAX_STAGES) stages = LOOP_MAX_STAGES;
+    if (stages < 2) return cudaErrorInvalidConfiguration;
+    pl.stages = stages;
+    pl.smem_bytes = pl.stat_bytes + (uint32_t)stages * pl.stage_bytes + 1024;
+    *out = pl;
+    return cudaSuccess;
+}
+
+static thread_local LoopMaps t_loop_maps;
+static thread_local LoopPlan t_loop_plan;
+
+cudaError_t loop_prepare(Call& c) {
+    cudaError_t e = get_encode_loop();
+    if (e != cudaSuccess) return e;
+    LoopPlan& pl = t_loop_plan;
+    if ((e = loop_plan(c, &pl)) != cudaSuccess) return e;
+    LoopMaps& M = t_loop_maps;
+    const wind_model_t& m = c.m;
+#define WIND_MAP(call_) do { e = (call_); if (e != cudaSuccess) return e; } while (0)
+    WIND_MAP(loop_map(&M.w_out, m.w_out, (uint64_t)m.V + 1, m.H, 128));
+    WIND_MAP(loop_map(&M.z, c.z(), (uint64_t)c.lay.rows_pad, m.H, pl.nj));
+    WIND_MAP(loop_map(&M.w_pred, m.w_pred, m.H, m.P, pl.np));
+    for (int l = 0; l < m.L; ++l) {
+        if (l > 0) WIND_MAP(loop_map(&M.w_ih[l], c.w_ih[l], 4ull * m.P, m.P, pl.slots));
+        WIND_MAP(loop_map(&M.w_hh[l], c.w_hh[l], 4ull * m.P, m.P, pl.slots));
+        for (int par = 0; par < 2; ++par) WIND_MAP(loop_map(&M.hb[par][l], c.hb(par, l), c.lay.Bpad, m.P, 128));
+    }
+#undef WIND_MAP
+    {
+        std::lock_guard<std::mutex> lock(g_loop_mutex);
+        if ((int)pl.smem_bytes > g_attr_smem) {
+            e = cudaFuncSetAttribute(loop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
+            if (e != cudaSuccess) return e;
+            g_attr_smem = (int)pl.smem_bytes;
+        }
+    }
+    return cudaSuccess;
+}
+
+cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* prefix_len, float* logits_out) {
+    const LoopPlan& pl = t_loop_plan;
+    LoopParams p{};
+    p.ctrl = c.ctrl();
+    p.B = c.B; p.T = c.T; p.W = c.W; p.S = c.S; p.max_out = c.max_out;
+    p.H = c.m.H; p.P = c.m.P; p.NV = c.m.V + 1; p.blank = c.m.blank_id; p.act = c.m.act; p.L = c.m.L;
+    p.rows = c.B * c.W; p.rows_pad = c.lay.rows_pad; p.Bpad = c.lay.Bpad;
+    long long cap = (long long)c.T * (c.S + 1) + 2;
+    p.step_cap = cap > 0x7fffffff ? 0x7fffffff : (int)cap;
+    p.nj = pl.nj; p.vt_count = pl.vt_count; p.rg_count = pl.rg_count; p.j_items = pl.j_items; p.j_stationary = pl.j_stationary;
+    p.slots = pl.slots; p.ul = pl.ul; p.ug_count = pl.ug_count; p.mt_count = pl.mt_count; p.l_items = pl.l_items;
+    p.np = pl.np; p.hg_count = pl.hg_count; p.p_items = pl.p_items;
+    p.kb_h = pl.kb_h; p.kb_p = pl.kb_p;
+    p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.stat_bytes = pl.stat_bytes;
+    p.enc_len = c.enc_len; p.t2 = c.t(); p.count = c.count(); p.emit_tok = c.emit_tok(); p.keys2 = c.keys();
+    p.out_tokens = c.out_tokens; p.out_frames = c.out_frames; p.out_len = c.out_len;
+    p.c_state = c.c(); p.hb = c.hb(0, 0); p.z = c.z(); p.enc_proj = (const __nv_bfloat16*)c.enc_proj(); p.g0 = c.g0();
+    for (int l = 0; l < c.m.L; ++l) { p.b_ih[l] = c.b_ih[l]; p.b_hh[l] = c.b_hh[l]; }
+    p.b_pred = c.m.b_pred; p.b_out = c.m.b_out;
+    p.forced = logits_out != nullptr; p.prefix = prefix; p.U = U; p.prefix_len = prefix_len; p.logits_out = logits_out;
+    void* args[2] = {(void*)&t_loop_maps, (void*)&p};
+    return cudaLaunchCooperativeKernel((const void*)loop_kernel, dim3((unsigned)pl.grid), dim3(LOOP_THREADS), args, pl.smem_bytes,
+                                       c.stream);
+}
+
+}  // namespace wind

@@ -1,0 +1,72 @@
+// Parameter blocks of the persistent decoding-loop kernel.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "wind_internal.cuh"
+
+namespace wind {
+
+// Tensor maps of one call; all bf16, 64-column boxes, 128-byte swizzle.
+struct LoopMaps {
+    CUtensorMap w_out;                 // [V+1, H], box 128 rows
+    CUtensorMap z;                     // [rows_pad, H], box nj rows
+    CUtensorMap w_pred;                // [H, P], box np rows
+    CUtensorMap w_ih[kMaxLayers];      // [4P, P], box `slots` rows (layers > 0)
+    CUtensorMap w_hh[kMaxLayers];      // [4P, P], box `slots` rows
+    CUtensorMap hb[2][kMaxLayers];     // [Bpad, P], box 128 rows
+};
+
+// How the three phases are cut into items and how shared memory is used (host-chosen).
+struct LoopPlan {
+    int grid;
+    int kb_h, kb_p;                        // K blocks of 64 in H and in P
+    int nj, vt_count, rg_count, j_items;   // joint: window rows per item, vocabulary tiles, row groups
+    int j_stationary;                      // every CTA owns one joint item: its W_out tile stays in shared memory
+    int slots, ul, ug_count, mt_count, l_items;  // decoder: rows per gate block, units per item, unit groups, utterance tiles
+    int np, hg_count, p_items;             // projection: H columns per item, H slices
+    int stages;
+    uint32_t stage_bytes, stat_bytes, smem_bytes;
+};
+
+struct LoopParams {
+    Ctrl* ctrl;
+    int B, T, W, S, max_out, H, P, NV, blank, act, L;
+    int rows, rows_pad, Bpad, step_cap;
+    int nj, vt_count, rg_count, j_items, j_stationary;
+    int slots, ul, ug_count, mt_count, l_items;
+    int np, hg_count, p_items;
+    int kb_h, kb_p;
+    int stages;
+    uint32_t stage_bytes, stat_bytes;
+    const int32_t* enc_len;
+    int32_t* t2;                   // [2][B]
+    int32_t* count;                // [B]
+    int32_t* emit_tok;             // [B]
+    unsigned long long* keys2;     // [2][rows_pad]
+    int32_t* out_tokens;
+    int32_t* out_frames;
+    int32_t* out_len;
+    float* c_state;                // [L][B][P]
+    __nv_bfloat16* hb;             // [2][L][Bpad][P]
+    __nv_bfloat16* z;              // [rows_pad][H]
+    const __nv_bfloat16* enc_proj; // [B*T][H]
+    const float* g0;               // [V+1][4P]
+    const float* b_ih[kMaxLayers];
+    const float* b_hh[kMaxLayers];
+    const float* b_pred;
+    const float* b_out;
+    // teacher forcing (wind_eval_joint_window): feed prefix tokens, then store the window logits
+    int forced;
+    const int32_t* prefix;
+    int U;
+    const int32_t* prefix_len;
+    float* logits_out;
+};
+
+cudaError_t loop_plan(const Call& c, LoopPlan* out);
+cudaError_t loop_prepare(Call& c);   // plan + tensor maps + shared-memory opt-in (host only; not inside a capture)
+
+}  // namespace wind

@@ -40,20 +40,22 @@ def test_status_strings(lib):
     assert pkg.wind_status_string(99) == "WIND_ERR_UNKNOWN"
 
 
-def test_workspace_grows_with_window_only_by_the_key_array(lib):
+def test_workspace_grows_with_window_only_by_keys_and_activations(lib):
     # The paper's memory analysis: WIND's only extra state is the window's logits,
     # W x (V+1) floats per utterance (16 x 1025 = 16400 floats for W = 16).  Here the
-    # logits stay on chip and only an 8-byte argmax key per window row is kept.
+    # logits stay on chip; per window row the workspace keeps two 8-byte argmax keys (double
+    # buffered by step parity) and the joint's H bf16 activations.
     m = large_model()
     B, T = 128, 2500
-    base = pkg.wind_workspace_bytes(m, B, T, 1)
-    for W in (2, 4, 8, 16, 64):
+    base = pkg.wind_workspace_bytes(m, B, T, 2)   # B * W = 256 rows: no row padding at even W
+    for W in (4, 8, 16, 64):
         extra = pkg.wind_workspace_bytes(m, B, T, W) - base
-        assert extra == 8 * B * (W - 1)
-        assert extra <= 4 * B * W * (m.V + 1)  # far below the paper's W x (V+1) floats per utterance
+        assert extra == B * (W - 2) * (2 * 8 + 2 * m.H)
+        assert extra <= 4 * B * W * (m.V + 1)  # below the paper's W x (V+1) floats per utterance
     assert 16 * 1025 == 16400
-    # dominated by enc_proj [B, T, H] in bf16
-    assert base >= 2 * B * T * m.H and base < 2 * B * T * m.H * 1.02 + (1 << 22)
+    # dominated by enc_proj [B, T, H] in bf16; the gate table adds (V+1) x 4P floats
+    table = 4 * (m.V + 1) * 4 * m.P
+    assert base >= 2 * B * T * m.H + table and base < 2 * B * T * m.H * 1.02 + table + (1 << 22)
 
 
 def test_invalid_arguments_are_rejected_on_the_host(lib):
