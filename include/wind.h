@@ -220,6 +220,27 @@ wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const 
 /* Copies the counters of the last decode that used `workspace` to host memory (synchronises `stream`). */
 wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t* host_out);
 
+/*
+ * Timeline of the persistent loop kernel (tensor-core path), a debugging and measurement aid.
+ * wind_set_trace(s) makes later decodes record, for lock steps s and s + 1 (s = -1 is the start of
+ * sequence), when the role threads of CTA 0 pass fixed points of each phase; s < -1 switches it off
+ * (default).  Returns the previous setting.  Recording costs a few stores and does not change results.
+ * wind_read_trace copies the records of the last decode that used `workspace` (same m, B, T, W).
+ *   role:  0 TMA issuer, 1 MMA issuer, 2 first epilogue thread, 3 grid barrier
+ *   phase: 0 joint, 1 decoder update, 2 projection
+ *   event: 0 phase entered, 1 first / 2 last TMA issued, 3 first operands arrived, 4 accumulator
+ *          committed, 5 epilogue inputs requested (token known), 6 accumulator ready, 7 epilogue
+ *          done, 8 barrier arrival, 9 barrier release
+ *   clock: SM cycle counter of CTA 0's SM
+ */
+typedef struct {
+    int32_t role, phase, event, step;
+    int64_t clock;
+} wind_trace_event_t;
+int32_t wind_set_trace(int32_t first_step);
+wind_status_t wind_read_trace(const wind_model_t* m, int32_t B, int32_t T, int32_t W, const void* workspace, void* stream,
+                              wind_trace_event_t* host_out, int32_t capacity, int32_t* n_out);
+
 /* Process-wide choice of kernels for the bf16 path (default AUTO).  Returns the previous value. */
 int32_t wind_set_kernels(int32_t kernels);
 

@@ -30,7 +30,7 @@ WIND_KERNELS_AUTO, WIND_KERNELS_SIMT, WIND_KERNELS_TENSOR = 0, 1, 2
 
 EXPORTS = [
     "wind_workspace_bytes", "wind_decode_greedy", "wind_host_staging_bytes", "wind_decode_greedy_host",
-    "wind_eval_joint_window", "wind_eval_joint_window_static", "wind_profile_decode", "wind_read_stats", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
+    "wind_eval_joint_window", "wind_eval_joint_window_static", "wind_profile_decode", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
 ]
 
 _vp = C.c_void_p
@@ -68,6 +68,10 @@ class wind_profile_t(C.Structure):
     ]
 
 
+class wind_trace_event_t(C.Structure):
+    _fields_ = [("role", C.c_int32), ("phase", C.c_int32), ("event", C.c_int32), ("step", C.c_int32), ("clock", C.c_int64)]
+
+
 _lib = None
 
 
@@ -100,6 +104,10 @@ def load_library():
     L.wind_eval_joint_window_static.restype = i32
     L.wind_read_stats.argtypes = [_vp, _vp, C.POINTER(wind_stats_t)]
     L.wind_read_stats.restype = i32
+    L.wind_set_trace.argtypes = [i32]
+    L.wind_set_trace.restype = i32
+    L.wind_read_trace.argtypes = [mp, i32, i32, i32, _vp, _vp, C.POINTER(wind_trace_event_t), i32, C.POINTER(i32)]
+    L.wind_read_trace.restype = i32
     L.wind_set_kernels.argtypes = [i32]
     L.wind_set_kernels.restype = i32
     L.wind_status_string.argtypes = [i32]
@@ -122,6 +130,22 @@ class WindError(RuntimeError):
 
 def wind_status_string(status: int) -> str:
     return load_library().wind_status_string(status).decode()
+
+
+def wind_set_trace(first_step: int) -> int:
+    """Record the loop kernel's timeline for lock steps first_step and first_step + 1 (< -1: off)."""
+    return load_library().wind_set_trace(first_step)
+
+
+def wind_read_trace(model: "WindModel", B: int, T: int, W: int, workspace, stream=None) -> List[Dict[str, int]]:
+    L = load_library()
+    cap = 4 * 512
+    buf = (wind_trace_event_t * cap)()
+    n = C.c_int32(0)
+    st = L.wind_read_trace(model.ref, B, T, W, _ws_ptr(workspace), _stream_ptr(stream), buf, cap, C.byref(n))
+    if st != WIND_OK:
+        raise WindError(st)
+    return [dict(role=e.role, phase=e.phase, event=e.event, step=e.step, clock=e.clock) for e in buf[: n.value]]
 
 
 def wind_set_kernels(kernels: int) -> int:

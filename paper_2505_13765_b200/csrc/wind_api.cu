@@ -12,6 +12,7 @@ namespace wind {
 
 static thread_local char g_cuda_err[256] = "";
 static int g_kernels = WIND_KERNELS_AUTO;
+static int g_trace_step = -2;   // first lock step of the loop kernel's timeline window; -2 = off
 
 static wind_status_t cuda_fail(cudaError_t e, const char* where) {
     snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", where, cudaGetErrorString(e));
@@ -173,7 +174,7 @@ static wind_status_t enqueue_decode(Call& c) {
         WIND_CUDA(launch_init(c, WIND_KERNELS_TENSOR, 0, tc_setup_launches(c)));
         WIND_CUDA(tc_enc_proj(c));
         WIND_CUDA(tc_gate_table(c));
-        WIND_CUDA(tc_loop(c, nullptr, 0, nullptr, nullptr));
+        WIND_CUDA(tc_loop(c, nullptr, 0, nullptr, nullptr, g_trace_step));
         return WIND_OK;
     }
     const int per_step = 2 + simt_pred_launches(c);
@@ -319,7 +320,7 @@ wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, con
         WIND_CUDA(tc_enc_proj(c));
         WIND_CUDA(tc_gate_table(c));
         WIND_CUDA(launch_set_t(c, t0));
-        WIND_CUDA(tc_loop(c, prefix, U, prefix_len, logits));
+        WIND_CUDA(tc_loop(c, prefix, U, prefix_len, logits, -2));
         return read_status(c);
     }
     WIND_CUDA(launch_init(c, WIND_KERNELS_SIMT, 0, 0));
@@ -395,7 +396,7 @@ wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const 
         WIND_CUDA(tc_enc_proj(c));
         WIND_CUDA(cudaEventRecord(e1, c.stream));
         WIND_CUDA(tc_gate_table(c));
-        WIND_CUDA(tc_loop(c, nullptr, 0, nullptr, nullptr));
+        WIND_CUDA(tc_loop(c, nullptr, 0, nullptr, nullptr, g_trace_step));
         Ctrl hc;
         WIND_CUDA(cudaMemcpyAsync(&hc, c.ctrl(), sizeof(Ctrl), cudaMemcpyDeviceToHost, c.stream));
         WIND_CUDA(cudaStreamSynchronize(c.stream));
@@ -484,6 +485,42 @@ wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t*
     host_out->launches_per_step = hc.launches_per_step;
     host_out->launches_setup = hc.launches_setup;
     host_out->kernels = hc.kernels;
+    return WIND_OK;
+}
+
+int32_t wind_set_trace(int32_t first_step) {
+    int32_t prev = g_trace_step;
+    g_trace_step = first_step < -1 ? -2 : first_step;
+    return prev;
+}
+
+wind_status_t wind_read_trace(const wind_model_t* m, int32_t B, int32_t T, int32_t W, const void* workspace, void* stream,
+                              wind_trace_event_t* host_out, int32_t capacity, int32_t* n_out) {
+    wind_status_t s = check_model(m);
+    if (s != WIND_OK) return s;
+    s = check_shape(m, B, T, W);
+    if (s != WIND_OK) return s;
+    if (!workspace || !host_out || !n_out || capacity < 0) return WIND_ERR_INVALID_ARG;
+    *n_out = 0;
+    if (m->dtype != WIND_DT_BF16) return WIND_OK;
+    Layout lay = make_layout(*m, B, T, W, 1);
+    std::vector<TraceEvent> ev((size_t)kTraceRoles * kTraceEvents);
+    WIND_CUDA(cudaMemcpyAsync(ev.data(), static_cast<const uint8_t*>(workspace) + lay.trace, ev.size() * sizeof(TraceEvent),
+                              cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    WIND_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    int n = 0;
+    for (int r = 0; r < kTraceRoles; ++r)
+        for (int k = 0; k < kTraceEvents; ++k) {
+            const TraceEvent& t = ev[(size_t)r * kTraceEvents + k];
+            if (t.clock == 0 || n >= capacity) continue;
+            host_out[n].role = r;
+            host_out[n].phase = (int32_t)(t.tag / 16);
+            host_out[n].event = (int32_t)(t.tag % 16);
+            host_out[n].step = t.step;
+            host_out[n].clock = t.clock;
+            ++n;
+        }
+    *n_out = n;
     return WIND_OK;
 }
 

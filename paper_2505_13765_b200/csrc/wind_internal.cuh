@@ -14,6 +14,15 @@ constexpr int kMaxLayers = 8;
 constexpr int kMaxWindow = 64;
 constexpr size_t kAlign = 256;
 
+// Timeline of the loop kernel (debug aid, off unless a step window is set): one record per event.
+struct TraceEvent {
+    uint32_t tag;      // phase * 16 + event
+    int32_t step;
+    long long clock;   // clock64 of the SM that runs CTA 0
+};
+constexpr int kTraceRoles = 4;     // TMA issuer, MMA issuer, first epilogue thread, barrier
+constexpr int kTraceEvents = 512;
+
 // Device control block, first thing in the workspace.
 struct Ctrl {
     int32_t status;   // wind_status_t, sticky (first error wins)
@@ -49,6 +58,7 @@ struct Layout {
     size_t hb;         // bf16 [2][L][Bpad][P] LSTM hidden state as tensor-core operand rows (tensor path)
     size_t z;          // bf16 [rows_pad][H] joint activations act(enc_proj + pred_proj), the joint GEMM's operand (tensor path)
     size_t g0;         // fp32 [V+1][4P] layer-0 gate pre-activations of every token: W_ih emb[tok] + b_ih + b_hh (tensor path)
+    size_t trace;      // TraceEvent [kTraceRoles][kTraceEvents]: optional timeline of CTA 0 of the loop kernel
     size_t enc_proj;   // elem [B*T][H]
     size_t total;
     // host staging (wind_decode_greedy_host), placed after `total`
@@ -78,6 +88,7 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     L.hb = take(bf ? 2 * (size_t)m.L * L.Bpad * m.P * 2 : 0);
     L.z = take(bf ? (size_t)L.rows_pad * m.H * 2 : 0);
     L.g0 = take(bf ? sizeof(float) * (size_t)(m.V + 1) * 4 * m.P : 0);
+    L.trace = take(bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents : 0);
     L.enc_proj = take(es * (size_t)B * T * m.H);
     L.total = off;
     L.st_enc = take(es * (size_t)B * T * m.D);
@@ -120,6 +131,7 @@ struct Call {
     void* enc_proj() const { return ws + lay.enc_proj; }
     __nv_bfloat16* z() const { return reinterpret_cast<__nv_bfloat16*>(ws + lay.z); }
     float* g0() const { return reinterpret_cast<float*>(ws + lay.g0); }
+    TraceEvent* trace() const { return reinterpret_cast<TraceEvent*>(ws + lay.trace); }
     __nv_bfloat16* hb(int parity, int l) const {
         return reinterpret_cast<__nv_bfloat16*>(ws + lay.hb) + ((size_t)parity * m.L + l) * lay.Bpad * m.P;
     }
@@ -164,7 +176,8 @@ cudaError_t tc_gate_table(const Call& c);  // g0[tok] = W_ih[0] emb[tok] + b_ih[
 // The whole decoding loop as one persistent cooperative kernel.  prefix == nullptr: greedy
 // decoding until every utterance is done.  Otherwise teacher forcing: feed prefix tokens, then
 // store the window logits at t (set beforehand in both t buffers) to logits_out.
-cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* prefix_len, float* logits_out);
+cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* prefix_len, float* logits_out,
+                    int trace_step);
 int tc_setup_launches(const Call& c);
 
 }  // namespace wind

@@ -28,6 +28,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <cstdlib>
 #include <mutex>
 
 #include "wind_internal.cuh"
@@ -37,7 +38,7 @@
 namespace wind {
 
 constexpr int LOOP_THREADS = 192;
-constexpr int LOOP_MAX_STAGES = 12;
+constexpr int LOOP_MAX_STAGES = 28;
 constexpr uint32_t LOOP_A_BYTES = 128 * BK * 2;  // one K block of a 128-row operand tile
 constexpr uint32_t LOOP_TMEM_COLS = 512;
 
@@ -85,14 +86,46 @@ __device__ __forceinline__ void argmax_exchange(float* v, int* id, int lane) {
     }
 }
 
-struct PipeState {
-    uint32_t it;    // K blocks pushed (producer) or consumed (MMA issuer) so far, over the whole kernel
-    uint32_t acc;   // accumulator uses so far (MMA issuer and epilogue count the same items)
-};
+// Timeline record of CTA 0 (one of the role threads calls this; n is that thread's event counter).
+__device__ __forceinline__ void trace_event(const LoopParams& p, int role, int& n, int step, int phase, int ev) {
+    if (p.trace && blockIdx.x == 0 && step >= p.trace_step && step < p.trace_step + 2 && n < kTraceEvents) {
+        TraceEvent t;
+        t.tag = (uint32_t)(phase * 16 + ev);
+        t.step = step;
+        t.clock = clock64();
+        p.trace[role * kTraceEvents + n] = t;
+        ++n;
+    }
+}
+enum { TR_J = 0, TR_L = 1, TR_P = 2 };
+enum { EV_START = 0, EV_FIRST_ISSUE = 1, EV_LAST_ISSUE = 2, EV_FIRST_DATA = 3, EV_COMMIT = 4, EV_TOK = 5, EV_ACC = 6, EV_EPI_DONE = 7,
+       EV_ARRIVE = 8, EV_RELEASE = 9 };
+
+// 32 lanes x 16 consecutive columns, registers -> tensor memory
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+        "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// D[tmem] (+)= A[tmem] * B[smem]^T: A rows on lanes, two bf16 K elements per 32-bit column
+__device__ __forceinline__ void tc_mma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+enum { J_STREAM = 0, J_SMEM = 1, J_TMEM = 2 };   // where the joint's W_out tile lives
 
 __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_constant__ LoopMaps M, const LoopParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[LOOP_MAX_STAGES], empty_bar[LOOP_MAX_STAGES], stat_bar, acc_full, acc_empty;
+    __shared__ uint64_t full_bar[LOOP_MAX_STAGES], empty_bar[LOOP_MAX_STAGES], stat_bar;
+    __shared__ uint64_t acc_full[3], acc_empty[3];   // accumulators: joint, decoder, projection
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;      // this CTA has given up
     __shared__ int s_active;     // utterances still decoding (set in the projection phase)
@@ -101,20 +134,21 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cta = blockIdx.x, G = gridDim.x;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t* stat = smem;                       // stationary W_out tile: kb_h blocks of 128 x 64 bf16
-    uint8_t* ring = smem + p.stat_bytes;        // stages of [128-row operand block | small operand block]
-    const int S = p.stages;
+    uint8_t* stat = smem;                       // W_out tile kept in shared memory (J_SMEM): kb_h blocks of 128 x 64 bf16
+    uint8_t* ring = smem + p.stat_bytes;        // operand stages; geometry differs per phase, drained in between
 
     if (threadIdx.x == 0) {
         s_abort = 0;
         s_active = 0;
-        for (int s = 0; s < S; ++s) {
+        for (int s = 0; s < LOOP_MAX_STAGES; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
         mbar_init(&stat_bar, 1);
-        mbar_init(&acc_full, 1);
-        mbar_init(&acc_empty, 4);
+        for (int k = 0; k < 3; ++k) {
+            mbar_init(&acc_full[k], 1);
+            mbar_init(&acc_empty[k], 4);
+        }
         fence_barrier_init();
     }
     if (warp == 1) tmem_alloc(&tmem_slot, LOOP_TMEM_COLS);
@@ -122,28 +156,65 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
+    const uint32_t tm_j = tmem_base + (uint32_t)p.tm_j, tm_l = tmem_base + (uint32_t)p.tm_l, tm_p = tmem_base + (uint32_t)p.tm_p;
 
-    if (p.j_stationary && cta < p.j_items && threadIdx.x == 0) {
-        const int vt = cta % p.vt_count;
+    const int e = threadIdx.x - 64;            // epilogue thread 0..127 (warps 2..5)
+    const int q = warp & 3;                    // tensor-memory lane quadrant of this warp
+    const int row_in_tile = q * 32 + lane;     // the tensor-memory lane (accumulator row) of this thread
+    const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+    const bool has_j = cta < p.j_items;
+    const int my_vt = cta % p.vt_count;        // vocabulary tile of this CTA's joint item when it has exactly one
+
+    // ----- the joint's W_out tile, loaded once when every CTA owns one joint item -----
+    if (p.j_mode == J_SMEM && has_j && threadIdx.x == 0) {
         mbar_expect_tx(&stat_bar, (uint32_t)p.kb_h * LOOP_A_BYTES);
-        for (int kb = 0; kb < p.kb_h; ++kb) tma_load_2d(stat + (size_t)kb * LOOP_A_BYTES, &M.w_out, kb * BK, vt * 128, &stat_bar);
+        for (int kb = 0; kb < p.kb_h; ++kb) tma_load_2d(stat + (size_t)kb * LOOP_A_BYTES, &M.w_out, kb * BK, my_vt * 128, &stat_bar);
+    }
+    if (p.j_mode == J_TMEM) {
+        if (warp >= 2 && has_j) {
+            // tensor memory, lane = vocabulary entry, 32-bit column j = W_out[v, 2j], W_out[v, 2j + 1]
+            const int v = my_vt * 128 + row_in_tile;
+            const uint4* src = reinterpret_cast<const uint4*>(p.w_out + (size_t)(v < p.NV ? v : 0) * p.H);
+            for (int c0 = 0; c0 < p.H / 2; c0 += 16) {
+                uint32_t r[16];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint4 x = v < p.NV ? src[c0 / 4 + j] : make_uint4(0, 0, 0, 0);
+                    r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
+                }
+                tmem_st16(tmem_base + lane_off + (uint32_t)c0, r);
+            }
+            tmem_st_wait();
+        }
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
     }
 
-    PipeState ps{0u, 0u};
-    uint32_t epoch = 0;          // grid barrier target (thread 0)
-    int step = -1;               // -1: start of sequence
-    int pin = 0;                 // hb[pin] holds the current decoder state
+    // ----- pipeline state of the role threads -----
+    uint32_t pe_bits = 0xffffffffu;   // TMA issuer: parity to wait for on empty_bar[s]
+    uint32_t cf_bits = 0u;            // MMA issuer: parity to wait for on full_bar[s]
+    uint32_t acc_n[3] = {0u, 0u, 0u}; // uses of each accumulator so far (MMA issuer and epilogue threads count alike)
+    int cur = 0;                      // stage cursor, reset whenever the ring has drained
+    uint32_t epoch = 0;               // grid barrier target (thread 0)
+    int step = -1;                    // -1: start of sequence
+    int pin = 0;                      // hb[pin] holds the current decoder state
     long long clk_last = 0, cyc[3] = {0, 0, 0};
     unsigned long long ns0 = 0;
     if (cta == 0 && threadIdx.x == 0) { clk_last = clock64(); ns0 = globaltimer_ns(); }
     int exit_status = 0;
+    int tr_n = 0;                     // trace events written by this thread
+    const bool early = p.l_early != 0;   // layer 0's GEMM is issued one phase ahead of its cell update
 
-    // ----- helpers -------------------------------------------------------------------------
+    const uint32_t sb_lp = p.stage_lp, sb_j = p.stage_j;   // stage bytes of the decoder/projection phases and of the joint phase
+    const int S_lp = p.stages_lp, S_j = p.stages_j;
+
     // Grid barrier for all threads of all CTAs; false when the kernel is being abandoned.
     auto grid_sync = [&](int phase_kind) -> bool {
         __syncthreads();
         if (threadIdx.x == 0) {
             epoch += (uint32_t)G;
+            trace_event(p, 3, tr_n, step, phase_kind, EV_ARRIVE);
             if (s_abort) {
                 atomicExch(&p.ctrl->abort, 1);
             } else {
@@ -161,6 +232,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                 }
                 __threadfence();
             }
+            trace_event(p, 3, tr_n, step, phase_kind, EV_RELEASE);
             if (cta == 0) {
                 const long long now = clock64();
                 cyc[phase_kind] += now - clk_last;
@@ -171,249 +243,313 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         return s_abort == 0;
     };
 
-    const int e = threadIdx.x - 64;            // epilogue thread 0..127 (warps 2..5)
-    const int q = warp & 3;                    // tensor-memory lane quadrant of this warp
-    const int row_in_tile = q * 32 + lane;     // the tensor-memory lane (accumulator row) of this thread
-    const uint32_t tq = tmem_base + ((uint32_t)(q * 32) << 16);
+    // ----- TMA issuer (warp 0, lane 0) -----
+    auto acquire = [&](uint32_t sb) -> uint8_t* {   // next free stage, nullptr when giving up
+        if (!mbar_wait(&empty_bar[cur], (pe_bits >> cur) & 1u, &s_abort)) return nullptr;
+        pe_bits ^= 1u << cur;
+        return ring + (size_t)cur * sb;
+    };
+    // decoder GEMM operands of layer l for this CTA's items
+    auto produce_L = [&](int l) -> bool {
+        const uint32_t b_bytes = (uint32_t)(4 * p.slots) * BK * 2;
+        const int segs = l == 0 ? 1 : 2;
+        for (int i = cta; i < p.l_items; i += G) {
+            const int mt = i / p.ug_count, ug = i - mt * p.ug_count;
+            for (int sg = 0; sg < segs; ++sg) {
+                const CUtensorMap* ma = (l == 0 || sg == 1) ? &M.hb[pin][l] : &M.hb[pin ^ 1][l - 1];
+                const CUtensorMap* mb = (l == 0 || sg == 1) ? &M.w_hh[l] : &M.w_ih[l];
+                for (int kb = 0; kb < p.kb_p; ++kb) {
+                    uint8_t* a_dst = acquire(sb_lp);
+                    if (!a_dst) return false;
+                    uint8_t* b_dst = a_dst + LOOP_A_BYTES;
+                    mbar_expect_tx(&full_bar[cur], LOOP_A_BYTES + b_bytes);
+                    tma_load_2d(a_dst, ma, kb * BK, mt * 128, &full_bar[cur]);
+                    for (int g = 0; g < 4; ++g)
+                        tma_load_2d(b_dst + (size_t)g * p.slots * 128, mb, kb * BK, g * p.P + ug * p.ul, &full_bar[cur]);
+                    cur = cur + 1 == S_lp ? 0 : cur + 1;
+                }
+            }
+        }
+        return true;
+    };
+    // ----- MMA issuer (warp 1, lane 0) -----
+    auto consume = [&]() -> bool {
+        if (!mbar_wait(&full_bar[cur], (cf_bits >> cur) & 1u, &s_abort)) return false;
+        cf_bits ^= 1u << cur;
+        tc_fence_after();
+        return true;
+    };
+    auto begin_acc = [&](int k) -> bool {   // the epilogue has drained the previous use of accumulator k
+        if (!mbar_wait(&acc_empty[k], (acc_n[k] & 1u) ^ 1u, &s_abort)) return false;
+        tc_fence_after();
+        return true;
+    };
+    auto mma_L = [&](int l) -> bool {
+        const uint32_t idesc = idesc_bf16(128, 4 * p.slots);
+        const int kbs = (l == 0 ? 1 : 2) * p.kb_p;
+        for (int i = cta; i < p.l_items; i += G) {
+            if (!begin_acc(1)) return false;
+            for (int kb = 0; kb < kbs; ++kb) {
+                if (!consume()) return false;
+                const uint32_t a_addr = smem_u32(ring + (size_t)cur * sb_lp);
+                const uint64_t adesc = smem_desc_sw128(a_addr);
+                const uint64_t bdesc = smem_desc_sw128(a_addr + LOOP_A_BYTES);
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)
+                    tc_mma_bf16(tm_l, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+                tc_commit(&empty_bar[cur]);
+                cur = cur + 1 == S_lp ? 0 : cur + 1;
+            }
+            tc_commit(&acc_full[1]);
+            ++acc_n[1];
+        }
+        return true;
+    };
+    // ----- epilogue of the decoder phase of layer l: control step (layer 0 while decoding) + LSTM cell update -----
+    auto epilogue_L = [&](int l) -> bool {
+        const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
+        int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
+        const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
+        unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
+        for (int i = cta; i < p.l_items; i += G) {
+            const int mt = i / p.ug_count, ug = i - mt * p.ug_count;
+            const int b = mt * 128 + row_in_tile;
+            const bool in = b < p.B;
+            const int bb = in ? b : 0;
+            float* cst = p.c_state + ((size_t)l * p.B + bb) * p.P;
+            const __nv_bfloat16* hin = p.hb + (((size_t)pin * p.L + l) * p.Bpad + bb) * p.P;
+            __nv_bfloat16* hout = p.hb + (((size_t)(pin ^ 1) * p.L + l) * p.Bpad + bb) * p.P;
+            const int unit0 = ug * p.ul;
+            // ---- which token does utterance b feed to its decoder in this step? ----
+            int tok = -1;
+            if (in) {
+                if (step < 0) {
+                    tok = p.blank;
+                } else if (p.forced) {
+                    tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
+                } else if (l > 0) {
+                    tok = p.emit_tok[b];
+                } else {
+                    // control step (Algorithm 2's branch): first non-blank row of the window.
+                    // Everything it needs is requested at once; the keys of all W rows are readable.
+                    int t = t_cur[b];
+                    const int len = p.enc_len[b];
+                    const bool writer = ug == 0;
+                    int cnt = 0, pos = 0;
+                    if (writer) { cnt = p.count[b]; pos = p.out_len[b]; }
+                    unsigned long long kk[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) kk[j] = j < p.W ? keys_cur[(size_t)b * p.W + j] : 0ull;
+                    if (t < len) {
+                        const int n = min(p.W, len - t);
+                        int first = -1, label = p.blank;
+                        bool bad = false;
+                        for (int w0 = 0; w0 < n && first < 0; w0 += 8) {
+                            if (w0 > 0) {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) kk[j] = (w0 + j < n) ? keys_cur[(size_t)b * p.W + w0 + j] : 0ull;
+                            }
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                if (w0 + j < n && first < 0) {
+                                    uint32_t lab = key_label(kk[j]);
+                                    if (kk[j] == 0ull || lab >= (uint32_t)p.NV) { bad = true; lab = (uint32_t)p.blank; }
+                                    if ((int)lab != p.blank) { first = w0 + j; label = (int)lab; }
+                                }
+                            }
+                        }
+                        if (first >= 0) tok = label;
+                        if (writer) {
+                            // this CTA records the step for its utterances
+                            int jump, forced = 0, emitted = 0;
+                            if (first < 0) {
+                                jump = n;
+                                t += n;
+                                cnt = 0;
+                            } else {
+                                jump = first;
+                                if (first > 0) cnt = 0;
+                                t += first;
+                                if (pos < p.max_out) {
+                                    p.out_tokens[(size_t)b * p.max_out + pos] = label;
+                                    p.out_frames[(size_t)b * p.max_out + pos] = t;
+                                    p.out_len[b] = pos + 1;
+                                    emitted = 1;
+                                    cnt += 1;
+                                    if (cnt == p.S) { t += 1; cnt = 0; forced = 1; }
+                                } else {
+                                    set_status(p.ctrl, WIND_ERR_OUTPUT_OVERFLOW);  // this utterance stops here
+                                    t = len;
+                                    tok = -1;
+                                }
+                            }
+                            if (bad) set_status(p.ctrl, WIND_ERR_INTERNAL);
+                            t_nxt[b] = t;
+                            p.count[b] = cnt;
+                            for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
+                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
+                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->joint_rows), (unsigned long long)n);
+                            if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
+                            if (forced) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
+                        }
+                    } else if (writer) {
+                        t_nxt[b] = t;
+                    }
+                    if (writer) p.emit_tok[b] = tok;
+                }
+            }
+            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
+            const bool live = in && tok >= 0;
+            // what the cell update needs from memory, requested before the accumulator is waited for
+            float add[4][8], cold[8];
+            auto load_operands = [&](int u0) {
+                if (live) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int unit = unit0 + u0 + j;
+                        const bool ok = u0 + j < p.ul && unit < p.P;
+                        cold[j] = ok ? cst[unit] : 0.f;
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            if (l == 0) add[g][j] = ok ? p.g0[(size_t)tok * 4 * p.P + (size_t)g * p.P + unit] : 0.f;
+                            else add[g][j] = ok ? p.b_ih[l][g * p.P + unit] + p.b_hh[l][g * p.P + unit] : 0.f;
+                        }
+                    }
+                }
+            };
+            load_operands(0);
+            const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, &s_abort));
+            tc_fence_after();
+            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
+            if (ready) {
+                for (int u0 = 0; u0 < p.ul; u0 += 8) {
+                    if (u0 > 0) load_operands(u0);
+                    float pre[4][8];
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) tmem_ld8(tm_l + lane_off + (uint32_t)(g * p.slots + u0), pre[g]);
+                    if (in) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const int unit = unit0 + u0 + j;
+                            if (u0 + j < p.ul && unit < p.P) {
+                                if (live) {
+                                    const float gi = sigmoid_f(pre[0][j] + add[0][j]);
+                                    const float gf = sigmoid_f(pre[1][j] + add[1][j]);
+                                    const float gg = tanhf(pre[2][j] + add[2][j]);
+                                    const float go = sigmoid_f(pre[3][j] + add[3][j]);
+                                    const float cc = gf * cold[j] + gi * gg;
+                                    cst[unit] = cc;
+                                    hout[unit] = __float2bfloat16_rn(go * tanhf(cc));
+                                } else {
+                                    hout[unit] = hin[unit];
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[1]);
+            ++acc_n[1];
+            if (!ready) return false;
+        }
+        if (cta == 0 && e == 0 && l == 0 && step >= 0 && !p.forced) p.ctrl->step = step + 1;
+        fence_proxy_async_all();
+        if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_EPI_DONE);
+        return true;
+    };
+
+    // ----- before the loop: layer 0's GEMM on the initial (zero) state -----
+    if (early) {
+        if (warp == 0) {
+            if (lane == 0) { fence_proxy_async_all(); cur = 0; produce_L(0); }
+        } else if (warp == 1) {
+            if (lane == 0) { cur = 0; mma_L(0); }
+        }
+    }
 
     for (;;) {
         // =====================================================================================
-        // L phases: control step (layer 0 of a decoding step) + LSTM cell update, one phase per layer
+        // decoder phases: control step + LSTM cell update (layer 0), then one GEMM + update phase per upper layer
         // =====================================================================================
         for (int l = 0; l < p.L; ++l) {
-            const int n_tile = 4 * p.slots;
-            const int segs = l == 0 ? 1 : 2;
-            const uint32_t b_bytes = (uint32_t)n_tile * BK * 2;
+            const bool gemm_here = l > 0 || !early;
             if (warp == 0) {
-                if (lane == 0) {
-                    fence_proxy_async_all();
-                    for (int i = cta; i < p.l_items; i += G) {
-                        const int mt = i / p.ug_count, ug = i - mt * p.ug_count;
-                        for (int sg = 0; sg < segs; ++sg) {
-                            const CUtensorMap* ma = (l == 0 || sg == 1) ? &M.hb[pin][l] : &M.hb[pin ^ 1][l - 1];
-                            const CUtensorMap* mb = (l == 0 || sg == 1) ? &M.w_hh[l] : &M.w_ih[l];
-                            for (int kb = 0; kb < p.kb_p; ++kb) {
-                                const int s = ps.it % S;
-                                if (!mbar_wait(&empty_bar[s], ((ps.it / S) & 1) ^ 1, &s_abort)) goto l_done;
-                                uint8_t* a_dst = ring + (size_t)s * p.stage_bytes;
-                                uint8_t* b_dst = a_dst + LOOP_A_BYTES;
-                                mbar_expect_tx(&full_bar[s], LOOP_A_BYTES + b_bytes);
-                                tma_load_2d(a_dst, ma, kb * BK, mt * 128, &full_bar[s]);
-                                for (int g = 0; g < 4; ++g)
-                                    tma_load_2d(b_dst + (size_t)g * p.slots * 128, mb, kb * BK, g * p.P + ug * p.ul, &full_bar[s]);
-                                ++ps.it;
-                            }
-                        }
-                    }
-                }
+                if (lane == 0 && gemm_here) { fence_proxy_async_all(); cur = 0; produce_L(l); }
             } else if (warp == 1) {
-                if (lane == 0) {
-                    const uint32_t idesc = idesc_bf16(128, n_tile);
-                    for (int i = cta; i < p.l_items; i += G) {
-                        if (!mbar_wait(&acc_empty, (ps.acc & 1) ^ 1, &s_abort)) goto l_done;
-                        tc_fence_after();
-                        const int kbs = segs * p.kb_p;
-                        for (int kb = 0; kb < kbs; ++kb) {
-                            const int s = ps.it % S;
-                            if (!mbar_wait(&full_bar[s], (ps.it / S) & 1, &s_abort)) goto l_done;
-                            tc_fence_after();
-                            const uint32_t a_addr = smem_u32(ring + (size_t)s * p.stage_bytes);
-                            const uint64_t adesc = smem_desc_sw128(a_addr);
-                            const uint64_t bdesc = smem_desc_sw128(a_addr + LOOP_A_BYTES);
-#pragma unroll
-                            for (int k = 0; k < BK / 16; ++k)
-                                tc_mma_bf16(tmem_base, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
-                            tc_commit(&empty_bar[s]);
-                            ++ps.it;
-                        }
-                        tc_commit(&acc_full);
-                        ++ps.acc;
-                    }
-                }
+                if (lane == 0 && gemm_here) { cur = 0; mma_L(l); }
             } else {
-                const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
-                int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
-                const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
-                unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
-                for (int i = cta; i < p.l_items; i += G) {
-                    const int mt = i / p.ug_count, ug = i - mt * p.ug_count;
-                    const int b = mt * 128 + row_in_tile;
-                    // ---- which token does utterance b feed to its decoder in this step? ----
-                    int tok = -1;
-                    if (b < p.B) {
-                        if (step < 0) {
-                            tok = p.blank;
-                        } else if (p.forced) {
-                            tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
-                        } else if (l > 0) {
-                            tok = p.emit_tok[b];
-                        } else {
-                            // control step (Algorithm 2's branch): first non-blank row of the window
-                            int t = t_cur[b];
-                            const int len = p.enc_len[b];
-                            if (t < len) {
-                                const int n = min(p.W, len - t);
-                                int first = -1, label = p.blank;
-                                bool bad = false;
-                                for (int w0 = 0; w0 < n && first < 0; w0 += 8) {
-                                    unsigned long long kk[8];
-#pragma unroll
-                                    for (int j = 0; j < 8; ++j) kk[j] = (w0 + j < n) ? keys_cur[(size_t)b * p.W + w0 + j] : 0ull;
-#pragma unroll
-                                    for (int j = 0; j < 8; ++j) {
-                                        if (w0 + j < n && first < 0) {
-                                            uint32_t lab = key_label(kk[j]);
-                                            if (kk[j] == 0ull || lab >= (uint32_t)p.NV) { bad = true; lab = (uint32_t)p.blank; }
-                                            if ((int)lab != p.blank) { first = w0 + j; label = (int)lab; }
-                                        }
-                                    }
-                                }
-                                if (first >= 0) tok = label;
-                                if (ug == 0) {
-                                    // this CTA records the step for its utterances
-                                    int cnt = p.count[b];
-                                    int jump, forced = 0, emitted = 0;
-                                    if (first < 0) {
-                                        jump = n;
-                                        t += n;
-                                        cnt = 0;
-                                    } else {
-                                        jump = first;
-                                        if (first > 0) cnt = 0;
-                                        t += first;
-                                        const int pos = p.out_len[b];
-                                        if (pos < p.max_out) {
-                                            p.out_tokens[(size_t)b * p.max_out + pos] = label;
-                                            p.out_frames[(size_t)b * p.max_out + pos] = t;
-                                            p.out_len[b] = pos + 1;
-                                            emitted = 1;
-                                            cnt += 1;
-                                            if (cnt == p.S) { t += 1; cnt = 0; forced = 1; }
-                                        } else {
-                                            set_status(p.ctrl, WIND_ERR_OUTPUT_OVERFLOW);  // this utterance stops here
-                                            t = len;
-                                            tok = -1;
-                                        }
-                                    }
-                                    if (bad) set_status(p.ctrl, WIND_ERR_INTERNAL);
-                                    t_nxt[b] = t;
-                                    p.count[b] = cnt;
-                                    for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
-                                    atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
-                                    atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->joint_rows), (unsigned long long)n);
-                                    if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
-                                    if (forced) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
-                                }
-                            } else if (ug == 0) {
-                                t_nxt[b] = t;
-                            }
-                            if (ug == 0) p.emit_tok[b] = tok;
-                        }
-                    }
-                    // ---- LSTM cell update of units [ug*ul, ug*ul + ul) for utterance b ----
-                    const float* bi = p.b_ih[l];
-                    const float* bh = p.b_hh[l];
-                    float* cst = p.c_state + ((size_t)l * p.B + (b < p.B ? b : 0)) * p.P;
-                    const __nv_bfloat16* hin = p.hb + (((size_t)pin * p.L + l) * p.Bpad + (b < p.B ? b : 0)) * p.P;
-                    __nv_bfloat16* hout = p.hb + (((size_t)(pin ^ 1) * p.L + l) * p.Bpad + (b < p.B ? b : 0)) * p.P;
-                    const bool live = b < p.B && tok >= 0;
-                    const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full, ps.acc & 1, &s_abort));
-                    tc_fence_after();
-                    if (ready) {
-                        for (int u0 = 0; u0 < p.ul; u0 += 8) {
-                            float pre[4][8];
-#pragma unroll
-                            for (int g = 0; g < 4; ++g) tmem_ld8(tq + (uint32_t)(g * p.slots + u0), pre[g]);
-                            if (b < p.B) {
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) {
-                                    const int unit = ug * p.ul + u0 + j;
-                                    if (u0 + j < p.ul && unit < p.P) {
-                                        if (live) {
-                                            float add[4];
-#pragma unroll
-                                            for (int g = 0; g < 4; ++g)
-                                                add[g] = l == 0 ? p.g0[(size_t)tok * 4 * p.P + (size_t)g * p.P + unit]
-                                                                : bi[g * p.P + unit] + bh[g * p.P + unit];
-                                            const float gi = sigmoid_f(pre[0][j] + add[0]);
-                                            const float gf = sigmoid_f(pre[1][j] + add[1]);
-                                            const float gg = tanhf(pre[2][j] + add[2]);
-                                            const float go = sigmoid_f(pre[3][j] + add[3]);
-                                            const float cc = gf * cst[unit] + gi * gg;
-                                            cst[unit] = cc;
-                                            hout[unit] = __float2bfloat16_rn(go * tanhf(cc));
-                                        } else {
-                                            hout[unit] = hin[unit];
-                                        }
-                                    }
-                                }
-                            }
-                        }
-                    }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&acc_empty);
-                    ++ps.acc;
-                    if (!ready) goto l_done;
-                }
-                if (cta == 0 && e == 0 && l == 0 && step >= 0 && !p.forced) p.ctrl->step = step + 1;
-                fence_proxy_async_all();
+                if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_START);
+                epilogue_L(l);
             }
-        l_done:
-            // keep the role threads' counters in step: the MMA issuer and the epilogue count items alike,
-            // producer and MMA issuer count K blocks alike; lanes other than 0 of warps 0/1 hold no state
-            if (!grid_sync(1)) goto done;
+            if (!grid_sync(TR_L)) goto done;
         }
         pin ^= 1;
-        if (p.forced && step + 1 < p.U) { ++step; continue; }
+        if (p.forced && step + 1 < p.U) {
+            // teacher forcing: more prefix tokens to feed before the window is evaluated
+            if (early) {
+                if (warp == 0) {
+                    if (lane == 0) { fence_proxy_async_all(); cur = 0; produce_L(0); }
+                } else if (warp == 1) {
+                    if (lane == 0) { cur = 0; mma_L(0); }
+                }
+            }
+            ++step;
+            continue;
+        }
 
         // =====================================================================================
-        // P phase: pred_proj for every utterance, then the next window's joint activations z
+        // projection phase: pred_proj for every utterance, then the next window's joint activations z;
+        // behind it, layer 0's GEMM of the next step (its result waits in tensor memory)
         // =====================================================================================
         {
             const int n_tile = p.np;
             const uint32_t b_bytes = (uint32_t)n_tile * BK * 2;
             const int32_t* t_new = p.t2 + (size_t)((step + 1) & 1) * p.B;
+            const int i0 = p.p_items <= G ? G - 1 - cta : cta;   // projection items start at the far end of the grid
             if (warp == 0) {
                 if (lane == 0) {
                     fence_proxy_async_all();
-                    for (int i = cta; i < p.p_items; i += G) {
+                    cur = 0;
+                    bool ok = true;
+                    for (int i = i0; i < p.p_items && ok; i += G) {
                         const int mt = i / p.hg_count, hg = i - mt * p.hg_count;
                         for (int kb = 0; kb < p.kb_p; ++kb) {
-                            const int s = ps.it % S;
-                            if (!mbar_wait(&empty_bar[s], ((ps.it / S) & 1) ^ 1, &s_abort)) goto p_done;
-                            uint8_t* a_dst = ring + (size_t)s * p.stage_bytes;
-                            mbar_expect_tx(&full_bar[s], LOOP_A_BYTES + b_bytes);
-                            tma_load_2d(a_dst, &M.hb[pin][p.L - 1], kb * BK, mt * 128, &full_bar[s]);
-                            tma_load_2d(a_dst + LOOP_A_BYTES, &M.w_pred, kb * BK, hg * p.np, &full_bar[s]);
-                            ++ps.it;
+                            uint8_t* a_dst = acquire(sb_lp);
+                            if (!a_dst) { ok = false; break; }
+                            mbar_expect_tx(&full_bar[cur], LOOP_A_BYTES + b_bytes);
+                            tma_load_2d(a_dst, &M.hb[pin][p.L - 1], kb * BK, mt * 128, &full_bar[cur]);
+                            tma_load_2d(a_dst + LOOP_A_BYTES, &M.w_pred, kb * BK, hg * p.np, &full_bar[cur]);
+                            cur = cur + 1 == S_lp ? 0 : cur + 1;
                         }
                     }
+                    if (ok && early) produce_L(0);
                 }
             } else if (warp == 1) {
                 if (lane == 0) {
                     const uint32_t idesc = idesc_bf16(128, n_tile);
-                    for (int i = cta; i < p.p_items; i += G) {
-                        if (!mbar_wait(&acc_empty, (ps.acc & 1) ^ 1, &s_abort)) goto p_done;
-                        tc_fence_after();
+                    cur = 0;
+                    bool ok = true;
+                    for (int i = i0; i < p.p_items && ok; i += G) {
+                        if (!begin_acc(2)) { ok = false; break; }
                         for (int kb = 0; kb < p.kb_p; ++kb) {
-                            const int s = ps.it % S;
-                            if (!mbar_wait(&full_bar[s], (ps.it / S) & 1, &s_abort)) goto p_done;
-                            tc_fence_after();
-                            const uint32_t a_addr = smem_u32(ring + (size_t)s * p.stage_bytes);
+                            if (!consume()) { ok = false; break; }
+                            const uint32_t a_addr = smem_u32(ring + (size_t)cur * sb_lp);
                             const uint64_t adesc = smem_desc_sw128(a_addr);
                             const uint64_t bdesc = smem_desc_sw128(a_addr + LOOP_A_BYTES);
 #pragma unroll
                             for (int k = 0; k < BK / 16; ++k)
-                                tc_mma_bf16(tmem_base, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
-                            tc_commit(&empty_bar[s]);
-                            ++ps.it;
+                                tc_mma_bf16(tm_p, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+                            tc_commit(&empty_bar[cur]);
+                            cur = cur + 1 == S_lp ? 0 : cur + 1;
                         }
-                        tc_commit(&acc_full);
-                        ++ps.acc;
+                        if (ok) { tc_commit(&acc_full[2]); ++acc_n[2]; }
                     }
+                    if (ok && early) mma_L(0);
                 }
             } else {
+                if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_START);
                 // utterances still decoding, counted by every CTA (they all take the same exit)
                 {
                     int cnt = 0;
@@ -424,7 +560,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                     asm volatile("bar.sync 1, 128;" ::: "memory");
                     if (e == 0) s_active = s_red[0] + s_red[1] + s_red[2] + s_red[3];
                 }
-                for (int i = cta; i < p.p_items; i += G) {
+                for (int i = i0; i < p.p_items; i += G) {
                     const int mt = i / p.hg_count, hg = i - mt * p.hg_count;
                     const int b = mt * 128 + row_in_tile;
                     const int h0 = hg * p.np;
@@ -433,24 +569,37 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                         t = t_new[b];
                         n = min(p.W, p.enc_len[b] - t);   // <= 0 when the utterance is done
                     }
-                    const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full, ps.acc & 1, &s_abort));
+                    // the first rows of the window, requested before the accumulator is ready (np == 16)
+                    uint4 ev[4][2];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (j < n) {
+                            const uint4* src = reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + t + j) * p.H + h0);
+                            ev[j][0] = src[0];
+                            ev[j][1] = src[1];
+                        }
+                    }
+                    if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
+                    const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[2], acc_n[2] & 1u, &s_abort));
                     tc_fence_after();
+                    if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
                     if (ready) {
                         for (int c0 = 0; c0 < n_tile; c0 += 16) {
                             float g[16];
-                            tmem_ld16(tq + (uint32_t)c0, g);
+                            tmem_ld16(tm_p + lane_off + (uint32_t)c0, g);
                             if (b < p.B && n > 0) {
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) g[j] += p.b_pred[h0 + c0 + j];
                                 for (int w0 = 0; w0 < p.W; w0 += 4) {
-                                    uint4 ev[4][2];
+                                    if (w0 > 0 || c0 > 0) {
 #pragma unroll
-                                    for (int j = 0; j < 4; ++j) {
-                                        if (w0 + j < n) {
-                                            const uint4* src = reinterpret_cast<const uint4*>(
-                                                p.enc_proj + ((size_t)b * p.T + t + w0 + j) * p.H + h0 + c0);
-                                            ev[j][0] = src[0];
-                                            ev[j][1] = src[1];
+                                        for (int j = 0; j < 4; ++j) {
+                                            if (w0 + j < n) {
+                                                const uint4* src = reinterpret_cast<const uint4*>(
+                                                    p.enc_proj + ((size_t)b * p.T + t + w0 + j) * p.H + h0 + c0);
+                                                ev[j][0] = src[0];
+                                                ev[j][1] = src[1];
+                                            }
                                         }
                                     }
 #pragma unroll
@@ -482,21 +631,21 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                     }
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&acc_empty);
-                    ++ps.acc;
-                    if (!ready) goto p_done;
+                    if (lane == 0) mbar_arrive(&acc_empty[2]);
+                    ++acc_n[2];
+                    if (!ready) break;
                 }
                 fence_proxy_async_all();
+                if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
             }
-        p_done:
-            if (!grid_sync(2)) goto done;
+            if (!grid_sync(TR_P)) goto done;
         }
         if (!p.forced && s_active == 0) break;
         if (!p.forced && step + 1 >= p.step_cap) { exit_status = WIND_ERR_INTERNAL; break; }
         ++step;
 
         // =====================================================================================
-        // J phase: window logits on tensor cores, per-row argmax in the epilogue
+        // joint phase: window logits on tensor cores, per-row argmax in the epilogue
         // =====================================================================================
         {
             const int n_tile = p.nj;
@@ -505,65 +654,76 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
             if (warp == 0) {
                 if (lane == 0) {
                     fence_proxy_async_all();
-                    for (int i = cta; i < p.j_items; i += G) {
+                    cur = 0;
+                    bool ok = true;
+                    trace_event(p, 0, tr_n, step, TR_J, EV_FIRST_ISSUE);
+                    for (int i = cta; i < p.j_items && ok; i += G) {
                         const int rg = i / p.vt_count, vt = i - rg * p.vt_count;
                         for (int kb = 0; kb < p.kb_h; ++kb) {
-                            const int s = ps.it % S;
-                            if (!mbar_wait(&empty_bar[s], ((ps.it / S) & 1) ^ 1, &s_abort)) goto j_done;
-                            uint8_t* a_dst = ring + (size_t)s * p.stage_bytes;
-                            if (p.j_stationary) {
-                                mbar_expect_tx(&full_bar[s], z_bytes);
-                                tma_load_2d(a_dst, &M.z, kb * BK, rg * n_tile, &full_bar[s]);
+                            uint8_t* dst = acquire(sb_j);
+                            if (!dst) { ok = false; break; }
+                            if (p.j_mode != J_STREAM) {
+                                mbar_expect_tx(&full_bar[cur], z_bytes);
+                                tma_load_2d(dst, &M.z, kb * BK, rg * n_tile, &full_bar[cur]);
                             } else {
-                                mbar_expect_tx(&full_bar[s], LOOP_A_BYTES + z_bytes);
-                                tma_load_2d(a_dst, &M.w_out, kb * BK, vt * 128, &full_bar[s]);
-                                tma_load_2d(a_dst + LOOP_A_BYTES, &M.z, kb * BK, rg * n_tile, &full_bar[s]);
+                                mbar_expect_tx(&full_bar[cur], LOOP_A_BYTES + z_bytes);
+                                tma_load_2d(dst, &M.w_out, kb * BK, vt * 128, &full_bar[cur]);
+                                tma_load_2d(dst + LOOP_A_BYTES, &M.z, kb * BK, rg * n_tile, &full_bar[cur]);
                             }
-                            ++ps.it;
+                            cur = cur + 1 == S_j ? 0 : cur + 1;
                         }
                     }
+                    trace_event(p, 0, tr_n, step, TR_J, EV_LAST_ISSUE);
                 }
             } else if (warp == 1) {
                 if (lane == 0) {
                     const uint32_t idesc = idesc_bf16(128, n_tile);
-                    if (p.j_stationary && cta < p.j_items) {
-                        if (!mbar_wait(&stat_bar, 0, &s_abort)) goto j_done;
-                    }
-                    for (int i = cta; i < p.j_items; i += G) {
-                        if (!mbar_wait(&acc_empty, (ps.acc & 1) ^ 1, &s_abort)) goto j_done;
-                        tc_fence_after();
+                    cur = 0;
+                    bool ok = true;
+                    if (p.j_mode == J_SMEM && has_j) ok = mbar_wait(&stat_bar, 0, &s_abort);
+                    for (int i = cta; i < p.j_items && ok; i += G) {
+                        if (!begin_acc(0)) { ok = false; break; }
                         for (int kb = 0; kb < p.kb_h; ++kb) {
-                            const int s = ps.it % S;
-                            if (!mbar_wait(&full_bar[s], (ps.it / S) & 1, &s_abort)) goto j_done;
-                            tc_fence_after();
-                            const uint32_t st_addr = smem_u32(ring + (size_t)s * p.stage_bytes);
-                            const uint64_t adesc = smem_desc_sw128(p.j_stationary ? smem_u32(stat + (size_t)kb * LOOP_A_BYTES) : st_addr);
-                            const uint64_t bdesc = smem_desc_sw128(p.j_stationary ? st_addr : st_addr + LOOP_A_BYTES);
+                            if (!consume()) { ok = false; break; }
+                            if (kb == 0) trace_event(p, 1, tr_n, step, TR_J, EV_FIRST_DATA);
+                            const uint32_t st_addr = smem_u32(ring + (size_t)cur * sb_j);
+                            if (p.j_mode == J_TMEM) {
+                                const uint64_t bdesc = smem_desc_sw128(st_addr);
 #pragma unroll
-                            for (int k = 0; k < BK / 16; ++k)
-                                tc_mma_bf16(tmem_base, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
-                            tc_commit(&empty_bar[s]);
-                            ++ps.it;
+                                for (int k = 0; k < BK / 16; ++k)
+                                    tc_mma_bf16_ts(tm_j, tmem_base + (uint32_t)(kb * (BK / 2) + k * 8), bdesc + (uint64_t)(k * 2), idesc,
+                                                   (kb | k) != 0);
+                            } else {
+                                const uint64_t adesc =
+                                    smem_desc_sw128(p.j_mode == J_SMEM ? smem_u32(stat + (size_t)kb * LOOP_A_BYTES) : st_addr);
+                                const uint64_t bdesc = smem_desc_sw128(p.j_mode == J_SMEM ? st_addr : st_addr + LOOP_A_BYTES);
+#pragma unroll
+                                for (int k = 0; k < BK / 16; ++k)
+                                    tc_mma_bf16(tm_j, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+                            }
+                            tc_commit(&empty_bar[cur]);
+                            cur = cur + 1 == S_j ? 0 : cur + 1;
                         }
-                        tc_commit(&acc_full);
-                        ++ps.acc;
+                        if (ok) { tc_commit(&acc_full[0]); ++acc_n[0]; trace_event(p, 1, tr_n, step, TR_J, EV_COMMIT); }
                     }
                 }
             } else {
+                if (e == 0) trace_event(p, 2, tr_n, step, TR_J, EV_START);
                 const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
                 for (int i = cta; i < p.j_items; i += G) {
                     const int rg = i / p.vt_count, vt = i - rg * p.vt_count;
                     const int v = vt * 128 + row_in_tile;            // this thread's vocabulary entry
                     const bool v_ok = v < p.NV;
                     const float bias = v_ok ? p.b_out[v] : 0.f;
-                    const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full, ps.acc & 1, &s_abort));
+                    const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[0], acc_n[0] & 1u, &s_abort));
                     tc_fence_after();
+                    if (e == 0) trace_event(p, 2, tr_n, step, TR_J, EV_ACC);
                     if (ready) {
                         for (int c0 = 0; c0 < n_tile; c0 += 32) {
                             float val[32];
-                            tmem_ld16(tq + (uint32_t)c0, val);
+                            tmem_ld16(tm_j + lane_off + (uint32_t)c0, val);
                             if (c0 + 16 < n_tile) {
-                                tmem_ld16(tq + (uint32_t)(c0 + 16), val + 16);
+                                tmem_ld16(tm_j + lane_off + (uint32_t)(c0 + 16), val + 16);
                             } else {
 #pragma unroll
                                 for (int j = 16; j < 32; ++j) val[j] = -INFINITY;
@@ -599,17 +759,20 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                     }
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&acc_empty);
-                    ++ps.acc;
-                    if (!ready) goto j_done;
+                    if (lane == 0) mbar_arrive(&acc_empty[0]);
+                    ++acc_n[0];
+                    if (!ready) break;
                 }
+                if (e == 0) trace_event(p, 2, tr_n, step, TR_J, EV_EPI_DONE);
             }
-        j_done:
-            if (!grid_sync(0)) goto done;
+            if (!grid_sync(TR_J)) goto done;
         }
         if (p.forced) break;
     }
 done:
+    // an accumulator may still hold an unused early GEMM; nothing reads it, the MMAs have completed
+    // before the last barrier (the issuing thread waited for none of them, so wait for them here)
+    if (early && warp == 1 && lane == 0 && !s_abort) mbar_wait(&acc_full[1], acc_n[1] & 1u ? 0u : 1u, &s_abort);
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -700,9 +863,16 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
     }
     pl.rg_count = (rows + pl.nj - 1) / pl.nj;
     pl.j_items = pl.vt_count * pl.rg_count;
-    // decoder: utterance tiles of 128 x unit groups of ul (4 gates x `slots` rows per item)
+    // projection: utterance tiles of 128 x H slices of np, placed at the far end of the grid
     pl.mt_count = (c.B + 127) / 128;
-    int groups_wanted = G / pl.mt_count;
+    pl.np = 16;
+    pl.hg_count = m.H / pl.np;
+    pl.p_items = pl.mt_count * pl.hg_count;
+    // decoder: utterance tiles of 128 x unit groups of ul (4 gates x `slots` rows per item), on the
+    // CTAs the projection leaves free when there are enough of them
+    int free_ctas = G - pl.p_items;
+    if (free_ctas < G / 2) free_ctas = G;
+    int groups_wanted = free_ctas / pl.mt_count;
     if (groups_wanted < 1) groups_wanted = 1;
     pl.ul = (m.P + groups_wanted - 1) / groups_wanted;
     if (pl.ul > 64) pl.ul = 64;
@@ -710,30 +880,34 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
     while (pl.slots < pl.ul) pl.slots *= 2;
     pl.ug_count = (m.P + pl.ul - 1) / pl.ul;
     pl.l_items = pl.mt_count * pl.ug_count;
-    // projection: utterance tiles x H slices of np
-    pl.np = 16;
-    pl.hg_count = m.H / pl.np;
-    pl.p_items = pl.mt_count * pl.hg_count;
-    // shared memory: [stationary W_out tile] [ring of stages]
-    const int budget = smem_optin - 2048;   // static shared memory of the kernel and the 1 KB alignment slack
+    pl.l_early = pl.l_items <= G;
+    // where the joint's W_out tile lives, tensor-memory columns, shared-memory ring
+    const int budget = smem_optin - 2048 - 1024;   // static shared memory of the kernel, 1 KB alignment slack
     const uint32_t small_ops = (uint32_t)(4 * pl.slots > pl.np ? 4 * pl.slots : pl.np) * BK * 2;
+    pl.stage_lp = LOOP_A_BYTES + (small_ops + 1023u) / 1024u * 1024u;
     const uint32_t stat_bytes = (uint32_t)pl.kb_h * LOOP_A_BYTES;
-    const uint32_t stage_stat = LOOP_A_BYTES + small_ops;
-    pl.j_stationary = pl.j_items <= G && pl.nj <= 128 && (long long)stat_bytes + 3ll * stage_stat + 1024 <= budget;
-    if (pl.j_stationary) {
-        pl.stat_bytes = stat_bytes;
-        pl.stage_bytes = stage_stat;
-    } else {
-        const uint32_t zb = (uint32_t)pl.nj * BK * 2;
-        pl.stat_bytes = 0;
-        pl.stage_bytes = LOOP_A_BYTES + (zb > small_ops ? zb : small_ops);
+    const bool one_wave = pl.j_items <= G;
+    const bool tmem_fits = m.H / 2 + pl.nj + 4 * pl.slots + pl.np <= (int)LOOP_TMEM_COLS;
+    const bool smem_fits = pl.nj <= 128 && (long long)stat_bytes + 3ll * pl.stage_lp <= budget;
+    pl.j_mode = one_wave && tmem_fits ? J_TMEM : (one_wave && smem_fits ? J_SMEM : J_STREAM);
+    if (const char* env = getenv("WIND_J_MODE")) {   // experiments: force a placement when it is feasible
+        const int want = atoi(env);
+        if (want == J_STREAM || (want == J_SMEM && one_wave && smem_fits) || (want == J_TMEM && one_wave && tmem_fits)) pl.j_mode = want;
     }
-    pl.stage_bytes = (pl.stage_bytes + 1023u) / 1024u * 1024u;
-    int stages = (int)((budget - 1024 - (long long)pl.stat_bytes) / pl.stage_bytes);
-    if (stages > LOOP_MAX_STAGES) stages = LOOP_MAX_STAGES;
-    if (stages < 2) return cudaErrorInvalidConfiguration;
-    pl.stages = stages;
-    pl.smem_bytes = pl.stat_bytes + (uint32_t)stages * pl.stage_bytes + 1024;
+    pl.stat_bytes = pl.j_mode == J_SMEM ? stat_bytes : 0;
+    pl.stage_j = ((pl.j_mode == J_STREAM ? LOOP_A_BYTES : 0u) + (uint32_t)pl.nj * BK * 2 + 1023u) / 1024u * 1024u;
+    const long long ring = (long long)budget - pl.stat_bytes;
+    pl.stages_lp = (int)(ring / pl.stage_lp);
+    pl.stages_j = (int)(ring / pl.stage_j);
+    if (pl.stages_lp > LOOP_MAX_STAGES) pl.stages_lp = LOOP_MAX_STAGES;
+    if (pl.stages_j > LOOP_MAX_STAGES) pl.stages_j = LOOP_MAX_STAGES;
+    if (pl.stages_lp < 2 || pl.stages_j < 2) return cudaErrorInvalidConfiguration;
+    pl.tm_j = pl.j_mode == J_TMEM ? m.H / 2 : 0;
+    pl.tm_l = pl.tm_j + pl.nj;
+    pl.tm_p = pl.tm_l + 4 * pl.slots;
+    if (pl.tm_p + pl.np > (int)LOOP_TMEM_COLS) return cudaErrorInvalidConfiguration;
+    const uint32_t ring_lp = (uint32_t)pl.stages_lp * pl.stage_lp, ring_j = (uint32_t)pl.stages_j * pl.stage_j;
+    pl.smem_bytes = pl.stat_bytes + (ring_lp > ring_j ? ring_lp : ring_j) + 1024;
     *out = pl;
     return cudaSuccess;
 }
@@ -769,7 +943,8 @@ cudaError_t loop_prepare(Call& c) {
     return cudaSuccess;
 }
 
-cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* prefix_len, float* logits_out) {
+cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* prefix_len, float* logits_out,
+                    int trace_step) {
     const LoopPlan& pl = t_loop_plan;
     LoopParams p{};
     p.ctrl = c.ctrl();
@@ -778,17 +953,20 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.rows = c.B * c.W; p.rows_pad = c.lay.rows_pad; p.Bpad = c.lay.Bpad;
     long long cap = (long long)c.T * (c.S + 1) + 2;
     p.step_cap = cap > 0x7fffffff ? 0x7fffffff : (int)cap;
-    p.nj = pl.nj; p.vt_count = pl.vt_count; p.rg_count = pl.rg_count; p.j_items = pl.j_items; p.j_stationary = pl.j_stationary;
+    p.nj = pl.nj; p.vt_count = pl.vt_count; p.rg_count = pl.rg_count; p.j_items = pl.j_items; p.j_mode = pl.j_mode;
+    p.tm_j = pl.tm_j; p.tm_l = pl.tm_l; p.tm_p = pl.tm_p; p.l_early = pl.l_early;
+    p.stage_lp = pl.stage_lp; p.stage_j = pl.stage_j; p.stages_lp = pl.stages_lp; p.stages_j = pl.stages_j;
     p.slots = pl.slots; p.ul = pl.ul; p.ug_count = pl.ug_count; p.mt_count = pl.mt_count; p.l_items = pl.l_items;
     p.np = pl.np; p.hg_count = pl.hg_count; p.p_items = pl.p_items;
     p.kb_h = pl.kb_h; p.kb_p = pl.kb_p;
-    p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.stat_bytes = pl.stat_bytes;
+    p.stat_bytes = pl.stat_bytes;
     p.enc_len = c.enc_len; p.t2 = c.t(); p.count = c.count(); p.emit_tok = c.emit_tok(); p.keys2 = c.keys();
     p.out_tokens = c.out_tokens; p.out_frames = c.out_frames; p.out_len = c.out_len;
     p.c_state = c.c(); p.hb = c.hb(0, 0); p.z = c.z(); p.enc_proj = (const __nv_bfloat16*)c.enc_proj(); p.g0 = c.g0();
     for (int l = 0; l < c.m.L; ++l) { p.b_ih[l] = c.b_ih[l]; p.b_hh[l] = c.b_hh[l]; }
-    p.b_pred = c.m.b_pred; p.b_out = c.m.b_out;
+    p.b_pred = c.m.b_pred; p.b_out = c.m.b_out; p.w_out = (const __nv_bfloat16*)c.m.w_out;
     p.forced = logits_out != nullptr; p.prefix = prefix; p.U = U; p.prefix_len = prefix_len; p.logits_out = logits_out;
+    p.trace = trace_step >= -1 ? c.trace() : nullptr; p.trace_step = trace_step;
     void* args[2] = {(void*)&t_loop_maps, (void*)&p};
     return cudaLaunchCooperativeKernel((const void*)loop_kernel, dim3((unsigned)pl.grid), dim3(LOOP_THREADS), args, pl.smem_bytes,
                                        c.stream);

@@ -24,23 +24,27 @@ struct LoopPlan {
     int grid;
     int kb_h, kb_p;                        // K blocks of 64 in H and in P
     int nj, vt_count, rg_count, j_items;   // joint: window rows per item, vocabulary tiles, row groups
-    int j_stationary;                      // every CTA owns one joint item: its W_out tile stays in shared memory
+    int j_mode;                            // where the joint's W_out tile lives: 0 streamed through the ring, 1 kept in
+                                           // shared memory, 2 kept in tensor memory (1, 2: every CTA owns one joint item)
+    int tm_j, tm_l, tm_p;                  // tensor-memory columns of the joint / decoder / projection accumulators
+    int l_early;                           // layer 0's GEMM runs one phase ahead of its cell update
     int slots, ul, ug_count, mt_count, l_items;  // decoder: rows per gate block, units per item, unit groups, utterance tiles
     int np, hg_count, p_items;             // projection: H columns per item, H slices
-    int stages;
-    uint32_t stage_bytes, stat_bytes, smem_bytes;
+    int stages_lp, stages_j;               // ring stages in the decoder/projection phases and in the joint phase
+    uint32_t stage_lp, stage_j, stat_bytes, smem_bytes;
 };
 
 struct LoopParams {
     Ctrl* ctrl;
     int B, T, W, S, max_out, H, P, NV, blank, act, L;
     int rows, rows_pad, Bpad, step_cap;
-    int nj, vt_count, rg_count, j_items, j_stationary;
+    int nj, vt_count, rg_count, j_items, j_mode;
+    int tm_j, tm_l, tm_p, l_early;
     int slots, ul, ug_count, mt_count, l_items;
     int np, hg_count, p_items;
     int kb_h, kb_p;
-    int stages;
-    uint32_t stage_bytes, stat_bytes;
+    int stages_lp, stages_j;
+    uint32_t stage_lp, stage_j, stat_bytes;
     const int32_t* enc_len;
     int32_t* t2;                   // [2][B]
     int32_t* count;                // [B]
@@ -58,12 +62,16 @@ struct LoopParams {
     const float* b_hh[kMaxLayers];
     const float* b_pred;
     const float* b_out;
+    const __nv_bfloat16* w_out;    // [V+1][H]
     // teacher forcing (wind_eval_joint_window): feed prefix tokens, then store the window logits
     int forced;
     const int32_t* prefix;
     int U;
     const int32_t* prefix_len;
     float* logits_out;
+    // timeline of CTA 0 for lock steps [trace_step, trace_step + 2); trace == nullptr: off
+    TraceEvent* trace;
+    int trace_step;
 };
 
 cudaError_t loop_plan(const Call& c, LoopPlan* out);
