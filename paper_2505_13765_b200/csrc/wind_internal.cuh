@@ -20,7 +20,7 @@ struct TraceEvent {
     int32_t step;
     long long clock;   // clock64 of the SM that runs CTA 0
 };
-constexpr int kTraceRoles = 4;     // TMA issuer, MMA issuer, first epilogue thread, barrier
+constexpr int kTraceRoles = 8;     // TMA issuer, MMA issuer, first epilogue thread, barrier: of CTA 0, then of the last CTA
 constexpr int kTraceEvents = 512;
 
 // Device control block, first thing in the workspace.

@@ -86,9 +86,11 @@ __device__ __forceinline__ void argmax_exchange(float* v, int* id, int lane) {
     }
 }
 
-// Timeline record of CTA 0 (one of the role threads calls this; n is that thread's event counter).
+// Timeline record of CTA 0 and of the last CTA (a role thread calls this; n is that thread's event counter).
 __device__ __forceinline__ void trace_event(const LoopParams& p, int role, int& n, int step, int phase, int ev) {
-    if (p.trace && blockIdx.x == 0 && step >= p.trace_step && step < p.trace_step + 2 && n < kTraceEvents) {
+    if (p.trace && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) && step >= p.trace_step && step < p.trace_step + 2 &&
+        n < kTraceEvents) {
+        if (blockIdx.x != 0) role += 4;   // the last CTA's records go to the second half of the table
         TraceEvent t;
         t.tag = (uint32_t)(phase * 16 + ev);
         t.step = step;
@@ -169,6 +171,24 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
     if (p.j_mode == J_SMEM && has_j && threadIdx.x == 0) {
         mbar_expect_tx(&stat_bar, (uint32_t)p.kb_h * LOOP_A_BYTES);
         for (int kb = 0; kb < p.kb_h; ++kb) tma_load_2d(stat + (size_t)kb * LOOP_A_BYTES, &M.w_out, kb * BK, my_vt * 128, &stat_bar);
+    }
+    // resident-weights mode: CTAs [0, l_items) keep a W_hh tile (4 gates x 16 units), the last p_items CTAs a W_pred
+    // tile (64 rows), loaded once; `stat` holds kb_p blocks of 64 rows x 64 columns
+    const bool res_l = p.resident && cta < p.l_items;
+    const bool res_p = p.resident && !res_l && G - 1 - cta < p.p_items;
+    const int r_ut = cta % p.ut_count, r_ql = cta / p.ut_count;                      // unit tile / utterance group of an L CTA
+    const int r_ht = (G - 1 - cta) % p.ht_count, r_qp = (G - 1 - cta) / p.ht_count;  // H tile / utterance group of a P CTA
+    constexpr uint32_t RES_A_BYTES = 64 * BK * 2;
+    if (threadIdx.x == 0 && (res_l || res_p)) {
+        mbar_expect_tx(&stat_bar, (uint32_t)p.kb_p * RES_A_BYTES);
+        for (int kb = 0; kb < p.kb_p; ++kb) {
+            uint8_t* dst = stat + (size_t)kb * RES_A_BYTES;
+            if (res_l) {
+                for (int g = 0; g < 4; ++g) tma_load_2d(dst + g * 16 * 128, &M.w_hh_r, kb * BK, g * p.P + r_ut * 16, &stat_bar);
+            } else {
+                tma_load_2d(dst, &M.w_pred_r, kb * BK, r_ht * 64, &stat_bar);
+            }
+        }
     }
     if (p.j_mode == J_TMEM) {
         if (warp >= 2 && has_j) {
@@ -460,8 +480,303 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         return true;
     };
 
+    // =========================================================================================
+    // resident-weights mode.  Every per-step operand is ONE three-dimensional TMA box (all K blocks at once) into
+    // the single operand buffer, and every GEMM is one wait, kb x 4 MMAs back to back, two commits: the issuing
+    // threads pay for as few asynchronous instructions as possible.
+    //   decoder:    D[4 gates x 16 units, nl utterances] = W_hh tile . h^T   (warp q of the epilogue = gate q)
+    //   projection: D[64 H rows, np utterances] = W_pred tile . h^T
+    // With 64 accumulator rows, row m sits in lane (m % 16) of quadrant m / 16.
+    // =========================================================================================
+    float* stage_f = reinterpret_cast<float*>(smem + p.stage_off);   // epilogue staging
+    auto produce_one = [&](const CUtensorMap* map, int row0, uint32_t bytes) -> bool {
+        cur = 0;
+        uint8_t* dst = acquire(0);
+        if (!dst) return false;
+        mbar_expect_tx(&full_bar[0], bytes);
+        tma_load_3d(dst, map, 0, row0, 0, &full_bar[0]);
+        return true;
+    };
+    auto mma_one = [&](int k_acc, uint32_t tm_d, int n_tile, int kbs, bool a_tmem) -> bool {
+        const uint32_t idesc = idesc_bf16(a_tmem ? 128 : 64, n_tile);
+        if (!a_tmem && !mbar_wait(&stat_bar, 0, &s_abort)) return false;
+        if (!begin_acc(k_acc)) return false;
+        cur = 0;
+        if (!consume()) return false;
+        const uint32_t b_addr = smem_u32(ring);
+        const uint32_t b_block = (uint32_t)n_tile * BK * 2;
+        for (int kb = 0; kb < kbs; ++kb) {
+            const uint64_t bdesc = smem_desc_sw128(b_addr + (uint32_t)kb * b_block);
+            if (a_tmem) {
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)
+                    tc_mma_bf16_ts(tm_d, tmem_base + (uint32_t)(kb * (BK / 2) + k * 8), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+            } else {
+                const uint64_t adesc = smem_desc_sw128(smem_u32(stat + (size_t)kb * RES_A_BYTES));
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)
+                    tc_mma_bf16(tm_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+            }
+        }
+        tc_commit(&empty_bar[0]);
+        tc_commit(&acc_full[k_acc]);
+        ++acc_n[k_acc];
+        return true;
+    };
+    // control step + LSTM cell update of an L CTA: units [r_ut*16, +16), utterances [r_ql*nl, +nl)
+    auto epilogue_res_L = [&]() -> bool {
+        const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
+        int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
+        const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
+        unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
+        const int u16 = lane & 15;
+        const int unit = r_ut * 16 + u16;        // this thread's hidden unit; its gate is q
+        const bool row_ok = lane < 16;           // lanes 16..31 of a quadrant hold no accumulator row
+        const bool writer = r_ut == 0 && q == 0; // one warp per utterance group records the step
+        float* cst = p.c_state + unit;
+        const __nv_bfloat16* hin = p.hb + ((size_t)pin * p.Bpad) * p.P + unit;
+        __nv_bfloat16* hout = p.hb + ((size_t)(pin ^ 1) * p.Bpad) * p.P + unit;
+        const float* g0u = p.g0 + (size_t)q * p.P + unit;
+        const uint32_t g0_stride = 4u * (uint32_t)p.P;
+        bool ready = true;
+        for (int c0 = 0; c0 < p.nl; c0 += 32) {
+            // ---- lane j: which token does utterance b0 + j feed to its decoder in this step? ----
+            const int b0 = r_ql * p.nl + c0;
+            const int b = b0 + lane;
+            const bool in = c0 + lane < p.nl && b < p.B;
+            int tok = -1;
+            if (in) {
+                if (step < 0) {
+                    tok = p.blank;
+                } else if (p.forced) {
+                    tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
+                } else {
+                    // control step (Algorithm 2's branch); everything it reads is requested at once
+                    int t = t_cur[b];
+                    const int len = p.enc_len[b];
+                    int cnt = 0, pos = 0;
+                    if (writer) { cnt = p.count[b]; pos = p.out_len[b]; }
+                    unsigned long long kk[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) kk[j] = j < p.W ? keys_cur[(size_t)b * p.W + j] : 0ull;
+                    if (t < len) {
+                        const int n = min(p.W, len - t);
+                        int first = -1, label = p.blank;
+                        bool bad = false;
+                        for (int w0 = 0; w0 < n && first < 0; w0 += 8) {
+                            if (w0 > 0) {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) kk[j] = (w0 + j < n) ? keys_cur[(size_t)b * p.W + w0 + j] : 0ull;
+                            }
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                if (w0 + j < n && first < 0) {
+                                    uint32_t lab = key_label(kk[j]);
+                                    if (kk[j] == 0ull || lab >= (uint32_t)p.NV) { bad = true; lab = (uint32_t)p.blank; }
+                                    if ((int)lab != p.blank) { first = w0 + j; label = (int)lab; }
+                                }
+                            }
+                        }
+                        if (first >= 0) tok = label;
+                        if (writer) {
+                            int jump, forced = 0, emitted = 0;
+                            if (first < 0) {
+                                jump = n;
+                                t += n;
+                                cnt = 0;
+                            } else {
+                                jump = first;
+                                if (first > 0) cnt = 0;
+                                t += first;
+                                if (pos < p.max_out) {
+                                    p.out_tokens[(size_t)b * p.max_out + pos] = label;
+                                    p.out_frames[(size_t)b * p.max_out + pos] = t;
+                                    p.out_len[b] = pos + 1;
+                                    emitted = 1;
+                                    cnt += 1;
+                                    if (cnt == p.S) { t += 1; cnt = 0; forced = 1; }
+                                } else {
+                                    set_status(p.ctrl, WIND_ERR_OUTPUT_OVERFLOW);  // this utterance stops here
+                                    t = len;
+                                    tok = -1;
+                                }
+                            }
+                            if (bad) set_status(p.ctrl, WIND_ERR_INTERNAL);
+                            t_nxt[b] = t;
+                            p.count[b] = cnt;
+                            for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
+                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
+                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->joint_rows), (unsigned long long)n);
+                            if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
+                            if (forced) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
+                        }
+                    } else if (writer) {
+                        t_nxt[b] = t;
+                    }
+                }
+            }
+            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
+            // ---- operands of the cell update: the old cell state of the four (utterance, unit) pairs this thread
+            //      finishes, and the token's gate-table entry for this thread's gate and unit ----
+            float cold[4];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                const int j = (lane >> 4) + 2 * q + 8 * jj;
+                const int bj = b0 + j;
+                cold[jj] = (c0 + j < p.nl && bj < p.B) ? cst[(size_t)bj * p.P] : 0.f;
+            }
+            float add[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int tj = __shfl_sync(0xffffffffu, tok, j);
+                add[j] = (row_ok && tj >= 0) ? g0u[(uint32_t)tj * g0_stride] : 0.f;
+            }
+            if (c0 == 0) {
+                ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, &s_abort));
+                tc_fence_after();
+                if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
+            }
+            if (ready) {
+                float pre[32];
+                tmem_ld16(tm_l + lane_off + (uint32_t)c0, pre);
+                if (c0 + 16 < p.nl) {
+                    tmem_ld16(tm_l + lane_off + (uint32_t)(c0 + 16), pre + 16);
+                } else {
+#pragma unroll
+                    for (int j = 16; j < 32; ++j) pre[j] = 0.f;
+                }
+                // warp q holds gate q: tanh for the cell candidate (q == 2), logistic for the other three,
+                // written as 0.5 tanh(x / 2) + 0.5 so that both are one hardware tanh
+                const float sc = q == 2 ? 1.f : 0.5f, of = q == 2 ? 0.f : 0.5f;
+                if (row_ok) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) stage_f[(q * 32 + j) * 16 + u16] = fmaf(tanh_fast((pre[j] + add[j]) * sc), sc, of);
+                }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (ready) {
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = (lane >> 4) + 2 * q + 8 * jj;
+                    const int bj = b0 + j;
+                    const int tj = __shfl_sync(0xffffffffu, tok, j);
+                    if (c0 + j < p.nl && bj < p.B) {
+                        if (tj >= 0) {
+                            const float gi = stage_f[(0 * 32 + j) * 16 + u16], gf = stage_f[(1 * 32 + j) * 16 + u16];
+                            const float gg = stage_f[(2 * 32 + j) * 16 + u16], go = stage_f[(3 * 32 + j) * 16 + u16];
+                            const float cc = gf * cold[jj] + gi * gg;
+                            cst[(size_t)bj * p.P] = cc;
+                            hout[(size_t)bj * p.P] = __float2bfloat16_rn(go * tanh_fast(cc));
+                        } else {
+                            hout[(size_t)bj * p.P] = hin[(size_t)bj * p.P];
+                        }
+                    }
+                }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[1]);
+        ++acc_n[1];
+        fence_proxy_async_all();
+        if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_EPI_DONE);
+        return ready;
+    };
+    // projection epilogue of a P CTA: pred_proj rows [r_ht*64, +64) of utterances [r_qp*np, +np), then z
+    auto epilogue_res_P = [&]() -> bool {
+        const int32_t* t_new = p.t2 + (size_t)((step + 1) & 1) * p.B;
+        const int h0 = r_ht * 64;
+        const int rows_here = p.np * p.W;          // z rows of this CTA: (utterance, window row) pairs
+        // fetch the 64 enc_proj values of z row r (8 x 16 bytes); false when the row lies outside the window
+        auto fetch = [&](int r, uint4* ev) -> bool {
+            const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
+            if (r >= rows_here || b >= p.B) return false;
+            const int t = t_new[b];
+            if (w >= min(p.W, p.enc_len[b] - t)) return false;
+            const uint4* src = reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + t + w) * p.H + h0);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) ev[k] = src[k];
+            return true;
+        };
+        // z row r = act(enc_proj row + pred_proj of its utterance), or zeros outside the window
+        auto emit = [&](int r, bool have, const uint4* ev) {
+            const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
+            if (r >= rows_here || b >= p.B) return;
+            if (t_new[b] >= p.enc_len[b]) return;    // utterance done: its z rows are never used again
+            uint4* dst = reinterpret_cast<uint4*>(p.z + ((size_t)b * p.W + w) * p.H + h0);
+            const float* gs = stage_f + bl * 65;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                uint4 o = make_uint4(0, 0, 0, 0);
+                if (have) {
+                    const __nv_bfloat162* eb = reinterpret_cast<const __nv_bfloat162*>(&ev[k]);
+                    uint32_t wds[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float2 e2 = __bfloat1622float2(eb[i]);
+                        float z0 = e2.x + gs[k * 8 + 2 * i], z1 = e2.y + gs[k * 8 + 2 * i + 1];
+                        z0 = p.act == WIND_ACT_RELU ? fmaxf(z0, 0.f) : tanh_fast(z0);
+                        z1 = p.act == WIND_ACT_RELU ? fmaxf(z1, 0.f) : tanh_fast(z1);
+                        wds[i] = pack_bf16x2(z0, z1);
+                    }
+                    o = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+                }
+                dst[k] = o;
+            }
+        };
+        // the first two z rows of this thread are requested before the accumulator is ready
+        uint4 ev0[8], ev1[8];
+        const bool have0 = fetch(e, ev0), have1 = fetch(e + 128, ev1);
+        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
+        const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[2], acc_n[2] & 1u, &s_abort));
+        tc_fence_after();
+        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
+        if (ready) {
+            const int hl = 16 * q + (lane & 15);
+            const float bias = p.b_pred[h0 + hl];
+            for (int c0 = 0; c0 < p.np; c0 += 16) {
+                float g[16];
+                tmem_ld16(tm_p + lane_off + (uint32_t)c0, g);
+                if (lane < 16) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) stage_f[(c0 + j) * 65 + hl] = g[j] + bias;
+                }
+            }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[2]);
+        ++acc_n[2];
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ready) {
+            emit(e, have0, ev0);
+            emit(e + 128, have1, ev1);
+            for (int r = e + 256; r < rows_here; r += 128) {
+                const bool have = fetch(r, ev0);
+                emit(r, have, ev0);
+            }
+        }
+        fence_proxy_async_all();
+        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
+        return ready;
+    };
+    // the decoder GEMM of the next step, on the state hb[pin] (TMA and MMA issuers of an L CTA)
+    auto early_res = [&]() {
+        if (warp == 0) {
+            if (lane == 0 && res_l) {
+                fence_proxy_async_all();
+                produce_one(&M.hb_l3[pin], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u);
+            }
+        } else if (warp == 1) {
+            if (lane == 0 && res_l) mma_one(1, tm_l, p.nl, p.kb_p, false);
+        }
+    };
+
     // ----- before the loop: layer 0's GEMM on the initial (zero) state -----
-    if (early) {
+    if (p.resident) {
+        early_res();
+    } else if (early) {
         if (warp == 0) {
             if (lane == 0) { fence_proxy_async_all(); cur = 0; produce_L(0); }
         } else if (warp == 1) {
@@ -473,7 +788,15 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         // =====================================================================================
         // decoder phases: control step + LSTM cell update (layer 0), then one GEMM + update phase per upper layer
         // =====================================================================================
-        for (int l = 0; l < p.L; ++l) {
+        if (p.resident) {
+            if (warp >= 2) {
+                if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_START);
+                if (res_l) epilogue_res_L();
+                if (cta == 0 && e == 0 && step >= 0 && !p.forced) p.ctrl->step = step + 1;
+            }
+            if (!grid_sync(TR_L)) goto done;
+        }
+        for (int l = 0; l < p.L && !p.resident; ++l) {
             const bool gemm_here = l > 0 || !early;
             if (warp == 0) {
                 if (lane == 0 && gemm_here) { fence_proxy_async_all(); cur = 0; produce_L(l); }
@@ -488,7 +811,9 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         pin ^= 1;
         if (p.forced && step + 1 < p.U) {
             // teacher forcing: more prefix tokens to feed before the window is evaluated
-            if (early) {
+            if (p.resident) {
+                early_res();
+            } else if (early) {
                 if (warp == 0) {
                     if (lane == 0) { fence_proxy_async_all(); cur = 0; produce_L(0); }
                 } else if (warp == 1) {
@@ -508,7 +833,27 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
             const uint32_t b_bytes = (uint32_t)n_tile * BK * 2;
             const int32_t* t_new = p.t2 + (size_t)((step + 1) & 1) * p.B;
             const int i0 = p.p_items <= G ? G - 1 - cta : cta;   // projection items start at the far end of the grid
-            if (warp == 0) {
+            if (p.resident) {
+                if (warp == 0) {
+                    if (lane == 0 && res_p) {
+                        fence_proxy_async_all();
+                        produce_one(&M.hb_p3[pin], r_qp * p.np, (uint32_t)p.np * (uint32_t)p.P * 2u);
+                    }
+                } else if (warp == 1) {
+                    if (lane == 0 && res_p) mma_one(2, tm_p, p.np, p.kb_p, false);
+                } else {
+                    if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_START);
+                    int cnt = 0;
+                    for (int b = e; b < p.B; b += 128) cnt += t_new[b] < p.enc_len[b];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+                    if (lane == 0) s_red[warp - 2] = cnt;
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (e == 0) s_active = s_red[0] + s_red[1] + s_red[2] + s_red[3];
+                    if (res_p) epilogue_res_P();
+                }
+                early_res();
+            } else if (warp == 0) {
                 if (lane == 0) {
                     fence_proxy_async_all();
                     cur = 0;
@@ -651,7 +996,20 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
             const int n_tile = p.nj;
             const uint32_t z_bytes = (uint32_t)n_tile * BK * 2;
             unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
-            if (warp == 0) {
+            if (p.resident && warp < 2) {
+                // one box for the whole z tile, then every MMA back to back (A = W_out tile in tensor memory)
+                if (lane == 0 && has_j) {
+                    if (warp == 0) {
+                        fence_proxy_async_all();
+                        trace_event(p, 0, tr_n, step, TR_J, EV_FIRST_ISSUE);
+                        produce_one(&M.z3, (cta / p.vt_count) * n_tile, (uint32_t)n_tile * (uint32_t)p.H * 2u);
+                        trace_event(p, 0, tr_n, step, TR_J, EV_LAST_ISSUE);
+                    } else {
+                        mma_one(0, tm_j, n_tile, p.kb_h, true);
+                        trace_event(p, 1, tr_n, step, TR_J, EV_COMMIT);
+                    }
+                }
+            } else if (warp == 0) {
                 if (lane == 0) {
                     fence_proxy_async_all();
                     cur = 0;
@@ -841,6 +1199,19 @@ static cudaError_t loop_map(CUtensorMap* map, const void* base, uint64_t rows, u
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// the same matrix seen as (64 columns, rows, cols / 64 blocks): one box of (64, box_rows, all blocks) lands in shared
+// memory as cols / 64 consecutive K blocks of box_rows x 128 bytes, each with the 128-byte swizzle
+static cudaError_t loop_map3(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    cuuint64_t dims[3] = {(cuuint64_t)BK, rows, cols / BK};
+    cuuint64_t strides[2] = {cols * 2, (cuuint64_t)BK * 2};
+    cuuint32_t box[3] = {(cuuint32_t)BK, box_rows, (cuuint32_t)(cols / BK)};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode_loop(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
 // Tile plan: how each phase's GEMM is cut into items (one item = one accumulator), sized so that a
 // phase is one wave over the grid whenever the shapes allow.
 cudaError_t loop_plan(const Call& c, LoopPlan* out) {
@@ -908,6 +1279,51 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
     if (pl.tm_p + pl.np > (int)LOOP_TMEM_COLS) return cudaErrorInvalidConfiguration;
     const uint32_t ring_lp = (uint32_t)pl.stages_lp * pl.stage_lp, ring_j = (uint32_t)pl.stages_j * pl.stage_j;
     pl.smem_bytes = pl.stat_bytes + (ring_lp > ring_j ? ring_lp : ring_j) + 1024;
+
+    // Resident-weights mode (one LSTM layer, W_out tile in tensor memory): W_hh in tiles of 4 gates x 16 units and
+    // W_pred in tiles of 64 rows stay in the shared memory of disjoint CTA sets for the whole decode; per step a CTA
+    // fetches only its utterance group's rows of the state, as one box.
+    const char* res_env = getenv("WIND_RESIDENT");
+    if (m.L == 1 && one_wave && m.H / 2 + pl.nj <= (int)LOOP_TMEM_COLS && !(res_env && atoi(res_env) == 0)) {
+        LoopPlan r = pl;
+        r.ut_count = m.P / 16;
+        r.ht_count = m.H / 64;
+        bool found = false;
+        for (int nl : {16, 32, 64, 128}) {
+            for (int npr : {16, 32, 64, 128}) {
+                const int ql = (c.B + nl - 1) / nl, qp = (c.B + npr - 1) / npr;
+                if (r.ut_count * ql + r.ht_count * qp <= G) {
+                    r.nl = nl; r.np = npr; r.ql_count = ql; r.qp_count = qp;
+                    found = true;
+                    break;
+                }
+            }
+            if (found) break;
+        }
+        if (found) {
+            const uint32_t staging = 17408;
+            const uint32_t tile = (uint32_t)r.kb_p * 64u * BK * 2u;
+            uint32_t buf = (uint32_t)r.nj * (uint32_t)m.H * 2u;
+            if ((uint32_t)r.nl * m.P * 2u > buf) buf = (uint32_t)r.nl * m.P * 2u;
+            if ((uint32_t)r.np * m.P * 2u > buf) buf = (uint32_t)r.np * m.P * 2u;
+            buf = (buf + 1023u) / 1024u * 1024u;
+            r.resident = 1;
+            r.j_mode = J_TMEM;
+            r.stat_bytes = tile;
+            r.buf_off = tile;
+            r.stage_off = tile + buf;
+            r.smem_bytes = tile + buf + staging + 1024;
+            r.stages_lp = r.stages_j = 1;
+            r.stage_lp = r.stage_j = 0;
+            r.tm_j = m.H / 2;
+            r.tm_l = r.tm_p = r.tm_j + r.nj;
+            r.l_items = r.ut_count * r.ql_count;
+            r.p_items = r.ht_count * r.qp_count;
+            r.l_early = 1;
+            const int acc_cols = r.nl > r.np ? r.nl : r.np;
+            if ((long long)r.smem_bytes <= (long long)budget + 1024 && r.tm_l + acc_cols <= (int)LOOP_TMEM_COLS) pl = r;
+        }
+    }
     *out = pl;
     return cudaSuccess;
 }
@@ -930,6 +1346,15 @@ cudaError_t loop_prepare(Call& c) {
         if (l > 0) WIND_MAP(loop_map(&M.w_ih[l], c.w_ih[l], 4ull * m.P, m.P, pl.slots));
         WIND_MAP(loop_map(&M.w_hh[l], c.w_hh[l], 4ull * m.P, m.P, pl.slots));
         for (int par = 0; par < 2; ++par) WIND_MAP(loop_map(&M.hb[par][l], c.hb(par, l), c.lay.Bpad, m.P, 128));
+    }
+    if (pl.resident) {
+        WIND_MAP(loop_map(&M.w_hh_r, c.w_hh[0], 4ull * m.P, m.P, 16));
+        WIND_MAP(loop_map(&M.w_pred_r, m.w_pred, m.H, m.P, 64));
+        for (int par = 0; par < 2; ++par) {
+            WIND_MAP(loop_map3(&M.hb_l3[par], c.hb(par, 0), c.lay.Bpad, m.P, pl.nl));
+            WIND_MAP(loop_map3(&M.hb_p3[par], c.hb(par, 0), c.lay.Bpad, m.P, pl.np));
+        }
+        WIND_MAP(loop_map3(&M.z3, c.z(), (uint64_t)c.lay.rows_pad, m.H, pl.nj));
     }
 #undef WIND_MAP
     {
@@ -955,6 +1380,8 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.step_cap = cap > 0x7fffffff ? 0x7fffffff : (int)cap;
     p.nj = pl.nj; p.vt_count = pl.vt_count; p.rg_count = pl.rg_count; p.j_items = pl.j_items; p.j_mode = pl.j_mode;
     p.tm_j = pl.tm_j; p.tm_l = pl.tm_l; p.tm_p = pl.tm_p; p.l_early = pl.l_early;
+    p.resident = pl.resident; p.nl = pl.nl; p.ut_count = pl.ut_count > 0 ? pl.ut_count : 1; p.ht_count = pl.ht_count > 0 ? pl.ht_count : 1;
+    p.ql_count = pl.ql_count; p.qp_count = pl.qp_count; p.buf_off = pl.buf_off; p.stage_off = pl.stage_off;
     p.stage_lp = pl.stage_lp; p.stage_j = pl.stage_j; p.stages_lp = pl.stages_lp; p.stages_j = pl.stages_j;
     p.slots = pl.slots; p.ul = pl.ul; p.ug_count = pl.ug_count; p.mt_count = pl.mt_count; p.l_items = pl.l_items;
     p.np = pl.np; p.hg_count = pl.hg_count; p.p_items = pl.p_items;

@@ -17,6 +17,13 @@ struct LoopMaps {
     CUtensorMap w_ih[kMaxLayers];      // [4P, P], box `slots` rows (layers > 0)
     CUtensorMap w_hh[kMaxLayers];      // [4P, P], box `slots` rows
     CUtensorMap hb[2][kMaxLayers];     // [Bpad, P], box 128 rows
+    // resident-weights mode (one LSTM layer): weight tiles of 64 rows loaded once; per-step operands as ONE
+    // three-dimensional box each (64 columns, rows, all K blocks)
+    CUtensorMap w_hh_r;                // [4P, P], box 16 rows (one gate's 16 units)
+    CUtensorMap w_pred_r;              // [H, P], box 64 rows
+    CUtensorMap hb_l3[2];              // [Bpad, P] as (64, rows, P/64), box (64, nl, P/64)
+    CUtensorMap hb_p3[2];              // same, box (64, np, P/64)
+    CUtensorMap z3;                    // [rows_pad, H] as (64, rows, H/64), box (64, nj, H/64)
 };
 
 // How the three phases are cut into items and how shared memory is used (host-chosen).
@@ -28,6 +35,10 @@ struct LoopPlan {
                                            // shared memory, 2 kept in tensor memory (1, 2: every CTA owns one joint item)
     int tm_j, tm_l, tm_p;                  // tensor-memory columns of the joint / decoder / projection accumulators
     int l_early;                           // layer 0's GEMM runs one phase ahead of its cell update
+    // resident-weights mode: W_hh tiles (4 gates x 16 units) and W_pred tiles (64 rows) stay in the shared memory of
+    // disjoint CTA sets; accumulators are [64 weight rows, nl or np utterances]
+    int resident, nl, ut_count, ht_count, ql_count, qp_count;
+    uint32_t buf_off, stage_off;           // the per-step operand buffer and the epilogue staging area (after the tile)
     int slots, ul, ug_count, mt_count, l_items;  // decoder: rows per gate block, units per item, unit groups, utterance tiles
     int np, hg_count, p_items;             // projection: H columns per item, H slices
     int stages_lp, stages_j;               // ring stages in the decoder/projection phases and in the joint phase
@@ -40,6 +51,8 @@ struct LoopParams {
     int rows, rows_pad, Bpad, step_cap;
     int nj, vt_count, rg_count, j_items, j_mode;
     int tm_j, tm_l, tm_p, l_early;
+    int resident, nl, ut_count, ht_count, ql_count, qp_count;
+    uint32_t buf_off, stage_off;
     int slots, ul, ug_count, mt_count, l_items;
     int np, hg_count, p_items;
     int kb_h, kb_p;
