@@ -250,7 +250,8 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                         else if (now - t0 > kWaitLimitNs) { s_abort = 1; atomicExch(&p.ctrl->abort, 1); break; }
                     }
                 }
-                __threadfence();
+                // the acquire load orders this thread after every arrival; the block barrier below extends that to
+                // the other threads of the CTA
             }
             trace_event(p, 3, tr_n, step, phase_kind, EV_RELEASE);
             if (cta == 0) {
@@ -523,113 +524,128 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         ++acc_n[k_acc];
         return true;
     };
-    // control step + LSTM cell update of an L CTA: units [r_ut*16, +16), utterances [r_ql*nl, +nl)
+    // control step + LSTM cell update of an L CTA: units [r_ut*16, +16), utterances [r_ql*nl, +nl), 64 utterances per
+    // pass.  All global reads of a pass are requested together: first everything the control step needs, then the
+    // gate-table rows of the chosen tokens; lanes 16..31 of a warp hold no accumulator row (64-row tile), so they
+    // take the second 32 utterances of the pass.
+    struct ScanIn { int t, len, cnt, pos; unsigned long long kk[8]; };
     auto epilogue_res_L = [&]() -> bool {
         const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
         int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
         const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
         unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
-        const int u16 = lane & 15;
+        const int u16 = lane & 15, half = lane >> 4;
         const int unit = r_ut * 16 + u16;        // this thread's hidden unit; its gate is q
-        const bool row_ok = lane < 16;           // lanes 16..31 of a quadrant hold no accumulator row
         const bool writer = r_ut == 0 && q == 0; // one warp per utterance group records the step
+        const bool decode = step >= 0 && !p.forced;
         float* cst = p.c_state + unit;
         const __nv_bfloat16* hin = p.hb + ((size_t)pin * p.Bpad) * p.P + unit;
         __nv_bfloat16* hout = p.hb + ((size_t)(pin ^ 1) * p.Bpad) * p.P + unit;
         const float* g0u = p.g0 + (size_t)q * p.P + unit;
         const uint32_t g0_stride = 4u * (uint32_t)p.P;
-        bool ready = true;
-        for (int c0 = 0; c0 < p.nl; c0 += 32) {
-            // ---- lane j: which token does utterance b0 + j feed to its decoder in this step? ----
-            const int b0 = r_ql * p.nl + c0;
-            const int b = b0 + lane;
-            const bool in = c0 + lane < p.nl && b < p.B;
-            int tok = -1;
-            if (in) {
-                if (step < 0) {
-                    tok = p.blank;
-                } else if (p.forced) {
-                    tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
-                } else {
-                    // control step (Algorithm 2's branch); everything it reads is requested at once
-                    int t = t_cur[b];
-                    const int len = p.enc_len[b];
-                    int cnt = 0, pos = 0;
-                    if (writer) { cnt = p.count[b]; pos = p.out_len[b]; }
-                    unsigned long long kk[8];
+        auto scan_load = [&](int b, bool in, ScanIn& si) {
+            si.t = 0; si.len = 0; si.cnt = 0; si.pos = 0;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) kk[j] = j < p.W ? keys_cur[(size_t)b * p.W + j] : 0ull;
-                    if (t < len) {
-                        const int n = min(p.W, len - t);
-                        int first = -1, label = p.blank;
-                        bool bad = false;
-                        for (int w0 = 0; w0 < n && first < 0; w0 += 8) {
-                            if (w0 > 0) {
+            for (int j = 0; j < 8; ++j) si.kk[j] = 0ull;
+            if (in && decode) {
+                si.t = t_cur[b];
+                si.len = p.enc_len[b];
+                if (writer) { si.cnt = p.count[b]; si.pos = p.out_len[b]; }
 #pragma unroll
-                                for (int j = 0; j < 8; ++j) kk[j] = (w0 + j < n) ? keys_cur[(size_t)b * p.W + w0 + j] : 0ull;
-                            }
+                for (int j = 0; j < 8; ++j)
+                    if (j < p.W) si.kk[j] = keys_cur[(size_t)b * p.W + j];
+            }
+        };
+        // the token utterance b feeds to its decoder in this step (-1: none); the writer warp also records the step
+        auto scan_decide = [&](int b, bool in, ScanIn& si) -> int {
+            if (!in) return -1;
+            if (step < 0) return p.blank;
+            if (p.forced) return step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
+            int t = si.t, tok = -1;
+            const int len = si.len;
+            if (t < len) {
+                // control step (Algorithm 2's branch): first non-blank row of the window
+                const int n = min(p.W, len - t);
+                int first = -1, label = p.blank;
+                bool bad = false;
+                for (int w0 = 0; w0 < n && first < 0; w0 += 8) {
+                    if (w0 > 0) {
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                if (w0 + j < n && first < 0) {
-                                    uint32_t lab = key_label(kk[j]);
-                                    if (kk[j] == 0ull || lab >= (uint32_t)p.NV) { bad = true; lab = (uint32_t)p.blank; }
-                                    if ((int)lab != p.blank) { first = w0 + j; label = (int)lab; }
-                                }
-                            }
+                        for (int j = 0; j < 8; ++j) si.kk[j] = (w0 + j < n) ? keys_cur[(size_t)b * p.W + w0 + j] : 0ull;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (w0 + j < n && first < 0) {
+                            uint32_t lab = key_label(si.kk[j]);
+                            if (si.kk[j] == 0ull || lab >= (uint32_t)p.NV) { bad = true; lab = (uint32_t)p.blank; }
+                            if ((int)lab != p.blank) { first = w0 + j; label = (int)lab; }
                         }
-                        if (first >= 0) tok = label;
-                        if (writer) {
-                            int jump, forced = 0, emitted = 0;
-                            if (first < 0) {
-                                jump = n;
-                                t += n;
-                                cnt = 0;
-                            } else {
-                                jump = first;
-                                if (first > 0) cnt = 0;
-                                t += first;
-                                if (pos < p.max_out) {
-                                    p.out_tokens[(size_t)b * p.max_out + pos] = label;
-                                    p.out_frames[(size_t)b * p.max_out + pos] = t;
-                                    p.out_len[b] = pos + 1;
-                                    emitted = 1;
-                                    cnt += 1;
-                                    if (cnt == p.S) { t += 1; cnt = 0; forced = 1; }
-                                } else {
-                                    set_status(p.ctrl, WIND_ERR_OUTPUT_OVERFLOW);  // this utterance stops here
-                                    t = len;
-                                    tok = -1;
-                                }
-                            }
-                            if (bad) set_status(p.ctrl, WIND_ERR_INTERNAL);
-                            t_nxt[b] = t;
-                            p.count[b] = cnt;
-                            for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
-                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
-                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->joint_rows), (unsigned long long)n);
-                            if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
-                            if (forced) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
-                        }
-                    } else if (writer) {
-                        t_nxt[b] = t;
                     }
                 }
+                if (first >= 0) tok = label;
+                if (writer) {
+                    int cnt = si.cnt, jump, forced = 0, emitted = 0;
+                    if (first < 0) {
+                        jump = n;
+                        t += n;
+                        cnt = 0;
+                    } else {
+                        jump = first;
+                        if (first > 0) cnt = 0;
+                        t += first;
+                        if (si.pos < p.max_out) {
+                            p.out_tokens[(size_t)b * p.max_out + si.pos] = label;
+                            p.out_frames[(size_t)b * p.max_out + si.pos] = t;
+                            p.out_len[b] = si.pos + 1;
+                            emitted = 1;
+                            cnt += 1;
+                            if (cnt == p.S) { t += 1; cnt = 0; forced = 1; }
+                        } else {
+                            set_status(p.ctrl, WIND_ERR_OUTPUT_OVERFLOW);  // this utterance stops here
+                            t = len;
+                            tok = -1;
+                        }
+                    }
+                    if (bad) set_status(p.ctrl, WIND_ERR_INTERNAL);
+                    t_nxt[b] = t;
+                    p.count[b] = cnt;
+                    for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
+                    atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
+                    atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->joint_rows), (unsigned long long)n);
+                    if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
+                    if (forced) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
+                }
+            } else if (writer) {
+                t_nxt[b] = t;
             }
-            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
-            // ---- operands of the cell update: the old cell state of the four (utterance, unit) pairs this thread
-            //      finishes, and the token's gate-table entry for this thread's gate and unit ----
-            float cold[4];
+            return tok;
+        };
+        bool ready = true;
+        for (int c0 = 0; c0 < p.nl; c0 += 64) {
+            const int b0 = r_ql * p.nl + c0;
+            // ---- lane j decides for utterances b0 + j and b0 + 32 + j ----
+            const int ba = b0 + lane, bb = b0 + 32 + lane;
+            const bool in_a = c0 + lane < p.nl && ba < p.B, in_b = c0 + 32 + lane < p.nl && bb < p.B;
+            ScanIn sa, sb;
+            scan_load(ba, in_a, sa);
+            scan_load(bb, in_b, sb);
+            // old cell state of the eight (utterance, unit) pairs this thread finishes
+            float cold[8];
 #pragma unroll
-            for (int jj = 0; jj < 4; ++jj) {
-                const int j = (lane >> 4) + 2 * q + 8 * jj;
-                const int bj = b0 + j;
-                cold[jj] = (c0 + j < p.nl && bj < p.B) ? cst[(size_t)bj * p.P] : 0.f;
+            for (int jj = 0; jj < 8; ++jj) {
+                const int j = half + 2 * q + 8 * jj;
+                cold[jj] = (c0 + j < p.nl && b0 + j < p.B) ? cst[(size_t)(b0 + j) * p.P] : 0.f;
             }
+            const int tok_a = scan_decide(ba, in_a, sa);
+            const int tok_b = scan_decide(bb, in_b, sb);
+            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
+            // ---- gate-table entries (this thread's gate and unit) of the tokens of this lane half's 32 utterances ----
             float add[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-                const int tj = __shfl_sync(0xffffffffu, tok, j);
-                add[j] = (row_ok && tj >= 0) ? g0u[(uint32_t)tj * g0_stride] : 0.f;
+                const int ta = __shfl_sync(0xffffffffu, tok_a, j), tb = __shfl_sync(0xffffffffu, tok_b, j);
+                const int tj = half ? tb : ta;
+                add[j] = tj >= 0 ? g0u[(uint32_t)tj * g0_stride] : 0.f;
             }
             if (c0 == 0) {
                 ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, &s_abort));
@@ -637,33 +653,38 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                 if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
             }
             if (ready) {
-                float pre[32];
-                tmem_ld16(tm_l + lane_off + (uint32_t)c0, pre);
-                if (c0 + 16 < p.nl) {
-                    tmem_ld16(tm_l + lane_off + (uint32_t)(c0 + 16), pre + 16);
-                } else {
+                // lanes 0..15 read their row's 64 columns; columns 32..63 then move to lanes 16..31
+                float x[32], hi[32];
 #pragma unroll
-                    for (int j = 16; j < 32; ++j) pre[j] = 0.f;
+                for (int j = 0; j < 32; ++j) { x[j] = 0.f; hi[j] = 0.f; }
+                tmem_ld16(tm_l + lane_off + (uint32_t)c0, x);
+                if (c0 + 16 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(c0 + 16), x + 16);
+                if (c0 + 32 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(c0 + 32), hi);
+                if (c0 + 48 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(c0 + 48), hi + 16);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float v = __shfl_sync(0xffffffffu, hi[j], u16);
+                    if (half) x[j] = v;
                 }
                 // warp q holds gate q: tanh for the cell candidate (q == 2), logistic for the other three,
                 // written as 0.5 tanh(x / 2) + 0.5 so that both are one hardware tanh
                 const float sc = q == 2 ? 1.f : 0.5f, of = q == 2 ? 0.f : 0.5f;
-                if (row_ok) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) stage_f[(q * 32 + j) * 16 + u16] = fmaf(tanh_fast((pre[j] + add[j]) * sc), sc, of);
-                }
+                for (int j = 0; j < 32; ++j) stage_f[(q * 64 + half * 32 + j) * 16 + u16] = fmaf(tanh_fast((x[j] + add[j]) * sc), sc, of);
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, 10);
             if (ready) {
 #pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                    const int j = (lane >> 4) + 2 * q + 8 * jj;
+                for (int jj = 0; jj < 8; ++jj) {
+                    const int j = half + 2 * q + 8 * jj;     // 0..63
                     const int bj = b0 + j;
-                    const int tj = __shfl_sync(0xffffffffu, tok, j);
+                    const int ta = __shfl_sync(0xffffffffu, tok_a, j & 31), tb = __shfl_sync(0xffffffffu, tok_b, j & 31);
+                    const int tj = j < 32 ? ta : tb;
                     if (c0 + j < p.nl && bj < p.B) {
                         if (tj >= 0) {
-                            const float gi = stage_f[(0 * 32 + j) * 16 + u16], gf = stage_f[(1 * 32 + j) * 16 + u16];
-                            const float gg = stage_f[(2 * 32 + j) * 16 + u16], go = stage_f[(3 * 32 + j) * 16 + u16];
+                            const float gi = stage_f[(0 * 64 + j) * 16 + u16], gf = stage_f[(1 * 64 + j) * 16 + u16];
+                            const float gg = stage_f[(2 * 64 + j) * 16 + u16], go = stage_f[(3 * 64 + j) * 16 + u16];
                             const float cc = gf * cold[jj] + gi * gg;
                             cst[(size_t)bj * p.P] = cc;
                             hout[(size_t)bj * p.P] = __float2bfloat16_rn(go * tanh_fast(cc));
@@ -688,34 +709,37 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         const int32_t* t_new = p.t2 + (size_t)((step + 1) & 1) * p.B;
         const int h0 = r_ht * 64;
         const int rows_here = p.np * p.W;          // z rows of this CTA: (utterance, window row) pairs
-        // fetch the 64 enc_proj values of z row r (8 x 16 bytes); false when the row lies outside the window
-        auto fetch = [&](int r, uint4* ev) -> bool {
+        // z row r: 0 = nothing to write (outside the batch, or the utterance is done), 1 = zeros (past the end of
+        // the utterance), 2 = act(enc_proj row + pred_proj); for 2 the row's 64 enc_proj values are fetched
+        auto fetch = [&](int r, uint4* ev) -> int {
             const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
-            if (r >= rows_here || b >= p.B) return false;
+            if (r >= rows_here || b >= p.B) return 0;
             const int t = t_new[b];
-            if (w >= min(p.W, p.enc_len[b] - t)) return false;
+            const int left = p.enc_len[b] - t;
+            if (left <= 0) return 0;
+            if (w >= left) return 1;
             const uint4* src = reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + t + w) * p.H + h0);
 #pragma unroll
             for (int k = 0; k < 8; ++k) ev[k] = src[k];
-            return true;
+            return 2;
         };
-        // z row r = act(enc_proj row + pred_proj of its utterance), or zeros outside the window
-        auto emit = [&](int r, bool have, const uint4* ev) {
+        auto emit = [&](int r, int kind, const uint4* ev) {
+            if (kind == 0) return;
             const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
-            if (r >= rows_here || b >= p.B) return;
-            if (t_new[b] >= p.enc_len[b]) return;    // utterance done: its z rows are never used again
             uint4* dst = reinterpret_cast<uint4*>(p.z + ((size_t)b * p.W + w) * p.H + h0);
-            const float* gs = stage_f + bl * 65;
+            const float4* gs = reinterpret_cast<const float4*>(stage_f + bl * 68);
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 uint4 o = make_uint4(0, 0, 0, 0);
-                if (have) {
+                if (kind == 2) {
                     const __nv_bfloat162* eb = reinterpret_cast<const __nv_bfloat162*>(&ev[k]);
+                    const float4 ga = gs[2 * k], gb = gs[2 * k + 1];
+                    const float gg[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
                     uint32_t wds[4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const float2 e2 = __bfloat1622float2(eb[i]);
-                        float z0 = e2.x + gs[k * 8 + 2 * i], z1 = e2.y + gs[k * 8 + 2 * i + 1];
+                        float z0 = e2.x + gg[2 * i], z1 = e2.y + gg[2 * i + 1];
                         z0 = p.act == WIND_ACT_RELU ? fmaxf(z0, 0.f) : tanh_fast(z0);
                         z1 = p.act == WIND_ACT_RELU ? fmaxf(z1, 0.f) : tanh_fast(z1);
                         wds[i] = pack_bf16x2(z0, z1);
@@ -727,7 +751,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         };
         // the first two z rows of this thread are requested before the accumulator is ready
         uint4 ev0[8], ev1[8];
-        const bool have0 = fetch(e, ev0), have1 = fetch(e + 128, ev1);
+        const int kind0 = fetch(e, ev0), kind1 = fetch(e + 128, ev1);
         if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
         const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[2], acc_n[2] & 1u, &s_abort));
         tc_fence_after();
@@ -740,7 +764,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                 tmem_ld16(tm_p + lane_off + (uint32_t)c0, g);
                 if (lane < 16) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) stage_f[(c0 + j) * 65 + hl] = g[j] + bias;
+                    for (int j = 0; j < 16; ++j) stage_f[(c0 + j) * 68 + hl] = g[j] + bias;
                 }
             }
         }
@@ -749,14 +773,16 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         if (lane == 0) mbar_arrive(&acc_empty[2]);
         ++acc_n[2];
         asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 10);
         if (ready) {
-            emit(e, have0, ev0);
-            emit(e + 128, have1, ev1);
+            emit(e, kind0, ev0);
+            emit(e + 128, kind1, ev1);
             for (int r = e + 256; r < rows_here; r += 128) {
-                const bool have = fetch(r, ev0);
-                emit(r, have, ev0);
+                const int kind = fetch(r, ev0);
+                emit(r, kind, ev0);
             }
         }
+        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 11);
         fence_proxy_async_all();
         if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
         return ready;
