@@ -124,6 +124,9 @@ __device__ __forceinline__ void tc_mma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a,
 
 enum { J_STREAM = 0, J_SMEM = 1, J_TMEM = 2 };   // where the joint's W_out tile lives
 
+// RES: resident-weights mode (compile-time, so that each instantiation carries only its own code paths: the loop
+// body runs once per lock step, straight through, and instruction fetch is a visible cost at that scale).
+template <bool RES>
 __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_constant__ LoopMaps M, const LoopParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[LOOP_MAX_STAGES], empty_bar[LOOP_MAX_STAGES], stat_bar;
@@ -142,13 +145,15 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
     if (threadIdx.x == 0) {
         s_abort = 0;
         s_active = 0;
+        // resident-weights mode: two threads issue the MMAs of a GEMM (each its half of the K blocks), both commit
+        const uint32_t issuers = RES ? 2u : 1u;
         for (int s = 0; s < LOOP_MAX_STAGES; ++s) {
             mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], 1);
+            mbar_init(&empty_bar[s], s == 0 ? issuers : 1u);
         }
         mbar_init(&stat_bar, 1);
         for (int k = 0; k < 3; ++k) {
-            mbar_init(&acc_full[k], 1);
+            mbar_init(&acc_full[k], issuers);
             mbar_init(&acc_empty[k], 4);
         }
         fence_barrier_init();
@@ -174,8 +179,8 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
     }
     // resident-weights mode: CTAs [0, l_items) keep a W_hh tile (4 gates x 16 units), the last p_items CTAs a W_pred
     // tile (64 rows), loaded once; `stat` holds kb_p blocks of 64 rows x 64 columns
-    const bool res_l = p.resident && cta < p.l_items;
-    const bool res_p = p.resident && !res_l && G - 1 - cta < p.p_items;
+    const bool res_l = RES && cta < p.l_items;
+    const bool res_p = RES && !res_l && G - 1 - cta < p.p_items;
     const int r_ut = cta % p.ut_count, r_ql = cta / p.ut_count;                      // unit tile / utterance group of an L CTA
     const int r_ht = (G - 1 - cta) % p.ht_count, r_qp = (G - 1 - cta) / p.ht_count;  // H tile / utterance group of a P CTA
     constexpr uint32_t RES_A_BYTES = 64 * BK * 2;
@@ -498,7 +503,10 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         tma_load_3d(dst, map, 0, row0, 0, &full_bar[0]);
         return true;
     };
-    auto mma_one = [&](int k_acc, uint32_t tm_d, int n_tile, int kbs, bool a_tmem) -> bool {
+    // One issuing thread's share of a GEMM: K blocks [kb_lo, kb_hi) into the accumulator at tm_d.  Two threads call
+    // this for every GEMM (warp 1 and, after it has issued the TMA box, warp 0), with disjoint K ranges and
+    // separate accumulator copies that the epilogue adds; an empty range only takes part in the commits.
+    auto mma_part = [&](int k_acc, uint32_t tm_d, int n_tile, int kb_lo, int kb_hi, bool a_tmem) -> bool {
         const uint32_t idesc = idesc_bf16(a_tmem ? 128 : 64, n_tile);
         if (!a_tmem && !mbar_wait(&stat_bar, 0, &s_abort)) return false;
         if (!begin_acc(k_acc)) return false;
@@ -506,17 +514,18 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         if (!consume()) return false;
         const uint32_t b_addr = smem_u32(ring);
         const uint32_t b_block = (uint32_t)n_tile * BK * 2;
-        for (int kb = 0; kb < kbs; ++kb) {
+        for (int kb = kb_lo; kb < kb_hi; ++kb) {
             const uint64_t bdesc = smem_desc_sw128(b_addr + (uint32_t)kb * b_block);
             if (a_tmem) {
 #pragma unroll
                 for (int k = 0; k < BK / 16; ++k)
-                    tc_mma_bf16_ts(tm_d, tmem_base + (uint32_t)(kb * (BK / 2) + k * 8), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+                    tc_mma_bf16_ts(tm_d, tmem_base + (uint32_t)(kb * (BK / 2) + k * 8), bdesc + (uint64_t)(k * 2), idesc,
+                                   kb != kb_lo || k != 0);
             } else {
                 const uint64_t adesc = smem_desc_sw128(smem_u32(stat + (size_t)kb * RES_A_BYTES));
 #pragma unroll
                 for (int k = 0; k < BK / 16; ++k)
-                    tc_mma_bf16(tm_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+                    tc_mma_bf16(tm_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, kb != kb_lo || k != 0);
             }
         }
         tc_commit(&empty_bar[0]);
@@ -673,7 +682,6 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                 for (int j = 0; j < 32; ++j) stage_f[(q * 64 + half * 32 + j) * 16 + u16] = fmaf(tanh_fast((x[j] + add[j]) * sc), sc, of);
             }
             asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, 10);
             if (ready) {
 #pragma unroll
                 for (int jj = 0; jj < 8; ++jj) {
@@ -760,11 +768,12 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
             const int hl = 16 * q + (lane & 15);
             const float bias = p.b_pred[h0 + hl];
             for (int c0 = 0; c0 < p.np; c0 += 16) {
-                float g[16];
+                float g[16], more[16];
                 tmem_ld16(tm_p + lane_off + (uint32_t)c0, g);
+                tmem_ld16(tm_p + lane_off + (uint32_t)(p.np + c0), more);   // the other issuing thread's K blocks
                 if (lane < 16) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) stage_f[(c0 + j) * 68 + hl] = g[j] + bias;
+                    for (int j = 0; j < 16; ++j) stage_f[(c0 + j) * 68 + hl] = g[j] + more[j] + bias;
                 }
             }
         }
@@ -773,7 +782,6 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         if (lane == 0) mbar_arrive(&acc_empty[2]);
         ++acc_n[2];
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 10);
         if (ready) {
             emit(e, kind0, ev0);
             emit(e + 128, kind1, ev1);
@@ -782,7 +790,6 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                 emit(r, kind, ev0);
             }
         }
-        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 11);
         fence_proxy_async_all();
         if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
         return ready;
@@ -792,15 +799,16 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         if (warp == 0) {
             if (lane == 0 && res_l) {
                 fence_proxy_async_all();
-                produce_one(&M.hb_l3[pin], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u);
+                if (produce_one(&M.hb_l3[pin], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u))
+                    mma_part(1, tm_l, p.nl, p.kb_p, p.kb_p, false);   // one accumulator: warp 1 issues all of it
             }
         } else if (warp == 1) {
-            if (lane == 0 && res_l) mma_one(1, tm_l, p.nl, p.kb_p, false);
+            if (lane == 0 && res_l) mma_part(1, tm_l, p.nl, 0, p.kb_p, false);
         }
     };
 
     // ----- before the loop: layer 0's GEMM on the initial (zero) state -----
-    if (p.resident) {
+    if constexpr (RES) {
         early_res();
     } else if (early) {
         if (warp == 0) {
@@ -814,7 +822,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         // =====================================================================================
         // decoder phases: control step + LSTM cell update (layer 0), then one GEMM + update phase per upper layer
         // =====================================================================================
-        if (p.resident) {
+        if constexpr (RES) {
             if (warp >= 2) {
                 if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_START);
                 if (res_l) epilogue_res_L();
@@ -822,7 +830,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
             }
             if (!grid_sync(TR_L)) goto done;
         }
-        for (int l = 0; l < p.L && !p.resident; ++l) {
+        for (int l = 0; l < p.L && !RES; ++l) {
             const bool gemm_here = l > 0 || !early;
             if (warp == 0) {
                 if (lane == 0 && gemm_here) { fence_proxy_async_all(); cur = 0; produce_L(l); }
@@ -837,7 +845,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         pin ^= 1;
         if (p.forced && step + 1 < p.U) {
             // teacher forcing: more prefix tokens to feed before the window is evaluated
-            if (p.resident) {
+            if constexpr (RES) {
                 early_res();
             } else if (early) {
                 if (warp == 0) {
@@ -859,14 +867,15 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
             const uint32_t b_bytes = (uint32_t)n_tile * BK * 2;
             const int32_t* t_new = p.t2 + (size_t)((step + 1) & 1) * p.B;
             const int i0 = p.p_items <= G ? G - 1 - cta : cta;   // projection items start at the far end of the grid
-            if (p.resident) {
+            if constexpr (RES) {
                 if (warp == 0) {
                     if (lane == 0 && res_p) {
                         fence_proxy_async_all();
-                        produce_one(&M.hb_p3[pin], r_qp * p.np, (uint32_t)p.np * (uint32_t)p.P * 2u);
+                        if (produce_one(&M.hb_p3[pin], r_qp * p.np, (uint32_t)p.np * (uint32_t)p.P * 2u))
+                            mma_part(2, tm_p + (uint32_t)p.np, p.np, p.kb_p / 2, p.kb_p, false);
                     }
                 } else if (warp == 1) {
-                    if (lane == 0 && res_p) mma_one(2, tm_p, p.np, p.kb_p, false);
+                    if (lane == 0 && res_p) mma_part(2, tm_p, p.np, 0, p.kb_p / 2, false);
                 } else {
                     if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_START);
                     int cnt = 0;
@@ -1022,16 +1031,18 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
             const int n_tile = p.nj;
             const uint32_t z_bytes = (uint32_t)n_tile * BK * 2;
             unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
-            if (p.resident && warp < 2) {
+            if (RES && warp < 2) {
                 // one box for the whole z tile, then every MMA back to back (A = W_out tile in tensor memory)
                 if (lane == 0 && has_j) {
                     if (warp == 0) {
                         fence_proxy_async_all();
                         trace_event(p, 0, tr_n, step, TR_J, EV_FIRST_ISSUE);
-                        produce_one(&M.z3, (cta / p.vt_count) * n_tile, (uint32_t)n_tile * (uint32_t)p.H * 2u);
+                        const bool ok = produce_one(&M.z3, (cta / p.vt_count) * n_tile, (uint32_t)n_tile * (uint32_t)p.H * 2u);
                         trace_event(p, 0, tr_n, step, TR_J, EV_LAST_ISSUE);
+                        if (ok) mma_part(0, tm_j + (uint32_t)n_tile, n_tile, p.kb_h / 2, p.kb_h, true);
+                        trace_event(p, 0, tr_n, step, TR_J, EV_COMMIT);
                     } else {
-                        mma_one(0, tm_j, n_tile, p.kb_h, true);
+                        mma_part(0, tm_j, n_tile, 0, p.kb_h / 2, true);
                         trace_event(p, 1, tr_n, step, TR_J, EV_COMMIT);
                     }
                 }
@@ -1111,6 +1122,17 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                             } else {
 #pragma unroll
                                 for (int j = 16; j < 32; ++j) val[j] = -INFINITY;
+                            }
+                            if (RES) {   // second accumulator copy (the other issuing thread's K blocks)
+                                float more[16];
+                                tmem_ld16(tm_j + lane_off + (uint32_t)(n_tile + c0), more);
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) val[j] += more[j];
+                                if (c0 + 16 < n_tile) {
+                                    tmem_ld16(tm_j + lane_off + (uint32_t)(n_tile + c0 + 16), more);
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) val[16 + j] += more[j];
+                                }
                             }
 #pragma unroll
                             for (int j = 0; j < 32; ++j) val[j] = v_ok ? val[j] + bias : -INFINITY;
@@ -1310,7 +1332,7 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
     // W_pred in tiles of 64 rows stay in the shared memory of disjoint CTA sets for the whole decode; per step a CTA
     // fetches only its utterance group's rows of the state, as one box.
     const char* res_env = getenv("WIND_RESIDENT");
-    if (m.L == 1 && one_wave && m.H / 2 + pl.nj <= (int)LOOP_TMEM_COLS && !(res_env && atoi(res_env) == 0)) {
+    if (m.L == 1 && one_wave && m.H / 2 + 2 * pl.nj <= (int)LOOP_TMEM_COLS && !(res_env && atoi(res_env) == 0)) {
         LoopPlan r = pl;
         r.ut_count = m.P / 16;
         r.ht_count = m.H / 64;
@@ -1342,11 +1364,11 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
             r.stages_lp = r.stages_j = 1;
             r.stage_lp = r.stage_j = 0;
             r.tm_j = m.H / 2;
-            r.tm_l = r.tm_p = r.tm_j + r.nj;
+            r.tm_l = r.tm_p = r.tm_j + 2 * r.nj;   // two copies of the joint accumulator, then decoder / projection
             r.l_items = r.ut_count * r.ql_count;
             r.p_items = r.ht_count * r.qp_count;
             r.l_early = 1;
-            const int acc_cols = r.nl > r.np ? r.nl : r.np;
+            const int acc_cols = r.nl > 2 * r.np ? r.nl : 2 * r.np;
             if ((long long)r.smem_bytes <= (long long)budget + 1024 && r.tm_l + acc_cols <= (int)LOOP_TMEM_COLS) pl = r;
         }
     }
@@ -1386,7 +1408,9 @@ cudaError_t loop_prepare(Call& c) {
     {
         std::lock_guard<std::mutex> lock(g_loop_mutex);
         if ((int)pl.smem_bytes > g_attr_smem) {
-            e = cudaFuncSetAttribute(loop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
+            e = cudaFuncSetAttribute(loop_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
+            if (e != cudaSuccess) return e;
+            e = cudaFuncSetAttribute(loop_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
             if (e != cudaSuccess) return e;
             g_attr_smem = (int)pl.smem_bytes;
         }
@@ -1421,7 +1445,7 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.forced = logits_out != nullptr; p.prefix = prefix; p.U = U; p.prefix_len = prefix_len; p.logits_out = logits_out;
     p.trace = trace_step >= -1 ? c.trace() : nullptr; p.trace_step = trace_step;
     void* args[2] = {(void*)&t_loop_maps, (void*)&p};
-    return cudaLaunchCooperativeKernel((const void*)loop_kernel, dim3((unsigned)pl.grid), dim3(LOOP_THREADS), args, pl.smem_bytes,
+    return cudaLaunchCooperativeKernel(pl.resident ? (const void*)loop_kernel<true> : (const void*)loop_kernel<false>, dim3((unsigned)pl.grid), dim3(LOOP_THREADS), args, pl.smem_bytes,
                                        c.stream);
 }
 
