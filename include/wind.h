@@ -199,10 +199,11 @@ wind_status_t wind_eval_joint_window_static(const wind_model_t* m, const void* e
 typedef struct {
     double enc_proj_ms, joint_ms, control_ms, pred_ms;
     int64_t enc_proj_launches, joint_launches, control_launches, pred_launches;
-    /* tensor-core path only (zero otherwise): the decoding loop is one persistent kernel, so the
-     * figures above are its phases, timed from inside the kernel; loop_ms is its wall time,
-     * lstm_ms + proj_ms = pred_ms */
-    double loop_ms, lstm_ms, proj_ms;
+    /* tensor-core path only (zero otherwise): the decoding loop is one persistent kernel; loop_ms is its
+     * duration between two CUDA events, split into joint_ms + lstm_ms + proj_ms (= pred_ms) in proportion to
+     * the SM cycles its first CTA spent in each phase (barrier waits included); gate_table_ms is the one-shot
+     * GEMM that tabulates layer 0's input term for every token */
+    double loop_ms, lstm_ms, proj_ms, gate_table_ms;
 } wind_profile_t;
 
 /*

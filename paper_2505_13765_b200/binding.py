@@ -64,7 +64,7 @@ class wind_profile_t(C.Structure):
         ("enc_proj_ms", C.c_double), ("joint_ms", C.c_double), ("control_ms", C.c_double), ("pred_ms", C.c_double),
         ("enc_proj_launches", C.c_int64), ("joint_launches", C.c_int64), ("control_launches", C.c_int64),
         ("pred_launches", C.c_int64),
-        ("loop_ms", C.c_double), ("lstm_ms", C.c_double), ("proj_ms", C.c_double),
+        ("loop_ms", C.c_double), ("lstm_ms", C.c_double), ("proj_ms", C.c_double), ("gate_table_ms", C.c_double),
     ]
 
 

@@ -385,36 +385,39 @@ wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const 
     if (c.m.dtype == WIND_DT_BF16 && g_kernels == WIND_KERNELS_TENSOR && !tensor) return WIND_ERR_UNSUPPORTED;
     memset(host_out, 0, sizeof(*host_out));
     if (tensor) {
-        // the loop is one kernel: its phases are timed from inside (SM cycles of CTA 0, scaled by the
-        // kernel's wall time from the global timer); the projection is bracketed by events as usual
-        cudaEvent_t e0, e1;
-        WIND_CUDA(cudaEventCreate(&e0));
-        WIND_CUDA(cudaEventCreate(&e1));
+        // every kernel is bracketed by CUDA events on the stream; the loop is one kernel, so its phases are
+        // split by the SM cycles CTA 0 counted in each of them
+        cudaEvent_t ev[4];
+        for (auto& e : ev) WIND_CUDA(cudaEventCreate(&e));
         WIND_CUDA(tc_prepare(c));
         WIND_CUDA(launch_init(c, WIND_KERNELS_TENSOR, 0, tc_setup_launches(c)));
-        WIND_CUDA(cudaEventRecord(e0, c.stream));
+        WIND_CUDA(cudaEventRecord(ev[0], c.stream));
         WIND_CUDA(tc_enc_proj(c));
-        WIND_CUDA(cudaEventRecord(e1, c.stream));
+        WIND_CUDA(cudaEventRecord(ev[1], c.stream));
         WIND_CUDA(tc_gate_table(c));
+        WIND_CUDA(cudaEventRecord(ev[2], c.stream));
         WIND_CUDA(tc_loop(c, nullptr, 0, nullptr, nullptr, g_trace_step));
+        WIND_CUDA(cudaEventRecord(ev[3], c.stream));
         Ctrl hc;
         WIND_CUDA(cudaMemcpyAsync(&hc, c.ctrl(), sizeof(Ctrl), cudaMemcpyDeviceToHost, c.stream));
         WIND_CUDA(cudaStreamSynchronize(c.stream));
-        float ms = 0.f;
-        cudaEventElapsedTime(&ms, e0, e1);
-        cudaEventDestroy(e0);
-        cudaEventDestroy(e1);
-        host_out->enc_proj_ms = ms;
+        float ms_proj = 0.f, ms_table = 0.f, ms_loop = 0.f;
+        cudaEventElapsedTime(&ms_proj, ev[0], ev[1]);
+        cudaEventElapsedTime(&ms_table, ev[1], ev[2]);
+        cudaEventElapsedTime(&ms_loop, ev[2], ev[3]);
+        for (auto& e : ev) cudaEventDestroy(e);
+        host_out->enc_proj_ms = ms_proj;
         host_out->enc_proj_launches = 1;
+        host_out->gate_table_ms = ms_table;
         const double cyc = (double)(hc.phase_cycles[0] + hc.phase_cycles[1] + hc.phase_cycles[2]);
-        const double ms_per_cycle = cyc > 0 ? (double)hc.loop_ns * 1e-6 / cyc : 0.0;
+        const double ms_per_cycle = cyc > 0 ? (double)ms_loop / cyc : 0.0;
         host_out->joint_ms = hc.phase_cycles[0] * ms_per_cycle;
         host_out->pred_ms = (hc.phase_cycles[1] + hc.phase_cycles[2]) * ms_per_cycle;
         host_out->control_ms = 0.0;   // the control step runs inside the decoder-update phase
         host_out->joint_launches = hc.step;       // phases, not launches: one joint phase per lock step
         host_out->pred_launches = hc.step + 1;
         host_out->control_launches = 0;
-        host_out->loop_ms = (double)hc.loop_ns * 1e-6;
+        host_out->loop_ms = ms_loop;
         host_out->lstm_ms = hc.phase_cycles[1] * ms_per_cycle;
         host_out->proj_ms = hc.phase_cycles[2] * ms_per_cycle;
         return (wind_status_t)hc.status;

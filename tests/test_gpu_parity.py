@@ -259,6 +259,57 @@ def test_cfg3_full_batch_sampled_utterances(pkg):
         assert np.all((tok[b, : olen[b]] >= 0) & (tok[b, : olen[b]] < cfg.V))
 
 
+def test_bf16_tensor_path_is_window_invariant_on_the_gpu(pkg):
+    # A window row's logits come from the same operands in the same order whatever W is, so the tensor-core path
+    # must emit the same (token, frame) sequences for every window size, bit for bit (the paper's claim that
+    # WIND leaves the result unchanged, here for the GPU path by itself).
+    cfg = ws.small_variant(ws.CONFIGS["cfg3_large_b128"], 12, 5, 140)
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="nan")
+    model = pkg.WindModel(weights)
+    ref = None
+    for W in (1, 2, 4, 8, 16, 64):
+        tok, frm, olen, stats, st = pkg.decode(model, enc, lens, W, cfg.S)
+        assert st == 0 and stats["kernels"] == 2
+        if ref is None:
+            ref = (tok, frm, olen)
+        else:
+            assert np.array_equal(olen, ref[2]), W
+            assert np.array_equal(tok, ref[0]) and np.array_equal(frm, ref[1]), W
+
+
+def test_loop_kernel_timeline_can_be_recorded_without_changing_results(pkg):
+    cfg = ws.small_variant(ws.CONFIGS["cfg3_large_b128"], 8, 30, 80)
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="zero")
+    model = pkg.WindModel(weights)
+    d = model.device
+    B, T, _ = enc.shape
+    max_out = T * cfg.S
+    enc_d = pkg.to_device_enc(model, enc)
+    len_d = torch.from_numpy(lens).to(d)
+    outs = []
+    wsb = pkg.alloc_workspace(model, B, T, cfg.W)
+    for first in (-2, 3):
+        tok = torch.full((B, max_out), -1, dtype=torch.int32, device=d)
+        frm = tok.clone()
+        ol = torch.zeros(B, dtype=torch.int32, device=d)
+        prev = pkg.wind_set_trace(first)
+        try:
+            pkg.wind_decode_greedy(model, enc_d, len_d, cfg.W, cfg.S, tok, frm, ol, wsb)
+        finally:
+            pkg.wind_set_trace(prev)
+        outs.append((tok.cpu().numpy(), frm.cpu().numpy(), ol.cpu().numpy()))
+        ev = pkg.wind_read_trace(model, B, T, cfg.W, wsb)
+        if first < -1:
+            assert ev == []
+        else:
+            assert ev and {e["step"] for e in ev} <= {3, 4}
+            assert {e["phase"] for e in ev} == {0, 1, 2} and all(0 <= e["role"] < 8 and e["clock"] > 0 for e in ev)
+    for a, b in zip(outs[0], outs[1]):
+        assert np.array_equal(a, b)
+
+
 # ---------------------------------------------------------------------------
 # behaviour of the interface
 # ---------------------------------------------------------------------------
