@@ -37,7 +37,8 @@
 
 namespace wind {
 
-constexpr int LOOP_THREADS = 192;
+constexpr int LOOP_THREADS = 192;       // streaming mode: TMA warp, MMA warp, 4 epilogue warps
+constexpr int LOOP_THREADS_RES = 320;   // resident-weights mode: 8 epilogue warps (two per tensor-memory lane quadrant)
 constexpr int LOOP_MAX_STAGES = 28;
 constexpr uint32_t LOOP_A_BYTES = 128 * BK * 2;  // one K block of a 128-row operand tile
 constexpr uint32_t LOOP_TMEM_COLS = 512;
@@ -127,14 +128,14 @@ enum { J_STREAM = 0, J_SMEM = 1, J_TMEM = 2 };   // where the joint's W_out tile
 // RES: resident-weights mode (compile-time, so that each instantiation carries only its own code paths: the loop
 // body runs once per lock step, straight through, and instruction fetch is a visible cost at that scale).
 template <bool RES>
-__global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_constant__ LoopMaps M, const LoopParams p) {
+__global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop_kernel(const __grid_constant__ LoopMaps M, const LoopParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[LOOP_MAX_STAGES], empty_bar[LOOP_MAX_STAGES], stat_bar;
     __shared__ uint64_t acc_full[3], acc_empty[3];   // accumulators: joint, decoder, projection
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;      // this CTA has given up
     __shared__ int s_active;     // utterances still decoding (set in the projection phase)
-    __shared__ int s_red[4];
+    __shared__ int s_red[8];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cta = blockIdx.x, G = gridDim.x;
@@ -154,7 +155,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         mbar_init(&stat_bar, 1);
         for (int k = 0; k < 3; ++k) {
             mbar_init(&acc_full[k], issuers);
-            mbar_init(&acc_empty[k], 4);
+            mbar_init(&acc_empty[k], RES ? 8u : 4u);   // one arrival per epilogue warp
         }
         fence_barrier_init();
     }
@@ -165,7 +166,8 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
     const uint32_t tmem_base = tmem_slot;
     const uint32_t tm_j = tmem_base + (uint32_t)p.tm_j, tm_l = tmem_base + (uint32_t)p.tm_l, tm_p = tmem_base + (uint32_t)p.tm_p;
 
-    const int e = threadIdx.x - 64;            // epilogue thread 0..127 (warps 2..5)
+    const int e = threadIdx.x - 64;            // epilogue thread: 0..127 (warps 2..5), 0..255 (warps 2..9) in resident mode
+    const int sub = (warp - 2) >> 2;           // resident mode: which of the two warps of a lane quadrant (0 otherwise)
     const int q = warp & 3;                    // tensor-memory lane quadrant of this warp
     const int row_in_tile = q * 32 + lane;     // the tensor-memory lane (accumulator row) of this thread
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
@@ -534,9 +536,9 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         return true;
     };
     // control step + LSTM cell update of an L CTA: units [r_ut*16, +16), utterances [r_ql*nl, +nl), 64 utterances per
-    // pass.  All global reads of a pass are requested together: first everything the control step needs, then the
-    // gate-table rows of the chosen tokens; lanes 16..31 of a warp hold no accumulator row (64-row tile), so they
-    // take the second 32 utterances of the pass.
+    // pass.  Warp (q, sub) of the epilogue owns gate q and the pass's utterances [32 sub, 32 sub + 32).  All global reads
+    // of a pass are requested together: first everything the control step needs, then the gate-table rows of the
+    // chosen tokens.  Lanes 16..31 hold no accumulator row (64-row tile); they take the second 16 utterances.
     struct ScanIn { int t, len, cnt, pos; unsigned long long kk[8]; };
     auto epilogue_res_L = [&]() -> bool {
         const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
@@ -545,14 +547,21 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
         const int u16 = lane & 15, half = lane >> 4;
         const int unit = r_ut * 16 + u16;        // this thread's hidden unit; its gate is q
-        const bool writer = r_ut == 0 && q == 0; // one warp per utterance group records the step
+        const bool writer = r_ut == 0 && q == 0; // the two gate-0 warps of one CTA per utterance group record the step
         const bool decode = step >= 0 && !p.forced;
         float* cst = p.c_state + unit;
         const __nv_bfloat16* hin = p.hb + ((size_t)pin * p.Bpad) * p.P + unit;
         __nv_bfloat16* hout = p.hb + ((size_t)(pin ^ 1) * p.Bpad) * p.P + unit;
         const float* g0u = p.g0 + (size_t)q * p.P + unit;
         const uint32_t g0_stride = 4u * (uint32_t)p.P;
-        auto scan_load = [&](int b, bool in, ScanIn& si) {
+        bool ready = true;
+        for (int c0 = 0; c0 < p.nl; c0 += 64) {
+            const int b0 = r_ql * p.nl + c0;
+            // ---- lane j decides for utterance b0 + 32 sub + j ----
+            const int jl = 32 * sub + lane;
+            const int b = b0 + jl;
+            const bool in = c0 + jl < p.nl && b < p.B;
+            ScanIn si;
             si.t = 0; si.len = 0; si.cnt = 0; si.pos = 0;
 #pragma unroll
             for (int j = 0; j < 8; ++j) si.kk[j] = 0ull;
@@ -564,114 +573,107 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                 for (int j = 0; j < 8; ++j)
                     if (j < p.W) si.kk[j] = keys_cur[(size_t)b * p.W + j];
             }
-        };
-        // the token utterance b feeds to its decoder in this step (-1: none); the writer warp also records the step
-        auto scan_decide = [&](int b, bool in, ScanIn& si) -> int {
-            if (!in) return -1;
-            if (step < 0) return p.blank;
-            if (p.forced) return step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
-            int t = si.t, tok = -1;
-            const int len = si.len;
-            if (t < len) {
-                // control step (Algorithm 2's branch): first non-blank row of the window
-                const int n = min(p.W, len - t);
-                int first = -1, label = p.blank;
-                bool bad = false;
-                for (int w0 = 0; w0 < n && first < 0; w0 += 8) {
-                    if (w0 > 0) {
+            // old cell state of the four (utterance, unit) pairs this thread finishes
+            float cold[4];
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) si.kk[j] = (w0 + j < n) ? keys_cur[(size_t)b * p.W + w0 + j] : 0ull;
-                    }
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (w0 + j < n && first < 0) {
-                            uint32_t lab = key_label(si.kk[j]);
-                            if (si.kk[j] == 0ull || lab >= (uint32_t)p.NV) { bad = true; lab = (uint32_t)p.blank; }
-                            if ((int)lab != p.blank) { first = w0 + j; label = (int)lab; }
-                        }
-                    }
-                }
-                if (first >= 0) tok = label;
-                if (writer) {
-                    int cnt = si.cnt, jump, forced = 0, emitted = 0;
-                    if (first < 0) {
-                        jump = n;
-                        t += n;
-                        cnt = 0;
-                    } else {
-                        jump = first;
-                        if (first > 0) cnt = 0;
-                        t += first;
-                        if (si.pos < p.max_out) {
-                            p.out_tokens[(size_t)b * p.max_out + si.pos] = label;
-                            p.out_frames[(size_t)b * p.max_out + si.pos] = t;
-                            p.out_len[b] = si.pos + 1;
-                            emitted = 1;
-                            cnt += 1;
-                            if (cnt == p.S) { t += 1; cnt = 0; forced = 1; }
-                        } else {
-                            set_status(p.ctrl, WIND_ERR_OUTPUT_OVERFLOW);  // this utterance stops here
-                            t = len;
-                            tok = -1;
-                        }
-                    }
-                    if (bad) set_status(p.ctrl, WIND_ERR_INTERNAL);
-                    t_nxt[b] = t;
-                    p.count[b] = cnt;
-                    for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
-                    atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
-                    atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->joint_rows), (unsigned long long)n);
-                    if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
-                    if (forced) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
-                }
-            } else if (writer) {
-                t_nxt[b] = t;
-            }
-            return tok;
-        };
-        bool ready = true;
-        for (int c0 = 0; c0 < p.nl; c0 += 64) {
-            const int b0 = r_ql * p.nl + c0;
-            // ---- lane j decides for utterances b0 + j and b0 + 32 + j ----
-            const int ba = b0 + lane, bb = b0 + 32 + lane;
-            const bool in_a = c0 + lane < p.nl && ba < p.B, in_b = c0 + 32 + lane < p.nl && bb < p.B;
-            ScanIn sa, sb;
-            scan_load(ba, in_a, sa);
-            scan_load(bb, in_b, sb);
-            // old cell state of the eight (utterance, unit) pairs this thread finishes
-            float cold[8];
-#pragma unroll
-            for (int jj = 0; jj < 8; ++jj) {
-                const int j = half + 2 * q + 8 * jj;
+            for (int jj = 0; jj < 4; ++jj) {
+                const int j = half + 2 * q + 8 * sub + 16 * jj;     // 0..63 over the CTA's 256 epilogue threads
                 cold[jj] = (c0 + j < p.nl && b0 + j < p.B) ? cst[(size_t)(b0 + j) * p.P] : 0.f;
             }
-            const int tok_a = scan_decide(ba, in_a, sa);
-            const int tok_b = scan_decide(bb, in_b, sb);
-            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
-            // ---- gate-table entries (this thread's gate and unit) of the tokens of this lane half's 32 utterances ----
-            float add[32];
+            // the token utterance b feeds to its decoder in this step (-1: none)
+            int tok = -1;
+            if (in) {
+                if (step < 0) {
+                    tok = p.blank;
+                } else if (p.forced) {
+                    tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
+                } else {
+                    int t = si.t;
+                    const int len = si.len;
+                    if (t < len) {
+                        // control step (Algorithm 2's branch): first non-blank row of the window
+                        const int n = min(p.W, len - t);
+                        int first = -1, label = p.blank;
+                        bool bad = false;
+                        for (int w0 = 0; w0 < n && first < 0; w0 += 8) {
+                            if (w0 > 0) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const int ta = __shfl_sync(0xffffffffu, tok_a, j), tb = __shfl_sync(0xffffffffu, tok_b, j);
+                                for (int j = 0; j < 8; ++j) si.kk[j] = (w0 + j < n) ? keys_cur[(size_t)b * p.W + w0 + j] : 0ull;
+                            }
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                if (w0 + j < n && first < 0) {
+                                    uint32_t lab = key_label(si.kk[j]);
+                                    if (si.kk[j] == 0ull || lab >= (uint32_t)p.NV) { bad = true; lab = (uint32_t)p.blank; }
+                                    if ((int)lab != p.blank) { first = w0 + j; label = (int)lab; }
+                                }
+                            }
+                        }
+                        if (first >= 0) tok = label;
+                        if (writer) {
+                            int cnt = si.cnt, jump, forced = 0, emitted = 0;
+                            if (first < 0) {
+                                jump = n;
+                                t += n;
+                                cnt = 0;
+                            } else {
+                                jump = first;
+                                if (first > 0) cnt = 0;
+                                t += first;
+                                if (si.pos < p.max_out) {
+                                    p.out_tokens[(size_t)b * p.max_out + si.pos] = label;
+                                    p.out_frames[(size_t)b * p.max_out + si.pos] = t;
+                                    p.out_len[b] = si.pos + 1;
+                                    emitted = 1;
+                                    cnt += 1;
+                                    if (cnt == p.S) { t += 1; cnt = 0; forced = 1; }
+                                } else {
+                                    set_status(p.ctrl, WIND_ERR_OUTPUT_OVERFLOW);  // this utterance stops here
+                                    t = len;
+                                    tok = -1;
+                                }
+                            }
+                            if (bad) set_status(p.ctrl, WIND_ERR_INTERNAL);
+                            t_nxt[b] = t;
+                            p.count[b] = cnt;
+                            for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
+                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
+                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->joint_rows), (unsigned long long)n);
+                            if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
+                            if (forced) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
+                        }
+                    } else if (writer) {
+                        t_nxt[b] = t;
+                    }
+                }
+            }
+            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
+            // ---- gate-table entries (this thread's gate and unit) of the tokens of this lane half's 16 utterances ----
+            float add[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int ta = __shfl_sync(0xffffffffu, tok, j), tb = __shfl_sync(0xffffffffu, tok, 16 + j);
                 const int tj = half ? tb : ta;
                 add[j] = tj >= 0 ? g0u[(uint32_t)tj * g0_stride] : 0.f;
             }
+            // the other warps need the tokens for the cell update below: through shared memory
+            int* tok_s = reinterpret_cast<int*>(stage_f + 4 * 64 * 16);
+            if (q == 0) tok_s[jl] = tok;
             if (c0 == 0) {
                 ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, &s_abort));
                 tc_fence_after();
                 if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
             }
             if (ready) {
-                // lanes 0..15 read their row's 64 columns; columns 32..63 then move to lanes 16..31
-                float x[32], hi[32];
+                // lanes 0..15 read their row's 32 columns; columns 16..31 then move to lanes 16..31
+                float x[16], hi[16];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) { x[j] = 0.f; hi[j] = 0.f; }
-                tmem_ld16(tm_l + lane_off + (uint32_t)c0, x);
-                if (c0 + 16 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(c0 + 16), x + 16);
-                if (c0 + 32 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(c0 + 32), hi);
-                if (c0 + 48 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(c0 + 48), hi + 16);
+                for (int j = 0; j < 16; ++j) { x[j] = 0.f; hi[j] = 0.f; }
+                const int col = c0 + 32 * sub;
+                if (col < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)col, x);
+                if (col + 16 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(col + 16), hi);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
+                for (int j = 0; j < 16; ++j) {
                     const float v = __shfl_sync(0xffffffffu, hi[j], u16);
                     if (half) x[j] = v;
                 }
@@ -679,18 +681,17 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                 // written as 0.5 tanh(x / 2) + 0.5 so that both are one hardware tanh
                 const float sc = q == 2 ? 1.f : 0.5f, of = q == 2 ? 0.f : 0.5f;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) stage_f[(q * 64 + half * 32 + j) * 16 + u16] = fmaf(tanh_fast((x[j] + add[j]) * sc), sc, of);
+                for (int j = 0; j < 16; ++j)
+                    stage_f[(q * 64 + 32 * sub + 16 * half + j) * 16 + u16] = fmaf(tanh_fast((x[j] + add[j]) * sc), sc, of);
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             if (ready) {
 #pragma unroll
-                for (int jj = 0; jj < 8; ++jj) {
-                    const int j = half + 2 * q + 8 * jj;     // 0..63
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = half + 2 * q + 8 * sub + 16 * jj;     // 0..63
                     const int bj = b0 + j;
-                    const int ta = __shfl_sync(0xffffffffu, tok_a, j & 31), tb = __shfl_sync(0xffffffffu, tok_b, j & 31);
-                    const int tj = j < 32 ? ta : tb;
                     if (c0 + j < p.nl && bj < p.B) {
-                        if (tj >= 0) {
+                        if (tok_s[j] >= 0) {
                             const float gi = stage_f[(0 * 64 + j) * 16 + u16], gf = stage_f[(1 * 64 + j) * 16 + u16];
                             const float gg = stage_f[(2 * 64 + j) * 16 + u16], go = stage_f[(3 * 64 + j) * 16 + u16];
                             const float cc = gf * cold[jj] + gi * gg;
@@ -702,7 +703,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                     }
                 }
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
         }
         tc_fence_before();
         __syncwarp();
@@ -757,9 +758,9 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                 dst[k] = o;
             }
         };
-        // the first two z rows of this thread are requested before the accumulator is ready
-        uint4 ev0[8], ev1[8];
-        const int kind0 = fetch(e, ev0), kind1 = fetch(e + 128, ev1);
+        // the first z row of this thread is requested before the accumulator is ready
+        uint4 ev0[8];
+        const int kind0 = fetch(e, ev0);
         if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
         const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[2], acc_n[2] & 1u, &s_abort));
         tc_fence_after();
@@ -767,7 +768,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         if (ready) {
             const int hl = 16 * q + (lane & 15);
             const float bias = p.b_pred[h0 + hl];
-            for (int c0 = 0; c0 < p.np; c0 += 16) {
+            for (int c0 = 16 * sub; c0 < p.np; c0 += 32) {
                 float g[16], more[16];
                 tmem_ld16(tm_p + lane_off + (uint32_t)c0, g);
                 tmem_ld16(tm_p + lane_off + (uint32_t)(p.np + c0), more);   // the other issuing thread's K blocks
@@ -781,11 +782,10 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[2]);
         ++acc_n[2];
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (ready) {
             emit(e, kind0, ev0);
-            emit(e + 128, kind1, ev1);
-            for (int r = e + 256; r < rows_here; r += 128) {
+            for (int r = e + 256; r < rows_here; r += 256) {
                 const int kind = fetch(r, ev0);
                 emit(r, kind, ev0);
             }
@@ -879,12 +879,12 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                 } else {
                     if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_START);
                     int cnt = 0;
-                    for (int b = e; b < p.B; b += 128) cnt += t_new[b] < p.enc_len[b];
+                    for (int b = e; b < p.B; b += 256) cnt += t_new[b] < p.enc_len[b];
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
                     if (lane == 0) s_red[warp - 2] = cnt;
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                    if (e == 0) s_active = s_red[0] + s_red[1] + s_red[2] + s_red[3];
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    if (e == 0) s_active = s_red[0] + s_red[1] + s_red[2] + s_red[3] + s_red[4] + s_red[5] + s_red[6] + s_red[7];
                     if (res_p) epilogue_res_P();
                 }
                 early_res();
@@ -1114,7 +1114,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                     tc_fence_after();
                     if (e == 0) trace_event(p, 2, tr_n, step, TR_J, EV_ACC);
                     if (ready) {
-                        for (int c0 = 0; c0 < n_tile; c0 += 32) {
+                        for (int c0 = RES ? 32 * sub : 0; c0 < n_tile; c0 += RES ? 64 : 32) {
                             float val[32];
                             tmem_ld16(tm_j + lane_off + (uint32_t)c0, val);
                             if (c0 + 16 < n_tile) {
@@ -1445,7 +1445,7 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.forced = logits_out != nullptr; p.prefix = prefix; p.U = U; p.prefix_len = prefix_len; p.logits_out = logits_out;
     p.trace = trace_step >= -1 ? c.trace() : nullptr; p.trace_step = trace_step;
     void* args[2] = {(void*)&t_loop_maps, (void*)&p};
-    return cudaLaunchCooperativeKernel(pl.resident ? (const void*)loop_kernel<true> : (const void*)loop_kernel<false>, dim3((unsigned)pl.grid), dim3(LOOP_THREADS), args, pl.smem_bytes,
+    return cudaLaunchCooperativeKernel(pl.resident ? (const void*)loop_kernel<true> : (const void*)loop_kernel<false>, dim3((unsigned)pl.grid), dim3(pl.resident ? LOOP_THREADS_RES : LOOP_THREADS), args, pl.smem_bytes,
                                        c.stream);
 }
 
