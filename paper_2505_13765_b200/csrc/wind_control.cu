@@ -6,7 +6,7 @@
 namespace wind {
 
 // Reset all per-call state.  Block 0 also fills the control block.
-__global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, int32_t* count, int32_t* emit_tok,
+__global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsigned long long* t_pub, int32_t* count, int32_t* emit_tok,
                                                    unsigned long long* keys, float* h, float* c, uint32_t* hb, uint32_t* z,
                                                    uint32_t* trace, size_t n_trace_words, int32_t* out_len, const int32_t* __restrict__ enc_len, int B, size_t n_keys,
                                                    size_t n_h, size_t n_c, size_t n_hb_words, size_t n_z_words,
@@ -23,6 +23,7 @@ __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, int32
     for (size_t i = gtid; i < (size_t)B; i += gstride) {
         t[i] = 0;
         t[B + i] = 0;
+        t_pub[i] = 0ull;
         count[i] = 0;
         emit_tok[i] = blank;  // start of sequence: every decoder is fed the blank id once
         out_len[i] = 0;
@@ -76,7 +77,7 @@ cudaError_t launch_init(const Call& c, int kernels_used, int launches_per_step, 
     int blocks = (int)((biggest + 255) / 256);
     if (blocks > 592) blocks = 592;
     if (blocks < 1) blocks = 1;
-    init_kernel<<<blocks, 256, 0, c.stream>>>(c.ctrl(), c.t(), c.count(), c.emit_tok(), c.keys(), c.h(0), c.c(),
+    init_kernel<<<blocks, 256, 0, c.stream>>>(c.ctrl(), c.t(), c.t_pub(), c.count(), c.emit_tok(), c.keys(), c.h(0), c.c(),
                                               reinterpret_cast<uint32_t*>(c.hb(0, 0)), reinterpret_cast<uint32_t*>(c.z()),
                                               reinterpret_cast<uint32_t*>(c.trace()),
                                               bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents / 4 : 0, c.out_len, c.enc_len, c.B, 2 * (size_t)c.lay.rows_pad, n_h, n_c, n_hb_words,

@@ -49,6 +49,7 @@ struct Ctrl {
 struct Layout {
     size_t ctrl;       // Ctrl
     size_t t;          // int32 [2][B] current frame per utterance (the loop kernel ping-pongs by step parity)
+    size_t t_pub;      // uint64 [B]  (lock step + 2) << 32 | next frame: published early in a step for the projection CTAs
     size_t count;      // int32 [B]   consecutive emissions on the current frame
     size_t emit_tok;   // int32 [B]   token to feed to the decoder this step, -1 = none
     size_t keys;       // uint64 [2][rows_pad] packed (logit, label) argmax keys, 0 = empty (second half: loop kernel)
@@ -78,6 +79,7 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     const bool bf = m.dtype == WIND_DT_BF16;
     L.rows_pad = (int32_t)(((size_t)B * W + 255) / 256 * 256);
     L.t = take(sizeof(int32_t) * 2 * B);
+    L.t_pub = take(sizeof(uint64_t) * B);
     L.count = take(sizeof(int32_t) * B);
     L.emit_tok = take(sizeof(int32_t) * B);
     L.keys = take(sizeof(uint64_t) * 2 * (size_t)L.rows_pad);
@@ -120,6 +122,7 @@ struct Call {
 
     Ctrl* ctrl() const { return reinterpret_cast<Ctrl*>(ws + lay.ctrl); }
     int32_t* t() const { return reinterpret_cast<int32_t*>(ws + lay.t); }   // [2][B]; the per-phase kernels use [0]
+    unsigned long long* t_pub() const { return reinterpret_cast<unsigned long long*>(ws + lay.t_pub); }
     int32_t* count() const { return reinterpret_cast<int32_t*>(ws + lay.count); }
     int32_t* emit_tok() const { return reinterpret_cast<int32_t*>(ws + lay.emit_tok); }
     unsigned long long* keys() const { return reinterpret_cast<unsigned long long*>(ws + lay.keys); }  // [2][rows_pad]

@@ -95,7 +95,9 @@ __device__ __forceinline__ void trace_event(const LoopParams& p, int role, int& 
         TraceEvent t;
         t.tag = (uint32_t)(phase * 16 + ev);
         t.step = step;
-        t.clock = clock64();
+        long long now;
+        asm volatile("mov.u64 %0, %%clock64;" : "=l"(now)::"memory");   // not to be moved across the memory operations around it
+        t.clock = now;
         p.trace[role * kTraceEvents + n] = t;
         ++n;
     }
@@ -581,7 +583,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 cold[jj] = (c0 + j < p.nl && b0 + j < p.B) ? cst[(size_t)(b0 + j) * p.P] : 0.f;
             }
             // the token utterance b feeds to its decoder in this step (-1: none)
-            int tok = -1;
+            int tok = -1, t_out = 0;
             if (in) {
                 if (step < 0) {
                     tok = p.blank;
@@ -635,6 +637,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                             }
                             if (bad) set_status(p.ctrl, WIND_ERR_INTERNAL);
                             t_nxt[b] = t;
+                            t_out = t;
                             p.count[b] = cnt;
                             for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
                             atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
@@ -644,8 +647,12 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                         }
                     } else if (writer) {
                         t_nxt[b] = t;
+                        t_out = t;
                     }
                 }
+                // the next frame goes out at once, stamped with the step, for the projection CTAs (which fetch their
+                // enc_proj rows while this phase is still running)
+                if (writer && !p.forced) p.t_pub[b] = ((unsigned long long)(uint32_t)(step + 2) << 32) | (uint32_t)t_out;
             }
             if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
             // ---- gate-table entries (this thread's gate and unit) of the tokens of this lane half's 16 utterances ----
@@ -713,61 +720,132 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_EPI_DONE);
         return ready;
     };
+    // z rows of a P CTA: row r = (utterance bl = r / W of the CTA's group, window row w = r % W), 64 columns = 128 bytes =
+    // eight 16-byte chunks.  Thread e owns chunk (e & 7) of rows (e >> 3) + 32 i, so that eight neighbouring lanes
+    // read and write one whole 128-byte row segment.  Row kinds: 0 nothing to write (outside the batch, or the
+    // utterance is done), 1 zeros (past the utterance's end), 2 act(enc_proj row + pred_proj).
+    //
+    // During the decoder-update phase a P CTA has nothing else to do: it waits for the next frame of its
+    // utterances to be published and starts copying the enc_proj chunks of its first 256 rows into a shared-memory
+    // stash (asynchronous copies, collected in the projection epilogue).  pre_kinds: 2 bits per row, -1 = no prefetch.
+    uint8_t* stash = ring + (size_t)p.np * p.P * 2;   // behind the projection's own operand box
+    int pre_kinds = -1;
+    const int p_chunk = e & 7, p_row0 = e >> 3;
+    // the (utterance, window row) of this thread's first eight rows never changes: worked out once, so that the
+    // per-step code has no integer division; -1 = no such row
+    int p_bw[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        p_bw[i] = -1;
+        if (res_p && e >= 0) {
+            const int r = p_row0 + 32 * i;
+            const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
+            if (r < p.np * p.W && b < p.B) p_bw[i] = (b << 8) | w;
+        }
+    }
+    // b_pred of this thread's accumulator row: constant for the whole decode, read once
+    const float p_bias = (res_p && e >= 0) ? p.b_pred[r_ht * 64 + 16 * q + (lane & 15)] : 0.f;
+    // kind of a row at frame position t of its utterance, and the row's enc_proj frame
+    auto row_kind = [&](int b, int w, int t, int& frame) -> int {
+        const int left = p.enc_len[b] - t;
+        frame = t + w;
+        return left <= 0 ? 0 : (w >= left ? 1 : 2);
+    };
+    auto prefetch_res_P = [&]() {
+        pre_kinds = -1;
+        if (p.forced) return;
+        const uint32_t want = (uint32_t)(step + 2);
+        // the published frames of this thread's rows, all requested together, until every stamp is this step's
+        unsigned long long v[8];
+        unsigned long long t0 = 0;
+        for (uint32_t it = 1;; ++it) {
+            bool all = true;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                v[i] = (unsigned long long)want << 32;
+                if (p_bw[i] >= 0) asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(v[i]) : "l"(p.t_pub + (p_bw[i] >> 8)) : "memory");
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) all = all && (uint32_t)(v[i] >> 32) == want;
+            if (all) break;
+            if ((it & 15u) == 0u) {
+                if (s_abort || ld_volatile_i32(&p.ctrl->abort)) return;
+                const unsigned long long now = globaltimer_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > kWaitLimitNs) { s_abort = 1; return; }
+            }
+        }
+        int kinds = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (p_bw[i] < 0) continue;
+            const int b = p_bw[i] >> 8, w = p_bw[i] & 255;
+            int frame = 0;
+            const int kind = row_kind(b, w, (int)(uint32_t)v[i], frame);
+            kinds |= kind << (2 * i);
+            if (kind == 2) {
+                const __nv_bfloat16* src = p.enc_proj + ((size_t)b * p.T + frame) * p.H + r_ht * 64 + p_chunk * 8;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(stash + (size_t)(p_row0 + 32 * i) * 128 + p_chunk * 16)),
+                             "l"(src)
+                             : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        pre_kinds = kinds;
+    };
     // projection epilogue of a P CTA: pred_proj rows [r_ht*64, +64) of utterances [r_qp*np, +np), then z
     auto epilogue_res_P = [&]() -> bool {
         const int32_t* t_new = p.t2 + (size_t)((step + 1) & 1) * p.B;
         const int h0 = r_ht * 64;
-        const int rows_here = p.np * p.W;          // z rows of this CTA: (utterance, window row) pairs
-        // z row r: 0 = nothing to write (outside the batch, or the utterance is done), 1 = zeros (past the end of
-        // the utterance), 2 = act(enc_proj row + pred_proj); for 2 the row's 64 enc_proj values are fetched
-        auto fetch = [&](int r, uint4* ev) -> int {
-            const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
-            if (r >= rows_here || b >= p.B) return 0;
-            const int t = t_new[b];
-            const int left = p.enc_len[b] - t;
-            if (left <= 0) return 0;
-            if (w >= left) return 1;
-            const uint4* src = reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + t + w) * p.H + h0);
+        const int rows_here = p.np * p.W;
+        // one 16-byte chunk of a z row: act(enc_proj chunk + pred_proj chunk), zeros past the utterance's end
+        auto z_chunk = [&](int bl, int kind, uint4 ev) -> uint4 {
+            const float4* gs = reinterpret_cast<const float4*>(stage_f + bl * 68 + p_chunk * 8);
+            const float4 ga = gs[0], gb = gs[1];
+            const float gg[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+            const __nv_bfloat162* eb = reinterpret_cast<const __nv_bfloat162*>(&ev);
+            uint32_t wds[4];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) ev[k] = src[k];
-            return 2;
-        };
-        auto emit = [&](int r, int kind, const uint4* ev) {
-            if (kind == 0) return;
-            const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
-            uint4* dst = reinterpret_cast<uint4*>(p.z + ((size_t)b * p.W + w) * p.H + h0);
-            const float4* gs = reinterpret_cast<const float4*>(stage_f + bl * 68);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                uint4 o = make_uint4(0, 0, 0, 0);
-                if (kind == 2) {
-                    const __nv_bfloat162* eb = reinterpret_cast<const __nv_bfloat162*>(&ev[k]);
-                    const float4 ga = gs[2 * k], gb = gs[2 * k + 1];
-                    const float gg[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
-                    uint32_t wds[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float2 e2 = __bfloat1622float2(eb[i]);
-                        float z0 = e2.x + gg[2 * i], z1 = e2.y + gg[2 * i + 1];
-                        z0 = p.act == WIND_ACT_RELU ? fmaxf(z0, 0.f) : tanh_fast(z0);
-                        z1 = p.act == WIND_ACT_RELU ? fmaxf(z1, 0.f) : tanh_fast(z1);
-                        wds[i] = pack_bf16x2(z0, z1);
-                    }
-                    o = make_uint4(wds[0], wds[1], wds[2], wds[3]);
-                }
-                dst[k] = o;
+            for (int i = 0; i < 4; ++i) {
+                const float2 e2 = __bfloat1622float2(eb[i]);
+                float z0 = e2.x + gg[2 * i], z1 = e2.y + gg[2 * i + 1];
+                z0 = p.act == WIND_ACT_RELU ? fmaxf(z0, 0.f) : tanh_fast(z0);
+                z1 = p.act == WIND_ACT_RELU ? fmaxf(z1, 0.f) : tanh_fast(z1);
+                wds[i] = kind == 2 ? pack_bf16x2(z0, z1) : 0u;
             }
+            return make_uint4(wds[0], wds[1], wds[2], wds[3]);
         };
-        // the first z row of this thread is requested before the accumulator is ready
-        uint4 ev0[8];
-        const int kind0 = fetch(e, ev0);
+        // the chunks of this thread's first eight rows: prefetched, or requested now before the accumulator is ready
+        uint4 ev[8];
+        int kinds = pre_kinds;
+        if (kinds < 0) {
+            kinds = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                ev[i] = make_uint4(0, 0, 0, 0);
+                if (p_bw[i] >= 0) {
+                    const int b = p_bw[i] >> 8, w = p_bw[i] & 255;
+                    int frame = 0;
+                    const int kind = row_kind(b, w, t_new[b], frame);
+                    kinds |= kind << (2 * i);
+                    if (kind == 2) ev[i] = *reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + frame) * p.H + h0 + p_chunk * 8);
+                }
+            }
+        } else {
+            asm volatile("cp.async.wait_all;" ::: "memory");
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                ev[i] = make_uint4(0, 0, 0, 0);
+                if (((kinds >> (2 * i)) & 3) == 2) ev[i] = *reinterpret_cast<const uint4*>(stash + (size_t)(p_row0 + 32 * i) * 128 + p_chunk * 16);
+            }
+        }
         if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
         const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[2], acc_n[2] & 1u, &s_abort));
         tc_fence_after();
         if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
         if (ready) {
             const int hl = 16 * q + (lane & 15);
-            const float bias = p.b_pred[h0 + hl];
+            const float bias = p_bias;
             for (int c0 = 16 * sub; c0 < p.np; c0 += 32) {
                 float g[16], more[16];
                 tmem_ld16(tm_p + lane_off + (uint32_t)c0, g);
@@ -778,18 +856,41 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 }
             }
         }
+        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 10);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[2]);
         ++acc_n[2];
         asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 11);
         if (ready) {
-            emit(e, kind0, ev0);
-            for (int r = e + 256; r < rows_here; r += 256) {
-                const int kind = fetch(r, ev0);
-                emit(r, kind, ev0);
+            uint4 out[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int bl = p_bw[i] >= 0 ? (p_bw[i] >> 8) - r_qp * p.np : 0;
+                out[i] = z_chunk(bl, (kinds >> (2 * i)) & 3, ev[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (p_bw[i] >= 0 && ((kinds >> (2 * i)) & 3) != 0) {
+                    const int b = p_bw[i] >> 8, w = p_bw[i] & 255;
+                    *reinterpret_cast<uint4*>(p.z + ((size_t)b * p.W + w) * p.H + h0 + p_chunk * 8) = out[i];
+                }
+            }
+            if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 12);
+            // rows beyond the first 256 of this CTA (wide windows): same chunking, fetched here
+            for (int r = p_row0 + 256; r < rows_here; r += 32) {
+                const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
+                if (b >= p.B) break;
+                int frame = 0;
+                const int kind = row_kind(b, w, t_new[b], frame);
+                if (kind == 0) continue;
+                uint4 x = make_uint4(0, 0, 0, 0);
+                if (kind == 2) x = *reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + frame) * p.H + h0 + p_chunk * 8);
+                *reinterpret_cast<uint4*>(p.z + ((size_t)b * p.W + w) * p.H + h0 + p_chunk * 8) = z_chunk(bl, kind, x);
             }
         }
+        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 13);
         fence_proxy_async_all();
         if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
         return ready;
@@ -826,6 +927,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             if (warp >= 2) {
                 if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_START);
                 if (res_l) epilogue_res_L();
+                else if (res_p) prefetch_res_P();
                 if (cta == 0 && e == 0 && step >= 0 && !p.forced) p.ctrl->step = step + 1;
             }
             if (!grid_sync(TR_L)) goto done;
@@ -1353,7 +1455,9 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
             const uint32_t tile = (uint32_t)r.kb_p * 64u * BK * 2u;
             uint32_t buf = (uint32_t)r.nj * (uint32_t)m.H * 2u;
             if ((uint32_t)r.nl * m.P * 2u > buf) buf = (uint32_t)r.nl * m.P * 2u;
-            if ((uint32_t)r.np * m.P * 2u > buf) buf = (uint32_t)r.np * m.P * 2u;
+            // a projection CTA also keeps, behind its operand box, the prefetched enc_proj rows of its first 256 z rows
+            const uint32_t stash_rows = (uint32_t)(r.np * c.W < 256 ? r.np * c.W : 256);
+            if ((uint32_t)r.np * m.P * 2u + stash_rows * 128u > buf) buf = (uint32_t)r.np * m.P * 2u + stash_rows * 128u;
             buf = (buf + 1023u) / 1024u * 1024u;
             r.resident = 1;
             r.j_mode = J_TMEM;
@@ -1437,7 +1541,7 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.np = pl.np; p.hg_count = pl.hg_count; p.p_items = pl.p_items;
     p.kb_h = pl.kb_h; p.kb_p = pl.kb_p;
     p.stat_bytes = pl.stat_bytes;
-    p.enc_len = c.enc_len; p.t2 = c.t(); p.count = c.count(); p.emit_tok = c.emit_tok(); p.keys2 = c.keys();
+    p.enc_len = c.enc_len; p.t2 = c.t(); p.t_pub = c.t_pub(); p.count = c.count(); p.emit_tok = c.emit_tok(); p.keys2 = c.keys();
     p.out_tokens = c.out_tokens; p.out_frames = c.out_frames; p.out_len = c.out_len;
     p.c_state = c.c(); p.hb = c.hb(0, 0); p.z = c.z(); p.enc_proj = (const __nv_bfloat16*)c.enc_proj(); p.g0 = c.g0();
     for (int l = 0; l < c.m.L; ++l) { p.b_ih[l] = c.b_ih[l]; p.b_hh[l] = c.b_hh[l]; }

@@ -60,6 +60,7 @@ struct LoopParams {
     uint32_t stage_lp, stage_j, stat_bytes;
     const int32_t* enc_len;
     int32_t* t2;                   // [2][B]
+    unsigned long long* t_pub;     // [B]
     int32_t* count;                // [B]
     int32_t* emit_tok;             // [B]
     unsigned long long* keys2;     // [2][rows_pad]
