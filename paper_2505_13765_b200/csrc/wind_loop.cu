@@ -602,14 +602,27 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
 #pragma unroll
                                 for (int j = 0; j < 8; ++j) si.kk[j] = (w0 + j < n) ? keys_cur[(size_t)b * p.W + w0 + j] : 0ull;
                             }
+                            // the eight rows side by side: which are inside the window, broken, non-blank
+                            uint32_t nonblank = 0u, broken = 0u;
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
-                                if (w0 + j < n && first < 0) {
-                                    uint32_t lab = key_label(si.kk[j]);
-                                    if (si.kk[j] == 0ull || lab >= (uint32_t)p.NV) { bad = true; lab = (uint32_t)p.blank; }
-                                    if ((int)lab != p.blank) { first = w0 + j; label = (int)lab; }
-                                }
+                                const uint32_t lab = key_label(si.kk[j]);
+                                const bool inside = w0 + j < n;
+                                const bool brk = si.kk[j] == 0ull || lab >= (uint32_t)p.NV;
+                                broken |= (uint32_t)(inside && brk) << j;
+                                nonblank |= (uint32_t)(inside && !brk && (int)lab != p.blank) << j;
                             }
+                            if (nonblank) {
+                                const int j = __ffs((int)nonblank) - 1;
+                                first = w0 + j;
+                                uint32_t lab = 0u;
+#pragma unroll
+                                for (int jj = 0; jj < 8; ++jj)
+                                    if (jj == j) lab = key_label(si.kk[jj]);
+                                label = (int)lab;
+                                broken &= (1u << j) - 1u;   // rows after the first non-blank one are not looked at
+                            }
+                            bad = bad || broken != 0u;
                         }
                         if (first >= 0) tok = label;
                         if (writer) {
@@ -856,13 +869,11 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 }
             }
         }
-        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 10);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[2]);
         ++acc_n[2];
         asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 11);
         if (ready) {
             uint4 out[8];
 #pragma unroll
@@ -877,7 +888,6 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     *reinterpret_cast<uint4*>(p.z + ((size_t)b * p.W + w) * p.H + h0 + p_chunk * 8) = out[i];
                 }
             }
-            if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 12);
             // rows beyond the first 256 of this CTA (wide windows): same chunking, fetched here
             for (int r = p_row0 + 256; r < rows_here; r += 32) {
                 const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
@@ -890,7 +900,6 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 *reinterpret_cast<uint4*>(p.z + ((size_t)b * p.W + w) * p.H + h0 + p_chunk * 8) = z_chunk(bl, kind, x);
             }
         }
-        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, 13);
         fence_proxy_async_all();
         if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
         return ready;
