@@ -96,16 +96,18 @@ struct GemmParams {
 };
 
 constexpr int GEMM_THREADS = 192;  // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..5: epilogue
-constexpr int GEMM_STAGES = 4;
+constexpr int GEMM_STAGES = 3;      // 3 x 32 KB per CTA, so that two CTAs share an SM: one's epilogue overlaps the other's main loop
 constexpr int GEMM_BN = 128;
 
 template <int MODE>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[GEMM_STAGES], empty_bar[GEMM_STAGES], accum_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ float s_bias[GEMM_BN];
+    __shared__ int s_valid[BM];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr uint32_t b_stage_bytes = GEMM_BN * BK * 2;
@@ -178,37 +180,59 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
     } else {
         const int q = warp & 3;            // tensor-memory lane quadrant this warp may read
-        const bool ready = __all_sync(0xffffffffu, mbar_wait(&accum_bar, 0, &abort_flag));
-        tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-        if (ready) {
-            const long long r = (long long)m_blk * BM + q * 32 + lane;
+        const int et = threadIdx.x - 64;   // 0..127
+        const int row = q * 32 + lane;     // accumulator row of this thread
+        // before the accumulator is ready: this tile's bias values and which of its rows are valid frames
+        {
+            const int n = n_tile_idx * GEMM_BN + et;
+            float bsum = 0.f;
+            if (n < p.N) bsum = p.bias0[n] + (MODE == MODE_GATE_TABLE ? p.bias1[n] : 0.f);
+            s_bias[et] = bsum;
+            const long long r = (long long)m_blk * BM + row;
             bool valid = r < p.rows;
             if (MODE == MODE_ENC_PROJ && valid) {
                 const int b = (int)(r / p.T);
                 valid = (int)(r - (long long)b * p.T) < p.enc_len[b];
             }
+            s_valid[row] = valid;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const bool ready = __all_sync(0xffffffffu, mbar_wait(&accum_bar, 0, &abort_flag));
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+        // The tile goes through shared memory (the pipeline's buffers: every MMA has completed), so that it leaves
+        // as whole row segments: 16 (bf16) or 32 (fp32) neighbouring threads write one row's 256 or 512 bytes.
+        constexpr int ELEM = MODE == MODE_ENC_PROJ ? 2 : 4;
+        constexpr int ROW_BYTES = GEMM_BN * ELEM + 16;          // padded: consecutive rows start in different banks
+        if (ready) {
+            uint8_t* my = smem + (size_t)row * ROW_BYTES;
             for (int c0 = 0; c0 < GEMM_BN; c0 += 16) {
                 float v[16];
                 tmem_ld16(taddr + c0, v);
-                const int n0 = n_tile_idx * GEMM_BN + c0;
-                if (valid && n0 < p.N) {   // N is a multiple of 64, so 16-column groups are all-in or all-out
-                    if (MODE == MODE_ENC_PROJ) {
-                        uint32_t w[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) w[i] = pack_bf16x2(v[2 * i] + p.bias0[n0 + 2 * i], v[2 * i + 1] + p.bias0[n0 + 2 * i + 1]);
-                        uint4* dst = reinterpret_cast<uint4*>(p.out_bf16 + r * p.N + n0);
-                        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-                    } else {
-                        float4* dst = reinterpret_cast<float4*>(p.out_f32 + r * p.N + n0);
+                for (int i = 0; i < 16; ++i) v[i] += s_bias[c0 + i];
+                if (MODE == MODE_ENC_PROJ) {
+                    uint4* dst = reinterpret_cast<uint4*>(my + c0 * 2);
+                    dst[0] = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+                    dst[1] = make_uint4(pack_bf16x2(v[8], v[9]), pack_bf16x2(v[10], v[11]), pack_bf16x2(v[12], v[13]), pack_bf16x2(v[14], v[15]));
+                } else {
+                    float4* dst = reinterpret_cast<float4*>(my + c0 * 4);
 #pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            dst[i] = make_float4(v[4 * i] + p.bias0[n0 + 4 * i] + p.bias1[n0 + 4 * i],
-                                                 v[4 * i + 1] + p.bias0[n0 + 4 * i + 1] + p.bias1[n0 + 4 * i + 1],
-                                                 v[4 * i + 2] + p.bias0[n0 + 4 * i + 2] + p.bias1[n0 + 4 * i + 2],
-                                                 v[4 * i + 3] + p.bias0[n0 + 4 * i + 3] + p.bias1[n0 + 4 * i + 3]);
-                    }
+                    for (int i = 0; i < 4; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                }
+            }
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ready) {
+            constexpr int CHUNKS = GEMM_BN * ELEM / 16;           // 16-byte chunks per row
+            const int n_cols = min(GEMM_BN, p.N - n_tile_idx * GEMM_BN);
+            uint8_t* out = MODE == MODE_ENC_PROJ ? reinterpret_cast<uint8_t*>(p.out_bf16) : reinterpret_cast<uint8_t*>(p.out_f32);
+            for (int ch = et; ch < BM * CHUNKS; ch += 128) {
+                const int rr = ch / CHUNKS, cc = ch - rr * CHUNKS;
+                if (s_valid[rr] && cc * 16 < n_cols * ELEM) {
+                    const uint4 x = *reinterpret_cast<const uint4*>(smem + (size_t)rr * ROW_BYTES + cc * 16);
+                    const long long r = (long long)m_blk * BM + rr;
+                    *reinterpret_cast<uint4*>(out + ((size_t)r * p.N + (size_t)n_tile_idx * GEMM_BN) * ELEM + cc * 16) = x;
                 }
             }
         }
