@@ -242,6 +242,16 @@ int32_t wind_set_trace(int32_t first_step);
 wind_status_t wind_read_trace(const wind_model_t* m, int32_t B, int32_t T, int32_t W, const void* workspace, void* stream,
                               wind_trace_event_t* host_out, int32_t capacity, int32_t* n_out);
 
+/*
+ * Test hook for the failure path of the persistent loop kernel: with extra_arrivals > 0 its grid barrier waits
+ * for that many arrivals more than there are CTAs, so the first barrier of the next decode can never fill.  Every
+ * wait in the kernel is bounded (about two seconds), so the decode then ends by itself: the CTAs give up, free
+ * their tensor memory and return, and the call reports WIND_ERR_TIMEOUT with undefined outputs; the CUDA context
+ * stays usable.  0 restores normal operation.  Returns the previous value.  The paper has no counterpart (its only
+ * mention of a safeguard is the beam-search footnote about not staying on one frame forever).
+ */
+int32_t wind_debug_stall_barrier(int32_t extra_arrivals);
+
 /* Process-wide choice of kernels for the bf16 path (default AUTO).  Returns the previous value. */
 int32_t wind_set_kernels(int32_t kernels);
 

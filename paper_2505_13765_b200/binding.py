@@ -30,7 +30,7 @@ WIND_KERNELS_AUTO, WIND_KERNELS_SIMT, WIND_KERNELS_TENSOR = 0, 1, 2
 
 EXPORTS = [
     "wind_workspace_bytes", "wind_decode_greedy", "wind_host_staging_bytes", "wind_decode_greedy_host",
-    "wind_eval_joint_window", "wind_eval_joint_window_static", "wind_profile_decode", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
+    "wind_eval_joint_window", "wind_eval_joint_window_static", "wind_profile_decode", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_debug_stall_barrier", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
 ]
 
 _vp = C.c_void_p
@@ -108,6 +108,8 @@ def load_library():
     L.wind_set_trace.restype = i32
     L.wind_read_trace.argtypes = [mp, i32, i32, i32, _vp, _vp, C.POINTER(wind_trace_event_t), i32, C.POINTER(i32)]
     L.wind_read_trace.restype = i32
+    L.wind_debug_stall_barrier.argtypes = [i32]
+    L.wind_debug_stall_barrier.restype = i32
     L.wind_set_kernels.argtypes = [i32]
     L.wind_set_kernels.restype = i32
     L.wind_status_string.argtypes = [i32]
@@ -146,6 +148,11 @@ def wind_read_trace(model: "WindModel", B: int, T: int, W: int, workspace, strea
     if st != WIND_OK:
         raise WindError(st)
     return [dict(role=e.role, phase=e.phase, event=e.event, step=e.step, clock=e.clock) for e in buf[: n.value]]
+
+
+def wind_debug_stall_barrier(extra_arrivals: int) -> int:
+    """Test hook: make the loop kernel's grid barrier unfillable (see wind.h); 0 restores normal operation."""
+    return load_library().wind_debug_stall_barrier(extra_arrivals)
 
 
 def wind_set_kernels(kernels: int) -> int:

@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "wind_internal.cuh"
+#include "wind_loop.cuh"
 
 namespace wind {
 
@@ -490,6 +491,8 @@ wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t*
     host_out->kernels = hc.kernels;
     return WIND_OK;
 }
+
+int32_t wind_debug_stall_barrier(int32_t extra_arrivals) { return loop_set_extra_arrivals(extra_arrivals); }
 
 int32_t wind_set_trace(int32_t first_step) {
     int32_t prev = g_trace_step;

@@ -242,7 +242,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
     auto grid_sync = [&](int phase_kind) -> bool {
         __syncthreads();
         if (threadIdx.x == 0) {
-            epoch += (uint32_t)G;
+            epoch += (uint32_t)(G + p.extra_arrivals);   // extra_arrivals > 0: a test hook, the barrier can then never fill
             trace_event(p, 3, tr_n, step, phase_kind, EV_ARRIVE);
             if (s_abort) {
                 atomicExch(&p.ctrl->abort, 1);
@@ -1289,7 +1289,11 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
 done:
     // an accumulator may still hold an unused early GEMM; nothing reads it, the MMAs have completed
     // before the last barrier (the issuing thread waited for none of them, so wait for them here)
-    if (early && warp == 1 && lane == 0 && !s_abort) mbar_wait(&acc_full[1], acc_n[1] & 1u ? 0u : 1u, &s_abort);
+    // (also when the kernel is being abandoned: a private flag, so that the wait is not cut short; it stays bounded)
+    if (early && warp == 1 && lane == 0) {
+        int gave_up = 0;
+        mbar_wait(&acc_full[1], acc_n[1] & 1u ? 0u : 1u, &gave_up);
+    }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -1315,6 +1319,8 @@ static std::mutex g_loop_mutex;
 static int g_sm_count[64] = {};
 static int g_smem_optin[64] = {};
 static int g_attr_smem = 0;
+static int g_loop_extra_arrivals = 0;
+int loop_set_extra_arrivals(int n) { int prev = g_loop_extra_arrivals; g_loop_extra_arrivals = n > 0 ? n : 0; return prev; }
 
 static cudaError_t loop_device_info(int* sms, int* smem_optin) {
     int dev = 0;
@@ -1557,6 +1563,7 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.b_pred = c.m.b_pred; p.b_out = c.m.b_out; p.w_out = (const __nv_bfloat16*)c.m.w_out;
     p.forced = logits_out != nullptr; p.prefix = prefix; p.U = U; p.prefix_len = prefix_len; p.logits_out = logits_out;
     p.trace = trace_step >= -1 ? c.trace() : nullptr; p.trace_step = trace_step;
+    p.extra_arrivals = g_loop_extra_arrivals;
     void* args[2] = {(void*)&t_loop_maps, (void*)&p};
     return cudaLaunchCooperativeKernel(pl.resident ? (const void*)loop_kernel<true> : (const void*)loop_kernel<false>, dim3((unsigned)pl.grid), dim3(pl.resident ? LOOP_THREADS_RES : LOOP_THREADS), args, pl.smem_bytes,
                                        c.stream);

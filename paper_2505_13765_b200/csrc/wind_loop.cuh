@@ -86,9 +86,11 @@ struct LoopParams {
     // timeline of CTA 0 for lock steps [trace_step, trace_step + 2); trace == nullptr: off
     TraceEvent* trace;
     int trace_step;
+    int extra_arrivals;            // test hook: arrivals the grid barrier waits for beyond the grid size (0 in normal use)
 };
 
 cudaError_t loop_plan(const Call& c, LoopPlan* out);
+int loop_set_extra_arrivals(int n);  // returns the previous value
 cudaError_t loop_prepare(Call& c);   // plan + tensor maps + shared-memory opt-in (host only; not inside a capture)
 
 }  // namespace wind

@@ -358,6 +358,28 @@ def test_host_buffer_entry_point_matches_device_entry_point(pkg):
         assert np.array_equal(frm_h.numpy()[b, : ref[2][b]], ref[1][b, : ref[2][b]])
 
 
+def test_unfillable_barrier_ends_in_timeout_status_and_the_context_stays_usable(pkg):
+    # Failure path of the persistent kernel without hanging anything: every wait in it is bounded, so a grid
+    # barrier that can never fill (test hook) makes the CTAs give up after about two seconds and the call return
+    # WIND_ERR_TIMEOUT; the next decode on the same context works and gives the usual result.
+    cfg = ws.small_variant(ws.CONFIGS["cfg3_large_b128"], 4, 10, 40)
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="zero")
+    model = pkg.WindModel(weights)
+    ref = pkg.decode(model, enc, lens, cfg.W, cfg.S)
+    assert ref[4] == 0 and ref[3]["kernels"] == 2
+    prev = pkg.wind_debug_stall_barrier(1)
+    try:
+        out = pkg.decode(model, enc, lens, cfg.W, cfg.S, check=False)
+    finally:
+        pkg.wind_debug_stall_barrier(prev)
+    assert out[4] == pkg.binding.WIND_ERR_TIMEOUT
+    again = pkg.decode(model, enc, lens, cfg.W, cfg.S)
+    assert again[4] == 0
+    for a, b in zip(again[:3], ref[:3]):
+        assert np.array_equal(a, b)
+
+
 def test_workspace_too_small_is_rejected(pkg):
     w, enc, lens = ragged_case(60, B=2, T=10, D=8, E=8, P=8, L=1, H=8, V=5)
     model = pkg.WindModel(w)
