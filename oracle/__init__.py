@@ -92,6 +92,8 @@ def lib():
         L.oracle_eval_joint_window.argtypes = [mp, f32p, C.c_int32, i32p, C.c_int32, C.c_int32, C.c_int32, f64p,
                                                f64p, f64p, f64p]
         L.oracle_eval_joint_window.restype = C.c_int32
+        L.oracle_first_output_logprobs.argtypes = [mp, f32p, C.c_int32, i32p, C.c_int32, C.c_int32, C.c_int32, f64p]
+        L.oracle_first_output_logprobs.restype = C.c_int32
     return _lib
 
 
@@ -185,6 +187,16 @@ def eval_joint_window(model: Model, enc_b: np.ndarray, T: int, prefix: Sequence[
                                        int(t0), int(W), _ptr(logits, f64p), _ptr(g, f64p), _ptr(h, f64p),
                                        _ptr(c, f64p))
     return logits[:n], g, h, c
+
+
+def first_output_logprobs(model: Model, enc_b: np.ndarray, T: int, prefix: Sequence[int], t0: int, W: int) -> np.ndarray:
+    """Eq. (1): log P'(v, t) for the window starting at t0, [n, V+1] fp64 (-inf where P' is zero)."""
+    enc_b = _f32(enc_b)
+    prefix = np.ascontiguousarray(prefix, dtype=np.int32)
+    out = np.zeros((max(W, 1), model.dims["V"] + 1), np.float64)
+    n = lib().oracle_first_output_logprobs(model.ref, _ptr(enc_b, f32p), int(T), _ptr(prefix, i32p), len(prefix),
+                                           int(t0), int(W), _ptr(out, f64p))
+    return out[:n]
 
 
 def linear(Wm: np.ndarray, b: Optional[np.ndarray], x: np.ndarray) -> np.ndarray:

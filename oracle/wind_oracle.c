@@ -380,3 +380,40 @@ int32_t oracle_eval_joint_window(const oracle_model_t* m, const float* enc, int3
     scratch_free(&s);
     return n;
 }
+
+/*
+ * Eq. (1): P'(v, t), the probability that v is the FIRST output in the window that starts at frame t0,
+ * emitted at frame t0 + t, under the current decoder state:
+ *   v != blank: P(v | t0 + t) * prod_{t' < t} P(blank | t0 + t')
+ *   v == blank: 0 for t < n - 1, and prod_{t' <= n - 1} P(blank | t0 + t') for t = n - 1
+ * with P(. | frame) = softmax of the joint's logits and n = min(W, T - t0) rows in the window (the paper writes
+ * the window size w; at the end of an utterance the window is the truncated one of Algorithm 3, n = min(N, T - t)).
+ * Output: natural-log probabilities, logp [n, V+1] (-INFINITY for the zero entries).  Returns n.
+ * Plain steps: logits (teacher-forced prefix), log-softmax per row, running sum of the blank log-probabilities.
+ */
+int32_t oracle_first_output_logprobs(const oracle_model_t* m, const float* enc, int32_t T, const int32_t* prefix,
+                                     int32_t prefix_len, int32_t t0, int32_t W, double* logp) {
+    const int NV = m->V + 1;
+    double* logits = (double*)malloc(sizeof(double) * (size_t)(W > 0 ? W : 1) * NV);
+    const int n = oracle_eval_joint_window(m, enc, T, prefix, prefix_len, t0, W, logits, NULL, NULL, NULL);
+    double blanks_before = 0.0; /* sum of log P(blank | t0 + t') for t' < t */
+    for (int t = 0; t < n; ++t) {
+        const double* row = logits + (size_t)t * NV;
+        double mx = row[0];
+        for (int v = 1; v < NV; ++v)
+            if (row[v] > mx) mx = row[v];
+        double se = 0.0;
+        for (int v = 0; v < NV; ++v) se += exp(row[v] - mx);
+        const double lse = mx + log(se);
+        for (int v = 0; v < NV; ++v) {
+            const double lp = row[v] - lse; /* log P(v | t0 + t) */
+            if (v != m->blank_id)
+                logp[(size_t)t * NV + v] = lp + blanks_before;
+            else
+                logp[(size_t)t * NV + v] = (t == n - 1) ? lp + blanks_before : -INFINITY;
+        }
+        blanks_before += row[m->blank_id] - lse;
+    }
+    free(logits);
+    return n;
+}

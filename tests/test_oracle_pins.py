@@ -356,3 +356,72 @@ def test_low_margin_count_matches_direct_count():
     _, _, _, stw = oracle.decode_batch(m, enc, lens, W=4, S=3, margin_thr=thr)
     assert st["low_margin"] == stw["low_margin"] and st["decisions"] == stw["decisions"]
     assert 0 < st["low_margin"] < st["decisions"]
+
+
+# ---------------------------------------------------------------------------
+# Eq. (1): P'(v, t), "v is the first output in the window, at offset t"
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("seed,blank0,W,t0", [(0, False, 4, 0), (1, True, 3, 2), (2, False, 8, 5), (3, True, 1, 1), (4, False, 6, 7)])
+def test_first_output_probabilities_match_direct_products(seed, blank0, W, t0):
+    # independent evaluator: softmax of the naive model's logits, then the products of Eq. (1) written out
+    r = rng(300 + seed)
+    T, V = 9, 6
+    w = random_weights(r, 5, 4, 6, 2, 7, V, blank_id=0 if blank0 else None, act=seed % 2, blank_bias=0.5, bias_scale=0.2)
+    enc = r.standard_normal((T, 5)).astype(np.float32)
+    prefix = [int(x) for x in r.integers(1 if blank0 else 0, V if blank0 else V - 1, size=3)]
+    prefix = [p for p in prefix if p != w["blank_id"]]
+    m = oracle.Model(w)
+    logp = oracle.first_output_logprobs(m, enc, T, prefix, t0, W)
+    n = min(W, T - t0)
+    assert logp.shape == (n, V + 1)
+    naive = NaiveModel(w)
+    probs = []
+    for t in range(n):
+        z = naive.logits(enc[t0 + t], prefix)
+        e = np.exp(z - z.max())
+        probs.append(e / e.sum())
+    blank = w["blank_id"]
+    expect = np.zeros((n, V + 1))
+    for t in range(n):
+        before = np.prod([probs[k][blank] for k in range(t)]) if t else 1.0
+        for v in range(V + 1):
+            if v != blank:
+                expect[t, v] = probs[t][v] * before
+            else:
+                expect[t, v] = before * probs[t][blank] if t == n - 1 else 0.0
+    got = np.exp(logp)
+    assert np.max(np.abs(got - expect)) < 1e-12
+    assert np.all(np.isneginf(logp[: n - 1, blank]))
+    # it is a distribution over "what comes first in the window, and where"
+    assert abs(got.sum() - 1.0) < 1e-12
+    # a window of one frame is the frame's own softmax
+    one = np.exp(oracle.first_output_logprobs(m, enc, T, prefix, t0, 1))
+    assert np.max(np.abs(one[0] - probs[0])) < 1e-12
+
+
+def test_first_output_argmax_is_the_greedy_jump_when_blank_dominates_or_not():
+    # With a very confident model (logits scaled up) the most probable first output is what Algorithm 2 emits: the
+    # first non-blank argmax row and its label, or blank at the last row when every row's argmax is blank.
+    r = rng(400)
+    T, V, W = 12, 5, 4
+    w = random_weights(r, 4, 3, 5, 1, 6, V, blank_bias=0.3)
+    w["w_out"] = (w["w_out"] * 40).astype(np.float32)
+    w["b_out"] = (w["b_out"] * 40).astype(np.float32)
+    enc = r.standard_normal((T, 4)).astype(np.float32)
+    m = oracle.Model(w)
+    checked = 0
+    for t0 in range(T):
+        logits, *_ = oracle.eval_joint_window(m, enc, T, [], t0, W)
+        labels = logits.argmax(axis=1)
+        logp = oracle.first_output_logprobs(m, enc, T, [], t0, W)
+        t_best, v_best = np.unravel_index(np.argmax(logp), logp.shape)
+        nonblank = [i for i, l in enumerate(labels) if l != w["blank_id"]]
+        top2 = np.sort(logits, axis=1)[:, -2:]
+        if np.min(top2[:, 1] - top2[:, 0]) < 0.5:
+            continue    # not confident enough for the argument to hold
+        checked += 1
+        if nonblank:
+            assert (t_best, v_best) == (nonblank[0], labels[nonblank[0]])
+        else:
+            assert (t_best, v_best) == (len(labels) - 1, w["blank_id"])
+    assert checked >= 4
