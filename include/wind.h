@@ -161,6 +161,24 @@ wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, con
                                      size_t workspace_bytes, void* stream);
 
 /*
+ * Eq. (1) of the paper's beam-search section: P'(v, t), the probability that v is the FIRST output in the window that
+ * starts at frame t0[b], emitted at frame t0[b] + t, given the decoder state after `prefix`:
+ *     v != blank:  P(v | t0 + t) * prod_{t' < t} P(blank | t0 + t')
+ *     v == blank:  0 for t < n - 1;  prod_{t' <= n - 1} P(blank | t0 + t') for t = n - 1
+ * with P(. | frame) the softmax of the joint's logits and n = min(W, enc_len[b] - t0[b]) (the truncated window of
+ * Algorithm 3, line "n = min(N, T - t)").  Same inputs as wind_eval_joint_window.
+ *   logp       [B, W, V+1] fp32 out: natural-log P'(v, t), -inf for the zero entries; rows w >= n are left untouched.
+ *   K          0, or how many of the most probable (label, offset) pairs to return per utterance: the expansions
+ *              Algorithm 3 takes "from all |V| x n combinations".  top_label, top_jump [B, K] int32, top_logp [B, K] fp32,
+ *              best first; equal values in order of (offset, label); -1 / -inf when the window has fewer than K entries.
+ * The logits stay in `logp` between the joint's store epilogue and the in-place pass; errors as wind_eval_joint_window.
+ */
+wind_status_t wind_window_first_output(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B, int32_t T,
+                                       int32_t W, const int32_t* prefix, int32_t U, const int32_t* prefix_len,
+                                       const int32_t* t0, float* logp, int32_t K, int32_t* top_label, int32_t* top_jump,
+                                       float* top_logp, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Largest workspace, in bytes, that wind_eval_joint_window_static can serve: the size of the
  * scratch array compiled into the library.
  */

@@ -30,7 +30,7 @@ WIND_KERNELS_AUTO, WIND_KERNELS_SIMT, WIND_KERNELS_TENSOR = 0, 1, 2
 
 EXPORTS = [
     "wind_workspace_bytes", "wind_decode_greedy", "wind_host_staging_bytes", "wind_decode_greedy_host",
-    "wind_eval_joint_window", "wind_eval_joint_window_static", "wind_profile_decode", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_debug_stall_barrier", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
+    "wind_eval_joint_window", "wind_window_first_output", "wind_eval_joint_window_static", "wind_profile_decode", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_debug_stall_barrier", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
 ]
 
 _vp = C.c_void_p
@@ -100,6 +100,8 @@ def load_library():
     L.wind_profile_decode.restype = i32
     L.wind_eval_joint_window.argtypes = [mp, _vp, _vp, i32, i32, i32, _vp, i32, _vp, _vp, _vp, _vp, C.c_size_t, _vp]
     L.wind_eval_joint_window.restype = i32
+    L.wind_window_first_output.argtypes = [mp, _vp, _vp, i32, i32, i32, _vp, i32, _vp, _vp, _vp, i32, _vp, _vp, _vp, _vp, C.c_size_t, _vp]
+    L.wind_window_first_output.restype = i32
     L.wind_eval_joint_window_static.argtypes = [mp, _vp, _vp, i32, i32, i32, _vp, i32, _vp, _vp, _vp, _vp]
     L.wind_eval_joint_window_static.restype = i32
     L.wind_read_stats.argtypes = [_vp, _vp, C.POINTER(wind_stats_t)]
@@ -315,6 +317,21 @@ def wind_eval_joint_window(model: WindModel, enc, enc_len, W: int, prefix, prefi
     st = L.wind_eval_joint_window(model.ref, enc.data_ptr(), enc_len.data_ptr(), B, T, W,
                                   prefix.data_ptr() if U else None, U, prefix_len.data_ptr(), t0.data_ptr(),
                                   logits.data_ptr(), _ws_ptr(workspace), _ws_bytes(workspace), _stream_ptr(stream))
+    if st != WIND_OK:
+        raise WindError(st)
+    return st
+
+
+def wind_window_first_output(model: WindModel, enc, enc_len, W: int, prefix, prefix_len, t0, logp, workspace, K: int = 0,
+                             top_label=None, top_jump=None, top_logp=None, stream=None) -> int:
+    """Eq. (1): log P'(v, t) of each utterance's window into ``logp`` [B, W, V+1]; optionally the K best (label, offset)."""
+    L = load_library()
+    B, T, D = enc.shape
+    U = prefix.shape[1] if prefix is not None and prefix.numel() else 0
+    st = L.wind_window_first_output(model.ref, enc.data_ptr(), enc_len.data_ptr(), B, T, W,
+                                    prefix.data_ptr() if U else None, U, prefix_len.data_ptr(), t0.data_ptr(),
+                                    logp.data_ptr(), K, top_label.data_ptr() if K else None, top_jump.data_ptr() if K else None,
+                                    top_logp.data_ptr() if K else None, _ws_ptr(workspace), _ws_bytes(workspace), _stream_ptr(stream))
     if st != WIND_OK:
         raise WindError(st)
     return st

@@ -297,9 +297,11 @@ wind_status_t wind_decode_greedy_host(const wind_model_t* m, const void* enc_hos
     return read_status(c);
 }
 
-wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B, int32_t T,
-                                     int32_t W, const int32_t* prefix, int32_t U, const int32_t* prefix_len, const int32_t* t0,
-                                     float* logits, void* workspace, size_t workspace_bytes, void* stream) {
+// Teacher-forced window logits, enqueued on the stream (no synchronisation); c receives the call's bundle.
+static wind_status_t enqueue_eval_joint_window(Call& c, const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B,
+                                               int32_t T, int32_t W, const int32_t* prefix, int32_t U, const int32_t* prefix_len,
+                                               const int32_t* t0, float* logits, void* workspace, size_t workspace_bytes,
+                                               void* stream) {
     wind_status_t s = check_model(m);
     if (s != WIND_OK) return s;
     s = check_weights(m);
@@ -308,7 +310,6 @@ wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, con
     if (s != WIND_OK) return s;
     if (!enc || !enc_len || !prefix_len || !t0 || !logits || !workspace || U < 0 || (U > 0 && !prefix)) return WIND_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return WIND_ERR_WORKSPACE;
-    Call c;
     // the control arrays double as scratch outputs here: out_len is reset by the init kernel
     fill_call(c, m, enc, enc_len, B, T, W, 1, nullptr, nullptr, nullptr, 1, workspace, (cudaStream_t)stream);
     if (workspace_bytes < c.lay.total) return WIND_ERR_WORKSPACE;
@@ -322,7 +323,7 @@ wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, con
         WIND_CUDA(tc_gate_table(c));
         WIND_CUDA(launch_set_t(c, t0));
         WIND_CUDA(tc_loop(c, prefix, U, prefix_len, logits, -2));
-        return read_status(c);
+        return WIND_OK;
     }
     WIND_CUDA(launch_init(c, WIND_KERNELS_SIMT, 0, 0));
     WIND_CUDA(simt_enc_proj(c));
@@ -337,6 +338,29 @@ wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, con
     }
     WIND_CUDA(launch_set_t(c, t0));
     WIND_CUDA(simt_joint(c, logits));
+    return WIND_OK;
+}
+
+wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B, int32_t T,
+                                     int32_t W, const int32_t* prefix, int32_t U, const int32_t* prefix_len, const int32_t* t0,
+                                     float* logits, void* workspace, size_t workspace_bytes, void* stream) {
+    Call c;
+    wind_status_t s = enqueue_eval_joint_window(c, m, enc, enc_len, B, T, W, prefix, U, prefix_len, t0, logits, workspace,
+                                                workspace_bytes, stream);
+    if (s != WIND_OK) return s;
+    return read_status(c);
+}
+
+wind_status_t wind_window_first_output(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B, int32_t T,
+                                       int32_t W, const int32_t* prefix, int32_t U, const int32_t* prefix_len, const int32_t* t0,
+                                       float* logp, int32_t K, int32_t* top_label, int32_t* top_jump, float* top_logp,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+    if (K < 0 || (K > 0 && (!top_label || !top_jump || !top_logp))) return WIND_ERR_INVALID_ARG;
+    Call c;
+    wind_status_t s = enqueue_eval_joint_window(c, m, enc, enc_len, B, T, W, prefix, U, prefix_len, t0, logp, workspace,
+                                                workspace_bytes, stream);
+    if (s != WIND_OK) return s;
+    WIND_CUDA(launch_first_output(logp, enc_len, t0, B, W, m->V + 1, m->blank_id, K, top_label, top_jump, top_logp, (cudaStream_t)stream));
     return read_status(c);
 }
 

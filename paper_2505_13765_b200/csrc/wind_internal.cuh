@@ -171,6 +171,10 @@ cudaError_t launch_control(const Call& c, cudaGraphConditionalHandle handle, int
 cudaError_t launch_force_tokens(const Call& c, const int32_t* prefix, int U, const int32_t* prefix_len, int u);
 cudaError_t launch_set_t(const Call& c, const int32_t* t0);
 
+// first-output distribution of a window (Eq. 1), in place on the window's logits
+cudaError_t launch_first_output(float* logp, const int32_t* enc_len, const int32_t* t0, int B, int W, int NV, int blank, int K,
+                                int32_t* top_label, int32_t* top_jump, float* top_logp, cudaStream_t stream);
+
 // tensor-core kernels (bf16 path)
 bool tc_supported(const wind_model_t& m, int B, int T, int W);
 cudaError_t tc_prepare(Call& c);         // builds the tensor maps and the tile plan of this call (host only), sets c.tc
