@@ -184,6 +184,8 @@ def main():
     ap.add_argument("--len-hi", type=int, default=0, help="override the longest utterance length, frames")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the W=1 comparison, e2e and per-kernel timing legs")
+    ap.add_argument("--op", default="decode", choices=["decode", "first_output"],
+                    help="first_output: time wind_window_first_output (Eq. 1 on one window per utterance) instead of the decode")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -196,6 +198,8 @@ def main():
 
     if args.impl == "reference":
         return reference_arm(args, cfg, W)
+    if args.op == "first_output":
+        return first_output_op(args, cfg, W)
 
     import torch
     import paper_2505_13765_b200 as pkg
@@ -370,6 +374,60 @@ def roofline(pkg, model, cfg, W, enc_d, len_d, tok_d, frm_d, ol_d, wsb, stream, 
     return {"kernel": "windowed joint (plain-ALU kernel)", "bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
             "frac": achieved / peak, "peak_source": peaks["source"] + " sustained bf16", "traffic": None,
             "avg_launch_us": dur_s * 1e6, "rows_per_launch": rows_per_launch, "enc_proj": enc, "per_kernel_ms": per_kernel}
+
+
+def first_output_op(args, cfg, W):
+    """Secondary measurement (one JSON line of its own): Eq. (1) for one window per utterance.
+
+    The call runs the projection, the decoder on an empty prefix and the joint's store epilogue, then the in-place
+    Eq. (1) pass with the 4 best (label, offset) pairs.  `value` is windows per second for the whole call; the
+    in-place kernel's own share is what `ncu -k regex:first_output` shows for the same command (see profiles/).
+    """
+    import torch
+    import wind_synth as ws
+    import paper_2505_13765_b200 as pkg
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    pkg.load_library()
+    weights = ws.make_model(cfg)
+    enc_np, lens_np = ws.make_enc(cfg, pad="zero")
+    model = pkg.WindModel(weights, device=dev)
+    B, T, _ = enc_np.shape
+    NV, K = cfg.V + 1, 4
+    enc_d = pkg.to_device_enc(model, enc_np)
+    len_d = torch.from_numpy(lens_np).to(dev)
+    rng = np.random.default_rng(7)
+    t0 = torch.from_numpy(np.array([rng.integers(0, max(1, l - W)) for l in lens_np], np.int32)).to(dev)
+    plen = torch.zeros(B, dtype=torch.int32, device=dev)
+    logp = torch.empty((B, W, NV), dtype=torch.float32, device=dev)
+    tl = torch.empty((B, K), dtype=torch.int32, device=dev)
+    tj = torch.empty((B, K), dtype=torch.int32, device=dev)
+    tv = torch.empty((B, K), dtype=torch.float32, device=dev)
+    wsb = pkg.alloc_workspace(model, B, T, W)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        pkg.wind_window_first_output(model, enc_d, len_d, W, None, plen, t0, logp, wsb, K=K, top_label=tl, top_jump=tj,
+                                     top_logp=tv, stream=stream)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    total = float(np.exp(logp.double().cpu().numpy()).sum())
+    print(json.dumps({
+        "metric": "windows/s, wind_window_first_output (projection + decoder start + joint store + Eq. 1 pass)", "op": "first_output",
+        "value": B / (ms * 1e-3), "unit": "windows/s", "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": B, "W": W, "K": K, "V": cfg.V},
+        "eq1_pass_algorithmic_bytes": 2 * B * W * NV * 4, "sum_of_probabilities_per_window": total / B,
+    }))
 
 
 def reference_arm(args, cfg, W):

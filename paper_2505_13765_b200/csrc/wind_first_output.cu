@@ -27,7 +27,6 @@ __global__ void __launch_bounds__(FO_THREADS) first_output_kernel(float* __restr
                                                                   const int32_t* __restrict__ t0, int W, int NV, int blank, int K,
                                                                   int32_t* __restrict__ top_label, int32_t* __restrict__ top_jump,
                                                                   float* __restrict__ top_logp) {
-    __shared__ float s_part[FO_THREADS / 32];
     __shared__ float s_lse[kMaxWindow], s_before[kMaxWindow];   // log-sum-exp of a row; sum of blank log-probs of the rows before it
     __shared__ float s_best_v[FO_THREADS / 32];
     __shared__ int s_best_i[FO_THREADS / 32];
@@ -38,30 +37,18 @@ __global__ void __launch_bounds__(FO_THREADS) first_output_kernel(float* __restr
     int n = enc_len[b] - t0[b];
     n = n < 0 ? 0 : (n > W ? W : n);
     float* base = logp + (size_t)b * W * NV;
-    // ---- log-sum-exp per row: row maximum, then the sum of exponentials ----
-    for (int w = 0; w < n; ++w) {
+    // ---- log-sum-exp per row, one warp per row (no block-wide synchronisation inside): maximum, then sum of exponentials ----
+    for (int w = warp; w < n; w += FO_THREADS / 32) {
         const float* row = base + (size_t)w * NV;
         float mx = -CUDART_INF_F;
-        for (int v = threadIdx.x; v < NV; v += FO_THREADS) mx = fmaxf(mx, row[v]);
+        for (int v = lane; v < NV; v += 32) mx = fmaxf(mx, row[v]);
         mx = fo_warp_max(mx);
-        if (lane == 0) s_part[warp] = mx;
-        __syncthreads();
-        mx = s_part[0];
-#pragma unroll
-        for (int k = 1; k < FO_THREADS / 32; ++k) mx = fmaxf(mx, s_part[k]);
-        __syncthreads();
         float se = 0.f;
-        for (int v = threadIdx.x; v < NV; v += FO_THREADS) se += expf(row[v] - mx);
+        for (int v = lane; v < NV; v += 32) se += expf(row[v] - mx);
         se = fo_warp_sum(se);
-        if (lane == 0) s_part[warp] = se;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            float tot = 0.f;
-            for (int k = 0; k < FO_THREADS / 32; ++k) tot += s_part[k];
-            s_lse[w] = mx + logf(tot);
-        }
-        __syncthreads();
+        if (lane == 0) s_lse[w] = mx + logf(se);
     }
+    __syncthreads();
     // ---- running sum of the blank log-probabilities (the product over earlier frames in Eq. 1) ----
     if (threadIdx.x == 0) {
         float before = 0.f;
@@ -71,11 +58,11 @@ __global__ void __launch_bounds__(FO_THREADS) first_output_kernel(float* __restr
         }
     }
     __syncthreads();
-    // ---- log P'(v, t) in place ----
-    for (int w = 0; w < n; ++w) {
+    // ---- log P'(v, t) in place, one warp per row ----
+    for (int w = warp; w < n; w += FO_THREADS / 32) {
         float* row = base + (size_t)w * NV;
         const float shift = s_before[w] - s_lse[w];
-        for (int v = threadIdx.x; v < NV; v += FO_THREADS) {
+        for (int v = lane; v < NV; v += 32) {
             const float x = row[v] + shift;
             row[v] = (v == blank && w != n - 1) ? -CUDART_INF_F : x;
         }
@@ -86,6 +73,63 @@ __global__ void __launch_bounds__(FO_THREADS) first_output_kernel(float* __restr
     if (threadIdx.x == 0) { s_prev_v = CUDART_INF_F; s_prev_i = -1; }
     __syncthreads();
     const int total = n * NV;
+    constexpr int KLOC = 8;
+    if (K <= KLOC) {
+        // one pass over the window: every thread keeps the K best of its own elements (sorted, best first), then K
+        // rounds pick the best of the threads' current heads; the winning thread moves on to its next one
+        float lv[KLOC];
+        int li[KLOC];
+#pragma unroll
+        for (int j = 0; j < KLOC; ++j) { lv[j] = -CUDART_INF_F; li[j] = 0x7fffffff; }
+        for (int i = threadIdx.x; i < total; i += FO_THREADS) {
+            float x = base[i];
+            int xi = i;
+            if (x > -CUDART_INF_F) {
+#pragma unroll
+                for (int j = 0; j < KLOC; ++j) {
+                    // i ascends, so on equal values the earlier element stays ahead
+                    if (j < K && x > lv[j]) {
+                        const float tv = lv[j]; const int ti = li[j];
+                        lv[j] = x; li[j] = xi;
+                        x = tv; xi = ti;
+                    }
+                }
+            }
+        }
+        for (int k = 0; k < K; ++k) {
+            float bv = lv[0];
+            int bi = li[0];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+            }
+            if (lane == 0) { s_best_v[warp] = bv; s_best_i[warp] = bi; }
+            __syncthreads();
+            bv = s_best_v[0]; bi = s_best_i[0];
+#pragma unroll
+            for (int q = 1; q < FO_THREADS / 32; ++q) {
+                const float ov = s_best_v[q];
+                const int oi = s_best_i[q];
+                if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+            }
+            const bool any = bv > -CUDART_INF_F;
+            if (any && li[0] == bi) {   // this thread's head was taken: shift its list
+#pragma unroll
+                for (int j = 0; j < KLOC - 1; ++j) { lv[j] = lv[j + 1]; li[j] = li[j + 1]; }
+                lv[KLOC - 1] = -CUDART_INF_F; li[KLOC - 1] = 0x7fffffff;
+            }
+            if (threadIdx.x == 0) {
+                const int off = any ? bi / NV : -1;
+                top_label[(size_t)b * K + k] = any ? bi - off * NV : -1;
+                top_jump[(size_t)b * K + k] = off;
+                top_logp[(size_t)b * K + k] = any ? bv : -CUDART_INF_F;
+            }
+            __syncthreads();
+        }
+        return;
+    }
     for (int k = 0; k < K; ++k) {
         const float pv = s_prev_v;
         const int pi = s_prev_i;

@@ -107,7 +107,7 @@ def test_first_output_fp32_odd_shapes(pkg):
     run_case(pkg, w, enc, lens, W=5, K=4, seed=1)
 
 
-@pytest.mark.parametrize("name,W,K", [("cfg3_large_b128", 8, 3), ("cfg5_bigvocab", 4, 8)])
+@pytest.mark.parametrize("name,W,K", [("cfg3_large_b128", 8, 3), ("cfg5_bigvocab", 4, 8), ("cfg3_large_b128", 4, 12)])
 def test_first_output_bf16_model_shapes(pkg, name, W, K):
     cfg = ws.small_variant(ws.CONFIGS[name], 6, 20, 70)
     weights = ws.make_model(cfg)
