@@ -77,6 +77,19 @@ def test_invalid_arguments_are_rejected_on_the_host(lib):
     assert lib.wind_decode_greedy_host(*args) == bd.WIND_ERR_INVALID_ARG
     assert lib.wind_eval_joint_window(ref, None, None, 1, 10, 4, None, 0, None, None, None, None, 0, None) == bd.WIND_ERR_INVALID_ARG
     assert lib.wind_read_stats(None, None, None) == bd.WIND_ERR_INVALID_ARG
+    fo = [ref, None, None, 1, 10, 4, None, 0, None, None, None, 0, None, None, None, None, 0, None]
+    assert lib.wind_window_first_output(*fo) == bd.WIND_ERR_INVALID_ARG
+    fo[11] = -1
+    assert lib.wind_window_first_output(*fo) == bd.WIND_ERR_INVALID_ARG      # K < 0
+    fo[11] = 3
+    assert lib.wind_window_first_output(*fo) == bd.WIND_ERR_INVALID_ARG      # K > 0 without output arrays
+    n_ev = C.c_int32(0)
+    assert lib.wind_read_trace(ref, 1, 10, 4, None, None, None, 0, C.byref(n_ev)) == bd.WIND_ERR_INVALID_ARG
+
+
+def test_debug_hooks_round_trip(lib):
+    assert pkg.wind_set_trace(5) == -2 and pkg.wind_set_trace(-9) == 5 and pkg.wind_set_trace(-2) == -2
+    assert pkg.wind_debug_stall_barrier(2) == 0 and pkg.wind_debug_stall_barrier(0) == 2
 
 
 def test_set_kernels_round_trip(lib):
