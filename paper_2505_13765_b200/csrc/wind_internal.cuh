@@ -58,6 +58,7 @@ struct Layout {
     size_t pred_proj;  // fp32 [B][H]        (plain-ALU path)
     size_t hb;         // bf16 [2][L][Bpad][P] LSTM hidden state as tensor-core operand rows (tensor path)
     size_t z;          // bf16 [rows_pad][H] joint activations act(enc_proj + pred_proj), the joint GEMM's operand (tensor path)
+    size_t dh;         // fp32 [B][4P] layer 1's recurrent term, handed from its CTAs to the layer's update (tensor path, L >= 2)
     size_t g0;         // fp32 [V+1][4P] layer-0 gate pre-activations of every token: W_ih emb[tok] + b_ih + b_hh (tensor path)
     size_t trace;      // TraceEvent [kTraceRoles][kTraceEvents]: optional timeline of CTA 0 of the loop kernel
     size_t enc_proj;   // elem [B*T][H]
@@ -89,6 +90,7 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     L.Bpad = (B + 127) / 128 * 128;
     L.hb = take(bf ? 2 * (size_t)m.L * L.Bpad * m.P * 2 : 0);
     L.z = take(bf ? (size_t)L.rows_pad * m.H * 2 : 0);
+    L.dh = take(bf && m.L >= 2 ? sizeof(float) * (size_t)B * 4 * m.P : 0);
     L.g0 = take(bf ? sizeof(float) * (size_t)(m.V + 1) * 4 * m.P : 0);
     L.trace = take(bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents : 0);
     L.enc_proj = take(es * (size_t)B * T * m.H);
@@ -134,6 +136,7 @@ struct Call {
     void* enc_proj() const { return ws + lay.enc_proj; }
     __nv_bfloat16* z() const { return reinterpret_cast<__nv_bfloat16*>(ws + lay.z); }
     float* g0() const { return reinterpret_cast<float*>(ws + lay.g0); }
+    float* dh() const { return reinterpret_cast<float*>(ws + lay.dh); }
     TraceEvent* trace() const { return reinterpret_cast<TraceEvent*>(ws + lay.trace); }
     __nv_bfloat16* hb(int parity, int l) const {
         return reinterpret_cast<__nv_bfloat16*>(ws + lay.hb) + ((size_t)parity * m.L + l) * lay.Bpad * m.P;

@@ -183,17 +183,25 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
     }
     // resident-weights mode: CTAs [0, l_items) keep a W_hh tile (4 gates x 16 units), the last p_items CTAs a W_pred
     // tile (64 rows), loaded once; `stat` holds kb_p blocks of 64 rows x 64 columns
+    // With two LSTM layers two more CTA sets follow the layer-0 set: "x1" keeps a W_ih[1] tile (layer 1's GEMM on the
+    // new layer-0 state, in its own phase) and "h1" a W_hh[1] tile (layer 1's recurrent term, issued a phase ahead
+    // like layer 0's GEMM and handed over through global memory).
+    const int r_role = RES ? cta / p.l_items : 0;                  // 0 layer 0, 1 x1, 2 h1 (while below the L CTA count)
+    const int r_idx = RES ? cta - r_role * p.l_items : 0;
     const bool res_l = RES && cta < p.l_items;
-    const bool res_p = RES && !res_l && G - 1 - cta < p.p_items;
-    const int r_ut = cta % p.ut_count, r_ql = cta / p.ut_count;                      // unit tile / utterance group of an L CTA
+    const bool res_x1 = RES && p.L == 2 && r_role == 1;
+    const bool res_h1 = RES && p.L == 2 && r_role == 2;
+    const bool res_p = RES && !res_l && !res_x1 && !res_h1 && G - 1 - cta < p.p_items;
+    const int r_ut = r_idx % p.ut_count, r_ql = r_idx / p.ut_count;                  // unit tile / utterance group of an L CTA
     const int r_ht = (G - 1 - cta) % p.ht_count, r_qp = (G - 1 - cta) / p.ht_count;  // H tile / utterance group of a P CTA
     constexpr uint32_t RES_A_BYTES = 64 * BK * 2;
-    if (threadIdx.x == 0 && (res_l || res_p)) {
+    if (threadIdx.x == 0 && (res_l || res_x1 || res_h1 || res_p)) {
         mbar_expect_tx(&stat_bar, (uint32_t)p.kb_p * RES_A_BYTES);
         for (int kb = 0; kb < p.kb_p; ++kb) {
             uint8_t* dst = stat + (size_t)kb * RES_A_BYTES;
-            if (res_l) {
-                for (int g = 0; g < 4; ++g) tma_load_2d(dst + g * 16 * 128, &M.w_hh_r, kb * BK, g * p.P + r_ut * 16, &stat_bar);
+            if (!res_p) {
+                const CUtensorMap* wm = res_l ? &M.w_hh_r : (res_x1 ? &M.w_ih1_r : &M.w_hh1_r);
+                for (int g = 0; g < 4; ++g) tma_load_2d(dst + g * 16 * 128, wm, kb * BK, g * p.P + r_ut * 16, &stat_bar);
             } else {
                 tma_load_2d(dst, &M.w_pred_r, kb * BK, r_ht * 64, &stat_bar);
             }
@@ -542,18 +550,19 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
     // of a pass are requested together: first everything the control step needs, then the gate-table rows of the
     // chosen tokens.  Lanes 16..31 hold no accumulator row (64-row tile); they take the second 16 utterances.
     struct ScanIn { int t, len, cnt, pos; unsigned long long kk[8]; };
-    auto epilogue_res_L = [&]() -> bool {
+    auto epilogue_res_L = [&](const int layer) -> bool {
         const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
         int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
         const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
         unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
         const int u16 = lane & 15, half = lane >> 4;
         const int unit = r_ut * 16 + u16;        // this thread's hidden unit; its gate is q
-        const bool writer = r_ut == 0 && q == 0; // the two gate-0 warps of one CTA per utterance group record the step
-        const bool decode = step >= 0 && !p.forced;
-        float* cst = p.c_state + unit;
-        const __nv_bfloat16* hin = p.hb + ((size_t)pin * p.Bpad) * p.P + unit;
-        __nv_bfloat16* hout = p.hb + ((size_t)(pin ^ 1) * p.Bpad) * p.P + unit;
+        const bool writer = layer == 0 && r_ut == 0 && q == 0; // the two gate-0 warps of one CTA per utterance group record the step
+        const bool decode = step >= 0 && !p.forced && layer == 0;
+        float* cst = p.c_state + (size_t)layer * p.B * p.P + unit;
+        const __nv_bfloat16* hin = p.hb + ((size_t)(pin * p.L + layer) * p.Bpad) * p.P + unit;
+        __nv_bfloat16* hout = p.hb + ((size_t)((pin ^ 1) * p.L + layer) * p.Bpad) * p.P + unit;
+        const float bias1 = layer == 0 ? 0.f : p.b_ih[1][q * p.P + unit] + p.b_hh[1][q * p.P + unit];
         const float* g0u = p.g0 + (size_t)q * p.P + unit;
         const uint32_t g0_stride = 4u * (uint32_t)p.P;
         bool ready = true;
@@ -589,6 +598,8 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     tok = p.blank;
                 } else if (p.forced) {
                     tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
+                } else if (layer > 0) {
+                    tok = p.emit_tok[b];     // decided by layer 0's CTAs one phase earlier
                 } else {
                     int t = si.t;
                     const int len = si.len;
@@ -666,6 +677,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 // the next frame goes out at once, stamped with the step, for the projection CTAs (which fetch their
                 // enc_proj rows while this phase is still running)
                 if (writer && !p.forced) p.t_pub[b] = ((unsigned long long)(uint32_t)(step + 2) << 32) | (uint32_t)t_out;
+                if (writer && p.L > 1 && decode) p.emit_tok[b] = tok;   // the upper layer's CTAs read it in their phase
             }
             if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
             // ---- gate-table entries (this thread's gate and unit) of the tokens of this lane half's 16 utterances ----
@@ -674,7 +686,13 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             for (int j = 0; j < 16; ++j) {
                 const int ta = __shfl_sync(0xffffffffu, tok, j), tb = __shfl_sync(0xffffffffu, tok, 16 + j);
                 const int tj = half ? tb : ta;
-                add[j] = tj >= 0 ? g0u[(uint32_t)tj * g0_stride] : 0.f;
+                if (layer == 0) {
+                    add[j] = tj >= 0 ? g0u[(uint32_t)tj * g0_stride] : 0.f;
+                } else {
+                    // layer 1: the recurrent term W_hh h computed a phase ahead by the h1 CTAs, plus the biases
+                    const int bj2 = b0 + 32 * sub + 16 * half + j;
+                    add[j] = (tj >= 0 && bj2 < p.B) ? p.dh[(size_t)bj2 * g0_stride + (size_t)q * p.P + unit] + bias1 : 0.f;
+                }
             }
             // the other warps need the tokens for the cell update below: through shared memory
             int* tok_s = reinterpret_cast<int*>(stage_f + 4 * 64 * 16);
@@ -905,15 +923,49 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         return ready;
     };
     // the decoder GEMM of the next step, on the state hb[pin] (TMA and MMA issuers of an L CTA)
+    // h1 CTAs: the finished recurrent term of layer 1 goes to global memory (fp32 [B][4P], gate-major like the gate
+    // table); the x1 CTAs add it one or two phases later
+    auto store_res_h1 = [&]() {
+        const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, &s_abort));
+        tc_fence_after();
+        if (ready) {
+            const int unit = r_ut * 16 + (lane & 15);
+            for (int c0 = 0; c0 < p.nl; c0 += 64) {
+                const int col = c0 + 32 * sub;
+                float x[16], hi[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) { x[j] = 0.f; hi[j] = 0.f; }
+                if (col < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)col, x);
+                if (col + 16 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(col + 16), hi);
+                if (lane < 16) {
+                    float* dst = p.dh + (size_t)q * p.P + unit;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int ba = r_ql * p.nl + col + j, bb = ba + 16;
+                        if (col + j < p.nl && ba < p.B) dst[(size_t)ba * 4 * p.P] = x[j];
+                        if (col + 16 + j < p.nl && bb < p.B) dst[(size_t)bb * 4 * p.P] = hi[j];
+                    }
+                }
+            }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[1]);
+        ++acc_n[1];
+    };
+    // GEMMs that need only the state, issued a phase ahead: layer 0's (its result waits in tensor memory for the
+    // next control step) and, with two layers, layer 1's recurrent term (stored by store_res_h1)
     auto early_res = [&]() {
         if (warp == 0) {
-            if (lane == 0 && res_l) {
+            if (lane == 0 && (res_l || res_h1)) {
                 fence_proxy_async_all();
-                if (produce_one(&M.hb_l3[pin], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u))
+                if (produce_one(res_l ? &M.hb_l3[pin] : &M.hb_l3_1[pin], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u))
                     mma_part(1, tm_l, p.nl, p.kb_p, p.kb_p, false);   // one accumulator: warp 1 issues all of it
             }
         } else if (warp == 1) {
-            if (lane == 0 && res_l) mma_part(1, tm_l, p.nl, 0, p.kb_p, false);
+            if (lane == 0 && (res_l || res_h1)) mma_part(1, tm_l, p.nl, 0, p.kb_p, false);
+        } else if (res_h1) {
+            store_res_h1();
         }
     };
 
@@ -935,11 +987,26 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         if constexpr (RES) {
             if (warp >= 2) {
                 if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_START);
-                if (res_l) epilogue_res_L();
+                if (res_l) epilogue_res_L(0);
                 else if (res_p) prefetch_res_P();
                 if (cta == 0 && e == 0 && step >= 0 && !p.forced) p.ctrl->step = step + 1;
             }
             if (!grid_sync(TR_L)) goto done;
+            if (p.L == 2) {
+                // layer 1: W_ih[1] . (new layer-0 state) on the x1 CTAs, then their cell update
+                if (warp == 0) {
+                    if (lane == 0 && res_x1) {
+                        fence_proxy_async_all();
+                        if (produce_one(&M.hb_l3[pin ^ 1], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u))
+                            mma_part(1, tm_l, p.nl, p.kb_p, p.kb_p, false);
+                    }
+                } else if (warp == 1) {
+                    if (lane == 0 && res_x1) mma_part(1, tm_l, p.nl, 0, p.kb_p, false);
+                } else if (res_x1) {
+                    epilogue_res_L(1);
+                }
+                if (!grid_sync(TR_L)) goto done;
+            }
         }
         for (int l = 0; l < p.L && !RES; ++l) {
             const bool gemm_here = l > 0 || !early;
@@ -1449,7 +1516,8 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
     // W_pred in tiles of 64 rows stay in the shared memory of disjoint CTA sets for the whole decode; per step a CTA
     // fetches only its utterance group's rows of the state, as one box.
     const char* res_env = getenv("WIND_RESIDENT");
-    if (m.L == 1 && one_wave && m.H / 2 + 2 * pl.nj <= (int)LOOP_TMEM_COLS && !(res_env && atoi(res_env) == 0)) {
+    if (m.L <= 2 && one_wave && m.H / 2 + 2 * pl.nj <= (int)LOOP_TMEM_COLS && !(res_env && atoi(res_env) == 0)) {
+        const int l_sets = m.L == 2 ? 3 : 1;   // layer 0; with two layers also layer 1's input and recurrent halves
         LoopPlan r = pl;
         r.ut_count = m.P / 16;
         r.ht_count = m.H / 64;
@@ -1457,7 +1525,7 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
         for (int nl : {16, 32, 64, 128}) {
             for (int npr : {16, 32, 64, 128}) {
                 const int ql = (c.B + nl - 1) / nl, qp = (c.B + npr - 1) / npr;
-                if (r.ut_count * ql + r.ht_count * qp <= G) {
+                if (l_sets * r.ut_count * ql + r.ht_count * qp <= G) {
                     r.nl = nl; r.np = npr; r.ql_count = ql; r.qp_count = qp;
                     found = true;
                     break;
@@ -1517,9 +1585,14 @@ cudaError_t loop_prepare(Call& c) {
     if (pl.resident) {
         WIND_MAP(loop_map(&M.w_hh_r, c.w_hh[0], 4ull * m.P, m.P, 16));
         WIND_MAP(loop_map(&M.w_pred_r, m.w_pred, m.H, m.P, 64));
+        if (m.L == 2) {
+            WIND_MAP(loop_map(&M.w_ih1_r, c.w_ih[1], 4ull * m.P, m.P, 16));
+            WIND_MAP(loop_map(&M.w_hh1_r, c.w_hh[1], 4ull * m.P, m.P, 16));
+        }
         for (int par = 0; par < 2; ++par) {
             WIND_MAP(loop_map3(&M.hb_l3[par], c.hb(par, 0), c.lay.Bpad, m.P, pl.nl));
-            WIND_MAP(loop_map3(&M.hb_p3[par], c.hb(par, 0), c.lay.Bpad, m.P, pl.np));
+            if (m.L == 2) WIND_MAP(loop_map3(&M.hb_l3_1[par], c.hb(par, 1), c.lay.Bpad, m.P, pl.nl));
+            WIND_MAP(loop_map3(&M.hb_p3[par], c.hb(par, m.L - 1), c.lay.Bpad, m.P, pl.np));
         }
         WIND_MAP(loop_map3(&M.z3, c.z(), (uint64_t)c.lay.rows_pad, m.H, pl.nj));
     }
@@ -1558,7 +1631,7 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.stat_bytes = pl.stat_bytes;
     p.enc_len = c.enc_len; p.t2 = c.t(); p.t_pub = c.t_pub(); p.count = c.count(); p.emit_tok = c.emit_tok(); p.keys2 = c.keys();
     p.out_tokens = c.out_tokens; p.out_frames = c.out_frames; p.out_len = c.out_len;
-    p.c_state = c.c(); p.hb = c.hb(0, 0); p.z = c.z(); p.enc_proj = (const __nv_bfloat16*)c.enc_proj(); p.g0 = c.g0();
+    p.c_state = c.c(); p.dh = c.dh(); p.hb = c.hb(0, 0); p.z = c.z(); p.enc_proj = (const __nv_bfloat16*)c.enc_proj(); p.g0 = c.g0();
     for (int l = 0; l < c.m.L; ++l) { p.b_ih[l] = c.b_ih[l]; p.b_hh[l] = c.b_hh[l]; }
     p.b_pred = c.m.b_pred; p.b_out = c.m.b_out; p.w_out = (const __nv_bfloat16*)c.m.w_out;
     p.forced = logits_out != nullptr; p.prefix = prefix; p.U = U; p.prefix_len = prefix_len; p.logits_out = logits_out;

@@ -21,7 +21,9 @@ struct LoopMaps {
     // three-dimensional box each (64 columns, rows, all K blocks)
     CUtensorMap w_hh_r;                // [4P, P], box 16 rows (one gate's 16 units)
     CUtensorMap w_pred_r;              // [H, P], box 64 rows
-    CUtensorMap hb_l3[2];              // [Bpad, P] as (64, rows, P/64), box (64, nl, P/64)
+    CUtensorMap w_ih1_r, w_hh1_r;      // layer 1 (two-layer models): [4P, P], box 16 rows
+    CUtensorMap hb_l3[2];              // layer 0 state [Bpad, P] as (64, rows, P/64), box (64, nl, P/64)
+    CUtensorMap hb_l3_1[2];            // layer 1 state, same box
     CUtensorMap hb_p3[2];              // same, box (64, np, P/64)
     CUtensorMap z3;                    // [rows_pad, H] as (64, rows, H/64), box (64, nj, H/64)
 };
@@ -68,6 +70,7 @@ struct LoopParams {
     int32_t* out_frames;
     int32_t* out_len;
     float* c_state;                // [L][B][P]
+    float* dh;                     // [B][4P] layer 1's recurrent term W_hh[1] h (two-layer resident mode)
     __nv_bfloat16* hb;             // [2][L][Bpad][P]
     __nv_bfloat16* z;              // [rows_pad][H]
     const __nv_bfloat16* enc_proj; // [B*T][H]
