@@ -881,6 +881,10 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 float g[16], more[16];
                 tmem_ld16(tm_p + lane_off + (uint32_t)c0, g);
                 tmem_ld16(tm_p + lane_off + (uint32_t)(p.np + c0), more);   // the other issuing thread's K blocks
+                if (p.kb_p < 2) {   // a single K block: the first copy's issuer had an empty range and wrote nothing
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) g[j] = 0.f;
+                }
                 if (lane < 16) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) stage_f[(c0 + j) * 68 + hl] = g[j] + more[j] + bias;
@@ -1303,6 +1307,10 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                             }
                             if (RES) {   // second accumulator copy (the other issuing thread's K blocks)
                                 float more[16];
+                                if (p.kb_h < 2) {   // a single K block: nothing was written to the first copy
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) val[j] = (j < 16 || c0 + 16 < n_tile) ? 0.f : val[j];
+                                }
                                 tmem_ld16(tm_j + lane_off + (uint32_t)(n_tile + c0), more);
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) val[j] += more[j];

@@ -242,6 +242,30 @@ def test_bf16_tensor_path_with_biases_and_other_blank_ids(pkg, L, blank0, act, B
     logits_parity(pkg, w, enc, lens, W=W, S=4, tol=TOL["bf16"], n_windows=2 * B, kernels=2)
 
 
+@pytest.mark.parametrize("resident", [1, 0])
+def test_bf16_tensor_path_more_utterances_than_one_tile(pkg, monkeypatch, resident):
+    # 150 utterances, one K block per GEMM (H = P = 64): ten utterance groups per weight tile in the resident-weights
+    # mode; two 128-row utterance tiles in the streaming mode (forced by the planner's environment switch)
+    if not resident:
+        monkeypatch.setenv("WIND_RESIDENT", "0")
+    w, enc, lens = ragged_case(91, B=150, T=24, D=64, E=64, P=64, L=1, H=64, V=140, act=0, bias=1.0, dtype="bf16")
+    rep, _ = check_against_oracle(pkg, w, enc, lens, 4, 3, kernels=2)
+    assert rep["stats"]["kernels"] == 2
+
+
+def test_bf16_tensor_path_output_overflow(pkg):
+    w, enc, lens = ragged_case(92, B=5, T=30, D=64, E=64, P=64, L=1, H=64, V=140, bias=-3.0, dtype="bf16")
+    model = pkg.WindModel(w)
+    full = pkg.decode(model, enc, lens, 4, 3)
+    assert full[4] == 0 and full[3]["kernels"] == 2 and full[2].max() > 5
+    tok, frm, olen, stats, st = pkg.decode(model, enc, lens, 4, 3, max_out=5, check=False)
+    assert st == pkg.binding.WIND_ERR_OUTPUT_OVERFLOW
+    assert olen.max() == 5
+    for b in range(5):
+        n = min(5, full[2][b])
+        assert olen[b] == n and np.array_equal(tok[b, :n], full[0][b, :n]) and np.array_equal(frm[b, :n], full[1][b, :n])
+
+
 def test_cfg2_large_b1(pkg):
     cfg = ws.CONFIGS["cfg2_large_b1"]
     weights = ws.make_model(cfg)
