@@ -253,6 +253,28 @@ def test_bf16_tensor_path_more_utterances_than_one_tile(pkg, monkeypatch, reside
     assert rep["stats"]["kernels"] == 2
 
 
+@pytest.mark.parametrize("B,W,S,P,H,V,L", [
+    (1, 3, 2, 128, 192, 127, 1),       # one utterance; V + 1 = exactly one vocabulary tile
+    (17, 20, 3, 192, 64, 300, 2),      # window wider than the control step's 8-row pass; one K block in the joint
+    (129, 1, 5, 64, 128, 140, 2),      # W = 1 (Algorithm 1), one utterance beyond a 128 tile
+    (200, 8, 3, 128, 128, 257, 1),     # third vocabulary tile holds two entries
+    (64, 5, 1, 192, 192, 200, 1),      # S = 1: every emission is followed by a forced advance
+    (300, 2, 3, 64, 64, 130, 1),
+    (40, 32, 4, 128, 64, 500, 2),
+    (148, 4, 3, 256, 256, 1000, 2),
+])
+@pytest.mark.parametrize("resident", [1, 0])
+def test_bf16_tensor_path_shape_sweep(pkg, monkeypatch, resident, B, W, S, P, H, V, L):
+    # shapes that send the tile planner of the loop kernel down its different branches, with the resident-weights
+    # mode allowed and with the planner's environment switch forcing the streaming mode
+    if not resident:
+        monkeypatch.setenv("WIND_RESIDENT", "0")
+    w, enc, lens = ragged_case(300 + B + W, B=B, T=20, D=64, E=64, P=P, L=L, H=H, V=V, act=B % 2, bias=1.5,
+                               dtype="bf16")
+    rep, _ = check_against_oracle(pkg, w, enc, lens, W, S, kernels=2)
+    assert rep["stats"]["kernels"] == 2
+
+
 def test_bf16_tensor_path_output_overflow(pkg):
     w, enc, lens = ragged_case(92, B=5, T=30, D=64, E=64, P=64, L=1, H=64, V=140, bias=-3.0, dtype="bf16")
     model = pkg.WindModel(w)
