@@ -233,8 +233,8 @@ def test_bf16_joint_logits(pkg, kernels, name, W):
 
 @pytest.mark.parametrize("L,blank0,act,B,W", [(1, True, 1, 9, 4), (1, False, 0, 70, 8), (2, True, 0, 5, 16), (2, False, 1, 33, 2)])
 def test_bf16_tensor_path_with_biases_and_other_blank_ids(pkg, L, blank0, act, B, W):
-    # tile-sized dimensions, so the tensor-core kernels run (one layer: weights resident in shared memory; two
-    # layers: streamed), with every bias vector non-zero and the blank either first or last
+    # tile-sized dimensions, so the tensor-core kernels run (weights resident in shared memory, for one and for two
+    # layers), with every bias vector non-zero and the blank either first or last
     w, enc, lens = ragged_case(70 + L + 2 * B, B=B, T=60, D=128, E=192, P=128, L=L, H=192, V=300, act=act,
                                blank_id=0 if blank0 else None, bias=1.0, dtype="bf16")
     rep, _ = check_against_oracle(pkg, w, enc, lens, W, 4, kernels=2)
@@ -251,6 +251,7 @@ def test_bf16_tensor_path_more_utterances_than_one_tile(pkg, monkeypatch, reside
     w, enc, lens = ragged_case(91, B=150, T=24, D=64, E=64, P=64, L=1, H=64, V=140, act=0, bias=1.0, dtype="bf16")
     rep, _ = check_against_oracle(pkg, w, enc, lens, 4, 3, kernels=2)
     assert rep["stats"]["kernels"] == 2
+    logits_parity(pkg, w, enc, lens, W=4, S=3, tol=TOL["bf16"], n_windows=150, kernels=2)
 
 
 @pytest.mark.parametrize("B,W,S,P,H,V,L", [
