@@ -357,9 +357,17 @@ def roofline(pkg, model, cfg, W, enc_d, len_d, tok_d, frm_d, ol_d, wsb, stream, 
         achieved = flop / dur_s / 1e12
         js = res["joint_ms"] * 1e-3
         dense = 2.0 * cfg.H * (cfg.V + 1) * cfg.B * W * stats["steps"]
+        # DRAM bytes per launch: ncu counters (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of this
+        # kernel on the same shapes with 18975 frames (profiles/loop_kernel_cfg3_b128_short.md): 37.1 MB, of which
+        # the enc_proj rows (2 H bytes per frame, each read once) grow with the workload and 12.8 MB (weights, gate
+        # table, outputs) do not.  Scaled by the frame count; other shapes have no capture.
+        traffic, traffic_source = None, None
+        if (cfg.name, W, cfg.B) == ("cfg3_large_b128", 8, 128):
+            traffic = 12.8e6 + 2.0 * cfg.H * frames
+            traffic_source = "ncu capture at 18975 frames, enc_proj part scaled by frames"
         return {"kernel": "decoding loop (one persistent launch: joint, decoder-update and projection phases)",
                 "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                "peak_source": peaks["source"] + " sustained bf16", "traffic": None,
+                "peak_source": peaks["source"] + " sustained bf16", "traffic": traffic, "traffic_source": traffic_source,
                 "launch_ms": res["loop_ms"], "algorithmic_gflop_per_launch": flop / 1e9,
                 "joint_phase": {"us_per_step": js * 1e6 / max(1, stats["steps"]), "achieved": joint_flop / js / 1e12,
                                 "frac": joint_flop / js / 1e12 / peak, "dense_issued_frac": dense / js / 1e12 / peak,
