@@ -94,6 +94,11 @@ def lib():
         L.oracle_eval_joint_window.restype = C.c_int32
         L.oracle_first_output_logprobs.argtypes = [mp, f32p, C.c_int32, i32p, C.c_int32, C.c_int32, C.c_int32, f64p]
         L.oracle_first_output_logprobs.restype = C.c_int32
+        L.oracle_decode_window_greedy_batch.argtypes = L.oracle_decode_batch.argtypes
+        L.oracle_decode_window_greedy_batch.restype = None
+        L.oracle_replay_verify_window.argtypes = [mp, f32p, C.c_int32, C.c_int32, C.c_int32, C.c_double, i32p, i32p,
+                                                  C.c_int32, i64p, i64p, i64p, i32p]
+        L.oracle_replay_verify_window.restype = C.c_int32
     return _lib
 
 
@@ -155,6 +160,39 @@ def decode_batch(model: Model, enc: np.ndarray, enc_len: np.ndarray, W: int, S: 
     lib().oracle_decode_batch(model.ref, _ptr(enc, f32p), _ptr(enc_len, i32p), B, T, W, S, margin_thr,
                               _ptr(tokens, i32p), _ptr(frames, i32p), _ptr(out_len, i32p), max_out, C.byref(st))
     return tokens, frames, out_len, st.as_dict()
+
+
+def decode_window_greedy_batch(model: Model, enc: np.ndarray, enc_len: np.ndarray, W: int, S: int,
+                               max_out: Optional[int] = None, margin_thr: float = 0.05):
+    """Window-based greedy decoding (the best (label, offset) pair of Eq. (1) at every step)."""
+    enc = _f32(enc)
+    B, T, D = enc.shape
+    assert D == model.dims["D"]
+    enc_len = np.ascontiguousarray(enc_len, dtype=np.int32)
+    if max_out is None:
+        max_out = max(1, T * S)
+    tokens = np.full((B, max_out), -1, np.int32)
+    frames = np.full((B, max_out), -1, np.int32)
+    out_len = np.zeros(B, np.int32)
+    st = OracleStats()
+    lib().oracle_decode_window_greedy_batch(model.ref, _ptr(enc, f32p), _ptr(enc_len, i32p), B, T, W, S, margin_thr,
+                                            _ptr(tokens, i32p), _ptr(frames, i32p), _ptr(out_len, i32p), max_out,
+                                            C.byref(st))
+    return tokens, frames, out_len, st.as_dict()
+
+
+def replay_verify_window(model: Model, enc_b: np.ndarray, T: int, W: int, S: int, tokens: np.ndarray,
+                         frames: np.ndarray, margin_thr: float = 0.05):
+    """Check one utterance's (token, frame) list against window-based greedy decoding with the same W and S."""
+    enc_b = _f32(enc_b)
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    frames = np.ascontiguousarray(frames, dtype=np.int32)
+    nd, nl, nn = C.c_int64(0), C.c_int64(0), C.c_int64(0)
+    bad = C.c_int32(-1)
+    rc = lib().oracle_replay_verify_window(model.ref, _ptr(enc_b, f32p), int(T), int(W), int(S), margin_thr,
+                                           _ptr(tokens, i32p), _ptr(frames, i32p), len(tokens),
+                                           C.byref(nd), C.byref(nl), C.byref(nn), C.byref(bad))
+    return dict(rc=int(rc), decisions=nd.value, low_margin=nl.value, not_argmax=nn.value, bad_pos=bad.value)
 
 
 def replay_verify(model: Model, enc_b: np.ndarray, T: int, S: int, tokens: np.ndarray, frames: np.ndarray,

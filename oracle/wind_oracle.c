@@ -22,6 +22,11 @@
  * the S-th token is still emitted and fed to the decoder, then t advances by
  * one.  The counter resets whenever t advances.
  *
+ * The file also holds Eq. (1) (first-output distribution of a window) and window-based greedy decoding, which
+ * takes the most probable (label, offset) pair of Eq. (1) at every step; their pins: the distribution sums to
+ * one, closed forms, W = 1 equals Algorithm 1, a step-by-step recomputation from Eq. (1) in the tests, and a
+ * hand-worked example where it differs from Algorithm 2.
+ *
  * Pins (see tests): WIND(W) == sequential for every W; brute-force tabulation
  * of joint argmaxes on tiny models; LSTM / linear layers against library fp64
  * routines and closed forms; S honoured; jump-size support.
@@ -298,6 +303,36 @@ void oracle_decode_batch(const oracle_model_t* m, const float* enc, const int32_
     free(sts);
 }
 
+/* forward declaration: defined at the end of the file */
+int32_t oracle_decode_window_greedy(const oracle_model_t* m, const float* enc, int32_t T, int32_t W, int32_t S,
+                                    double margin_thr, int32_t* out_tokens, int32_t* out_frames, int32_t max_out,
+                                    oracle_stats_t* st);
+
+/* Window-based greedy decoding of a batch: the same plain loop over utterances. */
+void oracle_decode_window_greedy_batch(const oracle_model_t* m, const float* enc, const int32_t* enc_len, int32_t B,
+                                       int32_t T, int32_t W, int32_t S, double margin_thr, int32_t* out_tokens,
+                                       int32_t* out_frames, int32_t* out_len, int32_t max_out, oracle_stats_t* st_total) {
+    oracle_stats_t* sts = (oracle_stats_t*)calloc((size_t)B, sizeof(oracle_stats_t));
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b)
+        out_len[b] = oracle_decode_window_greedy(m, enc + (size_t)b * T * m->D, enc_len[b], W, S, margin_thr,
+                                                 out_tokens + (size_t)b * max_out, out_frames + (size_t)b * max_out,
+                                                 max_out, &sts[b]);
+    if (st_total) {
+        memset(st_total, 0, sizeof(*st_total));
+        for (int b = 0; b < B; ++b) {
+            st_total->steps += sts[b].steps;
+            st_total->joint_rows += sts[b].joint_rows;
+            st_total->pred_updates += sts[b].pred_updates;
+            st_total->forced += sts[b].forced;
+            st_total->low_margin += sts[b].low_margin;
+            st_total->decisions += sts[b].decisions;
+            for (int k = 0; k < 65; ++k) st_total->jump_hist[k] += sts[b].jump_hist[k];
+        }
+    }
+    free(sts);
+}
+
 /*
  * Replay check of a (token, frame) sequence produced elsewhere against the
  * sequential definition.  Walk frames from 0; the sequence implies one choice
@@ -416,4 +451,161 @@ int32_t oracle_first_output_logprobs(const oracle_model_t* m, const float* enc, 
     }
     free(logits);
     return n;
+}
+
+/*
+ * Window-based greedy decoding: at every step the window's first-output distribution P'(v, t) of Eq. (1) is
+ * evaluated under the current decoder state and the single most probable (label, offset) pair is taken
+ * (the variant sketched beside Algorithm 2: "find the best prediction based on the whole window").
+ *   pair (v != blank, j): emit v at frame t + j, then t += j (the next window starts ON the emitting frame);
+ *   blank (only at the window's last row, i.e. the window is all blank): t += n.
+ * Candidates are compared in the order j ascending, label ascending, the all-blank candidate last; the first
+ * strict maximum wins.  The safeguard against staying on one frame is the one of the greedy decoders above.
+ * Unlike Algorithm 2 the result depends on W (W = 1 is Algorithm 1).
+ *
+ * window_scores(): log P' restricted to what the decision needs, from the logits of the n rows:
+ *   best[j]   = log P'(v_j, j) for the best non-blank label v_j of row j,
+ *   *all_blank = log P'(blank, n - 1).
+ */
+static void window_scores(const oracle_model_t* m, const double* logits, int n, double* best, int* best_label,
+                          double* all_blank) {
+    const int NV = m->V + 1;
+    double blanks_before = 0.0;
+    for (int j = 0; j < n; ++j) {
+        const double* row = logits + (size_t)j * NV;
+        double mx = row[0];
+        for (int v = 1; v < NV; ++v)
+            if (row[v] > mx) mx = row[v];
+        double se = 0.0;
+        for (int v = 0; v < NV; ++v) se += exp(row[v] - mx);
+        const double lse = mx + log(se);
+        int bl = -1;
+        for (int v = 0; v < NV; ++v)
+            if (v != m->blank_id && (bl < 0 || row[v] > row[bl])) bl = v;
+        best_label[j] = bl;
+        best[j] = blanks_before + row[bl] - lse;
+        blanks_before += row[m->blank_id] - lse;
+    }
+    *all_blank = blanks_before;
+}
+
+int32_t oracle_decode_window_greedy(const oracle_model_t* m, const float* enc, int32_t T, int32_t W, int32_t S,
+                                    double margin_thr, int32_t* out_tokens, int32_t* out_frames, int32_t max_out,
+                                    oracle_stats_t* st) {
+    if (W < 1 || W > 64) return -1;
+    scratch_t s;
+    scratch_alloc(m, T, &s);
+    oracle_enc_proj(m, enc, T, s.encp);
+    decoder_start(m, &s);
+    const int NV = m->V + 1;
+    double* logits = (double*)malloc(sizeof(double) * (size_t)W * NV);
+    int32_t n_out = 0, t = 0, count = 0;
+    while (t < T) {
+        const int n = (W < T - t) ? W : (T - t);
+        for (int w = 0; w < n; ++w)
+            oracle_joint_logits(m, s.encp + (size_t)(t + w) * m->H, s.g, s.z, logits + (size_t)w * NV);
+        double best[64], all_blank;
+        int best_label[64];
+        window_scores(m, logits, n, best, best_label, &all_blank);
+        int pick = -1; /* row of the chosen pair, -1 = all blank */
+        double top = -INFINITY, second = -INFINITY;
+        for (int j = 0; j <= n; ++j) {
+            const double sc = j < n ? best[j] : all_blank;
+            if (sc > top) { second = top; top = sc; pick = j < n ? j : -1; }
+            else if (sc > second) second = sc;
+        }
+        if (st) {
+            st->steps++;
+            st->joint_rows += n;
+            st->decisions++;
+            if (top - second < margin_thr) st->low_margin++;
+            st->jump_hist[pick < 0 ? n : pick]++;
+        }
+        if (pick < 0) { t += n; count = 0; continue; }
+        if (pick > 0) count = 0;
+        t += pick;
+        if (n_out < max_out) { out_tokens[n_out] = best_label[pick]; out_frames[n_out] = t; }
+        n_out++;
+        if (st) st->pred_updates++;
+        decoder_feed(m, &s, best_label[pick]);
+        count++;
+        if (count == S) { t += 1; count = 0; if (st) st->forced++; }
+    }
+    free(logits);
+    scratch_free(&s);
+    return n_out;
+}
+
+/*
+ * Replay check of a (token, frame) sequence produced elsewhere against window-based greedy decoding with the
+ * same W and S.  At every step the sequence implies one candidate: the next listed token if its frame lies
+ * inside the current window, else "all blank".  The implied candidate's log P' must be the maximum over the
+ * window's candidates, or lie within margin_thr of it (counted in *n_not_argmax when it is not the oracle's pick).
+ * The label of a pair must be the row's best non-blank label or within margin_thr of it in that row's logits.
+ * Return codes as in oracle_replay_verify.
+ */
+int32_t oracle_replay_verify_window(const oracle_model_t* m, const float* enc, int32_t T, int32_t W, int32_t S,
+                                    double margin_thr, const int32_t* tokens, const int32_t* frames, int32_t n_tok,
+                                    int64_t* n_decisions, int64_t* n_low_margin, int64_t* n_not_argmax,
+                                    int32_t* bad_pos) {
+    if (W < 1 || W > 64) return -1;
+    scratch_t s;
+    scratch_alloc(m, T, &s);
+    oracle_enc_proj(m, enc, T, s.encp);
+    decoder_start(m, &s);
+    const int NV = m->V + 1;
+    double* logits = (double*)malloc(sizeof(double) * (size_t)W * NV);
+    int32_t rc = 0, t = 0, count = 0, idx = 0;
+    int64_t dec = 0, low = 0, notmax = 0;
+    for (int k = 0; k < n_tok && !rc; ++k) {
+        if (tokens[k] < 0 || tokens[k] > m->V || tokens[k] == m->blank_id) { rc = 3; *bad_pos = k; }
+        if (frames[k] < 0 || frames[k] >= T || (k > 0 && frames[k] < frames[k - 1])) { rc = 2; *bad_pos = k; }
+    }
+    while (!rc && t < T) {
+        const int n = (W < T - t) ? W : (T - t);
+        for (int w = 0; w < n; ++w)
+            oracle_joint_logits(m, s.encp + (size_t)(t + w) * m->H, s.g, s.z, logits + (size_t)w * NV);
+        double best[64], all_blank;
+        int best_label[64];
+        window_scores(m, logits, n, best, best_label, &all_blank);
+        double top = all_blank, second = -INFINITY;
+        int pick = -1;
+        for (int j = 0; j < n; ++j) {
+            if (best[j] > top) { second = top; top = best[j]; pick = j; }
+            else if (best[j] > second) second = best[j];
+        }
+        if (idx < n_tok && frames[idx] < t) { rc = 2; *bad_pos = t; break; }
+        const int j = (idx < n_tok && frames[idx] < t + n) ? frames[idx] - t : -1;
+        dec++;
+        if (top - second < margin_thr) low++;
+        if (j < 0) {
+            if (pick >= 0) {
+                notmax++;
+                if (!(all_blank >= top - margin_thr)) { rc = 1; *bad_pos = t; break; }
+            }
+            t += n;
+            count = 0;
+            continue;
+        }
+        const int v = tokens[idx];
+        const double* row = logits + (size_t)j * NV;
+        const double sc = best[j] + (row[v] - row[best_label[j]]); /* log P'(v, j) */
+        if (j != pick || v != best_label[j]) {
+            notmax++;
+            if (!(sc >= top - margin_thr)) { rc = 1; *bad_pos = t; break; }
+        }
+        if (j > 0) count = 0;
+        t += j;
+        decoder_feed(m, &s, v);
+        idx++;
+        count++;
+        if (count == S) { t += 1; count = 0; }
+    }
+    if (!rc && idx != n_tok) { rc = 2; *bad_pos = T; }
+    if (n_decisions) *n_decisions = dec;
+    if (n_low_margin) *n_low_margin = low;
+    if (n_not_argmax) *n_not_argmax = notmax;
+    free(logits);
+    scratch_free(&s);
+    return rc;
 }

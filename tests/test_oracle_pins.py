@@ -425,3 +425,141 @@ def test_first_output_argmax_is_the_greedy_jump_when_blank_dominates_or_not():
         else:
             assert (t_best, v_best) == (len(labels) - 1, w["blank_id"])
     assert checked >= 4
+
+
+# ---------------------------------------------------------------------------
+# window-based greedy decoding (the best (label, offset) pair of Eq. (1) at every step)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("seed,bias,S", [(0, 1.0, 3), (1, 0.0, 2), (2, -1.0, 1), (3, 1.5, 10)])
+def test_window_greedy_with_a_one_frame_window_is_algorithm_1(seed, bias, S):
+    # one row: log P'(v, 0) = log softmax, whose argmax is the logits' argmax
+    w, enc, lens = small_case(80 + seed, bias=bias, S=S)
+    m = oracle.Model(w)
+    ref = oracle.decode_batch(m, enc, lens, W=0, S=S)
+    got = oracle.decode_window_greedy_batch(m, enc, lens, W=1, S=S)
+    assert np.array_equal(ref[2], got[2]) and np.array_equal(ref[0], got[0]) and np.array_equal(ref[1], got[1])
+    assert got[3]["forced"] == ref[3]["forced"]
+
+
+def brute_force_window_greedy(nm, enc, W, S):
+    """The variant's rules on independently evaluated logits: the whole table log P'(v, j) is built with library
+    routines (log_softmax, cumsum) and its first maximum in (row, label) order is taken, the all-blank entry last."""
+    T = enc.shape[0]
+    hyp, frames, t, count = [], [], 0, 0
+    while t < T:
+        n = min(W, T - t)
+        lg = np.stack([nm.logits(enc[t + j], hyp) for j in range(n)])
+        lp = torch.log_softmax(torch.tensor(lg), dim=1).numpy()
+        before = np.concatenate([[0.0], np.cumsum(lp[:, nm.blank])])   # blanks on rows < j
+        table = lp + before[:n, None]
+        table[:, nm.blank] = -np.inf
+        flat = int(np.argmax(table))                                   # first maximum, rows ascending then labels
+        j, v = divmod(flat, lp.shape[1])
+        if before[n] > table[j, v]:                                    # the all-blank candidate wins only strictly
+            t += n
+            count = 0
+            continue
+        if j > 0:
+            count = 0
+        t += j
+        hyp.append(v)
+        frames.append(t)
+        count += 1
+        if count == S:
+            t += 1
+            count = 0
+    return hyp, frames
+
+
+@pytest.mark.parametrize("seed,W,S,bias,blank0,act", [(0, 2, 3, 0.5, False, 0), (1, 4, 2, 1.0, True, 1), (2, 8, 3, 0.0, False, 0),
+                                                     (3, 3, 1, -0.5, False, 1), (4, 5, 4, 2.0, True, 0)])
+def test_window_greedy_matches_brute_force(seed, W, S, bias, blank0, act):
+    r = rng(900 + seed)
+    V = 9
+    w = random_weights(r, 6, 5, 6, 1 + seed % 2, 8, V, blank_id=0 if blank0 else None, act=act, blank_bias=bias, bias_scale=0.1)
+    T = 26
+    enc = r.standard_normal((1, T, 6)).astype(np.float32)
+    m = oracle.Model(w)
+    tok, frm, n, st = oracle.decode_window_greedy_batch(m, enc, np.array([T], np.int32), W=W, S=S)
+    hyp, frames = brute_force_window_greedy(NaiveModel(w), enc[0], W, S)
+    assert list(tok[0, : n[0]]) == hyp and list(frm[0, : n[0]]) == frames
+    hist = np.array(st["jump_hist"])
+    assert (hist * np.arange(65)).sum() + st["forced"] == T and hist[W + 1:].sum() == 0
+    assert st["pred_updates"] == n[0] and st["steps"] == st["decisions"] == hist.sum()
+
+
+def table_model(probs):
+    """A joiner whose output does not depend on the decoder: frame type k (a one-hot encoder frame) has the label
+    distribution probs[k] (labels 0..V-1, blank last)."""
+    probs = np.asarray(probs, np.float64)
+    K, NV = probs.shape
+    V = NV - 1
+    z = lambda *s: np.zeros(s, np.float32)
+    return dict(D=K, E=2, P=2, L=1, H=K, V=V, blank_id=V, act=0, dtype="f32", emb=z(NV, 2),
+                w_ih=[z(8, 2)], w_hh=[z(8, 2)], b_ih=[z(8)], b_hh=[z(8)],
+                w_enc=np.eye(K, dtype=np.float32), b_enc=z(K), w_pred=z(K, 2), b_pred=z(K),
+                w_out=np.log(probs).T.astype(np.float32), b_out=z(NV))
+
+
+def test_window_greedy_worked_example_differs_from_algorithm_2():
+    # frame types: A = (x .45, y .05, blank .5), B = (x .1, y .8, blank .1), C = (x .02, y .03, blank .95)
+    # utterance A B C C, W = 2, S = 1 (every emission is followed by a forced advance):
+    #   window [A, B]: P'(x,0) = .45, P'(y,0) = .05, P'(x,1) = .5 * .1, P'(y,1) = .5 * .8 = .4, all blank = .05  -> x at frame 0
+    #   window [B, C]: P'(y,0) = .8 is the largest                                                               -> y at frame 1
+    #   window [C, C]: all blank = .9025                                                                         -> end
+    # Algorithms 1 and 2 take the per-frame argmax: A -> blank (.5 > .45), B -> y, C -> blank: only y at frame 1.
+    w = table_model([[.45, .05, .5], [.1, .8, .1], [.02, .03, .95]])
+    enc = np.eye(3, dtype=np.float32)[[0, 1, 2, 2]][None]
+    lens = np.array([4], np.int32)
+    m = oracle.Model(w)
+    tok, frm, n, st = oracle.decode_window_greedy_batch(m, enc, lens, W=2, S=1)
+    assert list(tok[0, : n[0]]) == [0, 1] and list(frm[0, : n[0]]) == [0, 1]
+    assert st["steps"] == 3 and st["forced"] == 2 and st["jump_hist"][0] == 2 and st["jump_hist"][2] == 1
+    for W in (1, 2, 4):
+        tok2, frm2, n2, _ = oracle.decode_batch(m, enc, lens, W=W, S=1)
+        assert list(tok2[0, : n2[0]]) == [1] and list(frm2[0, : n2[0]]) == [1]
+    tok1, frm1, n1, _ = oracle.decode_window_greedy_batch(m, enc, lens, W=1, S=1)
+    assert list(tok1[0, : n1[0]]) == [1] and list(frm1[0, : n1[0]]) == [1]
+    # W = 3: window [A, B, C]: .45 for x at 0 still beats .4; then [B, C, C]: y at 1; then [C, C]
+    tok3, frm3, n3, _ = oracle.decode_window_greedy_batch(m, enc, lens, W=3, S=1)
+    assert list(tok3[0, : n3[0]]) == [0, 1] and list(frm3[0, : n3[0]]) == [0, 1]
+    # a later pair can win over an earlier one: A' = (x .3, y .1, blank .6): P'(y,1) = .6 * .8 = .48 > .3 -> jump to frame 1
+    w2 = table_model([[.3, .1, .6], [.1, .8, .1], [.02, .03, .95]])
+    tok4, frm4, n4, st4 = oracle.decode_window_greedy_batch(oracle.Model(w2), enc, lens, W=2, S=1)
+    assert list(tok4[0, : n4[0]]) == [1] and list(frm4[0, : n4[0]]) == [1] and st4["jump_hist"][1] == 1
+
+
+def test_window_replay_accepts_own_output_and_rejects_mistakes():
+    w, enc, lens = small_case(61, B=2, bias=0.9, S=3)
+    m = oracle.Model(w)
+    W = 4
+    tok, frm, n, st = oracle.decode_window_greedy_batch(m, enc, lens, W=W, S=3)
+    b, T = 0, int(lens[0])
+    tk, fr = tok[b, : n[b]].copy(), frm[b, : n[b]].copy()
+    assert n[b] >= 3
+    ok = oracle.replay_verify_window(m, enc[b], T, W, 3, tk, fr, margin_thr=0.0)
+    assert ok["rc"] == 0 and ok["not_argmax"] == 0
+    one = oracle.decode_window_greedy_batch(m, enc[b : b + 1], lens[b : b + 1], W=W, S=3)
+    assert ok["decisions"] == one[3]["decisions"]
+    # the same sequence is in general not what another window size produces
+    assert oracle.replay_verify_window(m, enc[b], T, W, 3, np.delete(tk, 1), np.delete(fr, 1), margin_thr=0.0)["rc"] == 1
+    fr2 = fr.copy()
+    fr2[0], fr2[-1] = fr[-1], fr[0]
+    if fr[0] != fr[-1]:
+        assert oracle.replay_verify_window(m, enc[b], T, W, 3, tk, fr2)["rc"] == 2
+    tk3 = tk.copy()
+    tk3[0] = w["blank_id"]
+    assert oracle.replay_verify_window(m, enc[b], T, W, 3, tk3, fr)["rc"] == 3
+    # a different label at the first decision passes only with a margin above its gap in log P'
+    lp = oracle.first_output_logprobs(m, enc[b], T, [], 0, W)
+    j = int(fr[0])
+    assert j < W
+    other = next(v for v in np.argsort(-lp[j]) if v != tk[0] and v != w["blank_id"])
+    gap = lp.max() - lp[j, other]
+    tk4 = tk.copy()
+    tk4[0] = other
+    res = oracle.replay_verify_window(m, enc[b], T, W, 3, tk4[:1], fr[:1], margin_thr=gap * 0.5)
+    assert res["rc"] == 1 and res["bad_pos"] == 0 and res["decisions"] == 1
+    # with a margin above the gap the first decision passes (whatever happens at the second one)
+    res = oracle.replay_verify_window(m, enc[b], T, W, 3, tk4[:1], fr[:1], margin_thr=gap * 1.01)
+    assert res["decisions"] >= 2 and res["not_argmax"] >= 1
