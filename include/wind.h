@@ -102,9 +102,10 @@ typedef struct {
 /*
  * Bytes of device workspace needed by wind_decode_greedy / wind_eval_joint_window for
  * batches up to B utterances of up to T frames and window W.  Holds enc_proj [B,T,H],
- * the decoder state, the per-row argmax keys (8 bytes per window row: the window logits
- * themselves -- W x (V+1) floats per utterance in the paper's memory analysis -- never
- * leave the chip) and control words.  Grows with W only by the key array.
+ * the decoder state, per window row a few argmax keys, the joint's activations and (for
+ * window-based decoding) per-tile softmax statistics -- the window logits themselves,
+ * W x (V+1) floats per utterance in the paper's memory analysis, never leave the chip --
+ * and control words.  Grows with W only by these per-row arrays.
  */
 wind_status_t wind_workspace_bytes(const wind_model_t* m, int32_t B, int32_t T, int32_t W, size_t* bytes);
 
@@ -129,6 +130,23 @@ wind_status_t wind_decode_greedy(const wind_model_t* m, const void* enc, const i
                                  int32_t T, int32_t W, int32_t max_symbols, int32_t* out_tokens,
                                  int32_t* out_frames, int32_t* out_len, int32_t max_out, void* workspace,
                                  size_t workspace_bytes, void* stream);
+
+/*
+ * Window-based greedy decoding: at every step the window's first-output distribution P'(v, t) of Eq. (1) is
+ * formed under the current decoder state and its most probable entry decides the step (the variant sketched
+ * beside Algorithm 2, which looks at the whole window instead of stopping at the first frame whose own argmax is
+ * not blank):
+ *   pair (v != blank, offset j): v is emitted at frame t + j and t += j;
+ *   the blank entry (only the window's last row has one: every row blank): t += n.
+ * Candidates are compared in the order offsets ascending, labels ascending, the blank entry last; the first
+ * strict maximum wins.  log-softmax, the running sum of blank log-probabilities and the comparison are fp32.
+ * The max_symbols rule, every argument, the outputs, the workspace (same size) and the status codes are those of
+ * wind_decode_greedy.  W == 1 gives Algorithm 1; for W > 1 the result depends on W.
+ */
+wind_status_t wind_decode_window_greedy(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B,
+                                        int32_t T, int32_t W, int32_t max_symbols, int32_t* out_tokens,
+                                        int32_t* out_frames, int32_t* out_len, int32_t max_out, void* workspace,
+                                        size_t workspace_bytes, void* stream);
 
 /*
  * Extra workspace (added to wind_workspace_bytes) that wind_decode_greedy_host needs for

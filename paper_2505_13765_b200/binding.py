@@ -29,7 +29,7 @@ WIND_DT_F32, WIND_DT_BF16 = 0, 1
 WIND_KERNELS_AUTO, WIND_KERNELS_SIMT, WIND_KERNELS_TENSOR = 0, 1, 2
 
 EXPORTS = [
-    "wind_workspace_bytes", "wind_decode_greedy", "wind_host_staging_bytes", "wind_decode_greedy_host",
+    "wind_workspace_bytes", "wind_decode_greedy", "wind_decode_window_greedy", "wind_host_staging_bytes", "wind_decode_greedy_host",
     "wind_eval_joint_window", "wind_window_first_output", "wind_eval_joint_window_static", "wind_profile_decode", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_debug_stall_barrier", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
 ]
 
@@ -93,6 +93,8 @@ def load_library():
     L.wind_host_staging_bytes.restype = i32
     dec = [mp, _vp, _vp, i32, i32, i32, i32, _vp, _vp, _vp, i32, _vp, C.c_size_t, _vp]
     L.wind_decode_greedy.argtypes = dec
+    L.wind_decode_window_greedy.argtypes = dec
+    L.wind_decode_window_greedy.restype = i32
     L.wind_decode_greedy.restype = i32
     L.wind_decode_greedy_host.argtypes = dec
     L.wind_decode_greedy_host.restype = i32
@@ -280,6 +282,21 @@ def wind_decode_greedy(model: WindModel, enc, enc_len, W: int, max_symbols: int,
     return st
 
 
+def wind_decode_window_greedy(model: WindModel, enc, enc_len, W: int, max_symbols: int, out_tokens, out_frames, out_len,
+                              workspace, stream=None, check: bool = True) -> int:
+    """Window-based greedy decoding; arguments as wind_decode_greedy."""
+    L = load_library()
+    B, T, D = enc.shape
+    assert enc.is_contiguous() and enc.dtype == model.torch_dtype and D == model.dims["D"]
+    max_out = out_tokens.shape[1]
+    st = L.wind_decode_window_greedy(model.ref, enc.data_ptr(), enc_len.data_ptr(), B, T, W, max_symbols,
+                                     out_tokens.data_ptr(), out_frames.data_ptr(), out_len.data_ptr(), max_out,
+                                     _ws_ptr(workspace), _ws_bytes(workspace), _stream_ptr(stream))
+    if check and st != WIND_OK:
+        raise WindError(st)
+    return st
+
+
 def wind_decode_greedy_host(model: WindModel, enc_host, enc_len_host, W: int, max_symbols: int, out_tokens_host,
                             out_frames_host, out_len_host, workspace, stream=None, check: bool = True) -> int:
     """Same as wind_decode_greedy with HOST (ideally pinned) torch tensors for enc, enc_len and the outputs."""
@@ -375,7 +392,7 @@ def to_device_enc(model: WindModel, enc_np: np.ndarray):
 
 
 def decode(model: WindModel, enc_np: np.ndarray, lens_np: np.ndarray, W: int, S: int, max_out: Optional[int] = None,
-           check: bool = True):
+           check: bool = True, window_greedy: bool = False):
     """Marshals numpy inputs to the device, decodes, returns numpy (tokens, frames, out_len, stats, status)."""
     torch = _torch()
     B, T, _ = enc_np.shape
@@ -387,6 +404,7 @@ def decode(model: WindModel, enc_np: np.ndarray, lens_np: np.ndarray, W: int, S:
     frm = torch.full((B, max_out), -1, dtype=torch.int32, device=model.device)
     olen = torch.zeros(B, dtype=torch.int32, device=model.device)
     ws = alloc_workspace(model, B, T, W)
-    st = wind_decode_greedy(model, enc, lens, W, S, tok, frm, olen, ws, check=check)
+    call = wind_decode_window_greedy if window_greedy else wind_decode_greedy
+    st = call(model, enc, lens, W, S, tok, frm, olen, ws, check=check)
     stats = wind_read_stats(ws)
     return tok.cpu().numpy(), frm.cpu().numpy(), olen.cpu().numpy(), stats, st

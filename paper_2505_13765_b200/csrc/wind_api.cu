@@ -268,6 +268,21 @@ wind_status_t wind_decode_greedy(const wind_model_t* m, const void* enc, const i
     return read_status(c);
 }
 
+wind_status_t wind_decode_window_greedy(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B, int32_t T,
+                                        int32_t W, int32_t max_symbols, int32_t* out_tokens, int32_t* out_frames,
+                                        int32_t* out_len, int32_t max_out, void* workspace, size_t workspace_bytes,
+                                        void* stream) {
+    wind_status_t s = check_decode_args(m, enc, enc_len, B, T, W, max_symbols, out_tokens, out_frames, out_len, max_out, workspace);
+    if (s != WIND_OK) return s;
+    Call c;
+    fill_call(c, m, enc, enc_len, B, T, W, max_symbols, out_tokens, out_frames, out_len, max_out, workspace, (cudaStream_t)stream);
+    c.mode = WIND_MODE_WINDOW;
+    if (workspace_bytes < c.lay.total) return WIND_ERR_WORKSPACE;
+    s = enqueue_decode(c);
+    if (s != WIND_OK) return s;
+    return read_status(c);
+}
+
 wind_status_t wind_decode_greedy_host(const wind_model_t* m, const void* enc_host, const int32_t* enc_len_host, int32_t B,
                                       int32_t T, int32_t W, int32_t max_symbols, int32_t* out_tokens_host,
                                       int32_t* out_frames_host, int32_t* out_len_host, int32_t max_out, void* workspace,

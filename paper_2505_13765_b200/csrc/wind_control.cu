@@ -80,7 +80,7 @@ cudaError_t launch_init(const Call& c, int kernels_used, int launches_per_step, 
     init_kernel<<<blocks, 256, 0, c.stream>>>(c.ctrl(), c.t(), c.t_pub(), c.count(), c.emit_tok(), c.keys(), c.h(0), c.c(),
                                               reinterpret_cast<uint32_t*>(c.hb(0, 0)), reinterpret_cast<uint32_t*>(c.z()),
                                               reinterpret_cast<uint32_t*>(c.trace()),
-                                              bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents / 4 : 0, c.out_len, c.enc_len, c.B, 2 * (size_t)c.lay.rows_pad, n_h, n_c, n_hb_words,
+                                              bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents / 4 : 0, c.out_len, c.enc_len, c.B, 3 * (size_t)c.lay.rows_pad, n_h, n_c, n_hb_words,
                                               n_z_words, c.m.blank_id, (int)step_cap, kernels_used, launches_per_step,
                                               launches_setup);
     return cudaGetLastError();

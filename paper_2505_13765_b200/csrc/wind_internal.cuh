@@ -10,6 +10,8 @@
 
 namespace wind {
 
+constexpr int WIND_MODE_FIRST_NONBLANK = 0;
+constexpr int WIND_MODE_WINDOW = 1;
 constexpr int kMaxLayers = 8;
 constexpr int kMaxWindow = 64;
 constexpr size_t kAlign = 256;
@@ -52,7 +54,10 @@ struct Layout {
     size_t t_pub;      // uint64 [B]  (lock step + 2) << 32 | next frame: published early in a step for the projection CTAs
     size_t count;      // int32 [B]   consecutive emissions on the current frame
     size_t emit_tok;   // int32 [B]   token to feed to the decoder this step, -1 = none
-    size_t keys;       // uint64 [2][rows_pad] packed (logit, label) argmax keys, 0 = empty (second half: loop kernel)
+    size_t keys;       // uint64 [3][rows_pad] packed (logit, label) argmax keys, 0 = empty ([1]: loop kernel's other step
+                       // parity; [2]: best non-blank key per row in window-based decoding)
+    size_t jpart;      // float2 [rows_pad][4 * vocabulary tiles] partial (maximum, sum of exponentials) of each row's logits
+    size_t jblank;     // fp32 [rows_pad] blank logit of each window row (both: window-based decoding on the tensor path)
     size_t h;          // fp32 [2][L][B][P]  LSTM hidden state, ping-pong by step parity (plain-ALU path)
     size_t c;          // fp32 [L][B][P]     LSTM cell state
     size_t pred_proj;  // fp32 [B][H]        (plain-ALU path)
@@ -83,7 +88,7 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     L.t_pub = take(sizeof(uint64_t) * B);
     L.count = take(sizeof(int32_t) * B);
     L.emit_tok = take(sizeof(int32_t) * B);
-    L.keys = take(sizeof(uint64_t) * 2 * (size_t)L.rows_pad);
+    L.keys = take(sizeof(uint64_t) * 3 * (size_t)L.rows_pad);
     L.h = take(sizeof(float) * 2 * (size_t)m.L * B * m.P);
     L.c = take(sizeof(float) * (size_t)m.L * B * m.P);
     L.pred_proj = take(sizeof(float) * (size_t)B * m.H);
@@ -93,6 +98,8 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     L.dh = take(bf && m.L >= 2 ? sizeof(float) * (size_t)B * 4 * m.P : 0);
     L.g0 = take(bf ? sizeof(float) * (size_t)(m.V + 1) * 4 * m.P : 0);
     L.trace = take(bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents : 0);
+    L.jpart = take(bf ? sizeof(float) * 2 * (size_t)L.rows_pad * 4 * ((size_t)(m.V + 1 + 127) / 128) : 0);
+    L.jblank = take(bf ? sizeof(float) * (size_t)L.rows_pad : 0);
     L.enc_proj = take(es * (size_t)B * T * m.H);
     L.total = off;
     L.st_enc = take(es * (size_t)B * T * m.D);
@@ -114,6 +121,7 @@ struct Call {
     const void* enc;
     const int32_t* enc_len;
     int32_t B, T, W, S, max_out;
+    int32_t mode;     // WIND_MODE_FIRST_NONBLANK (Algorithm 2) or WIND_MODE_WINDOW (best pair of Eq. (1) per step)
     int32_t* out_tokens;
     int32_t* out_frames;
     int32_t* out_len;
@@ -137,6 +145,8 @@ struct Call {
     __nv_bfloat16* z() const { return reinterpret_cast<__nv_bfloat16*>(ws + lay.z); }
     float* g0() const { return reinterpret_cast<float*>(ws + lay.g0); }
     float* dh() const { return reinterpret_cast<float*>(ws + lay.dh); }
+    float2* jpart() const { return reinterpret_cast<float2*>(ws + lay.jpart); }
+    float* jblank() const { return reinterpret_cast<float*>(ws + lay.jblank); }
     TraceEvent* trace() const { return reinterpret_cast<TraceEvent*>(ws + lay.trace); }
     __nv_bfloat16* hb(int parity, int l) const {
         return reinterpret_cast<__nv_bfloat16*>(ws + lay.hb) + ((size_t)parity * m.L + l) * lay.Bpad * m.P;
@@ -155,6 +165,10 @@ __device__ inline unsigned long long pack_key(float logit, uint32_t label) {
 }
 __host__ __device__ inline uint32_t key_label(unsigned long long key) {
     return 0xFFFFFFFFu - (uint32_t)(key & 0xFFFFFFFFull);
+}
+__device__ inline float key_logit(unsigned long long key) {
+    const uint32_t hi = (uint32_t)(key >> 32);
+    return __uint_as_float((hi & 0x80000000u) ? (hi & 0x7FFFFFFFu) : ~hi);
 }
 
 __device__ inline void set_status(Ctrl* ctrl, int32_t s) { atomicCAS(&ctrl->status, 0, s); }

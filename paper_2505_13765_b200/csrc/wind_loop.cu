@@ -1336,6 +1336,34 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                                     if (((okmask >> j) & 1u) && v_ok)
                                         p.logits_out[(size_t)(rg * n_tile + c0 + j) * p.NV + v] = val[j];
                             } else {
+                                unsigned long long* key_dst = keys_cur;
+                                if (p.window) {
+                                    // window-based decoding: this warp's 32 vocabulary entries give, per row, a partial
+                                    // (maximum, sum of exponentials) for the row's log-sum-exp; the blank's logit is
+                                    // stored on its own and the blank leaves the maximum search
+                                    float m_keep = -INFINITY, s_keep = 0.f;
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) {
+                                        float m = val[j];
+#pragma unroll
+                                        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+                                        float sm = val[j] > -INFINITY ? __expf(val[j] - m) : 0.f;
+#pragma unroll
+                                        for (int o = 16; o > 0; o >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, o);
+                                        if (lane == j) { m_keep = m; s_keep = sm; }
+                                    }
+                                    if (row < p.rows && c0 + lane < n_tile)
+                                        p.jpart[(size_t)row * p.parts + vt * 4 + q] = make_float2(m_keep, s_keep);
+                                    if (v == p.blank) {
+#pragma unroll
+                                        for (int j = 0; j < 32; ++j) {
+                                            const int rj = rg * n_tile + c0 + j;
+                                            if (rj < p.rows && c0 + j < n_tile) p.jblank[rj] = val[j];
+                                            val[j] = -INFINITY;
+                                        }
+                                    }
+                                    key_dst = p.nbkeys;
+                                }
                                 int id[32];
 #pragma unroll
                                 for (int j = 0; j < 32; ++j) id[j] = v;
@@ -1345,7 +1373,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                                 argmax_exchange<2>(val, id, lane);
                                 argmax_exchange<1>(val, id, lane);
                                 if (row < p.rows && c0 + lane < n_tile && val[0] > -INFINITY)
-                                    atomicMax(&keys_cur[row], pack_key(val[0], (uint32_t)id[0]));
+                                    atomicMax(&key_dst[row], pack_key(val[0], (uint32_t)id[0]));
                             }
                         }
                     }
@@ -1360,6 +1388,74 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             if (!grid_sync(TR_J)) goto done;
         }
         if (p.forced) break;
+        if (p.window) {
+            // =================================================================================
+            // window-based decoding: one warp per utterance turns the joint phase's per-row statistics into the
+            // most probable (label, offset) pair of Eq. (1) and leaves it in the keys in the form the control step
+            // reads (the chosen row carries its label, every other row the blank)
+            // =================================================================================
+            if (warp >= 2) {
+                const int n_ew = RES ? 8 : 4;
+                const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
+                unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
+                const unsigned long long blank_key = pack_key(0.f, (uint32_t)p.blank);
+                for (int b = (warp - 2) * G + cta; b < p.B; b += n_ew * G) {
+                    const int t = t_cur[b], len = p.enc_len[b];
+                    const int n = t < len ? min(p.W, len - t) : 0;
+                    float lpb[2], sc[2];
+                    unsigned long long key[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int j = lane + 32 * h;
+                        lpb[h] = 0.f; sc[h] = -INFINITY; key[h] = 0ull;
+                        if (j < n) {
+                            const size_t row = (size_t)b * p.W + j;
+                            const float2* part = p.jpart + row * p.parts;
+                            float mx = -INFINITY, se = 0.f;
+                            for (int k = 0; k < p.parts; ++k) {
+                                const float2 pr = part[k];
+                                if (pr.y > 0.f) {
+                                    if (pr.x > mx) { se = se * __expf(mx - pr.x) + pr.y; mx = pr.x; }
+                                    else se += pr.y * __expf(pr.x - mx);
+                                }
+                            }
+                            const float lse = mx + __logf(se);
+                            lpb[h] = p.jblank[row] - lse;
+                            key[h] = p.nbkeys[row];
+                            if (key[h] != 0ull) sc[h] = key_logit(key[h]) - lse;
+                        }
+                    }
+                    // blank log-probabilities of the rows before each row (rows 0..31 on the lanes, then rows 32..63)
+                    float incl0 = lpb[0], incl1 = lpb[1];
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const float a0 = __shfl_up_sync(0xffffffffu, incl0, o), a1 = __shfl_up_sync(0xffffffffu, incl1, o);
+                        if (lane >= o) { incl0 += a0; incl1 += a1; }
+                    }
+                    const float tot0 = __shfl_sync(0xffffffffu, incl0, 31), tot1 = __shfl_sync(0xffffffffu, incl1, 31);
+                    sc[0] += incl0 - lpb[0];
+                    sc[1] += tot0 + incl1 - lpb[1];
+                    // first strict maximum in row order; "all blank" (tot0 + tot1) wins only when strictly larger
+                    float top = sc[0];
+                    int pick = lane;
+                    if (sc[1] > top) { top = sc[1]; pick = lane + 32; }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const float ot = __shfl_xor_sync(0xffffffffu, top, o);
+                        const int op = __shfl_xor_sync(0xffffffffu, pick, o);
+                        if (ot > top || (ot == top && op < pick)) { top = ot; pick = op; }
+                    }
+                    if (!(top > -INFINITY) || tot0 + tot1 > top) pick = -1;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int j = lane + 32 * h;
+                        if (j < n) keys_cur[(size_t)b * p.W + j] = j == pick ? key[h] : blank_key;
+                        if (j < p.W) p.nbkeys[(size_t)b * p.W + j] = 0ull;
+                    }
+                }
+            }
+            if (!grid_sync(TR_J)) goto done;
+        }
     }
 done:
     // an accumulator may still hold an unused early GEMM; nothing reads it, the MMAs have completed
@@ -1645,6 +1741,8 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.forced = logits_out != nullptr; p.prefix = prefix; p.U = U; p.prefix_len = prefix_len; p.logits_out = logits_out;
     p.trace = trace_step >= -1 ? c.trace() : nullptr; p.trace_step = trace_step;
     p.extra_arrivals = g_loop_extra_arrivals;
+    p.window = c.mode == WIND_MODE_WINDOW && !logits_out;
+    p.nbkeys = c.keys() + 2 * (size_t)c.lay.rows_pad; p.jpart = c.jpart(); p.jblank = c.jblank(); p.parts = 4 * pl.vt_count;
     void* args[2] = {(void*)&t_loop_maps, (void*)&p};
     return cudaLaunchCooperativeKernel(pl.resident ? (const void*)loop_kernel<true> : (const void*)loop_kernel<false>, dim3((unsigned)pl.grid), dim3(pl.resident ? LOOP_THREADS_RES : LOOP_THREADS), args, pl.smem_bytes,
                                        c.stream);

@@ -89,6 +89,11 @@ struct LoopParams {
     // timeline of CTA 0 for lock steps [trace_step, trace_step + 2); trace == nullptr: off
     TraceEvent* trace;
     int trace_step;
+    // window-based decoding (the most probable pair of Eq. (1) per step instead of the first non-blank row)
+    int window, parts;             // parts = 4 per vocabulary tile: one (maximum, sum of exponentials) pair per epilogue warp
+    unsigned long long* nbkeys;    // [rows_pad] best non-blank (logit, label) per window row
+    float2* jpart;                 // [rows_pad][parts]
+    float* jblank;                 // [rows_pad] blank logit per window row
     int extra_arrivals;            // test hook: arrivals the grid barrier waits for beyond the grid size (0 in normal use)
 };
 

@@ -219,15 +219,25 @@ int simt_pred_launches(const Call& c) { return c.m.L + 1; }
 // logits[w, v] = W_out[v] . z[w] + b_out[v]; per-row argmax key (or the logits themselves).
 // Rows are taken in chunks of 8 so the activation tile stays small.
 // ---------------------------------------------------------------------------
-template <typename TW>
+//
+// WG (window-based greedy decoding): besides the row maximum over the non-blank labels the block gathers each
+// row's log-sum-exp and blank logit, picks the most probable (label, offset) pair of Eq. (1) (or "all blank") once
+// every row is done, and writes the keys in the form the control step reads: the chosen row carries its label, every
+// other row the blank, so that "first non-blank row" is the chosen pair.
+template <typename TW, bool WG>
 __global__ void __launch_bounds__(256) joint_simt_kernel(const Ctrl* __restrict__ ctrl, const int32_t* __restrict__ t_cur,
                                                          const int32_t* __restrict__ enc_len, const TW* __restrict__ enc_proj,
                                                          const float* __restrict__ pred_proj, const TW* __restrict__ w_out,
                                                          const float* __restrict__ b_out, unsigned long long* __restrict__ keys,
-                                                         float* __restrict__ logits_out, int T, int W, int H, int NV, int act) {
+                                                         float* __restrict__ logits_out, int T, int W, int H, int NV, int act,
+                                                         int blank) {
     if (ctrl->active == 0) return;
     extern __shared__ float z[];  // [8][H]
     __shared__ unsigned long long skey[8];
+    // window mode: per-warp running (maximum, sum of exponentials) of the chunk's rows; per-row results of the window
+    __shared__ float s_m[8][8], s_s[8][8];
+    __shared__ float s_lse[kMaxWindow], s_blank[kMaxWindow];
+    __shared__ unsigned long long s_best[kMaxWindow];
     const int b = blockIdx.x;
     const int t = t_cur[b], len = enc_len[b];
     if (t >= len) return;
@@ -244,6 +254,9 @@ __global__ void __launch_bounds__(256) joint_simt_kernel(const Ctrl* __restrict_
             z[e] = round_like<TW>(s);
         }
         __syncthreads();
+        float run_m[8], run_s[8];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) { run_m[w] = -INFINITY; run_s[w] = 0.f; }
         for (int v = warp; v < NV; v += nw) {
             float a[8];
 #pragma unroll
@@ -260,33 +273,72 @@ __global__ void __launch_bounds__(256) joint_simt_kernel(const Ctrl* __restrict_
                     float s = warp_sum(a[w]) + b_out[v];
                     if (lane == 0) {
                         if (logits_out) logits_out[((size_t)b * W + w0 + w) * NV + v] = s;
-                        atomicMax(&skey[w], pack_key(s, (uint32_t)v));
+                        if (!WG) {
+                            atomicMax(&skey[w], pack_key(s, (uint32_t)v));
+                        } else {
+                            if (v == blank) s_blank[w0 + w] = s;
+                            else atomicMax(&skey[w], pack_key(s, (uint32_t)v));
+                            if (s > run_m[w]) { run_s[w] = run_s[w] * __expf(run_m[w] - s) + 1.f; run_m[w] = s; }
+                            else run_s[w] += __expf(s - run_m[w]);
+                        }
                     }
                 }
             }
         }
+        if (WG && lane == 0) {
+#pragma unroll
+            for (int w = 0; w < 8; ++w) { s_m[warp][w] = run_m[w]; s_s[warp][w] = run_s[w]; }
+        }
         __syncthreads();
-        if (threadIdx.x < nc) keys[(size_t)b * W + w0 + threadIdx.x] = skey[threadIdx.x];
+        if (!WG) {
+            if (threadIdx.x < nc) keys[(size_t)b * W + w0 + threadIdx.x] = skey[threadIdx.x];
+        } else if (threadIdx.x < nc) {
+            const int w = threadIdx.x;
+            float mx = -INFINITY;
+            for (int k = 0; k < nw; ++k) mx = fmaxf(mx, s_m[k][w]);
+            float se = 0.f;
+            for (int k = 0; k < nw; ++k)
+                if (s_s[k][w] > 0.f) se += s_s[k][w] * __expf(s_m[k][w] - mx);
+            s_lse[w0 + w] = mx + __logf(se);
+            s_best[w0 + w] = skey[w];
+        }
+    }
+    if (WG) {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            // candidates in the order rows ascending (each row's best non-blank label), "all blank" last; first strict maximum
+            float before = 0.f, top = -INFINITY;
+            int pick = -1;
+            for (int j = 0; j < n; ++j) {
+                if (s_best[j] != 0ull) {
+                    const float sc = before + key_logit(s_best[j]) - s_lse[j];
+                    if (sc > top) { top = sc; pick = j; }
+                }
+                before += s_blank[j] - s_lse[j];
+            }
+            if (before > top) pick = -1;
+            const unsigned long long blank_key = pack_key(0.f, (uint32_t)blank);
+            for (int j = 0; j < n; ++j) keys[(size_t)b * W + j] = j == pick ? s_best[j] : blank_key;
+        }
     }
 }
 
-cudaError_t simt_joint(const Call& c, float* logits_out) {
-    size_t smem = sizeof(float) * 8 * (size_t)c.m.H;
-    if (c.B == 0) return cudaSuccess;
-    if (c.m.dtype == WIND_DT_BF16) {
-        if (smem > 48 * 1024)
-            cudaFuncSetAttribute(joint_simt_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        joint_simt_kernel<__nv_bfloat16><<<c.B, 256, smem, c.stream>>>(
-            c.ctrl(), c.t(), c.enc_len, (const __nv_bfloat16*)c.enc_proj(), c.pred_proj(), (const __nv_bfloat16*)c.m.w_out,
-            c.m.b_out, c.keys(), logits_out, c.T, c.W, c.m.H, c.m.V + 1, c.m.act);
-    } else {
-        if (smem > 48 * 1024)
-            cudaFuncSetAttribute(joint_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        joint_simt_kernel<float><<<c.B, 256, smem, c.stream>>>(c.ctrl(), c.t(), c.enc_len, (const float*)c.enc_proj(),
-                                                                c.pred_proj(), (const float*)c.m.w_out, c.m.b_out, c.keys(),
-                                                                logits_out, c.T, c.W, c.m.H, c.m.V + 1, c.m.act);
-    }
+template <typename TW, bool WG>
+static cudaError_t simt_joint_t(const Call& c, float* logits_out) {
+    const size_t smem = sizeof(float) * 8 * (size_t)c.m.H;
+    if (smem > 48 * 1024) cudaFuncSetAttribute(joint_simt_kernel<TW, WG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    joint_simt_kernel<TW, WG><<<c.B, 256, smem, c.stream>>>(c.ctrl(), c.t(), c.enc_len, (const TW*)c.enc_proj(), c.pred_proj(),
+                                                            (const TW*)c.m.w_out, c.m.b_out, c.keys(), logits_out, c.T, c.W,
+                                                            c.m.H, c.m.V + 1, c.m.act, c.m.blank_id);
     return cudaGetLastError();
+}
+
+cudaError_t simt_joint(const Call& c, float* logits_out) {
+    if (c.B == 0) return cudaSuccess;
+    const bool wg = c.mode == WIND_MODE_WINDOW && !logits_out;
+    if (c.m.dtype == WIND_DT_BF16)
+        return wg ? simt_joint_t<__nv_bfloat16, true>(c, logits_out) : simt_joint_t<__nv_bfloat16, false>(c, logits_out);
+    return wg ? simt_joint_t<float, true>(c, logits_out) : simt_joint_t<float, false>(c, logits_out);
 }
 
 }  // namespace wind

@@ -43,14 +43,16 @@ def test_status_strings(lib):
 def test_workspace_grows_with_window_only_by_keys_and_activations(lib):
     # The paper's memory analysis: WIND's only extra state is the window's logits,
     # W x (V+1) floats per utterance (16 x 1025 = 16400 floats for W = 16).  Here the
-    # logits stay on chip; per window row the workspace keeps two 8-byte argmax keys (double
-    # buffered by step parity) and the joint's H bf16 activations.
+    # logits stay on chip; per window row the workspace keeps three 8-byte argmax keys (two buffers by step
+    # parity, one for the best non-blank label in window-based decoding), the joint's H bf16 activations and, for
+    # window-based decoding, the blank logit and four (maximum, sum of exponentials) pairs per vocabulary tile.
     m = large_model()
     B, T = 128, 2500
+    tiles = (m.V + 1 + 127) // 128
     base = pkg.wind_workspace_bytes(m, B, T, 2)   # B * W = 256 rows: no row padding at even W
     for W in (4, 8, 16, 64):
         extra = pkg.wind_workspace_bytes(m, B, T, W) - base
-        assert extra == B * (W - 2) * (2 * 8 + 2 * m.H)
+        assert extra == B * (W - 2) * (3 * 8 + 2 * m.H + 4 + 8 * 4 * tiles)
         assert extra <= 4 * B * W * (m.V + 1)  # below the paper's W x (V+1) floats per utterance
     assert 16 * 1025 == 16400
     # dominated by enc_proj [B, T, H] in bf16; the gate table adds (V+1) x 4P floats
@@ -74,6 +76,7 @@ def test_invalid_arguments_are_rejected_on_the_host(lib):
     # null weights / buffers: rejected before any CUDA call (this machine may have no GPU at all)
     args = [ref, None, None, 1, 10, 4, 5, None, None, None, 50, None, 0, None]
     assert lib.wind_decode_greedy(*args) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_decode_window_greedy(*args) == bd.WIND_ERR_INVALID_ARG
     assert lib.wind_decode_greedy_host(*args) == bd.WIND_ERR_INVALID_ARG
     assert lib.wind_eval_joint_window(ref, None, None, 1, 10, 4, None, 0, None, None, None, None, 0, None) == bd.WIND_ERR_INVALID_ARG
     assert lib.wind_read_stats(None, None, None) == bd.WIND_ERR_INVALID_ARG
