@@ -87,6 +87,20 @@ __device__ __forceinline__ void argmax_exchange(float* v, int* id, int lane) {
     }
 }
 
+// The same exchange for a plain maximum or a plain sum of 32 columns: after the five calls (HALF = 16 .. 1) lane L
+// holds column L's result over the warp in v[0].
+template <int HALF, bool SUM>
+__device__ __forceinline__ void reduce_exchange(float* v, int lane) {
+    const bool up = (lane & HALF) != 0;
+#pragma unroll
+    for (int c = 0; c < HALF; ++c) {
+        const float send = up ? v[c] : v[c + HALF];
+        const float keep = up ? v[c + HALF] : v[c];
+        const float recv = __shfl_xor_sync(0xffffffffu, send, HALF);
+        v[c] = SUM ? keep + recv : fmaxf(keep, recv);
+    }
+}
+
 // Timeline record of CTA 0 and of the last CTA (a role thread calls this; n is that thread's event counter).
 __device__ __forceinline__ void trace_event(const LoopParams& p, int role, int& n, int step, int phase, int ev) {
     if (p.trace && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1) && step >= p.trace_step && step < p.trace_step + 2 &&
@@ -129,7 +143,9 @@ enum { J_STREAM = 0, J_SMEM = 1, J_TMEM = 2 };   // where the joint's W_out tile
 
 // RES: resident-weights mode (compile-time, so that each instantiation carries only its own code paths: the loop
 // body runs once per lock step, straight through, and instruction fetch is a visible cost at that scale).
-template <bool RES>
+// FULL: the kernel also carries teacher forcing with the logits store, window-based decoding and the timeline; the
+// plain decode runs the variant without them (a smaller instruction footprint: the loop is sensitive to it).
+template <bool RES, bool FULL>
 __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop_kernel(const __grid_constant__ LoopMaps M, const LoopParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[LOOP_MAX_STAGES], empty_bar[LOOP_MAX_STAGES], stat_bar;
@@ -251,7 +267,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         __syncthreads();
         if (threadIdx.x == 0) {
             epoch += (uint32_t)(G + p.extra_arrivals);   // extra_arrivals > 0: a test hook, the barrier can then never fill
-            trace_event(p, 3, tr_n, step, phase_kind, EV_ARRIVE);
+            if constexpr (FULL) trace_event(p, 3, tr_n, step, phase_kind, EV_ARRIVE);
             if (s_abort) {
                 atomicExch(&p.ctrl->abort, 1);
             } else {
@@ -270,7 +286,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 // the acquire load orders this thread after every arrival; the block barrier below extends that to
                 // the other threads of the CTA
             }
-            trace_event(p, 3, tr_n, step, phase_kind, EV_RELEASE);
+            if constexpr (FULL) trace_event(p, 3, tr_n, step, phase_kind, EV_RELEASE);
             if (cta == 0) {
                 const long long now = clock64();
                 cyc[phase_kind] += now - clk_last;
@@ -363,7 +379,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             if (in) {
                 if (step < 0) {
                     tok = p.blank;
-                } else if (p.forced) {
+                } else if ((FULL && p.forced)) {
                     tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
                 } else if (l > 0) {
                     tok = p.emit_tok[b];
@@ -436,7 +452,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     if (writer) p.emit_tok[b] = tok;
                 }
             }
-            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
+            if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
             const bool live = in && tok >= 0;
             // what the cell update needs from memory, requested before the accumulator is waited for
             float add[4][8], cold[8];
@@ -458,7 +474,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             load_operands(0);
             const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, &s_abort));
             tc_fence_after();
-            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
+            if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
             if (ready) {
                 for (int u0 = 0; u0 < p.ul; u0 += 8) {
                     if (u0 > 0) load_operands(u0);
@@ -492,9 +508,9 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             ++acc_n[1];
             if (!ready) return false;
         }
-        if (cta == 0 && e == 0 && l == 0 && step >= 0 && !p.forced) p.ctrl->step = step + 1;
+        if (cta == 0 && e == 0 && l == 0 && step >= 0 && !(FULL && p.forced)) p.ctrl->step = step + 1;
         fence_proxy_async_all();
-        if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_EPI_DONE);
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_EPI_DONE);
         return true;
     };
 
@@ -558,7 +574,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         const int u16 = lane & 15, half = lane >> 4;
         const int unit = r_ut * 16 + u16;        // this thread's hidden unit; its gate is q
         const bool writer = layer == 0 && r_ut == 0 && q == 0; // the two gate-0 warps of one CTA per utterance group record the step
-        const bool decode = step >= 0 && !p.forced && layer == 0;
+        const bool decode = step >= 0 && !(FULL && p.forced) && layer == 0;
         float* cst = p.c_state + (size_t)layer * p.B * p.P + unit;
         const __nv_bfloat16* hin = p.hb + ((size_t)(pin * p.L + layer) * p.Bpad) * p.P + unit;
         __nv_bfloat16* hout = p.hb + ((size_t)((pin ^ 1) * p.L + layer) * p.Bpad) * p.P + unit;
@@ -596,7 +612,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             if (in) {
                 if (step < 0) {
                     tok = p.blank;
-                } else if (p.forced) {
+                } else if ((FULL && p.forced)) {
                     tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
                 } else if (layer > 0) {
                     tok = p.emit_tok[b];     // decided by layer 0's CTAs one phase earlier
@@ -676,10 +692,10 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 }
                 // the next frame goes out at once, stamped with the step, for the projection CTAs (which fetch their
                 // enc_proj rows while this phase is still running)
-                if (writer && !p.forced) p.t_pub[b] = ((unsigned long long)(uint32_t)(step + 2) << 32) | (uint32_t)t_out;
+                if (writer && !(FULL && p.forced)) p.t_pub[b] = ((unsigned long long)(uint32_t)(step + 2) << 32) | (uint32_t)t_out;
                 if (writer && p.L > 1 && decode) p.emit_tok[b] = tok;   // the upper layer's CTAs read it in their phase
             }
-            if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
+            if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
             // ---- gate-table entries (this thread's gate and unit) of the tokens of this lane half's 16 utterances ----
             float add[16];
 #pragma unroll
@@ -700,7 +716,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             if (c0 == 0) {
                 ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, &s_abort));
                 tc_fence_after();
-                if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
             }
             if (ready) {
                 // lanes 0..15 read their row's 32 columns; columns 16..31 then move to lanes 16..31
@@ -748,7 +764,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         if (lane == 0) mbar_arrive(&acc_empty[1]);
         ++acc_n[1];
         fence_proxy_async_all();
-        if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_EPI_DONE);
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_EPI_DONE);
         return ready;
     };
     // z rows of a P CTA: row r = (utterance bl = r / W of the CTA's group, window row w = r % W), 64 columns = 128 bytes =
@@ -784,7 +800,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
     };
     auto prefetch_res_P = [&]() {
         pre_kinds = -1;
-        if (p.forced) return;
+        if ((FULL && p.forced)) return;
         const uint32_t want = (uint32_t)(step + 2);
         // the published frames of this thread's rows, all requested together, until every stamp is this step's
         unsigned long long v[8];
@@ -870,10 +886,10 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 if (((kinds >> (2 * i)) & 3) == 2) ev[i] = *reinterpret_cast<const uint4*>(stash + (size_t)(p_row0 + 32 * i) * 128 + p_chunk * 16);
             }
         }
-        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
         const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[2], acc_n[2] & 1u, &s_abort));
         tc_fence_after();
-        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
         if (ready) {
             const int hl = 16 * q + (lane & 15);
             const float bias = p_bias;
@@ -923,7 +939,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             }
         }
         fence_proxy_async_all();
-        if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
         return ready;
     };
     // the decoder GEMM of the next step, on the state hb[pin] (TMA and MMA issuers of an L CTA)
@@ -990,10 +1006,10 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         // =====================================================================================
         if constexpr (RES) {
             if (warp >= 2) {
-                if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_START);
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_START);
                 if (res_l) epilogue_res_L(0);
                 else if (res_p) prefetch_res_P();
-                if (cta == 0 && e == 0 && step >= 0 && !p.forced) p.ctrl->step = step + 1;
+                if (cta == 0 && e == 0 && step >= 0 && !(FULL && p.forced)) p.ctrl->step = step + 1;
             }
             if (!grid_sync(TR_L)) goto done;
             if (p.L == 2) {
@@ -1019,13 +1035,13 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             } else if (warp == 1) {
                 if (lane == 0 && gemm_here) { cur = 0; mma_L(l); }
             } else {
-                if (e == 0) trace_event(p, 2, tr_n, step, TR_L, EV_START);
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_START);
                 epilogue_L(l);
             }
             if (!grid_sync(TR_L)) goto done;
         }
         pin ^= 1;
-        if (p.forced && step + 1 < p.U) {
+        if ((FULL && p.forced) && step + 1 < p.U) {
             // teacher forcing: more prefix tokens to feed before the window is evaluated
             if constexpr (RES) {
                 early_res();
@@ -1059,7 +1075,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 } else if (warp == 1) {
                     if (lane == 0 && res_p) mma_part(2, tm_p, p.np, 0, p.kb_p / 2, false);
                 } else {
-                    if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_START);
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_START);
                     int cnt = 0;
                     for (int b = e; b < p.B; b += 256) cnt += t_new[b] < p.enc_len[b];
 #pragma unroll
@@ -1111,7 +1127,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     if (ok && early) mma_L(0);
                 }
             } else {
-                if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_START);
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_START);
                 // utterances still decoding, counted by every CTA (they all take the same exit)
                 {
                     int cnt = 0;
@@ -1141,10 +1157,10 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                             ev[j][1] = src[1];
                         }
                     }
-                    if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
                     const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[2], acc_n[2] & 1u, &s_abort));
                     tc_fence_after();
-                    if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
                     if (ready) {
                         for (int c0 = 0; c0 < n_tile; c0 += 16) {
                             float g[16];
@@ -1198,12 +1214,12 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     if (!ready) break;
                 }
                 fence_proxy_async_all();
-                if (e == 0) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
             }
             if (!grid_sync(TR_P)) goto done;
         }
-        if (!p.forced && s_active == 0) break;
-        if (!p.forced && step + 1 >= p.step_cap) { exit_status = WIND_ERR_INTERNAL; break; }
+        if (!(FULL && p.forced) && s_active == 0) break;
+        if (!(FULL && p.forced) && step + 1 >= p.step_cap) { exit_status = WIND_ERR_INTERNAL; break; }
         ++step;
 
         // =====================================================================================
@@ -1218,22 +1234,22 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 if (lane == 0 && has_j) {
                     if (warp == 0) {
                         fence_proxy_async_all();
-                        trace_event(p, 0, tr_n, step, TR_J, EV_FIRST_ISSUE);
+                        if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_FIRST_ISSUE);
                         const bool ok = produce_one(&M.z3, (cta / p.vt_count) * n_tile, (uint32_t)n_tile * (uint32_t)p.H * 2u);
-                        trace_event(p, 0, tr_n, step, TR_J, EV_LAST_ISSUE);
+                        if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_LAST_ISSUE);
                         if (ok) mma_part(0, tm_j + (uint32_t)n_tile, n_tile, p.kb_h / 2, p.kb_h, true);
-                        trace_event(p, 0, tr_n, step, TR_J, EV_COMMIT);
+                        if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_COMMIT);
                     } else {
                         mma_part(0, tm_j, n_tile, 0, p.kb_h / 2, true);
-                        trace_event(p, 1, tr_n, step, TR_J, EV_COMMIT);
+                        if constexpr (FULL) trace_event(p, 1, tr_n, step, TR_J, EV_COMMIT);
                     }
                 }
-            } else if (warp == 0) {
+            } else if (!RES && warp == 0) {
                 if (lane == 0) {
                     fence_proxy_async_all();
                     cur = 0;
                     bool ok = true;
-                    trace_event(p, 0, tr_n, step, TR_J, EV_FIRST_ISSUE);
+                    if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_FIRST_ISSUE);
                     for (int i = cta; i < p.j_items && ok; i += G) {
                         const int rg = i / p.vt_count, vt = i - rg * p.vt_count;
                         for (int kb = 0; kb < p.kb_h; ++kb) {
@@ -1250,9 +1266,9 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                             cur = cur + 1 == S_j ? 0 : cur + 1;
                         }
                     }
-                    trace_event(p, 0, tr_n, step, TR_J, EV_LAST_ISSUE);
+                    if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_LAST_ISSUE);
                 }
-            } else if (warp == 1) {
+            } else if (!RES && warp == 1) {
                 if (lane == 0) {
                     const uint32_t idesc = idesc_bf16(128, n_tile);
                     cur = 0;
@@ -1262,7 +1278,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                         if (!begin_acc(0)) { ok = false; break; }
                         for (int kb = 0; kb < p.kb_h; ++kb) {
                             if (!consume()) { ok = false; break; }
-                            if (kb == 0) trace_event(p, 1, tr_n, step, TR_J, EV_FIRST_DATA);
+                            if (kb == 0) if constexpr (FULL) trace_event(p, 1, tr_n, step, TR_J, EV_FIRST_DATA);
                             const uint32_t st_addr = smem_u32(ring + (size_t)cur * sb_j);
                             if (p.j_mode == J_TMEM) {
                                 const uint64_t bdesc = smem_desc_sw128(st_addr);
@@ -1281,11 +1297,11 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                             tc_commit(&empty_bar[cur]);
                             cur = cur + 1 == S_j ? 0 : cur + 1;
                         }
-                        if (ok) { tc_commit(&acc_full[0]); ++acc_n[0]; trace_event(p, 1, tr_n, step, TR_J, EV_COMMIT); }
+                        if (ok) { tc_commit(&acc_full[0]); ++acc_n[0]; if constexpr (FULL) trace_event(p, 1, tr_n, step, TR_J, EV_COMMIT); }
                     }
                 }
             } else {
-                if (e == 0) trace_event(p, 2, tr_n, step, TR_J, EV_START);
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_START);
                 const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
                 for (int i = cta; i < p.j_items; i += G) {
                     const int rg = i / p.vt_count, vt = i - rg * p.vt_count;
@@ -1294,7 +1310,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     const float bias = v_ok ? p.b_out[v] : 0.f;
                     const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[0], acc_n[0] & 1u, &s_abort));
                     tc_fence_after();
-                    if (e == 0) trace_event(p, 2, tr_n, step, TR_J, EV_ACC);
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_ACC);
                     if (ready) {
                         for (int c0 = RES ? 32 * sub : 0; c0 < n_tile; c0 += RES ? 64 : 32) {
                             float val[32];
@@ -1323,7 +1339,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
 #pragma unroll
                             for (int j = 0; j < 32; ++j) val[j] = v_ok ? val[j] + bias : -INFINITY;
                             const int row = rg * n_tile + c0 + lane;      // the window row whose result this lane ends up with
-                            if (p.logits_out) {
+                            if (FULL && p.logits_out) {
                                 // teacher-forced evaluation: store the logits of the rows inside the window
                                 bool row_ok = false;
                                 if (row < p.rows && c0 + lane < n_tile) {
@@ -1337,21 +1353,30 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                                         p.logits_out[(size_t)(rg * n_tile + c0 + j) * p.NV + v] = val[j];
                             } else {
                                 unsigned long long* key_dst = keys_cur;
-                                if (p.window) {
+                                if (FULL && p.window) {
                                     // window-based decoding: this warp's 32 vocabulary entries give, per row, a partial
                                     // (maximum, sum of exponentials) for the row's log-sum-exp; the blank's logit is
                                     // stored on its own and the blank leaves the maximum search
-                                    float m_keep = -INFINITY, s_keep = 0.f;
+                                    float tmp[32];
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) tmp[j] = val[j];
+                                    reduce_exchange<16, false>(tmp, lane);
+                                    reduce_exchange<8, false>(tmp, lane);
+                                    reduce_exchange<4, false>(tmp, lane);
+                                    reduce_exchange<2, false>(tmp, lane);
+                                    reduce_exchange<1, false>(tmp, lane);
+                                    const float m_keep = tmp[0];           // this lane's row: maximum over the warp's 32 entries
 #pragma unroll
                                     for (int j = 0; j < 32; ++j) {
-                                        float m = val[j];
-#pragma unroll
-                                        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-                                        float sm = val[j] > -INFINITY ? __expf(val[j] - m) : 0.f;
-#pragma unroll
-                                        for (int o = 16; o > 0; o >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, o);
-                                        if (lane == j) { m_keep = m; s_keep = sm; }
+                                        const float mj = __shfl_sync(0xffffffffu, m_keep, j);
+                                        tmp[j] = val[j] > -INFINITY ? __expf(val[j] - mj) : 0.f;
                                     }
+                                    reduce_exchange<16, true>(tmp, lane);
+                                    reduce_exchange<8, true>(tmp, lane);
+                                    reduce_exchange<4, true>(tmp, lane);
+                                    reduce_exchange<2, true>(tmp, lane);
+                                    reduce_exchange<1, true>(tmp, lane);
+                                    const float s_keep = tmp[0];
                                     if (row < p.rows && c0 + lane < n_tile)
                                         p.jpart[(size_t)row * p.parts + vt * 4 + q] = make_float2(m_keep, s_keep);
                                     if (v == p.blank) {
@@ -1383,12 +1408,12 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     ++acc_n[0];
                     if (!ready) break;
                 }
-                if (e == 0) trace_event(p, 2, tr_n, step, TR_J, EV_EPI_DONE);
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_EPI_DONE);
             }
             if (!grid_sync(TR_J)) goto done;
         }
-        if (p.forced) break;
-        if (p.window) {
+        if ((FULL && p.forced)) break;
+        if (FULL && p.window) {
             // =================================================================================
             // window-based decoding: one warp per utterance turns the joint phase's per-row statistics into the
             // most probable (label, offset) pair of Eq. (1) and leaves it in the keys in the form the control step
@@ -1399,30 +1424,72 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
                 unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
                 const unsigned long long blank_key = pack_key(0.f, (uint32_t)p.blank);
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_START);
                 for (int b = (warp - 2) * G + cta; b < p.B; b += n_ew * G) {
+                    // every load below is independent of the utterance's position: one round trip to L2 for all of them
                     const int t = t_cur[b], len = p.enc_len[b];
-                    const int n = t < len ? min(p.W, len - t) : 0;
-                    float lpb[2], sc[2];
+                    // lane j keeps rows j and j + 32: their blank logit and best non-blank key
+                    float lpb[2], sc[2], bl[2];
                     unsigned long long key[2];
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const int j = lane + 32 * h;
-                        lpb[h] = 0.f; sc[h] = -INFINITY; key[h] = 0ull;
-                        if (j < n) {
-                            const size_t row = (size_t)b * p.W + j;
-                            const float2* part = p.jpart + row * p.parts;
-                            float mx = -INFINITY, se = 0.f;
-                            for (int k = 0; k < p.parts; ++k) {
-                                const float2 pr = part[k];
-                                if (pr.y > 0.f) {
-                                    if (pr.x > mx) { se = se * __expf(mx - pr.x) + pr.y; mx = pr.x; }
-                                    else se += pr.y * __expf(pr.x - mx);
+                        lpb[h] = 0.f; sc[h] = -INFINITY; key[h] = 0ull; bl[h] = 0.f;
+                        if (j < p.W) {
+                            bl[h] = p.jblank[(size_t)b * p.W + j];
+                            key[h] = p.nbkeys[(size_t)b * p.W + j];
+                        }
+                    }
+                    float lse_own[2] = {0.f, 0.f};
+                    // log-sum-exp of every row from its partial (maximum, sum) pairs: eight rows at a time, the pairs of
+                    // a row spread over the lanes, then combined across the warp
+                    for (int j0 = 0; j0 < p.W; j0 += 8) {
+                        float m8[8], s8[8];
+#pragma unroll
+                        for (int r = 0; r < 8; ++r) { m8[r] = -INFINITY; s8[r] = 0.f; }
+                        for (int k = lane; k < p.parts; k += 32) {
+                            float2 pr[8];
+#pragma unroll
+                            for (int r = 0; r < 8; ++r)
+                                pr[r] = j0 + r < p.W ? p.jpart[((size_t)b * p.W + j0 + r) * p.parts + k] : make_float2(-INFINITY, 0.f);
+#pragma unroll
+                            for (int r = 0; r < 8; ++r) {
+                                if (pr[r].y > 0.f) {
+                                    if (pr[r].x > m8[r]) { s8[r] = s8[r] * __expf(m8[r] - pr[r].x) + pr[r].y; m8[r] = pr[r].x; }
+                                    else s8[r] += pr[r].y * __expf(pr[r].x - m8[r]);
                                 }
                             }
-                            const float lse = mx + __logf(se);
-                            lpb[h] = p.jblank[row] - lse;
-                            key[h] = p.nbkeys[row];
-                            if (key[h] != 0ull) sc[h] = key_logit(key[h]) - lse;
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                            for (int r = 0; r < 8; ++r) {
+                                const float om = __shfl_xor_sync(0xffffffffu, m8[r], o), os = __shfl_xor_sync(0xffffffffu, s8[r], o);
+                                const float mx = fmaxf(m8[r], om);
+                                const float a = s8[r] > 0.f ? s8[r] * __expf(m8[r] - mx) : 0.f;
+                                const float c = os > 0.f ? os * __expf(om - mx) : 0.f;
+                                m8[r] = mx; s8[r] = a + c;
+                            }
+                        }
+#pragma unroll
+                        for (int r = 0; r < 8; ++r) {
+                            const float lse = m8[r] + __logf(s8[r]);
+                            const int j = j0 + r;
+                            if ((j & 31) == lane) {
+                                if ((j >> 5) == 0) lse_own[0] = lse; else lse_own[1] = lse;
+                            }
+                        }
+                    }
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_ACC);
+                    const int n = t < len ? min(p.W, len - t) : 0;
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_TOK);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (lane + 32 * h < n) {
+                            lpb[h] = bl[h] - lse_own[h];
+                            if (key[h] != 0ull) sc[h] = key_logit(key[h]) - lse_own[h];
+                        } else {
+                            key[h] = 0ull;
                         }
                     }
                     // blank log-probabilities of the rows before each row (rows 0..31 on the lanes, then rows 32..63)
@@ -1453,6 +1520,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                         if (j < p.W) p.nbkeys[(size_t)b * p.W + j] = 0ull;
                     }
                 }
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_EPI_DONE);
             }
             if (!grid_sync(TR_J)) goto done;
         }
@@ -1704,10 +1772,11 @@ cudaError_t loop_prepare(Call& c) {
     {
         std::lock_guard<std::mutex> lock(g_loop_mutex);
         if ((int)pl.smem_bytes > g_attr_smem) {
-            e = cudaFuncSetAttribute(loop_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
-            if (e != cudaSuccess) return e;
-            e = cudaFuncSetAttribute(loop_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
-            if (e != cudaSuccess) return e;
+            for (const void* fn : {(const void*)loop_kernel<false, false>, (const void*)loop_kernel<false, true>,
+                                   (const void*)loop_kernel<true, false>, (const void*)loop_kernel<true, true>}) {
+                e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
+                if (e != cudaSuccess) return e;
+            }
             g_attr_smem = (int)pl.smem_bytes;
         }
     }
@@ -1744,7 +1813,10 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.window = c.mode == WIND_MODE_WINDOW && !logits_out;
     p.nbkeys = c.keys() + 2 * (size_t)c.lay.rows_pad; p.jpart = c.jpart(); p.jblank = c.jblank(); p.parts = 4 * pl.vt_count;
     void* args[2] = {(void*)&t_loop_maps, (void*)&p};
-    return cudaLaunchCooperativeKernel(pl.resident ? (const void*)loop_kernel<true> : (const void*)loop_kernel<false>, dim3((unsigned)pl.grid), dim3(pl.resident ? LOOP_THREADS_RES : LOOP_THREADS), args, pl.smem_bytes,
+    const bool full = p.forced || p.window || p.trace;
+    const void* fn = pl.resident ? (full ? (const void*)loop_kernel<true, true> : (const void*)loop_kernel<true, false>)
+                                 : (full ? (const void*)loop_kernel<false, true> : (const void*)loop_kernel<false, false>);
+    return cudaLaunchCooperativeKernel(fn, dim3((unsigned)pl.grid), dim3(pl.resident ? LOOP_THREADS_RES : LOOP_THREADS), args, pl.smem_bytes,
                                        c.stream);
 }
 

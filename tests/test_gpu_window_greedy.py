@@ -113,3 +113,34 @@ def test_bf16_both_kernel_sets(pkg, kernels, L, W, B):
     w, enc, lens = ragged_case(520 + L + W, B=B, T=40, D=64, E=64, P=128, L=L, H=128, V=300, act=L % 2, bias=1.5, dtype="bf16")
     rep, _ = check_window_greedy(pkg, w, enc, lens, W, 3, kernels=kernels)
     assert rep["stats"]["kernels"] == kernels
+
+
+def test_bf16_streaming_mode_of_the_loop_kernel(pkg, monkeypatch):
+    monkeypatch.setenv("WIND_RESIDENT", "0")
+    w, enc, lens = ragged_case(531, B=150, T=30, D=64, E=64, P=64, L=1, H=128, V=257, act=0, bias=1.5, dtype="bf16")
+    rep, _ = check_window_greedy(pkg, w, enc, lens, 8, 3, kernels=2)
+    assert rep["stats"]["kernels"] == 2
+
+
+def test_cfg3_full_batch_sampled_utterances(pkg):
+    # the benchmark's workload and launch configuration; the oracle replays a sample of the utterances
+    cfg = ws.CONFIGS["cfg3_large_b128"]
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="zero")
+    model = pkg.WindModel(weights)
+    tok, frm, olen, stats, st = pkg.decode(model, enc, lens, cfg.W, cfg.S, window_greedy=True)
+    assert st == 0 and stats["kernels"] == 2 and stats["frames"] == int(lens.sum()) and stats["tokens"] == int(olen.sum())
+    hist = np.array(stats["jump_hist"])
+    assert (hist * np.arange(65)).sum() + stats["forced"] == int(lens.sum())
+    om = oracle.Model(weights)
+    order = np.argsort(lens)
+    sample = [int(order[0]), int(order[len(order) // 3]), int(order[-1])]
+
+    def replay(b):
+        return oracle.replay_verify_window(om, enc[b], int(lens[b]), cfg.W, cfg.S, tok[b, : olen[b]], frm[b, : olen[b]], MARGIN)
+
+    with ThreadPoolExecutor(3) as ex:
+        reps = list(ex.map(replay, sample))
+    for b, r in zip(sample, reps):
+        assert r["rc"] == 0, f"utterance {b}: {r}"
+    print("[window-greedy cfg3]", [(b, int(lens[b]), r["decisions"], r["not_argmax"]) for b, r in zip(sample, reps)])
