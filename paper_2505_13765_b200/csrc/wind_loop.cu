@@ -153,6 +153,9 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
     __shared__ uint32_t tmem_slot;
     __shared__ int s_abort;      // this CTA has given up
     __shared__ int s_active;     // utterances still decoding (set in the projection phase)
+    // window-based decoding: per row of the window in hand, blank log-probability, best non-blank score and key
+    __shared__ float win_lpb[FULL ? kMaxWindow : 1], win_sc[FULL ? kMaxWindow : 1];
+    __shared__ unsigned long long win_key[FULL ? kMaxWindow : 1];
     __shared__ int s_red[8];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -1420,105 +1423,75 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             // reads (the chosen row carries its label, every other row the blank)
             // =================================================================================
             if (warp >= 2) {
-                const int n_ew = RES ? 8 : 4;
+                constexpr int n_ew = RES ? 8 : 4;
+                const int ew = warp - 2;
                 const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
                 unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
                 const unsigned long long blank_key = pack_key(0.f, (uint32_t)p.blank);
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_START);
-                for (int b = (warp - 2) * G + cta; b < p.B; b += n_ew * G) {
-                    // every load below is independent of the utterance's position: one round trip to L2 for all of them
-                    const int t = t_cur[b], len = p.enc_len[b];
-                    // lane j keeps rows j and j + 32: their blank logit and best non-blank key
-                    float lpb[2], sc[2], bl[2];
-                    unsigned long long key[2];
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int j = lane + 32 * h;
-                        lpb[h] = 0.f; sc[h] = -INFINITY; key[h] = 0ull; bl[h] = 0.f;
-                        if (j < p.W) {
-                            bl[h] = p.jblank[(size_t)b * p.W + j];
-                            key[h] = p.nbkeys[(size_t)b * p.W + j];
-                        }
-                    }
-                    float lse_own[2] = {0.f, 0.f};
-                    // log-sum-exp of every row from its partial (maximum, sum) pairs: eight rows at a time, the pairs of
-                    // a row spread over the lanes, then combined across the warp
-                    for (int j0 = 0; j0 < p.W; j0 += 8) {
-                        float m8[8], s8[8];
-#pragma unroll
-                        for (int r = 0; r < 8; ++r) { m8[r] = -INFINITY; s8[r] = 0.f; }
+                // one utterance per CTA at a time; each epilogue warp takes the rows ew, ew + n_ew, ... of its window
+                for (int b = cta; b < p.B; b += G) {
+                    int t = 0, len = 0;
+                    if (ew == 0) { t = t_cur[b]; len = p.enc_len[b]; }
+                    for (int j = ew; j < p.W; j += n_ew) {
+                        const size_t row = (size_t)b * p.W + j;
+                        float bl = 0.f;
+                        unsigned long long key = 0ull;
+                        if (lane == 0) { bl = p.jblank[row]; key = p.nbkeys[row]; }
+                        // the row's log-sum-exp from its partial (maximum, sum) pairs, spread over the lanes
+                        float m = -INFINITY, sm = 0.f;
                         for (int k = lane; k < p.parts; k += 32) {
-                            float2 pr[8];
-#pragma unroll
-                            for (int r = 0; r < 8; ++r)
-                                pr[r] = j0 + r < p.W ? p.jpart[((size_t)b * p.W + j0 + r) * p.parts + k] : make_float2(-INFINITY, 0.f);
-#pragma unroll
-                            for (int r = 0; r < 8; ++r) {
-                                if (pr[r].y > 0.f) {
-                                    if (pr[r].x > m8[r]) { s8[r] = s8[r] * __expf(m8[r] - pr[r].x) + pr[r].y; m8[r] = pr[r].x; }
-                                    else s8[r] += pr[r].y * __expf(pr[r].x - m8[r]);
-                                }
+                            const float2 pr = p.jpart[row * p.parts + k];
+                            if (pr.y > 0.f) {
+                                if (pr.x > m) { sm = sm * __expf(m - pr.x) + pr.y; m = pr.x; }
+                                else sm += pr.y * __expf(pr.x - m);
                             }
                         }
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-                            for (int r = 0; r < 8; ++r) {
-                                const float om = __shfl_xor_sync(0xffffffffu, m8[r], o), os = __shfl_xor_sync(0xffffffffu, s8[r], o);
-                                const float mx = fmaxf(m8[r], om);
-                                const float a = s8[r] > 0.f ? s8[r] * __expf(m8[r] - mx) : 0.f;
-                                const float c = os > 0.f ? os * __expf(om - mx) : 0.f;
-                                m8[r] = mx; s8[r] = a + c;
-                            }
+                            const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, sm, o);
+                            const float mx = fmaxf(m, om);
+                            const float a = sm > 0.f ? sm * __expf(m - mx) : 0.f;
+                            const float c = os > 0.f ? os * __expf(om - mx) : 0.f;
+                            m = mx; sm = a + c;
                         }
-#pragma unroll
-                        for (int r = 0; r < 8; ++r) {
-                            const float lse = m8[r] + __logf(s8[r]);
-                            const int j = j0 + r;
-                            if ((j & 31) == lane) {
-                                if ((j >> 5) == 0) lse_own[0] = lse; else lse_own[1] = lse;
-                            }
+                        if (lane == 0) {
+                            const float lse = m + __logf(sm);
+                            win_lpb[j] = bl - lse;
+                            win_sc[j] = key != 0ull ? key_logit(key) - lse : -INFINITY;
+                            win_key[j] = key;
+                            p.nbkeys[row] = 0ull;
                         }
                     }
-                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_ACC);
-                    const int n = t < len ? min(p.W, len - t) : 0;
-                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_TOK);
+                    asm volatile("bar.sync 1, %0;" ::"n"(n_ew * 32) : "memory");
+                    if (ew == 0) {
+                        const int n = t < len ? min(p.W, len - t) : 0;
+                        // lane j looks at rows j and j + 32: blank log-probabilities of the rows before each row
+                        float lpb0 = lane < n ? win_lpb[lane] : 0.f, lpb1 = lane + 32 < n ? win_lpb[lane + 32] : 0.f;
+                        float sc0 = lane < n ? win_sc[lane] : -INFINITY, sc1 = lane + 32 < n ? win_sc[lane + 32] : -INFINITY;
+                        float incl0 = lpb0, incl1 = lpb1;
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        if (lane + 32 * h < n) {
-                            lpb[h] = bl[h] - lse_own[h];
-                            if (key[h] != 0ull) sc[h] = key_logit(key[h]) - lse_own[h];
-                        } else {
-                            key[h] = 0ull;
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const float a0 = __shfl_up_sync(0xffffffffu, incl0, o), a1 = __shfl_up_sync(0xffffffffu, incl1, o);
+                            if (lane >= o) { incl0 += a0; incl1 += a1; }
                         }
-                    }
-                    // blank log-probabilities of the rows before each row (rows 0..31 on the lanes, then rows 32..63)
-                    float incl0 = lpb[0], incl1 = lpb[1];
+                        const float tot0 = __shfl_sync(0xffffffffu, incl0, 31), tot1 = __shfl_sync(0xffffffffu, incl1, 31);
+                        sc0 += incl0 - lpb0;
+                        sc1 += tot0 + incl1 - lpb1;
+                        // first strict maximum in row order; "all blank" (tot0 + tot1) wins only when strictly larger
+                        float top = sc0;
+                        int pick = lane;
+                        if (sc1 > top) { top = sc1; pick = lane + 32; }
 #pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const float a0 = __shfl_up_sync(0xffffffffu, incl0, o), a1 = __shfl_up_sync(0xffffffffu, incl1, o);
-                        if (lane >= o) { incl0 += a0; incl1 += a1; }
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const float ot = __shfl_xor_sync(0xffffffffu, top, o);
+                            const int op = __shfl_xor_sync(0xffffffffu, pick, o);
+                            if (ot > top || (ot == top && op < pick)) { top = ot; pick = op; }
+                        }
+                        if (!(top > -INFINITY) || tot0 + tot1 > top) pick = -1;
+                        for (int j = lane; j < n; j += 32) keys_cur[(size_t)b * p.W + j] = j == pick ? win_key[j] : blank_key;
                     }
-                    const float tot0 = __shfl_sync(0xffffffffu, incl0, 31), tot1 = __shfl_sync(0xffffffffu, incl1, 31);
-                    sc[0] += incl0 - lpb[0];
-                    sc[1] += tot0 + incl1 - lpb[1];
-                    // first strict maximum in row order; "all blank" (tot0 + tot1) wins only when strictly larger
-                    float top = sc[0];
-                    int pick = lane;
-                    if (sc[1] > top) { top = sc[1]; pick = lane + 32; }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        const float ot = __shfl_xor_sync(0xffffffffu, top, o);
-                        const int op = __shfl_xor_sync(0xffffffffu, pick, o);
-                        if (ot > top || (ot == top && op < pick)) { top = ot; pick = op; }
-                    }
-                    if (!(top > -INFINITY) || tot0 + tot1 > top) pick = -1;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int j = lane + 32 * h;
-                        if (j < n) keys_cur[(size_t)b * p.W + j] = j == pick ? key[h] : blank_key;
-                        if (j < p.W) p.nbkeys[(size_t)b * p.W + j] = 0ull;
-                    }
+                    if (b + G < p.B) asm volatile("bar.sync 1, %0;" ::"n"(n_ew * 32) : "memory");   // the arrays are reused
                 }
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_EPI_DONE);
             }
