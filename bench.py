@@ -361,7 +361,7 @@ def roofline(pkg, model, cfg, W, enc_d, len_d, tok_d, frm_d, ol_d, wsb, stream, 
         js = res["joint_ms"] * 1e-3
         dense = 2.0 * cfg.H * (cfg.V + 1) * cfg.B * W * stats["steps"]
         # DRAM bytes per launch: ncu counters (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of this
-        # kernel on the same shapes with 18975 frames (profiles/loop_kernel_cfg3_b128_short.md): 37.1 MB, of which
+        # kernel on the same shapes with 18975 frames (profiles/loop_kernel_cfg3_b128_short.md): 37.0 MB, of which
         # the enc_proj rows (2 H bytes per frame, each read once) grow with the workload and 12.8 MB (weights, gate
         # table, outputs) do not.  Scaled by the frame count; other shapes have no capture.
         traffic, traffic_source = None, None
