@@ -184,9 +184,10 @@ def main():
     ap.add_argument("--len-hi", type=int, default=0, help="override the longest utterance length, frames")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the W=1 comparison, e2e and per-kernel timing legs")
-    ap.add_argument("--op", default="decode", choices=["decode", "first_output", "window_greedy"],
+    ap.add_argument("--op", default="decode", choices=["decode", "first_output", "window_greedy", "dataset"],
                     help="first_output: time wind_window_first_output (Eq. 1 on one window per utterance) instead of the decode; "
-                         "window_greedy: time wind_decode_window_greedy on the whole workload")
+                         "window_greedy: time wind_decode_window_greedy on the whole workload; dataset: 4 x B utterances in "
+                         "arrival-order batches against length-aware batches")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -203,6 +204,8 @@ def main():
         return first_output_op(args, cfg, W)
     if args.op == "window_greedy":
         return window_greedy_op(args, cfg, W)
+    if args.op == "dataset":
+        return dataset_op(args, cfg, W)
 
     import torch
     import paper_2505_13765_b200 as pkg
@@ -509,6 +512,76 @@ def window_greedy_op(args, cfg, W):
         "note": "random-weight models give flat label distributions, for which the best pair of Eq. (1) is almost always a "
                 "label on the window's first row: the variant then emits max_symbols tokens per frame, its worst case for "
                 "the number of steps; the per-step cost is what this line measures",
+    }))
+
+
+def dataset_op(args, cfg, W):
+    """Secondary measurement (one JSON line of its own): a set of 4 x B utterances decoded batch by batch.
+
+    The same utterances are packed into batches of B twice: in arrival order and by the library's length-aware plan
+    (wind_plan_batches).  Both packings are resident on the device before the clock starts; the timed region is the
+    decodes of all batches, back to back.  `value` is the planned packing's whole-set RTFx.
+    """
+    import torch
+    import wind_synth as ws
+    import paper_2505_13765_b200 as pkg
+    from dataclasses import replace
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    pkg.load_library()
+    pkg.wind_set_kernels(args.kernels)
+    B = cfg.B
+    big = replace(cfg, B=4 * B)
+    weights = ws.make_model(cfg)
+    enc_np, lens_np = ws.make_enc(big, pad="zero")
+    model = pkg.WindModel(weights, device=dev)
+    N = enc_np.shape[0]
+    stream = torch.cuda.current_stream()
+    order, batch_T = pkg.wind_plan_batches(lens_np, B)
+
+    def pack(idx_order):
+        batches = []
+        for k in range(0, N, B):
+            idx = idx_order[k: k + B]
+            T = int(lens_np[idx].max())
+            enc_d = pkg.to_device_enc(model, np.ascontiguousarray(enc_np[idx, :T]))
+            len_d = torch.from_numpy(np.ascontiguousarray(lens_np[idx])).to(dev)
+            max_out = T * cfg.S
+            tok = torch.full((len(idx), max_out), -1, dtype=torch.int32, device=dev)
+            batches.append((enc_d, len_d, tok, tok.clone(), torch.zeros(len(idx), dtype=torch.int32, device=dev),
+                            pkg.alloc_workspace(model, len(idx), T, W)))
+        return batches
+
+    def run(batches, k):
+        def once():
+            steps = 0
+            for enc_d, len_d, tok, frm, ol, wsb in batches:
+                pkg.wind_decode_greedy(model, enc_d, len_d, W, cfg.S, tok, frm, ol, wsb, stream=stream)
+                steps += pkg.wind_read_stats(wsb, stream)["steps"]
+            return steps
+        for _ in range(max(3, args.warmup)):
+            steps = once()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(k):
+            once()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / k, steps
+
+    ms_a, steps_a = run(pack(np.arange(N)), args.steps)
+    torch.cuda.empty_cache()
+    ms_p, steps_p = run(pack(order), args.steps)
+    audio_s = float(lens_np.sum()) * FRAME_SECONDS
+    print(json.dumps({
+        "metric": "greedy WIND RTFx of a set of utterances (audio-s/s at 80 ms/frame)", "op": "dataset",
+        "value": audio_s / (ms_p * 1e-3), "unit": "audio-s/s", "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": ms_p, "higher_is_better": True, "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "utterances": N, "B": B, "frames": int(lens_np.sum()), "W": W},
+        "length_aware": {"ms": ms_p, "lock_steps": steps_p, "batch_T": [int(t) for t in batch_T]},
+        "arrival_order": {"ms": ms_a, "lock_steps": steps_a, "value": audio_s / (ms_a * 1e-3)},
+        "speedup_vs_arrival_order": ms_a / ms_p, "gpu_launches": 4 * len(batch_T) * args.steps,
     }))
 
 

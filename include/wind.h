@@ -254,6 +254,21 @@ wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const 
                                   int32_t* out_frames, int32_t* out_len, int32_t max_out, void* workspace,
                                   size_t workspace_bytes, void* stream, wind_profile_t* host_out);
 
+/*
+ * Length-aware batching of a set of N utterances (host-only; no CUDA call).  The lock-step loop of a batch runs until
+ * its longest utterance is done, so batches of mixed lengths leave most rows idle for most steps: the paper's batched
+ * gain shrinks as the batch grows for the same reason.  The plan sorts the utterances by length, longest first (equal
+ * lengths keep their order), and cuts the sorted list into batches of B (the last one may be smaller), which
+ * minimises the sum over batches of the longest length.  With several GPUs, rank r of R takes batches r, r + R, ...
+ * (longest first, so that the ranks' loads differ by at most one batch of the shortest utterances).
+ *   enc_len  HOST [N] int32, each >= 0.     order    HOST [N] out: utterance indices, batch after batch.
+ *   batch_T  HOST [ceil(N / B)] out, may be null: longest length of each batch (the T to pack it with).
+ *   n_batches HOST out.
+ * WIND_ERR_INVALID_ARG: null pointer, N < 0, B < 1, a negative length.
+ */
+wind_status_t wind_plan_batches(const int32_t* enc_len, int32_t N, int32_t B, int32_t* order, int32_t* batch_T,
+                                int32_t* n_batches);
+
 /* Copies the counters of the last decode that used `workspace` to host memory (synchronises `stream`). */
 wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t* host_out);
 

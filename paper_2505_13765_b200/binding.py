@@ -30,7 +30,7 @@ WIND_KERNELS_AUTO, WIND_KERNELS_SIMT, WIND_KERNELS_TENSOR = 0, 1, 2
 
 EXPORTS = [
     "wind_workspace_bytes", "wind_decode_greedy", "wind_decode_window_greedy", "wind_host_staging_bytes", "wind_decode_greedy_host",
-    "wind_eval_joint_window", "wind_window_first_output", "wind_eval_joint_window_static", "wind_profile_decode", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_debug_stall_barrier", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
+    "wind_eval_joint_window", "wind_window_first_output", "wind_eval_joint_window_static", "wind_profile_decode", "wind_plan_batches", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_debug_stall_barrier", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
 ]
 
 _vp = C.c_void_p
@@ -106,6 +106,8 @@ def load_library():
     L.wind_window_first_output.restype = i32
     L.wind_eval_joint_window_static.argtypes = [mp, _vp, _vp, i32, i32, i32, _vp, i32, _vp, _vp, _vp, _vp]
     L.wind_eval_joint_window_static.restype = i32
+    L.wind_plan_batches.argtypes = [_vp, i32, i32, _vp, _vp, C.POINTER(i32)]
+    L.wind_plan_batches.restype = i32
     L.wind_read_stats.argtypes = [_vp, _vp, C.POINTER(wind_stats_t)]
     L.wind_read_stats.restype = i32
     L.wind_set_trace.argtypes = [i32]
@@ -389,6 +391,48 @@ def to_device_enc(model: WindModel, enc_np: np.ndarray):
     torch = _torch()
     t = torch.from_numpy(np.ascontiguousarray(enc_np, dtype=np.float32))
     return t.to(model.torch_dtype).to(model.device).contiguous()
+
+
+def wind_plan_batches(lens_np: np.ndarray, B: int):
+    """Length-aware batching plan: (order [N], batch_T [n_batches]); batch k = order[k*B : (k+1)*B]."""
+    L = load_library()
+    lens = np.ascontiguousarray(lens_np, dtype=np.int32)
+    N = int(lens.shape[0])
+    order = np.zeros(max(N, 1), np.int32)
+    batch_T = np.zeros(max((N + B - 1) // max(B, 1), 1), np.int32)
+    nb = C.c_int32(0)
+    st = L.wind_plan_batches(lens.ctypes.data, N, B, order.ctypes.data, batch_T.ctypes.data, C.byref(nb))
+    if st != WIND_OK:
+        raise WindError(st)
+    return order[:N], batch_T[: nb.value]
+
+
+def decode_dataset(model: WindModel, utterances, W: int, S: int, B: int, plan: bool = True, window_greedy: bool = False):
+    """Decodes a list of [T_i, D] numpy arrays in batches of B; results come back in the list's order.
+
+    plan=True groups utterances of similar length (wind_plan_batches); plan=False keeps the arrival order.  Packing the
+    batches is marshalling; every batch is one call of the decode entry point.  Returns (list of token arrays, list of
+    frame arrays, total lock steps).
+    """
+    lens = np.array([u.shape[0] for u in utterances], np.int32)
+    N = len(utterances)
+    if plan:
+        order, _ = wind_plan_batches(lens, B)
+    else:
+        order = np.arange(N, dtype=np.int32)
+    toks, frms, steps = [None] * N, [None] * N, 0
+    D = model.dims["D"]
+    for k in range(0, N, B):
+        idx = order[k: k + B]
+        T = max(1, int(lens[idx].max()))
+        enc = np.zeros((len(idx), T, D), np.float32)
+        for r, i in enumerate(idx):
+            enc[r, : lens[i]] = utterances[i]
+        tok, frm, olen, stats, _ = decode(model, enc, lens[idx], W, S, window_greedy=window_greedy)
+        steps += stats["steps"]
+        for r, i in enumerate(idx):
+            toks[i], frms[i] = tok[r, : olen[r]].copy(), frm[r, : olen[r]].copy()
+    return toks, frms, steps
 
 
 def decode(model: WindModel, enc_np: np.ndarray, lens_np: np.ndarray, W: int, S: int, max_out: Optional[int] = None,

@@ -1,5 +1,6 @@
 // C ABI entry points: argument checks, workspace carving, launch sequence, and the
 // device-resident decoding loop (a CUDA-graph WHILE node whose body is two lock steps).
+#include <algorithm>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -510,6 +511,20 @@ wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const 
     }
     destroy();
     return read_status(c);
+}
+
+wind_status_t wind_plan_batches(const int32_t* enc_len, int32_t N, int32_t B, int32_t* order, int32_t* batch_T,
+                                int32_t* n_batches) {
+    if (!enc_len || !order || !n_batches || N < 0 || B < 1) return WIND_ERR_INVALID_ARG;
+    for (int32_t i = 0; i < N; ++i)
+        if (enc_len[i] < 0) return WIND_ERR_INVALID_ARG;
+    for (int32_t i = 0; i < N; ++i) order[i] = i;
+    std::stable_sort(order, order + N, [&](int32_t a, int32_t b) { return enc_len[a] > enc_len[b]; });
+    const int32_t nb = (N + B - 1) / B;
+    if (batch_T)
+        for (int32_t k = 0; k < nb; ++k) batch_T[k] = enc_len[order[(size_t)k * B]];   // sorted: the batch's first is its longest
+    *n_batches = nb;
+    return WIND_OK;
 }
 
 wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t* host_out) {

@@ -289,6 +289,22 @@ def test_bf16_tensor_path_output_overflow(pkg):
         assert olen[b] == n and np.array_equal(tok[b, :n], full[0][b, :n]) and np.array_equal(frm[b, :n], full[1][b, :n])
 
 
+def test_length_aware_batches_give_the_same_transcripts_in_fewer_lock_steps(pkg):
+    # an utterance's result does not depend on what shares its batch: planned and arrival-order batches agree bit for bit
+    w, enc, lens = ragged_case(95, B=45, T=60, D=64, E=64, P=128, L=1, H=128, V=200, act=1, bias=1.5, dtype="bf16")
+    utts = [np.ascontiguousarray(enc[b, : lens[b]]) for b in range(45)]
+    model = pkg.WindModel(w)
+    t_a, f_a, steps_a = pkg.decode_dataset(model, utts, 4, 3, B=8, plan=False)
+    t_p, f_p, steps_p = pkg.decode_dataset(model, utts, 4, 3, B=8, plan=True)
+    for b in range(45):
+        assert np.array_equal(t_a[b], t_p[b]) and np.array_equal(f_a[b], f_p[b])
+    assert steps_p < steps_a
+    # and both equal one batch of everything
+    tok, frm, olen, _, _ = pkg.decode(model, np.nan_to_num(enc), lens, 4, 3)
+    for b in range(45):
+        assert np.array_equal(tok[b, : olen[b]], t_p[b]) and np.array_equal(frm[b, : olen[b]], f_p[b])
+
+
 def test_cfg2_large_b1(pkg):
     cfg = ws.CONFIGS["cfg2_large_b1"]
     weights = ws.make_model(cfg)

@@ -90,6 +90,46 @@ def test_invalid_arguments_are_rejected_on_the_host(lib):
     assert lib.wind_read_trace(ref, 1, 10, 4, None, None, None, 0, C.byref(n_ev)) == bd.WIND_ERR_INVALID_ARG
 
 
+def test_plan_batches_sorts_by_length_and_minimises_the_sum_of_batch_maxima(lib):
+    import itertools
+    import numpy as np
+    r = np.random.default_rng(5)
+    for N, B in ((0, 4), (1, 4), (7, 3), (128, 128), (300, 64), (12, 1)):
+        lens = r.integers(0, 50, size=N).astype(np.int32)
+        order, batch_T = pkg.wind_plan_batches(lens, B)
+        assert sorted(order.tolist()) == list(range(N))                      # a permutation
+        assert len(batch_T) == (N + B - 1) // B
+        sl = lens[order]
+        assert np.all(np.diff(sl) <= 0)                                      # longest first
+        for a, b in zip(order[:-1], order[1:]):                              # equal lengths keep their order
+            if lens[a] == lens[b]:
+                assert a < b
+        for k, T in enumerate(batch_T):
+            assert T == lens[order[k * B: (k + 1) * B]].max()
+        arrival = sum(int(lens[k: k + B].max()) for k in range(0, N, B))
+        assert int(batch_T.sum()) <= arrival
+    # ranks take batches r, r + R, ...: together every utterance exactly once, loads within one (shortest) batch
+    lens = r.integers(1, 2500, size=1000).astype(np.int32)
+    order, batch_T = pkg.wind_plan_batches(lens, 64)
+    shares = [[k for k in range(len(batch_T)) if k % 4 == rank] for rank in range(4)]
+    seen = sorted(int(i) for sh in shares for k in sh for i in order[k * 64: (k + 1) * 64])
+    assert seen == list(range(1000))
+    loads = [int(batch_T[sh].sum()) for sh in shares]
+    assert max(loads) - min(loads) <= int(batch_T[0])
+    # brute force on a tiny set: no grouping into batches of 2 has a smaller sum of batch maxima
+    lens = np.array([9, 2, 7, 7, 1, 4], np.int32)
+    order, batch_T = pkg.wind_plan_batches(lens, 2)
+    best = min(sum(max(lens[list(perm[k: k + 2])]) for k in range(0, 6, 2)) for perm in itertools.permutations(range(6)))
+    assert int(batch_T.sum()) == best
+    n = C.c_int32(0)
+    buf = (C.c_int32 * 4)()
+    assert lib.wind_plan_batches(None, 4, 2, buf, None, C.byref(n)) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_plan_batches(buf, 4, 0, buf, None, C.byref(n)) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_plan_batches(buf, -1, 2, buf, None, C.byref(n)) == bd.WIND_ERR_INVALID_ARG
+    neg = (C.c_int32 * 2)(3, -1)
+    assert lib.wind_plan_batches(neg, 2, 2, buf, None, C.byref(n)) == bd.WIND_ERR_INVALID_ARG
+
+
 def test_debug_hooks_round_trip(lib):
     assert pkg.wind_set_trace(5) == -2 and pkg.wind_set_trace(-9) == 5 and pkg.wind_set_trace(-2) == -2
     assert pkg.wind_debug_stall_barrier(2) == 0 and pkg.wind_debug_stall_barrier(0) == 2
