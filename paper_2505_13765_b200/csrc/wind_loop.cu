@@ -211,6 +211,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
     const bool res_x1 = RES && p.L == 2 && r_role == 1;
     const bool res_h1 = RES && p.L == 2 && r_role == 2;
     const bool res_p = RES && !res_l && !res_x1 && !res_h1 && G - 1 - cta < p.p_items;
+    const bool res_w = RES && cta >= p.w_first && cta < p.w_first + p.w_count;   // step-recording CTAs (none of the above)
     const int r_ut = r_idx % p.ut_count, r_ql = r_idx / p.ut_count;                  // unit tile / utterance group of an L CTA
     const int r_ht = (G - 1 - cta) % p.ht_count, r_qp = (G - 1 - cta) / p.ht_count;  // H tile / utterance group of a P CTA
     constexpr uint32_t RES_A_BYTES = 64 * BK * 2;
@@ -569,14 +570,20 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
     // of a pass are requested together: first everything the control step needs, then the gate-table rows of the
     // chosen tokens.  Lanes 16..31 hold no accumulator row (64-row tile); they take the second 16 utterances.
     struct ScanIn { int t, len, cnt, pos; unsigned long long kk[8]; };
-    auto epilogue_res_L = [&](const int layer) -> bool {
+    // ctl_only: the CTA is one of the step-recording CTAs (see the plan): it takes the control step of 64 utterances,
+    // records it (outputs, counters, next frame) and has no cell update; the L CTAs then record nothing.
+    auto epilogue_res_L = [&](const int layer, const bool ctl_only) -> bool {
+        if (ctl_only && q != 0) return true;
         const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
         int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
         const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
         unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
         const int u16 = lane & 15, half = lane >> 4;
         const int unit = r_ut * 16 + u16;        // this thread's hidden unit; its gate is q
-        const bool writer = layer == 0 && r_ut == 0 && q == 0; // the two gate-0 warps of one CTA per utterance group record the step
+        // without recording CTAs, the two gate-0 warps of one CTA per utterance group record the step
+        const bool writer = ctl_only ? true : (p.w_count == 0 && layer == 0 && r_ut == 0 && q == 0);
+        const int n_here = ctl_only ? 64 : p.nl;
+        const int base = ctl_only ? (cta - p.w_first) * 64 : r_ql * p.nl;
         const bool decode = step >= 0 && !(FULL && p.forced) && layer == 0;
         float* cst = p.c_state + (size_t)layer * p.B * p.P + unit;
         const __nv_bfloat16* hin = p.hb + ((size_t)(pin * p.L + layer) * p.Bpad) * p.P + unit;
@@ -585,12 +592,12 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         const float* g0u = p.g0 + (size_t)q * p.P + unit;
         const uint32_t g0_stride = 4u * (uint32_t)p.P;
         bool ready = true;
-        for (int c0 = 0; c0 < p.nl; c0 += 64) {
-            const int b0 = r_ql * p.nl + c0;
+        for (int c0 = 0; c0 < n_here; c0 += 64) {
+            const int b0 = base + c0;
             // ---- lane j decides for utterance b0 + 32 sub + j ----
             const int jl = 32 * sub + lane;
             const int b = b0 + jl;
-            const bool in = c0 + jl < p.nl && b < p.B;
+            const bool in = c0 + jl < n_here && b < p.B;
             ScanIn si;
             si.t = 0; si.len = 0; si.cnt = 0; si.pos = 0;
 #pragma unroll
@@ -608,7 +615,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
 #pragma unroll
             for (int jj = 0; jj < 4; ++jj) {
                 const int j = half + 2 * q + 8 * sub + 16 * jj;     // 0..63 over the CTA's 256 epilogue threads
-                cold[jj] = (c0 + j < p.nl && b0 + j < p.B) ? cst[(size_t)(b0 + j) * p.P] : 0.f;
+                cold[jj] = (!ctl_only && c0 + j < p.nl && b0 + j < p.B) ? cst[(size_t)(b0 + j) * p.P] : 0.f;
             }
             // the token utterance b feeds to its decoder in this step (-1: none)
             int tok = -1, t_out = 0;
@@ -699,6 +706,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 if (writer && p.L > 1 && decode) p.emit_tok[b] = tok;   // the upper layer's CTAs read it in their phase
             }
             if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
+            if (ctl_only) continue;
             // ---- gate-table entries (this thread's gate and unit) of the tokens of this lane half's 16 utterances ----
             float add[16];
 #pragma unroll
@@ -762,6 +770,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");
         }
+        if (ctl_only) return true;
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&acc_empty[1]);
@@ -1010,7 +1019,8 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         if constexpr (RES) {
             if (warp >= 2) {
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_START);
-                if (res_l) epilogue_res_L(0);
+                if (res_l) epilogue_res_L(0, false);
+                else if (res_w) epilogue_res_L(0, true);
                 else if (res_p) prefetch_res_P();
                 if (cta == 0 && e == 0 && step >= 0 && !(FULL && p.forced)) p.ctrl->step = step + 1;
             }
@@ -1026,7 +1036,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 } else if (warp == 1) {
                     if (lane == 0 && res_x1) mma_part(1, tm_l, p.nl, 0, p.kb_p, false);
                 } else if (res_x1) {
-                    epilogue_res_L(1);
+                    epilogue_res_L(1, false);
                 }
                 if (!grid_sync(TR_L)) goto done;
             }
@@ -1699,6 +1709,11 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
             r.tm_l = r.tm_p = r.tm_j + 2 * r.nj;   // two copies of the joint accumulator, then decoder / projection
             r.l_items = r.ut_count * r.ql_count;
             r.p_items = r.ht_count * r.qp_count;
+            // CTAs that hold no decoder or projection tile record the steps (outputs, counters, next frame), 64
+            // utterances each, so that no L CTA carries that work between its control step and its cell update
+            r.w_first = l_sets * r.l_items;
+            r.w_count = (c.B + 63) / 64;
+            if (r.w_first + r.w_count + r.p_items > G) r.w_count = 0;
             r.l_early = 1;
             const int acc_cols = r.nl > 2 * r.np ? r.nl : 2 * r.np;
             if ((long long)r.smem_bytes <= (long long)budget + 1024 && r.tm_l + acc_cols <= (int)LOOP_TMEM_COLS) pl = r;
@@ -1769,6 +1784,7 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.nj = pl.nj; p.vt_count = pl.vt_count; p.rg_count = pl.rg_count; p.j_items = pl.j_items; p.j_mode = pl.j_mode;
     p.tm_j = pl.tm_j; p.tm_l = pl.tm_l; p.tm_p = pl.tm_p; p.l_early = pl.l_early;
     p.resident = pl.resident; p.nl = pl.nl; p.ut_count = pl.ut_count > 0 ? pl.ut_count : 1; p.ht_count = pl.ht_count > 0 ? pl.ht_count : 1;
+    p.w_first = pl.w_first; p.w_count = pl.resident ? pl.w_count : 0;
     p.ql_count = pl.ql_count; p.qp_count = pl.qp_count; p.buf_off = pl.buf_off; p.stage_off = pl.stage_off;
     p.stage_lp = pl.stage_lp; p.stage_j = pl.stage_j; p.stages_lp = pl.stages_lp; p.stages_j = pl.stages_j;
     p.slots = pl.slots; p.ul = pl.ul; p.ug_count = pl.ug_count; p.mt_count = pl.mt_count; p.l_items = pl.l_items;

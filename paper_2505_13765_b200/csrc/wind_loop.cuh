@@ -40,6 +40,7 @@ struct LoopPlan {
     // resident-weights mode: W_hh tiles (4 gates x 16 units) and W_pred tiles (64 rows) stay in the shared memory of
     // disjoint CTA sets; accumulators are [64 weight rows, nl or np utterances]
     int resident, nl, ut_count, ht_count, ql_count, qp_count;
+    int w_first, w_count;                  // step-recording CTAs [w_first, w_first + w_count), 64 utterances each (0: the L CTAs record)
     uint32_t buf_off, stage_off;           // the per-step operand buffer and the epilogue staging area (after the tile)
     int slots, ul, ug_count, mt_count, l_items;  // decoder: rows per gate block, units per item, unit groups, utterance tiles
     int np, hg_count, p_items;             // projection: H columns per item, H slices
@@ -54,6 +55,7 @@ struct LoopParams {
     int nj, vt_count, rg_count, j_items, j_mode;
     int tm_j, tm_l, tm_p, l_early;
     int resident, nl, ut_count, ht_count, ql_count, qp_count;
+    int w_first, w_count;
     uint32_t buf_off, stage_off;
     int slots, ul, ug_count, mt_count, l_items;
     int np, hg_count, p_items;
