@@ -278,12 +278,15 @@ wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t*
  * sequence), when the role threads of CTA 0 pass fixed points of each phase; s < -1 switches it off
  * (default).  Returns the previous setting.  Recording costs a few stores and does not change results.
  * wind_read_trace copies the records of the last decode that used `workspace` (same m, B, T, W).
- *   role:  0 TMA issuer, 1 MMA issuer, 2 first epilogue thread, 3 grid barrier
+ *   role:  0 TMA issuer, 1 MMA issuer, 2 first epilogue thread, 3 grid barrier (4..7: the same of the last CTA);
+ *          8, 9, 10: barrier arrival of EVERY CTA at the end of the joint, decoder-update and projection phase
+ *          of lock step s; for these records `step` holds the CTA index and `clock` the global timer in
+ *          nanoseconds, which is comparable across SMs: who arrives last is what bounds the phase
  *   phase: 0 joint, 1 decoder update, 2 projection
  *   event: 0 phase entered, 1 first / 2 last TMA issued, 3 first operands arrived, 4 accumulator
  *          committed, 5 epilogue inputs requested (token known), 6 accumulator ready, 7 epilogue
  *          done, 8 barrier arrival, 9 barrier release
- *   clock: SM cycle counter of CTA 0's SM
+ *   clock: SM cycle counter of the recording CTA's SM (roles 0..7)
  */
 typedef struct {
     int32_t role, phase, event, step;

@@ -22,7 +22,8 @@ struct TraceEvent {
     int32_t step;
     long long clock;   // clock64 of the SM that runs CTA 0
 };
-constexpr int kTraceRoles = 8;     // TMA issuer, MMA issuer, first epilogue thread, barrier: of CTA 0, then of the last CTA
+constexpr int kTraceRoles = 11;    // TMA issuer, MMA issuer, first epilogue thread, barrier: of CTA 0, then of the last CTA;
+                                   // 8..10: barrier arrival of every CTA in the joint / decoder / projection phase
 constexpr int kTraceEvents = 512;
 
 // Device control block, first thing in the workspace.

@@ -272,6 +272,16 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         if (threadIdx.x == 0) {
             epoch += (uint32_t)(G + p.extra_arrivals);   // extra_arrivals > 0: a test hook, the barrier can then never fill
             if constexpr (FULL) trace_event(p, 3, tr_n, step, phase_kind, EV_ARRIVE);
+            if constexpr (FULL) {
+                // barrier arrival of every CTA in the first traced step, on the global timer (comparable across SMs)
+                if (p.trace && step == p.trace_step && cta < kTraceEvents) {
+                    TraceEvent t;
+                    t.tag = (uint32_t)(phase_kind * 16 + EV_ARRIVE);
+                    t.step = cta;
+                    t.clock = (long long)globaltimer_ns();
+                    p.trace[(8 + phase_kind) * kTraceEvents + cta] = t;
+                }
+            }
             if (s_abort) {
                 atomicExch(&p.ctrl->abort, 1);
             } else {

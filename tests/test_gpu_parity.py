@@ -378,8 +378,13 @@ def test_loop_kernel_timeline_can_be_recorded_without_changing_results(pkg):
         if first < -1:
             assert ev == []
         else:
-            assert ev and {e["step"] for e in ev} <= {3, 4}
-            assert {e["phase"] for e in ev} == {0, 1, 2} and all(0 <= e["role"] < 8 and e["clock"] > 0 for e in ev)
+            roles = [e for e in ev if e["role"] < 8]
+            assert roles and {e["step"] for e in roles} <= {3, 4}
+            assert {e["phase"] for e in roles} == {0, 1, 2} and all(e["clock"] > 0 for e in ev)
+            # barrier arrivals of every CTA in the first traced step, one record per CTA and phase
+            for ph in range(3):
+                ctas = sorted(e["step"] for e in ev if e["role"] == 8 + ph)
+                assert ctas == list(range(len(ctas))) and len(ctas) >= 100 and all(e["phase"] == ph for e in ev if e["role"] == 8 + ph)
     for a, b in zip(outs[0], outs[1]):
         assert np.array_equal(a, b)
 
