@@ -23,6 +23,19 @@
 // (one thread per tensor-memory lane).  State that one phase reads while another CTA writes it
 // is double-buffered by step parity (t, keys), so a phase never reads what it writes.
 //
+// Two modes (template parameter RES).  The description above is the streaming mode: weights flow
+// through a TMA ring every step.  In the resident-weights mode (one or two LSTM layers, shapes whose
+// tiles fit) the W_out tile of a CTA lives in tensor memory and 64-row tiles of W_hh / W_pred (and of
+// layer 1's matrices) in the shared memory of disjoint CTA sets for the whole decode; the GEMMs are
+// transposed (weights on the M axis, utterances on N), every per-step operand is one TMA box, two
+// threads issue the MMAs, eight warps run the epilogues, and CTAs without a weight tile record the
+// steps (outputs, counters, next frame).
+//
+// Two variants (template parameter FULL): teacher forcing with the logits store (wind_eval_joint_window),
+// window-based decoding (the best (label, offset) pair of Eq. (1) decides the step: per-row softmax
+// statistics in the joint's epilogue and a decision phase after it) and the timeline records are compiled
+// into the FULL variant only; a plain decode launches the smaller one.
+//
 // Every wait is bounded (mbarrier waits and the grid barrier): a CTA that runs out of patience
 // flags WIND_ERR_TIMEOUT, raises the global abort word, and every CTA leaves at its next wait.
 #include <cuda.h>
