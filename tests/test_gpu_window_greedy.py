@@ -144,3 +144,23 @@ def test_cfg3_full_batch_sampled_utterances(pkg):
     for b, r in zip(sample, reps):
         assert r["rc"] == 0, f"utterance {b}: {r}"
     print("[window-greedy cfg3]", [(b, int(lens[b]), r["decisions"], r["not_argmax"]) for b, r in zip(sample, reps)])
+
+
+@pytest.mark.parametrize("resident", [1, 0])
+def test_bf16_tensor_path_wide_window_and_overflow(pkg, monkeypatch, resident):
+    # W = 40: more window rows than lanes in the decision warp; then an output buffer that is too small
+    if not resident:
+        monkeypatch.setenv("WIND_RESIDENT", "0")
+    w, enc, lens = ragged_case(540, B=6, T=70, D=64, E=64, P=64, L=1, H=128, V=150, act=1, bias=3.0, dtype="bf16")
+    rep, (tok, frm, olen) = check_window_greedy(pkg, w, enc, lens, 40, 2, kernels=2)
+    assert rep["stats"]["kernels"] == 2 and olen.max() > 4
+    model = pkg.WindModel(w)
+    prev = pkg.wind_set_kernels(2)
+    try:
+        t2, f2, o2, _, st = pkg.decode(model, enc, lens, 40, 2, max_out=4, check=False, window_greedy=True)
+    finally:
+        pkg.wind_set_kernels(prev)
+    assert st == pkg.binding.WIND_ERR_OUTPUT_OVERFLOW and o2.max() == 4
+    for b in range(6):
+        n = min(4, olen[b])
+        assert o2[b] == n and np.array_equal(t2[b, :n], tok[b, :n]) and np.array_equal(f2[b, :n], frm[b, :n])
