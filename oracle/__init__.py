@@ -99,6 +99,9 @@ def lib():
         L.oracle_replay_verify_window.argtypes = [mp, f32p, C.c_int32, C.c_int32, C.c_int32, C.c_double, i32p, i32p,
                                                   C.c_int32, i64p, i64p, i64p, i32p]
         L.oracle_replay_verify_window.restype = C.c_int32
+        L.oracle_beam_search.argtypes = [mp, f32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                         i32p, i32p, i32p, f64p, f64p, i64p]
+        L.oracle_beam_search.restype = C.c_int32
     return _lib
 
 
@@ -179,6 +182,26 @@ def decode_window_greedy_batch(model: Model, enc: np.ndarray, enc_len: np.ndarra
                                             _ptr(tokens, i32p), _ptr(frames, i32p), _ptr(out_len, i32p), max_out,
                                             C.byref(st))
     return tokens, frames, out_len, st.as_dict()
+
+
+def beam_search(model: Model, enc_b: np.ndarray, T: int, W: int, K: int, S: int, max_hyps: int = 64,
+                max_out: Optional[int] = None):
+    """Algorithm 3 for one utterance.  Returns (list of (tokens, frames, score) most probable first, min_gap, steps)."""
+    enc_b = _f32(enc_b)
+    if max_out is None:
+        max_out = max(1, int(T) * S)
+    tok = np.full((max_hyps, max_out), -1, np.int32)
+    frm = np.full((max_hyps, max_out), -1, np.int32)
+    ln = np.zeros(max_hyps, np.int32)
+    sc = np.zeros(max_hyps, np.float64)
+    gap = C.c_double(0.0)
+    steps = C.c_int64(0)
+    n = lib().oracle_beam_search(model.ref, _ptr(enc_b, f32p), int(T), int(W), int(K), int(S), max_hyps, max_out,
+                                 _ptr(tok, i32p), _ptr(frm, i32p), _ptr(ln, i32p), _ptr(sc, f64p), C.byref(gap),
+                                 C.byref(steps))
+    assert n >= 0
+    hyps = [(tok[a, : ln[a]].copy(), frm[a, : ln[a]].copy(), float(sc[a])) for a in range(n)]
+    return hyps, gap.value, steps.value
 
 
 def replay_verify_window(model: Model, enc_b: np.ndarray, T: int, W: int, S: int, tokens: np.ndarray,

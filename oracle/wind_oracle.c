@@ -609,3 +609,205 @@ int32_t oracle_replay_verify_window(const oracle_model_t* m, const float* enc, i
     scratch_free(&s);
     return rc;
 }
+
+/*
+ * Algorithm 3, "WIND Beam-search Algorithm", for one utterance.
+ *
+ * A hypothesis is (tokens, score) plus what this code needs to continue it: the frame of every token, the decoder
+ * state after its tokens, and the count of consecutive emissions on its current frame.  t2hyps maps a frame t to the
+ * hypotheses that have been decoded up to t.  Every iteration takes the smallest t, recombines and prunes its
+ * hypotheses to the beam K, evaluates the joint over the window of n = min(W, T - t) frames for each of them, forms
+ * P'(v, t) of Eq. (1) and expands each hypothesis by its K most probable entries:
+ *   (v != blank, jump): tokens + [v], score + log P'(v, jump), goes to t + jump;
+ *   blank (row n - 1):  same tokens, score + log P'(blank, n - 1), goes to t + n.
+ * The best hypothesis of t2hyps[T] is the result.
+ *
+ * recombine_prune, as far as the paper states it without the cited prefix-search paper: (1) hypotheses with the
+ * same tokens become one, their probabilities summed (the frames of the more probable one are kept; the decoder
+ * states are equal).  Two hypotheses with the same tokens but different counts of emissions on the current frame
+ * are NOT the same under the safeguard (they may continue differently), so they stay apart: with this reading a beam
+ * that never prunes gives every token sequence its total probability over all alignments, for every window;
+ * (3) the K most probable stay.  Step (2), moving the mass of a hypothesis A into a
+ * longer B that A is a prefix of, is NOT part of this function.
+ * Order conventions: entries of P' are ranked by log-probability, then offset, then label; new hypotheses are
+ * appended in the order (hypothesis, rank); duplicates merge into their first occurrence; pruning is a stable sort.
+ * Safeguard against staying on one frame (the paper omits its details): the rule of the greedy decoders above;
+ * a hypothesis whose emission is the S-th in a row on its frame moves to the next frame without a blank factor.
+ * With K = 1 this is window-based greedy decoding.
+ *
+ * min_gap: the smallest difference in log-probability that decided anything (K-th against (K+1)-th entry of a
+ * hypothesis' P', K-th against (K+1)-th hypothesis at pruning, the two scores of a merged pair, best against second
+ * final hypothesis).  A comparison against results computed in lower precision is only meaningful above it.
+ */
+typedef struct {
+    int32_t* tok;
+    int32_t* frm;
+    int32_t len, count;
+    double score;
+    double *h, *c, *g;
+} beam_hyp_t;
+
+typedef struct { beam_hyp_t** v; int n, cap; } beam_list_t;
+typedef struct { double lp; int32_t j, v; } beam_cand_t;
+
+static void beam_push(beam_list_t* l, beam_hyp_t* h) {
+    if (l->n == l->cap) { l->cap = l->cap ? 2 * l->cap : 8; l->v = (beam_hyp_t**)realloc(l->v, sizeof(beam_hyp_t*) * (size_t)l->cap); }
+    l->v[l->n++] = h;
+}
+static void beam_free(beam_hyp_t* h) { free(h->tok); free(h->frm); free(h->h); free(h->c); free(h->g); free(h); }
+static beam_hyp_t* beam_clone(const oracle_model_t* m, const beam_hyp_t* a, int extra) {
+    beam_hyp_t* b = (beam_hyp_t*)malloc(sizeof(beam_hyp_t));
+    *b = *a;
+    b->tok = (int32_t*)malloc(sizeof(int32_t) * (size_t)(a->len + extra + 1));
+    b->frm = (int32_t*)malloc(sizeof(int32_t) * (size_t)(a->len + extra + 1));
+    memcpy(b->tok, a->tok, sizeof(int32_t) * (size_t)a->len);
+    memcpy(b->frm, a->frm, sizeof(int32_t) * (size_t)a->len);
+    const size_t ns = (size_t)m->L * m->P;
+    b->h = (double*)malloc(sizeof(double) * ns); memcpy(b->h, a->h, sizeof(double) * ns);
+    b->c = (double*)malloc(sizeof(double) * ns); memcpy(b->c, a->c, sizeof(double) * ns);
+    b->g = (double*)malloc(sizeof(double) * (size_t)m->H); memcpy(b->g, a->g, sizeof(double) * (size_t)m->H);
+    return b;
+}
+static int beam_cand_cmp(const void* pa, const void* pb) {
+    const beam_cand_t* a = (const beam_cand_t*)pa; const beam_cand_t* b = (const beam_cand_t*)pb;
+    if (a->lp != b->lp) return a->lp > b->lp ? -1 : 1;
+    if (a->j != b->j) return a->j < b->j ? -1 : 1;
+    return a->v < b->v ? -1 : (a->v > b->v ? 1 : 0);
+}
+static double log_add(double a, double b) {
+    if (a == -INFINITY) return b;
+    if (b == -INFINITY) return a;
+    return a > b ? a + log1p(exp(b - a)) : b + log1p(exp(a - b));
+}
+static void note_gap(double* min_gap, double g) { if (g >= 0 && g < *min_gap) *min_gap = g; }
+
+/* duplicates -> one (probabilities summed), then the K most probable, stable; freed hypotheses are released */
+static void beam_recombine_prune(beam_list_t* l, int K, double* min_gap) {
+    for (int a = 0; a < l->n; ++a) {
+        for (int b = a + 1; b < l->n;) {
+            beam_hyp_t *x = l->v[a], *y = l->v[b];
+            if (x->len == y->len && x->count == y->count && memcmp(x->tok, y->tok, sizeof(int32_t) * (size_t)x->len) == 0) {
+                note_gap(min_gap, fabs(x->score - y->score));
+                const double sum = log_add(x->score, y->score);
+                if (y->score > x->score) { l->v[a] = y; beam_free(x); x = y; } else beam_free(y);
+                x->score = sum;
+                for (int k = b; k + 1 < l->n; ++k) l->v[k] = l->v[k + 1];
+                l->n--;
+            } else {
+                ++b;
+            }
+        }
+    }
+    for (int a = 1; a < l->n; ++a) {   /* stable insertion sort, most probable first */
+        beam_hyp_t* x = l->v[a];
+        int k = a;
+        while (k > 0 && l->v[k - 1]->score < x->score) { l->v[k] = l->v[k - 1]; --k; }
+        l->v[k] = x;
+    }
+    if (l->n > K) {
+        note_gap(min_gap, l->v[K - 1]->score - l->v[K]->score);
+        for (int a = K; a < l->n; ++a) beam_free(l->v[a]);
+        l->n = K;
+    }
+}
+
+int32_t oracle_beam_search(const oracle_model_t* m, const float* enc, int32_t T, int32_t W, int32_t K, int32_t S,
+                           int32_t max_hyps_out, int32_t max_out, int32_t* out_tokens, int32_t* out_frames,
+                           int32_t* out_len, double* out_score, double* min_gap_out, int64_t* n_steps_out) {
+    if (W < 1 || W > 64 || K < 1 || S < 1 || T < 0) return -1;
+    const int NV = m->V + 1;
+    double* encp = (double*)malloc(sizeof(double) * (size_t)(T > 0 ? T : 1) * m->H);
+    oracle_enc_proj(m, enc, T, encp);
+    double* logits = (double*)malloc(sizeof(double) * (size_t)W * NV);
+    double* z = (double*)malloc(sizeof(double) * (size_t)m->H);
+    beam_cand_t* cand = (beam_cand_t*)malloc(sizeof(beam_cand_t) * (size_t)W * NV);
+    beam_list_t* t2hyps = (beam_list_t*)calloc((size_t)T + 1, sizeof(beam_list_t));
+    double min_gap = INFINITY;
+    int64_t steps = 0;
+    {   /* t2hyps = {0: [Hyp(tokens = [], score = 0)]} */
+        beam_hyp_t* h0 = (beam_hyp_t*)calloc(1, sizeof(beam_hyp_t));
+        h0->tok = (int32_t*)malloc(sizeof(int32_t)); h0->frm = (int32_t*)malloc(sizeof(int32_t));
+        h0->h = (double*)calloc((size_t)m->L * m->P, sizeof(double));
+        h0->c = (double*)calloc((size_t)m->L * m->P, sizeof(double));
+        h0->g = (double*)malloc(sizeof(double) * (size_t)m->H);
+        oracle_lstm_step(m, m->blank_id, h0->h, h0->c);
+        oracle_pred_proj(m, h0->h, h0->g);
+        beam_push(&t2hyps[0], h0);
+    }
+    for (int t = 0; t < T; ++t) {
+        beam_list_t* cur = &t2hyps[t];
+        while (cur->n > 0) {   /* a frame is taken again when an expansion stays on it (jump 0) */
+            beam_list_t hyps = *cur;
+            cur->v = NULL; cur->n = 0; cur->cap = 0;
+            beam_recombine_prune(&hyps, K, &min_gap);
+            const int n = (W < T - t) ? W : (T - t);
+            steps++;
+            for (int b = 0; b < hyps.n; ++b) {
+                beam_hyp_t* hy = hyps.v[b];
+                /* log P'(v, j) of Eq. (1) for this hypothesis' decoder state */
+                double blanks_before = 0.0;
+                int nc = 0;
+                for (int j = 0; j < n; ++j) {
+                    double* row = logits + (size_t)j * NV;
+                    oracle_joint_logits(m, encp + (size_t)(t + j) * m->H, hy->g, z, row);
+                    double mx = row[0];
+                    for (int v = 1; v < NV; ++v) if (row[v] > mx) mx = row[v];
+                    double se = 0.0;
+                    for (int v = 0; v < NV; ++v) se += exp(row[v] - mx);
+                    const double lse = mx + log(se);
+                    for (int v = 0; v < NV; ++v) {
+                        if (v == m->blank_id && j < n - 1) continue;
+                        cand[nc].lp = row[v] - lse + blanks_before; cand[nc].j = j; cand[nc].v = v; nc++;
+                    }
+                    blanks_before += row[m->blank_id] - lse;
+                }
+                qsort(cand, (size_t)nc, sizeof(beam_cand_t), beam_cand_cmp);
+                const int take = K < nc ? K : nc;
+                if (take < nc) note_gap(&min_gap, cand[take - 1].lp - cand[take].lp);
+                for (int k = 0; k < take; ++k) {
+                    if (cand[k].v != m->blank_id) {
+                        beam_hyp_t* nh = beam_clone(m, hy, 1);
+                        int tt = t + cand[k].j;
+                        nh->tok[nh->len] = cand[k].v; nh->frm[nh->len] = tt; nh->len++;
+                        nh->score += cand[k].lp;
+                        nh->count = cand[k].j == 0 ? hy->count + 1 : 1;
+                        oracle_lstm_step(m, cand[k].v, nh->h, nh->c);
+                        oracle_pred_proj(m, nh->h, nh->g);
+                        if (nh->count == S) { tt += 1; nh->count = 0; }
+                        beam_push(&t2hyps[tt], nh);
+                    } else {
+                        beam_hyp_t* nh = beam_clone(m, hy, 0);
+                        nh->score += cand[k].lp;
+                        nh->count = 0;
+                        beam_push(&t2hyps[t + n], nh);
+                    }
+                }
+            }
+            for (int b = 0; b < hyps.n; ++b) beam_free(hyps.v[b]);
+            free(hyps.v);
+        }
+        free(cur->v); cur->v = NULL;
+    }
+    /* best_hyp_in(t2hyps[T]): duplicates merged, most probable first */
+    beam_list_t* fin = &t2hyps[T];
+    beam_recombine_prune(fin, fin->n > 0 ? fin->n : 1, &min_gap);
+    if (fin->n > 1) note_gap(&min_gap, fin->v[0]->score - fin->v[1]->score);
+    int n_out = 0;
+    for (int a = 0; a < fin->n; ++a) {
+        if (a < max_hyps_out) {
+            const beam_hyp_t* h = fin->v[a];
+            out_len[a] = h->len; out_score[a] = h->score;
+            for (int k = 0; k < h->len && k < max_out; ++k) {
+                out_tokens[(size_t)a * max_out + k] = h->tok[k];
+                out_frames[(size_t)a * max_out + k] = h->frm[k];
+            }
+            n_out++;
+        }
+        beam_free(fin->v[a]);
+    }
+    free(fin->v);
+    free(t2hyps); free(cand); free(z); free(logits); free(encp);
+    if (min_gap_out) *min_gap_out = min_gap;
+    if (n_steps_out) *n_steps_out = steps;
+    return n_out;
+}

@@ -563,3 +563,85 @@ def test_window_replay_accepts_own_output_and_rejects_mistakes():
     # with a margin above the gap the first decision passes (whatever happens at the second one)
     res = oracle.replay_verify_window(m, enc[b], T, W, 3, tk4[:1], fr[:1], margin_thr=gap * 1.01)
     assert res["decisions"] >= 2 and res["not_argmax"] >= 1
+
+
+# ---------------------------------------------------------------------------
+# Algorithm 3: WIND beam search
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("seed,W,S,bias", [(0, 4, 3, 1.0), (1, 1, 2, 0.5), (2, 8, 1, 1.5), (3, 3, 10, 2.0)])
+def test_beam_search_with_beam_one_is_window_based_greedy(seed, W, S, bias):
+    w, enc, lens = small_case(90 + seed, B=1, T=30, bias=bias, S=S)
+    m = oracle.Model(w)
+    T = int(lens[0])
+    hyps, gap, steps = oracle.beam_search(m, enc[0], T, W, 1, S)
+    tok, frm, n, st = oracle.decode_window_greedy_batch(m, enc, lens, W=W, S=S)
+    assert len(hyps) == 1 and steps == st["steps"]
+    assert list(hyps[0][0]) == list(tok[0, : n[0]]) and list(hyps[0][1]) == list(frm[0, : n[0]])
+
+
+def brute_force_sequence_probabilities(nm, enc, S):
+    """Total probability of every token sequence: all alignments walked frame by frame on independently evaluated
+    logits (blank advances; a label stays on the frame, the S-th label in a row on a frame advances without a blank)."""
+    T = enc.shape[0]
+    cache, total = {}, {}
+
+    def logp(t, hyp):
+        key = (t, tuple(hyp))
+        if key not in cache:
+            cache[key] = torch.log_softmax(torch.tensor(nm.logits(enc[t], hyp)), dim=0).numpy()
+        return cache[key]
+
+    def walk(t, hyp, count, acc):
+        if t == T:
+            total[tuple(hyp)] = np.logaddexp(total.get(tuple(hyp), -np.inf), acc)
+            return
+        lp = logp(t, hyp)
+        walk(t + 1, hyp, 0, acc + lp[nm.blank])
+        for v in range(len(lp)):
+            if v != nm.blank:
+                if count + 1 == S:
+                    walk(t + 1, hyp + [v], 0, acc + lp[v])
+                else:
+                    walk(t, hyp + [v], count + 1, acc + lp[v])
+
+    walk(0, [], 0, 0.0)
+    return total
+
+
+@pytest.mark.parametrize("seed,blank0", [(0, False), (1, True)])
+def test_beam_search_without_pruning_sums_all_alignments_for_every_window(seed, blank0):
+    # a beam wider than the number of hypotheses never prunes: the final score of a token sequence is then the log of
+    # its total probability over all alignments, whatever the window
+    r = rng(950 + seed)
+    V, T, S = 2, 3, 2
+    w = random_weights(r, 4, 3, 4, 1, 5, V, blank_id=0 if blank0 else None, act=seed % 2, blank_bias=0.3, bias_scale=0.1)
+    enc = r.standard_normal((T, 4)).astype(np.float32)
+    want = brute_force_sequence_probabilities(NaiveModel(w), enc, S)
+    assert abs(np.logaddexp.reduce(list(want.values()))) < 1e-9            # the sequences' probabilities sum to one
+    m = oracle.Model(w)
+    for W in (1, 2, 3, 5):
+        hyps, gap, steps = oracle.beam_search(m, enc, T, W, 4096, S, max_hyps=4096)
+        got = {tuple(int(x) for x in h[0]): h[2] for h in hyps}
+        assert set(got) == set(want)
+        for k in want:
+            assert abs(got[k] - want[k]) < 1e-7, (W, k)
+        scores = [h[2] for h in hyps]
+        assert scores == sorted(scores, reverse=True)
+
+
+def test_beam_search_worked_example_beats_greedy():
+    # frame types A = (x .45, y .05, blank .5), B = (x .1, y .8, blank .1); utterance A B, W = 2, S = 1, K = 2:
+    #   t = 0, []: P'(x,0) = .45, P'(y,1) = .5 * .8 = .4 are the two best -> [x] (frame 0, then forced to t = 1) and
+    #              [y] (frame 1, forced to t = 2)
+    #   t = 1, [x]: window [B]: P'(y,0) = .8, then x and blank tie at .1 (the label comes first) -> [x,y] .36, [x,x] .045
+    #   t = 2 = T: [y] .4 > [x,y] .36 > [x,x] .045.   With K = 1 (window-based greedy): [x] then [x,y], .36.
+    w = table_model([[.45, .05, .5], [.1, .8, .1]])
+    enc = np.eye(2, dtype=np.float32)[[0, 1]]
+    m = oracle.Model(w)
+    hyps, gap, steps = oracle.beam_search(m, enc, 2, 2, 2, 1)
+    assert [list(h[0]) for h in hyps] == [[1], [0, 1], [0, 0]]
+    assert [list(h[1]) for h in hyps] == [[1], [0, 1], [0, 1]]
+    assert np.allclose([h[2] for h in hyps], np.log([.4, .36, .045]), atol=1e-6) and steps == 2
+    one, _, _ = oracle.beam_search(m, enc, 2, 2, 1, 1)
+    assert list(one[0][0]) == [0, 1] and abs(one[0][2] - np.log(.36)) < 1e-6
+    assert abs(gap - 0.0) < 1e-6      # the x / blank tie is reported as a zero gap
