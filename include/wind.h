@@ -255,6 +255,38 @@ wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const 
                                   size_t workspace_bytes, void* stream, wind_profile_t* host_out);
 
 /*
+ * WIND beam search (Algorithm 3) for ONE utterance, beam K, window W.
+ * A map from frames to partial hypotheses is worked off in frame order: the hypotheses of the smallest frame t are
+ * recombined and pruned to K, the joint is evaluated over the window of n = min(W, T - t) frames for each of them,
+ * P'(v, t) of Eq. (1) is formed and every hypothesis is expanded by its K most probable entries (a label at an
+ * offset: appended, continues at t + offset; the blank entry: continues at t + n).  The most probable hypotheses
+ * that reached frame T are returned, best first.
+ * Recombination: hypotheses with the same tokens (and the same count of emissions on the current frame) become one
+ * with their probabilities summed; then the K most probable stay.  The transfer of probability from a hypothesis to
+ * a longer one that it is a prefix of (the cited prefix search) is not part of this function.
+ * max_symbols: as in wind_decode_greedy (the paper leaves its safeguard for this algorithm to its code).
+ * Entries of P' are ranked by probability, then offset, then label.  Scores are natural-log probabilities; the
+ * window's log-softmax is fp32, sums over steps are fp64.  K = 1 gives wind_decode_window_greedy's result.
+ * The map, recombination and pruning run on the host; the model arithmetic (encoder projection, decoder updates of
+ * surviving hypotheses, windowed joint, Eq. (1) and its K best entries) runs in kernels on `stream`, which the call
+ * synchronises once per iteration to read K x K (label, offset, log-probability) triples.
+ *   enc        DEVICE [T, D], element type m->dtype.    T >= 1, 1 <= W <= 64, 1 <= K <= 16.
+ *   out_*      HOST: tokens/frames [max_hyps, max_out], lengths and scores [max_hyps], *n_hyps = hypotheses written
+ *              (at most max_hyps, best first); a hypothesis longer than max_out is cut in the token arrays, its
+ *              length is reported in full.  n_steps (may be null): iterations of the loop.
+ *   workspace  DEVICE, at least wind_beam_workspace_bytes(m, T, W, K, max_symbols); 256-byte aligned.
+ * WIND_ERR_WORKSPACE also when the pool of decoder states (sized for K (W + 2) (min(max_symbols, 32) + 2) live
+ * hypotheses) runs out.
+ */
+wind_status_t wind_beam_workspace_bytes(const wind_model_t* m, int32_t T, int32_t W, int32_t K, int32_t max_symbols,
+                                        size_t* bytes);
+wind_status_t wind_beam_search(const wind_model_t* m, const void* enc, int32_t T, int32_t W, int32_t K,
+                               int32_t max_symbols, int32_t max_hyps, int32_t max_out, int32_t* out_tokens_host,
+                               int32_t* out_frames_host, int32_t* out_len_host, double* out_score_host,
+                               int32_t* n_hyps_host, int64_t* n_steps_host, void* workspace, size_t workspace_bytes,
+                               void* stream);
+
+/*
  * Length-aware batching of a set of N utterances (host-only; no CUDA call).  The lock-step loop of a batch runs until
  * its longest utterance is done, so batches of mixed lengths leave most rows idle for most steps: the paper's batched
  * gain shrinks as the batch grows for the same reason.  The plan sorts the utterances by length, longest first (equal

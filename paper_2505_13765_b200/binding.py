@@ -30,7 +30,7 @@ WIND_KERNELS_AUTO, WIND_KERNELS_SIMT, WIND_KERNELS_TENSOR = 0, 1, 2
 
 EXPORTS = [
     "wind_workspace_bytes", "wind_decode_greedy", "wind_decode_window_greedy", "wind_host_staging_bytes", "wind_decode_greedy_host",
-    "wind_eval_joint_window", "wind_window_first_output", "wind_eval_joint_window_static", "wind_profile_decode", "wind_plan_batches", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_debug_stall_barrier", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
+    "wind_eval_joint_window", "wind_window_first_output", "wind_eval_joint_window_static", "wind_profile_decode", "wind_beam_workspace_bytes", "wind_beam_search", "wind_plan_batches", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_debug_stall_barrier", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
 ]
 
 _vp = C.c_void_p
@@ -106,6 +106,11 @@ def load_library():
     L.wind_window_first_output.restype = i32
     L.wind_eval_joint_window_static.argtypes = [mp, _vp, _vp, i32, i32, i32, _vp, i32, _vp, _vp, _vp, _vp]
     L.wind_eval_joint_window_static.restype = i32
+    L.wind_beam_workspace_bytes.argtypes = [mp, i32, i32, i32, i32, C.POINTER(C.c_size_t)]
+    L.wind_beam_workspace_bytes.restype = i32
+    L.wind_beam_search.argtypes = [mp, _vp, i32, i32, i32, i32, i32, i32, _vp, _vp, _vp, _vp, C.POINTER(i32),
+                                   C.POINTER(C.c_int64), _vp, C.c_size_t, _vp]
+    L.wind_beam_search.restype = i32
     L.wind_plan_batches.argtypes = [_vp, i32, i32, _vp, _vp, C.POINTER(i32)]
     L.wind_plan_batches.restype = i32
     L.wind_read_stats.argtypes = [_vp, _vp, C.POINTER(wind_stats_t)]
@@ -391,6 +396,37 @@ def to_device_enc(model: WindModel, enc_np: np.ndarray):
     torch = _torch()
     t = torch.from_numpy(np.ascontiguousarray(enc_np, dtype=np.float32))
     return t.to(model.torch_dtype).to(model.device).contiguous()
+
+
+def wind_beam_search(model: WindModel, enc_np: np.ndarray, W: int, K: int, S: int, max_hyps: int = 64,
+                     max_out: Optional[int] = None, check: bool = True):
+    """Algorithm 3 for one utterance [T, D] (numpy).  Returns (list of (tokens, frames, score) best first, steps, status)."""
+    torch = _torch()
+    L = load_library()
+    T = int(enc_np.shape[0])
+    enc = to_device_enc(model, enc_np[None])[0].contiguous()
+    if max_out is None:
+        max_out = max(1, T * S)
+    n = C.c_size_t(0)
+    st = L.wind_beam_workspace_bytes(model.ref, T, W, K, S, C.byref(n))
+    if st != WIND_OK:
+        if check:
+            raise WindError(st)
+        return [], 0, st
+    ws = torch.empty(n.value + 256, dtype=torch.uint8, device=model.device)
+    off = (-ws.data_ptr()) % 256
+    tok = np.full((max_hyps, max_out), -1, np.int32)
+    frm = np.full((max_hyps, max_out), -1, np.int32)
+    ln = np.zeros(max_hyps, np.int32)
+    sc = np.zeros(max_hyps, np.float64)
+    nh, steps = C.c_int32(0), C.c_int64(0)
+    st = L.wind_beam_search(model.ref, enc.data_ptr(), T, W, K, S, max_hyps, max_out, tok.ctypes.data, frm.ctypes.data,
+                            ln.ctypes.data, sc.ctypes.data, C.byref(nh), C.byref(steps), ws.data_ptr() + off, n.value,
+                            _stream_ptr(None))
+    if check and st != WIND_OK:
+        raise WindError(st)
+    hyps = [(tok[a, : min(ln[a], max_out)].copy(), frm[a, : min(ln[a], max_out)].copy(), float(sc[a])) for a in range(nh.value)]
+    return hyps, steps.value, st
 
 
 def wind_plan_batches(lens_np: np.ndarray, B: int):

@@ -513,6 +513,46 @@ wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const 
     return read_status(c);
 }
 
+static wind_status_t check_beam_args(const wind_model_t* m, int32_t T, int32_t W, int32_t K, int32_t S) {
+    wind_status_t s = check_model(m);
+    if (s != WIND_OK) return s;
+    if (K < 1 || S < 1) return WIND_ERR_INVALID_ARG;
+    if (K > 16) return WIND_ERR_UNSUPPORTED;
+    return check_shape(m, K, T, W);
+}
+
+wind_status_t wind_beam_workspace_bytes(const wind_model_t* m, int32_t T, int32_t W, int32_t K, int32_t max_symbols,
+                                        size_t* bytes) {
+    wind_status_t s = check_beam_args(m, T, W, K, max_symbols);
+    if (s != WIND_OK) return s;
+    if (!bytes) return WIND_ERR_INVALID_ARG;
+    *bytes = make_beam_layout(*m, T, W, K, max_symbols, make_layout(*m, K, T, W, 1).total).total;
+    return WIND_OK;
+}
+
+wind_status_t wind_beam_search(const wind_model_t* m, const void* enc, int32_t T, int32_t W, int32_t K, int32_t max_symbols,
+                               int32_t max_hyps, int32_t max_out, int32_t* out_tokens_host, int32_t* out_frames_host,
+                               int32_t* out_len_host, double* out_score_host, int32_t* n_hyps_host, int64_t* n_steps_host,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+    wind_status_t s = check_beam_args(m, T, W, K, max_symbols);
+    if (s != WIND_OK) return s;
+    s = check_weights(m);
+    if (s != WIND_OK) return s;
+    if (!enc || !out_tokens_host || !out_frames_host || !out_len_host || !out_score_host || !n_hyps_host || !workspace ||
+        max_hyps < 1 || max_out < 1)
+        return WIND_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return WIND_ERR_WORKSPACE;
+    Call cb;
+    fill_call(cb, m, enc, nullptr, K, T, W, max_symbols, nullptr, nullptr, nullptr, 1, workspace, (cudaStream_t)stream);
+    const BeamLayout bl = make_beam_layout(*m, T, W, K, max_symbols, cb.lay.total);
+    if (workspace_bytes < bl.total) return WIND_ERR_WORKSPACE;
+    cudaError_t ce = cudaSuccess;
+    s = beam_search_run(cb, bl, K, max_hyps, max_out, out_tokens_host, out_frames_host, out_len_host, out_score_host,
+                        n_hyps_host, n_steps_host, &ce);
+    if (s == WIND_ERR_CUDA) return cuda_fail(ce, "beam search");
+    return s;
+}
+
 wind_status_t wind_plan_batches(const int32_t* enc_len, int32_t N, int32_t B, int32_t* order, int32_t* batch_T,
                                 int32_t* n_batches) {
     if (!enc_len || !order || !n_batches || N < 0 || B < 1) return WIND_ERR_INVALID_ARG;

@@ -181,6 +181,7 @@ __device__ inline void set_status(Ctrl* ctrl, int32_t s) { atomicCAS(&ctrl->stat
 cudaError_t simt_enc_proj(const Call& c);
 cudaError_t simt_pred_step(const Call& c, int parity_in);            // all layers + pred_proj
 cudaError_t simt_joint(const Call& c, float* logits_out /*nullable*/);
+cudaError_t simt_joint_shared(const Call& c, float* logits_out);   // every row's window comes from utterance 0 (beam search)
 int simt_pred_launches(const Call& c);
 
 // control
@@ -190,6 +191,20 @@ cudaError_t launch_force_tokens(const Call& c, const int32_t* prefix, int U, con
 cudaError_t launch_set_t(const Call& c, const int32_t* t0);
 
 // first-output distribution of a window (Eq. 1), in place on the window's logits
+// beam search (Algorithm 3): workspace regions behind the call's own layout, and the host-driven search
+struct BeamLayout {
+    size_t h_pool, c_pool, g_pool;   // fp32 [slots][L][P] x 2, [slots][H]: decoder states of live hypotheses and their pred_proj
+    size_t ints;                     // int32 [8][K] per-iteration index arrays
+    size_t logits;                   // fp32 [K][W][V+1]
+    size_t top_label, top_jump, top_logp;   // [K][K]
+    size_t total;
+    int slots;
+};
+BeamLayout make_beam_layout(const wind_model_t& m, int T, int W, int K, int S, size_t base);
+wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyps, int max_out, int32_t* out_tokens,
+                              int32_t* out_frames, int32_t* out_len, double* out_score, int32_t* n_hyps, int64_t* n_steps,
+                              cudaError_t* cuda_err);
+
 cudaError_t launch_first_output(float* logp, const int32_t* enc_len, const int32_t* t0, int B, int W, int NV, int blank, int K,
                                 int32_t* top_label, int32_t* top_jump, float* top_logp, cudaStream_t stream);
 

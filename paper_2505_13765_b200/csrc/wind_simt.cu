@@ -333,6 +333,15 @@ static cudaError_t simt_joint_t(const Call& c, float* logits_out) {
     return cudaGetLastError();
 }
 
+// Beam search: the rows are hypotheses of ONE utterance; a frame stride of zero makes every block read utterance 0.
+cudaError_t simt_joint_shared(const Call& c, float* logits_out) {
+    Call one = c;
+    one.T = 0;
+    one.mode = WIND_MODE_FIRST_NONBLANK;
+    if (c.m.dtype == WIND_DT_BF16) return simt_joint_t<__nv_bfloat16, false>(one, logits_out);
+    return simt_joint_t<float, false>(one, logits_out);
+}
+
 cudaError_t simt_joint(const Call& c, float* logits_out) {
     if (c.B == 0) return cudaSuccess;
     const bool wg = c.mode == WIND_MODE_WINDOW && !logits_out;

@@ -86,6 +86,15 @@ def test_invalid_arguments_are_rejected_on_the_host(lib):
     assert lib.wind_window_first_output(*fo) == bd.WIND_ERR_INVALID_ARG      # K < 0
     fo[11] = 3
     assert lib.wind_window_first_output(*fo) == bd.WIND_ERR_INVALID_ARG      # K > 0 without output arrays
+    # beam search: shape limits and null pointers
+    assert lib.wind_beam_workspace_bytes(ref, 100, 8, 0, 3, C.byref(n)) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_beam_workspace_bytes(ref, 100, 8, 17, 3, C.byref(n)) == bd.WIND_ERR_UNSUPPORTED
+    assert lib.wind_beam_workspace_bytes(ref, 100, 65, 4, 3, C.byref(n)) == bd.WIND_ERR_UNSUPPORTED
+    assert lib.wind_beam_workspace_bytes(ref, 100, 8, 4, 3, None) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_beam_workspace_bytes(ref, 1500, 8, 4, 10, C.byref(n)) == bd.WIND_OK and 0 < n.value < (1 << 30)
+    nh, ns = C.c_int32(0), C.c_int64(0)
+    assert lib.wind_beam_search(ref, None, 100, 8, 4, 3, 8, 100, None, None, None, None, C.byref(nh), C.byref(ns), None, 0, None) \
+        == bd.WIND_ERR_INVALID_ARG
     n_ev = C.c_int32(0)
     assert lib.wind_read_trace(ref, 1, 10, 4, None, None, None, 0, C.byref(n_ev)) == bd.WIND_ERR_INVALID_ARG
 
