@@ -184,10 +184,10 @@ def main():
     ap.add_argument("--len-hi", type=int, default=0, help="override the longest utterance length, frames")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the W=1 comparison, e2e and per-kernel timing legs")
-    ap.add_argument("--op", default="decode", choices=["decode", "first_output", "window_greedy", "dataset"],
+    ap.add_argument("--op", default="decode", choices=["decode", "first_output", "window_greedy", "dataset", "beam"],
                     help="first_output: time wind_window_first_output (Eq. 1 on one window per utterance) instead of the decode; "
                          "window_greedy: time wind_decode_window_greedy on the whole workload; dataset: 4 x B utterances in "
-                         "arrival-order batches against length-aware batches")
+                         "arrival-order batches against length-aware batches; beam: wind_beam_search on one utterance, beams 2..4")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -206,6 +206,8 @@ def main():
         return window_greedy_op(args, cfg, W)
     if args.op == "dataset":
         return dataset_op(args, cfg, W)
+    if args.op == "beam":
+        return beam_op(args, cfg, W)
 
     import torch
     import paper_2505_13765_b200 as pkg
@@ -583,6 +585,51 @@ def dataset_op(args, cfg, W):
         "arrival_order": {"ms": ms_a, "lock_steps": steps_a, "value": audio_s / (ms_a * 1e-3)},
         "speedup_vs_arrival_order": ms_a / ms_p, "gpu_launches": 4 * len(batch_T) * args.steps,
     }))
+
+
+def beam_op(args, cfg, W):
+    """Secondary measurement (one JSON line per beam width): WIND beam search (Algorithm 3) on the first utterance of
+    the workload, beams 2, 3 and 4, through wind_beam_search (encoder frames resident on the device; the call's own
+    host-side bookkeeping and its one synchronisation per iteration are inside the timed region, which is wall clock
+    around the call: the search is driven from the host).  Beside it the oracle on the utterance's first frames."""
+    import torch
+    import wind_synth as ws
+    import paper_2505_13765_b200 as pkg
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    pkg.load_library()
+    weights = ws.make_model(cfg)
+    enc_np, lens_np = ws.make_enc(cfg, pad="zero")
+    b = int(np.argmax(lens_np))
+    T = int(lens_np[b])
+    enc = np.ascontiguousarray(enc_np[b, :T])
+    model = pkg.WindModel(weights, device=dev)
+    for K in (2, 3, 4):
+        for _ in range(2):
+            pkg.wind_beam_search(model, enc, W, K, cfg.S, max_hyps=8)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            hyps, steps, st = pkg.wind_beam_search(model, enc, W, K, cfg.S, max_hyps=8)
+        torch.cuda.synchronize()
+        dt = (time.perf_counter() - t0) / args.steps
+        cb = None
+        if not args.no_cpu_baseline:
+            import oracle
+            Tc = min(T, 24)
+            t1 = time.perf_counter()
+            _, _, osteps = oracle.beam_search(oracle.Model(weights), enc[:Tc], Tc, W, K, cfg.S)
+            od = time.perf_counter() - t1
+            cb = dict(value=Tc * FRAME_SECONDS / od, unit="audio-s/s", cores=1, kind="oracle",
+                      sample=f"first {Tc} frames of the utterance, {osteps} iterations, one run, {od:.1f} s")
+        print(json.dumps({
+            "metric": "WIND beam search RTFx, one utterance (audio-s/s at 80 ms/frame)", "op": "beam", "value": T * FRAME_SECONDS / dt,
+            "unit": "audio-s/s", "n_gpus": 1, "steps": args.steps, "warmup": 2, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": cfg.name, "utterance": b, "frames": T, "W": W, "K": K, "max_symbols": cfg.S},
+            "iterations": steps, "us_per_iteration": dt * 1e6 / max(1, steps), "best_tokens": int(len(hyps[0][0])),
+            "best_score": hyps[0][2], "final_hypotheses": len(hyps), "cpu_baseline": cb,
+        }))
 
 
 def reference_arm(args, cfg, W):

@@ -66,8 +66,14 @@ __global__ void beam_fill_kernel(int32_t* a, int n, int v) {
     if (i < n) a[i] = v;
 }
 
+// Token histories are shared: a hypothesis points at the node of its last token, a node at the node before it.
+struct Node {
+    int32_t parent, tok, frm, len;
+    uint64_t hash;          // of the token sequence up to here
+};
+
 struct Hyp {
-    std::vector<int32_t> tok, frm;
+    int32_t node = -1;      // -1: no tokens
     double score = 0.0;
     int count = 0;
     int slot = -1;          // decoder state after tok (-1: not evaluated yet)
@@ -94,9 +100,9 @@ BeamLayout make_beam_layout(const wind_model_t& m, int T, int W, int K, int S, s
     L.g_pool = take(sizeof(float) * (size_t)L.slots * m.H);
     L.ints = take(sizeof(int32_t) * 8 * (size_t)K);
     L.logits = take(sizeof(float) * (size_t)K * W * (m.V + 1));
-    L.top_label = take(sizeof(int32_t) * (size_t)K * K);
-    L.top_jump = take(sizeof(int32_t) * (size_t)K * K);
-    L.top_logp = take(sizeof(float) * (size_t)K * K);
+    L.top_label = take(sizeof(int32_t) * 3 * (size_t)K * K);   // labels, offsets, log-probabilities: one block, one copy
+    L.top_jump = L.top_label + sizeof(int32_t) * (size_t)K * K;
+    L.top_logp = L.top_jump + sizeof(int32_t) * (size_t)K * K;
     L.total = off;
     return L;
 }
@@ -147,15 +153,29 @@ wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyp
         refs[0]++;
         t2hyps[0].push_back(std::move(h0));
     }
-    std::vector<int32_t> host_ints(4 * (size_t)K), top_label((size_t)K * K), top_jump((size_t)K * K);
-    std::vector<float> top_logp((size_t)K * K);
+    std::vector<int32_t> host_ints(4 * (size_t)K), top(3 * (size_t)K * K);
+    const int32_t* top_label = top.data();
+    const int32_t* top_jump = top.data() + (size_t)K * K;
+    const float* top_logp = reinterpret_cast<const float*>(top.data() + 2 * (size_t)K * K);
     int64_t steps = 0;
     bool first = true;
 
+    std::vector<Node> nodes;
+    auto node_len = [&](int32_t n) { return n < 0 ? 0 : nodes[(size_t)n].len; };
+    auto node_hash = [&](int32_t n) { return n < 0 ? 0x9E3779B97F4A7C15ull : nodes[(size_t)n].hash; };
+    auto same_tokens = [&](int32_t x, int32_t y) {
+        if (node_len(x) != node_len(y) || node_hash(x) != node_hash(y)) return false;
+        while (x != y) {   // equal lengths: the chains end together, or meet at a shared node
+            if (nodes[(size_t)x].tok != nodes[(size_t)y].tok) return false;
+            x = nodes[(size_t)x].parent;
+            y = nodes[(size_t)y].parent;
+        }
+        return true;
+    };
     auto recombine_prune = [&](std::vector<Hyp>& l, size_t keep) {
         for (size_t a = 0; a < l.size(); ++a)
             for (size_t b = a + 1; b < l.size();) {
-                if (l[a].count == l[b].count && l[a].tok == l[b].tok) {
+                if (l[a].count == l[b].count && same_tokens(l[a].node, l[b].node)) {
                     const double sum = log_add(l[a].score, l[b].score);
                     if (l[b].score > l[a].score) std::swap(l[a], l[b]);
                     l[a].score = sum;
@@ -191,7 +211,7 @@ wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyp
                     free_slots.pop_back();
                     refs[s] = 1;
                     host_ints[nu] = h.parent;
-                    host_ints[K + nu] = first ? m.blank_id : h.tok.back();
+                    host_ints[K + nu] = first ? m.blank_id : nodes[(size_t)h.node].tok;
                     host_ints[2 * K + nu] = s;
                     h.slot = s;
                     ++nu;
@@ -213,9 +233,7 @@ wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyp
             // ---- window logits of every hypothesis, Eq. (1), the K best entries each ----
             BEAM_CUDA(simt_joint_shared(cb, logits));
             BEAM_CUDA(launch_first_output(logits, d_len, d_t, K, W, NV, m.blank_id, K, d_top_label, d_top_jump, d_top_logp, st));
-            BEAM_CUDA(cudaMemcpyAsync(top_label.data(), d_top_label, sizeof(int32_t) * K * K, cudaMemcpyDeviceToHost, st));
-            BEAM_CUDA(cudaMemcpyAsync(top_jump.data(), d_top_jump, sizeof(int32_t) * K * K, cudaMemcpyDeviceToHost, st));
-            BEAM_CUDA(cudaMemcpyAsync(top_logp.data(), d_top_logp, sizeof(float) * K * K, cudaMemcpyDeviceToHost, st));
+            BEAM_CUDA(cudaMemcpyAsync(top.data(), d_top_label, sizeof(int32_t) * 3 * K * K, cudaMemcpyDeviceToHost, st));
             BEAM_CUDA(cudaStreamSynchronize(st));
             // ---- expansions ----
             for (int b = 0; b < nh; ++b) {
@@ -228,15 +246,18 @@ wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyp
                     nhyp.score = h.score + (double)lp;
                     if (label != m.blank_id) {
                         int tt = t + jump;
-                        nhyp.tok = h.tok; nhyp.frm = h.frm;
-                        nhyp.tok.push_back(label); nhyp.frm.push_back(tt);
+                        Node nd;
+                        nd.parent = h.node; nd.tok = label; nd.frm = tt; nd.len = node_len(h.node) + 1;
+                        nd.hash = (node_hash(h.node) ^ (uint64_t)(uint32_t)label) * 0x100000001B3ull + 0x9E3779B97F4A7C15ull;
+                        nodes.push_back(nd);
+                        nhyp.node = (int32_t)nodes.size() - 1;
                         nhyp.count = jump == 0 ? h.count + 1 : 1;
                         nhyp.parent = h.slot;
                         refs[h.slot]++;
                         if (nhyp.count == S) { tt += 1; nhyp.count = 0; }
                         t2hyps[tt].push_back(std::move(nhyp));
                     } else {
-                        nhyp.tok = h.tok; nhyp.frm = h.frm;
+                        nhyp.node = h.node;
                         nhyp.count = 0;
                         nhyp.slot = h.slot;
                         refs[h.slot]++;
@@ -252,11 +273,16 @@ wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyp
     int n_out = 0;
     for (size_t a = 0; a < fin.size() && (int)a < max_hyps; ++a) {
         const Hyp& h = fin[a];
-        out_len[a] = (int32_t)h.tok.size();
+        const int len = node_len(h.node);
+        out_len[a] = len;
         out_score[a] = h.score;
-        for (size_t k = 0; k < h.tok.size() && (int)k < max_out; ++k) {
-            out_tokens[a * (size_t)max_out + k] = h.tok[k];
-            out_frames[a * (size_t)max_out + k] = h.frm[k];
+        int32_t nd = h.node;
+        for (int k = len - 1; k >= 0; --k) {   // walk the history back from the last token
+            if (k < max_out) {
+                out_tokens[a * (size_t)max_out + k] = nodes[(size_t)nd].tok;
+                out_frames[a * (size_t)max_out + k] = nodes[(size_t)nd].frm;
+            }
+            nd = nodes[(size_t)nd].parent;
         }
         ++n_out;
     }

@@ -333,13 +333,66 @@ static cudaError_t simt_joint_t(const Call& c, float* logits_out) {
     return cudaGetLastError();
 }
 
-// Beam search: the rows are hypotheses of ONE utterance; a frame stride of zero makes every block read utterance 0.
+// Beam search: the rows are hypotheses of ONE utterance (all read utterance 0's enc_proj rows), there are only a few
+// of them, and only the logits are wanted (Eq. (1) is a pass of its own): one block per (vocabulary slice of 64,
+// hypothesis), so that the joint of a handful of hypotheses still spreads over the SMs.
+template <typename TW>
+__global__ void __launch_bounds__(256) joint_logits_shared_kernel(const int32_t* __restrict__ t_cur, const int32_t* __restrict__ enc_len,
+                                                                  const TW* __restrict__ enc_proj, const float* __restrict__ pred_proj,
+                                                                  const TW* __restrict__ w_out, const float* __restrict__ b_out,
+                                                                  float* __restrict__ logits_out, int W, int H, int NV, int act) {
+    extern __shared__ float z[];  // [8][H]
+    const int b = blockIdx.y;
+    const int t = t_cur[b], len = enc_len[b];
+    if (t >= len) return;
+    const int n = min(W, len - t);
+    const int v0 = blockIdx.x * 64, v1 = min(NV, v0 + 64);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    for (int w0 = 0; w0 < n; w0 += 8) {
+        const int nc = min(8, n - w0);
+        __syncthreads();
+        for (int e = threadIdx.x; e < nc * H; e += blockDim.x) {
+            const int w = e / H, k = e - w * H;
+            float s = ldf(enc_proj + (size_t)(t + w0 + w) * H + k) + pred_proj[(size_t)b * H + k];
+            s = act == WIND_ACT_RELU ? fmaxf(s, 0.f) : tanhf(s);
+            z[e] = round_like<TW>(s);
+        }
+        __syncthreads();
+        for (int v = v0 + warp; v < v1; v += nw) {
+            float a[8];
+#pragma unroll
+            for (int w = 0; w < 8; ++w) a[w] = 0.f;
+            for (int k = lane; k < H; k += 32) {
+                const float wv = ldf(w_out + (size_t)v * H + k);
+#pragma unroll
+                for (int w = 0; w < 8; ++w)
+                    if (w < nc) a[w] = fmaf(wv, z[w * H + k], a[w]);
+            }
+#pragma unroll
+            for (int w = 0; w < 8; ++w) {
+                if (w < nc) {
+                    const float s = warp_sum(a[w]) + b_out[v];
+                    if (lane == 0) logits_out[((size_t)b * W + w0 + w) * NV + v] = s;
+                }
+            }
+        }
+    }
+}
+
+template <typename TW>
+static cudaError_t simt_joint_shared_t(const Call& c, float* logits_out) {
+    const size_t smem = sizeof(float) * 8 * (size_t)c.m.H;
+    if (smem > 48 * 1024) cudaFuncSetAttribute(joint_logits_shared_kernel<TW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    dim3 grid((unsigned)((c.m.V + 1 + 63) / 64), (unsigned)c.B);
+    joint_logits_shared_kernel<TW><<<grid, 256, smem, c.stream>>>(c.t(), c.enc_len, (const TW*)c.enc_proj(), c.pred_proj(),
+                                                                  (const TW*)c.m.w_out, c.m.b_out, logits_out, c.W, c.m.H,
+                                                                  c.m.V + 1, c.m.act);
+    return cudaGetLastError();
+}
+
 cudaError_t simt_joint_shared(const Call& c, float* logits_out) {
-    Call one = c;
-    one.T = 0;
-    one.mode = WIND_MODE_FIRST_NONBLANK;
-    if (c.m.dtype == WIND_DT_BF16) return simt_joint_t<__nv_bfloat16, false>(one, logits_out);
-    return simt_joint_t<float, false>(one, logits_out);
+    if (c.B == 0) return cudaSuccess;
+    return c.m.dtype == WIND_DT_BF16 ? simt_joint_shared_t<__nv_bfloat16>(c, logits_out) : simt_joint_shared_t<float>(c, logits_out);
 }
 
 cudaError_t simt_joint(const Call& c, float* logits_out) {
