@@ -25,7 +25,9 @@
  * The file also holds Eq. (1) (first-output distribution of a window) and window-based greedy decoding, which
  * takes the most probable (label, offset) pair of Eq. (1) at every step; their pins: the distribution sums to
  * one, closed forms, W = 1 equals Algorithm 1, a step-by-step recomputation from Eq. (1) in the tests, and a
- * hand-worked example where it differs from Algorithm 2.
+ * hand-worked example where it differs from Algorithm 2; and Algorithm 3 (beam search for one utterance), pinned
+ * by: beam 1 equals window-based greedy decoding, an unpruned beam gives every token sequence its total probability
+ * over all alignments for every window (brute force on independently evaluated logits), and a hand-worked example.
  *
  * Pins (see tests): WIND(W) == sequential for every W; brute-force tabulation
  * of joint argmaxes on tiny models; LSTM / linear layers against library fp64
