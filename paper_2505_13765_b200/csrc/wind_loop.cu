@@ -1712,7 +1712,9 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
             if (found) break;
         }
         if (found) {
-            const uint32_t staging = 17408;
+            // epilogue staging: 64 utterances x 4 gates x 16 units (+ their tokens) in the decoder phase, np utterances x
+            // (64 + 4 padding) pred_proj values in the projection phase
+            const uint32_t staging = r.np > 64 ? (uint32_t)r.np * 68u * 4u : 17408u;
             const uint32_t tile = (uint32_t)r.kb_p * 64u * BK * 2u;
             uint32_t buf = (uint32_t)r.nj * (uint32_t)m.H * 2u;
             if ((uint32_t)r.nl * m.P * 2u > buf) buf = (uint32_t)r.nl * m.P * 2u;

@@ -263,6 +263,7 @@ def test_bf16_tensor_path_more_utterances_than_one_tile(pkg, monkeypatch, reside
     (300, 2, 3, 64, 64, 130, 1),
     (40, 32, 4, 128, 64, 500, 2),
     (148, 4, 3, 256, 256, 1000, 2),
+    (129, 2, 2, 256, 128, 152, 2),     # the resident plan takes 128 utterances per projection CTA
 ])
 @pytest.mark.parametrize("resident", [1, 0])
 def test_bf16_tensor_path_shape_sweep(pkg, monkeypatch, resident, B, W, S, P, H, V, L):
