@@ -100,8 +100,10 @@ def lib():
                                                   C.c_int32, i64p, i64p, i64p, i32p]
         L.oracle_replay_verify_window.restype = C.c_int32
         L.oracle_beam_search.argtypes = [mp, f32p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
-                                         i32p, i32p, i32p, f64p, f64p, i64p]
+                                         C.c_int32, i32p, i32p, i32p, f64p, f64p, i64p]
         L.oracle_beam_search.restype = C.c_int32
+        L.oracle_beam_prefix_step.argtypes = [mp, f32p, C.c_int32, C.c_int32, i32p, i32p, f64p, i32p]
+        L.oracle_beam_prefix_step.restype = None
     return _lib
 
 
@@ -185,7 +187,7 @@ def decode_window_greedy_batch(model: Model, enc: np.ndarray, enc_len: np.ndarra
 
 
 def beam_search(model: Model, enc_b: np.ndarray, T: int, W: int, K: int, S: int, max_hyps: int = 64,
-                max_out: Optional[int] = None):
+                max_out: Optional[int] = None, prefix_search: bool = False):
     """Algorithm 3 for one utterance.  Returns (list of (tokens, frames, score) most probable first, min_gap, steps)."""
     enc_b = _f32(enc_b)
     if max_out is None:
@@ -196,12 +198,29 @@ def beam_search(model: Model, enc_b: np.ndarray, T: int, W: int, K: int, S: int,
     sc = np.zeros(max_hyps, np.float64)
     gap = C.c_double(0.0)
     steps = C.c_int64(0)
-    n = lib().oracle_beam_search(model.ref, _ptr(enc_b, f32p), int(T), int(W), int(K), int(S), max_hyps, max_out,
+    n = lib().oracle_beam_search(model.ref, _ptr(enc_b, f32p), int(T), int(W), int(K), int(S), int(bool(prefix_search)),
+                                 max_hyps, max_out,
                                  _ptr(tok, i32p), _ptr(frm, i32p), _ptr(ln, i32p), _ptr(sc, f64p), C.byref(gap),
                                  C.byref(steps))
     assert n >= 0
     hyps = [(tok[a, : ln[a]].copy(), frm[a, : ln[a]].copy(), float(sc[a])) for a in range(n)]
     return hyps, gap.value, steps.value
+
+
+def beam_prefix_step(model: Model, enc_t: np.ndarray, hyps: Sequence[Sequence[int]], scores: Sequence[float]):
+    """Step (2) of Algorithm 3's recombination on its own.  Returns (new scores, removed flags)."""
+    enc_t = _f32(enc_t)
+    n = len(hyps)
+    ml = max(1, max((len(h) for h in hyps), default=1))
+    tok = np.zeros((n, ml), np.int32)
+    for i, h in enumerate(hyps):
+        tok[i, : len(h)] = h
+    lens = np.array([len(h) for h in hyps], np.int32)
+    sc = np.array(scores, np.float64)
+    gone = np.zeros(n, np.int32)
+    lib().oracle_beam_prefix_step(model.ref, _ptr(enc_t, f32p), n, ml, _ptr(tok, i32p), _ptr(lens, i32p), _ptr(sc, f64p),
+                                  _ptr(gone, i32p))
+    return sc, gone.astype(bool)
 
 
 def replay_verify_window(model: Model, enc_b: np.ndarray, T: int, W: int, S: int, tokens: np.ndarray,

@@ -629,8 +629,8 @@ int32_t oracle_replay_verify_window(const oracle_model_t* m, const float* enc, i
  * states are equal).  Two hypotheses with the same tokens but different counts of emissions on the current frame
  * are NOT the same under the safeguard (they may continue differently), so they stay apart: with this reading a beam
  * that never prunes gives every token sequence its total probability over all alignments, for every window;
- * (3) the K most probable stay.  Step (2), moving the mass of a hypothesis A into a
- * longer B that A is a prefix of, is NOT part of this function.
+ * (3) the K most probable stay.  Step (2), moving the mass of a hypothesis A into a longer B that A is a prefix
+ * of, is optional (prefix_search != 0): see beam_prefix_step.
  * Order conventions: entries of P' are ranked by log-probability, then offset, then label; new hypotheses are
  * appended in the order (hypothesis, rank); duplicates merge into their first occurrence; pruning is a stable sort.
  * Safeguard against staying on one frame (the paper omits its details): the rule of the greedy decoders above;
@@ -684,7 +684,11 @@ static double log_add(double a, double b) {
 static void note_gap(double* min_gap, double g) { if (g >= 0 && g < *min_gap) *min_gap = g; }
 
 /* duplicates -> one (probabilities summed), then the K most probable, stable; freed hypotheses are released */
-static void beam_recombine_prune(beam_list_t* l, int K, double* min_gap) {
+static void beam_prefix_step(const oracle_model_t* m, const double* encp_t, beam_list_t* l);
+
+/* prefix_ctx_m == NULL: steps (1) and (3) only */
+static void beam_recombine_prune(beam_list_t* l, int K, double* min_gap, const oracle_model_t* prefix_ctx_m,
+                                 const double* encp_t) {
     for (int a = 0; a < l->n; ++a) {
         for (int b = a + 1; b < l->n;) {
             beam_hyp_t *x = l->v[a], *y = l->v[b];
@@ -700,6 +704,7 @@ static void beam_recombine_prune(beam_list_t* l, int K, double* min_gap) {
             }
         }
     }
+    if (prefix_ctx_m) beam_prefix_step(prefix_ctx_m, encp_t, l);
     for (int a = 1; a < l->n; ++a) {   /* stable insertion sort, most probable first */
         beam_hyp_t* x = l->v[a];
         int k = a;
@@ -713,9 +718,58 @@ static void beam_recombine_prune(beam_list_t* l, int K, double* min_gap) {
     }
 }
 
+/*
+ * Step (2) of recombine_prune as the paper states it: for all pairs (A, B) of the list where A's tokens are a proper
+ * prefix of B's, the probability of completing A into B by emitting B's extra tokens at the current frame t,
+ *     P(A) * prod_i P(b_i | frame t, decoder state after A + b_<i),
+ * is added to B; then every such A is removed.  Every completion uses the probabilities the hypotheses had when the
+ * step began, so the result does not depend on the order of the pairs.  (The details are in a cited paper that is
+ * not at hand; this is the sentence of the paper, taken literally.)
+ */
+static void beam_prefix_step(const oracle_model_t* m, const double* encp_t, beam_list_t* l) {
+    const int n = l->n, NV = m->V + 1;
+    if (n < 2) return;
+    double* add = (double*)malloc(sizeof(double) * (size_t)n);
+    int* gone = (int*)calloc((size_t)n, sizeof(int));
+    const size_t ns = (size_t)m->L * m->P;
+    double* h = (double*)malloc(sizeof(double) * ns);
+    double* c = (double*)malloc(sizeof(double) * ns);
+    double* g = (double*)malloc(sizeof(double) * (size_t)m->H);
+    double* z = (double*)malloc(sizeof(double) * (size_t)m->H);
+    double* row = (double*)malloc(sizeof(double) * (size_t)NV);
+    for (int b = 0; b < n; ++b) add[b] = -INFINITY;
+    for (int a = 0; a < n; ++a)
+        for (int b = 0; b < n; ++b) {
+            const beam_hyp_t *A = l->v[a], *B = l->v[b];
+            if (a == b || A->len >= B->len || memcmp(A->tok, B->tok, sizeof(int32_t) * (size_t)A->len) != 0) continue;
+            memcpy(h, A->h, sizeof(double) * ns); memcpy(c, A->c, sizeof(double) * ns);
+            memcpy(g, A->g, sizeof(double) * (size_t)m->H);
+            double acc = A->score;
+            for (int i = A->len; i < B->len; ++i) {
+                oracle_joint_logits(m, encp_t, g, z, row);
+                double mx = row[0];
+                for (int v = 1; v < NV; ++v) if (row[v] > mx) mx = row[v];
+                double se = 0.0;
+                for (int v = 0; v < NV; ++v) se += exp(row[v] - mx);
+                acc += row[B->tok[i]] - (mx + log(se));
+                if (i + 1 < B->len) { oracle_lstm_step(m, B->tok[i], h, c); oracle_pred_proj(m, h, g); }
+            }
+            add[b] = log_add(add[b], acc);
+            gone[a] = 1;
+        }
+    for (int b = 0; b < n; ++b) l->v[b]->score = log_add(l->v[b]->score, add[b]);
+    int k = 0;
+    for (int a = 0; a < n; ++a) {
+        if (gone[a]) beam_free(l->v[a]); else l->v[k++] = l->v[a];
+    }
+    l->n = k;
+    free(row); free(z); free(g); free(c); free(h); free(gone); free(add);
+}
+
 int32_t oracle_beam_search(const oracle_model_t* m, const float* enc, int32_t T, int32_t W, int32_t K, int32_t S,
-                           int32_t max_hyps_out, int32_t max_out, int32_t* out_tokens, int32_t* out_frames,
-                           int32_t* out_len, double* out_score, double* min_gap_out, int64_t* n_steps_out) {
+                           int32_t prefix_search, int32_t max_hyps_out, int32_t max_out, int32_t* out_tokens,
+                           int32_t* out_frames, int32_t* out_len, double* out_score, double* min_gap_out,
+                           int64_t* n_steps_out) {
     if (W < 1 || W > 64 || K < 1 || S < 1 || T < 0) return -1;
     const int NV = m->V + 1;
     double* encp = (double*)malloc(sizeof(double) * (size_t)(T > 0 ? T : 1) * m->H);
@@ -741,7 +795,7 @@ int32_t oracle_beam_search(const oracle_model_t* m, const float* enc, int32_t T,
         while (cur->n > 0) {   /* a frame is taken again when an expansion stays on it (jump 0) */
             beam_list_t hyps = *cur;
             cur->v = NULL; cur->n = 0; cur->cap = 0;
-            beam_recombine_prune(&hyps, K, &min_gap);
+            beam_recombine_prune(&hyps, K, &min_gap, prefix_search ? m : NULL, encp + (size_t)t * m->H);
             const int n = (W < T - t) ? W : (T - t);
             steps++;
             for (int b = 0; b < hyps.n; ++b) {
@@ -792,7 +846,7 @@ int32_t oracle_beam_search(const oracle_model_t* m, const float* enc, int32_t T,
     }
     /* best_hyp_in(t2hyps[T]): duplicates merged, most probable first */
     beam_list_t* fin = &t2hyps[T];
-    beam_recombine_prune(fin, fin->n > 0 ? fin->n : 1, &min_gap);
+    beam_recombine_prune(fin, fin->n > 0 ? fin->n : 1, &min_gap, NULL, NULL);
     if (fin->n > 1) note_gap(&min_gap, fin->v[0]->score - fin->v[1]->score);
     int n_out = 0;
     for (int a = 0; a < fin->n; ++a) {
@@ -812,4 +866,37 @@ int32_t oracle_beam_search(const oracle_model_t* m, const float* enc, int32_t T,
     if (min_gap_out) *min_gap_out = min_gap;
     if (n_steps_out) *n_steps_out = steps;
     return n_out;
+}
+
+/*
+ * Test access to step (2) alone: n hypotheses given by their tokens (row-major [n, max_len], lengths) and
+ * log-probabilities at one encoder frame (enc_t [D]).  scores are updated in place, gone[i] = 1 for removed ones.
+ */
+void oracle_beam_prefix_step(const oracle_model_t* m, const float* enc_t, int32_t n, int32_t max_len, const int32_t* tokens,
+                             const int32_t* lens, double* scores, int32_t* gone) {
+    double* encp = (double*)malloc(sizeof(double) * (size_t)m->H);
+    oracle_enc_proj(m, enc_t, 1, encp);
+    beam_list_t l = {NULL, 0, 0};
+    const size_t ns = (size_t)m->L * m->P;
+    beam_hyp_t** all = (beam_hyp_t**)malloc(sizeof(beam_hyp_t*) * (size_t)(n > 0 ? n : 1));
+    for (int i = 0; i < n; ++i) {
+        beam_hyp_t* h = (beam_hyp_t*)calloc(1, sizeof(beam_hyp_t));
+        h->len = lens[i];
+        h->tok = (int32_t*)malloc(sizeof(int32_t) * (size_t)(lens[i] + 1));
+        h->frm = (int32_t*)calloc((size_t)(lens[i] + 1), sizeof(int32_t));
+        memcpy(h->tok, tokens + (size_t)i * max_len, sizeof(int32_t) * (size_t)lens[i]);
+        h->h = (double*)calloc(ns, sizeof(double)); h->c = (double*)calloc(ns, sizeof(double));
+        h->g = (double*)malloc(sizeof(double) * (size_t)m->H);
+        oracle_lstm_step(m, m->blank_id, h->h, h->c);
+        for (int k = 0; k < lens[i]; ++k) oracle_lstm_step(m, h->tok[k], h->h, h->c);
+        oracle_pred_proj(m, h->h, h->g);
+        h->score = scores[i];
+        h->count = i;   /* tag: the position in the input, to find the survivors again */
+        beam_push(&l, h);
+        all[i] = h;
+    }
+    beam_prefix_step(m, encp, &l);
+    for (int i = 0; i < n; ++i) gone[i] = 1;
+    for (int k = 0; k < l.n; ++k) { gone[l.v[k]->count] = 0; scores[l.v[k]->count] = l.v[k]->score; beam_free(l.v[k]); }
+    free(l.v); free(all); free(encp);
 }

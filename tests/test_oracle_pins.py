@@ -645,3 +645,57 @@ def test_beam_search_worked_example_beats_greedy():
     one, _, _ = oracle.beam_search(m, enc, 2, 2, 1, 1)
     assert list(one[0][0]) == [0, 1] and abs(one[0][2] - np.log(.36)) < 1e-6
     assert abs(gap - 0.0) < 1e-6      # the x / blank tie is reported as a zero gap
+
+
+def test_beam_prefix_step_matches_an_independent_evaluation():
+    # completing A into B at one frame: P(A) * prod_i P(b_i | frame, decoder after A + b_<i), from the independent
+    # evaluator (whole-prefix LSTM re-run, library log-softmax); every proper prefix is removed
+    r = rng(970)
+    w = random_weights(r, 5, 4, 6, 2, 7, 6, act=1, blank_bias=0.5, bias_scale=0.1)
+    nm = NaiveModel(w)
+    enc_t = r.standard_normal(5).astype(np.float32)
+    hyps = [[1, 2], [1, 2, 3, 0], [1], [4, 4], [1, 2, 5], []]
+    scores = [-1.0, -3.5, -0.7, -2.0, -2.5, -4.0]
+
+    def completion(a, b):
+        acc = scores[a]
+        for i in range(len(hyps[a]), len(hyps[b])):
+            lp = torch.log_softmax(torch.tensor(nm.logits(enc_t, hyps[b][:i])), dim=0).numpy()
+            acc += lp[hyps[b][i]]
+        return acc
+
+    want = list(scores)
+    removed = [False] * len(hyps)
+    for a in range(len(hyps)):
+        for b in range(len(hyps)):
+            if a != b and len(hyps[a]) < len(hyps[b]) and hyps[b][: len(hyps[a])] == hyps[a]:
+                want[b] = np.logaddexp(want[b], completion(a, b))
+                removed[a] = True
+    got, gone = oracle.beam_prefix_step(oracle.Model(w), enc_t, hyps, scores)
+    assert list(gone) == removed == [True, False, True, False, False, True]
+    for b in range(len(hyps)):
+        if not removed[b]:
+            assert abs(got[b] - want[b]) < 1e-9
+
+
+def test_beam_search_with_prefix_step_worked_example():
+    # frame types A = (x .45, y .05, blank .5), B = (x .1, y .8, blank .1); utterance A B, W = 1, S = 2, K = 2.
+    # t = 0, []: x .45 -> [x] stays on frame 0; blank .5 -> [] goes to frame 1.
+    # t = 0 again, [x]: x .45 -> [x,x] .2025, second emission on the frame: forced to frame 1; blank .5 -> [x] .225 to frame 1.
+    # t = 1, {[] .5, [x,x] .2025, [x] .225}: [] is a prefix of both others, [x] of [x,x].  Completions at frame 1 (type B):
+    #     [] -> [x]: .5 * .1 = .05      [] -> [x,x]: .5 * .1 * .1 = .005      [x] -> [x,x]: .225 * .1 = .0225
+    #   [x,x] = .2025 + .005 + .0225 = .23; [] and [x] are removed (each is a prefix of something): one hypothesis is left.
+    #   [x,x]: y .8 -> [x,x,y] .184 stays; x .1 (label before blank on the tie) -> [x,x,x] .023 stays.
+    # t = 1 again: no prefix pair; every second emission is forced to T:
+    #   [x,x,y,y] .1472, [x,x,y,x] .0184, [x,x,x,y] .0184, [x,x,x,x] .0023.
+    w = table_model([[.45, .05, .5], [.1, .8, .1]])
+    enc = np.eye(2, dtype=np.float32)[[0, 1]]
+    m = oracle.Model(w)
+    pre, _, steps = oracle.beam_search(m, enc, 2, 1, 2, 2, prefix_search=True)
+    assert steps == 4
+    assert [list(h[0]) for h in pre] == [[0, 0, 1, 1], [0, 0, 1, 0], [0, 0, 0, 1], [0, 0, 0, 0]]
+    assert [list(h[1]) for h in pre] == [[0, 0, 1, 1]] * 4
+    assert np.allclose(np.exp([h[2] for h in pre]), [.1472, .0184, .0184, .0023], atol=1e-6)
+    # without the step the beam at t = 1 is {[] .5, [x] .225}: a different search
+    plain, _, _ = oracle.beam_search(m, enc, 2, 1, 2, 2)
+    assert abs(np.exp(plain[0][2]) - .1472) > 1e-3
