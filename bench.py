@@ -604,13 +604,13 @@ def beam_op(args, cfg, W):
     T = int(lens_np[b])
     enc = np.ascontiguousarray(enc_np[b, :T])
     model = pkg.WindModel(weights, device=dev)
-    for K in (2, 3, 4):
+    for K, prefix in ((2, False), (3, False), (4, False), (4, True)):
         for _ in range(2):
-            pkg.wind_beam_search(model, enc, W, K, cfg.S, max_hyps=8)
+            pkg.wind_beam_search(model, enc, W, K, cfg.S, max_hyps=8, prefix_search=prefix)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         for _ in range(args.steps):
-            hyps, steps, st = pkg.wind_beam_search(model, enc, W, K, cfg.S, max_hyps=8)
+            hyps, steps, st = pkg.wind_beam_search(model, enc, W, K, cfg.S, max_hyps=8, prefix_search=prefix)
         torch.cuda.synchronize()
         dt = (time.perf_counter() - t0) / args.steps
         cb = None
@@ -618,7 +618,7 @@ def beam_op(args, cfg, W):
             import oracle
             Tc = min(T, 24)
             t1 = time.perf_counter()
-            _, _, osteps = oracle.beam_search(oracle.Model(weights), enc[:Tc], Tc, W, K, cfg.S)
+            _, _, osteps = oracle.beam_search(oracle.Model(weights), enc[:Tc], Tc, W, K, cfg.S, prefix_search=prefix)
             od = time.perf_counter() - t1
             cb = dict(value=Tc * FRAME_SECONDS / od, unit="audio-s/s", cores=1, kind="oracle",
                       sample=f"first {Tc} frames of the utterance, {osteps} iterations, one run, {od:.1f} s")
@@ -626,7 +626,7 @@ def beam_op(args, cfg, W):
             "metric": "WIND beam search RTFx, one utterance (audio-s/s at 80 ms/frame)", "op": "beam", "value": T * FRAME_SECONDS / dt,
             "unit": "audio-s/s", "n_gpus": 1, "steps": args.steps, "warmup": 2, "ms_per_step": dt * 1e3, "higher_is_better": True,
             "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": cfg.name, "utterance": b, "frames": T, "W": W, "K": K, "max_symbols": cfg.S},
+            "config": {"workload": cfg.name, "utterance": b, "frames": T, "W": W, "K": K, "max_symbols": cfg.S, "prefix_search": prefix},
             "iterations": steps, "us_per_iteration": dt * 1e6 / max(1, steps), "best_tokens": int(len(hyps[0][0])),
             "best_score": hyps[0][2], "final_hypotheses": len(hyps), "cpu_baseline": cb,
         }))

@@ -262,8 +262,13 @@ wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const 
  * offset: appended, continues at t + offset; the blank entry: continues at t + n).  The most probable hypotheses
  * that reached frame T are returned, best first.
  * Recombination: hypotheses with the same tokens (and the same count of emissions on the current frame) become one
- * with their probabilities summed; then the K most probable stay.  The transfer of probability from a hypothesis to
- * a longer one that it is a prefix of (the cited prefix search) is not part of this function.
+ * with their probabilities summed; then the K most probable stay.  prefix_search != 0 adds the step between the
+ * two as the paper states it: for every pair (A, B) of the frame's hypotheses with A's tokens a proper prefix of B's,
+ * P(A) times the probability of emitting B's extra tokens at the current frame (each under the decoder state after
+ * the tokens before it) is added to B, then every such A is removed; completions use the probabilities the
+ * hypotheses had when the step began.  (The paper refers to another paper for the details of this step; what is
+ * built is its own sentence, taken literally.  It costs one more round of kernels and one synchronisation per extra
+ * token and K pairs.)
  * max_symbols: as in wind_decode_greedy (the paper leaves its safeguard for this algorithm to its code).
  * Entries of P' are ranked by probability, then offset, then label.  Scores are natural-log probabilities; the
  * window's log-softmax is fp32, sums over steps are fp64.  K = 1 gives wind_decode_window_greedy's result.
@@ -281,7 +286,8 @@ wind_status_t wind_profile_decode(const wind_model_t* m, const void* enc, const 
 wind_status_t wind_beam_workspace_bytes(const wind_model_t* m, int32_t T, int32_t W, int32_t K, int32_t max_symbols,
                                         size_t* bytes);
 wind_status_t wind_beam_search(const wind_model_t* m, const void* enc, int32_t T, int32_t W, int32_t K,
-                               int32_t max_symbols, int32_t max_hyps, int32_t max_out, int32_t* out_tokens_host,
+                               int32_t max_symbols, int32_t prefix_search, int32_t max_hyps, int32_t max_out,
+                               int32_t* out_tokens_host,
                                int32_t* out_frames_host, int32_t* out_len_host, double* out_score_host,
                                int32_t* n_hyps_host, int64_t* n_steps_host, void* workspace, size_t workspace_bytes,
                                void* stream);

@@ -108,7 +108,7 @@ def load_library():
     L.wind_eval_joint_window_static.restype = i32
     L.wind_beam_workspace_bytes.argtypes = [mp, i32, i32, i32, i32, C.POINTER(C.c_size_t)]
     L.wind_beam_workspace_bytes.restype = i32
-    L.wind_beam_search.argtypes = [mp, _vp, i32, i32, i32, i32, i32, i32, _vp, _vp, _vp, _vp, C.POINTER(i32),
+    L.wind_beam_search.argtypes = [mp, _vp, i32, i32, i32, i32, i32, i32, i32, _vp, _vp, _vp, _vp, C.POINTER(i32),
                                    C.POINTER(C.c_int64), _vp, C.c_size_t, _vp]
     L.wind_beam_search.restype = i32
     L.wind_plan_batches.argtypes = [_vp, i32, i32, _vp, _vp, C.POINTER(i32)]
@@ -399,7 +399,7 @@ def to_device_enc(model: WindModel, enc_np: np.ndarray):
 
 
 def wind_beam_search(model: WindModel, enc_np: np.ndarray, W: int, K: int, S: int, max_hyps: int = 64,
-                     max_out: Optional[int] = None, check: bool = True):
+                     max_out: Optional[int] = None, check: bool = True, prefix_search: bool = False):
     """Algorithm 3 for one utterance [T, D] (numpy).  Returns (list of (tokens, frames, score) best first, steps, status)."""
     torch = _torch()
     L = load_library()
@@ -420,7 +420,8 @@ def wind_beam_search(model: WindModel, enc_np: np.ndarray, W: int, K: int, S: in
     ln = np.zeros(max_hyps, np.int32)
     sc = np.zeros(max_hyps, np.float64)
     nh, steps = C.c_int32(0), C.c_int64(0)
-    st = L.wind_beam_search(model.ref, enc.data_ptr(), T, W, K, S, max_hyps, max_out, tok.ctypes.data, frm.ctypes.data,
+    st = L.wind_beam_search(model.ref, enc.data_ptr(), T, W, K, S, int(bool(prefix_search)), max_hyps, max_out,
+                            tok.ctypes.data, frm.ctypes.data,
                             ln.ctypes.data, sc.ctypes.data, C.byref(nh), C.byref(steps), ws.data_ptr() + off, n.value,
                             _stream_ptr(None))
     if check and st != WIND_OK:

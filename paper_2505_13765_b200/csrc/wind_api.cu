@@ -531,7 +531,7 @@ wind_status_t wind_beam_workspace_bytes(const wind_model_t* m, int32_t T, int32_
 }
 
 wind_status_t wind_beam_search(const wind_model_t* m, const void* enc, int32_t T, int32_t W, int32_t K, int32_t max_symbols,
-                               int32_t max_hyps, int32_t max_out, int32_t* out_tokens_host, int32_t* out_frames_host,
+                               int32_t prefix_search, int32_t max_hyps, int32_t max_out, int32_t* out_tokens_host, int32_t* out_frames_host,
                                int32_t* out_len_host, double* out_score_host, int32_t* n_hyps_host, int64_t* n_steps_host,
                                void* workspace, size_t workspace_bytes, void* stream) {
     wind_status_t s = check_beam_args(m, T, W, K, max_symbols);
@@ -547,7 +547,7 @@ wind_status_t wind_beam_search(const wind_model_t* m, const void* enc, int32_t T
     const BeamLayout bl = make_beam_layout(*m, T, W, K, max_symbols, cb.lay.total);
     if (workspace_bytes < bl.total) return WIND_ERR_WORKSPACE;
     cudaError_t ce = cudaSuccess;
-    s = beam_search_run(cb, bl, K, max_hyps, max_out, out_tokens_host, out_frames_host, out_len_host, out_score_host,
+    s = beam_search_run(cb, bl, K, prefix_search != 0, max_hyps, max_out, out_tokens_host, out_frames_host, out_len_host, out_score_host,
                         n_hyps_host, n_steps_host, &ce);
     if (s == WIND_ERR_CUDA) return cuda_fail(ce, "beam search");
     return s;

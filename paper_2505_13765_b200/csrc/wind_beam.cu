@@ -61,6 +61,12 @@ __global__ void beam_gather_g_kernel(const float* __restrict__ g_pool, const int
     for (int k = threadIdx.x; k < H; k += blockDim.x) pred_proj[(size_t)b * H + k] = g_pool[(size_t)s * H + k];
 }
 
+// log-probability of one label per row, from a [B][NV] table of log-softmax values (rows without a label: untouched)
+__global__ void beam_pick_kernel(const float* __restrict__ logp, const int32_t* __restrict__ label, float* __restrict__ out, int B, int NV) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B && label[b] >= 0) out[b] = logp[(size_t)b * NV + label[b]];
+}
+
 __global__ void beam_fill_kernel(int32_t* a, int n, int v) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) a[i] = v;
@@ -109,7 +115,7 @@ BeamLayout make_beam_layout(const wind_model_t& m, int T, int W, int K, int S, s
 
 // cb: a call bundle with B = K rows (the beam), T, W, S of the utterance, enc = the utterance's frames [T, D];
 // its enc_len / out_len pointers are set here.  Outputs are HOST arrays.
-wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyps, int max_out, int32_t* out_tokens,
+wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int prefix_search, int max_hyps, int max_out, int32_t* out_tokens,
                               int32_t* out_frames, int32_t* out_len, double* out_score, int32_t* n_hyps, int64_t* n_steps,
                               cudaError_t* cuda_err) {
     const wind_model_t& m = cb.m;
@@ -158,7 +164,6 @@ wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyp
     const int32_t* top_jump = top.data() + (size_t)K * K;
     const float* top_logp = reinterpret_cast<const float*>(top.data() + 2 * (size_t)K * K);
     int64_t steps = 0;
-    bool first = true;
 
     std::vector<Node> nodes;
     auto node_len = [&](int32_t n) { return n < 0 ? 0 : nodes[(size_t)n].len; };
@@ -172,7 +177,129 @@ wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyp
         }
         return true;
     };
-    auto recombine_prune = [&](std::vector<Hyp>& l, size_t keep) {
+    int32_t *d_pick = ints + 7 * K;
+    // decoder update of up to K (parent slot, token) pairs into fresh slots; the parents' references are released
+    auto run_update = [&](int nu) -> cudaError_t {   // host_ints [0..K) src, [K..2K) tokens, [2K..3K) dst are filled
+        cudaError_t e = cudaMemcpyAsync(ints, host_ints.data(), sizeof(int32_t) * 3 * K, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return e;
+        beam_gather_kernel<<<K, 128, 0, st>>>(h_pool, c_pool, d_src, d_tok, cb.h(0), cb.c(), cb.emit_tok(), K, m.L, m.P);
+        if ((e = simt_pred_step(cb, 0)) != cudaSuccess) return e;
+        beam_scatter_kernel<<<K, 128, 0, st>>>(cb.h(1), cb.c(), cb.pred_proj(), d_dst, h_pool, c_pool, g_pool, K, m.L, m.P, m.H);
+        for (int u = 0; u < nu; ++u) release(host_ints[u]);
+        return cudaGetLastError();
+    };
+    auto take_slot = [&]() -> int {
+        if (free_slots.empty()) return -1;
+        const int s = free_slots.back();
+        free_slots.pop_back();
+        refs[s] = 1;
+        return s;
+    };
+    // Step (2) of the recombination as the paper states it: for every pair (A, B) of the list with A's tokens a proper
+    // prefix of B's, P(A) * prod_i P(b_i | frame t, decoder after A + b_<i) is added to B, then every such A is removed.
+    // The per-label probabilities come from the same kernels as the expansion (one-row window at frame t), K pairs at a
+    // time, one round per extra token; completions use the probabilities the hypotheses had when the step began.
+    struct Pair { int a, b, cur; std::vector<int32_t> extra; double acc; };
+    auto prefix_step = [&](std::vector<Hyp>& l, int t) -> wind_status_t {
+        const int n = (int)l.size();
+        if (n < 2) return WIND_OK;
+        std::vector<Pair> pairs;
+        for (int a = 0; a < n; ++a)
+            for (int b = 0; b < n; ++b) {
+                const int la = node_len(l[a].node), lb = node_len(l[b].node);
+                if (a == b || la >= lb) continue;
+                std::vector<int32_t> extra((size_t)(lb - la));
+                int32_t x = l[b].node;
+                for (int k = lb - la - 1; k >= 0; --k) { extra[(size_t)k] = nodes[(size_t)x].tok; x = nodes[(size_t)x].parent; }
+                if (!same_tokens(l[a].node, x)) continue;
+                pairs.push_back(Pair{a, b, -1, std::move(extra), l[a].score});
+            }
+        if (pairs.empty()) return WIND_OK;
+        // the prefixes need their decoder state now
+        std::vector<char> is_prefix((size_t)n, 0);
+        for (const Pair& p : pairs) is_prefix[(size_t)p.a] = 1;
+        for (int a0 = 0; a0 < n;) {
+            int nu = 0;
+            for (int b = 0; b < K; ++b) { host_ints[b] = -1; host_ints[K + b] = -1; host_ints[2 * K + b] = -1; }
+            for (; a0 < n && nu < K; ++a0) {
+                Hyp& h = l[(size_t)a0];
+                if (!is_prefix[(size_t)a0] || h.slot >= 0) continue;
+                const int s = take_slot();
+                if (s < 0) return WIND_ERR_WORKSPACE;
+                host_ints[nu] = h.parent;
+                host_ints[K + nu] = h.node < 0 ? m.blank_id : nodes[(size_t)h.node].tok;
+                host_ints[2 * K + nu] = s;
+                h.slot = s;
+                ++nu;
+            }
+            if (nu > 0) BEAM_CUDA(run_update(nu));
+        }
+        for (Pair& p : pairs) { p.cur = l[(size_t)p.a].slot; refs[p.cur]++; }
+        std::vector<float> picked((size_t)K);
+        size_t depth = 0;
+        for (bool more = true; more; ++depth) {
+            more = false;
+            std::vector<size_t> act;
+            for (size_t i = 0; i < pairs.size(); ++i)
+                if (pairs[i].extra.size() > depth) act.push_back(i);
+            for (size_t c0 = 0; c0 < act.size(); c0 += (size_t)K) {
+                const int nr = (int)std::min((size_t)K, act.size() - c0);
+                // log-softmax at frame t under each pair's current state, and the extra token's entry
+                for (int b = 0; b < K; ++b) { host_ints[3 * K + b] = -1; host_ints[b] = -1; host_ints[K + b] = -1; host_ints[2 * K + b] = -1; }
+                std::vector<int32_t> labels((size_t)K, -1);
+                for (int r = 0; r < nr; ++r) {
+                    Pair& p = pairs[act[c0 + (size_t)r]];
+                    host_ints[3 * K + r] = p.cur;
+                    labels[(size_t)r] = p.extra[depth];
+                }
+                BEAM_CUDA(cudaMemcpyAsync(d_exp, host_ints.data() + 3 * K, sizeof(int32_t) * K, cudaMemcpyHostToDevice, st));
+                BEAM_CUDA(cudaMemcpyAsync(d_pick, labels.data(), sizeof(int32_t) * K, cudaMemcpyHostToDevice, st));
+                beam_gather_g_kernel<<<K, 128, 0, st>>>(g_pool, d_exp, cb.pred_proj(), d_t, t, T, m.H);
+                BEAM_CUDA(launch_set_t(cb, d_t));
+                Call one = cb;
+                one.W = 1;
+                BEAM_CUDA(simt_joint_shared(one, logits));
+                BEAM_CUDA(launch_first_output(logits, d_len, d_t, K, 1, NV, m.blank_id, 0, nullptr, nullptr, nullptr, st));
+                beam_pick_kernel<<<1, 32, 0, st>>>(logits, d_pick, d_top_logp, K, NV);
+                BEAM_CUDA(cudaMemcpyAsync(picked.data(), d_top_logp, sizeof(float) * K, cudaMemcpyDeviceToHost, st));
+                BEAM_CUDA(cudaStreamSynchronize(st));
+                // one more decoder update for the pairs that have a further token
+                int nu = 0;
+                for (int r = 0; r < nr; ++r) {
+                    Pair& p = pairs[act[c0 + (size_t)r]];
+                    p.acc += (double)picked[(size_t)r];
+                    if (p.extra.size() > depth + 1) {
+                        const int s = take_slot();
+                        if (s < 0) return WIND_ERR_WORKSPACE;
+                        host_ints[nu] = p.cur;               // released by run_update
+                        host_ints[K + nu] = p.extra[depth];
+                        host_ints[2 * K + nu] = s;
+                        p.cur = s;
+                        ++nu;
+                        more = true;
+                    } else {
+                        release(p.cur);
+                        p.cur = -1;
+                    }
+                }
+                if (nu > 0) BEAM_CUDA(run_update(nu));
+            }
+        }
+        std::vector<double> add((size_t)n, -INFINITY);
+        for (const Pair& p : pairs) add[(size_t)p.b] = log_add(add[(size_t)p.b], p.acc);
+        std::vector<Hyp> kept;
+        for (int a = 0; a < n; ++a) {
+            if (is_prefix[(size_t)a]) {
+                release(l[(size_t)a].slot >= 0 ? l[(size_t)a].slot : l[(size_t)a].parent);
+            } else {
+                l[(size_t)a].score = log_add(l[(size_t)a].score, add[(size_t)a]);
+                kept.push_back(l[(size_t)a]);
+            }
+        }
+        l.swap(kept);
+        return WIND_OK;
+    };
+    auto merge_duplicates = [&](std::vector<Hyp>& l) {
         for (size_t a = 0; a < l.size(); ++a)
             for (size_t b = a + 1; b < l.size();) {
                 if (l[a].count == l[b].count && same_tokens(l[a].node, l[b].node)) {
@@ -185,6 +312,8 @@ wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyp
                     ++b;
                 }
             }
+    };
+    auto prune = [&](std::vector<Hyp>& l, size_t keep) {
         std::stable_sort(l.begin(), l.end(), [](const Hyp& x, const Hyp& y) { return x.score > y.score; });
         while (l.size() > keep) {
             release(l.back().slot >= 0 ? l.back().slot : l.back().parent);
@@ -196,7 +325,12 @@ wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyp
         while (!t2hyps[t].empty()) {
             std::vector<Hyp> hyps;
             hyps.swap(t2hyps[t]);
-            recombine_prune(hyps, (size_t)K);
+            merge_duplicates(hyps);
+            if (prefix_search) {
+                const wind_status_t ps = prefix_step(hyps, t);
+                if (ps != WIND_OK) return ps;
+            }
+            prune(hyps, (size_t)K);
             const int nh = (int)hyps.size();
             const int n = W < T - t ? W : T - t;
             ++steps;
@@ -211,25 +345,20 @@ wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyp
                     free_slots.pop_back();
                     refs[s] = 1;
                     host_ints[nu] = h.parent;
-                    host_ints[K + nu] = first ? m.blank_id : nodes[(size_t)h.node].tok;
+                    host_ints[K + nu] = h.node < 0 ? m.blank_id : nodes[(size_t)h.node].tok;
                     host_ints[2 * K + nu] = s;
                     h.slot = s;
                     ++nu;
                 }
             }
             for (int b = 0; b < nh; ++b) host_ints[3 * K + b] = hyps[b].slot;
-            BEAM_CUDA(cudaMemcpyAsync(ints, host_ints.data(), sizeof(int32_t) * 4 * K, cudaMemcpyHostToDevice, st));
+            BEAM_CUDA(cudaMemcpyAsync(d_exp, host_ints.data() + 3 * K, sizeof(int32_t) * K, cudaMemcpyHostToDevice, st));
             beam_gather_g_kernel<<<K, 128, 0, st>>>(g_pool, d_exp, cb.pred_proj(), d_t, t, T, m.H);   // sets the frames first
             BEAM_CUDA(launch_set_t(cb, d_t));   // frames of the rows, and the control block's "active" word
             if (nu > 0) {
-                beam_gather_kernel<<<K, 128, 0, st>>>(h_pool, c_pool, d_src, d_tok, cb.h(0), cb.c(), cb.emit_tok(), K, m.L, m.P);
-                BEAM_CUDA(simt_pred_step(cb, 0));
-                beam_scatter_kernel<<<K, 128, 0, st>>>(cb.h(1), cb.c(), cb.pred_proj(), d_dst, h_pool, c_pool, g_pool, K, m.L, m.P, m.H);
-                // the parents are no longer needed by these hypotheses
-                for (int u = 0; u < nu; ++u) release(host_ints[u]);
+                BEAM_CUDA(run_update(nu));   // (the parents are no longer needed by these hypotheses)
                 beam_gather_g_kernel<<<K, 128, 0, st>>>(g_pool, d_exp, cb.pred_proj(), d_t, t, T, m.H);
             }
-            first = false;
             // ---- window logits of every hypothesis, Eq. (1), the K best entries each ----
             BEAM_CUDA(simt_joint_shared(cb, logits));
             BEAM_CUDA(launch_first_output(logits, d_len, d_t, K, W, NV, m.blank_id, K, d_top_label, d_top_jump, d_top_logp, st));
@@ -269,7 +398,8 @@ wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyp
         }
     }
     std::vector<Hyp>& fin = t2hyps[T];
-    recombine_prune(fin, fin.size() > 0 ? fin.size() : 1);
+    merge_duplicates(fin);
+    prune(fin, fin.size() > 0 ? fin.size() : 1);
     int n_out = 0;
     for (size_t a = 0; a < fin.size() && (int)a < max_hyps; ++a) {
         const Hyp& h = fin[a];

@@ -201,7 +201,7 @@ struct BeamLayout {
     int slots;
 };
 BeamLayout make_beam_layout(const wind_model_t& m, int T, int W, int K, int S, size_t base);
-wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int max_hyps, int max_out, int32_t* out_tokens,
+wind_status_t beam_search_run(Call& cb, const BeamLayout& bl, int K, int prefix_search, int max_hyps, int max_out, int32_t* out_tokens,
                               int32_t* out_frames, int32_t* out_len, double* out_score, int32_t* n_hyps, int64_t* n_steps,
                               cudaError_t* cuda_err);
 

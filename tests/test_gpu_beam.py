@@ -46,11 +46,11 @@ def small_model(seed, dtype="f32", V=37, L=1, act=0, blank0=False, bias=1.5):
     return w, r
 
 
-def compare(pkg, w, enc, W, K, S, gap_needed, tol):
+def compare(pkg, w, enc, W, K, S, gap_needed, tol, prefix_search=False):
     """Returns True when the case was decidable and the GPU agreed with the oracle."""
     T = enc.shape[0]
-    want, gap, steps = oracle.beam_search(oracle.Model(w), enc, T, W, K, S, max_hyps=256)
-    got, gsteps, st = pkg.wind_beam_search(pkg.WindModel(w), enc, W, K, S, max_hyps=256)
+    want, gap, steps = oracle.beam_search(oracle.Model(w), enc, T, W, K, S, max_hyps=256, prefix_search=prefix_search)
+    got, gsteps, st = pkg.wind_beam_search(pkg.WindModel(w), enc, W, K, S, max_hyps=256, prefix_search=prefix_search)
     assert st == 0 and len(got) >= 1
     for tok, frm, sc in got:                      # always: well-formed hypotheses
         assert len(tok) == len(frm) and np.all(np.diff(frm) >= 0) and (len(frm) == 0 or frm.max() < T)
@@ -99,6 +99,35 @@ def test_fp32_matches_the_oracle_when_the_search_is_decidable(pkg, W, K, S, L, b
         decided += compare(pkg, w, enc, W, K, S, gap_needed=5e-5, tol=1e-4)
     print(f"[beam] W={W} K={K} S={S}: {decided}/8 cases decidable and equal to the oracle")
     assert decided >= 4
+
+
+def test_prefix_step_worked_example_fp32(pkg):
+    # A = (x .45, y .05, blank .5), B = (x .1, y .8, blank .1); utterance A B, W = 1, S = 2, K = 2 (derivation: the
+    # oracle's pin of the same example): at t = 1 the list {[] .5, [x,x] .2025, [x] .225} becomes {[x,x] .23}
+    w = table_model([[.45, .05, .5], [.1, .8, .1]])
+    enc = np.eye(2, dtype=np.float32)[[0, 1]]
+    hyps, steps, st = pkg.wind_beam_search(pkg.WindModel(w), enc, 1, 2, 2, prefix_search=True)
+    assert st == 0 and steps == 4
+    assert [list(h[0]) for h in hyps] == [[0, 0, 1, 1], [0, 0, 1, 0], [0, 0, 0, 1], [0, 0, 0, 0]]
+    assert np.allclose(np.exp([h[2] for h in hyps]), [.1472, .0184, .0184, .0023], atol=1e-6)
+
+
+@pytest.mark.parametrize("W,K,S,L,bias", [(1, 2, 3, 1, 2.5), (1, 4, 2, 2, 1.5), (8, 4, 2, 1, 2.5)])
+def test_fp32_with_the_prefix_step_matches_the_oracle_when_decidable(pkg, W, K, S, L, bias):
+    decided = changed = 0
+    for seed in range(8):
+        w, r = small_model(400 + seed + 10 * W, L=L, bias=bias)
+        T = int(r.integers(12, 24))
+        enc = r.standard_normal((T, 24)).astype(np.float32)
+        decided += compare(pkg, w, enc, W, K, S, gap_needed=5e-5, tol=1e-4, prefix_search=True)
+        a, _, _ = oracle.beam_search(oracle.Model(w), enc, T, W, K, S, max_hyps=256)
+        b, _, _ = oracle.beam_search(oracle.Model(w), enc, T, W, K, S, max_hyps=256, prefix_search=True)
+        da = {tuple(int(x) for x in h[0]): h[2] for h in a}
+        db = {tuple(int(x) for x in h[0]): h[2] for h in b}
+        changed += set(da) != set(db) or any(abs(da[k] - db[k]) > 1e-9 for k in da)
+    print(f"[beam] prefix step, W={W} K={K} S={S}: {decided}/8 cases decidable and equal to the oracle; "
+          f"the step changes the final hypotheses in {changed}/8")
+    assert decided >= 3 and changed >= 3       # the cases do contain prefix pairs
 
 
 def test_bf16_best_score_is_close_to_the_oracle(pkg):

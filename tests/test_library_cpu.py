@@ -93,7 +93,7 @@ def test_invalid_arguments_are_rejected_on_the_host(lib):
     assert lib.wind_beam_workspace_bytes(ref, 100, 8, 4, 3, None) == bd.WIND_ERR_INVALID_ARG
     assert lib.wind_beam_workspace_bytes(ref, 1500, 8, 4, 10, C.byref(n)) == bd.WIND_OK and 0 < n.value < (1 << 30)
     nh, ns = C.c_int32(0), C.c_int64(0)
-    assert lib.wind_beam_search(ref, None, 100, 8, 4, 3, 8, 100, None, None, None, None, C.byref(nh), C.byref(ns), None, 0, None) \
+    assert lib.wind_beam_search(ref, None, 100, 8, 4, 3, 0, 8, 100, None, None, None, None, C.byref(nh), C.byref(ns), None, 0, None) \
         == bd.WIND_ERR_INVALID_ARG
     n_ev = C.c_int32(0)
     assert lib.wind_read_trace(ref, 1, 10, 4, None, None, None, 0, C.byref(n_ev)) == bd.WIND_ERR_INVALID_ARG
