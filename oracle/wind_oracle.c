@@ -27,7 +27,8 @@
  * one, closed forms, W = 1 equals Algorithm 1, a step-by-step recomputation from Eq. (1) in the tests, and a
  * hand-worked example where it differs from Algorithm 2; and Algorithm 3 (beam search for one utterance), pinned
  * by: beam 1 equals window-based greedy decoding, an unpruned beam gives every token sequence its total probability
- * over all alignments for every window (brute force on independently evaluated logits), and a hand-worked example.
+ * over all alignments for every window (brute force on independently evaluated logits), hand-worked examples, and
+ * the optional prefix step against independently evaluated completions.
  *
  * Pins (see tests): WIND(W) == sequential for every W; brute-force tabulation
  * of joint argmaxes on tiny models; LSTM / linear layers against library fp64
