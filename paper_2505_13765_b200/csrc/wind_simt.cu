@@ -334,7 +334,7 @@ static cudaError_t simt_joint_t(const Call& c, float* logits_out) {
 }
 
 // Beam search: the rows are hypotheses of ONE utterance (all read utterance 0's enc_proj rows), there are only a few
-// of them, and only the logits are wanted (Eq. (1) is a pass of its own): one block per (vocabulary slice of 64,
+// of them, and only the logits are wanted (Eq. (1) is a pass of its own): one block per (vocabulary slice of 16,
 // hypothesis), so that the joint of a handful of hypotheses still spreads over the SMs.
 template <typename TW>
 __global__ void __launch_bounds__(256) joint_logits_shared_kernel(const int32_t* __restrict__ t_cur, const int32_t* __restrict__ enc_len,
@@ -346,7 +346,7 @@ __global__ void __launch_bounds__(256) joint_logits_shared_kernel(const int32_t*
     const int t = t_cur[b], len = enc_len[b];
     if (t >= len) return;
     const int n = min(W, len - t);
-    const int v0 = blockIdx.x * 64, v1 = min(NV, v0 + 64);
+    const int v0 = blockIdx.x * 16, v1 = min(NV, v0 + 16);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
     for (int w0 = 0; w0 < n; w0 += 8) {
         const int nc = min(8, n - w0);
@@ -383,7 +383,7 @@ template <typename TW>
 static cudaError_t simt_joint_shared_t(const Call& c, float* logits_out) {
     const size_t smem = sizeof(float) * 8 * (size_t)c.m.H;
     if (smem > 48 * 1024) cudaFuncSetAttribute(joint_logits_shared_kernel<TW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    dim3 grid((unsigned)((c.m.V + 1 + 63) / 64), (unsigned)c.B);
+    dim3 grid((unsigned)((c.m.V + 1 + 15) / 16), (unsigned)c.B);
     joint_logits_shared_kernel<TW><<<grid, 256, smem, c.stream>>>(c.t(), c.enc_len, (const TW*)c.enc_proj(), c.pred_proj(),
                                                                   (const TW*)c.m.w_out, c.m.b_out, logits_out, c.W, c.m.H,
                                                                   c.m.V + 1, c.m.act);
