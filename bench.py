@@ -309,9 +309,12 @@ def main():
             step_host()
             ke = max(1, min(args.steps, 3))
             ms_e = timed(step_host, ke)
+            # bytes that cross the bus: the valid frames and the lengths in, the lengths and the token / frame columns up
+            # to the longest transcript out
+            longest = int(ol_h.max())
             out["e2e"] = {"value": audio_s * ke / (ms_e * 1e-3), "unit": "audio-s/s",
-                          "h2d_bytes_per_step": int(enc_h.numel() * enc_h.element_size() + len_h.numel() * 4),
-                          "d2h_bytes_per_step": int((tok_h.numel() + frm_h.numel() + ol_h.numel()) * 4)}
+                          "h2d_bytes_per_step": int(int(lens_np.sum()) * D * enc_h.element_size() + len_h.numel() * 4),
+                          "d2h_bytes_per_step": int((2 * B * longest + ol_h.numel()) * 4)}
     elif world > 1:
         # every rank must take part in the same collectives: none are issued in the extras
         pass

@@ -156,8 +156,11 @@ wind_status_t wind_host_staging_bytes(const wind_model_t* m, int32_t B, int32_t 
 
 /*
  * Same decode, but enc, enc_len, out_tokens, out_frames and out_len are HOST pointers
- * (pinned memory gives asynchronous copies).  The call copies enc and enc_len to the
- * device, decodes, copies the outputs back and synchronises the stream.  The model's
+ * (pinned memory gives asynchronous copies).  The call copies enc_len and the valid frames
+ * of enc to the device, decodes, copies the lengths and then the token and frame columns up
+ * to the longest transcript back (entries of a row beyond its out_len are unspecified), and
+ * synchronises the stream.  enc_len_host is also read on the host: a value outside [0, T] is
+ * WIND_ERR_INVALID_ARG.  The model's
  * weights stay device pointers.  workspace: device, at least wind_workspace_bytes +
  * wind_host_staging_bytes.
  */

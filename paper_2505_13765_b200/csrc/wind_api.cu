@@ -301,16 +301,34 @@ wind_status_t wind_decode_greedy_host(const wind_model_t* m, const void* enc_hos
     int32_t* d_tok = reinterpret_cast<int32_t*>(ws + lay.st_tok);
     int32_t* d_frm = reinterpret_cast<int32_t*>(ws + lay.st_frm);
     int32_t* d_olen = reinterpret_cast<int32_t*>(ws + lay.st_olen);
-    WIND_CUDA(cudaMemcpyAsync(d_enc, enc_host, es * (size_t)B * T * m->D, cudaMemcpyHostToDevice, st));
+    // only the valid frames of every utterance cross the bus (padding frames are never read for a decision)
+    for (int b = 0; b < B; ++b) {
+        const int len = enc_len_host[b];
+        if (len < 0 || len > T) return WIND_ERR_INVALID_ARG;
+        if (len > 0)
+            WIND_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(d_enc) + es * (size_t)b * T * m->D,
+                                      static_cast<const uint8_t*>(enc_host) + es * (size_t)b * T * m->D, es * (size_t)len * m->D,
+                                      cudaMemcpyHostToDevice, st));
+    }
     WIND_CUDA(cudaMemcpyAsync(d_len, enc_len_host, sizeof(int32_t) * B, cudaMemcpyHostToDevice, st));
     Call c;
     fill_call(c, m, d_enc, d_len, B, T, W, max_symbols, d_tok, d_frm, d_olen, max_out, workspace, st);
     s = enqueue_decode(c);
     if (s != WIND_OK) return s;
-    WIND_CUDA(cudaMemcpyAsync(out_tokens_host, d_tok, sizeof(int32_t) * (size_t)B * max_out, cudaMemcpyDeviceToHost, st));
-    WIND_CUDA(cudaMemcpyAsync(out_frames_host, d_frm, sizeof(int32_t) * (size_t)B * max_out, cudaMemcpyDeviceToHost, st));
+    // lengths first, then the columns of the two output arrays that hold tokens (up to the longest transcript)
     WIND_CUDA(cudaMemcpyAsync(out_len_host, d_olen, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, st));
-    return read_status(c);
+    const wind_status_t status = read_status(c);   // synchronises the stream
+    if (status != WIND_OK && status != WIND_ERR_OUTPUT_OVERFLOW) return status;
+    int longest = 0;
+    for (int b = 0; b < B; ++b) longest = out_len_host[b] > longest ? out_len_host[b] : longest;
+    if (longest > max_out) longest = max_out;
+    if (longest > 0) {
+        const size_t pitch = sizeof(int32_t) * (size_t)max_out, width = sizeof(int32_t) * (size_t)longest;
+        WIND_CUDA(cudaMemcpy2DAsync(out_tokens_host, pitch, d_tok, pitch, width, (size_t)B, cudaMemcpyDeviceToHost, st));
+        WIND_CUDA(cudaMemcpy2DAsync(out_frames_host, pitch, d_frm, pitch, width, (size_t)B, cudaMemcpyDeviceToHost, st));
+        WIND_CUDA(cudaStreamSynchronize(st));
+    }
+    return status;
 }
 
 // Teacher-forced window logits, enqueued on the stream (no synchronisation); c receives the call's bundle.

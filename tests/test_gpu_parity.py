@@ -436,6 +436,24 @@ def test_host_buffer_entry_point_matches_device_entry_point(pkg):
     for b in range(B):
         assert np.array_equal(tok_h.numpy()[b, : ref[2][b]], ref[0][b, : ref[2][b]])
         assert np.array_equal(frm_h.numpy()[b, : ref[2][b]], ref[1][b, : ref[2][b]])
+    # only the columns up to the longest transcript come back
+    longest = int(ref[2].max())
+    assert longest < max_out and np.all(tok_h.numpy()[:, longest:] == -1) and np.all(frm_h.numpy()[:, longest:] == -1)
+    # only the valid frames go in: poison in the host padding and a zero-length utterance change nothing
+    enc2, lens2 = enc.copy(), lens.copy()
+    lens2[1] = 0
+    for b in range(B):
+        enc2[b, lens2[b]:] = np.nan
+    ref2 = pkg.decode(model, np.nan_to_num(enc2), lens2, 8, cfg.S)
+    enc_h2 = torch.from_numpy(enc2).to(model.torch_dtype).pin_memory()
+    len_h2 = torch.from_numpy(lens2).pin_memory()
+    pkg.wind_decode_greedy_host(model, enc_h2, len_h2, 8, cfg.S, tok_h, frm_h, ol_h, wsb)
+    assert np.array_equal(ol_h.numpy(), ref2[2]) and ol_h.numpy()[1] == 0
+    for b in range(B):
+        assert np.array_equal(tok_h.numpy()[b, : ref2[2][b]], ref2[0][b, : ref2[2][b]])
+    bad = len_h2.clone()
+    bad[0] = T + 1
+    assert pkg.wind_decode_greedy_host(model, enc_h2, bad, 8, cfg.S, tok_h, frm_h, ol_h, wsb, check=False) == pkg.binding.WIND_ERR_INVALID_ARG
 
 
 def test_unfillable_barrier_ends_in_timeout_status_and_the_context_stays_usable(pkg):
