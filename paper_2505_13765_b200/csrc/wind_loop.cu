@@ -205,7 +205,11 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
     const int q = warp & 3;                    // tensor-memory lane quadrant of this warp
     const int row_in_tile = q * 32 + lane;     // the tensor-memory lane (accumulator row) of this thread
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-    const bool has_j = cta < p.j_items;
+    // joint items of this CTA.  Streaming mode: items cta, cta + G, ... of the (row group, vocabulary tile) list.
+    // Resident mode: the CTA keeps ONE vocabulary tile (cta % vt_count) and takes the row groups j_first,
+    // j_first + rg_stride, ... (one per wave); CTAs beyond vt_count * rg_stride have none.
+    const int j_first = RES ? (cta < p.vt_count * p.rg_stride ? cta / p.vt_count : p.rg_count) : 0;
+    const bool has_j = RES ? j_first < p.rg_count : cta < p.j_items;
     const int my_vt = cta % p.vt_count;        // vocabulary tile of this CTA's joint item when it has exactly one
 
     // ----- the joint's W_out tile, loaded once when every CTA owns one joint item -----
@@ -1271,12 +1275,15 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     if (warp == 0) {
                         fence_proxy_async_all();
                         if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_FIRST_ISSUE);
-                        const bool ok = produce_one(&M.z3, (cta / p.vt_count) * n_tile, (uint32_t)n_tile * (uint32_t)p.H * 2u);
-                        if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_LAST_ISSUE);
-                        if (ok) mma_part(0, tm_j + (uint32_t)n_tile, n_tile, p.kb_h / 2, p.kb_h, true);
+                        for (int rg = j_first; rg < p.rg_count; rg += p.rg_stride) {
+                            const bool ok = produce_one(&M.z3, rg * n_tile, (uint32_t)n_tile * (uint32_t)p.H * 2u);
+                            if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_LAST_ISSUE);
+                            if (!ok || !mma_part(0, tm_j + (uint32_t)n_tile, n_tile, p.kb_h / 2, p.kb_h, true)) break;
+                        }
                         if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_COMMIT);
                     } else {
-                        mma_part(0, tm_j, n_tile, 0, p.kb_h / 2, true);
+                        for (int rg = j_first; rg < p.rg_count; rg += p.rg_stride)
+                            if (!mma_part(0, tm_j, n_tile, 0, p.kb_h / 2, true)) break;
                         if constexpr (FULL) trace_event(p, 1, tr_n, step, TR_J, EV_COMMIT);
                     }
                 }
@@ -1339,8 +1346,8 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             } else {
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_START);
                 const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
-                for (int i = cta; i < p.j_items; i += G) {
-                    const int rg = i / p.vt_count, vt = i - rg * p.vt_count;
+                for (int i = RES ? j_first : cta; i < (RES ? p.rg_count : p.j_items); i += RES ? p.rg_stride : G) {
+                    const int rg = RES ? i : i / p.vt_count, vt = RES ? my_vt : i - rg * p.vt_count;
                     const int v = vt * 128 + row_in_tile;            // this thread's vocabulary entry
                     const bool v_ok = v < p.NV;
                     const float bias = v_ok ? p.b_out[v] : 0.f;
@@ -1694,9 +1701,32 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
     // W_pred in tiles of 64 rows stay in the shared memory of disjoint CTA sets for the whole decode; per step a CTA
     // fetches only its utterance group's rows of the state, as one box.
     const char* res_env = getenv("WIND_RESIDENT");
-    if (m.L <= 2 && one_wave && m.H / 2 + 2 * pl.nj <= (int)LOOP_TMEM_COLS && !(res_env && atoi(res_env) == 0)) {
-        const int l_sets = m.L == 2 ? 3 : 1;   // layer 0; with two layers also layer 1's input and recurrent halves
+    // Its joint: every CTA keeps one vocabulary tile; G / vt_count CTAs share a tile and take one row group each per
+    // wave.  Row-group sizes are tried in order of preference -- the smallest that needs one wave, else from the largest
+    // down (fewest waves, at most four) -- until the whole plan fits shared and tensor memory.
+    const int per_wave = pl.vt_count <= G ? G / pl.vt_count : 0;
+    int cands[5], n_cands = 0;
+    {
+        const char* env = getenv("WIND_J_WAVES");   // experiments: 1 keeps the resident mode to one wave
+        const int max_waves = env && atoi(env) == 1 ? 1 : 4;
+        int one = 0;
+        for (int cand : {16, 32, 64, 96})
+            if (per_wave >= 1 && ((rows + cand - 1) / cand + per_wave - 1) / per_wave == 1) { one = cand; break; }
+        if (one) cands[n_cands++] = one;
+        for (int cand : {96, 64, 32, 16})
+            if (per_wave >= 1 && cand != one && ((rows + cand - 1) / cand + per_wave - 1) / per_wave <= max_waves && !one)
+                cands[n_cands++] = cand;
+    }
+    bool resident_done = false;
+    for (int ci = 0; ci < n_cands && !resident_done; ++ci) {
+        const int r_nj = cands[ci];
+        if (!(m.L <= 2 && m.H / 2 + 2 * r_nj <= (int)LOOP_TMEM_COLS && !(res_env && atoi(res_env) == 0))) continue;
         LoopPlan r = pl;
+        r.nj = r_nj;
+        r.rg_count = (rows + r_nj - 1) / r_nj;
+        r.j_items = r.vt_count * r.rg_count;
+        r.rg_stride = per_wave;
+        const int l_sets = m.L == 2 ? 3 : 1;   // layer 0; with two layers also layer 1's input and recurrent halves
         r.ut_count = m.P / 16;
         r.ht_count = m.H / 64;
         bool found = false;
@@ -1741,7 +1771,10 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
             if (r.w_first + r.w_count + r.p_items > G) r.w_count = 0;
             r.l_early = 1;
             const int acc_cols = r.nl > 2 * r.np ? r.nl : 2 * r.np;
-            if ((long long)r.smem_bytes <= (long long)budget + 1024 && r.tm_l + acc_cols <= (int)LOOP_TMEM_COLS) pl = r;
+            if ((long long)r.smem_bytes <= (long long)budget + 1024 && r.tm_l + acc_cols <= (int)LOOP_TMEM_COLS) {
+                pl = r;
+                resident_done = true;
+            }
         }
     }
     *out = pl;
@@ -1807,6 +1840,7 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     long long cap = (long long)c.T * (c.S + 1) + 2;
     p.step_cap = cap > 0x7fffffff ? 0x7fffffff : (int)cap;
     p.nj = pl.nj; p.vt_count = pl.vt_count; p.rg_count = pl.rg_count; p.j_items = pl.j_items; p.j_mode = pl.j_mode;
+    p.rg_stride = pl.rg_stride > 0 ? pl.rg_stride : 1;
     p.tm_j = pl.tm_j; p.tm_l = pl.tm_l; p.tm_p = pl.tm_p; p.l_early = pl.l_early;
     p.resident = pl.resident; p.nl = pl.nl; p.ut_count = pl.ut_count > 0 ? pl.ut_count : 1; p.ht_count = pl.ht_count > 0 ? pl.ht_count : 1;
     p.w_first = pl.w_first; p.w_count = pl.resident ? pl.w_count : 0;

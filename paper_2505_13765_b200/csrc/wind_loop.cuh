@@ -33,6 +33,7 @@ struct LoopPlan {
     int grid;
     int kb_h, kb_p;                        // K blocks of 64 in H and in P
     int nj, vt_count, rg_count, j_items;   // joint: window rows per item, vocabulary tiles, row groups
+    int rg_stride;                         // resident mode: row groups taken per wave (CTAs per vocabulary tile)
     int j_mode;                            // where the joint's W_out tile lives: 0 streamed through the ring, 1 kept in
                                            // shared memory, 2 kept in tensor memory (1, 2: every CTA owns one joint item)
     int tm_j, tm_l, tm_p;                  // tensor-memory columns of the joint / decoder / projection accumulators
@@ -52,7 +53,7 @@ struct LoopParams {
     Ctrl* ctrl;
     int B, T, W, S, max_out, H, P, NV, blank, act, L;
     int rows, rows_pad, Bpad, step_cap;
-    int nj, vt_count, rg_count, j_items, j_mode;
+    int nj, vt_count, rg_count, j_items, j_mode, rg_stride;
     int tm_j, tm_l, tm_p, l_early;
     int resident, nl, ut_count, ht_count, ql_count, qp_count;
     int w_first, w_count;

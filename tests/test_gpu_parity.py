@@ -264,6 +264,9 @@ def test_bf16_tensor_path_more_utterances_than_one_tile(pkg, monkeypatch, reside
     (40, 32, 4, 128, 64, 500, 2),
     (148, 4, 3, 256, 256, 1000, 2),
     (129, 2, 2, 256, 128, 152, 2),     # the resident plan takes 128 utterances per projection CTA
+    (60, 8, 3, 64, 64, 4099, 1),       # 33 vocabulary tiles: four CTAs per tile, the resident joint runs in two waves
+    (100, 8, 2, 128, 128, 2100, 2),    # two layers, 17 vocabulary tiles, two waves
+    (90, 16, 3, 64, 128, 3000, 1),     # 24 tiles, six CTAs per tile, three waves of 96-row groups
 ])
 @pytest.mark.parametrize("resident", [1, 0])
 def test_bf16_tensor_path_shape_sweep(pkg, monkeypatch, resident, B, W, S, P, H, V, L):

@@ -164,3 +164,10 @@ def test_bf16_tensor_path_wide_window_and_overflow(pkg, monkeypatch, resident):
     for b in range(6):
         n = min(4, olen[b])
         assert o2[b] == n and np.array_equal(t2[b, :n], tok[b, :n]) and np.array_equal(f2[b, :n], frm[b, :n])
+
+
+def test_bf16_resident_joint_in_waves(pkg):
+    # 33 vocabulary tiles leave four CTAs per tile: 480 window rows take two waves of 96-row groups per CTA
+    w, enc, lens = ragged_case(550, B=60, T=24, D=64, E=64, P=64, L=1, H=64, V=4099, act=0, bias=2.0, dtype="bf16")
+    rep, _ = check_window_greedy(pkg, w, enc, lens, 8, 3, kernels=2)
+    assert rep["stats"]["kernels"] == 2
