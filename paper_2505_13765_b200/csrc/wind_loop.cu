@@ -966,15 +966,29 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 }
             }
             // rows beyond the first 256 of this CTA (wide windows): same chunking, fetched here
-            for (int r = p_row0 + 256; r < rows_here; r += 32) {
-                const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
-                if (b >= p.B) break;
-                int frame = 0;
-                const int kind = row_kind(b, w, t_new[b], frame);
-                if (kind == 0) continue;
-                uint4 x = make_uint4(0, 0, 0, 0);
-                if (kind == 2) x = *reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + frame) * p.H + h0 + p_chunk * 8);
-                *reinterpret_cast<uint4*>(p.z + ((size_t)b * p.W + w) * p.H + h0 + p_chunk * 8) = z_chunk(bl, kind, x);
+            // (four rows at a time, their loads requested together)
+            for (int r0 = p_row0 + 256; r0 < rows_here; r0 += 128) {
+                uint4 x[4];
+                int kinds4[4], bls[4];
+                size_t zoff[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int r = r0 + 32 * i;
+                    const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
+                    x[i] = make_uint4(0, 0, 0, 0);
+                    kinds4[i] = 0; bls[i] = 0; zoff[i] = 0;
+                    if (r < rows_here && b < p.B) {
+                        int frame = 0;
+                        kinds4[i] = row_kind(b, w, t_new[b], frame);
+                        bls[i] = bl;
+                        zoff[i] = ((size_t)b * p.W + w) * p.H + h0 + p_chunk * 8;
+                        if (kinds4[i] == 2)
+                            x[i] = *reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + frame) * p.H + h0 + p_chunk * 8);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (kinds4[i] != 0) *reinterpret_cast<uint4*>(p.z + zoff[i]) = z_chunk(bls[i], kinds4[i], x[i]);
             }
         }
         fence_proxy_async_all();
