@@ -69,7 +69,7 @@ cudaError_t tc_prepare(Call& c) {
     const wind_model_t& m = c.m;
 #define WIND_MAP(call_) do { e = (call_); if (e != cudaSuccess) return e; } while (0)
     WIND_MAP(make_map(&M.enc, c.enc, (uint64_t)c.B * c.T, m.D, BM));
-    WIND_MAP(make_map(&M.w_enc, m.w_enc, m.H, m.D, 128));
+    WIND_MAP(make_map(&M.w_enc, m.w_enc, m.H, m.D, 256));
     WIND_MAP(make_map(&M.emb, m.emb, (uint64_t)m.V + 1, m.E, BM));
     WIND_MAP(make_map(&M.w_ih0, c.w_ih[0], 4ull * m.P, m.E, 128));
 #undef WIND_MAP
@@ -96,19 +96,22 @@ struct GemmParams {
 };
 
 constexpr int GEMM_THREADS = 192;  // warp 0: TMA, warp 1: MMA + tensor memory, warps 2..5: epilogue
-constexpr int GEMM_STAGES = 3;      // 3 x 32 KB per CTA, so that two CTAs share an SM: one's epilogue overlaps the other's main loop
-constexpr int GEMM_BN = 128;
+// Two CTAs share an SM, so that one's epilogue overlaps the other's main loop.  The encoder projection uses 128 x 256
+// tiles (the kernel is paced by its two issuing threads: half as many TMA and MMA instructions per flop as with 128 x
+// 128) with two 48 KB stages; the gate table (fp32 output, staged through the same buffers) 128 x 128 with three.
+template <int MODE> struct GemmShape { static constexpr int BN = MODE == 0 ? 256 : 128; static constexpr int STAGES = MODE == 0 ? 2 : 3; };
 
 template <int MODE>
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[GEMM_STAGES], empty_bar[GEMM_STAGES], accum_bar;
+    __shared__ uint64_t full_bar[GemmShape<MODE>::STAGES], empty_bar[GemmShape<MODE>::STAGES], accum_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ float s_bias[GEMM_BN];
+    __shared__ float s_bias[GemmShape<MODE>::BN];
     __shared__ int s_valid[BM];
 
+    constexpr int GEMM_BN = GemmShape<MODE>::BN, GEMM_STAGES = GemmShape<MODE>::STAGES;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr uint32_t b_stage_bytes = GEMM_BN * BK * 2;
     constexpr uint32_t stage_bytes = A_STAGE_BYTES + b_stage_bytes;
@@ -184,10 +187,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         const int row = q * 32 + lane;     // accumulator row of this thread
         // before the accumulator is ready: this tile's bias values and which of its rows are valid frames
         {
-            const int n = n_tile_idx * GEMM_BN + et;
-            float bsum = 0.f;
-            if (n < p.N) bsum = p.bias0[n] + (MODE == MODE_GATE_TABLE ? p.bias1[n] : 0.f);
-            s_bias[et] = bsum;
+            for (int k = et; k < GEMM_BN; k += 128) {
+                const int n = n_tile_idx * GEMM_BN + k;
+                float bsum = 0.f;
+                if (n < p.N) bsum = p.bias0[n] + (MODE == MODE_GATE_TABLE ? p.bias1[n] : 0.f);
+                s_bias[k] = bsum;
+            }
             const long long r = (long long)m_blk * BM + row;
             bool valid = r < p.rows;
             if (MODE == MODE_ENC_PROJ && valid) {
@@ -246,7 +251,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (threadIdx.x == 0 && abort_flag) set_status(p.ctrl, WIND_ERR_TIMEOUT);
 }
 
-constexpr size_t gemm_smem_bytes() { return (size_t)GEMM_STAGES * (A_STAGE_BYTES + (size_t)GEMM_BN * BK * 2) + 1024; }
+template <int MODE>
+constexpr size_t gemm_smem_bytes() { return (size_t)GemmShape<MODE>::STAGES * (A_STAGE_BYTES + (size_t)GemmShape<MODE>::BN * BK * 2) + 1024; }
 
 // Shared-memory opt-in of the kernels of this file.
 static cudaError_t tc_set_attributes() {
@@ -254,8 +260,8 @@ static cudaError_t tc_set_attributes() {
     std::lock_guard<std::mutex> lock(g_tc_mutex);
     if (done) return cudaSuccess;
     cudaError_t e;
-    if ((e = cudaFuncSetAttribute(gemm_kernel<MODE_ENC_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem_bytes())) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(gemm_kernel<MODE_GATE_TABLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem_bytes())) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(gemm_kernel<MODE_ENC_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem_bytes<MODE_ENC_PROJ>())) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(gemm_kernel<MODE_GATE_TABLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem_bytes<MODE_GATE_TABLE>())) != cudaSuccess) return e;
     done = true;
     return cudaSuccess;
 }
@@ -269,8 +275,9 @@ cudaError_t tc_enc_proj(const Call& c) {
     p.N = c.m.H;
     p.enc_len = c.enc_len; p.T = c.T;
     p.out_bf16 = (__nv_bfloat16*)c.enc_proj(); p.bias0 = c.m.b_enc;
-    dim3 grid((unsigned)(((c.m.H + GEMM_BN - 1) / GEMM_BN) * ((p.rows + BM - 1) / BM)));
-    gemm_kernel<MODE_ENC_PROJ><<<grid, GEMM_THREADS, gemm_smem_bytes(), c.stream>>>(M.enc, M.w_enc, p);
+    constexpr int BN = GemmShape<MODE_ENC_PROJ>::BN;
+    dim3 grid((unsigned)(((c.m.H + BN - 1) / BN) * ((p.rows + BM - 1) / BM)));
+    gemm_kernel<MODE_ENC_PROJ><<<grid, GEMM_THREADS, gemm_smem_bytes<MODE_ENC_PROJ>(), c.stream>>>(M.enc, M.w_enc, p);
     return cudaGetLastError();
 }
 
@@ -282,8 +289,9 @@ cudaError_t tc_gate_table(const Call& c) {
     p.rows = (long long)c.m.V + 1;
     p.N = 4 * c.m.P;
     p.out_f32 = c.g0(); p.bias0 = c.b_ih[0]; p.bias1 = c.b_hh[0];
-    dim3 grid((unsigned)(((p.N + GEMM_BN - 1) / GEMM_BN) * ((p.rows + BM - 1) / BM)));
-    gemm_kernel<MODE_GATE_TABLE><<<grid, GEMM_THREADS, gemm_smem_bytes(), c.stream>>>(M.emb, M.w_ih0, p);
+    constexpr int BN = GemmShape<MODE_GATE_TABLE>::BN;
+    dim3 grid((unsigned)(((p.N + BN - 1) / BN) * ((p.rows + BM - 1) / BM)));
+    gemm_kernel<MODE_GATE_TABLE><<<grid, GEMM_THREADS, gemm_smem_bytes<MODE_GATE_TABLE>(), c.stream>>>(M.emb, M.w_ih0, p);
     return cudaGetLastError();
 }
 
