@@ -29,9 +29,22 @@
  *   - Every pointer is a DEVICE pointer unless the parameter comment says "host".
  *   - All buffers are caller-owned and borrowed for the duration of the call; the
  *     library allocates no device memory.  Weight matrices are row-major [out, in].
- *   - dtype WIND_DT_BF16: enc, emb and all weight matrices are bf16 (uint16 bit
- *     patterns), biases fp32, all accumulation and recurrent state fp32.
- *     dtype WIND_DT_F32: everything fp32, plain FMA arithmetic (no tf32).
+ *   - dtype WIND_DT_F32: everything fp32, plain FMA arithmetic (no tf32); joint logits agree
+ *     with an fp64 evaluation within 1e-4.
+ *   - dtype WIND_DT_BF16: enc, emb and all weight matrices are bf16 (uint16 bit patterns),
+ *     biases fp32.  Every product is accumulated in fp32 and the LSTM cell state c is kept in
+ *     fp32.  Three intermediate quantities are rounded to bf16 (nearest even) because they are
+ *     tensor-core operands: enc_proj (stored once per call), the LSTM hidden state h wherever it
+ *     is consumed (the recurrent term of the next update, the input of the layer above and
+ *     pred_proj -- the recurrence therefore feeds back a bf16 h), and the joint's activations
+ *     act(enc_proj + pred_proj).  Both kernel sets (wind_kernels_t) round in the same places.
+ *     The tensor-core kernels evaluate the gate nonlinearities (and tanh activations) with the
+ *     hardware tanh approximation (absolute error about 5e-4, below the bf16 rounding of h) when
+ *     the weights are resident on chip; the plain-ALU kernels use tanhf / expf.  Joint logits
+ *     agree with an fp64 evaluation of the same bf16 weights within 2e-2, also after hundreds
+ *     of decoder updates; decisions whose top-two margin is smaller than such differences can
+ *     come out differently between kernel sets (AUTO picks the set by shape), never between two
+ *     runs of one set, and never between window sizes.
  *   - Calls enqueue work on `stream`, synchronise that stream once at the end to read the
  *     device status word, and return it.  Errors detectable on the host return before
  *     any launch.  Every device-side wait is bounded; a wait that runs out sets
@@ -113,7 +126,9 @@ wind_status_t wind_workspace_bytes(const wind_model_t* m, int32_t B, int32_t T, 
  * Batched greedy decoding (Algorithm 2; Algorithm 1 when W == 1).
  *   enc        [B, T, D] row-major, element type m->dtype.  Frames t >= enc_len[b] are
  *              never read for a decision (they may hold NaN).
- *   enc_len    [B] int32, 0 <= enc_len[b] <= T.
+ *   enc_len    [B] int32, 0 <= enc_len[b] <= T.  The values live on the device, so they are checked there, before
+ *              the loop starts: if one lies outside [0, T] nothing is decoded (no frame is read through
+ *              it), the outputs are undefined and the call returns WIND_ERR_INVALID_ARG.
  *   W          window, 1 <= W <= 64.   max_symbols >= 1.
  *   out_tokens [B, max_out] int32; out_frames [B, max_out] int32 (0-based encoder frame at
  *              which the token was emitted, non-decreasing, each value at most
@@ -175,6 +190,9 @@ wind_status_t wind_decode_greedy_host(const wind_model_t* m, const void* enc_hos
  *   prefix [B, U] int32, prefix_len [B] (tokens fed after the start-of-sequence blank;
  *   U >= max prefix_len), t0 [B] window start (0 <= t0[b] <= enc_len[b]).
  *   logits [B, W, V+1] fp32; rows w >= min(W, enc_len[b] - t0[b]) are left untouched.
+ * A length outside [0, T] is handled as in wind_decode_greedy.  A prefix token outside [0, V] is replaced
+ * by the blank and a window start outside [0, enc_len[b]] is moved inside (so that nothing is read out of
+ * range); in both cases the call returns WIND_ERR_INVALID_ARG and the logits are undefined.
  */
 wind_status_t wind_eval_joint_window(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t B,
                                      int32_t T, int32_t W, const int32_t* prefix, int32_t U,
@@ -218,11 +236,17 @@ wind_status_t wind_window_first_output(const wind_model_t* m, const void* enc, c
  * WIND_STATIC_WORKSPACE_BYTES that is part of the library image: every GPU on which the
  * library's kernels are loaded holds those bytes until the process exits.
  *
- *   - Nothing is allocated or freed, here or in any library routine the call uses.
+ *   - The call makes no cudaMalloc / cudaFree and uses no library routine that allocates.
  *   - If wind_workspace_bytes(m, B, T, W) exceeds WIND_STATIC_WORKSPACE_BYTES the call returns
  *     WIND_ERR_WORKSPACE before any launch; use wind_eval_joint_window with your own workspace.
- *   - The first call on each device looks up the device address of the array (with that
- *     device current).  Make that first call outside any stream capture.
+ *   - The first call on each device is a set-up step: with that device current it looks up the
+ *     device address of the array.  With CUDA's lazy loading this is also the moment the driver
+ *     loads the library's image on that device, which reserves the array's bytes and may
+ *     synchronise the device; if the device has no room left the call fails with WIND_ERR_CUDA.
+ *     Make that first call at start-up, outside any stream capture and before memory gets tight;
+ *     later calls on the device only read the cached address.  The address belongs to the
+ *     device's primary context: after cudaDeviceReset it is stale and this entry point must not
+ *     be used again in the process.
  *   - All calls on one device share the one array, which still holds what the previous call
  *     left; every call re-initialises the parts that must start from zero.  Two calls that
  *     overlap on the GPU (different streams, or different host threads) race on it: serialise them.

@@ -334,14 +334,14 @@ def wind_profile_decode(model: WindModel, enc, enc_len, W: int, max_symbols: int
 
 
 def wind_eval_joint_window(model: WindModel, enc, enc_len, W: int, prefix, prefix_len, t0, logits, workspace,
-                           stream=None) -> int:
+                           stream=None, check: bool = True) -> int:
     L = load_library()
     B, T, D = enc.shape
     U = prefix.shape[1] if prefix is not None and prefix.numel() else 0
     st = L.wind_eval_joint_window(model.ref, enc.data_ptr(), enc_len.data_ptr(), B, T, W,
                                   prefix.data_ptr() if U else None, U, prefix_len.data_ptr(), t0.data_ptr(),
                                   logits.data_ptr(), _ws_ptr(workspace), _ws_bytes(workspace), _stream_ptr(stream))
-    if st != WIND_OK:
+    if check and st != WIND_OK:
         raise WindError(st)
     return st
 

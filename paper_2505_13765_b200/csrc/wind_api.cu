@@ -301,10 +301,11 @@ wind_status_t wind_decode_greedy_host(const wind_model_t* m, const void* enc_hos
     int32_t* d_tok = reinterpret_cast<int32_t*>(ws + lay.st_tok);
     int32_t* d_frm = reinterpret_cast<int32_t*>(ws + lay.st_frm);
     int32_t* d_olen = reinterpret_cast<int32_t*>(ws + lay.st_olen);
+    for (int b = 0; b < B; ++b)
+        if (enc_len_host[b] < 0 || enc_len_host[b] > T) return WIND_ERR_INVALID_ARG;   // before anything is enqueued
     // only the valid frames of every utterance cross the bus (padding frames are never read for a decision)
     for (int b = 0; b < B; ++b) {
         const int len = enc_len_host[b];
-        if (len < 0 || len > T) return WIND_ERR_INVALID_ARG;
         if (len > 0)
             WIND_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(d_enc) + es * (size_t)b * T * m->D,
                                       static_cast<const uint8_t*>(enc_host) + es * (size_t)b * T * m->D, es * (size_t)len * m->D,

@@ -8,7 +8,7 @@ namespace wind {
 // Reset all per-call state.  Block 0 also fills the control block.
 __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsigned long long* t_pub, int32_t* count, int32_t* emit_tok,
                                                    unsigned long long* keys, float* h, float* c, uint32_t* hb, uint32_t* z,
-                                                   uint32_t* trace, size_t n_trace_words, int32_t* out_len, const int32_t* __restrict__ enc_len, int B, size_t n_keys,
+                                                   uint32_t* trace, size_t n_trace_words, int32_t* out_len, const int32_t* __restrict__ enc_len, int B, int T, size_t n_keys,
                                                    size_t n_h, size_t n_c, size_t n_hb_words, size_t n_z_words,
                                                    int blank, int step_cap, int kernels_used, int launches_per_step,
                                                    int launches_setup) {
@@ -29,14 +29,15 @@ __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsig
         out_len[i] = 0;
     }
     if (blockIdx.x == 0) {
-        __shared__ int s_active;
+        __shared__ int s_active, s_bad;
         __shared__ unsigned long long s_frames;
-        if (threadIdx.x == 0) { s_active = 0; s_frames = 0ull; }
+        if (threadIdx.x == 0) { s_active = 0; s_frames = 0ull; s_bad = 0; }
         __syncthreads();
         int a = 0;
         unsigned long long f = 0;
         for (int b = threadIdx.x; b < B; b += blockDim.x) {
             int len = enc_len[b];
+            if (len < 0 || len > T) s_bad = 1;   // a caller's mistake: nothing may be read through this length
             a += len > 0;
             f += (unsigned long long)(len > 0 ? len : 0);
         }
@@ -44,8 +45,9 @@ __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsig
         atomicAdd(&s_frames, f);
         __syncthreads();
         if (threadIdx.x == 0) {
-            ctrl->status = 0;
-            ctrl->active = s_active;
+            ctrl->status = s_bad ? WIND_ERR_INVALID_ARG : 0;
+            ctrl->bad_input = s_bad;
+            ctrl->active = s_bad ? 0 : s_active;
             ctrl->step = 0;
             ctrl->step_cap = step_cap;
             ctrl->joint_rows = 0;
@@ -56,7 +58,6 @@ __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsig
             ctrl->launches_per_step = launches_per_step;
             ctrl->launches_setup = launches_setup;
             ctrl->kernels = kernels_used;
-            ctrl->pad = 0;
             ctrl->bar = 0u;
             ctrl->abort = 0;
             for (int k = 0; k < 4; ++k) ctrl->phase_cycles[k] = 0;
@@ -80,7 +81,7 @@ cudaError_t launch_init(const Call& c, int kernels_used, int launches_per_step, 
     init_kernel<<<blocks, 256, 0, c.stream>>>(c.ctrl(), c.t(), c.t_pub(), c.count(), c.emit_tok(), c.keys(), c.h(0), c.c(),
                                               reinterpret_cast<uint32_t*>(c.hb(0, 0)), reinterpret_cast<uint32_t*>(c.z()),
                                               reinterpret_cast<uint32_t*>(c.trace()),
-                                              bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents / 4 : 0, c.out_len, c.enc_len, c.B, 3 * (size_t)c.lay.rows_pad, n_h, n_c, n_hb_words,
+                                              bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents / 4 : 0, c.out_len, c.enc_len, c.B, c.T, 3 * (size_t)c.lay.rows_pad, n_h, n_c, n_hb_words,
                                               n_z_words, c.m.blank_id, (int)step_cap, kernels_used, launches_per_step,
                                               launches_setup);
     return cudaGetLastError();
@@ -176,25 +177,41 @@ cudaError_t launch_control(const Call& c, cudaGraphConditionalHandle handle, int
     return cudaGetLastError();
 }
 
-// Teacher forcing (wind_eval_joint_window): token u of each prefix, -1 past its end.
+// Teacher forcing (wind_eval_joint_window): token u of each prefix, -1 past its end.  A token outside [0, V] is a
+// caller's mistake: the blank is fed instead and the call reports WIND_ERR_INVALID_ARG.
 __global__ void force_tokens_kernel(Ctrl* ctrl, int32_t* emit_tok, const int32_t* __restrict__ prefix, int U,
-                                    const int32_t* __restrict__ prefix_len, int u, int B) {
+                                    const int32_t* __restrict__ prefix_len, int u, int B, int NV, int blank) {
     int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b == 0) ctrl->active = B;
-    if (b < B) emit_tok[b] = (u < prefix_len[b]) ? prefix[(size_t)b * U + u] : -1;
+    if (b == 0 && !ctrl->bad_input) ctrl->active = B;
+    if (b < B) {
+        int tok = (u < prefix_len[b]) ? prefix[(size_t)b * U + u] : -1;
+        if (tok >= NV || tok < -1) { tok = blank; set_status(ctrl, WIND_ERR_INVALID_ARG); }
+        emit_tok[b] = tok;
+    }
 }
 cudaError_t launch_force_tokens(const Call& c, const int32_t* prefix, int U, const int32_t* prefix_len, int u) {
-    force_tokens_kernel<<<(c.B + 127) / 128, 128, 0, c.stream>>>(c.ctrl(), c.emit_tok(), prefix, U, prefix_len, u, c.B);
+    force_tokens_kernel<<<(c.B + 127) / 128, 128, 0, c.stream>>>(c.ctrl(), c.emit_tok(), prefix, U, prefix_len, u, c.B, c.m.V + 1,
+                                                                 c.m.blank_id);
     return cudaGetLastError();
 }
 
-__global__ void set_t_kernel(Ctrl* ctrl, int32_t* t, const int32_t* __restrict__ t0, int B) {
+// Window start of every utterance (teacher forcing, beam search).  A start outside [0, len] is a caller's mistake: it
+// is moved inside, so that nothing is read out of range, and the call reports WIND_ERR_INVALID_ARG.
+__global__ void set_t_kernel(Ctrl* ctrl, int32_t* t, const int32_t* __restrict__ t0, const int32_t* __restrict__ enc_len, int B) {
     int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b == 0) ctrl->active = B;
-    if (b < B) { t[b] = t0[b]; t[B + b] = t0[b]; }
+    if (b == 0 && !ctrl->bad_input) ctrl->active = B;
+    if (b < B) {
+        int v = t0[b];
+        if (enc_len) {
+            const int len = enc_len[b] > 0 ? enc_len[b] : 0;
+            if (v < 0 || v > len) { v = v < 0 ? 0 : len; set_status(ctrl, WIND_ERR_INVALID_ARG); }
+        }
+        t[b] = v;
+        t[B + b] = v;
+    }
 }
 cudaError_t launch_set_t(const Call& c, const int32_t* t0) {
-    set_t_kernel<<<(c.B + 127) / 128, 128, 0, c.stream>>>(c.ctrl(), c.t(), t0, c.B);
+    set_t_kernel<<<(c.B + 127) / 128, 128, 0, c.stream>>>(c.ctrl(), c.t(), t0, c.enc_len, c.B);
     return cudaGetLastError();
 }
 

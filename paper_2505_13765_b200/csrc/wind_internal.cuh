@@ -40,7 +40,7 @@ struct Ctrl {
     int32_t launches_per_step;
     int32_t launches_setup;
     int32_t kernels;
-    int32_t pad;
+    int32_t bad_input;  // set by the init kernel: a length outside [0, T]; the loops then do not start
     // persistent loop kernel
     uint32_t bar;             // grid barrier: arrivals so far (monotonic within a call)
     int32_t abort;            // some CTA gave up: everybody leaves

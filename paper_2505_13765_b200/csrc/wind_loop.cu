@@ -173,6 +173,8 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cta = blockIdx.x, G = gridDim.x;
+    // a length outside [0, T] (found by the init kernel, which ran before this launch): the status is set, no CTA starts
+    if (p.ctrl->bad_input) return;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* stat = smem;                       // W_out tile kept in shared memory (J_SMEM): kb_h blocks of 128 x 64 bf16
     uint8_t* ring = smem + p.stat_bytes;        // operand stages; geometry differs per phase, drained in between
@@ -412,6 +414,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     tok = p.blank;
                 } else if ((FULL && p.forced)) {
                     tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
+                    if (tok >= p.NV || tok < -1) { tok = p.blank; set_status(p.ctrl, WIND_ERR_INVALID_ARG); }   // caller's mistake
                 } else if (l > 0) {
                     tok = p.emit_tok[b];
                 } else {
@@ -651,6 +654,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     tok = p.blank;
                 } else if ((FULL && p.forced)) {
                     tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
+                    if (tok >= p.NV || tok < -1) { tok = p.blank; set_status(p.ctrl, WIND_ERR_INVALID_ARG); }   // caller's mistake
                 } else if (layer > 0) {
                     tok = p.emit_tok[b];     // decided by layer 0's CTAs one phase earlier
                 } else {

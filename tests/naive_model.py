@@ -66,3 +66,65 @@ def random_weights(rng, D, E, P, L, H, V, blank_id=None, act=0, blank_bias=0.0, 
         elif isinstance(v, list):
             w[k] = [a.astype(np.float32) for a in v]
     return w
+
+
+# ---------------------------------------------------------------------------
+# A model whose logits are set by hand, with EXACT ties, to pin the argmax tie rule (lowest index wins).
+# ---------------------------------------------------------------------------
+TIE_TYPES = 9   # frame types of tie_model
+
+
+def tie_model(V=299, blank_id=None, dim=64, dtype="f32"):
+    """Frame type k (a one-hot encoder frame) gives label v the logit target[v, k], whatever the decoder state:
+    W_enc = identity, W_pred = 0, ReLU, so z is the one-hot frame and logits = W_out[:, k] + b_out.  Every value is a
+    small dyadic number, exact in bf16 and in any summation order, so equal targets are equal logits bit for bit.
+    Biases differ per label (W_out compensates), so that the tie only exists after the bias is added.
+    Returns (weights, target, winners): winners[k] = lowest index among the maxima of type k (the expected argmax)."""
+    blank_id = V if blank_id is None else blank_id
+    NV = V + 1
+    assert NV >= 300 and dim >= TIE_TYPES and blank_id in (0, V)
+    lo, hi = -1.0, 2.0
+    tied = [
+        [3, 17],                 # two labels inside one group of 32 consecutive entries
+        [3, 40],                 # same 128-entry tile, different groups of 32
+        [70, 200],               # different 128-entry tiles
+        [200, blank_id],         # a label and the blank
+        [5, blank_id],           # a label and the blank, the label in the first tile
+        [blank_id],              # blank alone: no tie
+        [298],                   # one label alone: no tie
+        [10, 130, 260],          # three tiles
+        list(range(NV)),         # every entry equal
+    ]
+    target = np.full((NV, dim), lo, np.float64)
+    for k, labels in enumerate(tied):
+        target[labels, k] = hi
+    b_out = np.array([(-0.5, 0.0, 0.25, 0.5)[v % 4] for v in range(NV)], np.float64)
+    w_out = target - b_out[:, None]
+    winners = [min(labels) for labels in tied]
+    z = lambda *s: np.zeros(s, np.float32)
+    w = dict(D=dim, E=dim, P=dim, L=1, H=dim, V=V, blank_id=blank_id, act=0, dtype=dtype, emb=z(NV, dim),
+             w_ih=[z(4 * dim, dim)], w_hh=[z(4 * dim, dim)], b_ih=[z(4 * dim)], b_hh=[z(4 * dim)],
+             w_enc=np.eye(dim, dtype=np.float32), b_enc=z(dim), w_pred=z(dim, dim), b_pred=z(dim),
+             w_out=w_out.astype(np.float32), b_out=b_out.astype(np.float32))
+    return w, target, winners
+
+
+def tie_utterances(dim, types_per_utt):
+    """One-hot encoder frames for lists of frame types; returns (enc [B, T, dim] zero padded, lens)."""
+    T = max(len(u) for u in types_per_utt)
+    enc = np.zeros((len(types_per_utt), T, dim), np.float32)
+    for b, u in enumerate(types_per_utt):
+        for t, k in enumerate(u):
+            enc[b, t, k] = 1.0
+    return enc, np.array([len(u) for u in types_per_utt], np.int32)
+
+
+def tie_expected(types, winners, blank_id, S):
+    """Algorithm 1 written out for the tie model: the decision on a frame never depends on the decoder, so a frame
+    whose winner is a label emits it S times (the S-th emission forces the advance) and a blank frame emits nothing."""
+    tok, frm = [], []
+    for t, k in enumerate(types):
+        if winners[k] != blank_id:
+            tok += [winners[k]] * S
+            frm += [t] * S
+    return tok, frm

@@ -14,7 +14,7 @@ import pytest
 
 import oracle
 import wind_synth as ws
-from naive_model import random_weights
+from naive_model import random_weights, tie_expected, tie_model, tie_utterances
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -231,6 +231,45 @@ def test_bf16_joint_logits(pkg, kernels, name, W):
                   kernels=kernels)
 
 
+def test_bf16_joint_logits_after_a_long_prefix(pkg):
+    # The tensor path rounds the hidden state to bf16 at every update and feeds it back; this checks that the
+    # recurrence has not drifted after several hundred updates: windows of the 100 s utterance (large model)
+    # evaluated behind oracle prefixes of 500 to 3000 tokens, same tolerance as everywhere else.
+    cfg = ws.CONFIGS["cfg2_large_b1"]
+    weights = ws.make_model(cfg)
+    enc, lens = ws.make_enc(cfg, pad="nan")
+    om = oracle.Model(weights)
+    otok, ofrm, on, _ = oracle.decode_batch(om, enc, lens, W=0, S=cfg.S)
+    assert on[0] > 3000
+    T = int(lens[0])
+    W = 8
+    prev = pkg.wind_set_kernels(2)
+    try:
+        model = pkg.WindModel(weights)
+        d = model.device
+        enc_d = pkg.to_device_enc(model, enc)
+        wsb = pkg.alloc_workspace(model, 1, T, W)
+        worst = 0.0
+        for want in (500, 1200, 3000):
+            t0 = int(ofrm[0, want])                         # a frame reached after about `want` tokens
+            plen = int(np.searchsorted(ofrm[0, : on[0]], t0, side="left"))
+            assert plen >= want - 10 * cfg.S
+            prefix = np.ascontiguousarray(otok[:, :plen])
+            logits = torch.full((1, W, cfg.V + 1), float("nan"), dtype=torch.float32, device=d)
+            pkg.wind_eval_joint_window(model, enc_d, torch.from_numpy(lens).to(d), W, torch.from_numpy(prefix).to(d),
+                                       torch.tensor([plen], dtype=torch.int32, device=d),
+                                       torch.tensor([t0], dtype=torch.int32, device=d), logits, wsb)
+            ref, *_ = oracle.eval_joint_window(om, enc[0], T, prefix[0], t0, W)
+            n = ref.shape[0]
+            assert n == min(W, T - t0) and n > 0
+            err = float(np.max(np.abs(logits.cpu().numpy()[0, :n].astype(np.float64) - ref)))
+            print(f"[long prefix] {plen} tokens fed, window at frame {t0}: worst abs logit error {err:.3e}")
+            worst = max(worst, err)
+        assert worst < TOL["bf16"]
+    finally:
+        pkg.wind_set_kernels(prev)
+
+
 @pytest.mark.parametrize("L,blank0,act,B,W", [(1, True, 1, 9, 4), (1, False, 0, 70, 8), (2, True, 0, 5, 16), (2, False, 1, 33, 2)])
 def test_bf16_tensor_path_with_biases_and_other_blank_ids(pkg, L, blank0, act, B, W):
     # tile-sized dimensions, so the tensor-core kernels run (weights resident in shared memory, for one and for two
@@ -356,6 +395,39 @@ def test_bf16_tensor_path_is_window_invariant_on_the_gpu(pkg):
             assert np.array_equal(tok, ref[0]) and np.array_equal(frm, ref[1]), W
 
 
+TIE_UTTS = [[5, 0, 5, 5, 1, 2, 3, 4, 5, 6, 7, 8, 5], [8, 7, 6, 5, 5, 5, 5, 5, 5, 5, 4, 3, 2, 1, 0], [3], [5, 5, 4],
+            [2, 2, 3, 3, 4, 4, 8, 8], [], [0, 1, 2, 3, 4, 5, 6, 7, 8] * 3]
+
+
+@pytest.mark.parametrize("path", ["f32", "bf16_simt", "bf16_tensor", "bf16_tensor_streaming"])
+@pytest.mark.parametrize("blank_first", [False, True])
+def test_argmax_ties_go_to_the_lowest_index_on_the_gpu(pkg, monkeypatch, path, blank_first):
+    # Logits with exact ties by construction: two labels in one group of 32 vocabulary entries (one warp of the
+    # tensor path's epilogue), in different groups of one 128-entry tile, in different tiles (combined through the
+    # 64-bit keys), a label against the blank, and every entry equal.  The expected transcripts are written from the
+    # rule (lowest index wins), and the oracle must give the same.
+    if path == "bf16_tensor_streaming":
+        monkeypatch.setenv("WIND_RESIDENT", "0")
+    w, target, winners = tie_model(blank_id=0 if blank_first else None, dtype="f32" if path == "f32" else "bf16")
+    blank = w["blank_id"]
+    enc, lens = tie_utterances(w["D"], TIE_UTTS)
+    kernels = {"f32": 0, "bf16_simt": 1}.get(path, 2)
+    prev = pkg.wind_set_kernels(kernels)
+    try:
+        model = pkg.WindModel(w)
+        om = oracle.Model(w)
+        for W, S in ((1, 1), (4, 1), (8, 2), (16, 1)):
+            tok, frm, olen, stats, st = pkg.decode(model, enc, lens, W, S)
+            assert st == 0 and stats["kernels"] == (2 if kernels == 2 else 1)
+            otok, ofrm, on, _ = oracle.decode_batch(om, enc, lens, W=0, S=S)
+            for b, types in enumerate(TIE_UTTS):
+                want_tok, want_frm = tie_expected(types, winners, blank, S)
+                assert list(tok[b, : olen[b]]) == want_tok and list(frm[b, : olen[b]]) == want_frm, (W, S, b)
+                assert list(otok[b, : on[b]]) == want_tok and list(ofrm[b, : on[b]]) == want_frm
+    finally:
+        pkg.wind_set_kernels(prev)
+
+
 def test_loop_kernel_timeline_can_be_recorded_without_changing_results(pkg):
     cfg = ws.small_variant(ws.CONFIGS["cfg3_large_b128"], 8, 30, 80)
     weights = ws.make_model(cfg)
@@ -479,6 +551,57 @@ def test_unfillable_barrier_ends_in_timeout_status_and_the_context_stays_usable(
     assert again[4] == 0
     for a, b in zip(again[:3], ref[:3]):
         assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_device_side_inputs_out_of_range_are_reported_not_read(pkg, dtype):
+    # enc_len, prefix tokens and window starts live on the device; the kernels check them there: a length outside
+    # [0, T] stops the decode before any frame is read through it, a bad token or window start is replaced by a safe
+    # value, and the call returns WIND_ERR_INVALID_ARG.  The next correct call on the same workspace is unaffected.
+    dims = dict(D=64, E=64, P=64, L=1, H=64, V=140) if dtype == "bf16" else dict(D=20, E=12, P=24, L=2, H=40, V=30)
+    w, enc, lens = ragged_case(96, B=6, T=30, bias=1.0, dtype=dtype, **dims)
+    enc = np.nan_to_num(enc)
+    model = pkg.WindModel(w)
+    INVALID = pkg.binding.WIND_ERR_INVALID_ARG
+    ref = pkg.decode(model, enc, lens, 4, 3)
+    assert ref[4] == 0 and ref[3]["kernels"] == (2 if dtype == "bf16" else 1)
+    for bad_len in (31, -1, 2 ** 30):
+        bad = lens.copy()
+        bad[5] = bad_len
+        out = pkg.decode(model, enc, bad, 4, 3, check=False)
+        assert out[4] == INVALID and int(out[2].sum()) == 0
+    again = pkg.decode(model, enc, lens, 4, 3)
+    assert again[4] == 0
+    for a, b in zip(again[:3], ref[:3]):
+        assert np.array_equal(a, b)
+    # teacher forcing
+    d = model.device
+    B, T, _ = enc.shape
+    enc_d = pkg.to_device_enc(model, enc)
+    wsb = pkg.alloc_workspace(model, B, T, 4)
+    logits = torch.zeros((B, 4, dims["V"] + 1), dtype=torch.float32, device=d)
+    lens_d = torch.from_numpy(lens).to(d)
+    prefix = np.ones((B, 2), np.int32)
+    plen = np.full(B, 2, np.int32)
+    t0 = np.zeros(B, np.int32)
+
+    def call(prefix, t0, lens_t=lens_d):
+        pr, pl, tt = (torch.from_numpy(a).to(d) for a in (prefix, plen, t0))
+        return pkg.wind_eval_joint_window(model, enc_d, lens_t, 4, pr, pl, tt, logits, wsb, check=False)
+
+    assert call(prefix, t0) == 0
+    for tok in (dims["V"] + 1, -7, 2 ** 30):
+        bad = prefix.copy()
+        bad[3, 1] = tok
+        assert call(bad, t0) == INVALID
+    for start in (-1, T + 5):
+        bad = t0.copy()
+        bad[0] = start
+        assert call(prefix, bad) == INVALID
+    bad_lens = lens.copy()
+    bad_lens[2] = T + 1
+    assert call(prefix, t0, torch.from_numpy(bad_lens).to(d)) == INVALID
+    assert call(prefix, t0) == 0
 
 
 def test_workspace_too_small_is_rejected(pkg):

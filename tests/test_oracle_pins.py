@@ -17,7 +17,7 @@ import pytest
 import torch
 
 import oracle
-from naive_model import NaiveModel, random_weights
+from naive_model import NaiveModel, random_weights, tie_expected, tie_model, tie_utterances
 
 
 def rng(seed):
@@ -563,6 +563,41 @@ def test_window_replay_accepts_own_output_and_rejects_mistakes():
     # with a margin above the gap the first decision passes (whatever happens at the second one)
     res = oracle.replay_verify_window(m, enc[b], T, W, 3, tk4[:1], fr[:1], margin_thr=gap * 1.01)
     assert res["decisions"] >= 2 and res["not_argmax"] >= 1
+
+
+# ---------------------------------------------------------------------------
+# argmax tie rule: lowest index wins (the paper is silent; the reading is fixed here by exact ties)
+# ---------------------------------------------------------------------------
+TIE_UTTS = [[5, 0, 5, 5, 1, 2, 3, 4, 5, 6, 7, 8, 5], [8, 7, 6, 5, 5, 5, 5, 5, 5, 5, 4, 3, 2, 1, 0], [3], [5, 5, 4],
+            [2, 2, 3, 3, 4, 4, 8, 8], []]
+
+
+@pytest.mark.parametrize("blank_first", [False, True])
+@pytest.mark.parametrize("S", [1, 2])
+def test_argmax_ties_go_to_the_lowest_index(blank_first, S):
+    # Exact ties by construction (dyadic logits, ties only after the bias is added).  Expected winners are written
+    # down from the rule, not computed by the oracle: two labels -> the lower label; a label and the blank -> the
+    # label when the blank is the last index, the blank when it is index 0; everything equal -> index 0.
+    w, target, winners = tie_model(blank_id=0 if blank_first else None)
+    blank = w["blank_id"]
+    if blank_first:
+        assert winners == [3, 3, 70, 0, 0, 0, 298, 10, 0]
+    else:
+        assert winners == [3, 3, 70, 200, 5, 299, 298, 10, 0]
+    enc, lens = tie_utterances(w["D"], TIE_UTTS)
+    m = oracle.Model(w)
+    # the logits really are the hand-set targets, ties included
+    lg, *_ = oracle.eval_joint_window(m, enc[0], int(lens[0]), [], 0, 13)
+    for j, k in enumerate(TIE_UTTS[0]):
+        assert np.array_equal(lg[j], target[:, k])
+    for W in (0, 1, 2, 4, 8, 16):     # 0: Algorithm 1 as written; the others Algorithm 2
+        tok, frm, n, st = oracle.decode_batch(m, enc, lens, W=W, S=S)
+        for b, types in enumerate(TIE_UTTS):
+            want_tok, want_frm = tie_expected(types, winners, blank, S)
+            assert list(tok[b, : n[b]]) == want_tok and list(frm[b, : n[b]]) == want_frm, (W, b)
+    # the opposite rule (highest index on ties) would give something else on these inputs
+    other = [int(np.flatnonzero(target[:, k] == target[:, k].max())[-1]) for k in range(len(winners))]
+    assert tie_expected(TIE_UTTS[0], other, blank, S) != tie_expected(TIE_UTTS[0], winners, blank, S)
 
 
 # ---------------------------------------------------------------------------

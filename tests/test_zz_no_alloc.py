@@ -4,8 +4,10 @@ Some users of the library run where cudaMalloc (and torch's allocator) must not 
 section that may not synchronise the device, inside a process whose device memory is already
 handed out, or in a loop with a hard latency bound.  ``wind_eval_joint_window_static`` serves
 them from a scratch array built into the library.  This file checks it, through the C ABI,
-against ``wind_eval_joint_window`` (caller-allocated workspace) on the same inputs, twice in a row
-with different inputs, so that anything the first call left in the shared array would show.
+against ``wind_eval_joint_window`` (caller-allocated workspace) and against the CPU oracle on the
+same inputs, twice in a row with different inputs, so that anything the first call left in the
+shared array would show, and checks that the device's free memory is the same after a call as
+before it (the first call on a device may load the library's image and is not measured).
 
 Collected last on purpose: a run that stops at the first failure has then already run every
 other test.
@@ -13,6 +15,7 @@ other test.
 import numpy as np
 import pytest
 
+import oracle
 import wind_synth as ws
 from naive_model import random_weights
 
@@ -69,10 +72,26 @@ def _both(pkg, case, W):
     wsb = pkg.alloc_workspace(model, B, T, W)
     pkg.wind_eval_joint_window(model, enc_d, args[0], W, args[1], args[2], args[3], ref, wsb)
     got = torch.full((B, W, NV), float("nan"), dtype=torch.float32, device=d)
-    # everything the call needs is allocated by now; the call itself allocates nothing
+    # everything the call needs is allocated by now; the call itself allocates nothing.  One untimed call first:
+    # the very first use on a device resolves the array's address (and may load the library's image).
     pkg.wind_eval_joint_window_static(model, enc_d, args[0], W, args[1], args[2], args[3], got)
     torch.cuda.synchronize()
-    return ref.cpu().numpy(), got.cpu().numpy(), lens, t0
+    got.fill_(float("nan"))
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info(d)
+    reserved_before = torch.cuda.memory_reserved(d)
+    pkg.wind_eval_joint_window_static(model, enc_d, args[0], W, args[1], args[2], args[3], got)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info(d)
+    assert torch.cuda.memory_reserved(d) == reserved_before      # nothing taken from torch's allocator
+    assert free_after >= free_before, (free_before, free_after)   # nothing taken from the device
+    # the oracle's logits of the same windows
+    om = oracle.Model(w)
+    want = []
+    for b in range(B):
+        o, *_ = oracle.eval_joint_window(om, enc[b], int(lens[b]), prefix[b, : plen[b]], int(t0[b]), W)
+        want.append(o)
+    return ref.cpu().numpy(), got.cpu().numpy(), lens, t0, want
 
 
 @pytest.mark.parametrize("dtype,dims", [
@@ -82,13 +101,16 @@ def _both(pkg, case, W):
 def test_static_scratch_matches_caller_workspace_twice_in_a_row(pkg, dtype, dims):
     W = 4
     for call, seed in enumerate((1, 2)):  # second call: other weights and inputs, same shared array
-        ref, got, lens, t0 = _both(pkg, _case(seed, dtype, **dims), W)
+        ref, got, lens, t0, want = _both(pkg, _case(seed, dtype, **dims), W)
         rows = 0
         for b in range(ref.shape[0]):
             n = max(0, min(W, int(lens[b]) - int(t0[b])))
             rows += n
+            assert want[b].shape[0] == n
             assert np.all(np.isfinite(ref[b, :n]))
             assert np.max(np.abs(got[b, :n] - ref[b, :n])) <= TOL[dtype], (call, b)
+            if n:
+                assert np.max(np.abs(got[b, :n].astype(np.float64) - want[b])) <= TOL[dtype], (call, b)
             assert np.all(np.isnan(got[b, n:])) and np.all(np.isnan(ref[b, n:]))  # rows past the window untouched
         assert rows > 0
 

@@ -185,7 +185,11 @@ def make_enc(cfg: WindConfig, pad: str = "nan", seed_offset: int = 0) -> Tuple[n
     fill = {"nan": np.nan, "zero": 0.0}[pad]
     enc = np.full((cfg.B, cfg.T, cfg.D), fill, dtype=np.float32)
     for b in range(cfg.B):
-        n = int(lens[b])
-        x = _normal(cfg.seed + seed_offset, 1000 + b, (n, cfg.D), 1.0)
-        enc[b, :n] = bf16_round(x) if cfg.dtype == "bf16" else x
+        enc[b, : int(lens[b])] = make_utterance(cfg, b, int(lens[b]), seed_offset)
     return enc, lens
+
+
+def make_utterance(cfg: WindConfig, b: int, n: int, seed_offset: int = 0) -> np.ndarray:
+    """The ``n`` valid frames ``[n, D]`` of utterance ``b`` (the rows ``make_enc`` puts at ``enc[b, :n]``)."""
+    x = _normal(cfg.seed + seed_offset, 1000 + b, (n, cfg.D), 1.0)
+    return bf16_round(x) if cfg.dtype == "bf16" else x
