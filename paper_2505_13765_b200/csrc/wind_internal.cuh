@@ -67,12 +67,15 @@ struct Layout {
     size_t dh;         // fp32 [B][4P] layer 1's recurrent term, handed from its CTAs to the layer's update (tensor path, L >= 2)
     size_t g0;         // fp32 [V+1][4P] layer-0 gate pre-activations of every token: W_ih emb[tok] + b_ih + b_hh (tensor path)
     size_t trace;      // TraceEvent [kTraceRoles][kTraceEvents]: optional timeline of CTA 0 of the loop kernel
+    size_t flags;      // uint32 [n_flags] arrival counters between CTA groups of the resident-weights loop kernel
+    size_t pred_pub;   // (fp32, uint32) [B][H] pred_proj values, each stamped with the projection phase that wrote it
     size_t enc_proj;   // elem [B*T][H]
     size_t total;
     // host staging (wind_decode_greedy_host), placed after `total`
     size_t st_enc, st_len, st_tok, st_frm, st_olen, st_total;
     int32_t Bpad;      // B rounded up to 128 (tensor path operand rows)
     int32_t rows_pad;  // B*W rounded up to 256 (window rows incl. tile padding)
+    int32_t n_flags;   // one counter per 16 window rows and three per 16 utterances always suffice
 };
 
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -101,6 +104,9 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     L.trace = take(bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents : 0);
     L.jpart = take(bf ? sizeof(float) * 2 * (size_t)L.rows_pad * 4 * ((size_t)(m.V + 1 + 127) / 128) : 0);
     L.jblank = take(bf ? sizeof(float) * (size_t)L.rows_pad : 0);
+    L.n_flags = L.rows_pad / 16 + 3 * (B / 16 + 1);
+    L.flags = take(bf ? sizeof(uint32_t) * (size_t)L.n_flags : 0);
+    L.pred_pub = take(bf ? 8 * (size_t)B * m.H : 0);
     L.enc_proj = take(es * (size_t)B * T * m.H);
     L.total = off;
     L.st_enc = take(es * (size_t)B * T * m.D);
@@ -149,6 +155,8 @@ struct Call {
     float2* jpart() const { return reinterpret_cast<float2*>(ws + lay.jpart); }
     float* jblank() const { return reinterpret_cast<float*>(ws + lay.jblank); }
     TraceEvent* trace() const { return reinterpret_cast<TraceEvent*>(ws + lay.trace); }
+    uint32_t* flags() const { return reinterpret_cast<uint32_t*>(ws + lay.flags); }
+    unsigned long long* pred_pub() const { return reinterpret_cast<unsigned long long*>(ws + lay.pred_pub); }
     __nv_bfloat16* hb(int parity, int l) const {
         return reinterpret_cast<__nv_bfloat16*>(ws + lay.hb) + ((size_t)parity * m.L + l) * lay.Bpad * m.P;
     }

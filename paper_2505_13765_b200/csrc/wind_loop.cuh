@@ -25,7 +25,6 @@ struct LoopMaps {
     CUtensorMap hb_l3[2];              // layer 0 state [Bpad, P] as (64, rows, P/64), box (64, nl, P/64)
     CUtensorMap hb_l3_1[2];            // layer 1 state, same box
     CUtensorMap hb_p3[2];              // same, box (64, np, P/64)
-    CUtensorMap z3;                    // [rows_pad, H] as (64, rows, H/64), box (64, nj, H/64)
 };
 
 // How the three phases are cut into items and how shared memory is used (host-chosen).
@@ -43,6 +42,8 @@ struct LoopPlan {
     int resident, nl, ut_count, ht_count, ql_count, qp_count;
     int w_first, w_count;                  // step-recording CTAs [w_first, w_first + w_count), 64 utterances each (0: the L CTAs record)
     uint32_t buf_off, stage_off;           // the per-step operand buffer and the epilogue staging area (after the tile)
+    uint32_t z_off, z_off_p;               // resident mode: the joint's operand buffer (z_off_p: in CTAs with a W_pred tile);
+                                           // equal to buf_off where it shares the state box's memory
     int slots, ul, ug_count, mt_count, l_items;  // decoder: rows per gate block, units per item, unit groups, utterance tiles
     int np, hg_count, p_items;             // projection: H columns per item, H slices
     int stages_lp, stages_j;               // ring stages in the decoder/projection phases and in the joint phase
@@ -57,7 +58,7 @@ struct LoopParams {
     int tm_j, tm_l, tm_p, l_early;
     int resident, nl, ut_count, ht_count, ql_count, qp_count;
     int w_first, w_count;
-    uint32_t buf_off, stage_off;
+    uint32_t buf_off, stage_off, z_off, z_off_p;
     int slots, ul, ug_count, mt_count, l_items;
     int np, hg_count, p_items;
     int kb_h, kb_p;
@@ -97,10 +98,19 @@ struct LoopParams {
     unsigned long long* nbkeys;    // [rows_pad] best non-blank (logit, label) per window row
     float2* jpart;                 // [rows_pad][parts]
     float* jblank;                 // [rows_pad] blank logit per window row
-    int extra_arrivals;            // test hook: arrivals the grid barrier waits for beyond the grid size (0 in normal use)
+    int extra_arrivals;            // test hook: arrivals the first cross-CTA wait asks for beyond those that come (0 in normal use)
+    // resident-weights mode: arrival counters between CTA groups (keys of a row group complete, state of an utterance
+    // group written, ...) and the stamped pred_proj values
+    uint32_t* flags;
+    unsigned long long* pred_pub;  // [B][H] (fp32 value, stamp)
 };
 
 cudaError_t loop_plan(const Call& c, LoopPlan* out);
+// the plan as a pure function of the shapes and of the device's SM count and opt-in shared memory per block
+cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem_optin, LoopPlan* out);
+// launchers of the two kernels (wind_loop.cu: streaming mode; wind_loop_res.cu: resident-weights mode)
+cudaError_t loop_res_set_smem(int bytes);
+cudaError_t loop_res_launch(const LoopMaps& maps, const LoopParams& p, int grid, uint32_t smem_bytes, bool full, cudaStream_t stream);
 int loop_set_extra_arrivals(int n);  // returns the previous value
 cudaError_t loop_prepare(Call& c);   // plan + tensor maps + shared-memory opt-in (host only; not inside a capture)
 

@@ -1,0 +1,1004 @@
+// The decoding loop of the bf16 path, resident-weights mode (sm_100a): ONE persistent cooperative kernel in which
+// every weight matrix stays on chip for the whole decode and the CTAs hand results to one another through
+// per-group arrival counters and stamped data instead of grid-wide barriers.
+//
+// One CTA per SM.  A lock step of the batch (Algorithm 2 applied to every utterance at once) is three slots,
+// each a tensor-core GEMM with the weights as the stationary operand (M axis) and utterances / window rows on N:
+//
+//   J  joint      logits^T [128 vocabulary entries, nj window rows] = W_out tile . z^T.  The W_out tile lives in
+//                 TENSOR MEMORY (the A operand of tcgen05.mma) for the whole decode.  The CTA builds its own operand
+//                 z = act(enc_proj[b, t_b + w, :] + pred_proj[b, :]) in shared memory: the enc_proj rows of the row
+//                 group's utterances are copied in (cp.async, 128-byte swizzled K-major layout) as soon as the
+//                 control step has published the next frame, pred_proj arrives as stamped (value, stamp) pairs that
+//                 the CTA polls, the sum is activated in place.  Epilogue: per-row argmax over the tile's 128
+//                 entries by warp shuffles, 64-bit atomicMax of (logit, label) keys across the vocabulary tiles;
+//                 the logits never leave the chip.  Then one arrival on the row group's counter.
+//   L  decoder    gates [4 gates x 16 units, nl utterances] = W_hh tile . h^T, tile resident in shared memory.  The
+//                 GEMM needs only the state, so it is issued a slot ahead and its result waits in tensor memory; the
+//                 slot itself is: wait for the keys of the CTA's utterances (their row groups' counters), control
+//                 step (Algorithm 2's branch: first non-blank row of the window, jump, emission, max-symbols rule),
+//                 gate-table rows of the chosen tokens, LSTM cell update, new h (bf16) and c (fp32), one arrival on
+//                 the utterance group's counter.  CTAs without a weight tile record the steps (outputs, counters,
+//                 next frame, published at once as a stamped word per utterance).  With two layers, layer 1's input
+//                 GEMM runs on CTAs holding a W_ih[1] tile after layer 0's arrivals, its recurrent term a slot ahead
+//                 on CTAs holding a W_hh[1] tile.
+//   P  projection pred_proj [64 H rows, np utterances] = W_pred tile . h_top^T + b_pred after the state counters of
+//                 its utterances have filled; written as (fp32 value, stamp) pairs, which is what the joint CTAs poll.
+//
+// No CTA waits for the whole grid: utterances are independent (Algorithm 2 has no cross-utterance term), so a joint
+// CTA waits only for the pred_proj of its row group's utterances, a decoder CTA for the vocabulary tiles of its own
+// utterances' rows, a projection CTA for the unit tiles of its own utterance group.  Every wait is bounded (about two
+// seconds): a CTA that gives up flags WIND_ERR_TIMEOUT, raises the global abort word, and every CTA leaves at its next
+// wait and frees its tensor memory.  Roles per CTA: warp 0 issues TMA, warps 0 and 1 issue tcgen05.mma (half of the K
+// blocks each, into separate accumulators that the epilogue adds), warps 2..9 run the epilogues and build the operand.
+//
+// FULL: teacher forcing with the logits store (wind_eval_joint_window), window-based decoding (which keeps two grid
+// barriers around its decision phase) and the timeline records; a plain decode launches the smaller variant.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "wind_loop_dev.cuh"
+
+namespace wind {
+
+constexpr int kGroupUtts = 96;   // utterances one joint row group can touch (at most 96 rows, window >= 1)
+constexpr int kPrepItems = 3;    // (utterance, 16-byte chunk) items a thread finishes per round of the operand build
+
+__device__ __forceinline__ void ld_acquire_v2_u64(const unsigned long long* p, unsigned long long& a, unsigned long long& b) {
+    asm volatile("ld.acquire.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void st_relaxed_v2_u64(unsigned long long* p, unsigned long long a, unsigned long long b) {
+    asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(a), "l"(b) : "memory");
+}
+__device__ __forceinline__ unsigned long long stamped(float v, uint32_t stamp) {
+    return ((unsigned long long)stamp << 32) | (unsigned long long)__float_as_uint(v);
+}
+
+template <bool FULL>
+__global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __grid_constant__ LoopMaps M, const LoopParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[2], empty_bar[2], stat_bar;   // [0]: the state box, [1]: the joint's operand
+    __shared__ uint64_t acc_full[3], acc_empty[3];             // accumulators: joint, decoder, projection
+    __shared__ uint32_t tmem_slot;
+    __shared__ int s_abort;      // this CTA has given up (1: a wait of its own ran out, 2: it saw the global abort word)
+    __shared__ int s_active;     // utterances still decoding (set in the projection slot)
+    __shared__ float win_lpb[FULL ? kMaxWindow : 1], win_sc[FULL ? kMaxWindow : 1];
+    __shared__ unsigned long long win_key[FULL ? kMaxWindow : 1];
+    __shared__ int s_jt[kGroupUtts], s_jrem[kGroupUtts];       // operand build: frame and frames left of the group's utterances
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cta = blockIdx.x, G = gridDim.x;
+    // a length outside [0, T] (found by the init kernel, which ran before this launch): the status is set, no CTA starts
+    if (p.ctrl->bad_input) return;
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* stat = smem;                       // this CTA's resident weight tile: kb_p blocks of 64 rows x 64 columns
+    uint8_t* buf0 = smem + p.buf_off;           // the per-step state box
+    float* stage_f = reinterpret_cast<float*>(smem + p.stage_off);   // epilogue staging
+    volatile int* vabort = &s_abort;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        s_active = 1;
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 2);      // two threads issue the MMAs of a GEMM, both commit
+        }
+        mbar_init(&stat_bar, 1);
+        for (int k = 0; k < 3; ++k) {
+            mbar_init(&acc_full[k], 2);
+            mbar_init(&acc_empty[k], 8);      // one arrival per epilogue warp
+        }
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc(&tmem_slot, LOOP_TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    const uint32_t tm_j = tmem_base + (uint32_t)p.tm_j, tm_l = tmem_base + (uint32_t)p.tm_l, tm_p = tmem_base + (uint32_t)p.tm_p;
+
+    const int e = threadIdx.x - 64;            // epilogue thread: 0..255 (warps 2..9)
+    const int sub = (warp - 2) >> 2;           // which of the two warps of a tensor-memory lane quadrant
+    const int q = warp & 3;                    // tensor-memory lane quadrant of this warp
+    const int row_in_tile = q * 32 + lane;     // the tensor-memory lane (accumulator row) of this thread
+    const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+    const bool forced = FULL && p.forced;
+
+    // ----- roles -----
+    // joint: the CTA keeps ONE vocabulary tile (cta % vt_count) and takes the row groups j_first, j_first + rg_stride, ...
+    // (one per wave); CTAs beyond vt_count * rg_stride have none
+    const int j_first = cta < p.vt_count * p.rg_stride ? cta / p.vt_count : p.rg_count;
+    const bool has_j = j_first < p.rg_count;
+    const int my_vt = cta % p.vt_count;
+    // CTAs [0, l_items) keep a W_hh tile (4 gates x 16 units) of layer 0; with two layers the next two sets keep a
+    // W_ih[1] tile ("x1") and a W_hh[1] tile ("h1"); the last p_items CTAs keep a W_pred tile (64 rows); CTAs
+    // [w_first, w_first + w_count) record the steps
+    const int r_role = cta / p.l_items;
+    const int r_idx = cta - r_role * p.l_items;
+    const bool res_l = cta < p.l_items;
+    const bool res_x1 = p.L == 2 && r_role == 1;
+    const bool res_h1 = p.L == 2 && r_role == 2;
+    const bool res_p = !res_l && !res_x1 && !res_h1 && G - 1 - cta < p.p_items;
+    const bool res_w = cta >= p.w_first && cta < p.w_first + p.w_count;
+    const int r_ut = r_idx % p.ut_count, r_ql = r_idx / p.ut_count;                  // unit tile / utterance group of an L CTA
+    const int r_ht = (G - 1 - cta) % p.ht_count, r_qp = (G - 1 - cta) / p.ht_count;  // H tile / utterance group of a P CTA
+    constexpr uint32_t RES_A_BYTES = 64 * BK * 2;
+    uint8_t* zbuf = smem + (res_p ? p.z_off_p : p.z_off);     // the joint's operand: kb_h blocks of nj rows x 64 columns
+    const bool z_sh = zbuf == buf0 && (res_l || res_x1 || res_h1 || res_p);   // it shares the state box's memory
+
+    if (threadIdx.x == 0 && (res_l || res_x1 || res_h1 || res_p)) {
+        mbar_expect_tx(&stat_bar, (uint32_t)p.kb_p * RES_A_BYTES);
+        for (int kb = 0; kb < p.kb_p; ++kb) {
+            uint8_t* dst = stat + (size_t)kb * RES_A_BYTES;
+            if (!res_p) {
+                const CUtensorMap* wm = res_l ? &M.w_hh_r : (res_x1 ? &M.w_ih1_r : &M.w_hh1_r);
+                for (int g = 0; g < 4; ++g) tma_load_2d(dst + g * 16 * 128, wm, kb * BK, g * p.P + r_ut * 16, &stat_bar);
+            } else {
+                tma_load_2d(dst, &M.w_pred_r, kb * BK, r_ht * 64, &stat_bar);
+            }
+        }
+    }
+    if (warp >= 2 && has_j) {
+        // tensor memory, lane = vocabulary entry, 32-bit column j = W_out[v, 2j], W_out[v, 2j + 1]
+        const int v = my_vt * 128 + row_in_tile;
+        const uint4* src = reinterpret_cast<const uint4*>(p.w_out + (size_t)(v < p.NV ? v : 0) * p.H);
+        for (int c0 = 0; c0 < p.H / 2; c0 += 16) {
+            uint32_t r[16];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint4 x = v < p.NV ? src[c0 / 4 + j] : make_uint4(0, 0, 0, 0);
+                r[4 * j] = x.x; r[4 * j + 1] = x.y; r[4 * j + 2] = x.z; r[4 * j + 3] = x.w;
+            }
+            tmem_st16(tmem_base + lane_off + (uint32_t)c0, r);
+        }
+        tmem_st_wait();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    // ----- arrival counters (global, zeroed per call) -----
+    uint32_t* f_keys = p.flags;                  // [rg_count]  vocabulary tiles that have left their keys for a row group
+    uint32_t* f_h0 = f_keys + p.rg_count;        // [ql_count]  layer-0 state of an utterance group written (+ its steps recorded)
+    uint32_t* f_h1 = f_h0 + p.ql_count;          // [ql_count]  layer-1 state written (two layers)
+    uint32_t* f_dh = f_h1 + p.ql_count;          // [ql_count]  layer 1's recurrent term written (two layers)
+    // arrivals per decoder-update slot on group ql's layer-0 counter: its unit tiles, plus (when separate CTAs record
+    // the steps) one per block of 32 utterances that overlaps the group
+    auto arr_h0 = [&](int ql) -> uint32_t {
+        uint32_t a = (uint32_t)p.ut_count;
+        const int lo = ql * p.nl, hi = min(lo + p.nl, p.B);
+        if (p.w_count > 0 && hi > lo) a += (uint32_t)((hi - 1) / 32 - lo / 32 + 1);
+        return a;
+    };
+    // one thread waits until a counter has reached its target; false when the kernel is being abandoned
+    auto flag_wait = [&](const uint32_t* ptr, uint32_t target) -> bool {
+        unsigned long long t0 = 0;
+        for (uint32_t it = 1;; ++it) {
+            if ((int32_t)(ld_acquire_u32(ptr) - target) >= 0) return true;
+            if ((it & 63u) == 0u) {
+                if (*vabort) return false;
+                if (ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; return false; }
+                const unsigned long long now = globaltimer_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > kWaitLimitNs) { *vabort = 1; atomicExch(&p.ctrl->abort, 1); return false; }
+            }
+        }
+    };
+    // a whole warp waits for counters base[first .. first + count): lane i polls counter i (, i + 32, ...)
+    auto warp_flag_wait = [&](const uint32_t* base, int first, int count, uint32_t target) -> bool {
+        bool ok = true;
+        for (int i0 = 0; i0 < count && ok; i0 += 32) {
+            const int i = i0 + lane;
+            bool mine = i >= count;
+            unsigned long long t0 = 0;
+            for (uint32_t it = 1;; ++it) {
+                if (!mine) mine = (int32_t)(ld_acquire_u32(base + first + i) - target) >= 0;
+                if (__all_sync(0xffffffffu, mine)) break;
+                if ((it & 63u) == 0u) {
+                    bool quit = *vabort != 0;
+                    if (!quit && ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; quit = true; }
+                    const unsigned long long now = globaltimer_ns();
+                    if (t0 == 0) t0 = now;
+                    else if (!quit && now - t0 > kWaitLimitNs) { *vabort = 1; atomicExch(&p.ctrl->abort, 1); quit = true; }
+                    if (__any_sync(0xffffffffu, quit)) { ok = false; break; }
+                }
+            }
+        }
+        __syncwarp();
+        return ok;
+    };
+
+    // ----- per-thread pipeline state (every thread keeps the same counts) -----
+    uint32_t acc_n[3] = {0u, 0u, 0u}; // uses of each accumulator so far (issuing threads and epilogue threads count alike)
+    uint32_t use0 = 0, use1 = 0;      // uses of the state box and of the joint's operand buffer so far
+    uint32_t n_l = 0, n_p = 0, n_j = 0;   // decoder-update / projection / joint slots completed
+    int step = -1;                    // -1: start of sequence
+    int pin = 0;                      // hb[pin] holds the current decoder state
+    bool prepped = false;             // the copies of the next joint operand are already under way
+    long long clk_last = 0, cyc[3] = {0, 0, 0};
+    unsigned long long ns0 = 0;
+    if (cta == 0 && e == 0) { clk_last = clock64(); ns0 = globaltimer_ns(); }
+    int exit_status = 0;
+    int tr_n = 0;                     // trace events written by this thread
+    uint32_t epoch = 0;               // grid barrier target (window-based decoding only)
+
+    // this thread has finished its CTA's part of a slot: CTA 0 attributes the time, the timeline notes every CTA
+    auto slot_done = [&](int kind) {
+        if (cta == 0) {
+            const long long now = clock64();
+            cyc[kind] += now - clk_last;
+            clk_last = now;
+        }
+        if constexpr (FULL) trace_phase_done(p, step, kind);
+    };
+
+    // Grid barrier for all threads of all CTAs (window-based decoding: its decision phase needs every vocabulary
+    // tile's statistics of every row); false when the kernel is being abandoned.
+    auto grid_sync = [&]() -> bool {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            epoch += (uint32_t)G;
+            if (*vabort) {
+                atomicExch(&p.ctrl->abort, 1);
+            } else {
+                __threadfence();
+                atomicAdd(&p.ctrl->bar, 1u);
+                flag_wait(&p.ctrl->bar, epoch);
+            }
+        }
+        __syncthreads();
+        return *vabort == 0;
+    };
+
+    // ----- one issuing thread's share of a GEMM: K blocks [kb_lo, kb_hi) into the accumulator at tm_d -----
+    // Two threads call this for every GEMM (warp 1 and warp 0), with disjoint K ranges and separate accumulator
+    // copies that the epilogue adds; an empty range only takes part in the commits.  sidx / use: which operand
+    // buffer, and how often it has been used before.
+    auto mma_part = [&](int k_acc, uint32_t tm_d, int n_tile, int kb_lo, int kb_hi, bool a_tmem, int sidx, uint32_t use,
+                        const uint8_t* b_smem) -> bool {
+        const uint32_t idesc = idesc_bf16(a_tmem ? 128 : 64, n_tile);
+        if (!a_tmem && !mbar_wait(&stat_bar, 0, vabort)) return false;
+        if (!mbar_wait(&acc_empty[k_acc], (acc_n[k_acc] & 1u) ^ 1u, vabort)) return false;   // the epilogue has drained it
+        tc_fence_after();
+        if (!mbar_wait(&full_bar[sidx], use & 1u, vabort)) return false;
+        tc_fence_after();
+        const uint32_t b_addr = smem_u32(b_smem);
+        const uint32_t b_block = (uint32_t)n_tile * BK * 2;
+        for (int kb = kb_lo; kb < kb_hi; ++kb) {
+            const uint64_t bdesc = smem_desc_sw128(b_addr + (uint32_t)kb * b_block);
+            if (a_tmem) {
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)
+                    tc_mma_bf16_ts(tm_d, tmem_base + (uint32_t)(kb * (BK / 2) + k * 8), bdesc + (uint64_t)(k * 2), idesc,
+                                   kb != kb_lo || k != 0);
+            } else {
+                const uint64_t adesc = smem_desc_sw128(smem_u32(stat + (size_t)kb * RES_A_BYTES));
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)
+                    tc_mma_bf16(tm_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, kb != kb_lo || k != 0);
+            }
+        }
+        tc_commit(&empty_bar[sidx]);
+        tc_commit(&acc_full[k_acc]);
+        ++acc_n[k_acc];
+        return true;
+    };
+    // the state box of this step: ONE three-dimensional TMA box (64 columns, rows, all K blocks), once the MMAs
+    // that read the buffer last have completed
+    auto produce_box = [&](const CUtensorMap* map, int row0, uint32_t bytes) -> bool {
+        if (use0 > 0 && !mbar_wait(&empty_bar[0], (use0 - 1) & 1u, vabort)) return false;
+        if (z_sh && use1 > 0 && !mbar_wait(&empty_bar[1], (use1 - 1) & 1u, vabort)) return false;
+        mbar_expect_tx(&full_bar[0], bytes);
+        tma_load_3d(buf0, map, 0, row0, 0, &full_bar[0]);
+        return true;
+    };
+
+    // =========================================================================================
+    // decoder-update slot of an L CTA: units [r_ut*16, +16), utterances [r_ql*nl, +nl), 64 utterances per pass.
+    // Warp (q, sub) of the epilogue owns gate q and the pass's utterances [32 sub, 32 sub + 32).  All global reads of a
+    // pass are requested together: first everything the control step needs, then the gate-table rows of the chosen
+    // tokens.  Lanes 16..31 hold no accumulator row (64-row tile); they take the second 16 utterances.
+    // ctl_only: the CTA is one of the step-recording CTAs: it takes the control step of 64 utterances, records it
+    // (outputs, counters, next frame) and has no cell update; the L CTAs then record nothing.
+    // =========================================================================================
+    struct ScanIn { int t, len, cnt, pos; unsigned long long kk[8]; };
+    auto epilogue_res_L = [&](const int layer, const bool ctl_only) -> bool {
+        if (ctl_only && q != 0) return true;
+        const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
+        int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
+        const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
+        unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
+        const int u16 = lane & 15, half = lane >> 4;
+        const int unit = r_ut * 16 + u16;        // this thread's hidden unit; its gate is q
+        // without recording CTAs, the two gate-0 warps of one CTA per utterance group record the step
+        const bool writer = ctl_only ? true : (p.w_count == 0 && layer == 0 && r_ut == 0 && q == 0);
+        const int n_here = ctl_only ? 64 : p.nl;
+        const int base = ctl_only ? (cta - p.w_first) * 64 : r_ql * p.nl;
+        const bool decode = step >= 0 && !forced && layer == 0;
+        float* cst = p.c_state + (size_t)layer * p.B * p.P + unit;
+        const __nv_bfloat16* hin = p.hb + ((size_t)(pin * p.L + layer) * p.Bpad) * p.P + unit;
+        __nv_bfloat16* hout = p.hb + ((size_t)((pin ^ 1) * p.L + layer) * p.Bpad) * p.P + unit;
+        const float bias1 = layer == 0 ? 0.f : p.b_ih[1][q * p.P + unit] + p.b_hh[1][q * p.P + unit];
+        const float* g0u = p.g0 + (size_t)q * p.P + unit;
+        const uint32_t g0_stride = 4u * (uint32_t)p.P;
+        bool ready = true;
+        // ---- what this slot waits for from other CTAs ----
+        if (decode) {
+            // the keys of this CTA's utterances: every vocabulary tile of their row groups has arrived
+            const int b_hi = min(base + n_here, p.B);
+            if (b_hi > base) {
+                const int rg_lo = base * p.W / p.nj, rg_hi = (b_hi * p.W - 1) / p.nj;
+                ready = warp_flag_wait(f_keys, rg_lo, rg_hi - rg_lo + 1, n_j * (uint32_t)p.vt_count + (uint32_t)p.extra_arrivals);
+            }
+        } else if (layer > 0) {
+            // layer 1: the step's tokens (recorded with layer 0's arrivals) and the recurrent term computed a slot ahead
+            bool ok = true;
+            if (lane == 0) ok = flag_wait(f_h0 + r_ql, n_l * arr_h0(r_ql)) && flag_wait(f_dh + r_ql, n_l * (uint32_t)p.ut_count);
+            ready = __all_sync(0xffffffffu, ok);
+        }
+        for (int c0 = 0; c0 < n_here; c0 += 64) {
+            const int b0 = base + c0;
+            // ---- lane j decides for utterance b0 + 32 sub + j ----
+            const int jl = 32 * sub + lane;
+            const int b = b0 + jl;
+            const bool in = c0 + jl < n_here && b < p.B;
+            ScanIn si;
+            si.t = 0; si.len = 0; si.cnt = 0; si.pos = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) si.kk[j] = 0ull;
+            if (in && decode) {
+                si.t = __ldcg(t_cur + b);
+                si.len = p.enc_len[b];
+                if (writer) { si.cnt = __ldcg(p.count + b); si.pos = __ldcg(p.out_len + b); }
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (j < p.W) si.kk[j] = __ldcg(keys_cur + (size_t)b * p.W + j);
+            }
+            // old cell state of the four (utterance, unit) pairs this thread finishes
+            float cold[4];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                const int j = half + 2 * q + 8 * sub + 16 * jj;     // 0..63 over the CTA's 256 epilogue threads
+                cold[jj] = (!ctl_only && c0 + j < p.nl && b0 + j < p.B) ? cst[(size_t)(b0 + j) * p.P] : 0.f;
+            }
+            // the token utterance b feeds to its decoder in this step (-1: none)
+            int tok = -1, t_out = 0;
+            if (in) {
+                if (step < 0) {
+                    tok = p.blank;
+                } else if (forced) {
+                    tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
+                    if (tok >= p.NV || tok < -1) { tok = p.blank; set_status(p.ctrl, WIND_ERR_INVALID_ARG); }   // caller's mistake
+                } else if (layer > 0) {
+                    tok = __ldcg(p.emit_tok + b);     // decided by layer 0's CTAs one slot earlier
+                } else {
+                    int t = si.t;
+                    const int len = si.len;
+                    if (t < len) {
+                        // control step (Algorithm 2's branch): first non-blank row of the window
+                        const int n = min(p.W, len - t);
+                        int first = -1, label = p.blank;
+                        bool bad = false;
+                        for (int w0 = 0; w0 < n && first < 0; w0 += 8) {
+                            if (w0 > 0) {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) si.kk[j] = (w0 + j < n) ? __ldcg(keys_cur + (size_t)b * p.W + w0 + j) : 0ull;
+                            }
+                            // the eight rows side by side: which are inside the window, broken, non-blank
+                            uint32_t nonblank = 0u, broken = 0u;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const uint32_t lab = key_label(si.kk[j]);
+                                const bool inside = w0 + j < n;
+                                const bool brk = si.kk[j] == 0ull || lab >= (uint32_t)p.NV;
+                                broken |= (uint32_t)(inside && brk) << j;
+                                nonblank |= (uint32_t)(inside && !brk && (int)lab != p.blank) << j;
+                            }
+                            if (nonblank) {
+                                const int j = __ffs((int)nonblank) - 1;
+                                first = w0 + j;
+                                uint32_t lab = 0u;
+#pragma unroll
+                                for (int jj = 0; jj < 8; ++jj)
+                                    if (jj == j) lab = key_label(si.kk[jj]);
+                                label = (int)lab;
+                                broken &= (1u << j) - 1u;   // rows after the first non-blank one are not looked at
+                            }
+                            bad = bad || broken != 0u;
+                        }
+                        if (first >= 0) tok = label;
+                        if (writer) {
+                            int cnt = si.cnt, jump, forced_adv = 0, emitted = 0;
+                            if (first < 0) {
+                                jump = n;
+                                t += n;
+                                cnt = 0;
+                            } else {
+                                jump = first;
+                                if (first > 0) cnt = 0;
+                                t += first;
+                                if (si.pos < p.max_out) {
+                                    p.out_tokens[(size_t)b * p.max_out + si.pos] = label;
+                                    p.out_frames[(size_t)b * p.max_out + si.pos] = t;
+                                    p.out_len[b] = si.pos + 1;
+                                    emitted = 1;
+                                    cnt += 1;
+                                    if (cnt == p.S) { t += 1; cnt = 0; forced_adv = 1; }
+                                } else {
+                                    set_status(p.ctrl, WIND_ERR_OUTPUT_OVERFLOW);  // this utterance stops here
+                                    t = len;
+                                    tok = -1;
+                                }
+                            }
+                            if (bad && ready) set_status(p.ctrl, WIND_ERR_INTERNAL);
+                            t_nxt[b] = t;
+                            t_out = t;
+                            p.count[b] = cnt;
+                            for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
+                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
+                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->joint_rows), (unsigned long long)n);
+                            if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
+                            if (forced_adv) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
+                        }
+                    } else if (writer) {
+                        t_nxt[b] = t;
+                        t_out = t;
+                    }
+                }
+                if (writer && p.L > 1 && decode) p.emit_tok[b] = tok;   // the upper layer's CTAs read it in their slot
+                // the next frame goes out at once, stamped with the slot, for the CTAs that build the next window's
+                // operand and for everybody's count of the utterances still decoding.  Released: what this thread has
+                // written for the step (frame, counters, the cleared keys of the next step) is visible before it.
+                if (writer && !forced) {
+                    __threadfence();
+                    p.t_pub[b] = ((unsigned long long)(n_l + 1u) << 32) | (uint32_t)t_out;
+                }
+            }
+            if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
+            if (ctl_only) continue;
+            // ---- gate-table entries (this thread's gate and unit) of the tokens of this lane half's 16 utterances ----
+            float add[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int ta = __shfl_sync(0xffffffffu, tok, j), tb = __shfl_sync(0xffffffffu, tok, 16 + j);
+                const int tj = half ? tb : ta;
+                if (layer == 0) {
+                    add[j] = tj >= 0 ? g0u[(uint32_t)tj * g0_stride] : 0.f;
+                } else {
+                    // layer 1: the recurrent term W_hh h computed a slot ahead by the h1 CTAs, plus the biases
+                    const int bj2 = b0 + 32 * sub + 16 * half + j;
+                    add[j] = (tj >= 0 && bj2 < p.B) ? __ldcg(p.dh + (size_t)bj2 * g0_stride + (size_t)q * p.P + unit) + bias1 : 0.f;
+                }
+            }
+            // the other warps need the tokens for the cell update below: through shared memory
+            int* tok_s = reinterpret_cast<int*>(stage_f + 4 * 64 * 16);
+            if (q == 0) tok_s[jl] = tok;
+            if (c0 == 0) {
+                const bool acc_ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, vabort));
+                ready = ready && acc_ok;
+                tc_fence_after();
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
+            }
+            if (ready) {
+                // lanes 0..15 read their row's 32 columns; columns 16..31 then move to lanes 16..31
+                float x[16], hi[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) { x[j] = 0.f; hi[j] = 0.f; }
+                const int col = c0 + 32 * sub;
+                if (col < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)col, x);
+                if (col + 16 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(col + 16), hi);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float v = __shfl_sync(0xffffffffu, hi[j], u16);
+                    if (half) x[j] = v;
+                }
+                // warp q holds gate q: tanh for the cell candidate (q == 2), logistic for the other three,
+                // written as 0.5 tanh(x / 2) + 0.5 so that both are one hardware tanh
+                const float sc = q == 2 ? 1.f : 0.5f, of = q == 2 ? 0.f : 0.5f;
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    stage_f[(q * 64 + 32 * sub + 16 * half + j) * 16 + u16] = fmaf(tanh_fast((x[j] + add[j]) * sc), sc, of);
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (ready) {
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = half + 2 * q + 8 * sub + 16 * jj;     // 0..63
+                    const int bj = b0 + j;
+                    if (c0 + j < p.nl && bj < p.B) {
+                        if (tok_s[j] >= 0) {
+                            const float gi = stage_f[(0 * 64 + j) * 16 + u16], gf = stage_f[(1 * 64 + j) * 16 + u16];
+                            const float gg = stage_f[(2 * 64 + j) * 16 + u16], go = stage_f[(3 * 64 + j) * 16 + u16];
+                            const float cc = gf * cold[jj] + gi * gg;
+                            cst[(size_t)bj * p.P] = cc;
+                            hout[(size_t)bj * p.P] = __float2bfloat16_rn(go * tanh_fast(cc));
+                        } else {
+                            hout[(size_t)bj * p.P] = hin[(size_t)bj * p.P];
+                        }
+                    }
+                }
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+        }
+        if (ctl_only) {
+            // this warp's 32 utterances are recorded: one arrival on every utterance group they belong to
+            __syncwarp();
+            const int lo = base + 32 * sub, hi = min(lo + 32, p.B);
+            if (lane == 0 && hi > lo)
+                for (int g = lo / p.nl; g <= (hi - 1) / p.nl; ++g) red_release_add(f_h0 + g, 1u);
+            return true;
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[1]);
+        ++acc_n[1];
+        // the new state is complete for this CTA's units: visible to TMA reads, then one arrival for the group
+        fence_proxy_async_all();
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (e == 0) red_release_add((layer == 0 ? f_h0 : f_h1) + r_ql, 1u);
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_EPI_DONE);
+        return ready;
+    };
+
+    // b_pred of this thread's accumulator row: constant for the whole decode, read once
+    const float p_bias = (res_p && e >= 0) ? p.b_pred[r_ht * 64 + 16 * q + (lane & 15)] : 0.f;
+    // projection epilogue of a P CTA: pred_proj rows [r_ht*64, +64) of utterances [r_qp*np, +np), published as
+    // (value, stamp) pairs: a reader that finds the stamp of this slot has the value
+    auto epilogue_res_P = [&](uint32_t stamp) -> bool {
+        const int h0 = r_ht * 64;
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
+        const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[2], acc_n[2] & 1u, vabort));
+        tc_fence_after();
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
+        if (ready) {
+            const int hl = 16 * q + (lane & 15);
+            for (int c0 = 16 * sub; c0 < p.np; c0 += 32) {
+                float g[16], more[16];
+                tmem_ld16(tm_p + lane_off + (uint32_t)c0, g);
+                tmem_ld16(tm_p + lane_off + (uint32_t)(p.np + c0), more);   // the other issuing thread's K blocks
+                if (p.kb_p < 2) {   // a single K block: the first copy's issuer had an empty range and wrote nothing
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) g[j] = 0.f;
+                }
+                if (lane < 16) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) stage_f[(c0 + j) * 68 + hl] = g[j] + more[j] + p_bias;
+                }
+            }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[2]);
+        ++acc_n[2];
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (ready) {
+            // thread e: four consecutive H rows of utterances (e >> 4), (e >> 4) + 16, ...: 512 contiguous bytes per
+            // utterance and 16 threads.  One release fence, then the stamped pairs.
+            __threadfence();
+            const int hq = (e & 15) * 4;
+            for (int bl = e >> 4; bl < p.np; bl += 16) {
+                const int b = r_qp * p.np + bl;
+                if (b < p.B) {
+                    const float4 v = *reinterpret_cast<const float4*>(stage_f + bl * 68 + hq);
+                    unsigned long long* dst = p.pred_pub + (size_t)b * p.H + h0 + hq;
+                    st_relaxed_v2_u64(dst, stamped(v.x, stamp), stamped(v.y, stamp));
+                    st_relaxed_v2_u64(dst + 2, stamped(v.z, stamp), stamped(v.w, stamp));
+                }
+            }
+        }
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
+        return ready;
+    };
+    // h1 CTAs: the finished recurrent term of layer 1 goes to global memory (fp32 [B][4P], gate-major like the gate
+    // table); the x1 CTAs add it in the next decoder-update slot
+    auto store_res_h1 = [&]() {
+        const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, vabort));
+        tc_fence_after();
+        if (ready) {
+            const int unit = r_ut * 16 + (lane & 15);
+            for (int c0 = 0; c0 < p.nl; c0 += 64) {
+                const int col = c0 + 32 * sub;
+                float x[16], hi[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) { x[j] = 0.f; hi[j] = 0.f; }
+                if (col < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)col, x);
+                if (col + 16 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(col + 16), hi);
+                if (lane < 16) {
+                    float* dst = p.dh + (size_t)q * p.P + unit;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int ba = r_ql * p.nl + col + j, bb = ba + 16;
+                        if (col + j < p.nl && ba < p.B) dst[(size_t)ba * 4 * p.P] = x[j];
+                        if (col + 16 + j < p.nl && bb < p.B) dst[(size_t)bb * 4 * p.P] = hi[j];
+                    }
+                }
+            }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[1]);
+        ++acc_n[1];
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (e == 0) red_release_add(f_dh + r_ql, 1u);
+    };
+    // GEMMs that need only the state, issued a slot ahead: layer 0's (its result waits in tensor memory for the
+    // next control step) and, with two layers, layer 1's recurrent term (stored by store_res_h1)
+    auto early_res = [&]() {
+        const bool mine = res_l || res_h1;
+        if (warp == 0) {
+            if (lane == 0 && mine) {
+                // the state of this CTA's utterance group as the last decoder-update slot left it
+                const bool ok = res_l ? flag_wait(f_h0 + r_ql, n_l * arr_h0(r_ql)) : flag_wait(f_h1 + r_ql, n_l * (uint32_t)p.ut_count);
+                if (ok) {
+                    fence_proxy_async_all();
+                    if (produce_box(res_l ? &M.hb_l3[pin] : &M.hb_l3_1[pin], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u))
+                        mma_part(1, tm_l, p.nl, p.kb_p, p.kb_p, false, 0, use0, buf0);   // one accumulator: warp 1 issues all of it
+                }
+            }
+        } else if (warp == 1) {
+            if (lane == 0 && mine) mma_part(1, tm_l, p.nl, 0, p.kb_p, false, 0, use0, buf0);
+        } else if (res_h1) {
+            store_res_h1();
+        }
+        if (mine) ++use0;
+    };
+
+    // =========================================================================================
+    // The joint's operand, built by the epilogue warps in the 128-byte swizzled K-major layout the MMA reads:
+    // K block kb = 64 columns, nj rows of 128 bytes each, the 16-byte chunk c of row i at chunk position c ^ (i & 7).
+    // Work item = (utterance of the row group, chunk of 8 columns); thread e takes items e, e + 256, ...
+    // Part A (as soon as the next frames are known): copy the enc_proj chunks of the window rows in, zeros past an
+    // utterance's end.  Part B (when pred_proj has arrived): add, activate, convert, in place, by the thread that
+    // copied the chunk; then hand the buffer to the issuing threads.
+    // =========================================================================================
+    const int n_chunks = p.H >> 3;
+    auto group_span = [&](int rg, int& u_lo, int& n_utt) {
+        const int r_lo = rg * p.nj, r_hi = min(r_lo + p.nj, p.rows);
+        u_lo = r_lo / p.W;
+        n_utt = r_hi > r_lo ? (r_hi - 1) / p.W - u_lo + 1 : 0;
+    };
+    auto prep_A = [&](int rg, uint32_t want) {
+        int u_lo, n_utt;
+        group_span(rg, u_lo, n_utt);
+        if (e < n_utt) {
+            const int b = u_lo + e;
+            int t = 0;
+            if (forced) {
+                t = p.t2[b];
+            } else {
+                // acquire: what the recording thread wrote before publishing (the cleared keys of the next step
+                // among it) is ordered before everything this CTA does with the window
+                unsigned long long t0 = 0, v = 0;
+                for (uint32_t it = 1;; ++it) {
+                    v = ld_acquire_u64(p.t_pub + b);
+                    if ((uint32_t)(v >> 32) == want) break;
+                    if ((it & 63u) == 0u) {
+                        if (*vabort) break;
+                        if (ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; break; }
+                        const unsigned long long now = globaltimer_ns();
+                        if (t0 == 0) t0 = now;
+                        else if (now - t0 > kWaitLimitNs) { *vabort = 1; atomicExch(&p.ctrl->abort, 1); break; }
+                    }
+                }
+                t = (int)(uint32_t)v;
+            }
+            const int len = p.enc_len[b];
+            s_jt[e] = t < len ? t : 0;
+            s_jrem[e] = t < len ? len - t : 0;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        // the buffer is free once the MMAs that read it last have completed
+        bool ok = use1 == 0 || mbar_wait(&empty_bar[1], (use1 - 1) & 1u, vabort);
+        if (ok && z_sh && use0 > 0) ok = mbar_wait(&empty_bar[0], (use0 - 1) & 1u, vabort);
+        if (ok && *vabort == 0) {
+            for (int idx = e; idx < n_utt * n_chunks; idx += 256) {
+                const int ul = idx / n_chunks, c = idx - ul * n_chunks;
+                const int b = u_lo + ul, t = s_jt[ul], rem = s_jrem[ul];
+                const int w_lo = max(0, rg * p.nj - b * p.W), w_hi = min(p.W, (rg + 1) * p.nj - b * p.W);
+                uint8_t* dst_kb = zbuf + (size_t)(c >> 3) * ((size_t)p.nj * 128);
+                const __nv_bfloat16* src = p.enc_proj + ((size_t)b * p.T + t) * p.H + c * 8;
+                for (int w = w_lo; w < w_hi; ++w) {
+                    const int i = b * p.W + w - rg * p.nj;
+                    uint8_t* dst = dst_kb + i * 128 + (((c & 7) ^ (i & 7)) << 4);
+                    if (w < rem) {
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src + (size_t)w * p.H) : "memory");
+                    } else {
+                        *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+                    }
+                }
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    auto prep_B = [&](int rg, uint32_t want) {
+        int u_lo, n_utt;
+        group_span(rg, u_lo, n_utt);
+        const int n_items = n_utt * n_chunks;
+        bool waited = false;
+        for (int base = e; base < n_items; base += 256 * kPrepItems) {
+            float pv[kPrepItems][8];
+            int it_ul[kPrepItems], it_c[kPrepItems];
+#pragma unroll
+            for (int k = 0; k < kPrepItems; ++k) {
+                const int idx = base + k * 256;
+                it_ul[k] = -1; it_c[k] = 0;
+                if (idx < n_items) {
+                    const int ul = idx / n_chunks;
+                    if (s_jrem[ul] > 0) { it_ul[k] = ul; it_c[k] = idx - ul * n_chunks; }   // a finished utterance needs nothing
+                }
+            }
+            // pred_proj of this round's items, all requested together, until every stamp is this slot's
+            unsigned long long t0 = 0;
+            for (uint32_t it = 1;; ++it) {
+                bool all = true;
+#pragma unroll
+                for (int k = 0; k < kPrepItems; ++k) {
+                    if (it_ul[k] < 0) continue;
+                    const unsigned long long* src = p.pred_pub + (size_t)(u_lo + it_ul[k]) * p.H + it_c[k] * 8;
+                    unsigned long long x[8];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) ld_acquire_v2_u64(src + 2 * j, x[2 * j], x[2 * j + 1]);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        all = all && (uint32_t)(x[j] >> 32) == want;
+                        pv[k][j] = __uint_as_float((uint32_t)x[j]);
+                    }
+                }
+                if (all) break;
+                if ((it & 15u) == 0u) {
+                    if (*vabort) break;
+                    if (ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; break; }
+                    const unsigned long long now = globaltimer_ns();
+                    if (t0 == 0) t0 = now;
+                    else if (now - t0 > kWaitLimitNs) { *vabort = 1; atomicExch(&p.ctrl->abort, 1); break; }
+                }
+            }
+            if (!waited) { asm volatile("cp.async.wait_all;" ::: "memory"); waited = true; }
+#pragma unroll
+            for (int k = 0; k < kPrepItems; ++k) {
+                if (it_ul[k] < 0) continue;
+                const int b = u_lo + it_ul[k], c = it_c[k], rem = s_jrem[it_ul[k]];
+                const int w_lo = max(0, rg * p.nj - b * p.W), w_hi = min(min(p.W, (rg + 1) * p.nj - b * p.W), rem);
+                uint8_t* dst_kb = zbuf + (size_t)(c >> 3) * ((size_t)p.nj * 128);
+                for (int w = w_lo; w < w_hi; ++w) {
+                    const int i = b * p.W + w - rg * p.nj;
+                    uint4* dst = reinterpret_cast<uint4*>(dst_kb + i * 128 + (((c & 7) ^ (i & 7)) << 4));
+                    const uint4 ev = *dst;
+                    const __nv_bfloat162* eb = reinterpret_cast<const __nv_bfloat162*>(&ev);
+                    uint32_t wds[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float2 e2 = __bfloat1622float2(eb[j]);
+                        float z0 = e2.x + pv[k][2 * j], z1 = e2.y + pv[k][2 * j + 1];
+                        z0 = p.act == WIND_ACT_RELU ? fmaxf(z0, 0.f) : tanh_fast(z0);
+                        z1 = p.act == WIND_ACT_RELU ? fmaxf(z1, 0.f) : tanh_fast(z1);
+                        wds[j] = pack_bf16x2(z0, z1);
+                    }
+                    *dst = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+                }
+            }
+        }
+        if (!waited) asm volatile("cp.async.wait_all;" ::: "memory");
+        fence_proxy_async();      // this thread's shared-memory writes, for the MMAs (async proxy)
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (e == 0) mbar_arrive(&full_bar[1]);
+    };
+
+    // ----- before the loop: layer 0's GEMM on the initial (zero) state -----
+    early_res();
+
+    for (;;) {
+        // =====================================================================================
+        // decoder-update slot: control step + LSTM cell update (layer 0), then layer 1 on its own CTAs
+        // =====================================================================================
+        if (warp >= 2) {
+            if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_START);
+            if (res_l) epilogue_res_L(0, false);
+            else if (res_w) epilogue_res_L(0, true);
+            if (cta == 0 && e == 0 && step >= 0 && !forced) p.ctrl->step = step + 1;
+            // CTAs whose joint operand has a buffer of its own start on the next window now
+            if (has_j && !z_sh && !forced) { prep_A(j_first, n_l + 1u); prepped = true; }
+            if (e == 0 && p.L != 2) slot_done(TR_L);
+        }
+        ++n_l;
+        if (p.L == 2) {
+            // layer 1: W_ih[1] . (new layer-0 state) on the x1 CTAs, then their cell update
+            if (warp == 0) {
+                if (lane == 0 && res_x1) {
+                    if (flag_wait(f_h0 + r_ql, n_l * arr_h0(r_ql))) {
+                        fence_proxy_async_all();
+                        if (produce_box(&M.hb_l3[pin ^ 1], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u))
+                            mma_part(1, tm_l, p.nl, p.kb_p, p.kb_p, false, 0, use0, buf0);
+                    }
+                }
+            } else if (warp == 1) {
+                if (lane == 0 && res_x1) mma_part(1, tm_l, p.nl, 0, p.kb_p, false, 0, use0, buf0);
+            } else {
+                if (res_x1) epilogue_res_L(1, false);
+                if (e == 0) slot_done(TR_L);
+            }
+            if (res_x1) ++use0;
+        }
+        pin ^= 1;
+        if (forced && step + 1 < p.U) {
+            // teacher forcing: more prefix tokens to feed before the window is evaluated
+            early_res();
+            ++step;
+            continue;
+        }
+
+        // =====================================================================================
+        // projection slot: pred_proj for every utterance; behind it, layer 0's GEMM of the next step
+        // =====================================================================================
+        if (warp == 0) {
+            if (lane == 0 && res_p) {
+                // the top layer's state of this CTA's utterances: every utterance group they belong to has arrived
+                const uint32_t* f = p.L == 2 ? f_h1 : f_h0;
+                const int b_lo = r_qp * p.np, b_hi = min(b_lo + p.np, p.B);
+                bool ok = true;
+                if (b_hi > b_lo)
+                    for (int g = b_lo / p.nl; ok && g <= (b_hi - 1) / p.nl; ++g)
+                        ok = flag_wait(f + g, n_l * (p.L == 2 ? (uint32_t)p.ut_count : arr_h0(g)));
+                if (ok) {
+                    fence_proxy_async_all();
+                    if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_P, EV_FIRST_ISSUE);
+                    if (produce_box(&M.hb_p3[pin], r_qp * p.np, (uint32_t)p.np * (uint32_t)p.P * 2u))
+                        mma_part(2, tm_p + (uint32_t)p.np, p.np, p.kb_p / 2, p.kb_p, false, 0, use0, buf0);
+                }
+            }
+        } else if (warp == 1) {
+            if (lane == 0 && res_p) mma_part(2, tm_p, p.np, 0, p.kb_p / 2, false, 0, use0, buf0);
+        } else {
+            if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_START);
+            if (warp == 2 && !forced) {
+                // utterances still decoding, from the frames the recording threads have published for this step
+                // (every CTA reads the same words, so all take the same exit)
+                int alive = 0;
+                unsigned long long t0 = 0;
+                for (uint32_t it = 1;; ++it) {
+                    bool all = true;
+                    alive = 0;
+                    for (int b = lane; b < p.B; b += 32) {
+                        unsigned long long v;
+                        asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(v) : "l"(p.t_pub + b) : "memory");
+                        all = all && (uint32_t)(v >> 32) == n_l;
+                        alive += (int)(uint32_t)v < p.enc_len[b];
+                    }
+                    if (__all_sync(0xffffffffu, all)) break;
+                    if ((it & 15u) == 0u) {
+                        bool quit = *vabort != 0;
+                        if (!quit && ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; quit = true; }
+                        const unsigned long long now = globaltimer_ns();
+                        if (t0 == 0) t0 = now;
+                        else if (!quit && now - t0 > kWaitLimitNs) { *vabort = 1; atomicExch(&p.ctrl->abort, 1); quit = true; }
+                        if (__any_sync(0xffffffffu, quit)) break;
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) alive += __shfl_xor_sync(0xffffffffu, alive, o);
+                if (lane == 0) s_active = alive;
+            }
+            if (res_p) epilogue_res_P(n_p + 1u);
+        }
+        if (res_p) ++use0;
+        ++n_p;
+        early_res();
+        if (warp >= 2 && e == 0) slot_done(TR_P);
+        // the one CTA-wide meeting point of a step: everybody learns whether the kernel is being abandoned and how
+        // many utterances are still decoding
+        {
+            const int ab = __syncthreads_or(*vabort != 0);
+            if (ab) goto done;
+        }
+        if (!forced && s_active == 0) break;
+        if (!forced && step + 1 >= p.step_cap) { exit_status = WIND_ERR_INTERNAL; break; }
+        ++step;
+
+        // =====================================================================================
+        // joint slot: the CTA's vocabulary tile against the window rows of its row group(s)
+        // =====================================================================================
+        {
+            const int n_tile = p.nj;
+            unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
+            const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
+            for (int rg = j_first; rg < p.rg_count; rg += p.rg_stride) {
+                if (warp < 2) {
+                    if (lane == 0) {
+                        if constexpr (FULL) trace_event(p, warp, tr_n, step, TR_J, EV_FIRST_ISSUE);
+                        if (warp == 0) mma_part(0, tm_j + (uint32_t)n_tile, n_tile, p.kb_h / 2, p.kb_h, true, 1, use1, zbuf);
+                        else mma_part(0, tm_j, n_tile, 0, p.kb_h / 2, true, 1, use1, zbuf);
+                        if constexpr (FULL) trace_event(p, warp, tr_n, step, TR_J, EV_COMMIT);
+                    }
+                } else {
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_START);
+                    if (!prepped) prep_A(rg, n_l);
+                    prepped = false;
+                    prep_B(rg, n_p);
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_TOK);
+                    const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[0], acc_n[0] & 1u, vabort));
+                    tc_fence_after();
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_ACC);
+                    if (ready) joint_epilogue_item<true, FULL>(p, tm_j, lane_off, lane, q, sub, row_in_tile, rg, my_vt, n_tile, t_cur, keys_cur);
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[0]);
+                    ++acc_n[0];
+                    // this vocabulary tile's keys of the row group are out: one arrival
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    if (e == 0) red_release_add(f_keys + rg, 1u);
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_EPI_DONE);
+                }
+                ++use1;
+            }
+            ++n_j;
+            if (warp >= 2 && e == 0) slot_done(TR_J);
+        }
+        if (forced) break;
+        if (FULL && p.window) {
+            // window-based decoding: one warp per window row turns the joint's per-row statistics into the most
+            // probable (label, offset) pair of Eq. (1) and leaves it in the keys in the form the control step reads
+            if (!grid_sync()) goto done;
+            if (warp >= 2) {
+                const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
+                unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
+                window_decision<8>(p, cta, G, warp - 2, lane, t_cur, keys_cur, win_lpb, win_sc, win_key);
+            }
+            if (!grid_sync()) goto done;
+        }
+    }
+done:
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    // an accumulator may still hold an unused early GEMM; nothing reads it, but its MMAs must have completed before
+    // the tensor memory goes back (a private flag, so that the wait is not cut short; it stays bounded)
+    if (warp == 1 && lane == 0 && acc_n[1] > 0) {
+        int gave_up = 0;
+        mbar_wait(&acc_full[1], (acc_n[1] - 1u) & 1u, &gave_up);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, LOOP_TMEM_COLS);
+    }
+    if (threadIdx.x == 0) {
+        if (s_abort) atomicExch(&p.ctrl->abort, 1);
+        if (s_abort == 1) set_status(p.ctrl, WIND_ERR_TIMEOUT);
+    }
+    if (cta == 0 && e == 0) {
+        if (exit_status) set_status(p.ctrl, exit_status);
+        p.ctrl->active = s_active;
+        for (int k = 0; k < 3; ++k) p.ctrl->phase_cycles[k] = cyc[k];
+        p.ctrl->loop_ns = (long long)(globaltimer_ns() - ns0);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// host side of this kernel: shared-memory opt-in per device, launch
+// ---------------------------------------------------------------------------
+static std::mutex g_res_mutex;
+static int g_res_smem[64] = {};
+
+cudaError_t loop_res_set_smem(int bytes) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_res_mutex);
+    if (bytes > g_res_smem[dev]) {
+        for (const void* fn : {(const void*)loop_res_kernel<false>, (const void*)loop_res_kernel<true>}) {
+            e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+            if (e != cudaSuccess) return e;
+        }
+        g_res_smem[dev] = bytes;
+    }
+    return cudaSuccess;
+}
+
+cudaError_t loop_res_launch(const LoopMaps& maps, const LoopParams& p, int grid, uint32_t smem_bytes, bool full, cudaStream_t stream) {
+    void* args[2] = {(void*)&maps, (void*)&p};
+    const void* fn = full ? (const void*)loop_res_kernel<true> : (const void*)loop_res_kernel<false>;
+    return cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), dim3(LOOP_THREADS_RES), args, smem_bytes, stream);
+}
+
+}  // namespace wind

@@ -3,7 +3,7 @@
 The library decodes the whole batch (B = 128 / 64 / 32 utterances of up to 2500 / 5000 / 3000 frames).  Every
 transcript gets the checks that hold at any size (frames non-decreasing and inside the utterance, at most S tokens per
 frame, labels in range, counters consistent).  A sample of utterances -- the shortest few, one from the middle of the
-length order and the longest, listed in tests/golden/fullsize_oracle.json together with a digest of the oracle's own
+length order and (configurations 3 and 4 at rate 0.25) the longest, listed in tests/golden/fullsize_oracle.json together with a digest of the oracle's own
 transcript (written by tests/golden/make_golden.py --fullsize, which calls only the oracle and the input generator) --
 is compared with the oracle under the margin rule: the transcript is replayed through the oracle, every implied
 decision must be the oracle's argmax or lie within 0.05 of its maximum, and a transcript whose decisions are all the
