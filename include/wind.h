@@ -110,6 +110,9 @@ typedef struct {
     int32_t launches_per_step; /* kernel nodes in one loop iteration */
     int32_t launches_setup;    /* kernel launches outside the loop (projection, init, first decoder update) */
     int32_t kernels;           /* wind_kernels_t actually used */
+    int32_t timeout_site;      /* after WIND_ERR_TIMEOUT from the resident-weights loop kernel: a code for the wait that ran
+                                  out first (a diagnostic: grep the code in the kernel source) and the CTA it ran out in */
+    int32_t timeout_cta;
 } wind_stats_t;
 
 /*
@@ -370,6 +373,39 @@ wind_status_t wind_read_trace(const wind_model_t* m, int32_t B, int32_t T, int32
  * mention of a safeguard is the beam-search footnote about not staying on one frame forever).
  */
 int32_t wind_debug_stall_barrier(int32_t extra_arrivals);
+
+/*
+ * Options of the tensor-core loop's tile planner, process-wide (defaults: 1, -1, 4).  Meant for tests and
+ * measurements, which use them to reach every mode of the loop kernels on one shape; results do not depend on them.
+ *   resident         0: never choose the resident-weights mode (weights then stream through shared memory every
+ *                    step, as for shapes whose tiles do not fit on chip)
+ *   joint_placement  streaming mode only: where a CTA keeps its W_out tile when it owns one joint item: -1 the
+ *                    planner's choice, 0 streamed every step, 1 shared memory, 2 tensor memory (taken when feasible)
+ *   max_joint_waves  resident mode: most passes over row groups the joint may take per step (1..4)
+ */
+void wind_set_loop_options(int32_t resident, int32_t joint_placement, int32_t max_joint_waves);
+
+/*
+ * The tile plan the tensor-core loop would use for a model and batch on a device with `sms` multiprocessors and
+ * `smem_optin` bytes of opt-in shared memory per block: host arithmetic only, no CUDA call, so that the plan's
+ * invariants (every shared-memory region inside smem_bytes, tensor-memory columns within 512, disjoint CTA sets
+ * inside the grid) can be checked over many shapes without a GPU.  WIND_ERR_UNSUPPORTED: the shapes are outside the
+ * tensor-core path (dimensions not multiples of 64, fewer than 128 logits) or nothing fits.
+ * Resident mode (resident = 1): CTAs [0, l_sets * l_items) hold decoder tiles (l_items = ut_count unit tiles x ql_count
+ * utterance groups of nl), the last p_items = ht_count x qp_count CTAs hold W_pred tiles (np utterances each), CTAs
+ * [w_first, w_first + w_count) record the steps; shared memory of a CTA: tile_bytes at 0, the state box at buf_off, the
+ * joint's operand (nj rows x H) at z_off (z_off_p in W_pred CTAs), staging from stage_off to smem_bytes - 1024.
+ * Streaming mode: rings of stages_lp x stage_lp and stages_j x stage_j bytes behind tile_bytes.
+ */
+typedef struct {
+    int32_t grid, resident, smem_bytes;
+    int32_t nj, vt_count, rg_count, rg_stride, j_mode;
+    int32_t tm_j, tm_l, tm_p;
+    int32_t nl, np, ut_count, ht_count, ql_count, qp_count, l_items, p_items, w_first, w_count, l_sets;
+    int32_t tile_bytes, buf_off, z_off, z_off_p, stage_off;
+    int32_t slots, ul, ug_count, mt_count, hg_count, stages_lp, stages_j, stage_lp, stage_j;
+} wind_plan_t;
+wind_status_t wind_debug_plan(const wind_model_t* m, int32_t B, int32_t W, int32_t sms, int32_t smem_optin, wind_plan_t* out);
 
 /* Process-wide choice of kernels for the bf16 path (default AUTO).  Returns the previous value. */
 int32_t wind_set_kernels(int32_t kernels);

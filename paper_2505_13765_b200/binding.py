@@ -31,6 +31,7 @@ WIND_KERNELS_AUTO, WIND_KERNELS_SIMT, WIND_KERNELS_TENSOR = 0, 1, 2
 EXPORTS = [
     "wind_workspace_bytes", "wind_decode_greedy", "wind_decode_window_greedy", "wind_host_staging_bytes", "wind_decode_greedy_host",
     "wind_eval_joint_window", "wind_window_first_output", "wind_eval_joint_window_static", "wind_profile_decode", "wind_beam_workspace_bytes", "wind_beam_search", "wind_plan_batches", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_debug_stall_barrier", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
+    "wind_set_loop_options", "wind_debug_plan",
 ]
 
 _vp = C.c_void_p
@@ -51,6 +52,7 @@ class wind_stats_t(C.Structure):
         ("steps", C.c_int64), ("joint_rows", C.c_int64), ("tokens", C.c_int64), ("forced", C.c_int64),
         ("frames", C.c_int64), ("jump_hist", C.c_int64 * 65), ("status", C.c_int32),
         ("launches_per_step", C.c_int32), ("launches_setup", C.c_int32), ("kernels", C.c_int32),
+        ("timeout_site", C.c_int32), ("timeout_cta", C.c_int32),
     ]
 
     def as_dict(self) -> Dict[str, object]:
@@ -66,6 +68,17 @@ class wind_profile_t(C.Structure):
         ("pred_launches", C.c_int64),
         ("loop_ms", C.c_double), ("lstm_ms", C.c_double), ("proj_ms", C.c_double), ("gate_table_ms", C.c_double),
     ]
+
+
+class wind_plan_t(C.Structure):
+    _fields_ = [(k, C.c_int32) for k in (
+        "grid", "resident", "smem_bytes", "nj", "vt_count", "rg_count", "rg_stride", "j_mode", "tm_j", "tm_l", "tm_p",
+        "nl", "np", "ut_count", "ht_count", "ql_count", "qp_count", "l_items", "p_items", "w_first", "w_count", "l_sets",
+        "tile_bytes", "buf_off", "z_off", "z_off_p", "stage_off",
+        "slots", "ul", "ug_count", "mt_count", "hg_count", "stages_lp", "stages_j", "stage_lp", "stage_j")]
+
+    def as_dict(self) -> Dict[str, int]:
+        return {k: int(getattr(self, k)) for k, _ in self._fields_}
 
 
 class wind_trace_event_t(C.Structure):
@@ -123,6 +136,10 @@ def load_library():
     L.wind_debug_stall_barrier.restype = i32
     L.wind_set_kernels.argtypes = [i32]
     L.wind_set_kernels.restype = i32
+    L.wind_set_loop_options.argtypes = [i32, i32, i32]
+    L.wind_set_loop_options.restype = None
+    L.wind_debug_plan.argtypes = [mp, i32, i32, i32, i32, C.POINTER(wind_plan_t)]
+    L.wind_debug_plan.restype = i32
     L.wind_status_string.argtypes = [i32]
     L.wind_status_string.restype = C.c_char_p
     L.wind_last_cuda_error.argtypes = []
@@ -143,6 +160,25 @@ class WindError(RuntimeError):
 
 def wind_status_string(status: int) -> str:
     return load_library().wind_status_string(status).decode()
+
+
+def wind_set_loop_options(resident: bool = True, joint_placement: int = -1, max_joint_waves: int = 4) -> None:
+    """Options of the loop kernels' tile planner (process-wide); the defaults restore normal operation."""
+    load_library().wind_set_loop_options(int(bool(resident)), int(joint_placement), int(max_joint_waves))
+
+
+def wind_debug_plan(dims: Dict[str, int], B: int, W: int, sms: int = 148, smem_optin: int = 232448):
+    """The tile plan for bf16 model dimensions `dims` (D, E, P, L, H, V) on a device with the given SM count and
+    opt-in shared memory: host arithmetic only (no GPU needed).  Returns (status, dict of the plan's fields)."""
+    m = wind_model_t()
+    for k in ("D", "E", "P", "L", "H", "V"):
+        setattr(m, k, int(dims[k]))
+    m.blank_id = int(dims.get("blank_id", dims["V"]))
+    m.act = 0
+    m.dtype = WIND_DT_BF16
+    out = wind_plan_t()
+    st = load_library().wind_debug_plan(C.byref(m), B, W, sms, smem_optin, C.byref(out))
+    return st, out.as_dict()
 
 
 def wind_set_trace(first_step: int) -> int:

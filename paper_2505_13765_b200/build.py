@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libwind_b200.so")
-SOURCES = ["wind_api.cu", "wind_control.cu", "wind_simt.cu", "wind_tc.cu", "wind_loop.cu", "wind_first_output.cu", "wind_beam.cu"]
+SOURCES = ["wind_api.cu", "wind_control.cu", "wind_simt.cu", "wind_tc.cu", "wind_loop.cu", "wind_loop_res.cu", "wind_first_output.cu", "wind_beam.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
     "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC,

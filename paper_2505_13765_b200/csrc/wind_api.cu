@@ -184,22 +184,6 @@ static wind_status_t enqueue_decode(Call& c) {
     WIND_CUDA(launch_init(c, WIND_KERNELS_SIMT, per_step, setup));
     WIND_CUDA(simt_enc_proj(c));
     WIND_CUDA(simt_pred_step(c, 0));  // start of sequence: h[0] (zeros) -> h[1]
-    const char* mode = getenv("WIND_LOOP");
-    if (mode && strcmp(mode, "host") == 0) {
-        // bring-up aid: fixed-size bursts of steps, the host polls the active count between bursts
-        cudaGraphConditionalHandle none{};
-        for (;;) {
-            for (int k = 0; k < 8; ++k) {
-                WIND_CUDA(enqueue_step(c, false, 1, none, 0));
-                WIND_CUDA(enqueue_step(c, false, 0, none, 0));
-            }
-            Ctrl hc;
-            WIND_CUDA(cudaMemcpyAsync(&hc, c.ctrl(), sizeof(Ctrl), cudaMemcpyDeviceToHost, c.stream));
-            WIND_CUDA(cudaStreamSynchronize(c.stream));
-            if (hc.active == 0) break;
-        }
-        return WIND_OK;
-    }
     cudaGraphExec_t exec = nullptr;
     wind_status_t s = get_loop_graph(c, false, &exec);
     if (s != WIND_OK) return s;
@@ -602,10 +586,42 @@ wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t*
     host_out->launches_per_step = hc.launches_per_step;
     host_out->launches_setup = hc.launches_setup;
     host_out->kernels = hc.kernels;
+    host_out->timeout_site = hc.timeout_site;
+    host_out->timeout_cta = hc.timeout_cta;
     return WIND_OK;
 }
 
 int32_t wind_debug_stall_barrier(int32_t extra_arrivals) { return loop_set_extra_arrivals(extra_arrivals); }
+
+void wind_set_loop_options(int32_t resident, int32_t joint_placement, int32_t max_joint_waves) {
+    LoopOptions o;
+    o.resident = resident != 0;
+    o.joint_placement = joint_placement >= 0 && joint_placement <= 2 ? joint_placement : -1;
+    o.max_joint_waves = max_joint_waves >= 1 && max_joint_waves <= 4 ? max_joint_waves : 4;
+    loop_set_options(o);
+}
+
+wind_status_t wind_debug_plan(const wind_model_t* m, int32_t B, int32_t W, int32_t sms, int32_t smem_optin, wind_plan_t* out) {
+    wind_status_t s = check_model(m);
+    if (s != WIND_OK) return s;
+    if (!out || B < 1 || W < 1 || W > kMaxWindow || sms < 1 || smem_optin < 1) return WIND_ERR_INVALID_ARG;
+    memset(out, 0, sizeof(*out));
+    if (!(m->dtype == WIND_DT_BF16 && m->D % 64 == 0 && m->E % 64 == 0 && m->P % 64 == 0 && m->H % 64 == 0 && m->V + 1 >= 128))
+        return WIND_ERR_UNSUPPORTED;
+    LoopPlan pl;
+    if (loop_plan_for(*m, B, W, sms, smem_optin, &pl) != cudaSuccess) return WIND_ERR_UNSUPPORTED;
+    out->grid = pl.grid; out->resident = pl.resident; out->smem_bytes = (int32_t)pl.smem_bytes;
+    out->nj = pl.nj; out->vt_count = pl.vt_count; out->rg_count = pl.rg_count; out->rg_stride = pl.rg_stride; out->j_mode = pl.j_mode;
+    out->tm_j = pl.tm_j; out->tm_l = pl.tm_l; out->tm_p = pl.tm_p;
+    out->nl = pl.nl; out->np = pl.np; out->ut_count = pl.ut_count; out->ht_count = pl.ht_count; out->ql_count = pl.ql_count;
+    out->qp_count = pl.qp_count; out->l_items = pl.l_items; out->p_items = pl.p_items; out->w_first = pl.w_first; out->w_count = pl.w_count;
+    out->tile_bytes = (int32_t)pl.stat_bytes; out->buf_off = (int32_t)pl.buf_off; out->z_off = (int32_t)pl.z_off;
+    out->z_off_p = (int32_t)pl.z_off_p; out->stage_off = (int32_t)pl.stage_off;
+    out->slots = pl.slots; out->ul = pl.ul; out->ug_count = pl.ug_count; out->mt_count = pl.mt_count; out->hg_count = pl.hg_count;
+    out->stages_lp = pl.stages_lp; out->stages_j = pl.stages_j; out->stage_lp = (int32_t)pl.stage_lp; out->stage_j = (int32_t)pl.stage_j;
+    out->l_sets = pl.resident ? (m->L == 2 ? 3 : 1) : 0;
+    return WIND_OK;
+}
 
 int32_t wind_set_trace(int32_t first_step) {
     int32_t prev = g_trace_step;

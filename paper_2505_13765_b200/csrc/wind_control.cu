@@ -8,7 +8,7 @@ namespace wind {
 // Reset all per-call state.  Block 0 also fills the control block.
 __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsigned long long* t_pub, int32_t* count, int32_t* emit_tok,
                                                    unsigned long long* keys, float* h, float* c, uint32_t* hb, uint32_t* z,
-                                                   uint32_t* trace, size_t n_trace_words, int32_t* out_len, const int32_t* __restrict__ enc_len, int B, int T, size_t n_keys,
+                                                   uint32_t* trace, size_t n_trace_words, uint32_t* sync_words, size_t n_sync_words, int32_t* out_len, const int32_t* __restrict__ enc_len, int B, int T, size_t n_keys,
                                                    size_t n_h, size_t n_c, size_t n_hb_words, size_t n_z_words,
                                                    int blank, int step_cap, int kernels_used, int launches_per_step,
                                                    int launches_setup) {
@@ -19,6 +19,7 @@ __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsig
     for (size_t i = gtid; i < n_hb_words; i += gstride) hb[i] = 0u;
     for (size_t i = gtid; i < n_z_words; i += gstride) z[i] = 0u;
     for (size_t i = gtid; i < n_trace_words; i += gstride) trace[i] = 0u;
+    for (size_t i = gtid; i < n_sync_words; i += gstride) sync_words[i] = 0u;   // arrival counters and the stamps of pred_proj
     for (size_t i = gtid; i < n_keys; i += gstride) keys[i] = 0ull;
     for (size_t i = gtid; i < (size_t)B; i += gstride) {
         t[i] = 0;
@@ -62,6 +63,8 @@ __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsig
             ctrl->abort = 0;
             for (int k = 0; k < 4; ++k) ctrl->phase_cycles[k] = 0;
             ctrl->loop_ns = 0;
+            ctrl->timeout_site = 0;
+            ctrl->timeout_cta = 0;
         }
     }
 }
@@ -81,7 +84,9 @@ cudaError_t launch_init(const Call& c, int kernels_used, int launches_per_step, 
     init_kernel<<<blocks, 256, 0, c.stream>>>(c.ctrl(), c.t(), c.t_pub(), c.count(), c.emit_tok(), c.keys(), c.h(0), c.c(),
                                               reinterpret_cast<uint32_t*>(c.hb(0, 0)), reinterpret_cast<uint32_t*>(c.z()),
                                               reinterpret_cast<uint32_t*>(c.trace()),
-                                              bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents / 4 : 0, c.out_len, c.enc_len, c.B, c.T, 3 * (size_t)c.lay.rows_pad, n_h, n_c, n_hb_words,
+                                              bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents / 4 : 0,
+                                              reinterpret_cast<uint32_t*>(c.flags()), bf ? (c.lay.enc_proj - c.lay.flags) / 4 : 0,   // the counters and pred_pub lie side by side, before enc_proj
+                                              c.out_len, c.enc_len, c.B, c.T, 3 * (size_t)c.lay.rows_pad, n_h, n_c, n_hb_words,
                                               n_z_words, c.m.blank_id, (int)step_cap, kernels_used, launches_per_step,
                                               launches_setup);
     return cudaGetLastError();

@@ -46,6 +46,8 @@ struct Ctrl {
     int32_t abort;            // some CTA gave up: everybody leaves
     long long phase_cycles[4];  // SM cycles spent in the joint / decoder-update / projection phases (CTA 0), [3] unused
     long long loop_ns;        // wall time of the loop kernel (CTA 0, global timer)
+    int32_t timeout_site;     // which wait ran out first (resident-weights loop kernel; 0 = none), and in which CTA
+    int32_t timeout_cta;
 };
 
 // Byte offsets of every workspace region (all multiples of kAlign).
@@ -75,7 +77,7 @@ struct Layout {
     size_t st_enc, st_len, st_tok, st_frm, st_olen, st_total;
     int32_t Bpad;      // B rounded up to 128 (tensor path operand rows)
     int32_t rows_pad;  // B*W rounded up to 256 (window rows incl. tile padding)
-    int32_t n_flags;   // one counter per 16 window rows and three per 16 utterances always suffice
+    int32_t n_flags;   // one counter per 16 window rows of the widest window and three per 16 utterances always suffice
 };
 
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -104,7 +106,7 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     L.trace = take(bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents : 0);
     L.jpart = take(bf ? sizeof(float) * 2 * (size_t)L.rows_pad * 4 * ((size_t)(m.V + 1 + 127) / 128) : 0);
     L.jblank = take(bf ? sizeof(float) * (size_t)L.rows_pad : 0);
-    L.n_flags = L.rows_pad / 16 + 3 * (B / 16 + 1);
+    L.n_flags = B * (kMaxWindow / 16) + 16 + 3 * (B / 16 + 1);   // independent of W: row groups have at least 16 rows
     L.flags = take(bf ? sizeof(uint32_t) * (size_t)L.n_flags : 0);
     L.pred_pub = take(bf ? 8 * (size_t)B * m.H : 0);
     L.enc_proj = take(es * (size_t)B * T * m.H);

@@ -105,6 +105,13 @@ struct LoopParams {
     unsigned long long* pred_pub;  // [B][H] (fp32 value, stamp)
 };
 
+// Options of the tile planner (process-wide; wind_set_loop_options): whether the resident-weights mode may be chosen,
+// a forced placement of the streaming mode's W_out tile (-1: the planner's own choice; 0 streamed, 1 shared memory,
+// 2 tensor memory, taken when feasible), and the most waves the resident joint may run in (1..4).
+struct LoopOptions { int resident; int joint_placement; int max_joint_waves; };
+void loop_set_options(const LoopOptions& o);
+LoopOptions loop_get_options();
+bool loop_plan_ok(const wind_model_t& m, int B, int W);
 cudaError_t loop_plan(const Call& c, LoopPlan* out);
 // the plan as a pure function of the shapes and of the device's SM count and opt-in shared memory per block
 cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem_optin, LoopPlan* out);

@@ -164,15 +164,30 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
     uint32_t* f_h1 = f_h0 + p.ql_count;          // [ql_count]  layer-1 state written (two layers)
     uint32_t* f_dh = f_h1 + p.ql_count;          // [ql_count]  layer 1's recurrent term written (two layers)
     // arrivals per decoder-update slot on group ql's layer-0 counter: its unit tiles, plus (when separate CTAs record
-    // the steps) one per block of 32 utterances that overlaps the group
+    // the steps) one per block of 32 utterances that overlaps the group.  Under teacher forcing nothing is recorded
+    // and the recording CTAs stay out: a counter that sums arrivals over slots is only sound while no participant
+    // can run ahead of the others, and a CTA with nothing to wait for could.
     auto arr_h0 = [&](int ql) -> uint32_t {
         uint32_t a = (uint32_t)p.ut_count;
         const int lo = ql * p.nl, hi = min(lo + p.nl, p.B);
-        if (p.w_count > 0 && hi > lo) a += (uint32_t)((hi - 1) / 32 - lo / 32 + 1);
+        if (p.w_count > 0 && !forced && hi > lo) a += (uint32_t)((hi - 1) / 32 - lo / 32 + 1);
         return a;
     };
+    // a wait of this CTA ran out: note which one (the first in the grid stays), flag the CTA and everybody else
+    auto give_up = [&](int site) {
+        if (atomicCAS(&p.ctrl->timeout_site, 0, site) == 0) p.ctrl->timeout_cta = cta;
+        *vabort = 1;
+        atomicExch(&p.ctrl->abort, 1);
+    };
+    // bounded mbarrier wait that notes its site when it is the one that runs out
+    auto mwait = [&](uint64_t* bar, uint32_t parity, int site) -> bool {
+        const int before = *vabort;
+        const bool ok = mbar_wait(bar, parity, vabort);
+        if (!ok && before == 0 && *vabort == 1) give_up(site);
+        return ok;
+    };
     // one thread waits until a counter has reached its target; false when the kernel is being abandoned
-    auto flag_wait = [&](const uint32_t* ptr, uint32_t target) -> bool {
+    auto flag_wait = [&](const uint32_t* ptr, uint32_t target, int site) -> bool {
         unsigned long long t0 = 0;
         for (uint32_t it = 1;; ++it) {
             if ((int32_t)(ld_acquire_u32(ptr) - target) >= 0) return true;
@@ -181,12 +196,12 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                 if (ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; return false; }
                 const unsigned long long now = globaltimer_ns();
                 if (t0 == 0) t0 = now;
-                else if (now - t0 > kWaitLimitNs) { *vabort = 1; atomicExch(&p.ctrl->abort, 1); return false; }
+                else if (now - t0 > kWaitLimitNs) { give_up(site); return false; }
             }
         }
     };
     // a whole warp waits for counters base[first .. first + count): lane i polls counter i (, i + 32, ...)
-    auto warp_flag_wait = [&](const uint32_t* base, int first, int count, uint32_t target) -> bool {
+    auto warp_flag_wait = [&](const uint32_t* base, int first, int count, uint32_t target, int site) -> bool {
         bool ok = true;
         for (int i0 = 0; i0 < count && ok; i0 += 32) {
             const int i = i0 + lane;
@@ -200,7 +215,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                     if (!quit && ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; quit = true; }
                     const unsigned long long now = globaltimer_ns();
                     if (t0 == 0) t0 = now;
-                    else if (!quit && now - t0 > kWaitLimitNs) { *vabort = 1; atomicExch(&p.ctrl->abort, 1); quit = true; }
+                    else if (!quit && now - t0 > kWaitLimitNs) { give_up(site); quit = true; }
                     if (__any_sync(0xffffffffu, quit)) { ok = false; break; }
                 }
             }
@@ -244,7 +259,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
             } else {
                 __threadfence();
                 atomicAdd(&p.ctrl->bar, 1u);
-                flag_wait(&p.ctrl->bar, epoch);
+                flag_wait(&p.ctrl->bar, epoch, 1);
             }
         }
         __syncthreads();
@@ -258,10 +273,10 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
     auto mma_part = [&](int k_acc, uint32_t tm_d, int n_tile, int kb_lo, int kb_hi, bool a_tmem, int sidx, uint32_t use,
                         const uint8_t* b_smem) -> bool {
         const uint32_t idesc = idesc_bf16(a_tmem ? 128 : 64, n_tile);
-        if (!a_tmem && !mbar_wait(&stat_bar, 0, vabort)) return false;
-        if (!mbar_wait(&acc_empty[k_acc], (acc_n[k_acc] & 1u) ^ 1u, vabort)) return false;   // the epilogue has drained it
+        if (!a_tmem && !mwait(&stat_bar, 0, 10)) return false;
+        if (!mwait(&acc_empty[k_acc], (acc_n[k_acc] & 1u) ^ 1u, 11 + k_acc)) return false;   // the epilogue has drained it
         tc_fence_after();
-        if (!mbar_wait(&full_bar[sidx], use & 1u, vabort)) return false;
+        if (!mwait(&full_bar[sidx], use & 1u, 14 + sidx)) return false;
         tc_fence_after();
         const uint32_t b_addr = smem_u32(b_smem);
         const uint32_t b_block = (uint32_t)n_tile * BK * 2;
@@ -287,8 +302,8 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
     // the state box of this step: ONE three-dimensional TMA box (64 columns, rows, all K blocks), once the MMAs
     // that read the buffer last have completed
     auto produce_box = [&](const CUtensorMap* map, int row0, uint32_t bytes) -> bool {
-        if (use0 > 0 && !mbar_wait(&empty_bar[0], (use0 - 1) & 1u, vabort)) return false;
-        if (z_sh && use1 > 0 && !mbar_wait(&empty_bar[1], (use1 - 1) & 1u, vabort)) return false;
+        if (use0 > 0 && !mwait(&empty_bar[0], (use0 - 1) & 1u, 16)) return false;
+        if (z_sh && use1 > 0 && !mwait(&empty_bar[1], (use1 - 1) & 1u, 17)) return false;
         mbar_expect_tx(&full_bar[0], bytes);
         tma_load_3d(buf0, map, 0, row0, 0, &full_bar[0]);
         return true;
@@ -329,12 +344,19 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
             const int b_hi = min(base + n_here, p.B);
             if (b_hi > base) {
                 const int rg_lo = base * p.W / p.nj, rg_hi = (b_hi * p.W - 1) / p.nj;
-                ready = warp_flag_wait(f_keys, rg_lo, rg_hi - rg_lo + 1, n_j * (uint32_t)p.vt_count + (uint32_t)p.extra_arrivals);
+                ready = warp_flag_wait(f_keys, rg_lo, rg_hi - rg_lo + 1, n_j * (uint32_t)p.vt_count + (uint32_t)p.extra_arrivals, 20);
             }
+        } else if (forced && p.L == 2 && layer == 0 && n_l >= 2u) {
+            // Teacher forcing feeds tokens without waiting for keys, so nothing else holds layer 0 back: before this
+            // slot overwrites the state buffer it wrote two slots ago, layer 1's CTAs must have read it (their arrivals
+            // of the slot before last).  While decoding, the wait for the keys implies this.
+            bool ok = true;
+            if (lane == 0) ok = flag_wait(f_h1 + r_ql, (n_l - 1u) * (uint32_t)p.ut_count, 21);
+            ready = __all_sync(0xffffffffu, ok);
         } else if (layer > 0) {
             // layer 1: the step's tokens (recorded with layer 0's arrivals) and the recurrent term computed a slot ahead
             bool ok = true;
-            if (lane == 0) ok = flag_wait(f_h0 + r_ql, n_l * arr_h0(r_ql)) && flag_wait(f_dh + r_ql, n_l * (uint32_t)p.ut_count);
+            if (lane == 0) ok = flag_wait(f_h0 + r_ql, n_l * arr_h0(r_ql), 22) && flag_wait(f_dh + r_ql, n_l * (uint32_t)p.ut_count, 23);
             ready = __all_sync(0xffffffffu, ok);
         }
         for (int c0 = 0; c0 < n_here; c0 += 64) {
@@ -475,7 +497,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
             int* tok_s = reinterpret_cast<int*>(stage_f + 4 * 64 * 16);
             if (q == 0) tok_s[jl] = tok;
             if (c0 == 0) {
-                const bool acc_ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, vabort));
+                const bool acc_ok = __all_sync(0xffffffffu, mwait(&acc_full[1], acc_n[1] & 1u, 30));
                 ready = ready && acc_ok;
                 tc_fence_after();
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
@@ -548,7 +570,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
     auto epilogue_res_P = [&](uint32_t stamp) -> bool {
         const int h0 = r_ht * 64;
         if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
-        const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[2], acc_n[2] & 1u, vabort));
+        const bool ready = __all_sync(0xffffffffu, mwait(&acc_full[2], acc_n[2] & 1u, 31));
         tc_fence_after();
         if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
         if (ready) {
@@ -593,7 +615,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
     // h1 CTAs: the finished recurrent term of layer 1 goes to global memory (fp32 [B][4P], gate-major like the gate
     // table); the x1 CTAs add it in the next decoder-update slot
     auto store_res_h1 = [&]() {
-        const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, vabort));
+        const bool ready = __all_sync(0xffffffffu, mwait(&acc_full[1], acc_n[1] & 1u, 32));
         tc_fence_after();
         if (ready) {
             const int unit = r_ut * 16 + (lane & 15);
@@ -629,7 +651,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
         if (warp == 0) {
             if (lane == 0 && mine) {
                 // the state of this CTA's utterance group as the last decoder-update slot left it
-                const bool ok = res_l ? flag_wait(f_h0 + r_ql, n_l * arr_h0(r_ql)) : flag_wait(f_h1 + r_ql, n_l * (uint32_t)p.ut_count);
+                const bool ok = res_l ? flag_wait(f_h0 + r_ql, n_l * arr_h0(r_ql), 24) : flag_wait(f_h1 + r_ql, n_l * (uint32_t)p.ut_count, 25);
                 if (ok) {
                     fence_proxy_async_all();
                     if (produce_box(res_l ? &M.hb_l3[pin] : &M.hb_l3_1[pin], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u))
@@ -678,7 +700,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                         if (ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; break; }
                         const unsigned long long now = globaltimer_ns();
                         if (t0 == 0) t0 = now;
-                        else if (now - t0 > kWaitLimitNs) { *vabort = 1; atomicExch(&p.ctrl->abort, 1); break; }
+                        else if (now - t0 > kWaitLimitNs) { give_up(40); break; }
                     }
                 }
                 t = (int)(uint32_t)v;
@@ -689,8 +711,8 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
         }
         asm volatile("bar.sync 1, 256;" ::: "memory");
         // the buffer is free once the MMAs that read it last have completed
-        bool ok = use1 == 0 || mbar_wait(&empty_bar[1], (use1 - 1) & 1u, vabort);
-        if (ok && z_sh && use0 > 0) ok = mbar_wait(&empty_bar[0], (use0 - 1) & 1u, vabort);
+        bool ok = use1 == 0 || mwait(&empty_bar[1], (use1 - 1) & 1u, 18);
+        if (ok && z_sh && use0 > 0) ok = mwait(&empty_bar[0], (use0 - 1) & 1u, 19);
         if (ok && *vabort == 0) {
             for (int idx = e; idx < n_utt * n_chunks; idx += 256) {
                 const int ul = idx / n_chunks, c = idx - ul * n_chunks;
@@ -751,7 +773,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                     if (ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; break; }
                     const unsigned long long now = globaltimer_ns();
                     if (t0 == 0) t0 = now;
-                    else if (now - t0 > kWaitLimitNs) { *vabort = 1; atomicExch(&p.ctrl->abort, 1); break; }
+                    else if (now - t0 > kWaitLimitNs) { give_up(41); break; }
                 }
             }
             if (!waited) { asm volatile("cp.async.wait_all;" ::: "memory"); waited = true; }
@@ -795,7 +817,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
         if (warp >= 2) {
             if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_START);
             if (res_l) epilogue_res_L(0, false);
-            else if (res_w) epilogue_res_L(0, true);
+            else if (res_w && !forced) epilogue_res_L(0, true);
             if (cta == 0 && e == 0 && step >= 0 && !forced) p.ctrl->step = step + 1;
             // CTAs whose joint operand has a buffer of its own start on the next window now
             if (has_j && !z_sh && !forced) { prep_A(j_first, n_l + 1u); prepped = true; }
@@ -806,7 +828,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
             // layer 1: W_ih[1] . (new layer-0 state) on the x1 CTAs, then their cell update
             if (warp == 0) {
                 if (lane == 0 && res_x1) {
-                    if (flag_wait(f_h0 + r_ql, n_l * arr_h0(r_ql))) {
+                    if (flag_wait(f_h0 + r_ql, n_l * arr_h0(r_ql), 26)) {
                         fence_proxy_async_all();
                         if (produce_box(&M.hb_l3[pin ^ 1], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u))
                             mma_part(1, tm_l, p.nl, p.kb_p, p.kb_p, false, 0, use0, buf0);
@@ -839,7 +861,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                 bool ok = true;
                 if (b_hi > b_lo)
                     for (int g = b_lo / p.nl; ok && g <= (b_hi - 1) / p.nl; ++g)
-                        ok = flag_wait(f + g, n_l * (p.L == 2 ? (uint32_t)p.ut_count : arr_h0(g)));
+                        ok = flag_wait(f + g, n_l * (p.L == 2 ? (uint32_t)p.ut_count : arr_h0(g)), 27);
                 if (ok) {
                     fence_proxy_async_all();
                     if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_P, EV_FIRST_ISSUE);
@@ -854,6 +876,8 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
             if (warp == 2 && !forced) {
                 // utterances still decoding, from the frames the recording threads have published for this step
                 // (every CTA reads the same words, so all take the same exit)
+                // A CTA that lags may find a later stamp: the recording threads only go on when utterances are left,
+                // so a later stamp means "not finished" (the count itself is then of no interest).
                 int alive = 0;
                 unsigned long long t0 = 0;
                 for (uint32_t it = 1;; ++it) {
@@ -862,8 +886,9 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                     for (int b = lane; b < p.B; b += 32) {
                         unsigned long long v;
                         asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(v) : "l"(p.t_pub + b) : "memory");
-                        all = all && (uint32_t)(v >> 32) == n_l;
-                        alive += (int)(uint32_t)v < p.enc_len[b];
+                        const int32_t ahead = (int32_t)((uint32_t)(v >> 32) - n_l);
+                        all = all && ahead >= 0;
+                        alive += (ahead > 0 || (int)(uint32_t)v < p.enc_len[b]) ? 1 : 0;
                     }
                     if (__all_sync(0xffffffffu, all)) break;
                     if ((it & 15u) == 0u) {
@@ -871,7 +896,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                         if (!quit && ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; quit = true; }
                         const unsigned long long now = globaltimer_ns();
                         if (t0 == 0) t0 = now;
-                        else if (!quit && now - t0 > kWaitLimitNs) { *vabort = 1; atomicExch(&p.ctrl->abort, 1); quit = true; }
+                        else if (!quit && now - t0 > kWaitLimitNs) { give_up(42); quit = true; }
                         if (__any_sync(0xffffffffu, quit)) break;
                     }
                 }
@@ -916,7 +941,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                     prepped = false;
                     prep_B(rg, n_p);
                     if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_TOK);
-                    const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[0], acc_n[0] & 1u, vabort));
+                    const bool ready = __all_sync(0xffffffffu, mwait(&acc_full[0], acc_n[0] & 1u, 33));
                     tc_fence_after();
                     if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_ACC);
                     if (ready) joint_epilogue_item<true, FULL>(p, tm_j, lane_off, lane, q, sub, row_in_tile, rg, my_vt, n_tile, t_cur, keys_cur);

@@ -55,8 +55,9 @@ static cudaError_t make_map(CUtensorMap* map, const void* base, uint64_t rows, u
 }
 
 bool tc_supported(const wind_model_t& m, int B, int T, int W) {
-    (void)B; (void)T; (void)W;
-    return m.dtype == WIND_DT_BF16 && m.D % 64 == 0 && m.E % 64 == 0 && m.P % 64 == 0 && m.H % 64 == 0 && m.V + 1 >= 128;
+    (void)T;
+    if (!(m.dtype == WIND_DT_BF16 && m.D % 64 == 0 && m.E % 64 == 0 && m.P % 64 == 0 && m.H % 64 == 0 && m.V + 1 >= 128)) return false;
+    return loop_plan_ok(m, B, W);   // the loop kernels have a tile plan for these shapes on this device
 }
 
 static thread_local TcMaps t_maps;
@@ -256,10 +257,14 @@ constexpr size_t gemm_smem_bytes() { return (size_t)GemmShape<MODE>::STAGES * (A
 
 // Shared-memory opt-in of the kernels of this file.
 static cudaError_t tc_set_attributes() {
-    static bool done = false;
+    static bool done_on[64] = {};   // the attribute belongs to the (function, device) pair
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     std::lock_guard<std::mutex> lock(g_tc_mutex);
+    bool& done = done_on[dev];
     if (done) return cudaSuccess;
-    cudaError_t e;
     if ((e = cudaFuncSetAttribute(gemm_kernel<MODE_ENC_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem_bytes<MODE_ENC_PROJ>())) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(gemm_kernel<MODE_GATE_TABLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem_bytes<MODE_GATE_TABLE>())) != cudaSuccess) return e;
     done = true;

@@ -10,3 +10,12 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: test needs a CUDA device (run with -m gpu on a B200)")
+
+
+@pytest.fixture(autouse=True)
+def _restore_loop_options():
+    """Tests that force a mode of the loop kernels (wind_set_loop_options) leave the process-wide default behind them."""
+    yield
+    from paper_2505_13765_b200 import binding
+    if binding._lib is not None:
+        binding.wind_set_loop_options()

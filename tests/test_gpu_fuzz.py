@@ -38,7 +38,7 @@ def test_small_dimensions_many_utterances(pkg, monkeypatch, seed):
         W = int(r.choice([1, 2, 3, 5, 8, 13, 16, 24, 40])); L = int(r.choice([1, 1, 2, 2, 3])); S = int(r.integers(1, 6))
         act = int(r.integers(0, 2)); blank0 = bool(r.integers(0, 2)); res = int(r.integers(0, 2)); T = int(r.integers(8, 40))
         win = bool(r.integers(0, 3) == 0)
-        monkeypatch.setenv("WIND_RESIDENT", str(res))
+        pkg.wind_set_loop_options(resident=bool(res))
         w, enc, lens = tp.ragged_case(9000 + i, B=B, T=T, D=64, E=int(r.choice([64, 128])), P=P, L=L, H=H, V=V, act=act,
                                       blank_id=0 if blank0 else None, bias=float(r.uniform(0.5, 3.0)), dtype="bf16")
         print(f"case {i}: B={B} T={T} W={W} S={S} P={P} H={H} V={V} L={L} resident={res} window={win}", flush=True)
@@ -56,7 +56,7 @@ def test_large_dimensions(pkg, monkeypatch):
         W = int(r.choice([1, 2, 4, 8, 16, 32, 64])); L = int(r.choice([1, 2])); S = int(r.integers(1, 11)); act = int(r.integers(0, 2))
         res = int(r.integers(0, 2)); T = int(r.integers(4, 16)); kind = int(r.integers(0, 4)); D = int(r.choice([64, 512]))
         E = int(r.choice([64, 640]))
-        monkeypatch.setenv("WIND_RESIDENT", str(res))
+        pkg.wind_set_loop_options(resident=bool(res))
         w, enc, lens = tp.ragged_case(9500 + i, B=B, T=T, D=D, E=E, P=P, L=L, H=H, V=V, act=act, blank_id=0 if i % 3 == 0 else None,
                                       bias=float(r.uniform(0.5, 3.0)), dtype="bf16")
         print(f"case {i}: kind={kind} B={B} T={T} W={W} S={S} D={D} E={E} P={P} H={H} V={V} L={L} resident={res}", flush=True)

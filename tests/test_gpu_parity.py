@@ -284,9 +284,9 @@ def test_bf16_tensor_path_with_biases_and_other_blank_ids(pkg, L, blank0, act, B
 @pytest.mark.parametrize("resident", [1, 0])
 def test_bf16_tensor_path_more_utterances_than_one_tile(pkg, monkeypatch, resident):
     # 150 utterances, one K block per GEMM (H = P = 64): ten utterance groups per weight tile in the resident-weights
-    # mode; two 128-row utterance tiles in the streaming mode (forced by the planner's environment switch)
+    # mode; two 128-row utterance tiles in the streaming mode (forced through wind_set_loop_options)
     if not resident:
-        monkeypatch.setenv("WIND_RESIDENT", "0")
+        pkg.wind_set_loop_options(resident=False)
     w, enc, lens = ragged_case(91, B=150, T=24, D=64, E=64, P=64, L=1, H=64, V=140, act=0, bias=1.0, dtype="bf16")
     rep, _ = check_against_oracle(pkg, w, enc, lens, 4, 3, kernels=2)
     assert rep["stats"]["kernels"] == 2
@@ -310,9 +310,9 @@ def test_bf16_tensor_path_more_utterances_than_one_tile(pkg, monkeypatch, reside
 @pytest.mark.parametrize("resident", [1, 0])
 def test_bf16_tensor_path_shape_sweep(pkg, monkeypatch, resident, B, W, S, P, H, V, L):
     # shapes that send the tile planner of the loop kernel down its different branches, with the resident-weights
-    # mode allowed and with the planner's environment switch forcing the streaming mode
+    # mode allowed and with wind_set_loop_options forcing the streaming mode
     if not resident:
-        monkeypatch.setenv("WIND_RESIDENT", "0")
+        pkg.wind_set_loop_options(resident=False)
     w, enc, lens = ragged_case(300 + B + W, B=B, T=20, D=64, E=64, P=P, L=L, H=H, V=V, act=B % 2, bias=1.5,
                                dtype="bf16")
     rep, _ = check_against_oracle(pkg, w, enc, lens, W, S, kernels=2)
@@ -407,7 +407,7 @@ def test_argmax_ties_go_to_the_lowest_index_on_the_gpu(pkg, monkeypatch, path, b
     # 64-bit keys), a label against the blank, and every entry equal.  The expected transcripts are written from the
     # rule (lowest index wins), and the oracle must give the same.
     if path == "bf16_tensor_streaming":
-        monkeypatch.setenv("WIND_RESIDENT", "0")
+        pkg.wind_set_loop_options(resident=False)
     w, target, winners = tie_model(blank_id=0 if blank_first else None, dtype="f32" if path == "f32" else "bf16")
     blank = w["blank_id"]
     enc, lens = tie_utterances(w["D"], TIE_UTTS)

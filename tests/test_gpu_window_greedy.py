@@ -116,7 +116,7 @@ def test_bf16_both_kernel_sets(pkg, kernels, L, W, B):
 
 
 def test_bf16_streaming_mode_of_the_loop_kernel(pkg, monkeypatch):
-    monkeypatch.setenv("WIND_RESIDENT", "0")
+    pkg.wind_set_loop_options(resident=False)
     w, enc, lens = ragged_case(531, B=150, T=30, D=64, E=64, P=64, L=1, H=128, V=257, act=0, bias=1.5, dtype="bf16")
     rep, _ = check_window_greedy(pkg, w, enc, lens, 8, 3, kernels=2)
     assert rep["stats"]["kernels"] == 2
@@ -150,7 +150,7 @@ def test_cfg3_full_batch_sampled_utterances(pkg):
 def test_bf16_tensor_path_wide_window_and_overflow(pkg, monkeypatch, resident):
     # W = 40: more window rows than lanes in the decision warp; then an output buffer that is too small
     if not resident:
-        monkeypatch.setenv("WIND_RESIDENT", "0")
+        pkg.wind_set_loop_options(resident=False)
     w, enc, lens = ragged_case(540, B=6, T=70, D=64, E=64, P=64, L=1, H=128, V=150, act=1, bias=3.0, dtype="bf16")
     rep, (tok, frm, olen) = check_window_greedy(pkg, w, enc, lens, 40, 2, kernels=2)
     assert rep["stats"]["kernels"] == 2 and olen.max() > 4
