@@ -347,9 +347,13 @@ wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t*
  * (default).  Returns the previous setting.  Recording costs a few stores and does not change results.
  * wind_read_trace copies the records of the last decode that used `workspace` (same m, B, T, W).
  *   role:  0 TMA issuer, 1 MMA issuer, 2 first epilogue thread, 3 grid barrier (4..7: the same of the last CTA);
- *          8, 9, 10: barrier arrival of EVERY CTA at the end of the joint, decoder-update and projection phase
- *          of lock step s; for these records `step` holds the CTA index and `clock` the global timer in
- *          nanoseconds, which is comparable across SMs: who arrives last is what bounds the phase
+ *          8 + k: mark k of EVERY CTA in lock step s; for these records `step` holds the CTA index and `clock` the
+ *          global timer in nanoseconds, which is comparable across SMs (who is last is what bounds a phase).  Marks:
+ *          joint 0 entered, 1 copies of the window's enc_proj rows issued, 2 pred_proj arrived, 3 operand handed to the
+ *          issuing threads, 4 accumulator ready, 5 keys out; decoder update 6 keys of the CTA's utterances complete,
+ *          7 tokens known, 8 accumulator ready, 9 state written; projection 10 state counters seen, 11 accumulator
+ *          ready, 12 pred_proj published, 13 / 14 the GEMM issued ahead of the decoder update (counters seen /
+ *          issued), 15 done.  (The streaming mode records 5, 9 and 15: its barrier arrivals.)
  *   phase: 0 joint, 1 decoder update, 2 projection
  *   event: 0 phase entered, 1 first / 2 last TMA issued, 3 first operands arrived, 4 accumulator
  *          committed, 5 epilogue inputs requested (token known), 6 accumulator ready, 7 epilogue

@@ -188,7 +188,7 @@ def wind_set_trace(first_step: int) -> int:
 
 def wind_read_trace(model: "WindModel", B: int, T: int, W: int, workspace, stream=None) -> List[Dict[str, int]]:
     L = load_library()
-    cap = 4 * 512
+    cap = 24 * 512
     buf = (wind_trace_event_t * cap)()
     n = C.c_int32(0)
     st = L.wind_read_trace(model.ref, B, T, W, _ws_ptr(workspace), _stream_ptr(stream), buf, cap, C.byref(n))

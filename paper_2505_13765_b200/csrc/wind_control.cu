@@ -85,7 +85,7 @@ cudaError_t launch_init(const Call& c, int kernels_used, int launches_per_step, 
                                               reinterpret_cast<uint32_t*>(c.hb(0, 0)), reinterpret_cast<uint32_t*>(c.z()),
                                               reinterpret_cast<uint32_t*>(c.trace()),
                                               bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents / 4 : 0,
-                                              reinterpret_cast<uint32_t*>(c.flags()), bf ? (c.lay.enc_proj - c.lay.flags) / 4 : 0,   // the counters and pred_pub lie side by side, before enc_proj
+                                              reinterpret_cast<uint32_t*>(c.flags()), bf ? (c.lay.enc_proj - c.lay.flags) / 4 : 0,   // the counters, pred_pub and the key slots lie side by side, before enc_proj
                                               c.out_len, c.enc_len, c.B, c.T, 3 * (size_t)c.lay.rows_pad, n_h, n_c, n_hb_words,
                                               n_z_words, c.m.blank_id, (int)step_cap, kernels_used, launches_per_step,
                                               launches_setup);

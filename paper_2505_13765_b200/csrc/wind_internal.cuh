@@ -22,8 +22,8 @@ struct TraceEvent {
     int32_t step;
     long long clock;   // clock64 of the SM that runs CTA 0
 };
-constexpr int kTraceRoles = 11;    // TMA issuer, MMA issuer, first epilogue thread, barrier: of CTA 0, then of the last CTA;
-                                   // 8..10: barrier arrival of every CTA in the joint / decoder / projection phase
+constexpr int kTraceRoles = 24;    // TMA issuer, MMA issuer, first epilogue thread, barrier: of CTA 0, then of the last CTA;
+                                   // 8..23: marks of EVERY CTA in the first traced step (global timer), see trace_mark
 constexpr int kTraceEvents = 512;
 
 // Device control block, first thing in the workspace.
@@ -70,7 +70,8 @@ struct Layout {
     size_t g0;         // fp32 [V+1][4P] layer-0 gate pre-activations of every token: W_ih emb[tok] + b_ih + b_hh (tensor path)
     size_t trace;      // TraceEvent [kTraceRoles][kTraceEvents]: optional timeline of CTA 0 of the loop kernel
     size_t flags;      // uint32 [n_flags] arrival counters between CTA groups of the resident-weights loop kernel
-    size_t pred_pub;   // (fp32, uint32) [B][H] pred_proj values, each stamped with the projection phase that wrote it
+    size_t kslot;      // uint64 [window rows][vocabulary tiles, padded to even] stamped (logit, label) keys, one per window row and vocabulary tile
+    size_t pred_pub;   // (bf16 x 2, uint32) [B][H / 2] pred_proj values in pairs, each pair stamped with the projection phase that wrote it
     size_t enc_proj;   // elem [B*T][H]
     size_t total;
     // host staging (wind_decode_greedy_host), placed after `total`
@@ -108,7 +109,8 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     L.jblank = take(bf ? sizeof(float) * (size_t)L.rows_pad : 0);
     L.n_flags = B * (kMaxWindow / 16) + 16 + 3 * (B / 16 + 1);   // independent of W: row groups have at least 16 rows
     L.flags = take(bf ? sizeof(uint32_t) * (size_t)L.n_flags : 0);
-    L.pred_pub = take(bf ? 8 * (size_t)B * m.H : 0);
+    L.pred_pub = take(bf ? 4 * (size_t)B * m.H : 0);
+    L.kslot = take(bf ? 8 * ((size_t)L.rows_pad + 256) * (((size_t)(m.V + 1 + 127) / 128 + 1) & ~(size_t)1) : 0);
     L.enc_proj = take(es * (size_t)B * T * m.H);
     L.total = off;
     L.st_enc = take(es * (size_t)B * T * m.D);
@@ -159,6 +161,7 @@ struct Call {
     TraceEvent* trace() const { return reinterpret_cast<TraceEvent*>(ws + lay.trace); }
     uint32_t* flags() const { return reinterpret_cast<uint32_t*>(ws + lay.flags); }
     unsigned long long* pred_pub() const { return reinterpret_cast<unsigned long long*>(ws + lay.pred_pub); }
+    unsigned long long* kslot() const { return reinterpret_cast<unsigned long long*>(ws + lay.kslot); }
     __nv_bfloat16* hb(int parity, int l) const {
         return reinterpret_cast<__nv_bfloat16*>(ws + lay.hb) + ((size_t)parity * m.L + l) * lay.Bpad * m.P;
     }

@@ -864,7 +864,7 @@ cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem
     bool resident_done = false;
     for (int ci = 0; ci < n_cands && !resident_done; ++ci) {
         const int r_nj = cands[ci];
-        if (!(m.L <= 2 && m.H / 2 + 2 * r_nj <= (int)LOOP_TMEM_COLS && opt.resident != 0)) continue;
+        if (!(m.L <= 2 && m.H / 2 + 2 * r_nj <= (int)LOOP_TMEM_COLS && opt.resident != 0 && NV <= (1 << 20))) continue;   // (labels take 20 bits of a key slot)
         LoopPlan r = pl;
         r.nj = r_nj;
         r.rg_count = (rows + r_nj - 1) / r_nj;
@@ -1026,7 +1026,7 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.extra_arrivals = g_loop_extra_arrivals;
     p.window = c.mode == WIND_MODE_WINDOW && !logits_out;
     p.nbkeys = c.keys() + 2 * (size_t)c.lay.rows_pad; p.jpart = c.jpart(); p.jblank = c.jblank(); p.parts = 4 * pl.vt_count;
-    p.flags = c.flags(); p.pred_pub = c.pred_pub();
+    p.flags = c.flags(); p.pred_pub = c.pred_pub(); p.kslot = c.kslot();
     const bool full = p.forced || p.window || p.trace;
     if (pl.resident) return loop_res_launch(t_loop_maps, p, pl.grid, pl.smem_bytes, full, c.stream);
     void* args[2] = {(void*)&t_loop_maps, (void*)&p};

@@ -102,7 +102,8 @@ struct LoopParams {
     // resident-weights mode: arrival counters between CTA groups (keys of a row group complete, state of an utterance
     // group written, ...) and the stamped pred_proj values
     uint32_t* flags;
-    unsigned long long* pred_pub;  // [B][H] (fp32 value, stamp)
+    unsigned long long* pred_pub;  // [B][H / 2] (two bf16 values, stamp)
+    unsigned long long* kslot;     // [window rows][vocabulary tiles, padded to even] the tiles' stamped (logit, label) keys
 };
 
 // Options of the tile planner (process-wide; wind_set_loop_options): whether the resident-weights mode may be chosen,

@@ -29,6 +29,9 @@ __device__ __forceinline__ int ld_volatile_i32(const int* p) {
     return v;
 }
 // release: every write this thread has made or observed is visible device-wide before the counter moves
+__device__ __forceinline__ void red_relaxed_add(uint32_t* p, uint32_t v) {
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 __device__ __forceinline__ void red_release_add(uint32_t* p, uint32_t v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -115,15 +118,26 @@ __device__ __forceinline__ void trace_event(const LoopParams& p, int role, int& 
         ++n;
     }
 }
-// When this CTA finished its part of a phase in the first traced step, on the global timer (comparable across SMs).
-__device__ __forceinline__ void trace_phase_done(const LoopParams& p, int step, int phase_kind) {
+// Marks of every CTA in the first traced step, on the global timer (comparable across SMs): role 8 + mark, one
+// record per CTA (`step` holds the CTA index).  Joint: 0 slot entered, 1 copies of the window's enc_proj rows issued,
+// 2 pred_proj has arrived, 3 operand handed to the issuing threads, 4 accumulator ready, 5 keys out (slot done).
+// Decoder update: 6 keys of the CTA's utterances complete, 7 tokens known, 8 accumulator ready, 9 state written (slot
+// done).  Projection: 10 state counters seen by the TMA thread, 11 accumulator ready, 12 pred_proj published, 13
+// state counters seen for the GEMM issued a slot ahead, 14 that GEMM issued, 15 slot done.
+enum { MK_J_ENTER = 0, MK_J_COPIES = 1, MK_J_PRED = 2, MK_J_HANDOVER = 3, MK_J_ACC = 4, MK_J_DONE = 5, MK_L_KEYS = 6, MK_L_TOK = 7,
+       MK_L_ACC = 8, MK_L_DONE = 9, MK_P_FLAG = 10, MK_P_ACC = 11, MK_P_PUB = 12, MK_E_FLAG = 13, MK_E_ISSUED = 14, MK_P_DONE = 15 };
+__device__ __forceinline__ void trace_mark(const LoopParams& p, int step, int phase_kind, int mark) {
     if (p.trace && step == p.trace_step && (int)blockIdx.x < kTraceEvents) {
         TraceEvent t;
         t.tag = (uint32_t)(phase_kind * 16 + 8);
         t.step = (int)blockIdx.x;
         t.clock = (long long)globaltimer_ns();
-        p.trace[(8 + phase_kind) * kTraceEvents + blockIdx.x] = t;
+        p.trace[(8 + mark) * kTraceEvents + blockIdx.x] = t;
     }
+}
+// when this CTA finished its part of a phase
+__device__ __forceinline__ void trace_phase_done(const LoopParams& p, int step, int phase_kind) {
+    trace_mark(p, step, phase_kind, phase_kind == 0 ? MK_J_DONE : (phase_kind == 1 ? MK_L_DONE : MK_P_DONE));
 }
 enum { TR_J = 0, TR_L = 1, TR_P = 2 };
 enum { EV_START = 0, EV_FIRST_ISSUE = 1, EV_LAST_ISSUE = 2, EV_FIRST_DATA = 3, EV_COMMIT = 4, EV_TOK = 5, EV_ACC = 6, EV_EPI_DONE = 7,
@@ -138,7 +152,7 @@ enum { EV_START = 0, EV_FIRST_ISSUE = 1, EV_LAST_ISSUE = 2, EV_FIRST_DATA = 3, E
 template <bool RES, bool FULL>
 __device__ __forceinline__ void joint_epilogue_item(const LoopParams& p, uint32_t tm_j, uint32_t lane_off, int lane, int q, int sub,
                                                     int row_in_tile, int rg, int vt, int n_tile, const int32_t* t_cur,
-                                                    unsigned long long* keys_cur) {
+                                                    unsigned long long* keys_cur, unsigned long long* part = nullptr) {
     const int v = vt * 128 + row_in_tile;            // this thread's vocabulary entry
     const bool v_ok = v < p.NV;
     const float bias = v_ok ? p.b_out[v] : 0.f;
@@ -225,7 +239,13 @@ __device__ __forceinline__ void joint_epilogue_item(const LoopParams& p, uint32_
             argmax_exchange<4>(val, id, lane);
             argmax_exchange<2>(val, id, lane);
             argmax_exchange<1>(val, id, lane);
-            if (row < p.rows && c0 + lane < n_tile && val[0] > -INFINITY) atomicMax(&key_dst[row], pack_key(val[0], (uint32_t)id[0]));
+            if (part && !(FULL && p.window)) {
+                // this warp's winner of row c0 + lane (over its 32 vocabulary entries) goes to shared memory; the caller
+                // combines the four lane quadrants and puts the tile's key out
+                if (c0 + lane < n_tile) part[q * n_tile + c0 + lane] = (row < p.rows && val[0] > -INFINITY) ? pack_key(val[0], (uint32_t)id[0]) : 0ull;
+            } else if (row < p.rows && c0 + lane < n_tile && val[0] > -INFINITY) {
+                atomicMax(&key_dst[row], pack_key(val[0], (uint32_t)id[0]));
+            }
         }
     }
 }

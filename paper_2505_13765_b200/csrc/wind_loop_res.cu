@@ -45,14 +45,34 @@ namespace wind {
 constexpr int kGroupUtts = 96;   // utterances one joint row group can touch (at most 96 rows, window >= 1)
 constexpr int kPrepItems = 3;    // (utterance, 16-byte chunk) items a thread finishes per round of the operand build
 
-__device__ __forceinline__ void ld_acquire_v2_u64(const unsigned long long* p, unsigned long long& a, unsigned long long& b) {
-    asm volatile("ld.acquire.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+// relaxed (L2-coherent) loads: many may be in flight at once, which an acquire load does not allow
+__device__ __forceinline__ void ld_relaxed_v2_u64(const unsigned long long* p, unsigned long long& a, unsigned long long& b) {
+    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
 }
 __device__ __forceinline__ void st_relaxed_v2_u64(unsigned long long* p, unsigned long long a, unsigned long long b) {
     asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(a), "l"(b) : "memory");
 }
-__device__ __forceinline__ unsigned long long stamped(float v, uint32_t stamp) {
-    return ((unsigned long long)stamp << 32) | (unsigned long long)__float_as_uint(v);
+// two neighbouring pred_proj values as bf16, with the stamp of the slot that wrote them
+__device__ __forceinline__ unsigned long long stamped(float lo, float hi, uint32_t stamp) {
+    return ((unsigned long long)stamp << 32) | (unsigned long long)pack_bf16x2(lo, hi);
+}
+// z = act(e + g) on two bf16 pairs at once: one rounding for the sum (fused multiply-add with 1), then ReLU or tanh
+__device__ __forceinline__ uint32_t act_add_bf16x2(uint32_t e, uint32_t g, int act) {
+    const __nv_bfloat162 one = __floats2bfloat162_rn(1.f, 1.f);
+    __nv_bfloat162 s = __hfma2(*reinterpret_cast<const __nv_bfloat162*>(&e), one, *reinterpret_cast<const __nv_bfloat162*>(&g));
+    uint32_t r;
+    if (act == WIND_ACT_RELU) {
+        s = __hmax2(s, __floats2bfloat162_rn(0.f, 0.f));
+        r = *reinterpret_cast<uint32_t*>(&s);
+    } else {
+        asm("tanh.approx.bf16x2 %0, %1;" : "=r"(r) : "r"(*reinterpret_cast<uint32_t*>(&s)));
+    }
+    return r;
 }
 
 template <bool FULL>
@@ -164,13 +184,13 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
     uint32_t* f_h1 = f_h0 + p.ql_count;          // [ql_count]  layer-1 state written (two layers)
     uint32_t* f_dh = f_h1 + p.ql_count;          // [ql_count]  layer 1's recurrent term written (two layers)
     // arrivals per decoder-update slot on group ql's layer-0 counter: its unit tiles, plus (when separate CTAs record
-    // the steps) one per block of 32 utterances that overlaps the group.  Under teacher forcing nothing is recorded
+    // the steps) one per recording CTA (64 utterances) that overlaps the group.  Under teacher forcing nothing is recorded
     // and the recording CTAs stay out: a counter that sums arrivals over slots is only sound while no participant
     // can run ahead of the others, and a CTA with nothing to wait for could.
     auto arr_h0 = [&](int ql) -> uint32_t {
         uint32_t a = (uint32_t)p.ut_count;
         const int lo = ql * p.nl, hi = min(lo + p.nl, p.B);
-        if (p.w_count > 0 && !forced && hi > lo) a += (uint32_t)((hi - 1) / 32 - lo / 32 + 1);
+        if (p.w_count > 0 && !forced && hi > lo) a += (uint32_t)((hi - 1) / 64 - lo / 64 + 1);
         return a;
     };
     // a wait of this CTA ran out: note which one (the first in the grid stays), flag the CTA and everybody else
@@ -238,6 +258,9 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
     int tr_n = 0;                     // trace events written by this thread
     uint32_t epoch = 0;               // grid barrier target (window-based decoding only)
 
+    auto mark = [&](int kind, int id) {
+        if constexpr (FULL) trace_mark(p, step, kind, id);
+    };
     // this thread has finished its CTA's part of a slot: CTA 0 attributes the time, the timeline notes every CTA
     auto slot_done = [&](int kind) {
         if (cta == 0) {
@@ -317,36 +340,86 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
     // ctl_only: the CTA is one of the step-recording CTAs: it takes the control step of 64 utterances, records it
     // (outputs, counters, next frame) and has no cell update; the L CTAs then record nothing.
     // =========================================================================================
-    struct ScanIn { int t, len, cnt, pos; unsigned long long kk[8]; };
+    constexpr unsigned long long kStampMask = 0xFFFull << 20;   // bits of a key slot that hold the joint slot's stamp
+    const int vt_pad = (p.vt_count + 1) & ~1;   // key slots of a window row: one per vocabulary tile, padded to 16 bytes
+    // The (logit, label) keys of window rows wr and wr + 1 of utterance b (rows < n only): per row the maximum over the
+    // vocabulary tiles' slots, each of which must carry this step's stamp (the whole warp polls until all do).  Result
+    // per row: high word = orderable logit (0: nothing there), low 20 bits = 0xFFFFF - label.
+    auto fetch_keys2 = [&](int b, int wr, int n, bool live, unsigned long long& k0, unsigned long long& k1) -> bool {
+        const uint32_t want = n_j & 0xFFFu;
+        const bool in0 = live && wr < n, in1 = live && wr + 1 < n;
+        const int r0 = b * p.W + wr, r1 = r0 + 1;
+        const unsigned long long* s0 = p.kslot + (size_t)(in0 ? r0 : 0) * vt_pad;   // rows lie one after the other: (row group, row in it)
+        const unsigned long long* s1 = p.kslot + (size_t)(in1 ? r1 : 0) * vt_pad;
+        unsigned long long t0 = 0;
+        for (uint32_t it = 1;; ++it) {
+            bool ok = true;
+            k0 = 0ull; k1 = 0ull;
+            for (int v0 = 0; v0 < vt_pad; v0 += 10) {
+                unsigned long long x[10], y[10];
+#pragma unroll
+                for (int j = 0; j < 5; ++j) {
+                    x[2 * j] = x[2 * j + 1] = y[2 * j] = y[2 * j + 1] = 0ull;
+                    if (in0 && v0 + 2 * j < vt_pad) ld_relaxed_v2_u64(s0 + v0 + 2 * j, x[2 * j], x[2 * j + 1]);
+                    if (in1 && v0 + 2 * j < vt_pad) ld_relaxed_v2_u64(s1 + v0 + 2 * j, y[2 * j], y[2 * j + 1]);
+                }
+#pragma unroll
+                for (int j = 0; j < 10; ++j) {
+                    if (v0 + j < p.vt_count) {
+                        if (in0) {
+                            ok = ok && (uint32_t)((x[j] & kStampMask) >> 20) == want;
+                            const unsigned long long key = x[j] & ~kStampMask;
+                            k0 = key > k0 ? key : k0;
+                        }
+                        if (in1) {
+                            ok = ok && (uint32_t)((y[j] & kStampMask) >> 20) == want;
+                            const unsigned long long key = y[j] & ~kStampMask;
+                            k1 = key > k1 ? key : k1;
+                        }
+                    }
+                }
+            }
+            if (__all_sync(0xffffffffu, ok)) return true;
+            if ((it & 15u) == 0u) {
+                bool quit = *vabort != 0;
+                if (!quit && ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; quit = true; }
+                const unsigned long long now = globaltimer_ns();
+                if (t0 == 0) t0 = now;
+                else if (!quit && now - t0 > kWaitLimitNs) { give_up(43); quit = true; }
+                if (__any_sync(0xffffffffu, quit)) return false;
+            }
+        }
+    };
     auto epilogue_res_L = [&](const int layer, const bool ctl_only) -> bool {
-        if (ctl_only && q != 0) return true;
         const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
         int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
         const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
         unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
         const int u16 = lane & 15, half = lane >> 4;
         const int unit = r_ut * 16 + u16;        // this thread's hidden unit; its gate is q
-        // without recording CTAs, the two gate-0 warps of one CTA per utterance group record the step
-        const bool writer = ctl_only ? true : (p.w_count == 0 && layer == 0 && r_ut == 0 && q == 0);
+        // Control step: four neighbouring lanes per utterance (eight utterances per warp, 64 per pass over the eight
+        // epilogue warps); lane kq of a group looks at window rows 2 kq and 2 kq + 1 (+ 8 per round), the group's first
+        // lane decides and, where this CTA records the steps, records.  Without recording CTAs, one CTA per utterance
+        // group (unit tile 0) records.
+        const int kq = lane & 3;
+        const int ju = 8 * (warp - 2) + (lane >> 2);     // the group's utterance of the pass
+        const bool head = kq == 0;
+        const bool writer = head && (ctl_only ? true : (p.w_count == 0 && layer == 0 && r_ut == 0));
+        const bool mark_here = e == 0;
         const int n_here = ctl_only ? 64 : p.nl;
         const int base = ctl_only ? (cta - p.w_first) * 64 : r_ql * p.nl;
         const bool decode = step >= 0 && !forced && layer == 0;
+        const bool from_slots = !(FULL && p.window);   // window-based decoding leaves its decision in the key arrays
         float* cst = p.c_state + (size_t)layer * p.B * p.P + unit;
         const __nv_bfloat16* hin = p.hb + ((size_t)(pin * p.L + layer) * p.Bpad) * p.P + unit;
         __nv_bfloat16* hout = p.hb + ((size_t)((pin ^ 1) * p.L + layer) * p.Bpad) * p.P + unit;
         const float bias1 = layer == 0 ? 0.f : p.b_ih[1][q * p.P + unit] + p.b_hh[1][q * p.P + unit];
         const float* g0u = p.g0 + (size_t)q * p.P + unit;
         const uint32_t g0_stride = 4u * (uint32_t)p.P;
+        int* tok_s = reinterpret_cast<int*>(stage_f + 4 * 64 * 16);   // tokens of the pass's 64 utterances
         bool ready = true;
         // ---- what this slot waits for from other CTAs ----
-        if (decode) {
-            // the keys of this CTA's utterances: every vocabulary tile of their row groups has arrived
-            const int b_hi = min(base + n_here, p.B);
-            if (b_hi > base) {
-                const int rg_lo = base * p.W / p.nj, rg_hi = (b_hi * p.W - 1) / p.nj;
-                ready = warp_flag_wait(f_keys, rg_lo, rg_hi - rg_lo + 1, n_j * (uint32_t)p.vt_count + (uint32_t)p.extra_arrivals, 20);
-            }
-        } else if (forced && p.L == 2 && layer == 0 && n_l >= 2u) {
+        if (forced && p.L == 2 && layer == 0 && n_l >= 2u) {
             // Teacher forcing feeds tokens without waiting for keys, so nothing else holds layer 0 back: before this
             // slot overwrites the state buffer it wrote two slots ago, layer 1's CTAs must have read it (their arrivals
             // of the slot before last).  While decoding, the wait for the keys implies this.
@@ -361,22 +434,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
         }
         for (int c0 = 0; c0 < n_here; c0 += 64) {
             const int b0 = base + c0;
-            // ---- lane j decides for utterance b0 + 32 sub + j ----
-            const int jl = 32 * sub + lane;
-            const int b = b0 + jl;
-            const bool in = c0 + jl < n_here && b < p.B;
-            ScanIn si;
-            si.t = 0; si.len = 0; si.cnt = 0; si.pos = 0;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) si.kk[j] = 0ull;
-            if (in && decode) {
-                si.t = __ldcg(t_cur + b);
-                si.len = p.enc_len[b];
-                if (writer) { si.cnt = __ldcg(p.count + b); si.pos = __ldcg(p.out_len + b); }
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (j < p.W) si.kk[j] = __ldcg(keys_cur + (size_t)b * p.W + j);
-            }
+            const int jl = 32 * sub + lane;      // the utterance of the pass whose token this lane hands to the gate-table reads
             // old cell state of the four (utterance, unit) pairs this thread finishes
             float cold[4];
 #pragma unroll
@@ -384,54 +442,84 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                 const int j = half + 2 * q + 8 * sub + 16 * jj;     // 0..63 over the CTA's 256 epilogue threads
                 cold[jj] = (!ctl_only && c0 + j < p.nl && b0 + j < p.B) ? cst[(size_t)(b0 + j) * p.P] : 0.f;
             }
-            // the token utterance b feeds to its decoder in this step (-1: none)
-            int tok = -1, t_out = 0;
-            if (in) {
+            {
+                // ---- the token utterance b feeds to its decoder in this step (-1: none) ----
+                const int b = b0 + ju;
+                const bool in = c0 + ju < n_here && b < p.B;
+                int tok = -1, t_out = 0;
                 if (step < 0) {
-                    tok = p.blank;
+                    tok = in ? p.blank : -1;
                 } else if (forced) {
-                    tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
-                    if (tok >= p.NV || tok < -1) { tok = p.blank; set_status(p.ctrl, WIND_ERR_INVALID_ARG); }   // caller's mistake
+                    if (in) {
+                        tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
+                        if (tok >= p.NV || tok < -1) { tok = p.blank; set_status(p.ctrl, WIND_ERR_INVALID_ARG); }   // caller's mistake
+                    }
                 } else if (layer > 0) {
-                    tok = __ldcg(p.emit_tok + b);     // decided by layer 0's CTAs one slot earlier
+                    if (in) tok = __ldcg(p.emit_tok + b);     // decided by layer 0's CTAs one slot earlier
                 } else {
-                    int t = si.t;
-                    const int len = si.len;
-                    if (t < len) {
-                        // control step (Algorithm 2's branch): first non-blank row of the window
-                        const int n = min(p.W, len - t);
-                        int first = -1, label = p.blank;
-                        bool bad = false;
-                        for (int w0 = 0; w0 < n && first < 0; w0 += 8) {
-                            if (w0 > 0) {
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) si.kk[j] = (w0 + j < n) ? __ldcg(keys_cur + (size_t)b * p.W + w0 + j) : 0ull;
-                            }
-                            // the eight rows side by side: which are inside the window, broken, non-blank
-                            uint32_t nonblank = 0u, broken = 0u;
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                const uint32_t lab = key_label(si.kk[j]);
-                                const bool inside = w0 + j < n;
-                                const bool brk = si.kk[j] == 0ull || lab >= (uint32_t)p.NV;
-                                broken |= (uint32_t)(inside && brk) << j;
-                                nonblank |= (uint32_t)(inside && !brk && (int)lab != p.blank) << j;
-                            }
-                            if (nonblank) {
-                                const int j = __ffs((int)nonblank) - 1;
-                                first = w0 + j;
-                                uint32_t lab = 0u;
-#pragma unroll
-                                for (int jj = 0; jj < 8; ++jj)
-                                    if (jj == j) lab = key_label(si.kk[jj]);
-                                label = (int)lab;
-                                broken &= (1u << j) - 1u;   // rows after the first non-blank one are not looked at
-                            }
-                            bad = bad || broken != 0u;
+                    int t = 0, len = 0, cnt = 0, pos = 0;
+                    if (in) {
+                        t = __ldcg(t_cur + b);
+                        len = p.enc_len[b];
+                        if (writer) { cnt = __ldcg(p.count + b); pos = __ldcg(p.out_len + b); }
+                    }
+                    if (c0 == 0 && from_slots) {
+                        // A hint only (relaxed counters, no ordering; behind the loads above, so that their latency is
+                        // hidden): every vocabulary tile of the row groups of this CTA's utterances has put out its
+                        // keys.  The keys themselves are checked by their stamps.
+                        const int b_hi = min(base + n_here, p.B);
+                        if (b_hi > base) {
+                            const int rg_lo = base * p.W / p.nj, rg_hi = (b_hi * p.W - 1) / p.nj;
+                            ready = warp_flag_wait(f_keys, rg_lo, rg_hi - rg_lo + 1, n_j * (uint32_t)(p.vt_count * ((p.nj + 31) / 32)) + (uint32_t)p.extra_arrivals, 20);
                         }
+                        if (mark_here) mark(TR_L, MK_L_KEYS);
+                    }
+                    const bool live = in && t < len;
+                    const int n = live ? min(p.W, len - t) : 0;
+                    // control step (Algorithm 2's branch): first non-blank row of the window, eight rows per round
+                    int first = -1, label = p.blank;
+                    bool bad = false;
+                    const int n_max = __reduce_max_sync(0xffffffffu, n);
+                    for (int w0 = 0; w0 < n_max; w0 += 8) {
+                        const bool more = live && w0 < n && first < 0;     // the same in the four lanes of a group
+                        if (!__any_sync(0xffffffffu, more)) break;
+                        const int wr = w0 + 2 * kq;
+                        unsigned long long kk[2] = {0ull, 0ull};
+                        if (from_slots) {
+                            if (!fetch_keys2(in ? b : 0, wr, n, more, kk[0], kk[1])) ready = false;
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 2; ++j) {
+                                if (more && wr + j < n) {
+                                    const unsigned long long k = __ldcg(keys_cur + (size_t)b * p.W + wr + j);
+                                    if (k != 0ull) kk[j] = (k & 0xFFFFFFFF00000000ull) | (unsigned long long)(0xFFFFFu - key_label(k));
+                                }
+                            }
+                        }
+                        // this lane's two rows: the first non-blank one (row and label in one word) and the first broken one
+                        uint32_t fn = 0x7FFFFFFFu, fb = 0x7FFFFFFFu;
+#pragma unroll
+                        for (int j = 1; j >= 0; --j) {
+                            const uint32_t lab = 0xFFFFFu - (uint32_t)(kk[j] & 0xFFFFFull);
+                            const bool inside = more && wr + j < n;
+                            const bool brk = (kk[j] >> 32) == 0ull || lab >= (uint32_t)p.NV;
+                            if (inside && brk) fb = (uint32_t)(wr + j) << 20;
+                            if (inside && !brk && (int)lab != p.blank) fn = ((uint32_t)(wr + j) << 20) | lab;
+                        }
+#pragma unroll
+                        for (int o = 1; o <= 2; o <<= 1) {
+                            fn = min(fn, __shfl_xor_sync(0xffffffffu, fn, o));
+                            fb = min(fb, __shfl_xor_sync(0xffffffffu, fb, o));
+                        }
+                        if (more) {
+                            if (fn != 0x7FFFFFFFu) { first = (int)(fn >> 20); label = (int)(fn & 0xFFFFFu); }
+                            bad = bad || (fb >> 20) < (fn >> 20);     // rows after the first non-blank one are not looked at
+                        }
+                    }
+                    if (live) {
                         if (first >= 0) tok = label;
                         if (writer) {
-                            int cnt = si.cnt, jump, forced_adv = 0, emitted = 0;
+                            int jump, forced_adv = 0, emitted = 0;
                             if (first < 0) {
                                 jump = n;
                                 t += n;
@@ -440,10 +528,10 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                                 jump = first;
                                 if (first > 0) cnt = 0;
                                 t += first;
-                                if (si.pos < p.max_out) {
-                                    p.out_tokens[(size_t)b * p.max_out + si.pos] = label;
-                                    p.out_frames[(size_t)b * p.max_out + si.pos] = t;
-                                    p.out_len[b] = si.pos + 1;
+                                if (pos < p.max_out) {
+                                    p.out_tokens[(size_t)b * p.max_out + pos] = label;
+                                    p.out_frames[(size_t)b * p.max_out + pos] = t;
+                                    p.out_len[b] = pos + 1;
                                     emitted = 1;
                                     cnt += 1;
                                     if (cnt == p.S) { t += 1; cnt = 0; forced_adv = 1; }
@@ -457,28 +545,32 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                             t_nxt[b] = t;
                             t_out = t;
                             p.count[b] = cnt;
-                            for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
+                            if (!from_slots)
+                                for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
                             atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
                             atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->joint_rows), (unsigned long long)n);
                             if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
                             if (forced_adv) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
                         }
-                    } else if (writer) {
+                    } else if (in && writer) {
                         t_nxt[b] = t;
                         t_out = t;
                     }
                 }
-                if (writer && p.L > 1 && decode) p.emit_tok[b] = tok;   // the upper layer's CTAs read it in their slot
-                // the next frame goes out at once, stamped with the slot, for the CTAs that build the next window's
-                // operand and for everybody's count of the utterances still decoding.  Released: what this thread has
-                // written for the step (frame, counters, the cleared keys of the next step) is visible before it.
-                if (writer && !forced) {
-                    __threadfence();
-                    p.t_pub[b] = ((unsigned long long)(n_l + 1u) << 32) | (uint32_t)t_out;
+                if (in && writer) {
+                    if (p.L > 1 && decode) p.emit_tok[b] = tok;   // the upper layer's CTAs read it in their slot
+                    // the next frame goes out at once, stamped with the slot, for the CTAs that build the next window's
+                    // operand and for everybody's count of the utterances still decoding (readers need nothing but this
+                    // word; the frame and counter arrays are only read a whole step later)
+                    if (!forced) asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p.t_pub + b), "l"(((unsigned long long)(n_l + 1u) << 32) | (uint32_t)t_out) : "memory");
                 }
+                if (!ctl_only && head) tok_s[ju] = tok;
+                if (mark_here) mark(TR_L, MK_L_TOK);
             }
             if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
             if (ctl_only) continue;
+            asm volatile("bar.sync 1, 256;" ::: "memory");     // the tokens of the pass
+            const int tok = tok_s[jl];
             // ---- gate-table entries (this thread's gate and unit) of the tokens of this lane half's 16 utterances ----
             float add[16];
 #pragma unroll
@@ -493,14 +585,12 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                     add[j] = (tj >= 0 && bj2 < p.B) ? __ldcg(p.dh + (size_t)bj2 * g0_stride + (size_t)q * p.P + unit) + bias1 : 0.f;
                 }
             }
-            // the other warps need the tokens for the cell update below: through shared memory
-            int* tok_s = reinterpret_cast<int*>(stage_f + 4 * 64 * 16);
-            if (q == 0) tok_s[jl] = tok;
             if (c0 == 0) {
                 const bool acc_ok = __all_sync(0xffffffffu, mwait(&acc_full[1], acc_n[1] & 1u, 30));
                 ready = ready && acc_ok;
                 tc_fence_after();
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
+                if (e == 0) mark(TR_L, MK_L_ACC);
             }
             if (ready) {
                 // lanes 0..15 read their row's 32 columns; columns 16..31 then move to lanes 16..31
@@ -544,10 +634,10 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
             asm volatile("bar.sync 1, 256;" ::: "memory");
         }
         if (ctl_only) {
-            // this warp's 32 utterances are recorded: one arrival on every utterance group they belong to
-            __syncwarp();
-            const int lo = base + 32 * sub, hi = min(lo + 32, p.B);
-            if (lane == 0 && hi > lo)
+            // this CTA's 64 utterances are recorded: one arrival on every utterance group they belong to
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            const int lo = base, hi = min(lo + 64, p.B);
+            if (e == 0 && hi > lo)
                 for (int g = lo / p.nl; g <= (hi - 1) / p.nl; ++g) red_release_add(f_h0 + g, 1u);
             return true;
         }
@@ -573,6 +663,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
         const bool ready = __all_sync(0xffffffffu, mwait(&acc_full[2], acc_n[2] & 1u, 31));
         tc_fence_after();
         if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
+        if (e == 0) mark(TR_P, MK_P_ACC);
         if (ready) {
             const int hl = 16 * q + (lane & 15);
             for (int c0 = 16 * sub; c0 < p.np; c0 += 32) {
@@ -596,20 +687,21 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (ready) {
             // thread e: four consecutive H rows of utterances (e >> 4), (e >> 4) + 16, ...: 512 contiguous bytes per
-            // utterance and 16 threads.  One release fence, then the stamped pairs.
-            __threadfence();
+            // utterance and 16 threads.  No fence before the stamped pairs: a reader needs nothing but the pair itself,
+            // and what this CTA read of other CTAs' writes for this slot (the state box) had arrived in shared memory
+            // before the accumulator could be read, so a later overwrite of the state cannot reach it.
             const int hq = (e & 15) * 4;
             for (int bl = e >> 4; bl < p.np; bl += 16) {
                 const int b = r_qp * p.np + bl;
                 if (b < p.B) {
                     const float4 v = *reinterpret_cast<const float4*>(stage_f + bl * 68 + hq);
-                    unsigned long long* dst = p.pred_pub + (size_t)b * p.H + h0 + hq;
-                    st_relaxed_v2_u64(dst, stamped(v.x, stamp), stamped(v.y, stamp));
-                    st_relaxed_v2_u64(dst + 2, stamped(v.z, stamp), stamped(v.w, stamp));
+                    unsigned long long* dst = p.pred_pub + ((size_t)b * p.H + h0 + hq) / 2;
+                    st_relaxed_v2_u64(dst, stamped(v.x, v.y, stamp), stamped(v.z, v.w, stamp));
                 }
             }
         }
         if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
+        if (e == 0) mark(TR_P, MK_P_PUB);
         return ready;
     };
     // h1 CTAs: the finished recurrent term of layer 1 goes to global memory (fp32 [B][4P], gate-major like the gate
@@ -644,19 +736,24 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (e == 0) red_release_add(f_dh + r_ql, 1u);
     };
-    // GEMMs that need only the state, issued a slot ahead: layer 0's (its result waits in tensor memory for the
-    // next control step) and, with two layers, layer 1's recurrent term (stored by store_res_h1)
+    // GEMMs that need only the state, issued ahead of the decoder-update slot that uses them: layer 0's (its result
+    // waits in tensor memory for the next control step) and, with two layers, layer 1's recurrent term (stored by
+    // store_res_h1).  While decoding they are issued right behind the joint's MMAs: the state box then takes over the
+    // operand buffer the joint has just read, and the buffer is free for the next window's rows as soon as the
+    // decoder-update slot is over (the box and the joint's operand share memory in these CTAs).
     auto early_res = [&]() {
         const bool mine = res_l || res_h1;
         if (warp == 0) {
             if (lane == 0 && mine) {
                 // the state of this CTA's utterance group as the last decoder-update slot left it
                 const bool ok = res_l ? flag_wait(f_h0 + r_ql, n_l * arr_h0(r_ql), 24) : flag_wait(f_h1 + r_ql, n_l * (uint32_t)p.ut_count, 25);
+                mark(TR_P, MK_E_FLAG);
                 if (ok) {
                     fence_proxy_async_all();
                     if (produce_box(res_l ? &M.hb_l3[pin] : &M.hb_l3_1[pin], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u))
                         mma_part(1, tm_l, p.nl, p.kb_p, p.kb_p, false, 0, use0, buf0);   // one accumulator: warp 1 issues all of it
                 }
+                mark(TR_P, MK_E_ISSUED);
             }
         } else if (warp == 1) {
             if (lane == 0 && mine) mma_part(1, tm_l, p.nl, 0, p.kb_p, false, 0, use0, buf0);
@@ -680,10 +777,49 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
         u_lo = r_lo / p.W;
         n_utt = r_hi > r_lo ? (r_hi - 1) / p.W - u_lo + 1 : 0;
     };
-    auto prep_A = [&](int rg, uint32_t want) {
+    // Warp 2, once its CTA's decoder-slot work is over: the frames the recording threads have published for this step,
+    // all requested together (relaxed loads).  Gives the count of utterances still decoding (every CTA reads the same
+    // words, so all take the same exit) and the frames of the CTA's first row group for the operand copies.
+    // A CTA that lags may find a later stamp: the recording threads only go on while utterances are left, so a later
+    // stamp means "not finished" (the count itself is then of no interest).
+    auto poll_frames = [&](uint32_t want) {
+        int u_lo = 0, n_utt = 0;
+        if (has_j) group_span(j_first, u_lo, n_utt);
+        int alive = 0;
+        unsigned long long t0 = 0;
+        for (uint32_t it = 1;; ++it) {
+            bool all = true;
+            alive = 0;
+            for (int b = lane; b < p.B; b += 32) {
+                const unsigned long long v = ld_relaxed_u64(p.t_pub + b);
+                const int32_t ahead = (int32_t)((uint32_t)(v >> 32) - want);
+                const int t = (int)(uint32_t)v, len = p.enc_len[b];
+                all = all && ahead >= 0;
+                alive += (ahead > 0 || t < len) ? 1 : 0;
+                if (ahead == 0 && b >= u_lo && b < u_lo + n_utt) {
+                    s_jt[b - u_lo] = t < len ? t : 0;
+                    s_jrem[b - u_lo] = t < len ? len - t : 0;
+                }
+            }
+            if (__all_sync(0xffffffffu, all)) break;
+            if ((it & 15u) == 0u) {
+                bool quit = *vabort != 0;
+                if (!quit && ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; quit = true; }
+                const unsigned long long now = globaltimer_ns();
+                if (t0 == 0) t0 = now;
+                else if (!quit && now - t0 > kWaitLimitNs) { give_up(42); quit = true; }
+                if (__any_sync(0xffffffffu, quit)) break;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) alive += __shfl_xor_sync(0xffffffffu, alive, o);
+        if (lane == 0) s_active = alive;
+    };
+    // frames_known: s_jt / s_jrem of this row group were filled by poll_frames
+    auto prep_A = [&](int rg, uint32_t want, bool frames_known) {
         int u_lo, n_utt;
         group_span(rg, u_lo, n_utt);
-        if (e < n_utt) {
+        if (!frames_known && e < n_utt) {
             const int b = u_lo + e;
             int t = 0;
             if (forced) {
@@ -732,6 +868,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
             }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
+        if (e == 0) mark(TR_J, MK_J_COPIES);
     };
     auto prep_B = [&](int rg, uint32_t want) {
         int u_lo, n_utt;
@@ -739,7 +876,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
         const int n_items = n_utt * n_chunks;
         bool waited = false;
         for (int base = e; base < n_items; base += 256 * kPrepItems) {
-            float pv[kPrepItems][8];
+            uint32_t pv[kPrepItems][4];      // pred_proj of the item's eight columns, as four bf16 pairs
             int it_ul[kPrepItems], it_c[kPrepItems];
 #pragma unroll
             for (int k = 0; k < kPrepItems; ++k) {
@@ -750,32 +887,44 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                     if (s_jrem[ul] > 0) { it_ul[k] = ul; it_c[k] = idx - ul * n_chunks; }   // a finished utterance needs nothing
                 }
             }
-            // pred_proj of this round's items, all requested together, until every stamp is this slot's
+            // pred_proj of this round's items, all requested together, until every stamp is this slot's; between two
+            // such requests one word is polled until it carries the stamp (little traffic while the projection CTAs are
+            // still at work).  Relaxed loads: the values travel in the same 8-byte words as the stamps, and nothing else
+            // that another CTA writes is read behind them.
             unsigned long long t0 = 0;
             for (uint32_t it = 1;; ++it) {
                 bool all = true;
+                const unsigned long long* miss = nullptr;
 #pragma unroll
                 for (int k = 0; k < kPrepItems; ++k) {
                     if (it_ul[k] < 0) continue;
-                    const unsigned long long* src = p.pred_pub + (size_t)(u_lo + it_ul[k]) * p.H + it_c[k] * 8;
-                    unsigned long long x[8];
+                    const unsigned long long* src = p.pred_pub + ((size_t)(u_lo + it_ul[k]) * p.H + it_c[k] * 8) / 2;
+                    unsigned long long x[4];
+                    ld_relaxed_v2_u64(src, x[0], x[1]);
+                    ld_relaxed_v2_u64(src + 2, x[2], x[3]);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) ld_acquire_v2_u64(src + 2 * j, x[2 * j], x[2 * j + 1]);
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        all = all && (uint32_t)(x[j] >> 32) == want;
-                        pv[k][j] = __uint_as_float((uint32_t)x[j]);
+                    for (int j = 0; j < 4; ++j) {
+                        if ((uint32_t)(x[j] >> 32) != want) { all = false; miss = src + j; }
+                        pv[k][j] = (uint32_t)x[j];
                     }
                 }
                 if (all) break;
-                if ((it & 15u) == 0u) {
-                    if (*vabort) break;
-                    if (ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; break; }
-                    const unsigned long long now = globaltimer_ns();
-                    if (t0 == 0) t0 = now;
-                    else if (now - t0 > kWaitLimitNs) { give_up(41); break; }
+                bool quit = false;
+                for (uint32_t spin = 1; !quit; ++spin) {
+                    if ((uint32_t)(ld_relaxed_u64(miss) >> 32) == want) break;
+                    if ((spin & 15u) == 0u) {
+                        if (*vabort) quit = true;
+                        else if (ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; quit = true; }
+                        else {
+                            const unsigned long long now = globaltimer_ns();
+                            if (t0 == 0) t0 = now;
+                            else if (now - t0 > kWaitLimitNs) { give_up(41); quit = true; }
+                        }
+                    }
                 }
+                if (quit) break;
             }
+            if (e == 0 && !waited) mark(TR_J, MK_J_PRED);
             if (!waited) { asm volatile("cp.async.wait_all;" ::: "memory"); waited = true; }
 #pragma unroll
             for (int k = 0; k < kPrepItems; ++k) {
@@ -787,17 +936,8 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                     const int i = b * p.W + w - rg * p.nj;
                     uint4* dst = reinterpret_cast<uint4*>(dst_kb + i * 128 + (((c & 7) ^ (i & 7)) << 4));
                     const uint4 ev = *dst;
-                    const __nv_bfloat162* eb = reinterpret_cast<const __nv_bfloat162*>(&ev);
-                    uint32_t wds[4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float2 e2 = __bfloat1622float2(eb[j]);
-                        float z0 = e2.x + pv[k][2 * j], z1 = e2.y + pv[k][2 * j + 1];
-                        z0 = p.act == WIND_ACT_RELU ? fmaxf(z0, 0.f) : tanh_fast(z0);
-                        z1 = p.act == WIND_ACT_RELU ? fmaxf(z1, 0.f) : tanh_fast(z1);
-                        wds[j] = pack_bf16x2(z0, z1);
-                    }
-                    *dst = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+                    *dst = make_uint4(act_add_bf16x2(ev.x, pv[k][0], p.act), act_add_bf16x2(ev.y, pv[k][1], p.act),
+                                      act_add_bf16x2(ev.z, pv[k][2], p.act), act_add_bf16x2(ev.w, pv[k][3], p.act));
                 }
             }
         }
@@ -805,6 +945,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
         fence_proxy_async();      // this thread's shared-memory writes, for the MMAs (async proxy)
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (e == 0) mbar_arrive(&full_bar[1]);
+        if (e == 0) mark(TR_J, MK_J_HANDOVER);
     };
 
     // ----- before the loop: layer 0's GEMM on the initial (zero) state -----
@@ -819,8 +960,6 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
             if (res_l) epilogue_res_L(0, false);
             else if (res_w && !forced) epilogue_res_L(0, true);
             if (cta == 0 && e == 0 && step >= 0 && !forced) p.ctrl->step = step + 1;
-            // CTAs whose joint operand has a buffer of its own start on the next window now
-            if (has_j && !z_sh && !forced) { prep_A(j_first, n_l + 1u); prepped = true; }
             if (e == 0 && p.L != 2) slot_done(TR_L);
         }
         ++n_l;
@@ -842,6 +981,10 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
             }
             if (res_x1) ++use0;
         }
+        // The next window's enc_proj rows can be copied in from here on: the frames are published and this CTA's
+        // GEMMs on the state box are over.  (A CTA whose projection box shares the buffer does it behind that GEMM.)
+        if (warp == 2 && !forced) poll_frames(n_l);
+        if (warp >= 2 && has_j && !forced && !(res_p && z_sh)) { prep_A(j_first, n_l, true); prepped = true; }
         pin ^= 1;
         if (forced && step + 1 < p.U) {
             // teacher forcing: more prefix tokens to feed before the window is evaluated
@@ -862,6 +1005,7 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                 if (b_hi > b_lo)
                     for (int g = b_lo / p.nl; ok && g <= (b_hi - 1) / p.nl; ++g)
                         ok = flag_wait(f + g, n_l * (p.L == 2 ? (uint32_t)p.ut_count : arr_h0(g)), 27);
+                mark(TR_P, MK_P_FLAG);
                 if (ok) {
                     fence_proxy_async_all();
                     if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_P, EV_FIRST_ISSUE);
@@ -873,42 +1017,10 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
             if (lane == 0 && res_p) mma_part(2, tm_p, p.np, 0, p.kb_p / 2, false, 0, use0, buf0);
         } else {
             if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_START);
-            if (warp == 2 && !forced) {
-                // utterances still decoding, from the frames the recording threads have published for this step
-                // (every CTA reads the same words, so all take the same exit)
-                // A CTA that lags may find a later stamp: the recording threads only go on when utterances are left,
-                // so a later stamp means "not finished" (the count itself is then of no interest).
-                int alive = 0;
-                unsigned long long t0 = 0;
-                for (uint32_t it = 1;; ++it) {
-                    bool all = true;
-                    alive = 0;
-                    for (int b = lane; b < p.B; b += 32) {
-                        unsigned long long v;
-                        asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(v) : "l"(p.t_pub + b) : "memory");
-                        const int32_t ahead = (int32_t)((uint32_t)(v >> 32) - n_l);
-                        all = all && ahead >= 0;
-                        alive += (ahead > 0 || (int)(uint32_t)v < p.enc_len[b]) ? 1 : 0;
-                    }
-                    if (__all_sync(0xffffffffu, all)) break;
-                    if ((it & 15u) == 0u) {
-                        bool quit = *vabort != 0;
-                        if (!quit && ld_volatile_i32(&p.ctrl->abort)) { *vabort = 2; quit = true; }
-                        const unsigned long long now = globaltimer_ns();
-                        if (t0 == 0) t0 = now;
-                        else if (!quit && now - t0 > kWaitLimitNs) { give_up(42); quit = true; }
-                        if (__any_sync(0xffffffffu, quit)) break;
-                    }
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) alive += __shfl_xor_sync(0xffffffffu, alive, o);
-                if (lane == 0) s_active = alive;
-            }
             if (res_p) epilogue_res_P(n_p + 1u);
         }
         if (res_p) ++use0;
         ++n_p;
-        early_res();
         if (warp >= 2 && e == 0) slot_done(TR_P);
         // the one CTA-wide meeting point of a step: everybody learns whether the kernel is being abandoned and how
         // many utterances are still decoding
@@ -937,25 +1049,50 @@ __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __g
                     }
                 } else {
                     if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_START);
-                    if (!prepped) prep_A(rg, n_l);
+                    if (e == 0) mark(TR_J, MK_J_ENTER);
+                    if (!prepped) prep_A(rg, n_l, false);
                     prepped = false;
                     prep_B(rg, n_p);
                     if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_TOK);
                     const bool ready = __all_sync(0xffffffffu, mwait(&acc_full[0], acc_n[0] & 1u, 33));
                     tc_fence_after();
                     if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_ACC);
-                    if (ready) joint_epilogue_item<true, FULL>(p, tm_j, lane_off, lane, q, sub, row_in_tile, rg, my_vt, n_tile, t_cur, keys_cur);
+                    if (e == 0) mark(TR_J, MK_J_ACC);
+                    unsigned long long* part = reinterpret_cast<unsigned long long*>(stage_f);   // [4 lane quadrants][n_tile]
+                    if (ready) joint_epilogue_item<true, FULL>(p, tm_j, lane_off, lane, q, sub, row_in_tile, rg, my_vt, n_tile, t_cur, keys_cur, part);
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&acc_empty[0]);
                     ++acc_n[0];
-                    // this vocabulary tile's keys of the row group are out: one arrival
                     asm volatile("bar.sync 1, 256;" ::: "memory");
-                    if (e == 0) red_release_add(f_keys + rg, 1u);
+                    if (!forced && !(FULL && p.window)) {
+                        // This vocabulary tile's key of every row of the group goes out as ONE stamped word per row (no
+                        // atomics, no fence): high word the orderable logit (0: no entry), then the joint slot's stamp,
+                        // then 0xFFFFF - label.  Readers take the maximum over the tiles once every stamp is this step's.
+                        if (e < n_tile) {
+                            unsigned long long m = 0ull;
+                            if (ready) {
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    const unsigned long long x = part[k * n_tile + e];
+                                    m = x > m ? x : m;
+                                }
+                            }
+                            const unsigned long long stamp_bits = (unsigned long long)((n_j + 1u) & 0xFFFu) << 20;
+                            const unsigned long long word =
+                                m != 0ull ? ((m & 0xFFFFFFFF00000000ull) | stamp_bits | (unsigned long long)(0xFFFFFu - key_label(m))) : stamp_bits;
+                            asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p.kslot + ((size_t)rg * p.nj + e) * vt_pad + my_vt), "l"(word) : "memory");
+                        }
+                        // a hint for the readers' wait (relaxed: nothing is ordered by it), one per storing warp, behind
+                        // the warp's stores
+                        __syncwarp();
+                        if (lane == 0 && e < n_tile) red_relaxed_add(f_keys + rg, 1u);
+                    }
                     if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_EPI_DONE);
                 }
                 ++use1;
             }
+            if (!forced) early_res();     // behind the joint's MMAs: the GEMMs of the next decoder-update slot
             ++n_j;
             if (warp >= 2 && e == 0) slot_done(TR_J);
         }
