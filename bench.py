@@ -170,6 +170,15 @@ def run_cpu_baseline(cfg, weights, enc, lens, W, seconds_target=15.0):
                 seconds=dt, steps=st["steps"])
 
 
+def set_loop_mode(pkg, mode):
+    if mode == "barriers":
+        pkg.wind_set_loop_options(resident=True, dataflow=0)
+    elif mode == "counters":
+        pkg.wind_set_loop_options(resident=True, dataflow=1)
+    elif mode == "streaming":
+        pkg.wind_set_loop_options(resident=False)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -182,6 +191,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the number of utterances (profiling captures of a small case)")
     ap.add_argument("--len-lo", type=int, default=0, help="override the shortest utterance length, frames")
     ap.add_argument("--len-hi", type=int, default=0, help="override the longest utterance length, frames")
+    ap.add_argument("--loop-mode", default="auto", choices=["auto", "barriers", "counters", "streaming"],
+                    help="tensor-core loop: the planner's choice, or resident weights with grid barriers / with arrival counters, or streamed weights")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the W=1 comparison, e2e and per-kernel timing legs")
     ap.add_argument("--op", default="decode", choices=["decode", "first_output", "window_greedy", "dataset", "beam"],
@@ -219,6 +230,7 @@ def main():
     torch.cuda.set_device(dev)
     pkg.load_library()
     pkg.wind_set_kernels(args.kernels)
+    set_loop_mode(pkg, args.loop_mode)
     peaks = load_peaks()
 
     weights = ws.make_model(cfg)
@@ -463,6 +475,7 @@ def window_greedy_op(args, cfg, W):
     torch.cuda.set_device(dev)
     pkg.load_library()
     pkg.wind_set_kernels(args.kernels)
+    set_loop_mode(pkg, args.loop_mode)
     weights = ws.make_model(cfg)
     enc_np, lens_np = ws.make_enc(cfg, pad="zero")
     model = pkg.WindModel(weights, device=dev)
@@ -535,6 +548,7 @@ def dataset_op(args, cfg, W):
     torch.cuda.set_device(dev)
     pkg.load_library()
     pkg.wind_set_kernels(args.kernels)
+    set_loop_mode(pkg, args.loop_mode)
     B = cfg.B
     big = replace(cfg, B=4 * B)
     weights = ws.make_model(cfg)

@@ -37,7 +37,8 @@
  *     tensor-core operands: enc_proj (stored once per call), the LSTM hidden state h wherever it
  *     is consumed (the recurrent term of the next update, the input of the layer above and
  *     pred_proj -- the recurrence therefore feeds back a bf16 h), and the joint's activations
- *     act(enc_proj + pred_proj).  Both kernel sets (wind_kernels_t) round in the same places.
+ *     act(enc_proj + pred_proj).  Both kernel sets (wind_kernels_t) round in the same places; the
+ *     tensor-core kernels with on-chip weights also round pred_proj to bf16 before that sum.
  *     The tensor-core kernels evaluate the gate nonlinearities (and tanh activations) with the
  *     hardware tanh approximation (absolute error about 5e-4, below the bf16 rounding of h) when
  *     the weights are resident on chip; the plain-ALU kernels use tanhf / expf.  Joint logits
@@ -379,15 +380,20 @@ wind_status_t wind_read_trace(const wind_model_t* m, int32_t B, int32_t T, int32
 int32_t wind_debug_stall_barrier(int32_t extra_arrivals);
 
 /*
- * Options of the tensor-core loop's tile planner, process-wide (defaults: 1, -1, 4).  Meant for tests and
+ * Options of the tensor-core loop's tile planner, process-wide (defaults: 1, -1, 4, -1).  Meant for tests and
  * measurements, which use them to reach every mode of the loop kernels on one shape; results do not depend on them.
  *   resident         0: never choose the resident-weights mode (weights then stream through shared memory every
  *                    step, as for shapes whose tiles do not fit on chip)
  *   joint_placement  streaming mode only: where a CTA keeps its W_out tile when it owns one joint item: -1 the
  *                    planner's choice, 0 streamed every step, 1 shared memory, 2 tensor memory (taken when feasible)
  *   max_joint_waves  resident mode: most passes over row groups the joint may take per step (1..4)
+ *   dataflow         resident mode: which of its two kernels runs.  0: the phases of a lock step are separated by grid
+ *                    barriers.  1: no grid barrier; CTAs hand results on through per-group arrival counters and stamped
+ *                    data, and a joint CTA builds its own operand from pred_proj and prefetched enc_proj rows.
+ *                    -1: the planner's choice (the second for one-layer models and batches up to 64 utterances,
+ *                    where it measures faster; the first beyond).  The two give the same transcripts.
  */
-void wind_set_loop_options(int32_t resident, int32_t joint_placement, int32_t max_joint_waves);
+void wind_set_loop_options(int32_t resident, int32_t joint_placement, int32_t max_joint_waves, int32_t dataflow);
 
 /*
  * The tile plan the tensor-core loop would use for a model and batch on a device with `sms` multiprocessors and
@@ -395,14 +401,14 @@ void wind_set_loop_options(int32_t resident, int32_t joint_placement, int32_t ma
  * invariants (every shared-memory region inside smem_bytes, tensor-memory columns within 512, disjoint CTA sets
  * inside the grid) can be checked over many shapes without a GPU.  WIND_ERR_UNSUPPORTED: the shapes are outside the
  * tensor-core path (dimensions not multiples of 64, fewer than 128 logits) or nothing fits.
- * Resident mode (resident = 1): CTAs [0, l_sets * l_items) hold decoder tiles (l_items = ut_count unit tiles x ql_count
+ * Resident mode (resident = 1; dataflow: which of its two kernels): CTAs [0, l_sets * l_items) hold decoder tiles (l_items = ut_count unit tiles x ql_count
  * utterance groups of nl), the last p_items = ht_count x qp_count CTAs hold W_pred tiles (np utterances each), CTAs
  * [w_first, w_first + w_count) record the steps; shared memory of a CTA: tile_bytes at 0, the state box at buf_off, the
  * joint's operand (nj rows x H) at z_off (z_off_p in W_pred CTAs), staging from stage_off to smem_bytes - 1024.
  * Streaming mode: rings of stages_lp x stage_lp and stages_j x stage_j bytes behind tile_bytes.
  */
 typedef struct {
-    int32_t grid, resident, smem_bytes;
+    int32_t grid, resident, dataflow, smem_bytes;
     int32_t nj, vt_count, rg_count, rg_stride, j_mode;
     int32_t tm_j, tm_l, tm_p;
     int32_t nl, np, ut_count, ht_count, ql_count, qp_count, l_items, p_items, w_first, w_count, l_sets;

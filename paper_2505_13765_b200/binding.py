@@ -72,7 +72,7 @@ class wind_profile_t(C.Structure):
 
 class wind_plan_t(C.Structure):
     _fields_ = [(k, C.c_int32) for k in (
-        "grid", "resident", "smem_bytes", "nj", "vt_count", "rg_count", "rg_stride", "j_mode", "tm_j", "tm_l", "tm_p",
+        "grid", "resident", "dataflow", "smem_bytes", "nj", "vt_count", "rg_count", "rg_stride", "j_mode", "tm_j", "tm_l", "tm_p",
         "nl", "np", "ut_count", "ht_count", "ql_count", "qp_count", "l_items", "p_items", "w_first", "w_count", "l_sets",
         "tile_bytes", "buf_off", "z_off", "z_off_p", "stage_off",
         "slots", "ul", "ug_count", "mt_count", "hg_count", "stages_lp", "stages_j", "stage_lp", "stage_j")]
@@ -136,7 +136,7 @@ def load_library():
     L.wind_debug_stall_barrier.restype = i32
     L.wind_set_kernels.argtypes = [i32]
     L.wind_set_kernels.restype = i32
-    L.wind_set_loop_options.argtypes = [i32, i32, i32]
+    L.wind_set_loop_options.argtypes = [i32, i32, i32, i32]
     L.wind_set_loop_options.restype = None
     L.wind_debug_plan.argtypes = [mp, i32, i32, i32, i32, C.POINTER(wind_plan_t)]
     L.wind_debug_plan.restype = i32
@@ -162,9 +162,9 @@ def wind_status_string(status: int) -> str:
     return load_library().wind_status_string(status).decode()
 
 
-def wind_set_loop_options(resident: bool = True, joint_placement: int = -1, max_joint_waves: int = 4) -> None:
+def wind_set_loop_options(resident: bool = True, joint_placement: int = -1, max_joint_waves: int = 4, dataflow: int = -1) -> None:
     """Options of the loop kernels' tile planner (process-wide); the defaults restore normal operation."""
-    load_library().wind_set_loop_options(int(bool(resident)), int(joint_placement), int(max_joint_waves))
+    load_library().wind_set_loop_options(int(bool(resident)), int(joint_placement), int(max_joint_waves), int(dataflow))
 
 
 def wind_debug_plan(dims: Dict[str, int], B: int, W: int, sms: int = 148, smem_optin: int = 232448):

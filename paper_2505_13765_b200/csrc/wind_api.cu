@@ -593,11 +593,12 @@ wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t*
 
 int32_t wind_debug_stall_barrier(int32_t extra_arrivals) { return loop_set_extra_arrivals(extra_arrivals); }
 
-void wind_set_loop_options(int32_t resident, int32_t joint_placement, int32_t max_joint_waves) {
+void wind_set_loop_options(int32_t resident, int32_t joint_placement, int32_t max_joint_waves, int32_t dataflow) {
     LoopOptions o;
     o.resident = resident != 0;
     o.joint_placement = joint_placement >= 0 && joint_placement <= 2 ? joint_placement : -1;
     o.max_joint_waves = max_joint_waves >= 1 && max_joint_waves <= 4 ? max_joint_waves : 4;
+    o.dataflow = dataflow < 0 ? -1 : (dataflow != 0);
     loop_set_options(o);
 }
 
@@ -610,7 +611,7 @@ wind_status_t wind_debug_plan(const wind_model_t* m, int32_t B, int32_t W, int32
         return WIND_ERR_UNSUPPORTED;
     LoopPlan pl;
     if (loop_plan_for(*m, B, W, sms, smem_optin, &pl) != cudaSuccess) return WIND_ERR_UNSUPPORTED;
-    out->grid = pl.grid; out->resident = pl.resident; out->smem_bytes = (int32_t)pl.smem_bytes;
+    out->grid = pl.grid; out->resident = pl.resident; out->dataflow = pl.resident ? pl.dataflow : 0; out->smem_bytes = (int32_t)pl.smem_bytes;
     out->nj = pl.nj; out->vt_count = pl.vt_count; out->rg_count = pl.rg_count; out->rg_stride = pl.rg_stride; out->j_mode = pl.j_mode;
     out->tm_j = pl.tm_j; out->tm_l = pl.tm_l; out->tm_p = pl.tm_p;
     out->nl = pl.nl; out->np = pl.np; out->ut_count = pl.ut_count; out->ht_count = pl.ht_count; out->ql_count = pl.ql_count;

@@ -1,5 +1,5 @@
-// The decoding loop of the bf16 path as ONE persistent cooperative kernel (sm_100a): streaming mode, and the host
-// side of both modes (tile plan, tensor maps, launch).
+// The decoding loop of the bf16 path as ONE persistent cooperative kernel (sm_100a) whose phases are separated by
+// grid barriers, and the host side of all loop kernels (tile plan, tensor maps, launch).
 //
 // One CTA per SM stays resident for the whole decode.  A lock step of the batch
 // (Algorithm 2 applied to every utterance at once) is three phases separated by grid
@@ -24,9 +24,14 @@
 // (one thread per tensor-memory lane).  State that one phase reads while another CTA writes it
 // is double-buffered by step parity (t, keys), so a phase never reads what it writes.
 //
-// This file's kernel is the streaming mode: weights flow through a TMA ring every step (large vocabularies,
-// more than two LSTM layers, batches whose tiles outnumber the SMs).  Shapes whose weight tiles fit on chip run
-// the resident-weights kernel of wind_loop_res.cu instead (no grid barriers, operands built in place).
+// Two modes (template parameter RES).  The description above is the streaming mode: weights flow
+// through a TMA ring every step.  In the resident-weights mode (one or two LSTM layers, shapes whose
+// tiles fit) the W_out tile of a CTA lives in tensor memory and 64-row tiles of W_hh / W_pred (and of
+// layer 1's matrices) in the shared memory of disjoint CTA sets for the whole decode; the GEMMs are
+// transposed (weights on the M axis, utterances on N), every per-step operand is one TMA box, two
+// threads issue the MMAs, eight warps run the epilogues, and CTAs without a weight tile record the
+// steps (outputs, counters, next frame).  (wind_loop_res.cu holds a second kernel for the resident-weights
+// mode, without grid barriers; the tile planner below chooses between the two.)
 //
 // Two variants (template parameter FULL): teacher forcing with the logits store (wind_eval_joint_window),
 // window-based decoding (the best (label, offset) pair of Eq. (1) decides the step: per-row softmax
@@ -47,10 +52,15 @@ namespace wind {
 
 constexpr int LOOP_MAX_STAGES = 28;
 constexpr uint32_t LOOP_A_BYTES = 128 * BK * 2;  // one K block of a 128-row operand tile
+constexpr int kDataflowMaxBatch = 64;             // largest batch for which the planner picks the barrier-free resident kernel (one LSTM layer)
+constexpr int kDataflowMaxBatch2 = 0;             // the same with two LSTM layers (measured at 16 and 32 utterances: grid barriers ahead)
+
+// RES: resident-weights mode (compile-time, so that each instantiation carries only its own code paths: the loop
+// body runs once per lock step, straight through, and instruction fetch is a visible cost at that scale).
 // FULL: the kernel also carries teacher forcing with the logits store, window-based decoding and the timeline; the
 // plain decode runs the variant without them (a smaller instruction footprint: the loop is sensitive to it).
-template <bool FULL>
-__global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_constant__ LoopMaps M, const LoopParams p) {
+template <bool RES, bool FULL>
+__global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop_kernel(const __grid_constant__ LoopMaps M, const LoopParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[LOOP_MAX_STAGES], empty_bar[LOOP_MAX_STAGES], stat_bar;
     __shared__ uint64_t acc_full[3], acc_empty[3];   // accumulators: joint, decoder, projection
@@ -73,14 +83,16 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
     if (threadIdx.x == 0) {
         s_abort = 0;
         s_active = 0;
+        // resident-weights mode: two threads issue the MMAs of a GEMM (each its half of the K blocks), both commit
+        const uint32_t issuers = RES ? 2u : 1u;
         for (int s = 0; s < LOOP_MAX_STAGES; ++s) {
             mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], 1);
+            mbar_init(&empty_bar[s], s == 0 ? issuers : 1u);
         }
         mbar_init(&stat_bar, 1);
         for (int k = 0; k < 3; ++k) {
-            mbar_init(&acc_full[k], 1);
-            mbar_init(&acc_empty[k], 4);   // one arrival per epilogue warp
+            mbar_init(&acc_full[k], issuers);
+            mbar_init(&acc_empty[k], RES ? 8u : 4u);   // one arrival per epilogue warp
         }
         fence_barrier_init();
     }
@@ -91,18 +103,49 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
     const uint32_t tmem_base = tmem_slot;
     const uint32_t tm_j = tmem_base + (uint32_t)p.tm_j, tm_l = tmem_base + (uint32_t)p.tm_l, tm_p = tmem_base + (uint32_t)p.tm_p;
 
-    const int e = threadIdx.x - 64;            // epilogue thread: 0..127 (warps 2..5)
+    const int e = threadIdx.x - 64;            // epilogue thread: 0..127 (warps 2..5), 0..255 (warps 2..9) in resident mode
+    const int sub = (warp - 2) >> 2;           // resident mode: which of the two warps of a lane quadrant (0 otherwise)
     const int q = warp & 3;                    // tensor-memory lane quadrant of this warp
     const int row_in_tile = q * 32 + lane;     // the tensor-memory lane (accumulator row) of this thread
     const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-    // joint items of this CTA: items cta, cta + G, ... of the (row group, vocabulary tile) list
-    const bool has_j = cta < p.j_items;
+    // joint items of this CTA.  Streaming mode: items cta, cta + G, ... of the (row group, vocabulary tile) list.
+    // Resident mode: the CTA keeps ONE vocabulary tile (cta % vt_count) and takes the row groups j_first,
+    // j_first + rg_stride, ... (one per wave); CTAs beyond vt_count * rg_stride have none.
+    const int j_first = RES ? (cta < p.vt_count * p.rg_stride ? cta / p.vt_count : p.rg_count) : 0;
+    const bool has_j = RES ? j_first < p.rg_count : cta < p.j_items;
     const int my_vt = cta % p.vt_count;        // vocabulary tile of this CTA's joint item when it has exactly one
 
     // ----- the joint's W_out tile, loaded once when every CTA owns one joint item -----
     if (p.j_mode == J_SMEM && has_j && threadIdx.x == 0) {
         mbar_expect_tx(&stat_bar, (uint32_t)p.kb_h * LOOP_A_BYTES);
         for (int kb = 0; kb < p.kb_h; ++kb) tma_load_2d(stat + (size_t)kb * LOOP_A_BYTES, &M.w_out, kb * BK, my_vt * 128, &stat_bar);
+    }
+    // resident-weights mode: CTAs [0, l_items) keep a W_hh tile (4 gates x 16 units), the last p_items CTAs a W_pred
+    // tile (64 rows), loaded once; `stat` holds kb_p blocks of 64 rows x 64 columns
+    // With two LSTM layers two more CTA sets follow the layer-0 set: "x1" keeps a W_ih[1] tile (layer 1's GEMM on the
+    // new layer-0 state, in its own phase) and "h1" a W_hh[1] tile (layer 1's recurrent term, issued a phase ahead
+    // like layer 0's GEMM and handed over through global memory).
+    const int r_role = RES ? cta / p.l_items : 0;                  // 0 layer 0, 1 x1, 2 h1 (while below the L CTA count)
+    const int r_idx = RES ? cta - r_role * p.l_items : 0;
+    const bool res_l = RES && cta < p.l_items;
+    const bool res_x1 = RES && p.L == 2 && r_role == 1;
+    const bool res_h1 = RES && p.L == 2 && r_role == 2;
+    const bool res_p = RES && !res_l && !res_x1 && !res_h1 && G - 1 - cta < p.p_items;
+    const bool res_w = RES && cta >= p.w_first && cta < p.w_first + p.w_count;   // step-recording CTAs (none of the above)
+    const int r_ut = r_idx % p.ut_count, r_ql = r_idx / p.ut_count;                  // unit tile / utterance group of an L CTA
+    const int r_ht = (G - 1 - cta) % p.ht_count, r_qp = (G - 1 - cta) / p.ht_count;  // H tile / utterance group of a P CTA
+    constexpr uint32_t RES_A_BYTES = 64 * BK * 2;
+    if (threadIdx.x == 0 && (res_l || res_x1 || res_h1 || res_p)) {
+        mbar_expect_tx(&stat_bar, (uint32_t)p.kb_p * RES_A_BYTES);
+        for (int kb = 0; kb < p.kb_p; ++kb) {
+            uint8_t* dst = stat + (size_t)kb * RES_A_BYTES;
+            if (!res_p) {
+                const CUtensorMap* wm = res_l ? &M.w_hh_r : (res_x1 ? &M.w_ih1_r : &M.w_hh1_r);
+                for (int g = 0; g < 4; ++g) tma_load_2d(dst + g * 16 * 128, wm, kb * BK, g * p.P + r_ut * 16, &stat_bar);
+            } else {
+                tma_load_2d(dst, &M.w_pred_r, kb * BK, r_ht * 64, &stat_bar);
+            }
+        }
     }
     if (p.j_mode == J_TMEM) {
         if (warp >= 2 && has_j) {
@@ -149,7 +192,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         if (threadIdx.x == 0) {
             epoch += (uint32_t)(G + p.extra_arrivals);   // extra_arrivals > 0: a test hook, the barrier can then never fill
             if constexpr (FULL) trace_event(p, 3, tr_n, step, phase_kind, EV_ARRIVE);
-            if constexpr (FULL) trace_phase_done(p, step, phase_kind);   // when every CTA finished its part of the phase
+            if constexpr (FULL) trace_phase_done(p, step, phase_kind);   // when this CTA finished its part of the phase
             if (s_abort) {
                 atomicExch(&p.ctrl->abort, 1);
             } else {
@@ -397,8 +440,501 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         return true;
     };
 
+    // =========================================================================================
+    // resident-weights mode.  Every per-step operand is ONE three-dimensional TMA box (all K blocks at once) into
+    // the single operand buffer, and every GEMM is one wait, kb x 4 MMAs back to back, two commits: the issuing
+    // threads pay for as few asynchronous instructions as possible.
+    //   decoder:    D[4 gates x 16 units, nl utterances] = W_hh tile . h^T   (warp q of the epilogue = gate q)
+    //   projection: D[64 H rows, np utterances] = W_pred tile . h^T
+    // With 64 accumulator rows, row m sits in lane (m % 16) of quadrant m / 16.
+    // =========================================================================================
+    float* stage_f = reinterpret_cast<float*>(smem + p.stage_off);   // epilogue staging
+    auto produce_one = [&](const CUtensorMap* map, int row0, uint32_t bytes) -> bool {
+        cur = 0;
+        uint8_t* dst = acquire(0);
+        if (!dst) return false;
+        mbar_expect_tx(&full_bar[0], bytes);
+        tma_load_3d(dst, map, 0, row0, 0, &full_bar[0]);
+        return true;
+    };
+    // One issuing thread's share of a GEMM: K blocks [kb_lo, kb_hi) into the accumulator at tm_d.  Two threads call
+    // this for every GEMM (warp 1 and, after it has issued the TMA box, warp 0), with disjoint K ranges and
+    // separate accumulator copies that the epilogue adds; an empty range only takes part in the commits.
+    auto mma_part = [&](int k_acc, uint32_t tm_d, int n_tile, int kb_lo, int kb_hi, bool a_tmem) -> bool {
+        const uint32_t idesc = idesc_bf16(a_tmem ? 128 : 64, n_tile);
+        if (!a_tmem && !mbar_wait(&stat_bar, 0, &s_abort)) return false;
+        if (!begin_acc(k_acc)) return false;
+        cur = 0;
+        if (!consume()) return false;
+        const uint32_t b_addr = smem_u32(ring);
+        const uint32_t b_block = (uint32_t)n_tile * BK * 2;
+        for (int kb = kb_lo; kb < kb_hi; ++kb) {
+            const uint64_t bdesc = smem_desc_sw128(b_addr + (uint32_t)kb * b_block);
+            if (a_tmem) {
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)
+                    tc_mma_bf16_ts(tm_d, tmem_base + (uint32_t)(kb * (BK / 2) + k * 8), bdesc + (uint64_t)(k * 2), idesc,
+                                   kb != kb_lo || k != 0);
+            } else {
+                const uint64_t adesc = smem_desc_sw128(smem_u32(stat + (size_t)kb * RES_A_BYTES));
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)
+                    tc_mma_bf16(tm_d, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, kb != kb_lo || k != 0);
+            }
+        }
+        tc_commit(&empty_bar[0]);
+        tc_commit(&acc_full[k_acc]);
+        ++acc_n[k_acc];
+        return true;
+    };
+    // control step + LSTM cell update of an L CTA: units [r_ut*16, +16), utterances [r_ql*nl, +nl), 64 utterances per
+    // pass.  Warp (q, sub) of the epilogue owns gate q and the pass's utterances [32 sub, 32 sub + 32).  All global reads
+    // of a pass are requested together: first everything the control step needs, then the gate-table rows of the
+    // chosen tokens.  Lanes 16..31 hold no accumulator row (64-row tile); they take the second 16 utterances.
+    struct ScanIn { int t, len, cnt, pos; unsigned long long kk[8]; };
+    // ctl_only: the CTA is one of the step-recording CTAs (see the plan): it takes the control step of 64 utterances,
+    // records it (outputs, counters, next frame) and has no cell update; the L CTAs then record nothing.
+    auto epilogue_res_L = [&](const int layer, const bool ctl_only) -> bool {
+        if (ctl_only && q != 0) return true;
+        const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
+        int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
+        const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
+        unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
+        const int u16 = lane & 15, half = lane >> 4;
+        const int unit = r_ut * 16 + u16;        // this thread's hidden unit; its gate is q
+        // without recording CTAs, the two gate-0 warps of one CTA per utterance group record the step
+        const bool writer = ctl_only ? true : (p.w_count == 0 && layer == 0 && r_ut == 0 && q == 0);
+        const int n_here = ctl_only ? 64 : p.nl;
+        const int base = ctl_only ? (cta - p.w_first) * 64 : r_ql * p.nl;
+        const bool decode = step >= 0 && !(FULL && p.forced) && layer == 0;
+        float* cst = p.c_state + (size_t)layer * p.B * p.P + unit;
+        const __nv_bfloat16* hin = p.hb + ((size_t)(pin * p.L + layer) * p.Bpad) * p.P + unit;
+        __nv_bfloat16* hout = p.hb + ((size_t)((pin ^ 1) * p.L + layer) * p.Bpad) * p.P + unit;
+        const float bias1 = layer == 0 ? 0.f : p.b_ih[1][q * p.P + unit] + p.b_hh[1][q * p.P + unit];
+        const float* g0u = p.g0 + (size_t)q * p.P + unit;
+        const uint32_t g0_stride = 4u * (uint32_t)p.P;
+        bool ready = true;
+        for (int c0 = 0; c0 < n_here; c0 += 64) {
+            const int b0 = base + c0;
+            // ---- lane j decides for utterance b0 + 32 sub + j ----
+            const int jl = 32 * sub + lane;
+            const int b = b0 + jl;
+            const bool in = c0 + jl < n_here && b < p.B;
+            ScanIn si;
+            si.t = 0; si.len = 0; si.cnt = 0; si.pos = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) si.kk[j] = 0ull;
+            if (in && decode) {
+                si.t = t_cur[b];
+                si.len = p.enc_len[b];
+                if (writer) { si.cnt = p.count[b]; si.pos = p.out_len[b]; }
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (j < p.W) si.kk[j] = keys_cur[(size_t)b * p.W + j];
+            }
+            // old cell state of the four (utterance, unit) pairs this thread finishes
+            float cold[4];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                const int j = half + 2 * q + 8 * sub + 16 * jj;     // 0..63 over the CTA's 256 epilogue threads
+                cold[jj] = (!ctl_only && c0 + j < p.nl && b0 + j < p.B) ? cst[(size_t)(b0 + j) * p.P] : 0.f;
+            }
+            // the token utterance b feeds to its decoder in this step (-1: none)
+            int tok = -1, t_out = 0;
+            if (in) {
+                if (step < 0) {
+                    tok = p.blank;
+                } else if ((FULL && p.forced)) {
+                    tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
+                    if (tok >= p.NV || tok < -1) { tok = p.blank; set_status(p.ctrl, WIND_ERR_INVALID_ARG); }   // caller's mistake
+                } else if (layer > 0) {
+                    tok = p.emit_tok[b];     // decided by layer 0's CTAs one phase earlier
+                } else {
+                    int t = si.t;
+                    const int len = si.len;
+                    if (t < len) {
+                        // control step (Algorithm 2's branch): first non-blank row of the window
+                        const int n = min(p.W, len - t);
+                        int first = -1, label = p.blank;
+                        bool bad = false;
+                        for (int w0 = 0; w0 < n && first < 0; w0 += 8) {
+                            if (w0 > 0) {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) si.kk[j] = (w0 + j < n) ? keys_cur[(size_t)b * p.W + w0 + j] : 0ull;
+                            }
+                            // the eight rows side by side: which are inside the window, broken, non-blank
+                            uint32_t nonblank = 0u, broken = 0u;
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const uint32_t lab = key_label(si.kk[j]);
+                                const bool inside = w0 + j < n;
+                                const bool brk = si.kk[j] == 0ull || lab >= (uint32_t)p.NV;
+                                broken |= (uint32_t)(inside && brk) << j;
+                                nonblank |= (uint32_t)(inside && !brk && (int)lab != p.blank) << j;
+                            }
+                            if (nonblank) {
+                                const int j = __ffs((int)nonblank) - 1;
+                                first = w0 + j;
+                                uint32_t lab = 0u;
+#pragma unroll
+                                for (int jj = 0; jj < 8; ++jj)
+                                    if (jj == j) lab = key_label(si.kk[jj]);
+                                label = (int)lab;
+                                broken &= (1u << j) - 1u;   // rows after the first non-blank one are not looked at
+                            }
+                            bad = bad || broken != 0u;
+                        }
+                        if (first >= 0) tok = label;
+                        if (writer) {
+                            int cnt = si.cnt, jump, forced = 0, emitted = 0;
+                            if (first < 0) {
+                                jump = n;
+                                t += n;
+                                cnt = 0;
+                            } else {
+                                jump = first;
+                                if (first > 0) cnt = 0;
+                                t += first;
+                                if (si.pos < p.max_out) {
+                                    p.out_tokens[(size_t)b * p.max_out + si.pos] = label;
+                                    p.out_frames[(size_t)b * p.max_out + si.pos] = t;
+                                    p.out_len[b] = si.pos + 1;
+                                    emitted = 1;
+                                    cnt += 1;
+                                    if (cnt == p.S) { t += 1; cnt = 0; forced = 1; }
+                                } else {
+                                    set_status(p.ctrl, WIND_ERR_OUTPUT_OVERFLOW);  // this utterance stops here
+                                    t = len;
+                                    tok = -1;
+                                }
+                            }
+                            if (bad) set_status(p.ctrl, WIND_ERR_INTERNAL);
+                            t_nxt[b] = t;
+                            t_out = t;
+                            p.count[b] = cnt;
+                            for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
+                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->jump_hist[jump < 64 ? jump : 64]), 1ull);
+                            atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->joint_rows), (unsigned long long)n);
+                            if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
+                            if (forced) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
+                        }
+                    } else if (writer) {
+                        t_nxt[b] = t;
+                        t_out = t;
+                    }
+                }
+                // the next frame goes out at once, stamped with the step, for the projection CTAs (which fetch their
+                // enc_proj rows while this phase is still running)
+                if (writer && !(FULL && p.forced)) p.t_pub[b] = ((unsigned long long)(uint32_t)(step + 2) << 32) | (uint32_t)t_out;
+                if (writer && p.L > 1 && decode) p.emit_tok[b] = tok;   // the upper layer's CTAs read it in their phase
+            }
+            if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
+            if (ctl_only) continue;
+            // ---- gate-table entries (this thread's gate and unit) of the tokens of this lane half's 16 utterances ----
+            float add[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int ta = __shfl_sync(0xffffffffu, tok, j), tb = __shfl_sync(0xffffffffu, tok, 16 + j);
+                const int tj = half ? tb : ta;
+                if (layer == 0) {
+                    add[j] = tj >= 0 ? g0u[(uint32_t)tj * g0_stride] : 0.f;
+                } else {
+                    // layer 1: the recurrent term W_hh h computed a phase ahead by the h1 CTAs, plus the biases
+                    const int bj2 = b0 + 32 * sub + 16 * half + j;
+                    add[j] = (tj >= 0 && bj2 < p.B) ? p.dh[(size_t)bj2 * g0_stride + (size_t)q * p.P + unit] + bias1 : 0.f;
+                }
+            }
+            // the other warps need the tokens for the cell update below: through shared memory
+            int* tok_s = reinterpret_cast<int*>(stage_f + 4 * 64 * 16);
+            if (q == 0) tok_s[jl] = tok;
+            if (c0 == 0) {
+                ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, &s_abort));
+                tc_fence_after();
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_ACC);
+            }
+            if (ready) {
+                // lanes 0..15 read their row's 32 columns; columns 16..31 then move to lanes 16..31
+                float x[16], hi[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) { x[j] = 0.f; hi[j] = 0.f; }
+                const int col = c0 + 32 * sub;
+                if (col < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)col, x);
+                if (col + 16 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(col + 16), hi);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float v = __shfl_sync(0xffffffffu, hi[j], u16);
+                    if (half) x[j] = v;
+                }
+                // warp q holds gate q: tanh for the cell candidate (q == 2), logistic for the other three,
+                // written as 0.5 tanh(x / 2) + 0.5 so that both are one hardware tanh
+                const float sc = q == 2 ? 1.f : 0.5f, of = q == 2 ? 0.f : 0.5f;
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    stage_f[(q * 64 + 32 * sub + 16 * half + j) * 16 + u16] = fmaf(tanh_fast((x[j] + add[j]) * sc), sc, of);
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (ready) {
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = half + 2 * q + 8 * sub + 16 * jj;     // 0..63
+                    const int bj = b0 + j;
+                    if (c0 + j < p.nl && bj < p.B) {
+                        if (tok_s[j] >= 0) {
+                            const float gi = stage_f[(0 * 64 + j) * 16 + u16], gf = stage_f[(1 * 64 + j) * 16 + u16];
+                            const float gg = stage_f[(2 * 64 + j) * 16 + u16], go = stage_f[(3 * 64 + j) * 16 + u16];
+                            const float cc = gf * cold[jj] + gi * gg;
+                            cst[(size_t)bj * p.P] = cc;
+                            hout[(size_t)bj * p.P] = __float2bfloat16_rn(go * tanh_fast(cc));
+                        } else {
+                            hout[(size_t)bj * p.P] = hin[(size_t)bj * p.P];
+                        }
+                    }
+                }
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+        }
+        if (ctl_only) return true;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[1]);
+        ++acc_n[1];
+        fence_proxy_async_all();
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_EPI_DONE);
+        return ready;
+    };
+    // z rows of a P CTA: row r = (utterance bl = r / W of the CTA's group, window row w = r % W), 64 columns = 128 bytes =
+    // eight 16-byte chunks.  Thread e owns chunk (e & 7) of rows (e >> 3) + 32 i, so that eight neighbouring lanes
+    // read and write one whole 128-byte row segment.  Row kinds: 0 nothing to write (outside the batch, or the
+    // utterance is done), 1 zeros (past the utterance's end), 2 act(enc_proj row + pred_proj).
+    //
+    // During the decoder-update phase a P CTA has nothing else to do: it waits for the next frame of its
+    // utterances to be published and starts copying the enc_proj chunks of its first 256 rows into a shared-memory
+    // stash (asynchronous copies, collected in the projection epilogue).  pre_kinds: 2 bits per row, -1 = no prefetch.
+    uint8_t* stash = ring + (size_t)p.np * p.P * 2;   // behind the projection's own operand box
+    int pre_kinds = -1;
+    const int p_chunk = e & 7, p_row0 = e >> 3;
+    // the (utterance, window row) of this thread's first eight rows never changes: worked out once, so that the
+    // per-step code has no integer division; -1 = no such row
+    int p_bw[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        p_bw[i] = -1;
+        if (res_p && e >= 0) {
+            const int r = p_row0 + 32 * i;
+            const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
+            if (r < p.np * p.W && b < p.B) p_bw[i] = (b << 8) | w;
+        }
+    }
+    // b_pred of this thread's accumulator row: constant for the whole decode, read once
+    const float p_bias = (res_p && e >= 0) ? p.b_pred[r_ht * 64 + 16 * q + (lane & 15)] : 0.f;
+    // kind of a row at frame position t of its utterance, and the row's enc_proj frame
+    auto row_kind = [&](int b, int w, int t, int& frame) -> int {
+        const int left = p.enc_len[b] - t;
+        frame = t + w;
+        return left <= 0 ? 0 : (w >= left ? 1 : 2);
+    };
+    auto prefetch_res_P = [&]() {
+        pre_kinds = -1;
+        if ((FULL && p.forced)) return;
+        const uint32_t want = (uint32_t)(step + 2);
+        // the published frames of this thread's rows, all requested together, until every stamp is this step's
+        unsigned long long v[8];
+        unsigned long long t0 = 0;
+        for (uint32_t it = 1;; ++it) {
+            bool all = true;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                v[i] = (unsigned long long)want << 32;
+                if (p_bw[i] >= 0) asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(v[i]) : "l"(p.t_pub + (p_bw[i] >> 8)) : "memory");
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) all = all && (uint32_t)(v[i] >> 32) == want;
+            if (all) break;
+            if ((it & 15u) == 0u) {
+                if (s_abort || ld_volatile_i32(&p.ctrl->abort)) return;
+                const unsigned long long now = globaltimer_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > kWaitLimitNs) { s_abort = 1; return; }
+            }
+        }
+        int kinds = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (p_bw[i] < 0) continue;
+            const int b = p_bw[i] >> 8, w = p_bw[i] & 255;
+            int frame = 0;
+            const int kind = row_kind(b, w, (int)(uint32_t)v[i], frame);
+            kinds |= kind << (2 * i);
+            if (kind == 2) {
+                const __nv_bfloat16* src = p.enc_proj + ((size_t)b * p.T + frame) * p.H + r_ht * 64 + p_chunk * 8;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(stash + (size_t)(p_row0 + 32 * i) * 128 + p_chunk * 16)),
+                             "l"(src)
+                             : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        pre_kinds = kinds;
+    };
+    // projection epilogue of a P CTA: pred_proj rows [r_ht*64, +64) of utterances [r_qp*np, +np), then z
+    auto epilogue_res_P = [&]() -> bool {
+        const int32_t* t_new = p.t2 + (size_t)((step + 1) & 1) * p.B;
+        const int h0 = r_ht * 64;
+        const int rows_here = p.np * p.W;
+        // one 16-byte chunk of a z row: act(enc_proj chunk + pred_proj chunk), zeros past the utterance's end
+        // (pred_proj is rounded to bf16 and the sum is taken in bf16 arithmetic, one rounding: the same instruction
+        // sequence as in the resident kernel without grid barriers, so that the two give the same transcripts)
+        auto z_chunk = [&](int bl, int kind, uint4 ev) -> uint4 {
+            const float4* gs = reinterpret_cast<const float4*>(stage_f + bl * 68 + p_chunk * 8);
+            const float4 ga = gs[0], gb = gs[1];
+            if (kind != 2) return make_uint4(0, 0, 0, 0);
+            return make_uint4(act_add_bf16x2(ev.x, pack_bf16x2(ga.x, ga.y), p.act), act_add_bf16x2(ev.y, pack_bf16x2(ga.z, ga.w), p.act),
+                              act_add_bf16x2(ev.z, pack_bf16x2(gb.x, gb.y), p.act), act_add_bf16x2(ev.w, pack_bf16x2(gb.z, gb.w), p.act));
+        };
+        // the chunks of this thread's first eight rows: prefetched, or requested now before the accumulator is ready
+        uint4 ev[8];
+        int kinds = pre_kinds;
+        if (kinds < 0) {
+            kinds = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                ev[i] = make_uint4(0, 0, 0, 0);
+                if (p_bw[i] >= 0) {
+                    const int b = p_bw[i] >> 8, w = p_bw[i] & 255;
+                    int frame = 0;
+                    const int kind = row_kind(b, w, t_new[b], frame);
+                    kinds |= kind << (2 * i);
+                    if (kind == 2) ev[i] = *reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + frame) * p.H + h0 + p_chunk * 8);
+                }
+            }
+        } else {
+            asm volatile("cp.async.wait_all;" ::: "memory");
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                ev[i] = make_uint4(0, 0, 0, 0);
+                if (((kinds >> (2 * i)) & 3) == 2) ev[i] = *reinterpret_cast<const uint4*>(stash + (size_t)(p_row0 + 32 * i) * 128 + p_chunk * 16);
+            }
+        }
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
+        const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[2], acc_n[2] & 1u, &s_abort));
+        tc_fence_after();
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
+        if (ready) {
+            const int hl = 16 * q + (lane & 15);
+            const float bias = p_bias;
+            for (int c0 = 16 * sub; c0 < p.np; c0 += 32) {
+                float g[16], more[16];
+                tmem_ld16(tm_p + lane_off + (uint32_t)c0, g);
+                tmem_ld16(tm_p + lane_off + (uint32_t)(p.np + c0), more);   // the other issuing thread's K blocks
+                if (p.kb_p < 2) {   // a single K block: the first copy's issuer had an empty range and wrote nothing
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) g[j] = 0.f;
+                }
+                if (lane < 16) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) stage_f[(c0 + j) * 68 + hl] = g[j] + more[j] + bias;
+                }
+            }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[2]);
+        ++acc_n[2];
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (ready) {
+            uint4 out[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int bl = p_bw[i] >= 0 ? (p_bw[i] >> 8) - r_qp * p.np : 0;
+                out[i] = z_chunk(bl, (kinds >> (2 * i)) & 3, ev[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (p_bw[i] >= 0 && ((kinds >> (2 * i)) & 3) != 0) {
+                    const int b = p_bw[i] >> 8, w = p_bw[i] & 255;
+                    *reinterpret_cast<uint4*>(p.z + ((size_t)b * p.W + w) * p.H + h0 + p_chunk * 8) = out[i];
+                }
+            }
+            // rows beyond the first 256 of this CTA (wide windows): same chunking, fetched here
+            // (four rows at a time, their loads requested together)
+            for (int r0 = p_row0 + 256; r0 < rows_here; r0 += 128) {
+                uint4 x[4];
+                int kinds4[4], bls[4];
+                size_t zoff[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int r = r0 + 32 * i;
+                    const int bl = r / p.W, w = r - bl * p.W, b = r_qp * p.np + bl;
+                    x[i] = make_uint4(0, 0, 0, 0);
+                    kinds4[i] = 0; bls[i] = 0; zoff[i] = 0;
+                    if (r < rows_here && b < p.B) {
+                        int frame = 0;
+                        kinds4[i] = row_kind(b, w, t_new[b], frame);
+                        bls[i] = bl;
+                        zoff[i] = ((size_t)b * p.W + w) * p.H + h0 + p_chunk * 8;
+                        if (kinds4[i] == 2)
+                            x[i] = *reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + frame) * p.H + h0 + p_chunk * 8);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (kinds4[i] != 0) *reinterpret_cast<uint4*>(p.z + zoff[i]) = z_chunk(bls[i], kinds4[i], x[i]);
+            }
+        }
+        fence_proxy_async_all();
+        if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
+        return ready;
+    };
+    // the decoder GEMM of the next step, on the state hb[pin] (TMA and MMA issuers of an L CTA)
+    // h1 CTAs: the finished recurrent term of layer 1 goes to global memory (fp32 [B][4P], gate-major like the gate
+    // table); the x1 CTAs add it one or two phases later
+    auto store_res_h1 = [&]() {
+        const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[1], acc_n[1] & 1u, &s_abort));
+        tc_fence_after();
+        if (ready) {
+            const int unit = r_ut * 16 + (lane & 15);
+            for (int c0 = 0; c0 < p.nl; c0 += 64) {
+                const int col = c0 + 32 * sub;
+                float x[16], hi[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) { x[j] = 0.f; hi[j] = 0.f; }
+                if (col < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)col, x);
+                if (col + 16 < p.nl) tmem_ld16(tm_l + lane_off + (uint32_t)(col + 16), hi);
+                if (lane < 16) {
+                    float* dst = p.dh + (size_t)q * p.P + unit;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int ba = r_ql * p.nl + col + j, bb = ba + 16;
+                        if (col + j < p.nl && ba < p.B) dst[(size_t)ba * 4 * p.P] = x[j];
+                        if (col + 16 + j < p.nl && bb < p.B) dst[(size_t)bb * 4 * p.P] = hi[j];
+                    }
+                }
+            }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[1]);
+        ++acc_n[1];
+    };
+    // GEMMs that need only the state, issued a phase ahead: layer 0's (its result waits in tensor memory for the
+    // next control step) and, with two layers, layer 1's recurrent term (stored by store_res_h1)
+    auto early_res = [&]() {
+        if (warp == 0) {
+            if (lane == 0 && (res_l || res_h1)) {
+                fence_proxy_async_all();
+                if (produce_one(res_l ? &M.hb_l3[pin] : &M.hb_l3_1[pin], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u))
+                    mma_part(1, tm_l, p.nl, p.kb_p, p.kb_p, false);   // one accumulator: warp 1 issues all of it
+            }
+        } else if (warp == 1) {
+            if (lane == 0 && (res_l || res_h1)) mma_part(1, tm_l, p.nl, 0, p.kb_p, false);
+        } else if (res_h1) {
+            store_res_h1();
+        }
+    };
+
     // ----- before the loop: layer 0's GEMM on the initial (zero) state -----
-    if (early) {
+    if constexpr (RES) {
+        early_res();
+    } else if (early) {
         if (warp == 0) {
             if (lane == 0) { fence_proxy_async_all(); cur = 0; produce_L(0); }
         } else if (warp == 1) {
@@ -410,7 +946,32 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         // =====================================================================================
         // decoder phases: control step + LSTM cell update (layer 0), then one GEMM + update phase per upper layer
         // =====================================================================================
-        for (int l = 0; l < p.L; ++l) {
+        if constexpr (RES) {
+            if (warp >= 2) {
+                if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_START);
+                if (res_l) epilogue_res_L(0, false);
+                else if (res_w) epilogue_res_L(0, true);
+                else if (res_p) prefetch_res_P();
+                if (cta == 0 && e == 0 && step >= 0 && !(FULL && p.forced)) p.ctrl->step = step + 1;
+            }
+            if (!grid_sync(TR_L)) goto done;
+            if (p.L == 2) {
+                // layer 1: W_ih[1] . (new layer-0 state) on the x1 CTAs, then their cell update
+                if (warp == 0) {
+                    if (lane == 0 && res_x1) {
+                        fence_proxy_async_all();
+                        if (produce_one(&M.hb_l3[pin ^ 1], r_ql * p.nl, (uint32_t)p.nl * (uint32_t)p.P * 2u))
+                            mma_part(1, tm_l, p.nl, p.kb_p, p.kb_p, false);
+                    }
+                } else if (warp == 1) {
+                    if (lane == 0 && res_x1) mma_part(1, tm_l, p.nl, 0, p.kb_p, false);
+                } else if (res_x1) {
+                    epilogue_res_L(1, false);
+                }
+                if (!grid_sync(TR_L)) goto done;
+            }
+        }
+        for (int l = 0; l < p.L && !RES; ++l) {
             const bool gemm_here = l > 0 || !early;
             if (warp == 0) {
                 if (lane == 0 && gemm_here) { fence_proxy_async_all(); cur = 0; produce_L(l); }
@@ -425,7 +986,9 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
         pin ^= 1;
         if ((FULL && p.forced) && step + 1 < p.U) {
             // teacher forcing: more prefix tokens to feed before the window is evaluated
-            if (early) {
+            if constexpr (RES) {
+                early_res();
+            } else if (early) {
                 if (warp == 0) {
                     if (lane == 0) { fence_proxy_async_all(); cur = 0; produce_L(0); }
                 } else if (warp == 1) {
@@ -445,7 +1008,28 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
             const uint32_t b_bytes = (uint32_t)n_tile * BK * 2;
             const int32_t* t_new = p.t2 + (size_t)((step + 1) & 1) * p.B;
             const int i0 = p.p_items <= G ? G - 1 - cta : cta;   // projection items start at the far end of the grid
-            if (warp == 0) {
+            if constexpr (RES) {
+                if (warp == 0) {
+                    if (lane == 0 && res_p) {
+                        fence_proxy_async_all();
+                        if (produce_one(&M.hb_p3[pin], r_qp * p.np, (uint32_t)p.np * (uint32_t)p.P * 2u))
+                            mma_part(2, tm_p + (uint32_t)p.np, p.np, p.kb_p / 2, p.kb_p, false);
+                    }
+                } else if (warp == 1) {
+                    if (lane == 0 && res_p) mma_part(2, tm_p, p.np, 0, p.kb_p / 2, false);
+                } else {
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_START);
+                    int cnt = 0;
+                    for (int b = e; b < p.B; b += 256) cnt += t_new[b] < p.enc_len[b];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+                    if (lane == 0) s_red[warp - 2] = cnt;
+                    asm volatile("bar.sync 1, 256;" ::: "memory");
+                    if (e == 0) s_active = s_red[0] + s_red[1] + s_red[2] + s_red[3] + s_red[4] + s_red[5] + s_red[6] + s_red[7];
+                    if (res_p) epilogue_res_P();
+                }
+                early_res();
+            } else if (warp == 0) {
                 if (lane == 0) {
                     fence_proxy_async_all();
                     cur = 0;
@@ -588,7 +1172,25 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
             const int n_tile = p.nj;
             const uint32_t z_bytes = (uint32_t)n_tile * BK * 2;
             unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
-            if (warp == 0) {
+            if (RES && warp < 2) {
+                // one box for the whole z tile, then every MMA back to back (A = W_out tile in tensor memory)
+                if (lane == 0 && has_j) {
+                    if (warp == 0) {
+                        fence_proxy_async_all();
+                        if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_FIRST_ISSUE);
+                        for (int rg = j_first; rg < p.rg_count; rg += p.rg_stride) {
+                            const bool ok = produce_one(&M.z3, rg * n_tile, (uint32_t)n_tile * (uint32_t)p.H * 2u);
+                            if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_LAST_ISSUE);
+                            if (!ok || !mma_part(0, tm_j + (uint32_t)n_tile, n_tile, p.kb_h / 2, p.kb_h, true)) break;
+                        }
+                        if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_COMMIT);
+                    } else {
+                        for (int rg = j_first; rg < p.rg_count; rg += p.rg_stride)
+                            if (!mma_part(0, tm_j, n_tile, 0, p.kb_h / 2, true)) break;
+                        if constexpr (FULL) trace_event(p, 1, tr_n, step, TR_J, EV_COMMIT);
+                    }
+                }
+            } else if (!RES && warp == 0) {
                 if (lane == 0) {
                     fence_proxy_async_all();
                     cur = 0;
@@ -612,7 +1214,7 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
                     }
                     if constexpr (FULL) trace_event(p, 0, tr_n, step, TR_J, EV_LAST_ISSUE);
                 }
-            } else if (warp == 1) {
+            } else if (!RES && warp == 1) {
                 if (lane == 0) {
                     const uint32_t idesc = idesc_bf16(128, n_tile);
                     cur = 0;
@@ -647,12 +1249,105 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
             } else {
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_START);
                 const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
-                for (int i = cta; i < p.j_items; i += G) {
-                    const int rg = i / p.vt_count, vt = i - rg * p.vt_count;
+                for (int i = RES ? j_first : cta; i < (RES ? p.rg_count : p.j_items); i += RES ? p.rg_stride : G) {
+                    const int rg = RES ? i : i / p.vt_count, vt = RES ? my_vt : i - rg * p.vt_count;
+                    const int v = vt * 128 + row_in_tile;            // this thread's vocabulary entry
+                    const bool v_ok = v < p.NV;
+                    const float bias = v_ok ? p.b_out[v] : 0.f;
                     const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[0], acc_n[0] & 1u, &s_abort));
                     tc_fence_after();
                     if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_ACC);
-                    if (ready) joint_epilogue_item<false, FULL>(p, tm_j, lane_off, lane, q, 0, row_in_tile, rg, vt, n_tile, t_cur, keys_cur);
+                    if (ready) {
+                        for (int c0 = RES ? 32 * sub : 0; c0 < n_tile; c0 += RES ? 64 : 32) {
+                            float val[32];
+                            tmem_ld16(tm_j + lane_off + (uint32_t)c0, val);
+                            if (c0 + 16 < n_tile) {
+                                tmem_ld16(tm_j + lane_off + (uint32_t)(c0 + 16), val + 16);
+                            } else {
+#pragma unroll
+                                for (int j = 16; j < 32; ++j) val[j] = -INFINITY;
+                            }
+                            if (RES) {   // second accumulator copy (the other issuing thread's K blocks)
+                                float more[16];
+                                if (p.kb_h < 2) {   // a single K block: nothing was written to the first copy
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) val[j] = (j < 16 || c0 + 16 < n_tile) ? 0.f : val[j];
+                                }
+                                tmem_ld16(tm_j + lane_off + (uint32_t)(n_tile + c0), more);
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) val[j] += more[j];
+                                if (c0 + 16 < n_tile) {
+                                    tmem_ld16(tm_j + lane_off + (uint32_t)(n_tile + c0 + 16), more);
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) val[16 + j] += more[j];
+                                }
+                            }
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) val[j] = v_ok ? val[j] + bias : -INFINITY;
+                            const int row = rg * n_tile + c0 + lane;      // the window row whose result this lane ends up with
+                            if (FULL && p.logits_out) {
+                                // teacher-forced evaluation: store the logits of the rows inside the window
+                                bool row_ok = false;
+                                if (row < p.rows && c0 + lane < n_tile) {
+                                    const int b = row / p.W, w = row - b * p.W;
+                                    row_ok = t_cur[b] + w < p.enc_len[b];
+                                }
+                                const uint32_t okmask = __ballot_sync(0xffffffffu, row_ok);
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    if (((okmask >> j) & 1u) && v_ok)
+                                        p.logits_out[(size_t)(rg * n_tile + c0 + j) * p.NV + v] = val[j];
+                            } else {
+                                unsigned long long* key_dst = keys_cur;
+                                if (FULL && p.window) {
+                                    // window-based decoding: this warp's 32 vocabulary entries give, per row, a partial
+                                    // (maximum, sum of exponentials) for the row's log-sum-exp; the blank's logit is
+                                    // stored on its own and the blank leaves the maximum search
+                                    float tmp[32];
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) tmp[j] = val[j];
+                                    reduce_exchange<16, false>(tmp, lane);
+                                    reduce_exchange<8, false>(tmp, lane);
+                                    reduce_exchange<4, false>(tmp, lane);
+                                    reduce_exchange<2, false>(tmp, lane);
+                                    reduce_exchange<1, false>(tmp, lane);
+                                    const float m_keep = tmp[0];           // this lane's row: maximum over the warp's 32 entries
+#pragma unroll
+                                    for (int j = 0; j < 32; ++j) {
+                                        const float mj = __shfl_sync(0xffffffffu, m_keep, j);
+                                        tmp[j] = val[j] > -INFINITY ? __expf(val[j] - mj) : 0.f;
+                                    }
+                                    reduce_exchange<16, true>(tmp, lane);
+                                    reduce_exchange<8, true>(tmp, lane);
+                                    reduce_exchange<4, true>(tmp, lane);
+                                    reduce_exchange<2, true>(tmp, lane);
+                                    reduce_exchange<1, true>(tmp, lane);
+                                    const float s_keep = tmp[0];
+                                    if (row < p.rows && c0 + lane < n_tile)
+                                        p.jpart[(size_t)row * p.parts + vt * 4 + q] = make_float2(m_keep, s_keep);
+                                    if (v == p.blank) {
+#pragma unroll
+                                        for (int j = 0; j < 32; ++j) {
+                                            const int rj = rg * n_tile + c0 + j;
+                                            if (rj < p.rows && c0 + j < n_tile) p.jblank[rj] = val[j];
+                                            val[j] = -INFINITY;
+                                        }
+                                    }
+                                    key_dst = p.nbkeys;
+                                }
+                                int id[32];
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) id[j] = v;
+                                argmax_exchange<16>(val, id, lane);
+                                argmax_exchange<8>(val, id, lane);
+                                argmax_exchange<4>(val, id, lane);
+                                argmax_exchange<2>(val, id, lane);
+                                argmax_exchange<1>(val, id, lane);
+                                if (row < p.rows && c0 + lane < n_tile && val[0] > -INFINITY)
+                                    atomicMax(&key_dst[row], pack_key(val[0], (uint32_t)id[0]));
+                            }
+                        }
+                    }
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&acc_empty[0]);
@@ -671,10 +1366,76 @@ __global__ void __launch_bounds__(LOOP_THREADS, 1) loop_kernel(const __grid_cons
             // reads (the chosen row carries its label, every other row the blank)
             // =================================================================================
             if (warp >= 2) {
+                constexpr int n_ew = RES ? 8 : 4;
+                const int ew = warp - 2;
                 const int32_t* t_cur = p.t2 + (size_t)(step & 1) * p.B;
                 unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
+                const unsigned long long blank_key = pack_key(0.f, (uint32_t)p.blank);
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_START);
-                window_decision<4>(p, cta, G, warp - 2, lane, t_cur, keys_cur, win_lpb, win_sc, win_key);
+                // one utterance per CTA at a time; each epilogue warp takes the rows ew, ew + n_ew, ... of its window
+                for (int b = cta; b < p.B; b += G) {
+                    int t = 0, len = 0;
+                    if (ew == 0) { t = t_cur[b]; len = p.enc_len[b]; }
+                    for (int j = ew; j < p.W; j += n_ew) {
+                        const size_t row = (size_t)b * p.W + j;
+                        float bl = 0.f;
+                        unsigned long long key = 0ull;
+                        if (lane == 0) { bl = p.jblank[row]; key = p.nbkeys[row]; }
+                        // the row's log-sum-exp from its partial (maximum, sum) pairs, spread over the lanes
+                        float m = -INFINITY, sm = 0.f;
+                        for (int k = lane; k < p.parts; k += 32) {
+                            const float2 pr = p.jpart[row * p.parts + k];
+                            if (pr.y > 0.f) {
+                                if (pr.x > m) { sm = sm * __expf(m - pr.x) + pr.y; m = pr.x; }
+                                else sm += pr.y * __expf(pr.x - m);
+                            }
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, sm, o);
+                            const float mx = fmaxf(m, om);
+                            const float a = sm > 0.f ? sm * __expf(m - mx) : 0.f;
+                            const float c = os > 0.f ? os * __expf(om - mx) : 0.f;
+                            m = mx; sm = a + c;
+                        }
+                        if (lane == 0) {
+                            const float lse = m + __logf(sm);
+                            win_lpb[j] = bl - lse;
+                            win_sc[j] = key != 0ull ? key_logit(key) - lse : -INFINITY;
+                            win_key[j] = key;
+                            p.nbkeys[row] = 0ull;
+                        }
+                    }
+                    asm volatile("bar.sync 1, %0;" ::"n"(n_ew * 32) : "memory");
+                    if (ew == 0) {
+                        const int n = t < len ? min(p.W, len - t) : 0;
+                        // lane j looks at rows j and j + 32: blank log-probabilities of the rows before each row
+                        float lpb0 = lane < n ? win_lpb[lane] : 0.f, lpb1 = lane + 32 < n ? win_lpb[lane + 32] : 0.f;
+                        float sc0 = lane < n ? win_sc[lane] : -INFINITY, sc1 = lane + 32 < n ? win_sc[lane + 32] : -INFINITY;
+                        float incl0 = lpb0, incl1 = lpb1;
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const float a0 = __shfl_up_sync(0xffffffffu, incl0, o), a1 = __shfl_up_sync(0xffffffffu, incl1, o);
+                            if (lane >= o) { incl0 += a0; incl1 += a1; }
+                        }
+                        const float tot0 = __shfl_sync(0xffffffffu, incl0, 31), tot1 = __shfl_sync(0xffffffffu, incl1, 31);
+                        sc0 += incl0 - lpb0;
+                        sc1 += tot0 + incl1 - lpb1;
+                        // first strict maximum in row order; "all blank" (tot0 + tot1) wins only when strictly larger
+                        float top = sc0;
+                        int pick = lane;
+                        if (sc1 > top) { top = sc1; pick = lane + 32; }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const float ot = __shfl_xor_sync(0xffffffffu, top, o);
+                            const int op = __shfl_xor_sync(0xffffffffu, pick, o);
+                            if (ot > top || (ot == top && op < pick)) { top = ot; pick = op; }
+                        }
+                        if (!(top > -INFINITY) || tot0 + tot1 > top) pick = -1;
+                        for (int j = lane; j < n; j += 32) keys_cur[(size_t)b * p.W + j] = j == pick ? win_key[j] : blank_key;
+                    }
+                    if (b + G < p.B) asm volatile("bar.sync 1, %0;" ::"n"(n_ew * 32) : "memory");   // the arrays are reused
+                }
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_EPI_DONE);
             }
             if (!grid_sync(TR_J)) goto done;
@@ -705,6 +1466,7 @@ done:
     }
 }
 
+
 // ---------------------------------------------------------------------------
 // host side: tile plan, tensor maps, launch
 // ---------------------------------------------------------------------------
@@ -714,7 +1476,7 @@ static int g_sm_count[64] = {};
 static int g_smem_optin[64] = {};
 static int g_attr_smem[64] = {};       // opt-in shared memory already granted to the streaming kernel, per device
 static int g_loop_extra_arrivals = 0;
-static LoopOptions g_loop_options = {1, -1, 4};
+static LoopOptions g_loop_options = {1, -1, 4, -1};
 int loop_set_extra_arrivals(int n) { int prev = g_loop_extra_arrivals; g_loop_extra_arrivals = n > 0 ? n : 0; return prev; }
 void loop_set_options(const LoopOptions& o) { g_loop_options = o; }
 LoopOptions loop_get_options() { return g_loop_options; }
@@ -864,7 +1626,7 @@ cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem
     bool resident_done = false;
     for (int ci = 0; ci < n_cands && !resident_done; ++ci) {
         const int r_nj = cands[ci];
-        if (!(m.L <= 2 && m.H / 2 + 2 * r_nj <= (int)LOOP_TMEM_COLS && opt.resident != 0 && NV <= (1 << 20))) continue;   // (labels take 20 bits of a key slot)
+        if (!(m.L <= 2 && m.H / 2 + 2 * r_nj <= (int)LOOP_TMEM_COLS && opt.resident != 0)) continue;
         LoopPlan r = pl;
         r.nj = r_nj;
         r.rg_count = (rows + r_nj - 1) / r_nj;
@@ -886,10 +1648,35 @@ cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem
             if (found) break;
         }
         if (!found) continue;
+        // Which resident kernel: the one with grid barriers between the phases, or the one in which CTAs hand their
+        // results on through arrival counters and stamped data.  Measured on B200: the second is ahead while a lock step
+        // is mostly latency (config 3's model with 1 / 16 / 64 utterances: 12.1 / 13.4 / 14.8 against 13.2 / 13.9 / 15.4 us per
+        // lock step), the first once every CTA has work in every phase (128 utterances: 16.7 against 17.6 us).
+        r.dataflow = opt.dataflow >= 0 ? (opt.dataflow != 0) : (B <= (m.L == 1 ? kDataflowMaxBatch : kDataflowMaxBatch2));
+        if (NV > (1 << 20)) r.dataflow = 0;    // labels take 20 bits of a stamped key slot
+        auto up = [](uint32_t x) { return (x + 1023u) / 1024u * 1024u; };
+        if (!r.dataflow) {
+            // shared memory of a CTA: [weight tile][operand buffer][epilogue staging]; the buffer holds the step's one
+            // operand box (the joint's z rows, or the state rows) and, in CTAs with a W_pred tile, behind the state box
+            // the prefetched enc_proj rows of their first 256 z rows
+            const uint32_t staging = r.np > 64 ? (uint32_t)r.np * 68u * 4u : 17408u;
+            const uint32_t tile = (uint32_t)r.kb_p * 64u * BK * 2u;
+            uint32_t buf = (uint32_t)r.nj * (uint32_t)m.H * 2u;
+            if ((uint32_t)r.nl * m.P * 2u > buf) buf = (uint32_t)r.nl * m.P * 2u;
+            const uint32_t stash_rows = (uint32_t)(r.np * W < 256 ? r.np * W : 256);
+            if ((uint32_t)r.np * m.P * 2u + stash_rows * 128u > buf) buf = (uint32_t)r.np * m.P * 2u + stash_rows * 128u;
+            buf = up(buf);
+            r.resident = 1;
+            r.j_mode = J_TMEM;
+            r.stat_bytes = tile;
+            r.buf_off = tile;
+            r.z_off = r.z_off_p = tile;
+            r.stage_off = tile + buf;
+            r.smem_bytes = tile + buf + staging + 1024;
+        } else {
         // shared memory of a CTA: [weight tile][state box | joint operand][epilogue staging].  The joint's operand
         // (nj rows x H) shares the state box's memory where a CTA needs both; the CTAs with a W_pred tile (smaller box)
         // get an operand buffer of their own when it fits, so that they can start on the next window a slot earlier.
-        auto up = [](uint32_t x) { return (x + 1023u) / 1024u * 1024u; };
         // epilogue staging: 64 utterances x 4 gates x 16 units (+ their tokens) in the decoder slot, np utterances x
         // (64 + 4 padding) pred_proj values in the projection slot
         const uint32_t staging = r.np > 64 ? (uint32_t)r.np * 68u * 4u : 17408u;
@@ -908,6 +1695,7 @@ cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem
         r.z_off_p = own ? tile + box_p : tile;
         r.stage_off = end_l > end_p ? end_l : end_p;
         r.smem_bytes = r.stage_off + staging + 1024;
+        }
         r.stages_lp = r.stages_j = 1;
         r.stage_lp = r.stage_j = 0;
         r.tm_j = m.H / 2;
@@ -969,6 +1757,7 @@ cudaError_t loop_prepare(Call& c) {
             if (m.L == 2) WIND_MAP(loop_map3(&M.hb_l3_1[par], c.hb(par, 1), c.lay.Bpad, m.P, pl.nl));
             WIND_MAP(loop_map3(&M.hb_p3[par], c.hb(par, m.L - 1), c.lay.Bpad, m.P, pl.np));
         }
+        if (!pl.dataflow) WIND_MAP(loop_map3(&M.z3, c.z(), (uint64_t)c.lay.rows_pad, m.H, pl.nj));
     } else {
         WIND_MAP(loop_map(&M.w_out, m.w_out, (uint64_t)m.V + 1, m.H, 128));
         WIND_MAP(loop_map(&M.z, c.z(), (uint64_t)c.lay.rows_pad, m.H, pl.nj));
@@ -980,12 +1769,13 @@ cudaError_t loop_prepare(Call& c) {
         }
     }
 #undef WIND_MAP
-    if (pl.resident) return loop_res_set_smem((int)pl.smem_bytes);
+    if (pl.resident && pl.dataflow) return loop_res_set_smem((int)pl.smem_bytes);
     int sms = 0, optin = 0, dev = 0;
     if ((e = loop_device_info(&sms, &optin, &dev)) != cudaSuccess) return e;
     std::lock_guard<std::mutex> lock(g_loop_mutex);
     if ((int)pl.smem_bytes > g_attr_smem[dev]) {
-        for (const void* fn : {(const void*)loop_kernel<false>, (const void*)loop_kernel<true>}) {
+        for (const void* fn : {(const void*)loop_kernel<false, false>, (const void*)loop_kernel<false, true>,
+                               (const void*)loop_kernel<true, false>, (const void*)loop_kernel<true, true>}) {
             e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes);
             if (e != cudaSuccess) return e;
         }
@@ -1028,10 +1818,12 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.nbkeys = c.keys() + 2 * (size_t)c.lay.rows_pad; p.jpart = c.jpart(); p.jblank = c.jblank(); p.parts = 4 * pl.vt_count;
     p.flags = c.flags(); p.pred_pub = c.pred_pub(); p.kslot = c.kslot();
     const bool full = p.forced || p.window || p.trace;
-    if (pl.resident) return loop_res_launch(t_loop_maps, p, pl.grid, pl.smem_bytes, full, c.stream);
+    if (pl.resident && pl.dataflow) return loop_res_launch(t_loop_maps, p, pl.grid, pl.smem_bytes, full, c.stream);
     void* args[2] = {(void*)&t_loop_maps, (void*)&p};
-    const void* fn = full ? (const void*)loop_kernel<true> : (const void*)loop_kernel<false>;
-    return cudaLaunchCooperativeKernel(fn, dim3((unsigned)pl.grid), dim3(LOOP_THREADS), args, pl.smem_bytes, c.stream);
+    const void* fn = pl.resident ? (full ? (const void*)loop_kernel<true, true> : (const void*)loop_kernel<true, false>)
+                                 : (full ? (const void*)loop_kernel<false, true> : (const void*)loop_kernel<false, false>);
+    return cudaLaunchCooperativeKernel(fn, dim3((unsigned)pl.grid), dim3(pl.resident ? LOOP_THREADS_RES : LOOP_THREADS), args, pl.smem_bytes,
+                                       c.stream);
 }
 
 }  // namespace wind

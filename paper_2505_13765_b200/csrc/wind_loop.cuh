@@ -25,6 +25,7 @@ struct LoopMaps {
     CUtensorMap hb_l3[2];              // layer 0 state [Bpad, P] as (64, rows, P/64), box (64, nl, P/64)
     CUtensorMap hb_l3_1[2];            // layer 1 state, same box
     CUtensorMap hb_p3[2];              // same, box (64, np, P/64)
+    CUtensorMap z3;                    // [rows_pad, H] as (64, rows, H/64), box (64, nj, H/64) (resident kernel with grid barriers)
 };
 
 // How the three phases are cut into items and how shared memory is used (host-chosen).
@@ -40,6 +41,7 @@ struct LoopPlan {
     // resident-weights mode: W_hh tiles (4 gates x 16 units) and W_pred tiles (64 rows) stay in the shared memory of
     // disjoint CTA sets; accumulators are [64 weight rows, nl or np utterances]
     int resident, nl, ut_count, ht_count, ql_count, qp_count;
+    int dataflow;                          // resident mode: the kernel without grid barriers (wind_loop_res.cu)
     int w_first, w_count;                  // step-recording CTAs [w_first, w_first + w_count), 64 utterances each (0: the L CTAs record)
     uint32_t buf_off, stage_off;           // the per-step operand buffer and the epilogue staging area (after the tile)
     uint32_t z_off, z_off_p;               // resident mode: the joint's operand buffer (z_off_p: in CTAs with a W_pred tile);
@@ -108,8 +110,9 @@ struct LoopParams {
 
 // Options of the tile planner (process-wide; wind_set_loop_options): whether the resident-weights mode may be chosen,
 // a forced placement of the streaming mode's W_out tile (-1: the planner's own choice; 0 streamed, 1 shared memory,
-// 2 tensor memory, taken when feasible), and the most waves the resident joint may run in (1..4).
-struct LoopOptions { int resident; int joint_placement; int max_joint_waves; };
+// 2 tensor memory, taken when feasible), the most waves the resident joint may run in (1..4), and which resident kernel
+// (-1: the planner's choice by batch size; 0 the one with grid barriers; 1 the one with arrival counters).
+struct LoopOptions { int resident; int joint_placement; int max_joint_waves; int dataflow; };
 void loop_set_options(const LoopOptions& o);
 LoopOptions loop_get_options();
 bool loop_plan_ok(const wind_model_t& m, int B, int W);

@@ -70,6 +70,20 @@ __device__ __forceinline__ void tc_mma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a,
 
 enum { J_STREAM = 0, J_SMEM = 1, J_TMEM = 2 };   // where the joint's W_out tile lives
 
+// z = act(e + g) on two bf16 pairs at once: one rounding for the sum (fused multiply-add with 1), then ReLU or tanh
+__device__ __forceinline__ uint32_t act_add_bf16x2(uint32_t e, uint32_t g, int act) {
+    const __nv_bfloat162 one = __floats2bfloat162_rn(1.f, 1.f);
+    __nv_bfloat162 s = __hfma2(*reinterpret_cast<const __nv_bfloat162*>(&e), one, *reinterpret_cast<const __nv_bfloat162*>(&g));
+    uint32_t r;
+    if (act == WIND_ACT_RELU) {
+        s = __hmax2(s, __floats2bfloat162_rn(0.f, 0.f));
+        r = *reinterpret_cast<uint32_t*>(&s);
+    } else {
+        asm("tanh.approx.bf16x2 %0, %1;" : "=r"(r) : "r"(*reinterpret_cast<uint32_t*>(&s)));
+    }
+    return r;
+}
+
 // One stage of the exchange that turns "every lane holds 2*HALF columns" into "every lane holds HALF
 // columns, reduced over lane pairs": lanes with bit HALF set keep the upper columns.
 template <int HALF>

@@ -61,20 +61,6 @@ __device__ __forceinline__ void st_relaxed_v2_u64(unsigned long long* p, unsigne
 __device__ __forceinline__ unsigned long long stamped(float lo, float hi, uint32_t stamp) {
     return ((unsigned long long)stamp << 32) | (unsigned long long)pack_bf16x2(lo, hi);
 }
-// z = act(e + g) on two bf16 pairs at once: one rounding for the sum (fused multiply-add with 1), then ReLU or tanh
-__device__ __forceinline__ uint32_t act_add_bf16x2(uint32_t e, uint32_t g, int act) {
-    const __nv_bfloat162 one = __floats2bfloat162_rn(1.f, 1.f);
-    __nv_bfloat162 s = __hfma2(*reinterpret_cast<const __nv_bfloat162*>(&e), one, *reinterpret_cast<const __nv_bfloat162*>(&g));
-    uint32_t r;
-    if (act == WIND_ACT_RELU) {
-        s = __hmax2(s, __floats2bfloat162_rn(0.f, 0.f));
-        r = *reinterpret_cast<uint32_t*>(&s);
-    } else {
-        asm("tanh.approx.bf16x2 %0, %1;" : "=r"(r) : "r"(*reinterpret_cast<uint32_t*>(&s)));
-    }
-    return r;
-}
-
 template <bool FULL>
 __global__ void __launch_bounds__(LOOP_THREADS_RES, 1) loop_res_kernel(const __grid_constant__ LoopMaps M, const LoopParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -1158,6 +1144,10 @@ cudaError_t loop_res_set_smem(int bytes) {
 }
 
 cudaError_t loop_res_launch(const LoopMaps& maps, const LoopParams& p, int grid, uint32_t smem_bytes, bool full, cudaStream_t stream) {
+    // every array the kernel writes through must be there: a missing one is a host-side mistake, not something to find on the device
+    if (!p.ctrl || !p.flags || !p.pred_pub || !p.kslot || !p.t_pub || !p.t2 || !p.hb || !p.c_state || !p.enc_proj || !p.g0 || !p.keys2 ||
+        (p.L == 2 && (!p.dh || !p.emit_tok)))
+        return cudaErrorInvalidValue;
     void* args[2] = {(void*)&maps, (void*)&p};
     const void* fn = full ? (const void*)loop_res_kernel<true> : (const void*)loop_res_kernel<false>;
     return cudaLaunchCooperativeKernel(fn, dim3((unsigned)grid), dim3(LOOP_THREADS_RES), args, smem_bytes, stream);

@@ -19,3 +19,19 @@ def _restore_loop_options():
     from paper_2505_13765_b200 import binding
     if binding._lib is not None:
         binding.wind_set_loop_options()
+
+
+LOOP_MODES = ["barriers", "counters", "streaming"]
+
+
+def set_loop_mode(pkg, mode: str) -> None:
+    """The three modes of the tensor-core loop: resident weights with grid barriers between the phases, resident weights
+    with arrival counters and stamped data (no grid barrier), weights streamed through shared memory every step."""
+    if mode == "barriers":
+        pkg.wind_set_loop_options(resident=True, dataflow=0)
+    elif mode == "counters":
+        pkg.wind_set_loop_options(resident=True, dataflow=1)
+    elif mode == "streaming":
+        pkg.wind_set_loop_options(resident=False)
+    else:
+        raise ValueError(mode)

@@ -7,6 +7,8 @@ import sys
 
 import numpy as np
 import pytest
+
+from conftest import LOOP_MODES, set_loop_mode
 import torch
 
 sys.path.insert(0, os.path.join(os.path.dirname(__file__), ".."))
@@ -37,11 +39,12 @@ def test_small_dimensions_many_utterances(pkg, monkeypatch, seed):
         V = int(r.integers(127, 700)); B = int(r.choice([1, 2, 7, 31, 64, 65, 128, 129, 200, 333]))
         W = int(r.choice([1, 2, 3, 5, 8, 13, 16, 24, 40])); L = int(r.choice([1, 1, 2, 2, 3])); S = int(r.integers(1, 6))
         act = int(r.integers(0, 2)); blank0 = bool(r.integers(0, 2)); res = int(r.integers(0, 2)); T = int(r.integers(8, 40))
+        mode = LOOP_MODES[(2 * res + i) % 3]
         win = bool(r.integers(0, 3) == 0)
-        pkg.wind_set_loop_options(resident=bool(res))
+        set_loop_mode(pkg, mode)
         w, enc, lens = tp.ragged_case(9000 + i, B=B, T=T, D=64, E=int(r.choice([64, 128])), P=P, L=L, H=H, V=V, act=act,
                                       blank_id=0 if blank0 else None, bias=float(r.uniform(0.5, 3.0)), dtype="bf16")
-        print(f"case {i}: B={B} T={T} W={W} S={S} P={P} H={H} V={V} L={L} resident={res} window={win}", flush=True)
+        print(f"case {i}: B={B} T={T} W={W} S={S} P={P} H={H} V={V} L={L} mode={mode} window={win}", flush=True)
         if win:
             tw.check_window_greedy(pkg, w, enc, lens, W, S, kernels=2)
         else:
@@ -56,10 +59,11 @@ def test_large_dimensions(pkg, monkeypatch):
         W = int(r.choice([1, 2, 4, 8, 16, 32, 64])); L = int(r.choice([1, 2])); S = int(r.integers(1, 11)); act = int(r.integers(0, 2))
         res = int(r.integers(0, 2)); T = int(r.integers(4, 16)); kind = int(r.integers(0, 4)); D = int(r.choice([64, 512]))
         E = int(r.choice([64, 640]))
-        pkg.wind_set_loop_options(resident=bool(res))
+        mode = LOOP_MODES[(2 * res + i) % 3]
+        set_loop_mode(pkg, mode)
         w, enc, lens = tp.ragged_case(9500 + i, B=B, T=T, D=D, E=E, P=P, L=L, H=H, V=V, act=act, blank_id=0 if i % 3 == 0 else None,
                                       bias=float(r.uniform(0.5, 3.0)), dtype="bf16")
-        print(f"case {i}: kind={kind} B={B} T={T} W={W} S={S} D={D} E={E} P={P} H={H} V={V} L={L} resident={res}", flush=True)
+        print(f"case {i}: kind={kind} B={B} T={T} W={W} S={S} D={D} E={E} P={P} H={H} V={V} L={L} mode={mode}", flush=True)
         if kind == 0:
             tw.check_window_greedy(pkg, w, enc, lens, W, S, kernels=2)
         elif kind == 1:

@@ -14,6 +14,7 @@ import pytest
 
 import oracle
 import wind_synth as ws
+from conftest import LOOP_MODES, set_loop_mode
 from naive_model import random_weights, tie_expected, tie_model, tie_utterances
 
 torch = pytest.importorskip("torch")
@@ -281,12 +282,11 @@ def test_bf16_tensor_path_with_biases_and_other_blank_ids(pkg, L, blank0, act, B
     logits_parity(pkg, w, enc, lens, W=W, S=4, tol=TOL["bf16"], n_windows=2 * B, kernels=2)
 
 
-@pytest.mark.parametrize("resident", [1, 0])
-def test_bf16_tensor_path_more_utterances_than_one_tile(pkg, monkeypatch, resident):
+@pytest.mark.parametrize("mode", LOOP_MODES)
+def test_bf16_tensor_path_more_utterances_than_one_tile(pkg, mode):
     # 150 utterances, one K block per GEMM (H = P = 64): ten utterance groups per weight tile in the resident-weights
     # mode; two 128-row utterance tiles in the streaming mode (forced through wind_set_loop_options)
-    if not resident:
-        pkg.wind_set_loop_options(resident=False)
+    set_loop_mode(pkg, mode)
     w, enc, lens = ragged_case(91, B=150, T=24, D=64, E=64, P=64, L=1, H=64, V=140, act=0, bias=1.0, dtype="bf16")
     rep, _ = check_against_oracle(pkg, w, enc, lens, 4, 3, kernels=2)
     assert rep["stats"]["kernels"] == 2
@@ -307,12 +307,11 @@ def test_bf16_tensor_path_more_utterances_than_one_tile(pkg, monkeypatch, reside
     (100, 8, 2, 128, 128, 2100, 2),    # two layers, 17 vocabulary tiles, two waves
     (90, 16, 3, 64, 128, 3000, 1),     # 24 tiles, six CTAs per tile, three waves of 96-row groups
 ])
-@pytest.mark.parametrize("resident", [1, 0])
-def test_bf16_tensor_path_shape_sweep(pkg, monkeypatch, resident, B, W, S, P, H, V, L):
+@pytest.mark.parametrize("mode", LOOP_MODES)
+def test_bf16_tensor_path_shape_sweep(pkg, mode, B, W, S, P, H, V, L):
     # shapes that send the tile planner of the loop kernel down its different branches, with the resident-weights
     # mode allowed and with wind_set_loop_options forcing the streaming mode
-    if not resident:
-        pkg.wind_set_loop_options(resident=False)
+    set_loop_mode(pkg, mode)
     w, enc, lens = ragged_case(300 + B + W, B=B, T=20, D=64, E=64, P=P, L=L, H=H, V=V, act=B % 2, bias=1.5,
                                dtype="bf16")
     rep, _ = check_against_oracle(pkg, w, enc, lens, W, S, kernels=2)
@@ -395,19 +394,44 @@ def test_bf16_tensor_path_is_window_invariant_on_the_gpu(pkg):
             assert np.array_equal(tok, ref[0]) and np.array_equal(frm, ref[1]), W
 
 
+@pytest.mark.parametrize("case", ["large_model_w8", "two_layers_tanh_w3", "many_utterances_w1"])
+def test_the_two_resident_kernels_give_the_same_transcripts(pkg, case):
+    # The planner picks the resident kernel by batch size; an utterance's transcript must not depend on that choice
+    # (nor, therefore, on how many utterances share its batch): same arithmetic in both, bit for bit.
+    if case == "large_model_w8":
+        cfg = ws.small_variant(ws.CONFIGS["cfg3_large_b128"], 12, 5, 140)
+        w, (enc, lens), W, S = ws.make_model(cfg), ws.make_enc(cfg, pad="zero"), 8, cfg.S
+    elif case == "two_layers_tanh_w3":
+        w, enc, lens = ragged_case(501, B=20, T=40, D=64, E=64, P=128, L=2, H=192, V=300, act=1, bias=1.0, dtype="bf16")
+        enc, W, S = np.nan_to_num(enc), 3, 4
+    else:
+        w, enc, lens = ragged_case(502, B=150, T=24, D=64, E=64, P=64, L=1, H=64, V=140, act=0, bias=1.0, dtype="bf16")
+        enc, W, S = np.nan_to_num(enc), 1, 3
+    model = pkg.WindModel(w)
+    outs = {}
+    for mode in ("barriers", "counters"):
+        set_loop_mode(pkg, mode)
+        tok, frm, olen, stats, st = pkg.decode(model, enc, lens, W, S)
+        assert st == 0 and stats["kernels"] == 2
+        outs[mode] = (tok, frm, olen, stats["steps"])
+    for a, b in zip(outs["barriers"][:3], outs["counters"][:3]):
+        assert np.array_equal(a, b)
+    assert outs["barriers"][3] == outs["counters"][3]
+
+
 TIE_UTTS = [[5, 0, 5, 5, 1, 2, 3, 4, 5, 6, 7, 8, 5], [8, 7, 6, 5, 5, 5, 5, 5, 5, 5, 4, 3, 2, 1, 0], [3], [5, 5, 4],
             [2, 2, 3, 3, 4, 4, 8, 8], [], [0, 1, 2, 3, 4, 5, 6, 7, 8] * 3]
 
 
-@pytest.mark.parametrize("path", ["f32", "bf16_simt", "bf16_tensor", "bf16_tensor_streaming"])
+@pytest.mark.parametrize("path", ["f32", "bf16_simt", "bf16_tensor_barriers", "bf16_tensor_counters", "bf16_tensor_streaming"])
 @pytest.mark.parametrize("blank_first", [False, True])
 def test_argmax_ties_go_to_the_lowest_index_on_the_gpu(pkg, monkeypatch, path, blank_first):
     # Logits with exact ties by construction: two labels in one group of 32 vocabulary entries (one warp of the
     # tensor path's epilogue), in different groups of one 128-entry tile, in different tiles (combined through the
     # 64-bit keys), a label against the blank, and every entry equal.  The expected transcripts are written from the
     # rule (lowest index wins), and the oracle must give the same.
-    if path == "bf16_tensor_streaming":
-        pkg.wind_set_loop_options(resident=False)
+    if path.startswith("bf16_tensor_"):
+        set_loop_mode(pkg, path[len("bf16_tensor_"):])
     w, target, winners = tie_model(blank_id=0 if blank_first else None, dtype="f32" if path == "f32" else "bf16")
     blank = w["blank_id"]
     enc, lens = tie_utterances(w["D"], TIE_UTTS)
@@ -428,7 +452,9 @@ def test_argmax_ties_go_to_the_lowest_index_on_the_gpu(pkg, monkeypatch, path, b
         pkg.wind_set_kernels(prev)
 
 
-def test_loop_kernel_timeline_can_be_recorded_without_changing_results(pkg):
+@pytest.mark.parametrize("mode", ["barriers", "counters"])
+def test_loop_kernel_timeline_can_be_recorded_without_changing_results(pkg, mode):
+    set_loop_mode(pkg, mode)
     cfg = ws.small_variant(ws.CONFIGS["cfg3_large_b128"], 8, 30, 80)
     weights = ws.make_model(cfg)
     enc, lens = ws.make_enc(cfg, pad="zero")
@@ -532,10 +558,12 @@ def test_host_buffer_entry_point_matches_device_entry_point(pkg):
     assert pkg.wind_decode_greedy_host(model, enc_h2, bad, 8, cfg.S, tok_h, frm_h, ol_h, wsb, check=False) == pkg.binding.WIND_ERR_INVALID_ARG
 
 
-def test_unfillable_barrier_ends_in_timeout_status_and_the_context_stays_usable(pkg):
+@pytest.mark.parametrize("mode", ["barriers", "counters"])
+def test_unfillable_barrier_ends_in_timeout_status_and_the_context_stays_usable(pkg, mode):
     # Failure path of the persistent kernel without hanging anything: every wait in it is bounded, so a grid
     # barrier that can never fill (test hook) makes the CTAs give up after about two seconds and the call return
     # WIND_ERR_TIMEOUT; the next decode on the same context works and gives the usual result.
+    set_loop_mode(pkg, mode)
     cfg = ws.small_variant(ws.CONFIGS["cfg3_large_b128"], 4, 10, 40)
     weights = ws.make_model(cfg)
     enc, lens = ws.make_enc(cfg, pad="zero")

@@ -7,6 +7,8 @@ from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
 import pytest
+
+from conftest import LOOP_MODES, set_loop_mode
 import torch
 
 sys.path.insert(0, os.path.join(os.path.dirname(__file__), ".."))
@@ -146,11 +148,10 @@ def test_cfg3_full_batch_sampled_utterances(pkg):
     print("[window-greedy cfg3]", [(b, int(lens[b]), r["decisions"], r["not_argmax"]) for b, r in zip(sample, reps)])
 
 
-@pytest.mark.parametrize("resident", [1, 0])
-def test_bf16_tensor_path_wide_window_and_overflow(pkg, monkeypatch, resident):
+@pytest.mark.parametrize("mode", LOOP_MODES)
+def test_bf16_tensor_path_wide_window_and_overflow(pkg, mode):
     # W = 40: more window rows than lanes in the decision warp; then an output buffer that is too small
-    if not resident:
-        pkg.wind_set_loop_options(resident=False)
+    set_loop_mode(pkg, mode)
     w, enc, lens = ragged_case(540, B=6, T=70, D=64, E=64, P=64, L=1, H=128, V=150, act=1, bias=3.0, dtype="bf16")
     rep, (tok, frm, olen) = check_window_greedy(pkg, w, enc, lens, 40, 2, kernels=2)
     assert rep["stats"]["kernels"] == 2 and olen.max() > 4
