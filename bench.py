@@ -141,32 +141,36 @@ def aggregate_rtfx(audio_seconds_per_rank_step: float, steps: int, ms_local: flo
 # ---------------------------------------------------------------------------
 # CPU baseline: the oracle as it stands, on a bounded sample of the workload
 # ---------------------------------------------------------------------------
-def oracle_sample(cfg, enc, lens, seconds_target: float, cores: int):
-    """First k utterances (batch order) whose estimated oracle cost is about `seconds_target`."""
-    macs_per_row = cfg.H * (cfg.V + 1)
-    est_rate = 0.6e9 * cores  # fp64 MAC/s, rough
-    budget = seconds_target * est_rate
-    # rows per frame at window W on this generator: about (tokens per frame) * min(W, a few) + 1
-    rows_per_frame = 3.0 * min(cfg.W, 8) * 0.6 + 1.0
-    acc, k = 0.0, 0
-    while k < len(lens) and (k < 1 or acc + lens[k] * rows_per_frame * macs_per_row <= budget):
-        acc += lens[k] * rows_per_frame * macs_per_row
-        k += 1
-    return k
+def oracle_sample(cfg, lens, W, seconds_target: float, cores: int):
+    """The bounded sample both CPU legs time: the first k utterances, each cut to its first F frames.
+
+    The oracle runs one thread per utterance (OpenMP over utterances only), so k = min(cores, B) keeps every core busy
+    and the run lasts as long as its costliest utterance: F is chosen so that this is about `seconds_target` at a rough
+    0.5e9 fp64 multiply-adds per second and core.  Cost per frame on this generator: about 2.8 tokens (one decoder update
+    and one more window each) plus one window, a window being up to min(W, frames left) joint rows.
+    """
+    k = max(1, min(cores, len(lens)))
+    rows_per_frame = (2.8 + 1.0) * min(W, 4)            # jumps are short on this data: windows overlap heavily
+    lstm = sum(((cfg.E if l == 0 else cfg.P) + cfg.P) * 4 * cfg.P for l in range(cfg.L)) + cfg.P * cfg.H
+    macs_per_frame = cfg.D * cfg.H + rows_per_frame * cfg.H * (cfg.V + 1) + 2.8 * lstm
+    frames = int(max(8, seconds_target * 0.5e9 / macs_per_frame))
+    return k, frames
 
 
 def run_cpu_baseline(cfg, weights, enc, lens, W, seconds_target=15.0):
     import oracle
     cores = os.cpu_count() or 1
-    k = oracle_sample(cfg, enc, lens, seconds_target, cores)
+    k, frames = oracle_sample(cfg, lens, W, seconds_target, cores)
     om = oracle.Model(weights)
-    sub = np.ascontiguousarray(enc[:k])
+    sub_lens = np.minimum(lens[:k], frames).astype(np.int32)
+    sub = np.ascontiguousarray(enc[:k, : int(sub_lens.max())])
     t0 = time.perf_counter()
-    _, _, on, st = oracle.decode_batch(om, sub, lens[:k], W=W, S=cfg.S)
+    _, _, on, st = oracle.decode_batch(om, sub, sub_lens, W=W, S=cfg.S)
     dt = time.perf_counter() - t0
-    audio = float(lens[:k].sum()) * FRAME_SECONDS
-    return dict(value=audio / dt, unit="audio-s/s", cores=cores, kind="oracle",
-                sample=f"first {k} of {cfg.B} utterances ({int(lens[:k].sum())} frames), W={W}, one run, {dt:.1f} s",
+    audio = float(sub_lens.sum()) * FRAME_SECONDS
+    return dict(value=audio / dt, unit="audio-s/s", cores=min(cores, k), kind="oracle",
+                sample=f"first {k} of {cfg.B} utterances, each cut to its first {frames} frames ({int(sub_lens.sum())} frames in all), "
+                       f"W={W}, one run, {dt:.1f} s",
                 seconds=dt, steps=st["steps"])
 
 
@@ -195,7 +199,7 @@ def main():
                     help="tensor-core loop: the planner's choice, or resident weights with grid barriers / with arrival counters, or streamed weights")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the W=1 comparison, e2e and per-kernel timing legs")
-    ap.add_argument("--op", default="decode", choices=["decode", "first_output", "window_greedy", "dataset", "beam"],
+    ap.add_argument("--op", default="decode", choices=["decode", "first_output", "window_greedy", "dataset", "beam", "joint"],
                     help="first_output: time wind_window_first_output (Eq. 1 on one window per utterance) instead of the decode; "
                          "window_greedy: time wind_decode_window_greedy on the whole workload; dataset: 4 x B utterances in "
                          "arrival-order batches against length-aware batches; beam: wind_beam_search on one utterance, beams 2..4")
@@ -219,6 +223,8 @@ def main():
         return dataset_op(args, cfg, W)
     if args.op == "beam":
         return beam_op(args, cfg, W)
+    if args.op == "joint":
+        return joint_op(args, cfg, W)
 
     import torch
     import paper_2505_13765_b200 as pkg
@@ -346,6 +352,38 @@ def main():
         dist.destroy_process_group()
 
 
+def joint_standalone(pkg, model, cfg, W, peaks, iters=1000):
+    """The loop kernel's joint phase by itself: `iters` passes back to back inside one launch, on fixed activations of
+    all B * W window rows (wind_bench_joint), timed with CUDA events.  Algorithmic flop: 2 H (V+1) per window row;
+    issued: what the tiles cover (vocabulary padded to 128, rows to the row-group size)."""
+    import torch
+    wsb = pkg.alloc_workspace(model, cfg.B, 1, W)
+    r = pkg.wind_bench_joint(model, cfg.B, W, iters, wsb, stream=torch.cuda.current_stream())
+    s_per_iter = r["ms"] * 1e-3 / r["iters"]
+    alg = 2.0 * cfg.H * (cfg.V + 1) * r["rows"] / s_per_iter / 1e12
+    issued = 2.0 * cfg.H * r["labels_issued"] * r["rows_issued"] / s_per_iter / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    return {"us_per_pass": s_per_iter * 1e6, "passes": r["iters"], "rows": r["rows"], "rows_issued": r["rows_issued"],
+            "labels_issued": r["labels_issued"], "ctas": r["ctas"], "kernel": "resident weights" if r["resident"] else "streamed weights",
+            "achieved": alg, "issued": issued, "frac": alg / peak, "issued_frac": issued / peak, "unit": "TFLOP/s", "peak": peak,
+            "peak_source": peaks["source"] + " sustained bf16"}
+
+
+def measured_traffic(cfg, W, frames):
+    """DRAM bytes of one launch of the loop kernel, from the ncu counters of a small capture of the same shapes
+    (the package's measured_traffic.json: bytes that do not grow with the workload, and bytes per encoder frame),
+    scaled by the frame count.  None when the shapes have no capture."""
+    path = os.path.join(ROOT, "paper_2505_13765_b200", "measured_traffic.json")
+    if not os.path.exists(path):
+        return None, None
+    with open(path) as f:
+        table = json.load(f)
+    ent = table.get(f"{cfg.name}:W{W}")
+    if not ent:
+        return None, None
+    return ent["fixed_bytes"] + ent["bytes_per_frame"] * frames, ent["source"]
+
+
 def roofline(pkg, model, cfg, W, enc_d, len_d, tok_d, frm_d, ol_d, wsb, stream, stats, peaks, lens_np):
     """Roofline entry for the dominant kernel.
 
@@ -380,14 +418,10 @@ def roofline(pkg, model, cfg, W, enc_d, len_d, tok_d, frm_d, ol_d, wsb, stream, 
         achieved = flop / dur_s / 1e12
         js = res["joint_ms"] * 1e-3
         dense = 2.0 * cfg.H * (cfg.V + 1) * cfg.B * W * stats["steps"]
-        # DRAM bytes per launch: ncu counters (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of this
-        # kernel on the same shapes with 18975 frames (profiles/loop_kernel_cfg3_b128_short.md): 37.0 MB, of which
-        # the enc_proj rows (2 H bytes per frame, each read once) grow with the workload and 12.8 MB (weights, gate
-        # table, outputs) do not.  Scaled by the frame count; other shapes have no capture.
-        traffic, traffic_source = None, None
-        if (cfg.name, W, cfg.B) == ("cfg3_large_b128", 8, 128):
-            traffic = 12.8e6 + 2.0 * cfg.H * frames
-            traffic_source = "ncu capture at 18975 frames, enc_proj part scaled by frames"
+        # DRAM bytes per launch: ncu counters of a small capture of the same shapes, scaled by the frame count (the
+        # enc_proj rows, each read once, grow with the workload; weights, gate-table rows and outputs do not)
+        traffic, traffic_source = measured_traffic(cfg, W, frames)
+        standalone = joint_standalone(pkg, model, cfg, W, peaks)
         return {"kernel": "decoding loop (one persistent launch: joint, decoder-update and projection phases)",
                 "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                 "peak_source": peaks["source"] + " sustained bf16", "traffic": traffic, "traffic_source": traffic_source,
@@ -395,6 +429,7 @@ def roofline(pkg, model, cfg, W, enc_d, len_d, tok_d, frm_d, ol_d, wsb, stream, 
                 "joint_phase": {"us_per_step": js * 1e6 / max(1, stats["steps"]), "achieved": joint_flop / js / 1e12,
                                 "frac": joint_flop / js / 1e12 / peak, "dense_issued_frac": dense / js / 1e12 / peak,
                                 "rows_per_step": stats["joint_rows"] / max(1, stats["steps"])},
+                "joint_standalone": standalone,
                 "phase_us_per_step": {"joint": res["joint_ms"] * 1e3 / max(1, stats["steps"]),
                                       "decoder_update": res["lstm_ms"] * 1e3 / max(1, stats["steps"]),
                                       "projection": res["proj_ms"] * 1e3 / max(1, stats["steps"])},
@@ -412,7 +447,7 @@ def first_output_op(args, cfg, W):
 
     The call runs the projection, the decoder on an empty prefix and the joint's store epilogue, then the in-place
     Eq. (1) pass with the 4 best (label, offset) pairs.  `value` is windows per second for the whole call; the
-    in-place kernel's own share is what `ncu -k regex:first_output` shows for the same command (see profiles/).
+    in-place kernel's own share is what `ncu -k regex:first_output` shows for the same command.
     """
     import torch
     import wind_synth as ws
@@ -649,6 +684,23 @@ def beam_op(args, cfg, W):
         }))
 
 
+def joint_op(args, cfg, W):
+    """Secondary measurement (one JSON line of its own): the joint phase alone, back to back (see joint_standalone)."""
+    import torch
+    import wind_synth as ws
+    import paper_2505_13765_b200 as pkg
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    pkg.load_library()
+    peaks = load_peaks()
+    model = pkg.WindModel(ws.make_model(cfg), device=dev)
+    res = [joint_standalone(pkg, model, cfg, W, peaks, iters=1000) for _ in range(max(1, args.steps))]
+    best = min(res, key=lambda r: r["us_per_pass"])
+    print(json.dumps({"metric": "joint phase alone, TFLOP/s of algorithmic work (2 H (V+1) per window row)", "value": best["achieved"],
+                      "unit": "TFLOP/s", "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": cfg.name, "B": cfg.B, "W": W, "H": cfg.H, "V": cfg.V}, "joint_standalone": best}))
+
+
 def reference_arm(args, cfg, W):
     """The oracle as it stands, timed on the host cores (rank 0 only)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -657,7 +709,7 @@ def reference_arm(args, cfg, W):
     import wind_synth as ws
     weights = ws.make_model(cfg)
     enc_np, lens_np = ws.make_enc(cfg, pad="zero")
-    per_step_target = max(2.0, min(15.0, 120.0 / max(1, args.steps + args.warmup)))
+    per_step_target = max(2.0, min(15.0, 120.0 / max(1, args.steps + args.warmup)))   # the whole run within a few minutes
     for _ in range(args.warmup):
         run_cpu_baseline(cfg, weights, enc_np, lens_np, W, per_step_target)
     vals, secs = [], []

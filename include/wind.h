@@ -370,6 +370,27 @@ wind_status_t wind_read_trace(const wind_model_t* m, int32_t B, int32_t T, int32
                               wind_trace_event_t* host_out, int32_t capacity, int32_t* n_out);
 
 /*
+ * Measurement aid: the joint phase of the decoding loop by itself.  The loop kernel (the one that reads the joint's
+ * activations from the workspace: resident weights with grid barriers, or streamed weights, as the planner chooses for
+ * the shapes) runs ONLY its joint phase, `iters` times back to back, every CTA for itself, on fixed activations of all
+ * B * W window rows: the W_out contraction on tensor cores, the per-row argmax and the 64-bit key combine, exactly the
+ * code of a lock step's joint phase without the phases around it.  Timed with two CUDA events on `stream` around one
+ * launch (a short untimed launch goes first).  The paper has no counterpart; it is how the share of the tensor peak the
+ * joint can reach at a given size is told apart from the latency chain of the loop.
+ *   workspace  device, at least wind_workspace_bytes(m, B, 1, W); the model needs valid weight pointers.
+ *   host_out   ms for the timed launch; rows = B * W (algorithmic), rows_issued / labels_issued = what the tiles cover
+ *              (padding included); resident = which kernel ran; ctas = CTAs that had a joint item.
+ * flop per iteration: 2 * H * (V + 1) * rows (algorithmic), 2 * H * labels_issued * rows_issued (issued).
+ */
+typedef struct {
+    double ms;
+    int64_t rows, rows_issued, labels_issued;
+    int32_t iters, resident, ctas, reserved;
+} wind_joint_bench_t;
+wind_status_t wind_bench_joint(const wind_model_t* m, int32_t B, int32_t W, int32_t iters, void* workspace, size_t workspace_bytes,
+                               void* stream, wind_joint_bench_t* host_out);
+
+/*
  * Test hook for the failure path of the persistent loop kernel: with extra_arrivals > 0 its grid barrier waits
  * for that many arrivals more than there are CTAs, so the first barrier of the next decode can never fill.  Every
  * wait in the kernel is bounded (about two seconds), so the decode then ends by itself: the CTAs give up, free

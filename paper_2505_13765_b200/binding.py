@@ -31,7 +31,7 @@ WIND_KERNELS_AUTO, WIND_KERNELS_SIMT, WIND_KERNELS_TENSOR = 0, 1, 2
 EXPORTS = [
     "wind_workspace_bytes", "wind_decode_greedy", "wind_decode_window_greedy", "wind_host_staging_bytes", "wind_decode_greedy_host",
     "wind_eval_joint_window", "wind_window_first_output", "wind_eval_joint_window_static", "wind_profile_decode", "wind_beam_workspace_bytes", "wind_beam_search", "wind_plan_batches", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_debug_stall_barrier", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
-    "wind_set_loop_options", "wind_debug_plan",
+    "wind_set_loop_options", "wind_debug_plan", "wind_bench_joint",
 ]
 
 _vp = C.c_void_p
@@ -79,6 +79,11 @@ class wind_plan_t(C.Structure):
 
     def as_dict(self) -> Dict[str, int]:
         return {k: int(getattr(self, k)) for k, _ in self._fields_}
+
+
+class wind_joint_bench_t(C.Structure):
+    _fields_ = [("ms", C.c_double), ("rows", C.c_int64), ("rows_issued", C.c_int64), ("labels_issued", C.c_int64),
+                ("iters", C.c_int32), ("resident", C.c_int32), ("ctas", C.c_int32), ("reserved", C.c_int32)]
 
 
 class wind_trace_event_t(C.Structure):
@@ -140,6 +145,8 @@ def load_library():
     L.wind_set_loop_options.restype = None
     L.wind_debug_plan.argtypes = [mp, i32, i32, i32, i32, C.POINTER(wind_plan_t)]
     L.wind_debug_plan.restype = i32
+    L.wind_bench_joint.argtypes = [mp, i32, i32, i32, _vp, C.c_size_t, _vp, C.POINTER(wind_joint_bench_t)]
+    L.wind_bench_joint.restype = i32
     L.wind_status_string.argtypes = [i32]
     L.wind_status_string.restype = C.c_char_p
     L.wind_last_cuda_error.argtypes = []
@@ -179,6 +186,16 @@ def wind_debug_plan(dims: Dict[str, int], B: int, W: int, sms: int = 148, smem_o
     out = wind_plan_t()
     st = load_library().wind_debug_plan(C.byref(m), B, W, sms, smem_optin, C.byref(out))
     return st, out.as_dict()
+
+
+def wind_bench_joint(model: "WindModel", B: int, W: int, iters: int, workspace, stream=None) -> Dict[str, float]:
+    """The loop kernel's joint phase alone, `iters` times back to back on fixed activations (see wind.h)."""
+    out = wind_joint_bench_t()
+    st = load_library().wind_bench_joint(model.ref, B, W, iters, _ws_ptr(workspace), _ws_bytes(workspace), _stream_ptr(stream),
+                                         C.byref(out))
+    if st != WIND_OK:
+        raise WindError(st)
+    return {k: getattr(out, k) for k, _ in out._fields_ if k != "reserved"}
 
 
 def wind_set_trace(first_step: int) -> int:

@@ -591,6 +591,66 @@ wind_status_t wind_read_stats(const void* workspace, void* stream, wind_stats_t*
     return WIND_OK;
 }
 
+wind_status_t wind_bench_joint(const wind_model_t* m, int32_t B, int32_t W, int32_t iters, void* workspace, size_t workspace_bytes,
+                               void* stream, wind_joint_bench_t* host_out) {
+    wind_status_t s = check_model(m);
+    if (s != WIND_OK) return s;
+    s = check_shape(m, B, 1, W);
+    if (s != WIND_OK) return s;
+    if (!m->w_out || !m->b_out || !workspace || !host_out || iters < 1) return WIND_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return WIND_ERR_WORKSPACE;
+    memset(host_out, 0, sizeof(*host_out));
+    Call c;
+    memset(&c, 0, sizeof(c));
+    c.m = *m;
+    c.m.w_ih = nullptr; c.m.w_hh = nullptr; c.m.b_ih = nullptr; c.m.b_hh = nullptr;
+    for (int l = 0; l < m->L; ++l) {    // the tensor maps of the decoder's weights are built with the plan; nothing reads them here
+        c.w_ih[l] = m->w_ih ? m->w_ih[l] : nullptr; c.w_hh[l] = m->w_hh ? m->w_hh[l] : nullptr;
+        c.b_ih[l] = m->b_ih ? m->b_ih[l] : nullptr; c.b_hh[l] = m->b_hh ? m->b_hh[l] : nullptr;
+    }
+    c.B = B; c.T = 1; c.W = W; c.S = 1; c.max_out = 1;
+    c.ws = static_cast<uint8_t*>(workspace);
+    c.lay = make_layout(*m, B, 1, W, 1);
+    c.stream = (cudaStream_t)stream;
+    c.joint_iters = iters;
+    if (workspace_bytes < c.lay.total) return WIND_ERR_WORKSPACE;
+    if (!(m->dtype == WIND_DT_BF16 && tc_supported(c.m, B, 1, W)) || !m->w_pred || !c.w_hh[0]) return WIND_ERR_UNSUPPORTED;
+    // the kernel whose joint phase reads z from the workspace: grid barriers (resident weights) or streamed weights
+    const LoopOptions saved = loop_get_options();
+    LoopOptions o = saved;
+    o.dataflow = 0;
+    loop_set_options(o);
+    cudaError_t pe = loop_prepare(c);
+    LoopPlan pl;
+    cudaError_t pe2 = pe == cudaSuccess ? loop_plan(c, &pl) : pe;
+    loop_set_options(saved);
+    if (pe2 != cudaSuccess) return cuda_fail(pe2, "plan of the joint phase");
+    WIND_CUDA(cudaMemsetAsync(c.ctrl(), 0, sizeof(Ctrl), c.stream));
+    WIND_CUDA(cudaMemsetAsync(c.keys(), 0, sizeof(unsigned long long) * 3 * (size_t)c.lay.rows_pad, c.stream));
+    WIND_CUDA(launch_fill_z(c));
+    cudaEvent_t ev[2];
+    for (auto& e : ev) WIND_CUDA(cudaEventCreate(&e));
+    // one short launch first (first-use costs), then the timed one
+    c.joint_iters = iters < 8 ? iters : 8;
+    WIND_CUDA(tc_loop(c, nullptr, 0, nullptr, nullptr, -2));
+    c.joint_iters = iters;
+    WIND_CUDA(cudaEventRecord(ev[0], c.stream));
+    WIND_CUDA(tc_loop(c, nullptr, 0, nullptr, nullptr, -2));
+    WIND_CUDA(cudaEventRecord(ev[1], c.stream));
+    const wind_status_t st = read_status(c);
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, ev[0], ev[1]);
+    for (auto& e : ev) cudaEventDestroy(e);
+    host_out->ms = ms;
+    host_out->iters = iters;
+    host_out->resident = pl.resident;
+    host_out->rows = (int64_t)B * W;
+    host_out->rows_issued = (int64_t)pl.rg_count * pl.nj;
+    host_out->labels_issued = (int64_t)pl.vt_count * 128;
+    host_out->ctas = pl.resident ? (pl.vt_count * (pl.rg_count < pl.rg_stride ? pl.rg_count : pl.rg_stride)) : (pl.j_items < pl.grid ? pl.j_items : pl.grid);
+    return st;
+}
+
 int32_t wind_debug_stall_barrier(int32_t extra_arrivals) { return loop_set_extra_arrivals(extra_arrivals); }
 
 void wind_set_loop_options(int32_t resident, int32_t joint_placement, int32_t max_joint_waves, int32_t dataflow) {

@@ -220,4 +220,19 @@ cudaError_t launch_set_t(const Call& c, const int32_t* t0) {
     return cudaGetLastError();
 }
 
+// Measurement aid: joint activations of a plausible size in every row (a hash of the index mapped to [0, 2), as after a
+// ReLU), so that the joint phase can be timed alone on fixed operands.
+__global__ void fill_z_kernel(__nv_bfloat16* z, size_t n) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        uint32_t x = (uint32_t)i * 2654435761u + 12345u;
+        x ^= x >> 15; x *= 2246822519u; x ^= x >> 13;
+        z[i] = __float2bfloat16_rn((float)(x & 0xFFFFu) * (2.f / 65536.f));
+    }
+}
+cudaError_t launch_fill_z(const Call& c) {
+    fill_z_kernel<<<296, 256, 0, c.stream>>>(c.z(), (size_t)c.lay.rows_pad * c.m.H);
+    return cudaGetLastError();
+}
+
 }  // namespace wind

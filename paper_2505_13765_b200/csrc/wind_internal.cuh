@@ -133,6 +133,7 @@ struct Call {
     const int32_t* enc_len;
     int32_t B, T, W, S, max_out;
     int32_t mode;     // WIND_MODE_FIRST_NONBLANK (Algorithm 2) or WIND_MODE_WINDOW (best pair of Eq. (1) per step)
+    int32_t joint_iters;   // wind_bench_joint: run only the joint phase of the loop kernel, this many times
     int32_t* out_tokens;
     int32_t* out_frames;
     int32_t* out_len;
@@ -202,6 +203,7 @@ cudaError_t launch_init(const Call& c, int kernels_used, int launches_per_step, 
 cudaError_t launch_control(const Call& c, cudaGraphConditionalHandle handle, int use_handle);
 cudaError_t launch_force_tokens(const Call& c, const int32_t* prefix, int U, const int32_t* prefix_len, int u);
 cudaError_t launch_set_t(const Call& c, const int32_t* t0);
+cudaError_t launch_fill_z(const Call& c);   // measurement aid: fixed joint activations
 
 // first-output distribution of a window (Eq. 1), in place on the window's logits
 // beam search (Algorithm 3): workspace regions behind the call's own layout, and the host-driven search

@@ -931,6 +931,11 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         }
     };
 
+    // Measurement aid (FULL variant): the joint phase alone, joint_iters times back to back on the z rows the workspace
+    // holds, every CTA for itself (no barrier in between).
+    const bool jo = FULL && p.joint_iters > 0;
+    int jo_it = 0;
+    if (jo) { step = 0; goto joint_only_entry; }
     // ----- before the loop: layer 0's GEMM on the initial (zero) state -----
     if constexpr (RES) {
         early_res();
@@ -1168,6 +1173,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         // =====================================================================================
         // joint phase: window logits on tensor cores, per-row argmax in the epilogue
         // =====================================================================================
+joint_only_entry:
         {
             const int n_tile = p.nj;
             const uint32_t z_bytes = (uint32_t)n_tile * BK * 2;
@@ -1356,7 +1362,11 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 }
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_J, EV_EPI_DONE);
             }
-            if (!grid_sync(TR_J)) goto done;
+            if (!jo && !grid_sync(TR_J)) goto done;
+        }
+        if (jo) {
+            if (++jo_it < p.joint_iters) goto joint_only_entry;
+            goto done;
         }
         if ((FULL && p.forced)) break;
         if (FULL && p.window) {
@@ -1817,7 +1827,8 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.window = c.mode == WIND_MODE_WINDOW && !logits_out;
     p.nbkeys = c.keys() + 2 * (size_t)c.lay.rows_pad; p.jpart = c.jpart(); p.jblank = c.jblank(); p.parts = 4 * pl.vt_count;
     p.flags = c.flags(); p.pred_pub = c.pred_pub(); p.kslot = c.kslot();
-    const bool full = p.forced || p.window || p.trace;
+    p.joint_iters = c.joint_iters;
+    const bool full = p.forced || p.window || p.trace || p.joint_iters > 0;
     if (pl.resident && pl.dataflow) return loop_res_launch(t_loop_maps, p, pl.grid, pl.smem_bytes, full, c.stream);
     void* args[2] = {(void*)&t_loop_maps, (void*)&p};
     const void* fn = pl.resident ? (full ? (const void*)loop_kernel<true, true> : (const void*)loop_kernel<true, false>)

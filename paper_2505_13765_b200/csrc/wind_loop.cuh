@@ -105,6 +105,7 @@ struct LoopParams {
     // group written, ...) and the stamped pred_proj values
     uint32_t* flags;
     unsigned long long* pred_pub;  // [B][H / 2] (two bf16 values, stamp)
+    int joint_iters;               // measurement aid: > 0 runs only the joint phase, that many times (kernel with grid barriers, FULL)
     unsigned long long* kslot;     // [window rows][vocabulary tiles, padded to even] the tiles' stamped (logit, label) keys
 };
 
