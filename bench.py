@@ -573,7 +573,9 @@ def dataset_op(args, cfg, W):
 
     The same utterances are packed into batches of B twice: in arrival order and by the library's length-aware plan
     (wind_plan_batches).  Both packings are resident on the device before the clock starts; the timed region is the
-    decodes of all batches, back to back.  `value` is the planned packing's whole-set RTFx.
+    decodes of all batches, back to back.  `value` is the planned packing's whole-set RTFx.  `refilled_rows`: the same
+    set in ONE call on B batch rows that take the next utterance when theirs is finished (wind_decode_greedy_refill), in
+    arrival order and longest first.
     """
     import torch
     import wind_synth as ws
@@ -624,9 +626,41 @@ def dataset_op(args, cfg, W):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / k, steps
 
+    def run_refill(idx_order, k):
+        # all utterances resident at the set's T, decoded on B batch rows that are refilled inside the loop
+        T = int(lens_np.max())
+        enc_d = pkg.to_device_enc(model, np.ascontiguousarray(enc_np[idx_order, :T]))
+        len_d = torch.from_numpy(np.ascontiguousarray(lens_np[idx_order])).to(dev)
+        max_out = T * cfg.S
+        tok = torch.full((N, max_out), -1, dtype=torch.int32, device=dev)
+        frm = tok.clone()
+        ol = torch.zeros(N, dtype=torch.int32, device=dev)
+        wsb = torch.empty(pkg.wind_refill_workspace_bytes(model, N, T, B, W) + 256, dtype=torch.uint8, device=dev)
+        steps = 0
+        for _ in range(max(3, args.warmup)):
+            pkg.wind_decode_greedy_refill(model, enc_d, len_d, B, W, cfg.S, tok, frm, ol, wsb, stream=stream)
+            steps = pkg.wind_read_stats(wsb, stream)["steps"]
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(k):
+            pkg.wind_decode_greedy_refill(model, enc_d, len_d, B, W, cfg.S, tok, frm, ol, wsb, stream=stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / k, steps
+
     ms_a, steps_a = run(pack(np.arange(N)), args.steps)
     torch.cuda.empty_cache()
     ms_p, steps_p = run(pack(order), args.steps)
+    torch.cuda.empty_cache()
+    refill = {}
+    try:
+        for name, idx_order in (("arrival_order", np.arange(N)), ("longest_first", np.asarray(order))):
+            ms_r, steps_r = run_refill(idx_order, args.steps)
+            torch.cuda.empty_cache()
+            refill[name] = {"ms": ms_r, "lock_steps": steps_r, "value": float(lens_np.sum()) * FRAME_SECONDS / (ms_r * 1e-3)}
+    except pkg.WindError as e:      # shapes outside the tensor-core kernel set have no refilled rows
+        refill = {"unavailable": str(e)}
     audio_s = float(lens_np.sum()) * FRAME_SECONDS
     print(json.dumps({
         "metric": "greedy WIND RTFx of a set of utterances (audio-s/s at 80 ms/frame)", "op": "dataset",
@@ -635,7 +669,8 @@ def dataset_op(args, cfg, W):
         "config": {"workload": cfg.name, "utterances": N, "B": B, "frames": int(lens_np.sum()), "W": W},
         "length_aware": {"ms": ms_p, "lock_steps": steps_p, "batch_T": [int(t) for t in batch_T]},
         "arrival_order": {"ms": ms_a, "lock_steps": steps_a, "value": audio_s / (ms_a * 1e-3)},
-        "speedup_vs_arrival_order": ms_a / ms_p, "gpu_launches": 4 * len(batch_T) * args.steps,
+        "speedup_vs_arrival_order": ms_a / ms_p, "refilled_rows": refill,
+        "gpu_launches": 4 * len(batch_T) * args.steps,
     }))
 
 

@@ -151,6 +151,26 @@ wind_status_t wind_decode_greedy(const wind_model_t* m, const void* enc, const i
                                  size_t workspace_bytes, void* stream);
 
 /*
+ * Greedy decoding (Algorithm 2) of N utterances on B batch rows, B <= N or not: rows 0..B-1 start with utterances
+ * 0..B-1, and a row whose utterance is finished takes the next utterance that has none yet, inside the decoding loop
+ * (the row's decoder state is cleared in the lock step that finds it finished, the utterance moves in, and the step
+ * after that feeds start-of-sequence; two lock steps per change of utterance).  The batch therefore stays full until
+ * fewer than B utterances are left -- the length-sorted batches of wind_plan_batches shorten each batch's tail, this
+ * removes it.  Every utterance's result is the one wind_decode_greedy gives for it in any batch (Algorithm 2 treats
+ * the utterances of a batch independently); which row decodes which utterance is not part of the result.
+ *   enc [N, T, D], enc_len [N], out_tokens / out_frames [N, max_out], out_len [N]: as in wind_decode_greedy, per
+ *   utterance.  Workspace: wind_refill_workspace_bytes (enc_proj of all N utterances, everything else for B rows).
+ * Only the tensor-core kernel set refills rows: WIND_ERR_UNSUPPORTED for fp32 models and for shapes outside that set
+ * (see wind_decode_greedy), and when N * T * max(D, H) exceeds 2^31 - 1.  wind_read_stats counts over all N utterances.
+ * The paper decodes fixed batches; its batched decoding (Section 2.2) leaves the order of utterances to the caller.
+ */
+wind_status_t wind_refill_workspace_bytes(const wind_model_t* m, int32_t N, int32_t T, int32_t B, int32_t W, size_t* bytes);
+wind_status_t wind_decode_greedy_refill(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t N, int32_t T,
+                                        int32_t B, int32_t W, int32_t max_symbols, int32_t* out_tokens, int32_t* out_frames,
+                                        int32_t* out_len, int32_t max_out, void* workspace, size_t workspace_bytes,
+                                        void* stream);
+
+/*
  * Window-based greedy decoding: at every step the window's first-output distribution P'(v, t) of Eq. (1) is
  * formed under the current decoder state and its most probable entry decides the step (the variant sketched
  * beside Algorithm 2, which looks at the whole window instead of stopping at the first frame whose own argmax is

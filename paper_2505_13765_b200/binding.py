@@ -31,7 +31,7 @@ WIND_KERNELS_AUTO, WIND_KERNELS_SIMT, WIND_KERNELS_TENSOR = 0, 1, 2
 EXPORTS = [
     "wind_workspace_bytes", "wind_decode_greedy", "wind_decode_window_greedy", "wind_host_staging_bytes", "wind_decode_greedy_host",
     "wind_eval_joint_window", "wind_window_first_output", "wind_eval_joint_window_static", "wind_profile_decode", "wind_beam_workspace_bytes", "wind_beam_search", "wind_plan_batches", "wind_read_stats", "wind_set_trace", "wind_read_trace", "wind_debug_stall_barrier", "wind_set_kernels", "wind_status_string", "wind_last_cuda_error",
-    "wind_set_loop_options", "wind_debug_plan", "wind_bench_joint",
+    "wind_set_loop_options", "wind_debug_plan", "wind_bench_joint", "wind_refill_workspace_bytes", "wind_decode_greedy_refill",
 ]
 
 _vp = C.c_void_p
@@ -115,6 +115,10 @@ def load_library():
     L.wind_decode_window_greedy.restype = i32
     L.wind_decode_greedy.restype = i32
     L.wind_decode_greedy_host.argtypes = dec
+    L.wind_refill_workspace_bytes.argtypes = [mp, i32, i32, i32, i32, C.POINTER(C.c_size_t)]
+    L.wind_refill_workspace_bytes.restype = i32
+    L.wind_decode_greedy_refill.argtypes = [mp, _vp, _vp, i32, i32, i32, i32, i32, _vp, _vp, _vp, i32, _vp, C.c_size_t, _vp]
+    L.wind_decode_greedy_refill.restype = i32
     L.wind_decode_greedy_host.restype = i32
     L.wind_profile_decode.argtypes = dec + [C.POINTER(wind_profile_t)]
     L.wind_profile_decode.restype = i32
@@ -342,6 +346,31 @@ def wind_decode_greedy(model: WindModel, enc, enc_len, W: int, max_symbols: int,
     return st
 
 
+def wind_refill_workspace_bytes(model, N: int, T: int, B: int, W: int) -> int:
+    L = load_library()
+    n = C.c_size_t(0)
+    ref = model.ref if isinstance(model, WindModel) else C.byref(model)
+    st = L.wind_refill_workspace_bytes(ref, N, T, B, W, C.byref(n))
+    if st != WIND_OK:
+        raise WindError(st)
+    return int(n.value)
+
+
+def wind_decode_greedy_refill(model: WindModel, enc, enc_len, B: int, W: int, max_symbols: int, out_tokens, out_frames,
+                              out_len, workspace, stream=None, check: bool = True) -> int:
+    """N utterances on B batch rows, rows refilled inside the loop.  enc [N,T,D]; enc_len/out_* int32 device tensors [N...]."""
+    L = load_library()
+    N, T, D = enc.shape
+    assert enc.is_contiguous() and enc.dtype == model.torch_dtype and D == model.dims["D"]
+    max_out = out_tokens.shape[1]
+    st = L.wind_decode_greedy_refill(model.ref, enc.data_ptr(), enc_len.data_ptr(), N, T, B, W, max_symbols,
+                                     out_tokens.data_ptr(), out_frames.data_ptr(), out_len.data_ptr(), max_out,
+                                     _ws_ptr(workspace), _ws_bytes(workspace), _stream_ptr(stream))
+    if check and st != WIND_OK:
+        raise WindError(st)
+    return st
+
+
 def wind_decode_window_greedy(model: WindModel, enc, enc_len, W: int, max_symbols: int, out_tokens, out_frames, out_len,
                               workspace, stream=None, check: bool = True) -> int:
     """Window-based greedy decoding; arguments as wind_decode_greedy."""
@@ -523,6 +552,25 @@ def decode_dataset(model: WindModel, utterances, W: int, S: int, B: int, plan: b
         for r, i in enumerate(idx):
             toks[i], frms[i] = tok[r, : olen[r]].copy(), frm[r, : olen[r]].copy()
     return toks, frms, steps
+
+
+def decode_refill(model: WindModel, enc_np: np.ndarray, lens_np: np.ndarray, B: int, W: int, S: int,
+                  max_out: Optional[int] = None, check: bool = True):
+    """All N utterances of enc_np [N,T,D] on B batch rows that are refilled inside the loop (wind_decode_greedy_refill);
+    returns numpy (tokens [N, max_out], frames, out_len [N], stats, status)."""
+    torch = _torch()
+    N, T, _ = enc_np.shape
+    enc = to_device_enc(model, enc_np)
+    lens = torch.from_numpy(np.ascontiguousarray(lens_np, dtype=np.int32)).to(model.device)
+    if max_out is None:
+        max_out = max(1, T * S)
+    tok = torch.full((N, max_out), -1, dtype=torch.int32, device=model.device)
+    frm = torch.full((N, max_out), -1, dtype=torch.int32, device=model.device)
+    olen = torch.zeros(N, dtype=torch.int32, device=model.device)
+    ws = torch.empty(wind_refill_workspace_bytes(model, N, T, B, W) + 256, dtype=torch.uint8, device=model.device)
+    st = wind_decode_greedy_refill(model, enc, lens, B, W, S, tok, frm, olen, ws, check=check)
+    stats = wind_read_stats(ws)
+    return tok.cpu().numpy(), frm.cpu().numpy(), olen.cpu().numpy(), stats, st
 
 
 def decode(model: WindModel, enc_np: np.ndarray, lens_np: np.ndarray, W: int, S: int, max_out: Optional[int] = None,

@@ -268,6 +268,42 @@ wind_status_t wind_decode_window_greedy(const wind_model_t* m, const void* enc, 
     return read_status(c);
 }
 
+wind_status_t wind_refill_workspace_bytes(const wind_model_t* m, int32_t N, int32_t T, int32_t B, int32_t W, size_t* bytes) {
+    wind_status_t s = check_model(m);
+    if (s != WIND_OK) return s;
+    if (N < 1) return WIND_ERR_INVALID_ARG;
+    s = check_shape(m, N > B ? N : B, T, W);
+    if (s != WIND_OK) return s;
+    if (!bytes) return WIND_ERR_INVALID_ARG;
+    *bytes = make_layout(*m, B, T, W, 1, N).total;
+    return WIND_OK;
+}
+
+wind_status_t wind_decode_greedy_refill(const wind_model_t* m, const void* enc, const int32_t* enc_len, int32_t N, int32_t T,
+                                        int32_t B, int32_t W, int32_t max_symbols, int32_t* out_tokens, int32_t* out_frames,
+                                        int32_t* out_len, int32_t max_out, void* workspace, size_t workspace_bytes,
+                                        void* stream) {
+    if (N < 1) return WIND_ERR_INVALID_ARG;
+    wind_status_t s = check_decode_args(m, enc, enc_len, B, T, W, max_symbols, out_tokens, out_frames, out_len, max_out, workspace);
+    if (s != WIND_OK) return s;
+    s = check_shape(m, N > B ? N : B, T, W);
+    if (s != WIND_OK) return s;
+    if ((long long)N * max_out > 0x7fffffffLL) return WIND_ERR_UNSUPPORTED;
+    Call c;
+    fill_call(c, m, enc, enc_len, B, T, W, max_symbols, out_tokens, out_frames, out_len, max_out, workspace, (cudaStream_t)stream);
+    c.N = N;
+    c.lay = make_layout(*m, B, T, W, max_out, N);
+    if (workspace_bytes < c.lay.total) return WIND_ERR_WORKSPACE;
+    // rows are refilled inside the persistent loop kernel of the tensor-core set only
+    if (!use_tensor(c)) return WIND_ERR_UNSUPPORTED;
+    WIND_CUDA(tc_prepare(c));
+    WIND_CUDA(launch_init(c, WIND_KERNELS_TENSOR, 0, tc_setup_launches(c)));
+    WIND_CUDA(tc_enc_proj(c));
+    WIND_CUDA(tc_gate_table(c));
+    WIND_CUDA(tc_loop(c, nullptr, 0, nullptr, nullptr, g_trace_step));
+    return read_status(c);
+}
+
 wind_status_t wind_decode_greedy_host(const wind_model_t* m, const void* enc_host, const int32_t* enc_len_host, int32_t B,
                                       int32_t T, int32_t W, int32_t max_symbols, int32_t* out_tokens_host,
                                       int32_t* out_frames_host, int32_t* out_len_host, int32_t max_out, void* workspace,

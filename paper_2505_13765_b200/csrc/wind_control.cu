@@ -8,7 +8,7 @@ namespace wind {
 // Reset all per-call state.  Block 0 also fills the control block.
 __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsigned long long* t_pub, int32_t* count, int32_t* emit_tok,
                                                    unsigned long long* keys, float* h, float* c, uint32_t* hb, uint32_t* z,
-                                                   uint32_t* trace, size_t n_trace_words, uint32_t* sync_words, size_t n_sync_words, int32_t* out_len, const int32_t* __restrict__ enc_len, int B, int T, size_t n_keys,
+                                                   uint32_t* trace, size_t n_trace_words, uint32_t* sync_words, size_t n_sync_words, int32_t* out_len, const int32_t* __restrict__ enc_len, int32_t* slot, int N, int B, int T, size_t n_keys,
                                                    size_t n_h, size_t n_c, size_t n_hb_words, size_t n_z_words,
                                                    int blank, int step_cap, int kernels_used, int launches_per_step,
                                                    int launches_setup) {
@@ -27,8 +27,16 @@ __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsig
         t_pub[i] = 0ull;
         count[i] = 0;
         emit_tok[i] = blank;  // start of sequence: every decoder is fed the blank id once
-        out_len[i] = 0;
+        // batch row i starts with utterance i (the first B of N utterances; rows beyond N stay empty)
+        const int len = (int)i < N ? min(max(enc_len[i], 0), T) : 0;
+        slot[i] = len;
+        slot[B + i] = len;
+        slot[2 * B + i] = (int)i * T;
+        slot[3 * B + i] = (int)i * T;
+        slot[4 * B + i] = (int)i < N ? (int)i : 0;
+        slot[5 * B + i] = 0;
     }
+    for (size_t i = gtid; i < (size_t)N; i += gstride) out_len[i] = 0;
     if (blockIdx.x == 0) {
         __shared__ int s_active, s_bad;
         __shared__ unsigned long long s_frames;
@@ -36,7 +44,7 @@ __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsig
         __syncthreads();
         int a = 0;
         unsigned long long f = 0;
-        for (int b = threadIdx.x; b < B; b += blockDim.x) {
+        for (int b = threadIdx.x; b < N; b += blockDim.x) {
             int len = enc_len[b];
             if (len < 0 || len > T) s_bad = 1;   // a caller's mistake: nothing may be read through this length
             a += len > 0;
@@ -65,13 +73,19 @@ __global__ void __launch_bounds__(256) init_kernel(Ctrl* ctrl, int32_t* t, unsig
             ctrl->loop_ns = 0;
             ctrl->timeout_site = 0;
             ctrl->timeout_cta = 0;
+            ctrl->next_utt = N < B ? N : B;
+            ctrl->n_utt = N;
         }
     }
 }
 
 cudaError_t launch_init(const Call& c, int kernels_used, int launches_per_step, int launches_setup) {
     size_t n_h = 2 * (size_t)c.m.L * c.B * c.m.P, n_c = (size_t)c.m.L * c.B * c.m.P;
+    const int N = c.N > 0 ? c.N : c.B;
+    // every lock step moves some utterance forward (a frame, or one of at most S tokens on a frame), apart from the
+    // two steps around an utterance's start; with refilled rows the worst case is one utterance after the other
     long long step_cap = (long long)c.T * (c.S + 1) + 2;
+    if (c.N > 0) step_cap = (step_cap + 1) * c.N;
     if (step_cap > 0x7fffffff) step_cap = 0x7fffffff;
     const bool bf = c.m.dtype == WIND_DT_BF16;
     const size_t n_hb_words = bf ? (size_t)c.m.L * c.lay.Bpad * c.m.P : 0;       // 2 parities x bf16 = one word per element
@@ -86,7 +100,7 @@ cudaError_t launch_init(const Call& c, int kernels_used, int launches_per_step, 
                                               reinterpret_cast<uint32_t*>(c.trace()),
                                               bf ? sizeof(TraceEvent) * kTraceRoles * kTraceEvents / 4 : 0,
                                               reinterpret_cast<uint32_t*>(c.flags()), bf ? (c.lay.enc_proj - c.lay.flags) / 4 : 0,   // the counters, pred_pub and the key slots lie side by side, before enc_proj
-                                              c.out_len, c.enc_len, c.B, c.T, 3 * (size_t)c.lay.rows_pad, n_h, n_c, n_hb_words,
+                                              c.out_len, c.enc_len, c.slot(), N, c.B, c.T, 3 * (size_t)c.lay.rows_pad, n_h, n_c, n_hb_words,
                                               n_z_words, c.m.blank_id, (int)step_cap, kernels_used, launches_per_step,
                                               launches_setup);
     return cudaGetLastError();

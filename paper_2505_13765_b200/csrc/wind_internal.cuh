@@ -48,6 +48,8 @@ struct Ctrl {
     long long loop_ns;        // wall time of the loop kernel (CTA 0, global timer)
     int32_t timeout_site;     // which wait ran out first (resident-weights loop kernel; 0 = none), and in which CTA
     int32_t timeout_cta;
+    int32_t next_utt;         // first utterance that has not been given a batch row yet (more utterances than rows)
+    int32_t n_utt;
 };
 
 // Byte offsets of every workspace region (all multiples of kAlign).
@@ -55,6 +57,7 @@ struct Layout {
     size_t ctrl;       // Ctrl
     size_t t;          // int32 [2][B] current frame per utterance (the loop kernel ping-pongs by step parity)
     size_t t_pub;      // uint64 [B]  (lock step + 2) << 32 | next frame: published early in a step for the projection CTAs
+    size_t slot;       // int32 [6][B] the utterance of each batch row: frames [2][B], first enc_proj row [2][B], index, tokens so far
     size_t count;      // int32 [B]   consecutive emissions on the current frame
     size_t emit_tok;   // int32 [B]   token to feed to the decoder this step, -1 = none
     size_t keys;       // uint64 [3][rows_pad] packed (logit, label) argmax keys, 0 = empty ([1]: loop kernel's other step
@@ -72,7 +75,7 @@ struct Layout {
     size_t flags;      // uint32 [n_flags] arrival counters between CTA groups of the resident-weights loop kernel
     size_t kslot;      // uint64 [window rows][vocabulary tiles, padded to even] stamped (logit, label) keys, one per window row and vocabulary tile
     size_t pred_pub;   // (bf16 x 2, uint32) [B][H / 2] pred_proj values in pairs, each pair stamped with the projection phase that wrote it
-    size_t enc_proj;   // elem [B*T][H]
+    size_t enc_proj;   // elem [N*T][H] (N utterances; N = B unless rows are refilled)
     size_t total;
     // host staging (wind_decode_greedy_host), placed after `total`
     size_t st_enc, st_len, st_tok, st_frm, st_olen, st_total;
@@ -83,7 +86,7 @@ struct Layout {
 
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
-inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_out) {
+inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_out, int N = 0) {
     Layout L{};
     const size_t es = (m.dtype == WIND_DT_BF16) ? 2 : 4;
     size_t off = 0;
@@ -93,6 +96,7 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     L.rows_pad = (int32_t)(((size_t)B * W + 255) / 256 * 256);
     L.t = take(sizeof(int32_t) * 2 * B);
     L.t_pub = take(sizeof(uint64_t) * B);
+    L.slot = take(sizeof(int32_t) * 6 * B);
     L.count = take(sizeof(int32_t) * B);
     L.emit_tok = take(sizeof(int32_t) * B);
     L.keys = take(sizeof(uint64_t) * 3 * (size_t)L.rows_pad);
@@ -111,7 +115,7 @@ inline Layout make_layout(const wind_model_t& m, int B, int T, int W, int max_ou
     L.flags = take(bf ? sizeof(uint32_t) * (size_t)L.n_flags : 0);
     L.pred_pub = take(bf ? 4 * (size_t)B * m.H : 0);
     L.kslot = take(bf ? 8 * ((size_t)L.rows_pad + 256) * (((size_t)(m.V + 1 + 127) / 128 + 1) & ~(size_t)1) : 0);
-    L.enc_proj = take(es * (size_t)B * T * m.H);
+    L.enc_proj = take(es * (size_t)(N > B ? N : B) * T * m.H);
     L.total = off;
     L.st_enc = take(es * (size_t)B * T * m.D);
     L.st_len = take(sizeof(int32_t) * B);
@@ -132,6 +136,7 @@ struct Call {
     const void* enc;
     const int32_t* enc_len;
     int32_t B, T, W, S, max_out;
+    int32_t N;        // utterances when batch rows are refilled (wind_decode_greedy_refill), else 0: row b = utterance b
     int32_t mode;     // WIND_MODE_FIRST_NONBLANK (Algorithm 2) or WIND_MODE_WINDOW (best pair of Eq. (1) per step)
     int32_t joint_iters;   // wind_bench_joint: run only the joint phase of the loop kernel, this many times
     int32_t* out_tokens;
@@ -145,6 +150,7 @@ struct Call {
     Ctrl* ctrl() const { return reinterpret_cast<Ctrl*>(ws + lay.ctrl); }
     int32_t* t() const { return reinterpret_cast<int32_t*>(ws + lay.t); }   // [2][B]; the per-phase kernels use [0]
     unsigned long long* t_pub() const { return reinterpret_cast<unsigned long long*>(ws + lay.t_pub); }
+    int32_t* slot() const { return reinterpret_cast<int32_t*>(ws + lay.slot); }
     int32_t* count() const { return reinterpret_cast<int32_t*>(ws + lay.count); }
     int32_t* emit_tok() const { return reinterpret_cast<int32_t*>(ws + lay.emit_tok); }
     unsigned long long* keys() const { return reinterpret_cast<unsigned long long*>(ws + lay.keys); }  // [2][rows_pad]

@@ -290,6 +290,10 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
         const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
         unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
+        const int32_t* len_cur = p.slot_len2 + (size_t)(step & 1) * p.B;
+        int32_t* len_nxt = p.slot_len2 + (size_t)((step + 1) & 1) * p.B;
+        const int32_t* row_cur = p.slot_row2 + (size_t)(step & 1) * p.B;
+        int32_t* row_nxt = p.slot_row2 + (size_t)((step + 1) & 1) * p.B;
         for (int i = cta; i < p.l_items; i += G) {
             const int mt = i / p.ug_count, ug = i - mt * p.ug_count;
             const int b = mt * 128 + row_in_tile;
@@ -313,14 +317,23 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     // control step (Algorithm 2's branch): first non-blank row of the window.
                     // Everything it needs is requested at once; the keys of all W rows are readable.
                     int t = t_cur[b];
-                    const int len = p.enc_len[b];
+                    const int len_word = len_cur[b];
+                    const int len = len_word & kSlotLenMask;
                     const bool writer = ug == 0;
-                    int cnt = 0, pos = 0;
-                    if (writer) { cnt = p.count[b]; pos = p.out_len[b]; }
+                    int cnt = 0, pos = 0, s_row = 0, s_utt = 0;
+                    if (writer) { cnt = p.count[b]; pos = p.slot_pos[b]; s_row = row_cur[b]; s_utt = p.slot_utt[b]; }
+                    int len_out = len, row_out = s_row;
                     unsigned long long kk[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) kk[j] = j < p.W ? keys_cur[(size_t)b * p.W + j] : 0ull;
-                    if (t < len) {
+                    if (len_word & kSlotFresh) {
+                        // the row took a new utterance in the last step (its state is zero since then): start of sequence
+                        tok = p.blank;
+                        if (writer) {
+                            t_nxt[b] = t;
+                            for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
+                        }
+                    } else if (t < len) {
                         const int n = min(p.W, len - t);
                         int first = -1, label = p.blank;
                         bool bad = false;
@@ -351,9 +364,10 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                                 if (first > 0) cnt = 0;
                                 t += first;
                                 if (pos < p.max_out) {
-                                    p.out_tokens[(size_t)b * p.max_out + pos] = label;
-                                    p.out_frames[(size_t)b * p.max_out + pos] = t;
-                                    p.out_len[b] = pos + 1;
+                                    p.out_tokens[(size_t)s_utt * p.max_out + pos] = label;
+                                    p.out_frames[(size_t)s_utt * p.max_out + pos] = t;
+                                    p.out_len[s_utt] = pos + 1;
+                                    p.slot_pos[b] = pos + 1;
                                     emitted = 1;
                                     cnt += 1;
                                     if (cnt == p.S) { t += 1; cnt = 0; forced = 1; }
@@ -372,10 +386,31 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                             if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
                             if (forced) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
                         }
-                    } else if (writer) {
-                        t_nxt[b] = t;
+                    } else {
+                        // nothing left of this row's utterance: its decoder state is cleared, so that an utterance that
+                        // takes the row over starts from the zero state
+                        tok = -2;
+                        if (writer) {
+                            t_nxt[b] = t;
+                            if (ld_volatile_i32(&p.ctrl->next_utt) < p.n_utt) {
+                                const int u = atomicAdd(&p.ctrl->next_utt, 1);
+                                if (u < p.n_utt) {
+                                    // the next waiting utterance moves in; the coming step feeds it start-of-sequence
+                                    len_out = min(max(p.enc_len[u], 0), p.T) | kSlotFresh;
+                                    row_out = u * p.T;
+                                    p.slot_utt[b] = u;
+                                    p.slot_pos[b] = 0;
+                                    p.count[b] = 0;
+                                    t_nxt[b] = 0;
+                                }
+                            }
+                        }
                     }
-                    if (writer) p.emit_tok[b] = tok;
+                    if (writer) {
+                        len_nxt[b] = len_out;
+                        row_nxt[b] = row_out;
+                        p.emit_tok[b] = tok;
+                    }
                 }
             }
             if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
@@ -420,6 +455,9 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                                     const float cc = gf * cold[j] + gi * gg;
                                     cst[unit] = cc;
                                     hout[unit] = __float2bfloat16_rn(go * tanhf(cc));
+                                } else if (tok == -2) {
+                                    cst[unit] = 0.f;
+                                    hout[unit] = __float2bfloat16_rn(0.f);
                                 } else {
                                     hout[unit] = hin[unit];
                                 }
@@ -500,6 +538,10 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
         const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
         unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
+        const int32_t* len_cur = p.slot_len2 + (size_t)(step & 1) * p.B;
+        int32_t* len_nxt = p.slot_len2 + (size_t)((step + 1) & 1) * p.B;
+        const int32_t* row_cur = p.slot_row2 + (size_t)(step & 1) * p.B;
+        int32_t* row_nxt = p.slot_row2 + (size_t)((step + 1) & 1) * p.B;
         const int u16 = lane & 15, half = lane >> 4;
         const int unit = r_ut * 16 + u16;        // this thread's hidden unit; its gate is q
         // without recording CTAs, the two gate-0 warps of one CTA per utterance group record the step
@@ -524,10 +566,11 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             si.t = 0; si.len = 0; si.cnt = 0; si.pos = 0;
 #pragma unroll
             for (int j = 0; j < 8; ++j) si.kk[j] = 0ull;
+            int s_row = 0, s_utt = 0;
             if (in && decode) {
                 si.t = t_cur[b];
-                si.len = p.enc_len[b];
-                if (writer) { si.cnt = p.count[b]; si.pos = p.out_len[b]; }
+                si.len = len_cur[b];
+                if (writer) { si.cnt = p.count[b]; si.pos = p.slot_pos[b]; s_row = row_cur[b]; s_utt = p.slot_utt[b]; }
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     if (j < p.W) si.kk[j] = keys_cur[(size_t)b * p.W + j];
@@ -540,10 +583,12 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 cold[jj] = (!ctl_only && c0 + j < p.nl && b0 + j < p.B) ? cst[(size_t)(b0 + j) * p.P] : 0.f;
             }
             // the token utterance b feeds to its decoder in this step (-1: none)
-            int tok = -1, t_out = 0;
+            int tok = -1, t_out = 0, t_left = 0;
+            uint32_t t_row = 0u;
             if (in) {
                 if (step < 0) {
                     tok = p.blank;
+                    if (writer) { t_row = (uint32_t)row_cur[b]; t_left = len_cur[b] & kSlotLenMask; }   // frame 0 of the row's first utterance
                 } else if ((FULL && p.forced)) {
                     tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
                     if (tok >= p.NV || tok < -1) { tok = p.blank; set_status(p.ctrl, WIND_ERR_INVALID_ARG); }   // caller's mistake
@@ -551,8 +596,17 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     tok = p.emit_tok[b];     // decided by layer 0's CTAs one phase earlier
                 } else {
                     int t = si.t;
-                    const int len = si.len;
-                    if (t < len) {
+                    const int len = si.len & kSlotLenMask;
+                    int len_out = len, row_out = s_row;
+                    if (si.len & kSlotFresh) {
+                        // the row took a new utterance in the last step (its state is zero since then): start of sequence
+                        tok = p.blank;
+                        if (writer) {
+                            t_nxt[b] = t;
+                            t_out = t;
+                            for (int w = 0; w < p.W; ++w) keys_nxt[(size_t)b * p.W + w] = 0ull;
+                        }
+                    } else if (t < len) {
                         // control step (Algorithm 2's branch): first non-blank row of the window
                         const int n = min(p.W, len - t);
                         int first = -1, label = p.blank;
@@ -596,9 +650,10 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                                 if (first > 0) cnt = 0;
                                 t += first;
                                 if (si.pos < p.max_out) {
-                                    p.out_tokens[(size_t)b * p.max_out + si.pos] = label;
-                                    p.out_frames[(size_t)b * p.max_out + si.pos] = t;
-                                    p.out_len[b] = si.pos + 1;
+                                    p.out_tokens[(size_t)s_utt * p.max_out + si.pos] = label;
+                                    p.out_frames[(size_t)s_utt * p.max_out + si.pos] = t;
+                                    p.out_len[s_utt] = si.pos + 1;
+                                    p.slot_pos[b] = si.pos + 1;
                                     emitted = 1;
                                     cnt += 1;
                                     if (cnt == p.S) { t += 1; cnt = 0; forced = 1; }
@@ -618,14 +673,39 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                             if (emitted) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->tokens), 1ull);
                             if (forced) atomicAdd(reinterpret_cast<unsigned long long*>(&p.ctrl->forced), 1ull);
                         }
-                    } else if (writer) {
-                        t_nxt[b] = t;
-                        t_out = t;
+                    } else {
+                        // nothing left of this row's utterance: its decoder state is cleared, so that an utterance that
+                        // takes the row over starts from the zero state
+                        tok = -2;
+                        if (writer) {
+                            t_nxt[b] = t;
+                            t_out = t;
+                            if (ld_volatile_i32(&p.ctrl->next_utt) < p.n_utt) {
+                                const int u = atomicAdd(&p.ctrl->next_utt, 1);
+                                if (u < p.n_utt) {
+                                    // the next waiting utterance moves in; the coming step feeds it start-of-sequence
+                                    len_out = min(max(p.enc_len[u], 0), p.T) | kSlotFresh;
+                                    row_out = u * p.T;
+                                    p.slot_utt[b] = u;
+                                    p.slot_pos[b] = 0;
+                                    p.count[b] = 0;
+                                    t_nxt[b] = 0;
+                                    t_out = 0;
+                                }
+                            }
+                        }
+                    }
+                    if (writer) {
+                        len_nxt[b] = len_out;
+                        row_nxt[b] = row_out;
+                        t_row = (uint32_t)row_out + (uint32_t)t_out;
+                        t_left = (len_out & kSlotLenMask) - t_out;
                     }
                 }
                 // the next frame goes out at once, stamped with the step, for the projection CTAs (which fetch their
-                // enc_proj rows while this phase is still running)
-                if (writer && !(FULL && p.forced)) p.t_pub[b] = ((unsigned long long)(uint32_t)(step + 2) << 32) | (uint32_t)t_out;
+                // enc_proj rows while this phase is still running): enc_proj row of the frame, frames left (capped)
+                if (writer && !(FULL && p.forced))
+                    p.t_pub[b] = ((unsigned long long)(((uint32_t)(step + 2) << 8) | (uint32_t)min(max(t_left, 0), 255)) << 32) | t_row;
                 if (writer && p.L > 1 && decode) p.emit_tok[b] = tok;   // the upper layer's CTAs read it in their phase
             }
             if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_L, EV_TOK);
@@ -685,6 +765,9 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                             const float cc = gf * cold[jj] + gi * gg;
                             cst[(size_t)bj * p.P] = cc;
                             hout[(size_t)bj * p.P] = __float2bfloat16_rn(go * tanh_fast(cc));
+                        } else if (tok_s[j] == -2) {
+                            cst[(size_t)bj * p.P] = 0.f;
+                            hout[(size_t)bj * p.P] = __float2bfloat16_rn(0.f);
                         } else {
                             hout[(size_t)bj * p.P] = hin[(size_t)bj * p.P];
                         }
@@ -728,15 +811,11 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
     // b_pred of this thread's accumulator row: constant for the whole decode, read once
     const float p_bias = (res_p && e >= 0) ? p.b_pred[r_ht * 64 + 16 * q + (lane & 15)] : 0.f;
     // kind of a row at frame position t of its utterance, and the row's enc_proj frame
-    auto row_kind = [&](int b, int w, int t, int& frame) -> int {
-        const int left = p.enc_len[b] - t;
-        frame = t + w;
-        return left <= 0 ? 0 : (w >= left ? 1 : 2);
-    };
+    auto row_kind = [&](int w, int left) -> int { return left <= 0 ? 0 : (w >= left ? 1 : 2); };
     auto prefetch_res_P = [&]() {
         pre_kinds = -1;
         if ((FULL && p.forced)) return;
-        const uint32_t want = (uint32_t)(step + 2);
+        const uint32_t want = (uint32_t)(step + 2) & 0xFFFFFFu;
         // the published frames of this thread's rows, all requested together, until every stamp is this step's
         unsigned long long v[8];
         unsigned long long t0 = 0;
@@ -744,11 +823,11 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             bool all = true;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                v[i] = (unsigned long long)want << 32;
+                v[i] = (unsigned long long)want << 40;
                 if (p_bw[i] >= 0) asm volatile("ld.volatile.global.u64 %0, [%1];" : "=l"(v[i]) : "l"(p.t_pub + (p_bw[i] >> 8)) : "memory");
             }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) all = all && (uint32_t)(v[i] >> 32) == want;
+            for (int i = 0; i < 8; ++i) all = all && (uint32_t)(v[i] >> 40) == want;
             if (all) break;
             if ((it & 15u) == 0u) {
                 if (s_abort || ld_volatile_i32(&p.ctrl->abort)) return;
@@ -761,12 +840,11 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             if (p_bw[i] < 0) continue;
-            const int b = p_bw[i] >> 8, w = p_bw[i] & 255;
-            int frame = 0;
-            const int kind = row_kind(b, w, (int)(uint32_t)v[i], frame);
+            const int w = p_bw[i] & 255;
+            const int kind = row_kind(w, (int)((v[i] >> 32) & 255u));
             kinds |= kind << (2 * i);
             if (kind == 2) {
-                const __nv_bfloat16* src = p.enc_proj + ((size_t)b * p.T + frame) * p.H + r_ht * 64 + p_chunk * 8;
+                const __nv_bfloat16* src = p.enc_proj + ((size_t)(uint32_t)v[i] + w) * p.H + r_ht * 64 + p_chunk * 8;
                 asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(stash + (size_t)(p_row0 + 32 * i) * 128 + p_chunk * 16)),
                              "l"(src)
                              : "memory");
@@ -778,6 +856,8 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
     // projection epilogue of a P CTA: pred_proj rows [r_ht*64, +64) of utterances [r_qp*np, +np), then z
     auto epilogue_res_P = [&]() -> bool {
         const int32_t* t_new = p.t2 + (size_t)((step + 1) & 1) * p.B;
+        const int32_t* len_new = p.slot_len2 + (size_t)((step + 1) & 1) * p.B;
+        const int32_t* row_new = p.slot_row2 + (size_t)((step + 1) & 1) * p.B;
         const int h0 = r_ht * 64;
         const int rows_here = p.np * p.W;
         // one 16-byte chunk of a z row: act(enc_proj chunk + pred_proj chunk), zeros past the utterance's end
@@ -800,10 +880,10 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 ev[i] = make_uint4(0, 0, 0, 0);
                 if (p_bw[i] >= 0) {
                     const int b = p_bw[i] >> 8, w = p_bw[i] & 255;
-                    int frame = 0;
-                    const int kind = row_kind(b, w, t_new[b], frame);
+                    const int t = t_new[b];
+                    const int kind = row_kind(w, (len_new[b] & kSlotLenMask) - t);
                     kinds |= kind << (2 * i);
-                    if (kind == 2) ev[i] = *reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + frame) * p.H + h0 + p_chunk * 8);
+                    if (kind == 2) ev[i] = *reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)row_new[b] + t + w) * p.H + h0 + p_chunk * 8);
                 }
             }
         } else {
@@ -867,12 +947,12 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     x[i] = make_uint4(0, 0, 0, 0);
                     kinds4[i] = 0; bls[i] = 0; zoff[i] = 0;
                     if (r < rows_here && b < p.B) {
-                        int frame = 0;
-                        kinds4[i] = row_kind(b, w, t_new[b], frame);
+                        const int t = t_new[b];
+                        kinds4[i] = row_kind(w, (len_new[b] & kSlotLenMask) - t);
                         bls[i] = bl;
                         zoff[i] = ((size_t)b * p.W + w) * p.H + h0 + p_chunk * 8;
                         if (kinds4[i] == 2)
-                            x[i] = *reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + frame) * p.H + h0 + p_chunk * 8);
+                            x[i] = *reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)row_new[b] + t + w) * p.H + h0 + p_chunk * 8);
                     }
                 }
 #pragma unroll
@@ -1012,6 +1092,8 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             const int n_tile = p.np;
             const uint32_t b_bytes = (uint32_t)n_tile * BK * 2;
             const int32_t* t_new = p.t2 + (size_t)((step + 1) & 1) * p.B;
+            const int32_t* len_new = p.slot_len2 + (size_t)((step + 1) & 1) * p.B;
+            const int32_t* row_new = p.slot_row2 + (size_t)((step + 1) & 1) * p.B;
             const int i0 = p.p_items <= G ? G - 1 - cta : cta;   // projection items start at the far end of the grid
             if constexpr (RES) {
                 if (warp == 0) {
@@ -1024,8 +1106,9 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     if (lane == 0 && res_p) mma_part(2, tm_p, p.np, 0, p.kb_p / 2, false);
                 } else {
                     if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_START);
-                    int cnt = 0;
-                    for (int b = e; b < p.B; b += 256) cnt += t_new[b] < p.enc_len[b];
+                    // rows still decoding, plus one while utterances wait for a row
+                    int cnt = (e == 0 && ld_volatile_i32(&p.ctrl->next_utt) < p.n_utt) ? 1 : 0;
+                    for (int b = e; b < p.B; b += 256) cnt += t_new[b] < (len_new[b] & kSlotLenMask);
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
                     if (lane == 0) s_red[warp - 2] = cnt;
@@ -1078,8 +1161,8 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_START);
                 // utterances still decoding, counted by every CTA (they all take the same exit)
                 {
-                    int cnt = 0;
-                    for (int b = e; b < p.B; b += 128) cnt += t_new[b] < p.enc_len[b];
+                    int cnt = (e == 0 && ld_volatile_i32(&p.ctrl->next_utt) < p.n_utt) ? 1 : 0;   // utterances waiting for a row
+                    for (int b = e; b < p.B; b += 128) cnt += t_new[b] < (len_new[b] & kSlotLenMask);
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
                     if (lane == 0) s_red[warp - 2] = cnt;
@@ -1091,16 +1174,18 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     const int b = mt * 128 + row_in_tile;
                     const int h0 = hg * p.np;
                     int t = 0, n = 0;
+                    size_t row0 = 0;
                     if (b < p.B) {
                         t = t_new[b];
-                        n = min(p.W, p.enc_len[b] - t);   // <= 0 when the utterance is done
+                        n = min(p.W, (len_new[b] & kSlotLenMask) - t);   // <= 0 when the utterance is done
+                        row0 = (size_t)row_new[b] + t;                   // enc_proj row of the window's first frame
                     }
                     // the first rows of the window, requested before the accumulator is ready (np == 16)
                     uint4 ev[4][2];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         if (j < n) {
-                            const uint4* src = reinterpret_cast<const uint4*>(p.enc_proj + ((size_t)b * p.T + t + j) * p.H + h0);
+                            const uint4* src = reinterpret_cast<const uint4*>(p.enc_proj + (row0 + j) * p.H + h0);
                             ev[j][0] = src[0];
                             ev[j][1] = src[1];
                         }
@@ -1122,7 +1207,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                                         for (int j = 0; j < 4; ++j) {
                                             if (w0 + j < n) {
                                                 const uint4* src = reinterpret_cast<const uint4*>(
-                                                    p.enc_proj + ((size_t)b * p.T + t + w0 + j) * p.H + h0 + c0);
+                                                    p.enc_proj + (row0 + w0 + j) * p.H + h0 + c0);
                                                 ev[j][0] = src[0];
                                                 ev[j][1] = src[1];
                                             }
@@ -1550,9 +1635,10 @@ static cudaError_t loop_map3(CUtensorMap* map, const void* base, uint64_t rows, 
 // Tile plan: how each phase's GEMM is cut into items (one item = one accumulator), sized so that a phase is one wave
 // over the grid whenever the shapes allow.  A pure function of the shapes, the SM count and the opt-in shared memory
 // per block (so that it can be checked on the host over many shapes); cudaErrorInvalidConfiguration when nothing fits.
-cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem_optin, LoopPlan* out) {
+cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem_optin, LoopPlan* out, bool refill) {
     LoopPlan pl{};
-    const LoopOptions opt = g_loop_options;
+    LoopOptions opt = g_loop_options;
+    if (refill) opt.dataflow = 0;   // rows are refilled by loop_kernel only
     if (sms < 1 || m.H % BK || m.P % BK || m.H < BK || m.P < BK || B < 1 || W < 1) return cudaErrorInvalidConfiguration;
     const int G = sms;
     const int rows = B * W;
@@ -1733,7 +1819,7 @@ cudaError_t loop_plan(const Call& c, LoopPlan* out) {
     int sms = 0, smem_optin = 0;
     cudaError_t e = loop_device_info(&sms, &smem_optin, nullptr);
     if (e != cudaSuccess) return e;
-    return loop_plan_for(c.m, c.B, c.W, sms, smem_optin, out);
+    return loop_plan_for(c.m, c.B, c.W, sms, smem_optin, out, c.N > 0);
 }
 
 // whether the loop kernels have a plan for these shapes on the current device
@@ -1803,6 +1889,7 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.H = c.m.H; p.P = c.m.P; p.NV = c.m.V + 1; p.blank = c.m.blank_id; p.act = c.m.act; p.L = c.m.L;
     p.rows = c.B * c.W; p.rows_pad = c.lay.rows_pad; p.Bpad = c.lay.Bpad;
     long long cap = (long long)c.T * (c.S + 1) + 2;
+    if (c.N > 0) cap = (cap + 1) * c.N;    // refilled rows: at worst one utterance after the other
     p.step_cap = cap > 0x7fffffff ? 0x7fffffff : (int)cap;
     p.nj = pl.nj; p.vt_count = pl.vt_count; p.rg_count = pl.rg_count; p.j_items = pl.j_items; p.j_mode = pl.j_mode;
     p.rg_stride = pl.rg_stride > 0 ? pl.rg_stride : 1;
@@ -1816,6 +1903,8 @@ cudaError_t tc_loop(const Call& c, const int32_t* prefix, int U, const int32_t* 
     p.np = pl.np; p.hg_count = pl.hg_count; p.p_items = pl.p_items;
     p.kb_h = pl.kb_h; p.kb_p = pl.kb_p;
     p.stat_bytes = pl.stat_bytes;
+    p.slot_len2 = c.slot(); p.slot_row2 = c.slot() + 2 * (size_t)c.B; p.slot_utt = c.slot() + 4 * (size_t)c.B;
+    p.slot_pos = c.slot() + 5 * (size_t)c.B; p.n_utt = c.N > 0 ? c.N : c.B;
     p.enc_len = c.enc_len; p.t2 = c.t(); p.t_pub = c.t_pub(); p.count = c.count(); p.emit_tok = c.emit_tok(); p.keys2 = c.keys();
     p.out_tokens = c.out_tokens; p.out_frames = c.out_frames; p.out_len = c.out_len;
     p.c_state = c.c(); p.dh = c.dh(); p.hb = c.hb(0, 0); p.z = c.z(); p.enc_proj = (const __nv_bfloat16*)c.enc_proj(); p.g0 = c.g0();

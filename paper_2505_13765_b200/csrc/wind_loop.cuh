@@ -52,6 +52,9 @@ struct LoopPlan {
     uint32_t stage_lp, stage_j, stat_bytes, smem_bytes;
 };
 
+constexpr int kSlotFresh = 1 << 30;          // flag in a slot_len2 word
+constexpr int kSlotLenMask = kSlotFresh - 1;
+
 struct LoopParams {
     Ctrl* ctrl;
     int B, T, W, S, max_out, H, P, NV, blank, act, L;
@@ -66,7 +69,15 @@ struct LoopParams {
     int kb_h, kb_p;
     int stages_lp, stages_j;
     uint32_t stage_lp, stage_j, stat_bytes;
-    const int32_t* enc_len;
+    const int32_t* enc_len;        // [n_utt]
+    // Which utterance a batch row decodes (loop_kernel; the other kernels take row b = utterance b).  With more
+    // utterances than rows, a row whose utterance is finished takes the next waiting one.  Double-buffered by step
+    // parity like t2: a step's control threads write the copy the next step reads.
+    int n_utt;
+    int32_t* slot_len2;            // [2][B] frames of the row's utterance; kSlotFresh set in the step after it moved in
+    int32_t* slot_row2;            // [2][B] enc_proj row of the utterance's first frame
+    int32_t* slot_utt;             // [B] the utterance (index into the outputs); recording threads only
+    int32_t* slot_pos;             // [B] tokens emitted so far for it; recording threads only
     int32_t* t2;                   // [2][B]
     unsigned long long* t_pub;     // [B]
     int32_t* count;                // [B]
@@ -119,7 +130,7 @@ LoopOptions loop_get_options();
 bool loop_plan_ok(const wind_model_t& m, int B, int W);
 cudaError_t loop_plan(const Call& c, LoopPlan* out);
 // the plan as a pure function of the shapes and of the device's SM count and opt-in shared memory per block
-cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem_optin, LoopPlan* out);
+cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem_optin, LoopPlan* out, bool refill = false);
 // launchers of the two kernels (wind_loop.cu: streaming mode; wind_loop_res.cu: resident-weights mode)
 cudaError_t loop_res_set_smem(int bytes);
 cudaError_t loop_res_launch(const LoopMaps& maps, const LoopParams& p, int grid, uint32_t smem_bytes, bool full, cudaStream_t stream);

@@ -69,7 +69,7 @@ cudaError_t tc_prepare(Call& c) {
     TcMaps& M = t_maps;
     const wind_model_t& m = c.m;
 #define WIND_MAP(call_) do { e = (call_); if (e != cudaSuccess) return e; } while (0)
-    WIND_MAP(make_map(&M.enc, c.enc, (uint64_t)c.B * c.T, m.D, BM));
+    WIND_MAP(make_map(&M.enc, c.enc, (uint64_t)(c.N > 0 ? c.N : c.B) * c.T, m.D, BM));
     WIND_MAP(make_map(&M.w_enc, m.w_enc, m.H, m.D, 256));
     WIND_MAP(make_map(&M.emb, m.emb, (uint64_t)m.V + 1, m.E, BM));
     WIND_MAP(make_map(&M.w_ih0, c.w_ih[0], 4ull * m.P, m.E, 128));
@@ -276,7 +276,7 @@ cudaError_t tc_enc_proj(const Call& c) {
     GemmParams p{};
     p.ctrl = c.ctrl();
     p.k_blocks = c.m.D / BK;
-    p.rows = (long long)c.B * c.T;
+    p.rows = (long long)(c.N > 0 ? c.N : c.B) * c.T;
     p.N = c.m.H;
     p.enc_len = c.enc_len; p.T = c.T;
     p.out_bf16 = (__nv_bfloat16*)c.enc_proj(); p.bias0 = c.m.b_enc;

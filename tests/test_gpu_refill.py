@@ -1,0 +1,111 @@
+"""GPU parity of decoding N utterances on B batch rows that are refilled inside the persistent loop.
+
+Algorithm 2 treats the utterances of a batch independently, so what an utterance's row did before it moved in must not
+show in its transcript: every utterance's (tokens, frames) from wind_decode_greedy_refill must equal, bit for bit, the
+ones wind_decode_greedy gives for it with all N utterances in one batch (same kernel mode forced for both), for every
+number of rows -- one row (the utterances one after the other), a few, exactly N, more rows than utterances.  A sample
+is also replayed through the CPU oracle under the margin rule of the parity tests, and the counters are checked
+against what the transcripts say.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from conftest import set_loop_mode
+from test_gpu_parity import MARGIN, ragged_case
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pkg():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import __graft_entry__ as entry
+    entry.build()
+    import paper_2505_13765_b200 as p
+    p.load_library()
+    return p
+
+
+CASES = {
+    # name: (N, T, P, H, V, L, act, W, S, rows to try)
+    "one_layer_w4": (37, 40, 128, 128, 200, 1, 0, 4, 3, [1, 3, 8, 37, 50]),
+    "two_layers_w8": (29, 30, 192, 64, 300, 2, 1, 8, 2, [2, 5, 29]),
+    "algorithm1_many_rows": (210, 16, 64, 64, 140, 1, 0, 1, 4, [70, 150]),
+    "wide_window_two_waves": (40, 48, 64, 128, 3000, 1, 1, 16, 3, [6, 33]),
+}
+
+
+@pytest.mark.parametrize("mode", ["barriers", "streaming"])
+@pytest.mark.parametrize("case", list(CASES))
+def test_refilled_rows_give_every_utterance_its_single_batch_transcript(pkg, mode, case):
+    N, T, P, H, V, L, act, W, S, rows = CASES[case]
+    set_loop_mode(pkg, mode)
+    w, enc, lens = ragged_case(700 + N, B=N, T=T, D=64, E=64, P=P, L=L, H=H, V=V, act=act, bias=1.5, dtype="bf16")
+    lens[N // 2] = 0                       # an empty utterance in the middle of the queue
+    lens[-1] = T                           # and a full-length one at its end
+    enc = np.nan_to_num(enc)
+    for b in range(N):
+        enc[b, lens[b]:] = np.nan          # padding is never read
+    model = pkg.WindModel(w)
+    tok1, frm1, olen1, stats1, st1 = pkg.decode(model, enc, lens, W, S)
+    assert st1 == 0 and stats1["kernels"] == 2
+    om = oracle.Model(w)
+    for B in rows:
+        tok, frm, olen, stats, st = pkg.decode_refill(model, enc, lens, B, W, S)
+        assert st == 0 and stats["kernels"] == 2, (B, st)
+        assert np.array_equal(olen, olen1), f"{case} rows={B}: token counts differ"
+        for u in range(N):
+            assert np.array_equal(tok[u, : olen[u]], tok1[u, : olen1[u]]), f"{case} rows={B}: tokens of utterance {u}"
+            assert np.array_equal(frm[u, : olen[u]], frm1[u, : olen1[u]]), f"{case} rows={B}: frames of utterance {u}"
+            assert np.all(tok[u, olen[u]:] == -1)
+        assert stats["frames"] == int(lens.sum()) and stats["tokens"] == int(olen.sum())
+        hist = np.array(stats["jump_hist"])
+        assert (hist * np.arange(65)).sum() + stats["forced"] == int(lens.sum())
+        if B >= N:
+            assert stats["steps"] == stats1["steps"]      # nothing to refill: the same lock steps as one batch
+        else:
+            # fewer rows than utterances: more lock steps than one batch of everything, but far fewer than the
+            # utterances decoded one after the other
+            assert stats["steps"] >= stats1["steps"]
+        print(f"[refill] {case} {mode}: {N} utterances on {B} rows, {stats['steps']} lock steps "
+              f"(one batch of {N}: {stats1['steps']})")
+    # a sample against the oracle (margin rule), on the last row count
+    for u in (0, N // 3, N - 1):
+        r = oracle.replay_verify(om, enc[u], int(lens[u]), S, tok[u, : olen[u]], frm[u, : olen[u]], MARGIN)
+        assert r["rc"] == 0, f"utterance {u}: {r}"
+
+
+def test_refill_needs_fewer_lock_steps_than_planned_batches(pkg):
+    # lengths spread over 10..60 frames: with 8 rows, length-sorted batches still wait for each batch's longest
+    # utterance; refilled rows do not
+    w, enc, lens = ragged_case(801, B=64, T=60, D=64, E=64, P=128, L=1, H=128, V=200, act=0, bias=1.5, dtype="bf16")
+    lens = np.maximum(lens, 10).astype(np.int32)
+    enc = np.nan_to_num(enc)
+    model = pkg.WindModel(w)
+    utts = [np.ascontiguousarray(enc[b, : lens[b]]) for b in range(64)]
+    t_p, f_p, steps_planned = pkg.decode_dataset(model, utts, 4, 3, B=8, plan=True)
+    tok, frm, olen, stats, st = pkg.decode_refill(model, enc, lens, 8, 4, 3)
+    assert st == 0
+    for u in range(64):
+        assert np.array_equal(tok[u, : olen[u]], t_p[u]) and np.array_equal(frm[u, : olen[u]], f_p[u])
+    assert stats["steps"] < steps_planned, (stats["steps"], steps_planned)
+    print(f"[refill] 64 utterances on 8 rows: {stats['steps']} lock steps refilled, {steps_planned} in length-sorted batches")
+
+
+def test_refill_rejects_what_it_does_not_cover(pkg):
+    bd = pkg.binding
+    w, enc, lens = ragged_case(802, B=6, T=12, D=64, E=64, P=64, L=1, H=64, V=140, dtype="f32")
+    model = pkg.WindModel(w)
+    enc = np.nan_to_num(enc)
+    assert pkg.decode_refill(model, enc, lens, 2, 4, 3, check=False)[4] == bd.WIND_ERR_UNSUPPORTED   # fp32 model
+    w, enc, lens = ragged_case(803, B=6, T=12, D=64, E=64, P=64, L=1, H=64, V=140, dtype="bf16")
+    model = pkg.WindModel(w)
+    enc = np.nan_to_num(enc)
+    bad = lens.copy()
+    bad[5] = 13                                                                                      # beyond T, in the queue
+    assert pkg.decode_refill(model, enc, bad, 2, 4, 3, check=False)[4] == bd.WIND_ERR_INVALID_ARG
+    ok = pkg.decode_refill(model, enc, lens, 2, 4, 3)                                                # the context is fine
+    assert ok[4] == 0
