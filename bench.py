@@ -199,7 +199,7 @@ def main():
                     help="tensor-core loop: the planner's choice, or resident weights with grid barriers / with arrival counters, or streamed weights")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the W=1 comparison, e2e and per-kernel timing legs")
-    ap.add_argument("--op", default="decode", choices=["decode", "first_output", "window_greedy", "dataset", "beam", "joint"],
+    ap.add_argument("--op", default="decode", choices=["decode", "first_output", "window_greedy", "dataset", "beam", "joint", "schedule"],
                     help="first_output: time wind_window_first_output (Eq. 1 on one window per utterance) instead of the decode; "
                          "window_greedy: time wind_decode_window_greedy on the whole workload; dataset: 4 x B utterances in "
                          "arrival-order batches against length-aware batches; beam: wind_beam_search on one utterance, beams 2..4")
@@ -225,6 +225,8 @@ def main():
         return beam_op(args, cfg, W)
     if args.op == "joint":
         return joint_op(args, cfg, W)
+    if args.op == "schedule":
+        return schedule_op(args, cfg, W)
 
     import torch
     import paper_2505_13765_b200 as pkg
@@ -734,6 +736,98 @@ def joint_op(args, cfg, W):
     print(json.dumps({"metric": "joint phase alone, TFLOP/s of algorithmic work (2 H (V+1) per window row)", "value": best["achieved"],
                       "unit": "TFLOP/s", "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
                       "config": {"workload": cfg.name, "B": cfg.B, "W": W, "H": cfg.H, "V": cfg.V}, "joint_standalone": best}))
+
+
+def step_kinds(lens, tok_len, frames, W, S):
+    """Per utterance the kinds of its Algorithm 2 iterations, rebuilt from its transcript: True = the window held a non-blank
+    frame (one emission, one decoder update), False = every row blank (t += n)."""
+    out = []
+    for b in range(len(lens)):
+        f, n_tok, length = frames[b], int(tok_len[b]), int(lens[b])
+        t, k, cnt, kinds = 0, 0, 0, []
+        while t < length:
+            n = min(W, length - t)
+            if k < n_tok and f[k] < t + n:
+                cnt = (cnt if f[k] == t else 0) + 1
+                t = int(f[k])
+                k += 1
+                if cnt == S:
+                    t, cnt = t + 1, 0
+                kinds.append(True)
+            else:
+                t, cnt = t + n, 0
+                kinds.append(False)
+        out.append(np.array(kinds, dtype=bool))
+    return out
+
+
+def schedule_counts(kinds):
+    """Passes of the two batched schedules over the same per-utterance iterations.
+
+    Lock step (what the library runs): every pass is one joint evaluation, one masked decoder update and one projection for
+    the whole batch; an utterance takes one of its iterations per pass, so the passes are the longest utterance's.
+    Label looping proper: an outer iteration repeats the joint (with a fresh window, hence fresh activations) for the
+    utterances whose window was all blank until every utterance still decoding holds a non-blank frame, then runs ONE
+    decoder update and projection for all of them."""
+    lock = max((len(k) for k in kinds), default=0)
+    pos = [0] * len(kinds)
+    joint_passes = updates = 0
+    while True:
+        inner, any_emit = 0, False
+        for u, k in enumerate(kinds):
+            p = pos[u]
+            if p >= len(k):
+                continue
+            nxt = np.flatnonzero(k[p:])
+            blanks = int(nxt[0]) if len(nxt) else len(k) - p        # all-blank windows before the next emission
+            inner = max(inner, blanks + (1 if len(nxt) else 0))
+            any_emit = any_emit or len(nxt) > 0
+            pos[u] = p + blanks + (1 if len(nxt) else 0)
+        if inner == 0:
+            break
+        joint_passes += inner
+        updates += 1 if any_emit else 0
+    return {"lock_step_passes": lock, "label_looping_joint_passes": joint_passes, "label_looping_decoder_updates": updates}
+
+
+def schedule_op(args, cfg, W):
+    """Secondary measurement (one JSON line of its own): how many batched passes the label-looping schedule proper would
+    need on this workload against the lock-step schedule the library runs, counted on the transcripts the GPU produced, and
+    priced with the per-phase times of the same decode (wind_profile_decode)."""
+    import torch
+    import wind_synth as ws
+    import paper_2505_13765_b200 as pkg
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    pkg.load_library()
+    pkg.wind_set_kernels(args.kernels)
+    set_loop_mode(pkg, args.loop_mode)
+    enc_np, lens_np = ws.make_enc(cfg, pad="zero")
+    model = pkg.WindModel(ws.make_model(cfg), device=dev)
+    enc_d = pkg.to_device_enc(model, enc_np)
+    len_d = torch.from_numpy(lens_np).to(dev)
+    B, T, _ = enc_np.shape
+    tok = torch.full((B, T * cfg.S), -1, dtype=torch.int32, device=dev)
+    frm, ol = tok.clone(), torch.zeros(B, dtype=torch.int32, device=dev)
+    wsb = pkg.alloc_workspace(model, B, T, W)
+    stream = torch.cuda.current_stream()
+    for _ in range(max(3, args.warmup)):
+        pkg.wind_decode_greedy(model, enc_d, len_d, W, cfg.S, tok, frm, ol, wsb, stream=stream)
+    stats = pkg.wind_read_stats(wsb, stream)
+    prof = pkg.wind_profile_decode(model, enc_d, len_d, W, cfg.S, tok, frm, ol, wsb, stream=stream)
+    counts = schedule_counts(step_kinds(lens_np, ol.cpu().numpy(), frm.cpu().numpy(), W, cfg.S))
+    assert counts["lock_step_passes"] == stats["steps"], (counts, stats["steps"])
+    n = stats["steps"]
+    j, l, p = prof["joint_ms"] / n, prof["lstm_ms"] / n, prof["proj_ms"] / n      # ms per pass of each phase
+    # label looping proper: every joint pass needs its activations rebuilt (the projection phase's epilogue; priced as a
+    # whole projection phase: the phase is bound by its barrier and round trips, not by the GEMM), every update a decoder phase
+    est = counts["label_looping_joint_passes"] * (j + p) + counts["label_looping_decoder_updates"] * l
+    print(json.dumps({"metric": "batched passes per decode: lock step against label looping proper", "op": "schedule",
+                      "value": counts["label_looping_joint_passes"] / max(1, n), "unit": "joint passes relative to lock steps",
+                      "higher_is_better": False, "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+                      "config": {"workload": cfg.name, "B": B, "W": W}, **counts,
+                      "phase_ms_per_pass": {"joint": j, "decoder_update": l, "projection": p},
+                      "lock_step_ms": n * (j + l + p), "label_looping_ms_estimate": est}))
 
 
 def reference_arm(args, cfg, W):

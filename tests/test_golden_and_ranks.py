@@ -71,3 +71,28 @@ def test_two_rank_aggregation_takes_the_slowest_rank_and_sums_the_work():
         value, ms_per_step = res[rank]
         assert ms_per_step == pytest.approx(50.0)                       # 250 ms over 5 steps: the slower rank
         assert value == pytest.approx(1000.0 * 5 * 2 / 0.250)           # both replicas' audio over that time
+
+
+def test_schedule_counts_rebuilt_from_transcripts_match_the_oracle_and_a_hand_case():
+    # the benchmark's comparison of batched schedules counts passes on transcripts: the rebuilt per-utterance iterations
+    # must be the oracle's own (its step counter), and the two schedules' passes those of a case worked by hand
+    import bench
+    from naive_model import random_weights
+    r = np.random.default_rng(5)
+    w = random_weights(r, 8, 6, 10, 1, 12, 9, blank_bias=1.0)
+    om = oracle.Model(w)
+    lens = np.array([30, 17, 0, 25], np.int32)
+    enc = r.standard_normal((4, 30, 8)).astype(np.float32)
+    for W in (1, 3, 8):
+        for S in (1, 3):
+            tok, frm, on, st = oracle.decode_batch(om, enc, lens, W=W, S=S)
+            kinds = bench.step_kinds(lens, on, frm, W, S)
+            per_utt = [oracle.decode_batch(om, enc[b:b + 1], lens[b:b + 1], W=W, S=S)[3]["steps"] for b in range(4)]
+            assert [len(k) for k in kinds] == per_utt
+            assert [int(k.sum()) for k in kinds] == [int(x) for x in on]
+    # utterance A: blank, blank, emit, emit; utterance B: emit, blank, emit
+    kinds = [np.array([0, 0, 1, 1], bool), np.array([1, 0, 1], bool)]
+    c = bench.schedule_counts(kinds)
+    # lock step: 4 passes.  label looping: iteration 1 needs 3 joint passes (A's two blank windows), iteration 2 needs 2
+    # (B's blank window), then nothing is left: 5 joint passes, 2 decoder updates
+    assert c == {"lock_step_passes": 4, "label_looping_joint_passes": 5, "label_looping_decoder_updates": 2}
