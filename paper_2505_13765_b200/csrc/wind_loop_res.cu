@@ -11,11 +11,12 @@
 //                 group's utterances are copied in (cp.async, 128-byte swizzled K-major layout) as soon as the
 //                 control step has published the next frame, pred_proj arrives as stamped (value, stamp) pairs that
 //                 the CTA polls, the sum is activated in place.  Epilogue: per-row argmax over the tile's 128
-//                 entries by warp shuffles, 64-bit atomicMax of (logit, label) keys across the vocabulary tiles;
-//                 the logits never leave the chip.  Then one arrival on the row group's counter.
+//                 entries by warp shuffles; the winner of every (window row, vocabulary tile) goes, stamped with
+//                 the lock step, into its own key slot by a plain store; the logits never leave the chip.
 //   L  decoder    gates [4 gates x 16 units, nl utterances] = W_hh tile . h^T, tile resident in shared memory.  The
 //                 GEMM needs only the state, so it is issued a slot ahead and its result waits in tensor memory; the
-//                 slot itself is: wait for the keys of the CTA's utterances (their row groups' counters), control
+//                 slot itself is: poll the key slots of the CTA's utterances (four lanes per utterance read a
+//                 row's slots and take the maximum over the vocabulary tiles themselves), control
 //                 step (Algorithm 2's branch: first non-blank row of the window, jump, emission, max-symbols rule),
 //                 gate-table rows of the chosen tokens, LSTM cell update, new h (bf16) and c (fp32), one arrival on
 //                 the utterance group's counter.  CTAs without a weight tile record the steps (outputs, counters,
@@ -23,7 +24,8 @@
 //                 GEMM runs on CTAs holding a W_ih[1] tile after layer 0's arrivals, its recurrent term a slot ahead
 //                 on CTAs holding a W_hh[1] tile.
 //   P  projection pred_proj [64 H rows, np utterances] = W_pred tile . h_top^T + b_pred after the state counters of
-//                 its utterances have filled; written as (fp32 value, stamp) pairs, which is what the joint CTAs poll.
+//                 its utterances have filled; written as (bf16 pair, stamp) 8-byte words, which is what the joint
+//                 CTAs poll: data and "ready" arrive in one load.
 //
 // No CTA waits for the whole grid: utterances are independent (Algorithm 2 has no cross-utterance term), so a joint
 // CTA waits only for the pred_proj of its row group's utterances, a decoder CTA for the vocabulary tiles of its own
