@@ -156,8 +156,9 @@ wind_status_t wind_decode_greedy(const wind_model_t* m, const void* enc, const i
  * (the row's decoder state is cleared in the lock step that finds it finished, the utterance moves in, and the step
  * after that feeds start-of-sequence; two lock steps per change of utterance).  The batch therefore stays full until
  * fewer than B utterances are left -- the length-sorted batches of wind_plan_batches shorten each batch's tail, this
- * removes it.  Every utterance's result is the one wind_decode_greedy gives for it in any batch (Algorithm 2 treats
- * the utterances of a batch independently); which row decodes which utterance is not part of the result.
+ * removes it.  Every utterance's result is the one wind_decode_greedy gives for it in a batch of B rows (Algorithm 2
+ * treats the utterances of a batch independently; a batch size for which the library picks another kernel plan can
+ * differ at low-margin decisions, as stated at the top); which row decodes which utterance is not part of the result.
  *   enc [N, T, D], enc_len [N], out_tokens / out_frames [N, max_out], out_len [N]: as in wind_decode_greedy, per
  *   utterance.  Workspace: wind_refill_workspace_bytes (enc_proj of all N utterances, everything else for B rows).
  * Only the tensor-core kernel set refills rows: WIND_ERR_UNSUPPORTED for fp32 models and for shapes outside that set

@@ -70,3 +70,42 @@ def test_large_dimensions(pkg, monkeypatch):
             tp.logits_parity(pkg, w, enc, lens, W=W, S=S, tol=tp.TOL["bf16"], n_windows=B, kernels=2)
         else:
             tp.check_against_oracle(pkg, w, enc, lens, W, S, kernels=2)
+
+
+def refill_case(pkg, r, i, seed_base):
+    """One random (model, utterances, rows) case: refilled rows against one batch of all utterances, same loop mode."""
+    P = int(r.choice([64, 128, 192, 256, 640])); H = int(r.choice([64, 128, 256, 640]))
+    V = int(r.choice([127, 140, 300, 1024, 2100])); N = int(r.choice([1, 2, 9, 40, 77, 130, 200]))
+    B = int(r.choice([1, 2, 5, 16, 33, 64, 128, 150])); W = int(r.choice([1, 2, 4, 8, 13, 16, 32])); L = int(r.choice([1, 1, 2, 3]))
+    S = int(r.integers(1, 6)); act = int(r.integers(0, 2)); T = int(r.integers(4, 30))
+    mode = ["barriers", "streaming"][i % 2]
+    set_loop_mode(pkg, mode)
+    w, enc, lens = tp.ragged_case(seed_base + i, B=N, T=T, D=64, E=64, P=P, L=L, H=H, V=V, act=act,
+                                  blank_id=0 if i % 3 == 0 else None, bias=float(r.uniform(0.5, 3.0)), dtype="bf16")
+    enc = np.nan_to_num(enc)
+    print(f"refill case {i}: N={N} rows={B} T={T} W={W} S={S} P={P} H={H} V={V} L={L} mode={mode}", flush=True)
+    model = pkg.WindModel(w)
+    # the reference decodes the utterances in fixed batches of exactly B rows (the last one padded with empty utterances),
+    # so that both sides run the same tile plan, hence the same kernel and arithmetic
+    tok1 = np.full((N, max(1, T * S)), -1, np.int32); frm1 = tok1.copy(); olen1 = np.zeros(N, np.int32)
+    for k in range(0, N, B):
+        m = min(B, N - k)
+        e = np.zeros((B,) + enc.shape[1:], enc.dtype); l = np.zeros(B, np.int32)
+        e[:m], l[:m] = enc[k: k + m], lens[k: k + m]
+        t_, f_, o_, _, st1 = pkg.decode(model, e, l, W, S)
+        assert st1 == 0
+        tok1[k: k + m], frm1[k: k + m], olen1[k: k + m] = t_[:m], f_[:m], o_[:m]
+    tok, frm, olen, stats, st = pkg.decode_refill(model, enc, lens, B, W, S)
+    assert st == 0 and stats["kernels"] == 2
+    assert np.array_equal(olen, olen1)
+    for u in range(N):
+        assert np.array_equal(tok[u, : olen[u]], tok1[u, : olen1[u]]) and np.array_equal(frm[u, : olen[u]], frm1[u, : olen1[u]]), u
+    assert stats["frames"] == int(lens.sum()) and stats["tokens"] == int(olen.sum())
+    hist = np.array(stats["jump_hist"])
+    assert (hist * np.arange(65)).sum() + stats["forced"] == int(lens.sum())
+
+
+def test_refilled_rows_random_shapes(pkg):
+    r = np.random.default_rng(21)
+    for i in range(24):
+        refill_case(pkg, r, i, 9700)

@@ -3,7 +3,9 @@
 Algorithm 2 treats the utterances of a batch independently, so what an utterance's row did before it moved in must not
 show in its transcript: every utterance's (tokens, frames) from wind_decode_greedy_refill must equal, bit for bit, the
 ones wind_decode_greedy gives for it with all N utterances in one batch (same kernel mode forced for both), for every
-number of rows -- one row (the utterances one after the other), a few, exactly N, more rows than utterances.  A sample
+number of rows -- one row (the utterances one after the other), a few, exactly N, more rows than utterances (the shapes
+are such that every row count gets the same kind of tile plan as the batch of N; the randomised sweep in
+test_gpu_fuzz.py compares against fixed batches of exactly B rows instead, which holds for any shape).  A sample
 is also replayed through the CPU oracle under the margin rule of the parity tests, and the counters are checked
 against what the transcripts say.
 """
