@@ -1595,6 +1595,11 @@ static cudaError_t loop_device_info(int* sms, int* smem_optin, int* dev_out) {
     return cudaSuccess;
 }
 
+cudaError_t loop_sm_count(int* sms) {
+    int optin = 0;
+    return loop_device_info(sms, &optin, nullptr);
+}
+
 static cudaError_t get_encode_loop() {
     std::lock_guard<std::mutex> lock(g_loop_mutex);
     if (g_encode_loop) return cudaSuccess;

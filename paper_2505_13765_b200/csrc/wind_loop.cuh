@@ -129,6 +129,7 @@ void loop_set_options(const LoopOptions& o);
 LoopOptions loop_get_options();
 bool loop_plan_ok(const wind_model_t& m, int B, int W);
 cudaError_t loop_plan(const Call& c, LoopPlan* out);
+cudaError_t loop_sm_count(int* sms);   // SMs of the current device (cached per device)
 // the plan as a pure function of the shapes and of the device's SM count and opt-in shared memory per block
 cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem_optin, LoopPlan* out, bool refill = false);
 // launchers of the two kernels (wind_loop.cu: streaming mode; wind_loop_res.cu: resident-weights mode)

@@ -252,6 +252,196 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (threadIdx.x == 0 && abort_flag) set_status(p.ctrl, WIND_ERR_TIMEOUT);
 }
 
+// ---------------------------------------------------------------------------
+// Encoder projection, persistent form: one CTA per SM walks a static list of 128 x 256 output tiles.
+//
+// Row tiles are cut per utterance (rows b T + 128 j, j < ceil(len_b / 128)), so a tile never holds two utterances and
+// the tiles of padding are never enumerated: tile k of the list is found from the prefix sums of the utterances' tile
+// counts, which every CTA builds once in shared memory.  Column tile fastest, so that the CTAs working on one row tile
+// at the same time fetch it from DRAM once.  Four TMA stages of 48 KB feed one MMA-issuing thread; the accumulator is
+// double-buffered in tensor memory (2 x 256 columns), so that the epilogue of a tile (tensor memory -> registers ->
+// + bias -> bf16 -> 64 contiguous bytes per thread and store) runs under the next tile's MMAs.  Rows past the
+// utterance's end inside a tile are computed and not stored (rows of a GEMM are independent).
+// ---------------------------------------------------------------------------
+constexpr int EP_STAGES = 4;
+constexpr int EP_BN = 256;
+constexpr uint32_t EP_STAGE_BYTES = A_STAGE_BYTES + EP_BN * BK * 2;
+constexpr int EP_MAX_UTTS = 2048;     // prefix sums in shared memory; larger sets use the one-tile-per-CTA kernel
+constexpr int EP_MAX_H = 2048;        // bias values in shared memory
+
+// 256-bit store: one full 32-byte sector per thread (16-byte stores from 32 threads to 32 different rows would touch 32
+// sectors half-filled each, twice the traffic between the SM and L2)
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t* w) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]),
+                 "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+}
+
+struct EncProjParams {
+    Ctrl* ctrl;
+    int k_blocks, H, T, n_utts;
+    const int32_t* enc_len;
+    __nv_bfloat16* out;
+    const float* bias;
+};
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+enc_proj_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const EncProjParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[EP_STAGES], empty_bar[EP_STAGES], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ int s_prefix[EP_MAX_UTTS + 1];     // s_prefix[b] = row tiles of utterances before b
+    __shared__ float s_bias[EP_MAX_H];
+    __shared__ int s_scan[GEMM_THREADS / 32];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    if (p.ctrl->bad_input) return;   // a length outside [0, T]: nothing is read through it
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < EP_STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&acc_full[a], 1); mbar_init(&acc_empty[a], 4); }
+        fence_barrier_init();
+        prefetch_tmap(&map_a); prefetch_tmap(&map_b);
+    }
+    if (warp == 1) tmem_alloc(&tmem_slot, 512);
+    for (int i = threadIdx.x; i < p.H; i += GEMM_THREADS) s_bias[i] = p.bias[i];
+    // exclusive prefix sums of the utterances' row-tile counts (block-wide scan, GEMM_THREADS utterances per round)
+    {
+        int carry = 0;
+        for (int b0 = 0; b0 < p.n_utts; b0 += GEMM_THREADS) {
+            const int b = b0 + (int)threadIdx.x;
+            const int cnt = b < p.n_utts ? (p.enc_len[b] + BM - 1) / BM : 0;
+            int incl = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            if (lane == 31) s_scan[warp] = incl;
+            __syncthreads();
+            int before = carry;
+            for (int w = 0; w < warp; ++w) before += s_scan[w];
+            if (b < p.n_utts) s_prefix[b] = before + incl - cnt;
+            int total = 0;
+            for (int w = 0; w < GEMM_THREADS / 32; ++w) total += s_scan[w];
+            carry += total;
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) s_prefix[p.n_utts] = carry;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+
+    const int n_col_tiles = (p.H + EP_BN - 1) / EP_BN;
+    const int n_tiles = s_prefix[p.n_utts] * n_col_tiles;
+    // tile k -> (utterance, row tile inside it, column tile)
+    auto locate = [&](int k, int& b, int& j, int& nt) {
+        const int mt = k / n_col_tiles;
+        nt = k - mt * n_col_tiles;
+        int lo = 0, hi = p.n_utts;            // the last b with s_prefix[b] <= mt (utterances without frames have no tile)
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (s_prefix[mid] <= mt) lo = mid; else hi = mid;
+        }
+        b = lo;
+        j = mt - s_prefix[lo];
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int k = blockIdx.x; k < n_tiles && ok; k += gridDim.x) {
+                int b, j, nt;
+                locate(k, b, j, nt);
+                const int row0 = b * p.T + j * BM;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % EP_STAGES;
+                    if (!mbar_wait(&empty_bar[s], ((it / EP_STAGES) & 1) ^ 1, &abort_flag)) { ok = false; break; }
+                    uint8_t* a_dst = smem + (size_t)s * EP_STAGE_BYTES;
+                    mbar_expect_tx(&full_bar[s], EP_STAGE_BYTES);
+                    tma_load_2d(a_dst, &map_a, kb * BK, row0, &full_bar[s]);
+                    tma_load_2d(a_dst + A_STAGE_BYTES, &map_b, kb * BK, nt * EP_BN, &full_bar[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            uint32_t it = 0, n_acc = 0;
+            bool ok = true;
+            for (int k = blockIdx.x; k < n_tiles && ok; k += gridDim.x, ++n_acc) {
+                const int nt = k % n_col_tiles;
+                const int n_cols = min(EP_BN, p.H - nt * EP_BN);            // a multiple of 64
+                const uint32_t idesc = idesc_bf16(BM, n_cols);
+                const uint32_t a = n_acc & 1u;
+                if (!mbar_wait(&acc_empty[a], ((n_acc >> 1) & 1u) ^ 1u, &abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tm_d = tmem_base + a * EP_BN;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % EP_STAGES;
+                    if (!mbar_wait(&full_bar[s], (it / EP_STAGES) & 1, &abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(smem + (size_t)s * EP_STAGE_BYTES);
+                    const uint64_t adesc = smem_desc_sw128(a_addr);
+                    const uint64_t bdesc = smem_desc_sw128(a_addr + A_STAGE_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk)
+                        tc_mma_bf16(tm_d, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), idesc, (kb | kk) != 0);
+                    tc_commit(&empty_bar[s]);
+                }
+                if (ok) tc_commit(&acc_full[a]);
+            }
+        }
+    } else {
+        const int q = warp & 3;            // tensor-memory lane quadrant this warp may read
+        const int row = q * 32 + lane;     // accumulator row of this thread
+        uint32_t n_acc = 0;
+        for (int k = blockIdx.x; k < n_tiles; k += gridDim.x, ++n_acc) {
+            int b, j, nt;
+            locate(k, b, j, nt);
+            const int n_cols = min(EP_BN, p.H - nt * EP_BN);
+            const bool valid = j * BM + row < p.enc_len[b];
+            __nv_bfloat16* dst = p.out + ((size_t)b * p.T + (size_t)j * BM + row) * p.H + (size_t)nt * EP_BN;
+            const float* bias = s_bias + nt * EP_BN;
+            const uint32_t a = n_acc & 1u;
+            const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[a], (n_acc >> 1) & 1u, &abort_flag));
+            if (!ready) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + a * EP_BN + ((uint32_t)(q * 32) << 16);
+            for (int c0 = 0; c0 < n_cols; c0 += 32) {
+                float v[32];
+                tmem_ld16(taddr + c0, v);
+                tmem_ld16(taddr + c0 + 16, v + 16);
+                if (valid) {
+                    uint32_t w[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) w[i] = pack_bf16x2(v[2 * i] + bias[c0 + 2 * i], v[2 * i + 1] + bias[c0 + 2 * i + 1]);
+                    // whole 32-byte sectors per store (a row's segment is 32-byte aligned: H is a multiple of 64)
+                    st_global_v8(dst + c0, w);
+                    st_global_v8(dst + c0 + 16, w + 8);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[a]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && abort_flag) set_status(p.ctrl, WIND_ERR_TIMEOUT);
+}
+
+constexpr size_t enc_proj_smem_bytes() { return (size_t)EP_STAGES * EP_STAGE_BYTES + 1024; }
+
 template <int MODE>
 constexpr size_t gemm_smem_bytes() { return (size_t)GemmShape<MODE>::STAGES * (A_STAGE_BYTES + (size_t)GemmShape<MODE>::BN * BK * 2) + 1024; }
 
@@ -267,12 +457,27 @@ static cudaError_t tc_set_attributes() {
     if (done) return cudaSuccess;
     if ((e = cudaFuncSetAttribute(gemm_kernel<MODE_ENC_PROJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem_bytes<MODE_ENC_PROJ>())) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(gemm_kernel<MODE_GATE_TABLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_smem_bytes<MODE_GATE_TABLE>())) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(enc_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)enc_proj_smem_bytes())) != cudaSuccess) return e;
     done = true;
     return cudaSuccess;
 }
 
 cudaError_t tc_enc_proj(const Call& c) {
     const TcMaps& M = *static_cast<const TcMaps*>(c.tc);
+    const int n_utts = c.N > 0 ? c.N : c.B;
+    if (n_utts <= EP_MAX_UTTS && c.m.H <= EP_MAX_H) {
+        EncProjParams q{};
+        q.ctrl = c.ctrl();
+        q.k_blocks = c.m.D / BK; q.H = c.m.H; q.T = c.T; q.n_utts = n_utts;
+        q.enc_len = c.enc_len; q.out = (__nv_bfloat16*)c.enc_proj(); q.bias = c.m.b_enc;
+        int sms = 0;
+        cudaError_t e = loop_sm_count(&sms);
+        if (e != cudaSuccess) return e;
+        const long long most = ((long long)n_utts * ((c.T + BM - 1) / BM)) * ((c.m.H + EP_BN - 1) / EP_BN);
+        const int grid = (int)(most < sms ? (most < 1 ? 1 : most) : sms);
+        enc_proj_kernel<<<grid, GEMM_THREADS, enc_proj_smem_bytes(), c.stream>>>(M.enc, M.w_enc, q);
+        return cudaGetLastError();
+    }
     GemmParams p{};
     p.ctrl = c.ctrl();
     p.k_blocks = c.m.D / BK;
