@@ -111,3 +111,22 @@ def test_refill_rejects_what_it_does_not_cover(pkg):
     assert pkg.decode_refill(model, enc, bad, 2, 4, 3, check=False)[4] == bd.WIND_ERR_INVALID_ARG
     ok = pkg.decode_refill(model, enc, lens, 2, 4, 3)                                                # the context is fine
     assert ok[4] == 0
+
+
+def test_a_queue_longer_than_the_projection_kernels_prefix_table(pkg):
+    # more than 2048 utterances: the encoder projection takes its one-tile-per-CTA form (the persistent kernel keeps the
+    # utterances' tile counts in shared memory); short utterances, every one checked against fixed batches of 64 rows
+    N, T, B, W, S = 2100, 6, 64, 4, 2
+    w, enc, lens = ragged_case(804, B=N, T=T, D=64, E=64, P=64, L=1, H=128, V=140, bias=1.0, dtype="bf16")
+    enc = np.nan_to_num(enc)
+    model = pkg.WindModel(w)
+    tok, frm, olen, stats, st = pkg.decode_refill(model, enc, lens, B, W, S)
+    assert st == 0 and stats["frames"] == int(lens.sum()) and stats["tokens"] == int(olen.sum())
+    for k in range(0, N, B):
+        m = min(B, N - k)
+        e = np.zeros((B, T, 64), np.float32); l = np.zeros(B, np.int32)
+        e[:m], l[:m] = enc[k: k + m], lens[k: k + m]
+        t1, f1, o1, _, st1 = pkg.decode(model, e, l, W, S)
+        assert st1 == 0 and np.array_equal(o1[:m], olen[k: k + m])
+        for u in range(m):
+            assert np.array_equal(t1[u, : o1[u]], tok[k + u, : o1[u]]) and np.array_equal(f1[u, : o1[u]], frm[k + u, : o1[u]])
