@@ -1169,6 +1169,99 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     asm volatile("bar.sync 1, 128;" ::: "memory");
                     if (e == 0) s_active = s_red[0] + s_red[1] + s_red[2] + s_red[3];
                 }
+                // Projection epilogue of the streaming mode.  The accumulator holds pred_proj[utterance (lane), np columns];
+                // it goes through shared memory, and the z rows are then built by ALL epilogue threads: work item =
+                // (utterance, window row), 2 x 16 bytes of enc_proj each, four items per thread and round with their
+                // loads requested together.  (One thread per utterance, as the accumulator is laid out, left three
+                // quarters of the threads idle for batches of 32 and took W dependent rounds of loads.)
+                if (p.W > 4) {
+                float* pst = stage_f;                                                   // [128][np] pred_proj + b_pred
+                for (int i = i0; i < p.p_items; i += G) {
+                    const int mt = i / p.hg_count, hg = i - mt * p.hg_count;
+                    const int h0 = hg * p.np;
+                    const int rows_here = min(128, p.B - mt * 128);
+                    const int total = rows_here * p.W;
+                    // this thread's first four items, requested before the accumulator is ready
+                    uint4 ev[4][2];
+                    int it_r[4], it_w[4], it_n[4];
+                    auto fetch = [&](int base) {
+                        int t[4], len[4], row[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const int idx = base + k * 128 + e;
+                            it_n[k] = 0; it_r[k] = 0; it_w[k] = 0;
+                            t[k] = 0; len[k] = 0; row[k] = 0;
+                            if (idx < total) {
+                                it_r[k] = idx / p.W;
+                                it_w[k] = idx - it_r[k] * p.W;
+                                const int b = mt * 128 + it_r[k];
+                                t[k] = t_new[b]; len[k] = len_new[b]; row[k] = row_new[b];
+                            }
+                        }
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const int idx = base + k * 128 + e;
+                            if (idx < total) {
+                                it_n[k] = min(p.W, (len[k] & kSlotLenMask) - t[k]);   // <= 0 when the utterance is done
+                                if (it_w[k] < it_n[k]) {
+                                    const uint4* src = reinterpret_cast<const uint4*>(
+                                        p.enc_proj + ((size_t)row[k] + t[k] + it_w[k]) * p.H + h0);
+                                    ev[k][0] = src[0];
+                                    ev[k][1] = src[1];
+                                }
+                            }
+                        }
+                    };
+                    fetch(0);
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_TOK);
+                    const bool ready = __all_sync(0xffffffffu, mbar_wait(&acc_full[2], acc_n[2] & 1u, &s_abort));
+                    tc_fence_after();
+                    if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_ACC);
+                    if (ready) {
+                        float g[16];
+                        tmem_ld16(tm_p + lane_off, g);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) pst[row_in_tile * 16 + j] = g[j] + p.b_pred[h0 + j];
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[2]);
+                    ++acc_n[2];
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (ready) {
+                        for (int base = 0; base < total; base += 512) {
+                            if (base > 0) fetch(base);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                if (it_n[k] <= 0) continue;            // outside the batch, or the utterance is done: nothing to write
+                                uint4 o0 = make_uint4(0, 0, 0, 0), o1 = make_uint4(0, 0, 0, 0);
+                                if (it_w[k] < it_n[k]) {
+                                    const float* g = pst + it_r[k] * 16;
+                                    const __nv_bfloat162* eb = reinterpret_cast<const __nv_bfloat162*>(&ev[k][0]);
+                                    uint32_t wds[8];
+#pragma unroll
+                                    for (int c = 0; c < 8; ++c) {
+                                        const float2 e2 = __bfloat1622float2(eb[c]);
+                                        float z0 = e2.x + g[2 * c], z1 = e2.y + g[2 * c + 1];
+                                        z0 = p.act == WIND_ACT_RELU ? fmaxf(z0, 0.f) : tanh_fast(z0);
+                                        z1 = p.act == WIND_ACT_RELU ? fmaxf(z1, 0.f) : tanh_fast(z1);
+                                        wds[c] = pack_bf16x2(z0, z1);
+                                    }
+                                    o0 = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+                                    o1 = make_uint4(wds[4], wds[5], wds[6], wds[7]);
+                                }
+                                uint4* dst = reinterpret_cast<uint4*>(p.z + ((size_t)(mt * 128 + it_r[k]) * p.W + it_w[k]) * p.H + h0);
+                                dst[0] = o0;
+                                dst[1] = o1;
+                            }
+                        }
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");   // the staging arrays are reused by the CTA's next item
+                    if (s_abort) break;                               // the same decision in all four warps
+                }
+                } else {
+                // narrow windows: one thread per utterance (its accumulator lane), every load requested before the
+                // accumulator is ready; the staging above would only add a block barrier
                 for (int i = i0; i < p.p_items; i += G) {
                     const int mt = i / p.hg_count, hg = i - mt * p.hg_count;
                     const int b = mt * 128 + row_in_tile;
@@ -1245,6 +1338,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                     if (lane == 0) mbar_arrive(&acc_empty[2]);
                     ++acc_n[2];
                     if (!ready) break;
+                }
                 }
                 fence_proxy_async_all();
                 if (e == 0) if constexpr (FULL) trace_event(p, 2, tr_n, step, TR_P, EV_EPI_DONE);
@@ -1693,7 +1787,10 @@ cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem
     }
     pl.stat_bytes = pl.j_mode == J_SMEM ? stat_bytes : 0;
     pl.stage_j = ((pl.j_mode == J_STREAM ? LOOP_A_BYTES : 0u) + (uint32_t)pl.nj * BK * 2 + 1023u) / 1024u * 1024u;
-    const long long ring = (long long)budget - pl.stat_bytes;
+    // behind the ring: staging of the projection epilogue (pred_proj of a 128-utterance tile, np = 16 columns)
+    const uint32_t p_staging = 128u * (uint32_t)pl.np * 4u;
+    // (this mode's kernels have 1.6 KB of static shared memory, not the 4 KB the budget sets aside: half of the difference goes to the ring)
+    const long long ring = (long long)budget + 2048 - pl.stat_bytes - p_staging;
     pl.stages_lp = (int)(ring / pl.stage_lp);
     pl.stages_j = (int)(ring / pl.stage_j);
     if (pl.stages_lp > LOOP_MAX_STAGES) pl.stages_lp = LOOP_MAX_STAGES;
@@ -1704,7 +1801,8 @@ cudaError_t loop_plan_for(const wind_model_t& m, int B, int W, int sms, int smem
     pl.tm_p = pl.tm_l + 4 * pl.slots;
     if (pl.tm_p + pl.np > (int)LOOP_TMEM_COLS) streaming_ok = false;
     const uint32_t ring_lp = (uint32_t)(pl.stages_lp > 0 ? pl.stages_lp : 0) * pl.stage_lp, ring_j = (uint32_t)(pl.stages_j > 0 ? pl.stages_j : 0) * pl.stage_j;
-    pl.smem_bytes = pl.stat_bytes + (ring_lp > ring_j ? ring_lp : ring_j) + 1024;
+    pl.stage_off = pl.stat_bytes + (ring_lp > ring_j ? ring_lp : ring_j);
+    pl.smem_bytes = pl.stage_off + p_staging + 1024;
 
     // Resident-weights mode (one or two LSTM layers): the W_out tile of a CTA in tensor memory, W_hh in tiles of 4 gates x
     // 16 units and W_pred in tiles of 64 rows in the shared memory of disjoint CTA sets, for the whole decode; per step a

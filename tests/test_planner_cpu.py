@@ -14,6 +14,7 @@ import paper_2505_13765_b200 as pkg
 from paper_2505_13765_b200 import binding as bd
 
 STATIC_SMEM = 4096      # what the planner leaves for the kernels' static shared memory
+STREAMING_STATIC_SMEM = 2048   # the streaming-mode kernels declare 1.6 KB
 ALIGN_SLACK = 1024      # the kernels align their dynamic shared memory to 1 KB themselves
 
 
@@ -34,7 +35,8 @@ def check_plan(dims, B, W, sms, optin, pl):
     G = pl["grid"]
     assert G == sms
     usable = pl["smem_bytes"] - ALIGN_SLACK          # after the kernel's own alignment
-    assert pl["smem_bytes"] <= optin - STATIC_SMEM, "more dynamic shared memory than the device grants beside the static part"
+    static = STATIC_SMEM if pl["resident"] else STREAMING_STATIC_SMEM
+    assert pl["smem_bytes"] <= optin - static, "more dynamic shared memory than the device grants beside the static part"
     assert pl["vt_count"] == (NV + 127) // 128
     rows = B * W
     assert pl["nj"] % 16 == 0 and pl["rg_count"] == (rows + pl["nj"] - 1) // pl["nj"]
@@ -81,6 +83,9 @@ def check_plan(dims, B, W, sms, optin, pl):
         assert pl["stages_lp"] >= 2 and pl["stages_j"] >= 2
         ring = max(pl["stages_lp"] * pl["stage_lp"], pl["stages_j"] * pl["stage_j"])
         assert pl["tile_bytes"] + ring <= usable
+        # staging of the projection epilogue behind the ring: pred_proj of a 128-utterance tile
+        assert pl["np"] == 16 and pl["stage_off"] == pl["tile_bytes"] + ring
+        assert pl["stage_off"] + 128 * pl["np"] * 4 <= usable, "projection staging runs past the launch's shared memory"
         a_bytes = 128 * 64 * 2
         assert pl["stage_lp"] >= a_bytes + max(4 * pl["slots"], pl["np"]) * 64 * 2
         assert pl["stage_j"] >= (a_bytes if pl["j_mode"] == 0 else 0) + pl["nj"] * 64 * 2
