@@ -538,10 +538,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
         int32_t* t_nxt = p.t2 + (size_t)((step + 1) & 1) * p.B;
         const unsigned long long* keys_cur = p.keys2 + (size_t)(step & 1) * p.rows_pad;
         unsigned long long* keys_nxt = p.keys2 + (size_t)((step + 1) & 1) * p.rows_pad;
-        const int32_t* len_cur = p.slot_len2 + (size_t)(step & 1) * p.B;
-        int32_t* len_nxt = p.slot_len2 + (size_t)((step + 1) & 1) * p.B;
-        const int32_t* row_cur = p.slot_row2 + (size_t)(step & 1) * p.B;
-        int32_t* row_nxt = p.slot_row2 + (size_t)((step + 1) & 1) * p.B;
+        const int cur_off = (step & 1) * p.B, nxt_off = p.B - cur_off;   // the slot arrays' copy of this step and of the next
         const int u16 = lane & 15, half = lane >> 4;
         const int unit = r_ut * 16 + u16;        // this thread's hidden unit; its gate is q
         // without recording CTAs, the two gate-0 warps of one CTA per utterance group record the step
@@ -566,11 +563,11 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             si.t = 0; si.len = 0; si.cnt = 0; si.pos = 0;
 #pragma unroll
             for (int j = 0; j < 8; ++j) si.kk[j] = 0ull;
-            int s_row = 0, s_utt = 0;
+            int s_row = 0;
             if (in && decode) {
                 si.t = t_cur[b];
-                si.len = len_cur[b];
-                if (writer) { si.cnt = p.count[b]; si.pos = p.slot_pos[b]; s_row = row_cur[b]; s_utt = p.slot_utt[b]; }
+                si.len = p.slot_len2[cur_off + b];
+                if (writer) { si.cnt = p.count[b]; si.pos = p.slot_pos[b]; s_row = p.slot_row2[cur_off + b]; }
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
                     if (j < p.W) si.kk[j] = keys_cur[(size_t)b * p.W + j];
@@ -588,7 +585,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
             if (in) {
                 if (step < 0) {
                     tok = p.blank;
-                    if (writer) { t_row = (uint32_t)row_cur[b]; t_left = len_cur[b] & kSlotLenMask; }   // frame 0 of the row's first utterance
+                    if (writer) { t_row = (uint32_t)p.slot_row2[cur_off + b]; t_left = p.slot_len2[cur_off + b] & kSlotLenMask; }   // frame 0 of the row's first utterance
                 } else if ((FULL && p.forced)) {
                     tok = step < p.prefix_len[b] ? p.prefix[(size_t)b * p.U + step] : -1;
                     if (tok >= p.NV || tok < -1) { tok = p.blank; set_status(p.ctrl, WIND_ERR_INVALID_ARG); }   // caller's mistake
@@ -650,6 +647,7 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                                 if (first > 0) cnt = 0;
                                 t += first;
                                 if (si.pos < p.max_out) {
+                                    const int s_utt = p.slot_utt[b];   // which utterance the row decodes (index into the outputs)
                                     p.out_tokens[(size_t)s_utt * p.max_out + si.pos] = label;
                                     p.out_frames[(size_t)s_utt * p.max_out + si.pos] = t;
                                     p.out_len[s_utt] = si.pos + 1;
@@ -696,8 +694,8 @@ __global__ void __launch_bounds__(RES ? LOOP_THREADS_RES : LOOP_THREADS, 1) loop
                         }
                     }
                     if (writer) {
-                        len_nxt[b] = len_out;
-                        row_nxt[b] = row_out;
+                        p.slot_len2[nxt_off + b] = len_out;
+                        p.slot_row2[nxt_off + b] = row_out;
                         t_row = (uint32_t)row_out + (uint32_t)t_out;
                         t_left = (len_out & kSlotLenMask) - t_out;
                     }
