@@ -526,15 +526,32 @@ def wind_plan_batches(lens_np: np.ndarray, B: int):
     return order[:N], batch_T[: nb.value]
 
 
-def decode_dataset(model: WindModel, utterances, W: int, S: int, B: int, plan: bool = True, window_greedy: bool = False):
-    """Decodes a list of [T_i, D] numpy arrays in batches of B; results come back in the list's order.
+def decode_dataset(model: WindModel, utterances, W: int, S: int, B: int, plan: bool = True, window_greedy: bool = False,
+                   refill: bool = False):
+    """Decodes a list of [T_i, D] numpy arrays on B batch rows; results come back in the list's order.
 
     plan=True groups utterances of similar length (wind_plan_batches); plan=False keeps the arrival order.  Packing the
-    batches is marshalling; every batch is one call of the decode entry point.  Returns (list of token arrays, list of
-    frame arrays, total lock steps).
+    batches is marshalling; every batch is one call of the decode entry point.  refill=True hands the whole list to
+    wind_decode_greedy_refill in ONE call (longest first when plan=True): a row takes the next utterance as soon as its
+    own is finished; models and shapes that entry point does not cover fall back to the batches.  Returns (list of token
+    arrays, list of frame arrays, total lock steps).
     """
     lens = np.array([u.shape[0] for u in utterances], np.int32)
     N = len(utterances)
+    if refill and not window_greedy and N > 0:
+        order = wind_plan_batches(lens, B)[0] if plan else np.arange(N, dtype=np.int32)
+        T = max(1, int(lens.max()))
+        enc = np.zeros((N, T, model.dims["D"]), np.float32)
+        for r, i in enumerate(order):
+            enc[r, : lens[i]] = utterances[i]
+        tok, frm, olen, stats, st = decode_refill(model, enc, lens[order], B, W, S, check=False)
+        if st == WIND_OK:
+            toks, frms = [None] * N, [None] * N
+            for r, i in enumerate(order):
+                toks[i], frms[i] = tok[r, : olen[r]].copy(), frm[r, : olen[r]].copy()
+            return toks, frms, stats["steps"]
+        if st != WIND_ERR_UNSUPPORTED:
+            raise WindError(st)
     if plan:
         order, _ = wind_plan_batches(lens, B)
     else:

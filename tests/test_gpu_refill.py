@@ -95,6 +95,17 @@ def test_refill_needs_fewer_lock_steps_than_planned_batches(pkg):
         assert np.array_equal(tok[u, : olen[u]], t_p[u]) and np.array_equal(frm[u, : olen[u]], f_p[u])
     assert stats["steps"] < steps_planned, (stats["steps"], steps_planned)
     print(f"[refill] 64 utterances on 8 rows: {stats['steps']} lock steps refilled, {steps_planned} in length-sorted batches")
+    # the list helper: refilled rows, longest first, results back in the list's order; an fp32 model falls back to batches
+    t_r, f_r, steps_r = pkg.decode_dataset(model, utts, 4, 3, B=8, plan=True, refill=True)
+    for u in range(64):
+        assert np.array_equal(t_r[u], t_p[u]) and np.array_equal(f_r[u], f_p[u])
+    assert steps_r < steps_planned
+    w32, enc32, lens32 = ragged_case(805, B=10, T=12, D=64, E=64, P=64, L=1, H=64, V=140, dtype="f32")
+    m32 = pkg.WindModel(w32)
+    u32 = [np.ascontiguousarray(np.nan_to_num(enc32)[b, : lens32[b]]) for b in range(10)]
+    a = pkg.decode_dataset(m32, u32, 4, 3, B=4, refill=True)
+    b = pkg.decode_dataset(m32, u32, 4, 3, B=4, refill=False)
+    assert all(np.array_equal(x, y) for x, y in zip(a[0], b[0])) and a[2] == b[2]
 
 
 def test_refill_rejects_what_it_does_not_cover(pkg):
