@@ -34,6 +34,7 @@ class OracleModel(C.Structure):
         ("w_enc", f32p), ("b_enc", f32p),
         ("w_pred", f32p), ("b_pred", f32p),
         ("w_out", f32p), ("b_out", f32p),
+        ("round_bf16", C.c_int32),
     ]
 
 
@@ -69,6 +70,8 @@ def lib():
         mp = C.POINTER(OracleModel)
         L.oracle_linear.argtypes = [f32p, f32p, f64p, C.c_int, C.c_int, f64p]
         L.oracle_linear.restype = None
+        L.oracle_bf16_round.argtypes = [C.c_double]
+        L.oracle_bf16_round.restype = C.c_double
         L.oracle_lstm_step.argtypes = [mp, C.c_int32, f64p, f64p]
         L.oracle_lstm_step.restype = None
         L.oracle_pred_proj.argtypes = [mp, f64p, f64p]
@@ -118,7 +121,9 @@ def _ptr(a: np.ndarray, t):
 class Model:
     """Holds fp32 copies of the weights and the C struct that points at them."""
 
-    def __init__(self, w: Dict[str, object]):
+    def __init__(self, w: Dict[str, object], round_bf16: bool = False):
+        """round_bf16: enc_proj, the LSTM hidden state and the joint's activations are rounded to bf16 where they are
+        produced (the places a bf16 implementation rounds its matrix operands); the default keeps fp64 throughout."""
         self.dims = {k: int(w[k]) for k in ("D", "E", "P", "L", "H", "V", "blank_id", "act")}
         L = self.dims["L"]
         self._keep = []
@@ -142,6 +147,7 @@ class Model:
             w_enc=keep(w["w_enc"]), b_enc=keep(w["b_enc"]),
             w_pred=keep(w["w_pred"]), b_pred=keep(w["b_pred"]),
             w_out=keep(w["w_out"]), b_out=keep(w["b_out"]),
+            round_bf16=int(bool(round_bf16)),
         )
 
     @property
@@ -286,6 +292,11 @@ def linear(Wm: np.ndarray, b: Optional[np.ndarray], x: np.ndarray) -> np.ndarray
     bp = _ptr(_f32(b), f32p) if b is not None else None
     lib().oracle_linear(_ptr(Wm, f32p), bp, _ptr(x, f64p), Wm.shape[0], Wm.shape[1], _ptr(y, f64p))
     return y
+
+
+def bf16_round(x: float) -> float:
+    """The oracle's own rounding of one value to bf16 (what Model(round_bf16=True) applies)."""
+    return float(lib().oracle_bf16_round(float(x)))
 
 
 def lstm_step(model: Model, tok: int, h: np.ndarray, c: np.ndarray):

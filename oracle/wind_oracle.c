@@ -30,6 +30,11 @@
  * over all alignments for every window (brute force on independently evaluated logits), hand-worked examples, and
  * the optional prefix step against independently evaluated completions.
  *
+ * Precision: fp64 throughout by default.  With round_bf16 set in the model, enc_proj, the LSTM hidden state and the joint's
+ * activations are rounded to bf16 where they are produced and everything else stays fp64 (the paper runs its models under
+ * bf16 autocast and names no rounding points; these three are the matrix operands of a bf16 implementation).  Pins of this
+ * mode: the rounding against a library conversion, and each of the three places against a step-by-step recomputation.
+ *
  * Pins (see tests): WIND(W) == sequential for every W; brute-force tabulation
  * of joint argmaxes on tiny models; LSTM / linear layers against library fp64
  * routines and closed forms; S honoured; jump-size support.
@@ -56,6 +61,12 @@ typedef struct {
     const float* b_pred;      /* [H] */
     const float* w_out;       /* [V+1, H] */
     const float* b_out;       /* [V+1] */
+    int32_t round_bf16;       /* 0: fp64 throughout.  1: the three intermediate quantities that a bf16 implementation keeps
+                                 as matrix operands -- enc_proj, the LSTM hidden state h, and the joint's activations
+                                 act(enc_proj + pred_proj) -- are rounded to bf16 (nearest even) where they are produced;
+                                 everything else (sums, cell state c, pred_proj, logits) stays fp64.  The paper runs its
+                                 models under bf16 autocast and fixes no rounding points; these are the ones a decision
+                                 taken "in the kernel's precision" has to share. */
 } oracle_model_t;
 
 typedef struct {
@@ -83,6 +94,18 @@ void oracle_linear(const float* W, const float* b, const double* x, int n_out, i
 
 static double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
 
+/* nearest bf16 value (ties to even) of x: fp32 first, then the upper 16 bits of its pattern */
+double oracle_bf16_round(double x) {
+    float f = (float)x;
+    uint32_t u;
+    memcpy(&u, &f, sizeof(u));
+    if ((u & 0x7F800000u) == 0x7F800000u) return (double)f;   /* infinities and NaN pass */
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    u &= 0xFFFF0000u;
+    memcpy(&f, &u, sizeof(f));
+    return (double)f;
+}
+
 /*
  * One LSTM stack update for one token.  h, c: [L, P] fp64, updated in place.
  * Layer l: gates = W_ih x + b_ih + W_hh h + b_hh, split as (i, f, g, o);
@@ -108,6 +131,7 @@ void oracle_lstm_step(const oracle_model_t* m, int32_t tok, double* h, double* c
             double go = sigmoid(ga[3 * P + j] + gb[3 * P + j]);
             cl[j] = gf * cl[j] + gi * gg;
             hl[j] = go * tanh(cl[j]);
+            if (m->round_bf16) hl[j] = oracle_bf16_round(hl[j]);
         }
         for (int j = 0; j < P; ++j) x[j] = hl[j];
         n_in = P;
@@ -126,6 +150,8 @@ void oracle_enc_proj(const oracle_model_t* m, const float* enc, int T, double* o
     for (int t = 0; t < T; ++t) {
         for (int k = 0; k < m->D; ++k) x[k] = (double)enc[(size_t)t * m->D + k];
         oracle_linear(m->w_enc, m->b_enc, x, m->H, m->D, out + (size_t)t * m->H);
+        if (m->round_bf16)
+            for (int k = 0; k < m->H; ++k) out[(size_t)t * m->H + k] = oracle_bf16_round(out[(size_t)t * m->H + k]);
     }
     free(x);
 }
@@ -135,6 +161,7 @@ void oracle_joint_logits(const oracle_model_t* m, const double* encp, const doub
     for (int k = 0; k < m->H; ++k) {
         double s = encp[k] + g[k];
         z[k] = (m->act == 0) ? (s > 0.0 ? s : 0.0) : tanh(s);
+        if (m->round_bf16) z[k] = oracle_bf16_round(z[k]);
     }
     oracle_linear(m->w_out, m->b_out, z, m->V + 1, m->H, logits);
 }

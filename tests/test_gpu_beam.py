@@ -46,10 +46,12 @@ def small_model(seed, dtype="f32", V=37, L=1, act=0, blank0=False, bias=1.5):
     return w, r
 
 
-def compare(pkg, w, enc, W, K, S, gap_needed, tol, prefix_search=False):
-    """Returns True when the case was decidable and the GPU agreed with the oracle."""
+def compare(pkg, w, enc, W, K, S, gap_needed, tol, prefix_search=False, round_bf16=False):
+    """Returns True when the case was decidable and the GPU agreed with the oracle (round_bf16: the oracle that rounds
+    enc_proj, the hidden state and the joint's activations to bf16 where the bf16 kernels do)."""
     T = enc.shape[0]
-    want, gap, steps = oracle.beam_search(oracle.Model(w), enc, T, W, K, S, max_hyps=256, prefix_search=prefix_search)
+    want, gap, steps = oracle.beam_search(oracle.Model(w, round_bf16=round_bf16), enc, T, W, K, S, max_hyps=256,
+                                          prefix_search=prefix_search)
     got, gsteps, st = pkg.wind_beam_search(pkg.WindModel(w), enc, W, K, S, max_hyps=256, prefix_search=prefix_search)
     assert st == 0 and len(got) >= 1
     for tok, frm, sc in got:                      # always: well-formed hypotheses
@@ -145,6 +147,37 @@ def test_bf16_best_score_is_close_to_the_oracle(pkg):
         assert abs(got[0][2] - want[0][2]) < 0.02 * (len(want[0][0]) + T), (got[0][2], want[0][2])
         same += list(got[0][0]) == list(want[0][0])
     print(f"[beam bf16] best hypothesis equal to the oracle's in {same}/6 cases")
+
+
+@pytest.mark.parametrize("W,K,S,L,blank0,act,prefix", [(1, 2, 3, 1, False, 0, False), (4, 3, 3, 1, True, 1, False),
+                                                      (8, 4, 2, 2, False, 0, False), (4, 2, 3, 1, False, 0, True),
+                                                      (16, 4, 4, 1, True, 0, False)])
+def test_bf16_matches_the_oracle_that_rounds_where_the_kernels_do(pkg, W, K, S, L, blank0, act, prefix):
+    # bf16 weights: the kernels round enc_proj, the hidden state and the joint's activations to bf16.  Against the oracle
+    # in the same precision (Model(round_bf16=True): fp64 sums, the same three roundings) what is left is the kernels' fp32
+    # accumulation: scores agree to about 1e-6, except where an fp32 sum falls on the other side of a bf16 rounding
+    # boundary than the fp64 sum (one last-place step of one value: up to about 1e-3 in a score).  A case is decidable
+    # when the oracle's smallest deciding difference is four times the largest score difference measured in it; then
+    # every final hypothesis (tokens, frames) and the number of iterations must be the oracle's.
+    decided = 0
+    for seed in range(8):
+        w, r = small_model(500 + seed + 10 * W, dtype="bf16", L=L, act=act, blank0=blank0, bias=2.5)
+        T = int(r.integers(12, 24))
+        enc = ws.bf16_round(r.standard_normal((T, 24)).astype(np.float32))
+        want, gap, steps = oracle.beam_search(oracle.Model(w, round_bf16=True), enc, T, W, K, S, max_hyps=256, prefix_search=prefix)
+        got, gsteps, st = pkg.wind_beam_search(pkg.WindModel(w), enc, W, K, S, max_hyps=256, prefix_search=prefix)
+        assert st == 0 and len(got) >= 1
+        a = {tuple(int(x) for x in h[0]): h for h in want}
+        b = {tuple(int(x) for x in h[0]): h for h in got}
+        worst = max((abs(a[k][2] - b[k][2]) for k in a if k in b), default=0.0)
+        assert worst < 5e-3, (seed, worst)
+        if gap >= 4 * max(worst, 1e-6):
+            assert gsteps == steps and set(a) == set(b), (seed, gap, worst)
+            assert all(list(a[k][1]) == list(b[k][1]) for k in a)
+            assert list(got[0][0]) == list(want[0][0])
+            decided += 1
+    print(f"[beam bf16] W={W} K={K} S={S} prefix={prefix}: {decided}/8 cases decidable and equal to the rounding oracle")
+    assert decided >= 5
 
 
 def test_beam_one_equals_window_based_greedy_on_the_gpu(pkg):

@@ -35,8 +35,10 @@ def pkg():
     return p
 
 
-def check_against_oracle(pkg, weights, enc, lens, W, S, kernels=0, expect_exact=None, sample=None):
-    """Decode on the GPU, compare with the oracle.  Returns a report dict."""
+def check_against_oracle(pkg, weights, enc, lens, W, S, kernels=0, expect_exact=None, sample=None, round_bf16=False,
+                         margin=MARGIN):
+    """Decode on the GPU, compare with the oracle.  Returns a report dict.  round_bf16: the oracle that rounds enc_proj,
+    the hidden state and the joint's activations to bf16 where the bf16 kernels do (a smaller margin can then be asked)."""
     prev = pkg.wind_set_kernels(kernels)
     try:
         model = pkg.WindModel(weights)
@@ -44,15 +46,15 @@ def check_against_oracle(pkg, weights, enc, lens, W, S, kernels=0, expect_exact=
     finally:
         pkg.wind_set_kernels(prev)
     assert st == 0
-    om = oracle.Model(weights)
+    om = oracle.Model(weights, round_bf16=round_bf16)
     B = enc.shape[0]
     idx = list(range(B)) if sample is None else list(sample)
     sub = np.ascontiguousarray(enc[idx])
-    otok, ofrm, on, ost = oracle.decode_batch(om, sub, lens[idx], W=0, S=S, max_out=tok.shape[1])
+    otok, ofrm, on, ost = oracle.decode_batch(om, sub, lens[idx], W=0, S=S, max_out=tok.shape[1], margin_thr=margin)
 
     def replay(k):
         b = idx[k]
-        return oracle.replay_verify(om, enc[b], int(lens[b]), S, tok[b, : olen[b]], frm[b, : olen[b]], MARGIN)
+        return oracle.replay_verify(om, enc[b], int(lens[b]), S, tok[b, : olen[b]], frm[b, : olen[b]], margin)
 
     with ThreadPoolExecutor(8) as ex:
         reps = list(ex.map(replay, range(len(idx))))
@@ -83,7 +85,7 @@ def check_against_oracle(pkg, weights, enc, lens, W, S, kernels=0, expect_exact=
         assert (hist * np.arange(65)).sum() + stats["forced"] == int(lens.sum())
         assert hist[W + 1:].sum() == 0
     print(f"[parity] W={W} S={S} exact {exact}/{len(idx)} utterances, {off_argmax} decisions off the oracle argmax "
-          f"(all inside {MARGIN}); oracle low-margin decisions {ost['low_margin']}/{ost['decisions']}")
+          f"(all inside {margin}); oracle low-margin decisions {ost['low_margin']}/{ost['decisions']}")
     return rep, (tok, frm, olen)
 
 
@@ -156,9 +158,10 @@ def test_fp32_joint_logits(pkg):
     logits_parity(pkg, w, enc, lens, W=4, S=3, tol=TOL["f32"], n_windows=24)
 
 
-def logits_parity(pkg, weights, enc, lens, W, S, tol, n_windows, kernels=0, seed=0):
-    """Teacher-forced logits at oracle-chosen prefixes and frames."""
-    om = oracle.Model(weights)
+def logits_parity(pkg, weights, enc, lens, W, S, tol, n_windows, kernels=0, seed=0, round_bf16=False):
+    """Teacher-forced logits at oracle-chosen prefixes and frames.  round_bf16: against the oracle that rounds enc_proj, the
+    hidden state and the joint's activations to bf16 where the bf16 kernels do."""
+    om = oracle.Model(weights, round_bf16=round_bf16)
     B, T, _ = enc.shape
     otok, ofrm, on, _ = oracle.decode_batch(om, enc, lens, W=0, S=S)
     r = np.random.default_rng(seed)
@@ -196,6 +199,7 @@ def logits_parity(pkg, weights, enc, lens, W, S, tol, n_windows, kernels=0, seed
         pkg.wind_set_kernels(prev)
     print(f"[logits] {rows} rows, worst abs error {worst:.3e} (tolerance {tol})")
     assert rows > 0 and worst < tol
+    return worst
 
 
 # ---------------------------------------------------------------------------
@@ -207,6 +211,20 @@ def test_bf16_ragged_small(pkg, kernels):
     w, enc, lens = ragged_case(40, B=6, T=45, D=40, E=24, P=40, L=2, H=56, V=35, bias=1.0, dtype="bf16")
     check_against_oracle(pkg, w, enc, lens, 4, 3, kernels=kernels)
     logits_parity(pkg, w, enc, lens, W=4, S=3, tol=TOL["bf16"], n_windows=12, kernels=kernels)
+
+
+@pytest.mark.parametrize("L,act,W", [(2, 0, 4), (1, 1, 8), (3, 0, 1)])
+def test_bf16_plain_alu_path_against_the_oracle_in_the_same_precision(pkg, L, act, W):
+    # The plain-ALU bf16 kernels round enc_proj, the hidden state and the joint's activations to bf16 and nothing else; the
+    # oracle can do the same (Model(round_bf16=True): fp64 sums, the same three roundings).  What is left between the two
+    # is fp32 accumulation: logits agree to about 1e-6 unless an fp32 sum falls on the other side of a bf16 rounding
+    # boundary than the fp64 sum (one last-place step of one value: about 1e-3 in a logit), against 2e-2 for the fp64
+    # oracle.  Transcripts: the margin rule with a margin ten times smaller.
+    w, enc, lens = ragged_case(60 + L, B=6, T=45, D=40, E=24, P=40, L=L, H=56, V=35, act=act, bias=1.0, dtype="bf16")
+    rep, _ = check_against_oracle(pkg, w, enc, lens, W, 3, kernels=1, round_bf16=True, margin=5e-3)
+    assert rep["stats"]["kernels"] == 1 and rep["exact"] >= 5
+    worst = logits_parity(pkg, w, enc, lens, W=W, S=3, tol=2e-3, n_windows=24, kernels=1, round_bf16=True)
+    print(f"[same precision] L={L} act={act}: worst logit difference {worst:.2e}, {rep['exact']}/6 transcripts equal")
 
 
 @pytest.mark.parametrize("kernels", [1, 0])

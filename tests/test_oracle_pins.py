@@ -103,6 +103,69 @@ def test_lstm_matches_torch_lstm(L):
     assert np.max(np.abs(g - ref)) < 1e-12
 
 
+def to_bf16(a):
+    """Library rounding to bf16 (torch), as fp64 numpy."""
+    return torch.as_tensor(np.asarray(a, np.float64)).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+def test_bf16_rounding_matches_the_library_conversion():
+    r = rng(31)
+    xs = np.concatenate([r.standard_normal(2000), r.standard_normal(500) * 1e-3, r.standard_normal(500) * 1e4,
+                         # exact ties between two bf16 neighbours (even and odd), and values that are already bf16
+                         np.array([1.00390625, 1.01171875, -1.00390625, 0.0, 1.0, -2.5, 3.140625])])
+    ref = to_bf16(xs)
+    got = np.array([oracle.bf16_round(x) for x in xs])
+    assert np.array_equal(got, ref)
+    assert oracle.bf16_round(1.00390625) == 1.0 and oracle.bf16_round(1.01171875) == 1.015625    # ties go to the even pattern
+
+
+@pytest.mark.parametrize("L,act", [(1, 0), (2, 1)])
+def test_rounding_mode_rounds_enc_proj_hidden_state_and_activations_and_nothing_else(L, act):
+    # Model(round_bf16=True): the three quantities a bf16 implementation keeps as matrix operands are rounded where they
+    # are produced.  Recomputed here step by step with library fp64 routines and the library's bf16 conversion.
+    r = rng(40 + L)
+    D, E, P, H, V = 6, 5, 7, 8, 9
+    w = random_weights(r, D, E, P, L, H, V, act=act, bias_scale=0.4, emb_zero_blank=False)
+    m = oracle.Model(w, round_bf16=True)
+    m0 = oracle.Model(w)
+    f64 = lambda a: np.asarray(a, np.float64)
+    enc = r.standard_normal((5, D)).astype(np.float32)
+    ep = oracle.enc_proj(m, enc)
+    ref_ep = to_bf16(f64(enc) @ f64(w["w_enc"]).T + f64(w["b_enc"]))
+    assert np.array_equal(ep, ref_ep)
+    assert np.max(np.abs(ep - oracle.enc_proj(m0, enc))) > 1e-4          # the flag does something
+    # LSTM: the rounded h is what feeds the next layer and the next update; c is not rounded
+    sig = lambda x: 1.0 / (1.0 + np.exp(-x))
+    h = np.zeros((L, P)); c = np.zeros((L, P)); hr = np.zeros((L, P)); cr = np.zeros((L, P))
+    for tok in [w["blank_id"], 3, 8, 8, 0, 1]:
+        h, c = oracle.lstm_step(m, tok, h, c)
+        x = f64(w["emb"][tok])
+        for l in range(L):
+            g = f64(w["w_ih"][l]) @ x + f64(w["b_ih"][l]) + f64(w["w_hh"][l]) @ hr[l] + f64(w["b_hh"][l])
+            gi, gf, gg, go = sig(g[:P]), sig(g[P:2 * P]), np.tanh(g[2 * P:3 * P]), sig(g[3 * P:])
+            cr[l] = gf * cr[l] + gi * gg
+            hr[l] = to_bf16(go * np.tanh(cr[l]))
+            x = hr[l]
+        assert np.array_equal(h, hr)
+        assert np.max(np.abs(c - cr)) < 1e-12
+    assert np.max(np.abs(c - to_bf16(c))) > 1e-6                           # c keeps its precision
+    # pred_proj is not rounded; the joint's activations are
+    g = oracle.pred_proj(m, h)
+    ref_g = f64(w["w_pred"]) @ hr[-1] + f64(w["b_pred"])
+    assert np.max(np.abs(g - ref_g)) < 1e-12 and np.max(np.abs(g - to_bf16(g))) > 1e-6
+    lg = oracle.joint_logits(m, ep[2], g)
+    sgm = ref_ep[2] + ref_g
+    z = to_bf16(np.maximum(sgm, 0) if act == 0 else np.tanh(sgm))
+    assert np.max(np.abs(lg - (f64(w["w_out"]) @ z + f64(w["b_out"])))) < 1e-12
+    # and the decoding entry points go through the same functions: a decode with the flag differs from one without it only
+    # through these roundings (same code path: W-invariance still holds)
+    enc_b = r.standard_normal((2, 30, D)).astype(np.float32)
+    lens = np.array([30, 17], np.int32)
+    a = oracle.decode_batch(m, enc_b, lens, W=0, S=3)
+    b = oracle.decode_batch(m, enc_b, lens, W=5, S=3)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1]) and np.array_equal(a[2], b[2])
+
+
 @pytest.mark.parametrize("act", [0, 1])
 def test_enc_proj_and_joint_match_fp64(act):
     r = rng(20 + act)
