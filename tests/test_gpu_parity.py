@@ -227,6 +227,19 @@ def test_bf16_plain_alu_path_against_the_oracle_in_the_same_precision(pkg, L, ac
     print(f"[same precision] L={L} act={act}: worst logit difference {worst:.2e}, {rep['exact']}/6 transcripts equal")
 
 
+@pytest.mark.parametrize("L", [1, 2, 3])
+def test_bf16_streaming_tensor_path_against_the_oracle_in_the_same_precision(pkg, L):
+    # The tensor-core loop in its streaming mode rounds in the same three places as the plain-ALU kernels and uses tanhf /
+    # expf in the gates, so with a ReLU joint it too is the rounding oracle up to fp32 accumulation (the kernels with
+    # resident weights also round pred_proj and use the hardware tanh: they keep the fp64 oracle and its 2e-2).
+    set_loop_mode(pkg, "streaming")
+    w, enc, lens = ragged_case(80 + L, B=9, T=14, D=64, E=64, P=64, L=L, H=64, V=140, act=0, bias=1.0, dtype="bf16")
+    rep, _ = check_against_oracle(pkg, w, enc, lens, 4, 3, kernels=2, round_bf16=True, margin=5e-3)
+    assert rep["stats"]["kernels"] == 2 and rep["exact"] >= 8
+    worst = logits_parity(pkg, w, enc, lens, W=4, S=3, tol=2e-3, n_windows=36, kernels=2, round_bf16=True)
+    print(f"[same precision, streaming] L={L}: worst logit difference {worst:.2e}, {rep['exact']}/9 transcripts equal")
+
+
 @pytest.mark.parametrize("kernels", [1, 0])
 @pytest.mark.parametrize("name,B,lo,hi,W", [
     ("cfg3_large_b128", 5, 1, 150, 8), ("cfg3_large_b128", 3, 100, 300, 1), ("cfg4_xl_r25", 4, 20, 140, 16),
