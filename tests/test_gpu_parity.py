@@ -674,3 +674,32 @@ def test_workspace_too_small_is_rejected(pkg):
     st = pkg.wind_decode_greedy(model, enc_d, torch.from_numpy(lens).to(d), 4, 3, tok, tok.clone(), tok[:, 0].clone(), small,
                                 check=False)
     assert st == pkg.binding.WIND_ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("V,B,W,resident", [(300, 40, 8, 1), (3000, 90, 16, 1), (3000, 16, 16, 0)])
+def test_joint_alone_measurement_runs_and_leaves_the_workspace_usable(pkg, V, B, W, resident):
+    # wind_bench_joint: the joint phase of the loop kernel by itself (a measurement aid).  Its figures must be consistent with
+    # the tile plan, and a decode in the same workspace right after it must be what a decode in a fresh workspace gives.
+    w, enc, lens = ragged_case(95 + B, B=B, T=16, D=64, E=64, P=128, L=1, H=128, V=V, act=0, bias=1.5, dtype="bf16")
+    enc = np.nan_to_num(enc)
+    model = pkg.WindModel(w)
+    if not resident:
+        set_loop_mode(pkg, "streaming")
+    wsb = pkg.alloc_workspace(model, B, 16, W)
+    res = pkg.wind_bench_joint(model, B, W, 20, wsb)
+    st, plan = pkg.wind_debug_plan(model.dims, B, W)
+    assert st == 0
+    assert res["iters"] == 20 and res["ms"] > 0 and res["rows"] == B * W
+    assert res["rows_issued"] >= res["rows"] and res["rows_issued"] % 16 == 0
+    assert res["labels_issued"] == ((V + 1 + 127) // 128) * 128 and 1 <= res["ctas"] <= plan["grid"]
+    assert res["resident"] == resident
+    d = model.device
+    enc_d = pkg.to_device_enc(model, enc)
+    out = []
+    for ws_used in (wsb, pkg.alloc_workspace(model, B, 16, W)):
+        tok = torch.full((B, 48), -1, dtype=torch.int32, device=d)
+        frm = tok.clone()
+        ol = torch.zeros(B, dtype=torch.int32, device=d)
+        pkg.wind_decode_greedy(model, enc_d, torch.from_numpy(lens).to(d), W, 3, tok, frm, ol, ws_used)
+        out.append((tok.cpu().numpy(), frm.cpu().numpy(), ol.cpu().numpy()))
+    assert all(np.array_equal(a, b) for a, b in zip(out[0], out[1]))
