@@ -703,3 +703,35 @@ def test_joint_alone_measurement_runs_and_leaves_the_workspace_usable(pkg, V, B,
         pkg.wind_decode_greedy(model, enc_d, torch.from_numpy(lens).to(d), W, 3, tok, frm, ol, ws_used)
         out.append((tok.cpu().numpy(), frm.cpu().numpy(), ol.cpu().numpy()))
     assert all(np.array_equal(a, b) for a, b in zip(out[0], out[1]))
+
+
+@pytest.mark.parametrize("kernels,dtype", [(1, "f32"), (2, "bf16")])
+def test_profiled_decode_gives_the_same_transcripts_and_consistent_times(pkg, kernels, dtype):
+    # wind_profile_decode (the benchmark's per-kernel timing leg): same outputs as the decode entry point; on the plain-ALU
+    # path every launch is timed (host-driven loop), on the tensor-core path the loop kernel's time is split by its phase
+    # counters, so the parts add up to the loop
+    w, enc, lens = ragged_case(97, B=12, T=30, D=64, E=64, P=64, L=2, H=64, V=140, act=0, bias=1.5, dtype=dtype)
+    enc = np.nan_to_num(enc)
+    model = pkg.WindModel(w)
+    prev = pkg.wind_set_kernels(kernels)
+    try:
+        tok0, frm0, ol0, stats0, st0 = pkg.decode(model, enc, lens, 4, 3)
+        d = model.device
+        tok = torch.full((12, 90), -1, dtype=torch.int32, device=d)
+        frm = tok.clone()
+        ol = torch.zeros(12, dtype=torch.int32, device=d)
+        wsb = pkg.alloc_workspace(model, 12, 30, 4)
+        prof = pkg.wind_profile_decode(model, pkg.to_device_enc(model, enc), torch.from_numpy(lens).to(d), 4, 3, tok, frm, ol, wsb)
+    finally:
+        pkg.wind_set_kernels(prev)
+    assert st0 == 0
+    assert np.array_equal(ol.cpu().numpy(), ol0)
+    for b in range(12):
+        assert np.array_equal(tok.cpu().numpy()[b, : ol0[b]], tok0[b, : ol0[b]]) and np.array_equal(frm.cpu().numpy()[b, : ol0[b]], frm0[b, : ol0[b]])
+    assert prof["enc_proj_ms"] > 0 and prof["joint_ms"] > 0 and prof["pred_ms"] > 0
+    if kernels == 2:
+        assert prof["loop_ms"] > 0 and prof["gate_table_ms"] > 0
+        assert abs(prof["joint_ms"] + prof["pred_ms"] - prof["loop_ms"]) < 0.05 * prof["loop_ms"]
+        assert abs(prof["lstm_ms"] + prof["proj_ms"] - prof["pred_ms"]) < 1e-6 + 0.01 * prof["pred_ms"]
+    else:
+        assert prof["joint_launches"] == stats0["steps"] and prof["control_launches"] == stats0["steps"]

@@ -140,6 +140,24 @@ def test_plan_batches_sorts_by_length_and_minimises_the_sum_of_batch_maxima(lib)
     assert lib.wind_plan_batches(neg, 2, 2, buf, None, C.byref(n)) == bd.WIND_ERR_INVALID_ARG
 
 
+def test_workspace_of_refilled_rows_holds_the_projection_of_the_whole_set(lib):
+    # wind_refill_workspace_bytes(N utterances, B rows): everything per row as in wind_workspace_bytes(B), enc_proj for N
+    m = large_model()
+    T, B, W = 500, 32, 8
+    base = pkg.wind_workspace_bytes(m, B, T, W)
+    for N in (1, 32, 33, 256):
+        n = pkg.wind_refill_workspace_bytes(m, N, T, B, W)
+        extra = max(N, B) - B
+        assert 0 <= n - base - extra * T * m.H * 2 < 4096, (N, n - base)      # bf16 enc_proj rows, up to alignment
+    nb = C.c_size_t(0)
+    assert lib.wind_refill_workspace_bytes(C.byref(m), 0, T, B, W, C.byref(nb)) == bd.WIND_ERR_INVALID_ARG
+    assert lib.wind_refill_workspace_bytes(C.byref(m), 10 ** 6, 5000, B, W, C.byref(nb)) == bd.WIND_ERR_UNSUPPORTED
+    # host staging of the host-buffer entry point: input frames and the three output arrays
+    st = pkg.wind_host_staging_bytes(m, B, T, 100)
+    assert 0 <= st - (B * T * m.D * 2 + B * 4 + 2 * B * 100 * 4 + B * 4) < 8 * 256
+    assert isinstance(lib.wind_last_cuda_error(), bytes)      # empty until a CUDA call fails
+
+
 def test_debug_hooks_round_trip(lib):
     assert pkg.wind_set_trace(5) == -2 and pkg.wind_set_trace(-9) == 5 and pkg.wind_set_trace(-2) == -2
     assert pkg.wind_debug_stall_barrier(2) == 0 and pkg.wind_debug_stall_barrier(0) == 2
