@@ -19,6 +19,25 @@ template <typename T> __device__ __forceinline__ void stf(T* p, float x);
 template <> __device__ __forceinline__ void stf<float>(float* p, float x) { *p = x; }
 template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
 
+// n consecutive weights (n a multiple of 8, src 16-byte aligned) into shared memory as floats, 16 bytes per load
+__device__ __forceinline__ void load8(const __nv_bfloat16* src, float* dst) {
+    const uint4 v = *reinterpret_cast<const uint4*>(src);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(h[i]);
+        dst[2 * i] = f.x;
+        dst[2 * i + 1] = f.y;
+    }
+}
+__device__ __forceinline__ void load8(const float* src, float* dst) {
+    const float4 a = reinterpret_cast<const float4*>(src)[0], b = reinterpret_cast<const float4*>(src)[1];
+    dst[0] = a.x; dst[1] = a.y; dst[2] = a.z; dst[3] = a.w; dst[4] = b.x; dst[5] = b.y; dst[6] = b.z; dst[7] = b.w;
+}
+template <typename T> __device__ __forceinline__ bool aligned_rows(const T* p, int row_elems) {
+    return reinterpret_cast<uintptr_t>(p) % 32 == 0 && row_elems % 8 == 0;   // every row then starts on a 16-byte boundary (fp32: 32)
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -129,10 +148,19 @@ __global__ void __launch_bounds__(128) lstm_layer_simt_kernel(const Ctrl* __rest
     extern __shared__ float sm[];  // 4 rows x (n_in + P)
     const int j = blockIdx.x;
     const int K = n_in + P;
-    for (int e = threadIdx.x; e < 4 * K; e += blockDim.x) {
-        int g = e / K, k = e - g * K;
-        size_t row = (size_t)g * P + j;
-        sm[e] = (k < n_in) ? ldf(w_ih + row * n_in + k) : ldf(w_hh + row * P + (k - n_in));
+    if (aligned_rows(w_ih, n_in) && aligned_rows(w_hh, P)) {
+        // eight weights per load (a chunk never straddles a row or the boundary between the two matrices)
+        for (int c8 = threadIdx.x; c8 < 4 * K / 8; c8 += blockDim.x) {
+            const int e = 8 * c8, g = e / K, k = e - g * K;
+            const size_t row = (size_t)g * P + j;
+            load8(k < n_in ? w_ih + row * n_in + k : w_hh + row * P + (k - n_in), sm + e);
+        }
+    } else {
+        for (int e = threadIdx.x; e < 4 * K; e += blockDim.x) {
+            int g = e / K, k = e - g * K;
+            size_t row = (size_t)g * P + j;
+            sm[e] = (k < n_in) ? ldf(w_ih + row * n_in + k) : ldf(w_hh + row * P + (k - n_in));
+        }
     }
     __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
@@ -340,22 +368,44 @@ template <typename TW>
 __global__ void __launch_bounds__(256) joint_logits_shared_kernel(const int32_t* __restrict__ t_cur, const int32_t* __restrict__ enc_len,
                                                                   const TW* __restrict__ enc_proj, const float* __restrict__ pred_proj,
                                                                   const TW* __restrict__ w_out, const float* __restrict__ b_out,
-                                                                  float* __restrict__ logits_out, int W, int H, int NV, int act) {
-    extern __shared__ float z[];  // [8][H]
+                                                                  float* __restrict__ logits_out, int W, int H, int NV, int act, int stage_w) {
+    extern __shared__ float z[];  // [8][H] activations, then (stage_w) [16][H] the block's rows of W_out
+    float* wsm = z + 8 * (size_t)H;
     const int b = blockIdx.y;
     const int t = t_cur[b], len = enc_len[b];
     if (t >= len) return;
     const int n = min(W, len - t);
     const int v0 = blockIdx.x * 16, v1 = min(NV, v0 + 16);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+    const bool vec = aligned_rows(w_out, H) && aligned_rows(enc_proj, H);
+    // the block's rows of W_out, once (all loads in flight together instead of one dependent load per dot-product step)
+    if (stage_w && vec) {
+        for (int c8 = threadIdx.x; c8 < (v1 - v0) * H / 8; c8 += blockDim.x) load8(w_out + (size_t)v0 * H + 8 * (size_t)c8, wsm + 8 * c8);
+    } else if (stage_w) {
+        for (int e = threadIdx.x; e < (v1 - v0) * H; e += blockDim.x) wsm[e] = ldf(w_out + (size_t)v0 * H + e);
+    }
     for (int w0 = 0; w0 < n; w0 += 8) {
         const int nc = min(8, n - w0);
         __syncthreads();
-        for (int e = threadIdx.x; e < nc * H; e += blockDim.x) {
-            const int w = e / H, k = e - w * H;
-            float s = ldf(enc_proj + (size_t)(t + w0 + w) * H + k) + pred_proj[(size_t)b * H + k];
-            s = act == WIND_ACT_RELU ? fmaxf(s, 0.f) : tanhf(s);
-            z[e] = round_like<TW>(s);
+        if (vec) {
+            for (int c8 = threadIdx.x; c8 < nc * H / 8; c8 += blockDim.x) {
+                const int e = 8 * c8, w = e / H, k = e - w * H;
+                float x[8];
+                load8(enc_proj + (size_t)(t + w0 + w) * H + k, x);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float s = x[i] + pred_proj[(size_t)b * H + k + i];
+                    s = act == WIND_ACT_RELU ? fmaxf(s, 0.f) : tanhf(s);
+                    z[e + i] = round_like<TW>(s);
+                }
+            }
+        } else {
+            for (int e = threadIdx.x; e < nc * H; e += blockDim.x) {
+                const int w = e / H, k = e - w * H;
+                float s = ldf(enc_proj + (size_t)(t + w0 + w) * H + k) + pred_proj[(size_t)b * H + k];
+                s = act == WIND_ACT_RELU ? fmaxf(s, 0.f) : tanhf(s);
+                z[e] = round_like<TW>(s);
+            }
         }
         __syncthreads();
         for (int v = v0 + warp; v < v1; v += nw) {
@@ -363,7 +413,7 @@ __global__ void __launch_bounds__(256) joint_logits_shared_kernel(const int32_t*
 #pragma unroll
             for (int w = 0; w < 8; ++w) a[w] = 0.f;
             for (int k = lane; k < H; k += 32) {
-                const float wv = ldf(w_out + (size_t)v * H + k);
+                const float wv = stage_w ? wsm[(size_t)(v - v0) * H + k] : ldf(w_out + (size_t)v * H + k);
 #pragma unroll
                 for (int w = 0; w < 8; ++w)
                     if (w < nc) a[w] = fmaf(wv, z[w * H + k], a[w]);
@@ -381,12 +431,17 @@ __global__ void __launch_bounds__(256) joint_logits_shared_kernel(const int32_t*
 
 template <typename TW>
 static cudaError_t simt_joint_shared_t(const Call& c, float* logits_out) {
-    const size_t smem = sizeof(float) * 8 * (size_t)c.m.H;
-    if (smem > 48 * 1024) cudaFuncSetAttribute(joint_logits_shared_kernel<TW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // eight activation rows and, where they fit, the block's sixteen rows of W_out
+    const int stage_w = sizeof(float) * 24 * (size_t)c.m.H <= 160 * 1024;
+    const size_t smem = sizeof(float) * (stage_w ? 24 : 8) * (size_t)c.m.H;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(joint_logits_shared_kernel<TW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
     dim3 grid((unsigned)((c.m.V + 1 + 15) / 16), (unsigned)c.B);
     joint_logits_shared_kernel<TW><<<grid, 256, smem, c.stream>>>(c.t(), c.enc_len, (const TW*)c.enc_proj(), c.pred_proj(),
                                                                   (const TW*)c.m.w_out, c.m.b_out, logits_out, c.W, c.m.H,
-                                                                  c.m.V + 1, c.m.act);
+                                                                  c.m.V + 1, c.m.act, stage_w);
     return cudaGetLastError();
 }
 
