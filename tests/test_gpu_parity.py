@@ -259,7 +259,7 @@ def test_bf16_joint_logits(pkg, kernels, name, W):
     cfg = ws.small_variant(ws.CONFIGS[name], 8, 30, 90)
     weights = ws.make_model(cfg)
     enc, lens = ws.make_enc(cfg, pad="nan")
-    logits_parity(pkg, weights, enc, lens, W=W, S=cfg.S, tol=TOL["bf16"], n_windows=128 if name.startswith("cfg3") else 16,
+    logits_parity(pkg, weights, enc, lens, W=W, S=cfg.S, tol=TOL["bf16"], n_windows=64 if name.startswith("cfg3") else 16,
                   kernels=kernels)
 
 
